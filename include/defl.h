@@ -1,0 +1,167 @@
+/* defl.h -- C ABI of the B200 (sm_100a) spectrally deflated matrix filter.
+ *
+ * The library wraps an unchanged fixed-depth polynomial filter (Eq. 1) in spectral deflation
+ * (Section 2): estimate the dominant singular/eigen components, subtract them, normalise the
+ * residual, run the filter, restore the components (Eq. 3). Two primitives are exported:
+ *   defl_polar_batched  -- Algorithm 3 (batched randomized SVD) + Algorithm 1 (deflated polar factor)
+ *   defl_psd_project    -- Algorithm 2 (deflated PSD projection with a warm-started basis)
+ * plus the batched randomized SVD on its own, a counter-based Gaussian fill and diagnostics.
+ *
+ * Conventions
+ *   - Every matrix pointer is DEVICE memory unless the comment says "host". Matrices are
+ *     row-major and contiguous; a batch is b matrices back to back.
+ *   - The caller owns every buffer it passes; the library never frees or keeps a caller pointer
+ *     after the call returns. A context owns its own scratch memory and grows it (cudaMalloc)
+ *     when a call needs more than it holds, so repeated calls of one shape allocate once.
+ *   - All work is enqueued on the context's stream and the call returns without synchronising
+ *     (the only exception: growing the scratch memory synchronises the device).
+ *   - Return value: 0 = OK, < 0 = caller error, nothing was launched (see defl_status_string).
+ *     Numerical events (Cholesky breakdown, Jacobi sweep cap, zero residual, a device-side wait
+ *     that ran out) are reported per matrix in defl_info.status, never by a trap.
+ *   - There is no CPU fallback: without a CUDA device every compute entry point returns
+ *     DEFL_ERR_CUDA.
+ */
+#ifndef DEFL_H_
+#define DEFL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* storage types of G / out */
+#define DEFL_BF16 0 /* bf16 storage, bf16 tensor-core products, fp32 accumulation */
+#define DEFL_F32 1  /* fp32 storage; polar path: fp32 FMA products; PSD filter: tf32 tensor-core products */
+
+/* where the head is restored (polar) */
+#define DEFL_RESTORE_PADDED 0 /* Algorithm 1: X0 = R/||R||_F + U_k V_k^T / gamma, out = N^L(X0) */
+#define DEFL_RESTORE_ADD 1    /* Eq. 3:       X0 = R/||R||_F,                   out = N^L(X0) + U_k V_k^T */
+
+/* normalisation scale of the symmetric residual (PSD) */
+#define DEFL_NORM_LANCZOS 0   /* App. D.1: 20-step Lanczos upper estimate of ||R||_2 */
+#define DEFL_NORM_FROBENIUS 1 /* ||R||_F, a looser valid upper bound */
+
+/* which product engine runs the large matrix products */
+#define DEFL_ENGINE_AUTO 0   /* tensor cores whenever the shape and type allow */
+#define DEFL_ENGINE_SIMT 1   /* fp32 FMA tiles (reference engine inside the library) */
+#define DEFL_ENGINE_TENSOR 2 /* tcgen05 tiles; error if the shape is not supported */
+
+/* return codes */
+#define DEFL_OK 0
+#define DEFL_ERR_ARG (-1)       /* null pointer, non-positive size, aliasing, bad enum */
+#define DEFL_ERR_RANK (-2)      /* k + oversample leaves no room: need k < min(m,n) and l <= DEFL_MAX_L */
+#define DEFL_ERR_CUDA (-3)      /* a CUDA runtime call failed (no device, launch error, out of memory) */
+#define DEFL_ERR_UNSUPPORTED (-4) /* the requested engine cannot run this shape/type */
+
+/* per-matrix status bits in defl_info.status */
+#define DEFL_ST_CHOL_SHIFT 1   /* a Cholesky pivot was not positive; factorised with a diagonal shift */
+#define DEFL_ST_JACOBI_CAP 2   /* the Jacobi eigensolver hit its sweep cap */
+#define DEFL_ST_ZERO_RESIDUAL 4 /* ||R||_F was zero or not finite: residual treated as zero */
+#define DEFL_ST_DEVICE_WAIT 8  /* a bounded device-side wait ran out; the output is not valid */
+
+#define DEFL_MAX_L 64 /* largest sketch width k + oversample (and PSD basis width K) */
+#define DEFL_MAX_STEPS 32 /* largest filter depth L (or T) */
+#define DEFL_LANCZOS_STEPS 20
+
+typedef struct defl_ctx defl_ctx; /* opaque: device, stream, scratch memory */
+
+typedef struct defl_opts {
+  const float* sketch;   /* device, Omega[b, min(m,n), l] fp32 (Algorithm 3 line 2); NULL: drawn from `seed`
+                            with defl_fill_gaussian's generator, stream index = matrix index */
+  uint64_t seed;
+  int restore_mode;      /* DEFL_RESTORE_* */
+  float gamma;           /* padding margin gamma >= 1 (Algorithm 1 / 2); <= 0 means 1.01 */
+  int norm_mode;         /* DEFL_NORM_* (PSD only) */
+  const float* lanczos_start; /* device, [n] fp32 start vector of the Lanczos run; NULL: drawn from `seed` */
+  int warmup;            /* PSD: non-zero = gate off, return the undeflated projection of Eq. 7 but still
+                            advance the basis (the paper keeps the gate off while the basis stabilises) */
+  int engine;            /* DEFL_ENGINE_* */
+  int exploit_symmetry;  /* non-zero: compute only the upper tiles of X X^T and of A^2 and mirror them */
+} defl_opts;
+
+typedef struct defl_info {
+  float* s;      /* device, [b, l]: all l estimated singular values, descending (PSD: [K] Ritz values by
+                    decreasing magnitude); may be NULL */
+  float* rho;    /* device, [b]: ||R||_F used for normalisation (PSD: [1], the scale theta-hat); may be NULL */
+  int* status;   /* device, [b]: DEFL_ST_* bits (PSD: [1]); may be NULL */
+} defl_info;
+
+/* Context. `device` is a CUDA ordinal. defl_create makes no assumption about the current device
+ * and restores it. Not thread safe: one context per host thread or external locking. */
+int defl_create(defl_ctx** out, int device);
+int defl_destroy(defl_ctx* ctx);
+int defl_set_stream(defl_ctx* ctx, void* cuda_stream); /* cudaStream_t; NULL = default stream */
+
+/* Bytes of context scratch a polar / PSD call of this shape needs (what the context will hold). */
+size_t defl_polar_workspace_bytes(int b, int m, int n, int dtype, int k, int oversample);
+size_t defl_psd_workspace_bytes(int n, int K);
+
+/* Deflated polar factor of a batch (Algorithm 3 then Algorithm 1, fixed-k reading).
+ *   G    [b,m,n] dtype, not modified.         out [b,m,n] dtype, must not overlap G.
+ *   k            number of triplets deflated; k = 0 runs the plain filter X0 = G/||G||_F (Algorithm 1, else-branch).
+ *   oversample   extra sketch columns p; l = min(min(m,n), k+p) columns are sketched (Algorithm 3 line 1).
+ *   power_iters  J subspace iterations (Algorithm 3 lines 4-6).
+ *   coeff_schedule  host, [L][3] = (a_t, b_t, c_t) of X <- a X + b (X X^T) X + c (X X^T)^2 X (Eq. 2), applied
+ *                for t = 1..L in order. L = 0 returns X0.
+ * Wide matrices (m < n) are handled as the transpose without moving data (polar(M^T) = polar(M)^T).
+ * Errors: DEFL_ERR_ARG, DEFL_ERR_RANK (k >= min(m,n) or l > DEFL_MAX_L or L > DEFL_MAX_STEPS), DEFL_ERR_CUDA,
+ * DEFL_ERR_UNSUPPORTED. opts and info may be NULL. */
+int defl_polar_batched(defl_ctx* ctx, const void* G, void* out, int b, int m, int n, int dtype,
+                       int k, int oversample, int power_iters,
+                       const float* coeff_schedule, int L,
+                       const defl_opts* opts, const defl_info* info);
+
+/* Batched randomized SVD alone (Algorithm 3) in the caller's orientation:
+ *   G ~ P diag(s) W^T with P [b,m,l], s [b,l] descending, W [b,n,l], all fp32; l = min(min(m,n), k+oversample).
+ * Any of P, s, W may be NULL. The sketch comes from opts as above. */
+int defl_brsvd_batched(defl_ctx* ctx, const void* G, int b, int m, int n, int dtype,
+                       int k, int oversample, int power_iters,
+                       float* P, float* s, float* W, const defl_opts* opts, int* status);
+
+/* Deflated PSD projection (Algorithm 2, fixed-k reading) of one symmetric matrix.
+ *   X  [n,n] fp32 symmetric, not modified.   P [n,n] fp32, exactly symmetric on return, must not overlap X.
+ *   warm_basis [n,K] fp32 with orthonormal columns, IN/OUT: on return the orthonormalised Z V (line 9).
+ *   k  Ritz pairs of largest magnitude to deflate (k <= K); k = 0 or opts->warmup: Eq. 7.
+ *   coeff_schedule host, [T][3]: the composite odd filter g = p_T o ... o p_1, p_t(x) = a x + b x^3 + c x^5.
+ * The only state carried between calls is warm_basis, which the caller owns. */
+int defl_psd_project(defl_ctx* ctx, const void* X, void* P, int n, int k,
+                     float* warm_basis, int K,
+                     const float* coeff_schedule, int T,
+                     const defl_opts* opts, const defl_info* info);
+
+/* Counter-based standard-normal fill (the sketch of Algorithm 3 when none is passed):
+ *   h(x): x += 0x9E3779B97F4A7C15; x = (x ^ x>>30) * 0xBF58476D1CE4E5B9; x = (x ^ x>>27) * 0x94D049BB133111EB; x ^ x>>31
+ *   j = idx/2; r1 = h(h(seed) ^ 2j); r2 = h(h(seed) ^ (2j+1)); u1 = ((r1>>11)+1) 2^-53; u2 = (r2>>11) 2^-53
+ *   value(idx) = sqrt(-2 ln u1) * (idx even ? cos(2 pi u2) : sin(2 pi u2)), evaluated in fp64, rounded to dtype.
+ * dst is device memory of `count` elements of dtype (DEFL_BF16 or DEFL_F32). */
+int defl_fill_gaussian(defl_ctx* ctx, void* dst, size_t count, int dtype, uint64_t seed);
+
+/* Diagnostics: one batched product C[b,M,N] = alpha * opA(A) opB(B) through a chosen engine, used by the
+ * tests to check the tensor-core tile engine against the fp32 engine (no counterpart in the paper).
+ * A element (i,kk) is A[i*sa_i + kk*sa_k], B element (kk,j) is B[kk*sb_k + j*sb_j]; C is row-major [M,N].
+ * in_dtype / out_dtype are DEFL_BF16 or DEFL_F32; strides in elements. */
+int defl_debug_gemm(defl_ctx* ctx, int engine, int batch, int M, int N, int K,
+                    const void* A, long long sa_i, long long sa_k, long long batch_a,
+                    const void* B, long long sb_k, long long sb_j, long long batch_b,
+                    void* C, int in_dtype, int out_dtype, float alpha, int exploit_symmetry);
+
+/* Stage timing: when enabled, the context records CUDA events between the stages of each call;
+ * defl_get_stage_ms synchronises the stream and writes up to `cap` stage durations (ms) of the last
+ * call, returning how many stages there were. Polar stages: 0 randomized SVD (Algorithm 3),
+ * 1 deflate + normalise, 2 filter, 3 restore. PSD stages: 0 block step + Rayleigh-Ritz, 1 deflate,
+ * 2 Lanczos scale, 3 initialisation, 4 filter, 5 reconstruction, 6 basis update. */
+int defl_set_profiling(defl_ctx* ctx, int enabled);
+int defl_get_stage_ms(defl_ctx* ctx, float* ms, int cap);
+
+/* Number of kernels the library launched on this context since creation. */
+long long defl_launch_count(defl_ctx* ctx);
+
+const char* defl_status_string(int code);
+const char* defl_last_error(defl_ctx* ctx); /* text of the last CUDA failure, "" if none */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DEFL_H_ */

@@ -1,0 +1,282 @@
+"""Thin ctypes binding of libdeflpolar.so: argument marshalling only.
+
+Every function has the name and meaning of the C entry point declared in include/defl.h. Tensors
+are torch CUDA tensors used purely as device memory; all computation happens in the library's
+CUDA kernels. There is no fallback: if the shared library is missing the import of this module's
+`lib()` fails, and without a CUDA device every compute call raises.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdeflpolar.so")
+
+BF16, F32 = 0, 1
+RESTORE_PADDED, RESTORE_ADD = 0, 1
+NORM_LANCZOS, NORM_FROBENIUS = 0, 1
+ENGINE_AUTO, ENGINE_SIMT, ENGINE_TENSOR = 0, 1, 2
+ST_CHOL_SHIFT, ST_JACOBI_CAP, ST_ZERO_RESIDUAL, ST_DEVICE_WAIT = 1, 2, 4, 8
+MAX_L, MAX_STEPS = 64, 32
+
+MUON_QUINTIC = (3.4445, -4.7750, 2.0315)
+CLASSICAL_QUINTIC = (1.875, -1.25, 0.375)
+
+EXPORTS = [
+    "defl_create", "defl_destroy", "defl_set_stream", "defl_polar_workspace_bytes", "defl_psd_workspace_bytes",
+    "defl_polar_batched", "defl_brsvd_batched", "defl_psd_project", "defl_fill_gaussian", "defl_debug_gemm",
+    "defl_set_profiling", "defl_get_stage_ms", "defl_launch_count", "defl_status_string", "defl_last_error",
+]
+
+
+class DeflOpts(ctypes.Structure):
+    _fields_ = [("sketch", ctypes.c_void_p), ("seed", ctypes.c_uint64), ("restore_mode", ctypes.c_int),
+                ("gamma", ctypes.c_float), ("norm_mode", ctypes.c_int), ("lanczos_start", ctypes.c_void_p),
+                ("warmup", ctypes.c_int), ("engine", ctypes.c_int), ("exploit_symmetry", ctypes.c_int)]
+
+
+class DeflInfo(ctypes.Structure):
+    _fields_ = [("s", ctypes.c_void_p), ("rho", ctypes.c_void_p), ("status", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def lib():
+    """Load the shared library (raises OSError if it has not been built)."""
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(LIB_PATH)
+        L.defl_create.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.c_int]
+        L.defl_destroy.argtypes = [ctypes.c_void_p]
+        L.defl_set_stream.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+        L.defl_polar_workspace_bytes.restype = ctypes.c_size_t
+        L.defl_polar_workspace_bytes.argtypes = [ctypes.c_int] * 6
+        L.defl_psd_workspace_bytes.restype = ctypes.c_size_t
+        L.defl_psd_workspace_bytes.argtypes = [ctypes.c_int] * 2
+        L.defl_polar_batched.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 7 + [
+            ctypes.POINTER(ctypes.c_float), ctypes.c_int, ctypes.POINTER(DeflOpts), ctypes.POINTER(DeflInfo)]
+        L.defl_brsvd_batched.argtypes = [ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 7 + [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(DeflOpts), ctypes.c_void_p]
+        L.defl_psd_project.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                       ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_float), ctypes.c_int,
+                                       ctypes.POINTER(DeflOpts), ctypes.POINTER(DeflInfo)]
+        L.defl_fill_gaussian.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint64]
+        L.defl_debug_gemm.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                      ctypes.c_void_p, ctypes.c_longlong, ctypes.c_longlong, ctypes.c_longlong,
+                                      ctypes.c_void_p, ctypes.c_longlong, ctypes.c_longlong, ctypes.c_longlong,
+                                      ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_float, ctypes.c_int]
+        L.defl_set_profiling.argtypes = [ctypes.c_void_p, ctypes.c_int]
+        L.defl_get_stage_ms.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_float), ctypes.c_int]
+        L.defl_launch_count.restype = ctypes.c_longlong
+        L.defl_launch_count.argtypes = [ctypes.c_void_p]
+        L.defl_status_string.restype = ctypes.c_char_p
+        L.defl_status_string.argtypes = [ctypes.c_int]
+        L.defl_last_error.restype = ctypes.c_char_p
+        L.defl_last_error.argtypes = [ctypes.c_void_p]
+        _lib = L
+    return _lib
+
+
+class DeflError(RuntimeError):
+    def __init__(self, code, detail=""):
+        self.code = code
+        msg = lib().defl_status_string(code).decode()
+        super().__init__("defl error %d: %s%s" % (code, msg, (" [" + detail + "]") if detail else ""))
+
+
+def _dtype_code(t):
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return F32
+    raise TypeError("only bfloat16 and float32 tensors are supported")
+
+
+def _ptr(t):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def _dev(t, what):
+    if not (t.is_cuda and t.is_contiguous()):
+        raise ValueError("%s must be a contiguous CUDA tensor" % what)
+    return t
+
+
+def _schedule(coeffs, steps=None):
+    c = torch.as_tensor(coeffs, dtype=torch.float64)
+    if c.ndim == 1:
+        c = c.unsqueeze(0).repeat(steps, 1)
+    flat = [float(x) for x in c.reshape(-1).tolist()]
+    arr = (ctypes.c_float * max(len(flat), 1))(*flat)
+    return arr, c.shape[0]
+
+
+class Context:
+    """defl_ctx bound to one CUDA device; work is enqueued on torch's current stream at call time."""
+
+    def __init__(self, device=0):
+        self.device = torch.device("cuda", device) if not isinstance(device, torch.device) else device
+        h = ctypes.c_void_p()
+        rc = lib().defl_create(ctypes.byref(h), self.device.index or 0)
+        if rc != 0:
+            raise DeflError(rc)
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().defl_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _sync_stream(self):
+        s = torch.cuda.current_stream(self.device)
+        lib().defl_set_stream(self._h, ctypes.c_void_p(s.cuda_stream))
+
+    def _check(self, rc):
+        if rc != 0:
+            raise DeflError(rc, lib().defl_last_error(self._h).decode())
+
+    def _opts(self, sketch=None, seed=0, restore_mode=RESTORE_PADDED, gamma=0.0, norm_mode=NORM_LANCZOS,
+              lanczos_start=None, warmup=False, engine=ENGINE_AUTO, exploit_symmetry=False):
+        o = DeflOpts()
+        o.sketch = sketch.data_ptr() if sketch is not None else None
+        o.seed = seed
+        o.restore_mode = restore_mode
+        o.gamma = gamma
+        o.norm_mode = norm_mode
+        o.lanczos_start = lanczos_start.data_ptr() if lanczos_start is not None else None
+        o.warmup = int(bool(warmup))
+        o.engine = engine
+        o.exploit_symmetry = int(bool(exploit_symmetry))
+        return o
+
+    # ------------------------------------------------------------------------------------------
+    def defl_polar_batched(self, G, k, oversample, power_iters, coeff_schedule, steps=None, out=None, sketch=None,
+                           seed=0, restore_mode=RESTORE_PADDED, gamma=0.0, engine=ENGINE_AUTO,
+                           exploit_symmetry=False, want_info=False):
+        """out[b,m,n] = deflated polar factor of every G[b] (Algorithm 3 + Algorithm 1)."""
+        _dev(G, "G")
+        if G.ndim != 3:
+            raise ValueError("G must be [b, m, n]")
+        b, m, n = G.shape
+        out = torch.empty_like(G) if out is None else _dev(out, "out")
+        sched, L = _schedule(coeff_schedule, steps)
+        if sketch is not None:
+            _dev(sketch, "sketch")
+            if sketch.dtype != torch.float32:
+                raise TypeError("sketch must be float32")
+        opts = self._opts(sketch=sketch, seed=seed, restore_mode=restore_mode, gamma=gamma, engine=engine,
+                          exploit_symmetry=exploit_symmetry)
+        info = DeflInfo()
+        extras = None
+        if want_info:
+            l = min(min(m, n), k + oversample) if k > 0 else 0
+            s = torch.zeros((b, max(l, 1)), dtype=torch.float32, device=G.device)
+            rho = torch.zeros((b,), dtype=torch.float32, device=G.device)
+            status = torch.zeros((b,), dtype=torch.int32, device=G.device)
+            info.s, info.rho, info.status = s.data_ptr(), rho.data_ptr(), status.data_ptr()
+            extras = {"s": s[:, :l], "rho": rho, "status": status}
+        self._sync_stream()
+        rc = lib().defl_polar_batched(self._h, _ptr(G), _ptr(out), b, m, n, _dtype_code(G), k, oversample, power_iters,
+                                      sched, L, ctypes.byref(opts), ctypes.byref(info))
+        self._check(rc)
+        return (out, extras) if want_info else out
+
+    def defl_brsvd_batched(self, G, k, oversample, power_iters, sketch=None, seed=0, engine=ENGINE_AUTO):
+        """Algorithm 3 in the caller's orientation: returns (P[b,m,l], s[b,l], W[b,n,l], status[b])."""
+        _dev(G, "G")
+        b, m, n = G.shape
+        l = min(min(m, n), k + oversample)
+        P = torch.empty((b, m, l), dtype=torch.float32, device=G.device)
+        W = torch.empty((b, n, l), dtype=torch.float32, device=G.device)
+        s = torch.empty((b, l), dtype=torch.float32, device=G.device)
+        status = torch.zeros((b,), dtype=torch.int32, device=G.device)
+        opts = self._opts(sketch=sketch, seed=seed, engine=engine)
+        self._sync_stream()
+        rc = lib().defl_brsvd_batched(self._h, _ptr(G), b, m, n, _dtype_code(G), k, oversample, power_iters,
+                                      _ptr(P), _ptr(s), _ptr(W), ctypes.byref(opts), _ptr(status))
+        self._check(rc)
+        return P, s, W, status
+
+    def defl_psd_project(self, X, k, warm_basis, coeff_schedule, steps=None, out=None, gamma=0.0,
+                         norm_mode=NORM_LANCZOS, lanczos_start=None, seed=0, warmup=False, engine=ENGINE_AUTO,
+                         exploit_symmetry=False, want_info=False):
+        """P = deflated PSD projection of the symmetric X[n,n] (Algorithm 2); warm_basis[n,K] is updated in place."""
+        _dev(X, "X")
+        n = X.shape[0]
+        if X.dtype != torch.float32 or X.shape != (n, n):
+            raise ValueError("X must be a square float32 matrix")
+        K = 0
+        if warm_basis is not None:
+            _dev(warm_basis, "warm_basis")
+            K = warm_basis.shape[1]
+        out = torch.empty_like(X) if out is None else _dev(out, "out")
+        sched, T = _schedule(coeff_schedule, steps)
+        opts = self._opts(gamma=gamma, norm_mode=norm_mode, lanczos_start=lanczos_start, seed=seed, warmup=warmup,
+                          engine=engine, exploit_symmetry=exploit_symmetry)
+        info = DeflInfo()
+        extras = None
+        if want_info:
+            lam = torch.zeros((max(K, 1),), dtype=torch.float32, device=X.device)
+            theta = torch.zeros((1,), dtype=torch.float32, device=X.device)
+            status = torch.zeros((1,), dtype=torch.int32, device=X.device)
+            info.s, info.rho, info.status = lam.data_ptr(), theta.data_ptr(), status.data_ptr()
+            extras = {"lam": lam[:K], "theta": theta, "status": status}
+        self._sync_stream()
+        rc = lib().defl_psd_project(self._h, _ptr(X), _ptr(out), n, k, _ptr(warm_basis), K, sched, T,
+                                    ctypes.byref(opts), ctypes.byref(info))
+        self._check(rc)
+        return (out, extras) if want_info else out
+
+    def defl_fill_gaussian(self, dst, seed):
+        _dev(dst, "dst")
+        self._sync_stream()
+        self._check(lib().defl_fill_gaussian(self._h, _ptr(dst), dst.numel(), _dtype_code(dst), seed))
+        return dst
+
+    def defl_debug_gemm(self, A, B, trans_a=False, trans_b=False, engine=ENGINE_AUTO, out_dtype=None, alpha=1.0,
+                        exploit_symmetry=False):
+        """C[b] = alpha * op(A[b]) op(B[b]); op = transpose of the stored matrix when the flag is set."""
+        _dev(A, "A"), _dev(B, "B")
+        b = A.shape[0]
+        if trans_a:
+            K, M = A.shape[1], A.shape[2]
+            sa_i, sa_k = 1, M
+        else:
+            M, K = A.shape[1], A.shape[2]
+            sa_i, sa_k = K, 1
+        if trans_b:
+            N = B.shape[1]
+            sb_k, sb_j = 1, B.shape[2]
+        else:
+            N = B.shape[2]
+            sb_k, sb_j = N, 1
+        out_dtype = out_dtype or A.dtype
+        C = torch.empty((b, M, N), dtype=out_dtype, device=A.device)
+        self._sync_stream()
+        rc = lib().defl_debug_gemm(self._h, engine, b, M, N, K, _ptr(A), sa_i, sa_k, A.shape[1] * A.shape[2],
+                                   _ptr(B), sb_k, sb_j, B.shape[1] * B.shape[2], _ptr(C), _dtype_code(A),
+                                   BF16 if out_dtype == torch.bfloat16 else F32, alpha, int(exploit_symmetry))
+        self._check(rc)
+        return C
+
+    def defl_set_profiling(self, enabled):
+        lib().defl_set_profiling(self._h, int(bool(enabled)))
+
+    def defl_get_stage_ms(self):
+        buf = (ctypes.c_float * 16)()
+        n = lib().defl_get_stage_ms(self._h, buf, 16)
+        return [buf[i] for i in range(max(n, 0))]
+
+    def defl_launch_count(self):
+        return int(lib().defl_launch_count(self._h))
+
+    def polar_workspace_bytes(self, b, m, n, dtype, k, oversample):
+        return int(lib().defl_polar_workspace_bytes(b, m, n, BF16 if dtype == torch.bfloat16 else F32, k, oversample))

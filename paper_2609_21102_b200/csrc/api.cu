@@ -1,0 +1,519 @@
+// C ABI of the library: context, scratch memory, and the orchestration of the deflated polar factor
+// (Algorithm 3 + Algorithm 1) as a sequence of kernel launches on one stream. The PSD projection
+// lives in psd.cu. Nothing here computes on the host beyond choosing launch parameters.
+#include "../../include/defl.h"
+#include "common.cuh"
+#include "panel.cuh"
+#include "ctx.cuh"
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+using namespace defl;
+
+namespace defl {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool ctx_fail(defl_ctx* c, cudaError_t e, const char* where) {
+  if (e == cudaSuccess) return false;
+  snprintf(c->err, sizeof(c->err), "%s: %s", where, cudaGetErrorString(e));
+  return true;
+}
+
+int ctx_reserve(defl_ctx* c, size_t bytes) {
+  if (bytes <= c->ws_bytes) return DEFL_OK;
+  if (c->ws) {
+    cudaDeviceSynchronize();
+    cudaFree(c->ws);
+    c->ws = nullptr;
+    c->ws_bytes = 0;
+  }
+  void* p = nullptr;
+  if (ctx_fail(c, cudaMalloc(&p, bytes), "cudaMalloc(workspace)")) return DEFL_ERR_CUDA;
+  c->ws = p;
+  c->ws_bytes = bytes;
+  return DEFL_OK;
+}
+
+void ctx_stage_mark(defl_ctx* c) {
+  if (!c->profiling || c->n_marks >= DEFL_MAX_MARKS) return;
+  cudaEventRecord(c->marks[c->n_marks++], c->stream);
+}
+
+// Which engine a product runs on. AUTO sends bf16 products to the tensor cores and keeps fp32
+// products on exact fp32 FMA; ENGINE_TENSOR also sends fp32 products there (as tf32).
+bool use_tensor_engine(const GemmDesc& g, int engine) {
+  if (engine == DEFL_ENGINE_SIMT) return false;
+  if (engine == DEFL_ENGINE_AUTO && g.in_dtype != BF16) return false;
+  return gemm_tc_supported(g);
+}
+
+// Run one product on the engine the options ask for. Returns a DEFL_* code.
+int run_gemm(defl_ctx* c, const GemmDesc& g, int engine, const char* what) {
+  const bool tc = use_tensor_engine(g, engine);
+  if (engine == DEFL_ENGINE_TENSOR && !tc) {
+    snprintf(c->err, sizeof(c->err), "%s: shape/type not supported by the tensor engine", what);
+    return DEFL_ERR_UNSUPPORTED;
+  }
+  cudaError_t e;
+  if (tc) e = gemm_tc_launch(g, c->stream, c->wait_status, c->num_sms, &c->launches);
+  else e = gemm_simt_launch(g, c->stream, &c->launches);
+  if (ctx_fail(c, e, what)) return DEFL_ERR_CUDA;
+  return DEFL_OK;
+}
+
+int partials_per_batch(const GemmDesc& g, int engine) {
+  if (use_tensor_engine(g, engine)) return gemm_tc_partials_per_batch(g);
+  return gemm_simt_partials_per_batch(g);
+}
+
+struct Carver {
+  char* base; size_t off;
+  explicit Carver(void* p) : base(reinterpret_cast<char*>(p)), off(0) {}
+  template <typename T> T* take(size_t count) {
+    T* r = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off = align_up(off + count * sizeof(T), 256);
+    return r;
+  }
+};
+
+// Workspace layout of one polar call (also used, with a null base, to size it).
+struct PolarWs {
+  void* X;            // [b,m,n] dtype   second iterate buffer (the other one is `out`)
+  void* Am; void* Bm; // [b,ms,ms] dtype  A_t = X X^T and B_t = a I + b A_t + c A_t^2
+  float* Lp;          // [b,ml,l]  long-side panel  (Y, then Q)
+  float* Sp;          // [b,ms,l]  short-side panel (A^T Q and its orthonormalisation; finally (Q^T A)^T)
+  double* gram;       // [b,nchunk,l,l]
+  float* Rinv; float* E; float* Es; float* sv;   // [b,l,l] x3, [b,l]
+  float* Uk; float* Vk;   // [b,ml,k], [b,ms,k]  leading triplets in the tall orientation
+  float* Ws;          // [b,n,k] scaled copy of the right factor
+  double* npart;      // [b,nper] Frobenius partial sums
+  float* rho; float* inv_rho; float* inv_rho2;   // [b]
+  int* status;        // [b]
+  float* sketch;      // [b,ms,l] when the library draws the sketch
+  size_t bytes;
+};
+
+PolarWs carve_polar(void* base, int b, int m, int n, int dtype, int k, int l) {
+  const int ms = m < n ? m : n, ml = m < n ? n : m;
+  const size_t es = dtype_size(dtype);
+  Carver cv(base);
+  PolarWs w;
+  w.X = cv.take<char>((size_t)b * m * n * es);
+  w.Am = cv.take<char>((size_t)b * ms * ms * es);
+  w.Bm = cv.take<char>((size_t)b * ms * ms * es);
+  const int le = l > 0 ? l : 1, ke = k > 0 ? k : 1;
+  w.Lp = cv.take<float>((size_t)b * ml * le);
+  w.Sp = cv.take<float>((size_t)b * ms * le);
+  w.gram = cv.take<double>((size_t)b * gram_num_chunks(ml) * le * le);
+  w.Rinv = cv.take<float>((size_t)b * le * le);
+  w.E = cv.take<float>((size_t)b * le * le);
+  w.Es = cv.take<float>((size_t)b * le * le);
+  w.sv = cv.take<float>((size_t)b * le);
+  w.Uk = cv.take<float>((size_t)b * ml * ke);
+  w.Vk = cv.take<float>((size_t)b * ms * ke);
+  w.Ws = cv.take<float>((size_t)b * n * ke);
+  // norm partials: enough for either engine's tiling of an m x n output
+  const size_t nper = (size_t)((m + 63) / 64) * ((n + 15) / 16) * 4 + 1184;
+  w.npart = cv.take<double>((size_t)b * nper);
+  w.rho = cv.take<float>(b);
+  w.inv_rho = cv.take<float>(b);
+  w.inv_rho2 = cv.take<float>(b);
+  w.status = cv.take<int>(b);
+  w.sketch = cv.take<float>((size_t)b * ms * le);
+  w.bytes = cv.off;
+  return w;
+}
+
+// CholeskyQR2 of the panel P[b, rows, l] in place: twice { W = P^T P; W = R^T R; P <- P R^-1 }.
+int orthonormalise(defl_ctx* c, float* P, int b, int rows, int l, const PolarWs& w, int* status) {
+  const int nchunk = gram_num_chunks(rows);
+  for (int pass = 0; pass < 2; ++pass) {
+    if (ctx_fail(c, gram_partial_launch(P, (long long)rows * l, b, rows, l, l, w.gram, c->stream, &c->launches), "gram"))
+      return DEFL_ERR_CUDA;
+    if (ctx_fail(c, chol_inv_launch(w.gram, nchunk, b, l, w.Rinv, status, c->stream, &c->launches), "cholesky"))
+      return DEFL_ERR_CUDA;
+    if (ctx_fail(c, panel_apply_launch(P, (long long)rows * l, l, w.Rinv, l, b, rows, l, l, P, (long long)rows * l, l,
+                                       c->stream, &c->launches), "panel apply"))
+      return DEFL_ERR_CUDA;
+  }
+  return DEFL_OK;
+}
+
+// Algorithm 3 on the batch: on return w.Lp = Q U_G (left vectors of A, all l), w.Sp... see below.
+// Outputs: w.sv[b,l], w.Uk[b,ml,k_keep] and w.Vk[b,ms,k_keep] (leading k_keep triplets of A = G or G^T).
+int run_brsvd(defl_ctx* c, const void* G, int b, int m, int n, int dtype, int l, int J, int k_keep,
+              const float* sketch, const PolarWs& w, int engine) {
+  const bool tall = m >= n;
+  const int ms = tall ? n : m, ml = tall ? m : n;
+  // element (i,j) of A (ml x ms): tall G[i*n+j]; wide G[j*n+i]
+  const long long a_si = tall ? n : 1, a_sj = tall ? 1 : n;
+  int rc;
+  auto mul_A = [&](const float* Bp, float* Cp) {   // C[ml,l] = A B,  B[ms,l]
+    GemmDesc g = gemm_desc_zero();
+    g.batch = b; g.M = ml; g.N = l; g.K[0] = ms;
+    g.A[0] = G; g.sa_i[0] = a_si; g.sa_k[0] = a_sj; g.batch_a[0] = (long long)m * n; g.in_dtype = dtype;
+    g.B[0] = Bp; g.sb_k[0] = l; g.sb_j[0] = 1; g.batch_b[0] = (long long)ms * l; g.b_dtype = F32;
+    g.C = Cp; g.ldc = l; g.batch_c = (long long)ml * l; g.out_dtype = F32;
+    g.epilogue = EPI_STORE;
+    return run_gemm(c, g, DEFL_ENGINE_SIMT, "A*panel");
+  };
+  auto mul_At = [&](const float* Bp, float* Cp) {  // C[ms,l] = A^T B, B[ml,l]
+    GemmDesc g = gemm_desc_zero();
+    g.batch = b; g.M = ms; g.N = l; g.K[0] = ml;
+    g.A[0] = G; g.sa_i[0] = a_sj; g.sa_k[0] = a_si; g.batch_a[0] = (long long)m * n; g.in_dtype = dtype;
+    g.B[0] = Bp; g.sb_k[0] = l; g.sb_j[0] = 1; g.batch_b[0] = (long long)ml * l; g.b_dtype = F32;
+    g.C = Cp; g.ldc = l; g.batch_c = (long long)ms * l; g.out_dtype = F32;
+    g.epilogue = EPI_STORE;
+    return run_gemm(c, g, DEFL_ENGINE_SIMT, "A^T*panel");
+  };
+  if ((rc = mul_A(sketch, w.Lp))) return rc;                               // Y = A Omega
+  if ((rc = orthonormalise(c, w.Lp, b, ml, l, w, w.status))) return rc;    // Q
+  for (int j = 0; j < J; ++j) {
+    if ((rc = mul_At(w.Lp, w.Sp))) return rc;                              // A^T Q
+    if ((rc = orthonormalise(c, w.Sp, b, ms, l, w, w.status))) return rc;
+    if ((rc = mul_A(w.Sp, w.Lp))) return rc;                               // A Y
+    if ((rc = orthonormalise(c, w.Lp, b, ml, l, w, w.status))) return rc;
+  }
+  if ((rc = mul_At(w.Lp, w.Sp))) return rc;                                // (Q^T A)^T, [ms, l]
+  // thin SVD of Q^T A through the Gram core: (Q^T A)(Q^T A)^T = E diag(s^2) E^T
+  if (ctx_fail(c, gram_partial_launch(w.Sp, (long long)ms * l, b, ms, l, l, w.gram, c->stream, &c->launches), "gram core"))
+    return DEFL_ERR_CUDA;
+  if (ctx_fail(c, jacobi_eig_launch(w.gram, gram_num_chunks(ms), b, l, 0, w.sv, w.E, w.Es, w.status, c->stream,
+                                    &c->launches), "jacobi"))
+    return DEFL_ERR_CUDA;
+  if (k_keep > 0) {
+    // U = Q E (long side), V = (Q^T A)^T E diag(1/s) (short side); keep the leading k_keep columns
+    if (ctx_fail(c, panel_apply_launch(w.Lp, (long long)ml * l, l, w.E, l, b, ml, l, k_keep, w.Uk, (long long)ml * k_keep,
+                                       k_keep, c->stream, &c->launches), "U = Q E"))
+      return DEFL_ERR_CUDA;
+    if (ctx_fail(c, panel_apply_launch(w.Sp, (long long)ms * l, l, w.Es, l, b, ms, l, k_keep, w.Vk, (long long)ms * k_keep,
+                                       k_keep, c->stream, &c->launches), "V = B^T E / s"))
+      return DEFL_ERR_CUDA;
+  }
+  return DEFL_OK;
+}
+
+const float* resolve_sketch(defl_ctx* c, const defl_opts* opts, int b, int ms, int l, const PolarWs& w, int* rc) {
+  *rc = DEFL_OK;
+  if (opts && opts->sketch) return opts->sketch;
+  const unsigned long long seed = opts ? opts->seed : 0ull;
+  if (ctx_fail(c, fill_gaussian_launch(w.sketch, (long long)b * ms * l, F32, seed, (long long)ms * l, 1ull, c->stream,
+                                       &c->launches), "sketch"))
+    *rc = DEFL_ERR_CUDA;
+  return w.sketch;
+}
+
+}  // namespace defl
+
+// ================================================================================================
+extern "C" {
+
+int defl_create(defl_ctx** out, int device) {
+  if (!out) return DEFL_ERR_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return DEFL_ERR_CUDA;
+  int prev = 0;
+  cudaGetDevice(&prev);
+  if (cudaSetDevice(device) != cudaSuccess) return DEFL_ERR_CUDA;
+  defl_ctx* c = new (std::nothrow) defl_ctx();
+  if (!c) return DEFL_ERR_CUDA;
+  memset(c, 0, sizeof(*c));
+  c->device = device;
+  cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device);
+  int ok = 1;
+  if (cudaMalloc(&c->wait_status, sizeof(int)) != cudaSuccess) ok = 0;
+  if (ok) cudaMemset(c->wait_status, 0, sizeof(int));
+  for (int i = 0; ok && i < DEFL_MAX_MARKS; ++i)
+    if (cudaEventCreate(&c->marks[i]) != cudaSuccess) ok = 0;
+  cudaSetDevice(prev);
+  if (!ok) { delete c; return DEFL_ERR_CUDA; }
+  *out = c;
+  return DEFL_OK;
+}
+
+int defl_destroy(defl_ctx* c) {
+  if (!c) return DEFL_ERR_ARG;
+  int prev = 0;
+  cudaGetDevice(&prev);
+  cudaSetDevice(c->device);
+  cudaDeviceSynchronize();
+  if (c->ws) cudaFree(c->ws);
+  if (c->wait_status) cudaFree(c->wait_status);
+  for (int i = 0; i < DEFL_MAX_MARKS; ++i)
+    if (c->marks[i]) cudaEventDestroy(c->marks[i]);
+  cudaSetDevice(prev);
+  delete c;
+  return DEFL_OK;
+}
+
+int defl_set_stream(defl_ctx* c, void* s) {
+  if (!c) return DEFL_ERR_ARG;
+  c->stream = reinterpret_cast<cudaStream_t>(s);
+  return DEFL_OK;
+}
+
+size_t defl_polar_workspace_bytes(int b, int m, int n, int dtype, int k, int oversample) {
+  if (b <= 0 || m <= 0 || n <= 0 || k < 0 || oversample < 0) return 0;
+  const int ms = m < n ? m : n;
+  int l = k > 0 ? k + oversample : 0;
+  if (l > ms) l = ms;
+  return carve_polar(nullptr, b, m, n, dtype, k, l).bytes;
+}
+
+int defl_set_profiling(defl_ctx* c, int enabled) {
+  if (!c) return DEFL_ERR_ARG;
+  c->profiling = enabled != 0;
+  return DEFL_OK;
+}
+
+int defl_get_stage_ms(defl_ctx* c, float* ms, int cap) {
+  if (!c || !ms) return DEFL_ERR_ARG;
+  if (c->n_marks < 2) return 0;
+  cudaStreamSynchronize(c->stream);
+  const int n = c->n_marks - 1;
+  for (int i = 0; i < n && i < cap; ++i) cudaEventElapsedTime(&ms[i], c->marks[i], c->marks[i + 1]);
+  return n;
+}
+
+long long defl_launch_count(defl_ctx* c) { return c ? c->launches : 0; }
+
+const char* defl_status_string(int code) {
+  switch (code) {
+    case DEFL_OK: return "ok";
+    case DEFL_ERR_ARG: return "bad argument (null pointer, non-positive size, overlap or bad enum)";
+    case DEFL_ERR_RANK: return "rank/width out of range (need k < min(m,n), k+oversample <= 64, depth <= 32)";
+    case DEFL_ERR_CUDA: return "CUDA runtime failure (see defl_last_error)";
+    case DEFL_ERR_UNSUPPORTED: return "requested engine cannot run this shape or type";
+    default: return "unknown status";
+  }
+}
+
+const char* defl_last_error(defl_ctx* c) { return c ? c->err : ""; }
+
+int defl_fill_gaussian(defl_ctx* c, void* dst, size_t count, int dtype, uint64_t seed) {
+  if (!c || !dst || (dtype != DEFL_BF16 && dtype != DEFL_F32)) return DEFL_ERR_ARG;
+  cudaSetDevice(c->device);
+  if (ctx_fail(c, fill_gaussian_launch(dst, (long long)count, dtype, seed, 0, 0ull, c->stream, &c->launches), "fill"))
+    return DEFL_ERR_CUDA;
+  return DEFL_OK;
+}
+
+int defl_debug_gemm(defl_ctx* c, int engine, int batch, int M, int N, int K, const void* A, long long sa_i,
+                    long long sa_k, long long batch_a, const void* B, long long sb_k, long long sb_j, long long batch_b,
+                    void* C, int in_dtype, int out_dtype, float alpha, int exploit_symmetry) {
+  if (!c || !A || !B || !C || batch <= 0 || M <= 0 || N <= 0 || K <= 0) return DEFL_ERR_ARG;
+  cudaSetDevice(c->device);
+  GemmDesc g = gemm_desc_zero();
+  g.batch = batch; g.M = M; g.N = N; g.K[0] = K;
+  g.A[0] = A; g.sa_i[0] = sa_i; g.sa_k[0] = sa_k; g.batch_a[0] = batch_a;
+  g.B[0] = B; g.sb_k[0] = sb_k; g.sb_j[0] = sb_j; g.batch_b[0] = batch_b;
+  g.in_dtype = in_dtype; g.b_dtype = in_dtype;
+  g.C = C; g.ldc = N; g.batch_c = (long long)M * N; g.out_dtype = out_dtype;
+  g.epilogue = EPI_STORE; g.alpha = alpha; g.symmetric = exploit_symmetry ? 1 : 0;
+  return run_gemm(c, g, engine, "debug gemm");
+}
+
+int defl_brsvd_batched(defl_ctx* c, const void* G, int b, int m, int n, int dtype, int k, int oversample,
+                       int power_iters, float* P, float* s, float* W, const defl_opts* opts, int* status) {
+  if (!c || !G || b <= 0 || m <= 0 || n <= 0 || k <= 0 || oversample < 0 || power_iters < 0) return DEFL_ERR_ARG;
+  if (dtype != DEFL_BF16 && dtype != DEFL_F32) return DEFL_ERR_ARG;
+  const bool tall = m >= n;
+  const int ms = tall ? n : m, ml = tall ? m : n;
+  int l = k + oversample;
+  if (l > ms) l = ms;
+  if (l > DEFL_MAX_L) return DEFL_ERR_RANK;
+  cudaSetDevice(c->device);
+  const size_t need = carve_polar(nullptr, b, m, n, dtype, l, l).bytes;
+  int rc = ctx_reserve(c, need);
+  if (rc) return rc;
+  PolarWs w = carve_polar(c->ws, b, m, n, dtype, l, l);
+  const int engine = opts ? opts->engine : DEFL_ENGINE_AUTO;
+  if (ctx_fail(c, fill_int_launch(w.status, b, 0, c->stream, &c->launches), "status")) return DEFL_ERR_CUDA;
+  const float* sk = resolve_sketch(c, opts, b, ms, l, w, &rc);
+  if (rc) return rc;
+  if ((rc = run_brsvd(c, G, b, m, n, dtype, l, power_iters, l, sk, w, engine))) return rc;
+  // tall: G = U S V^T with U on m rows; wide: A = G^T so the left factor of G is V
+  const float* left = tall ? w.Uk : w.Vk;
+  const float* right = tall ? w.Vk : w.Uk;
+  if (P && ctx_fail(c, cudaMemcpyAsync(P, left, (size_t)b * m * l * sizeof(float), cudaMemcpyDeviceToDevice, c->stream), "copy P"))
+    return DEFL_ERR_CUDA;
+  if (W && ctx_fail(c, cudaMemcpyAsync(W, right, (size_t)b * n * l * sizeof(float), cudaMemcpyDeviceToDevice, c->stream), "copy W"))
+    return DEFL_ERR_CUDA;
+  if (s && ctx_fail(c, cudaMemcpyAsync(s, w.sv, (size_t)b * l * sizeof(float), cudaMemcpyDeviceToDevice, c->stream), "copy s"))
+    return DEFL_ERR_CUDA;
+  if (status && ctx_fail(c, cudaMemcpyAsync(status, w.status, (size_t)b * sizeof(int), cudaMemcpyDeviceToDevice, c->stream), "copy status"))
+    return DEFL_ERR_CUDA;
+  (void)ml;
+  return DEFL_OK;
+}
+
+int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int n, int dtype, int k, int oversample,
+                       int power_iters, const float* coeff_schedule, int L, const defl_opts* opts,
+                       const defl_info* info) {
+  if (!c || !G || !out || b <= 0 || m <= 0 || n <= 0 || k < 0 || oversample < 0 || power_iters < 0 || L < 0)
+    return DEFL_ERR_ARG;
+  if (dtype != DEFL_BF16 && dtype != DEFL_F32) return DEFL_ERR_ARG;
+  if (L > 0 && !coeff_schedule) return DEFL_ERR_ARG;
+  const size_t es = dtype_size(dtype);
+  const size_t gbytes = (size_t)b * m * n * es;
+  {
+    const char* g0 = reinterpret_cast<const char*>(G);
+    const char* o0 = reinterpret_cast<const char*>(out);
+    if (g0 < o0 + gbytes && o0 < g0 + gbytes) return DEFL_ERR_ARG;
+  }
+  const bool tall = m >= n;     // tall: Gram on the n side, X <- X B; otherwise Gram on the m side, X <- B X
+  const bool wide = m <= n;
+  const int ms = m < n ? m : n, ml = m < n ? n : m;
+  int l = k > 0 ? k + oversample : 0;
+  if (l > ms) l = ms;
+  if (k >= ms || l > DEFL_MAX_L || L > DEFL_MAX_STEPS) return DEFL_ERR_RANK;
+  const int engine = opts ? opts->engine : DEFL_ENGINE_AUTO;
+  const int mode = opts ? opts->restore_mode : DEFL_RESTORE_PADDED;
+  if (mode != DEFL_RESTORE_PADDED && mode != DEFL_RESTORE_ADD) return DEFL_ERR_ARG;
+  if (engine < 0 || engine > 2) return DEFL_ERR_ARG;
+  const float gamma = (opts && opts->gamma > 0.f) ? opts->gamma : 1.01f;
+  const int sym = (opts && opts->exploit_symmetry) ? 1 : 0;
+
+  cudaSetDevice(c->device);
+  int rc = ctx_reserve(c, carve_polar(nullptr, b, m, n, dtype, k, l).bytes);
+  if (rc) return rc;
+  PolarWs w = carve_polar(c->ws, b, m, n, dtype, k, l);
+  c->n_marks = 0;
+  c->err[0] = 0;
+  ctx_stage_mark(c);
+  if (ctx_fail(c, fill_int_launch(w.status, b, 0, c->stream, &c->launches), "status")) return DEFL_ERR_CUDA;
+
+  // ---- stage 0: Algorithm 3 ------------------------------------------------------------------
+  if (k > 0) {
+    const float* sk = resolve_sketch(c, opts, b, ms, l, w, &rc);
+    if (rc) return rc;
+    if ((rc = run_brsvd(c, G, b, m, n, dtype, l, power_iters, k, sk, w, engine))) return rc;
+  }
+  ctx_stage_mark(c);
+
+  // iterate buffers: the chain must end in `out`
+  void* bufs[2] = {w.X, out};
+  int cur = (L % 2 == 0) ? 1 : 0;        // X0 goes to bufs[cur]; after L swaps the result is in out
+
+  // ---- stage 1: R = G - P diag(s) W^T, rho = ||R||_F, X0 = R/rho (+ P W^T / gamma) ----------------
+  const float* left = tall ? w.Uk : w.Vk;     // [b,m,k]
+  const float* right = tall ? w.Vk : w.Uk;    // [b,n,k]
+  if (k > 0) {
+    // pass 1: norm of the residual, nothing stored
+    if (ctx_fail(c, scale_cols_launch(right, (long long)n * k, k, b, n, k, w.sv, l, nullptr, 1.f, 0.f, w.Ws,
+                                      (long long)n * k, k, c->stream, &c->launches), "W diag(s)"))
+      return DEFL_ERR_CUDA;
+    GemmDesc g = gemm_desc_zero();
+    g.batch = b; g.M = m; g.N = n; g.K[0] = k;
+    g.A[0] = left; g.sa_i[0] = k; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * k; g.in_dtype = F32;
+    g.B[0] = w.Ws; g.sb_k[0] = 1; g.sb_j[0] = k; g.batch_b[0] = (long long)n * k; g.b_dtype = F32;
+    g.aux = G; g.ld_aux = n; g.batch_aux = (long long)m * n; g.aux_dtype = dtype;
+    g.epilogue = EPI_RESID_NORM; g.partials = w.npart;
+    const int deng = DEFL_ENGINE_SIMT;   // fp32 panels: exact fp32 products
+    g.partials_per_batch = partials_per_batch(g, deng);
+    if ((rc = run_gemm(c, g, deng, "residual norm"))) return rc;
+    if (ctx_fail(c, rho_finalize_launch(w.npart, g.partials_per_batch, b, w.rho, w.inv_rho, w.inv_rho2, w.status,
+                                        c->stream, &c->launches), "rho"))
+      return DEFL_ERR_CUDA;
+    // pass 2: X0 = G/rho - P diag(s/rho - 1/gamma) W^T   (ADD mode: without the 1/gamma term)
+    const float pad = (mode == DEFL_RESTORE_PADDED) ? 1.f / gamma : 0.f;
+    if (ctx_fail(c, scale_cols_launch(right, (long long)n * k, k, b, n, k, w.sv, l, w.inv_rho, -1.f, pad, w.Ws,
+                                      (long long)n * k, k, c->stream, &c->launches), "W diag(coef)"))
+      return DEFL_ERR_CUDA;
+    g.epilogue = EPI_AUX_PLUS; g.partials = nullptr;
+    g.aux_scale = 1.f; g.aux_scale_dev = w.inv_rho; g.alpha = 1.f;
+    g.C = bufs[cur]; g.ldc = n; g.batch_c = (long long)m * n; g.out_dtype = dtype;
+    if ((rc = run_gemm(c, g, deng, "deflate+normalise"))) return rc;
+  } else {
+    const int nblk = 296;
+    if (ctx_fail(c, frob_partial_launch(G, dtype, b, (long long)m * n, nblk, w.npart, c->stream, &c->launches), "frobenius"))
+      return DEFL_ERR_CUDA;
+    if (ctx_fail(c, rho_finalize_launch(w.npart, nblk, b, w.rho, w.inv_rho, w.inv_rho2, w.status, c->stream,
+                                        &c->launches), "rho"))
+      return DEFL_ERR_CUDA;
+    if (ctx_fail(c, scale_launch(G, dtype, bufs[cur], dtype, b, (long long)m * n, w.inv_rho, c->stream, &c->launches), "normalise"))
+      return DEFL_ERR_CUDA;
+  }
+  ctx_stage_mark(c);
+
+  // ---- stage 2: X <- a X + b (X X^T) X + c (X X^T)^2 X, L times, through the short-side Gram -------
+  for (int t = 0; t < L; ++t) {
+    const float ca = coeff_schedule[3 * t], cb = coeff_schedule[3 * t + 1], cc = coeff_schedule[3 * t + 2];
+    const void* X = bufs[cur];
+    void* Xn = bufs[cur ^ 1];
+    GemmDesc g = gemm_desc_zero();
+    g.batch = b; g.in_dtype = dtype; g.b_dtype = dtype; g.out_dtype = dtype;
+    // A_t = X X^T (wide) or X^T X (tall), ms x ms, symmetric
+    g.M = ms; g.N = ms; g.K[0] = ml;
+    g.A[0] = X; g.B[0] = X; g.batch_a[0] = g.batch_b[0] = (long long)m * n;
+    if (wide) { g.sa_i[0] = n; g.sa_k[0] = 1; g.sb_k[0] = 1; g.sb_j[0] = n; }
+    else { g.sa_i[0] = 1; g.sa_k[0] = n; g.sb_k[0] = n; g.sb_j[0] = 1; }
+    g.C = w.Am; g.ldc = ms; g.batch_c = (long long)ms * ms;
+    g.epilogue = EPI_STORE; g.symmetric = sym;
+    if ((rc = run_gemm(c, g, engine, "gram"))) return rc;
+    // B_t = a I + b A_t + c A_t A_t
+    g = gemm_desc_zero();
+    g.batch = b; g.in_dtype = dtype; g.b_dtype = dtype; g.out_dtype = dtype;
+    g.M = ms; g.N = ms; g.K[0] = ms;
+    g.A[0] = w.Am; g.sa_i[0] = ms; g.sa_k[0] = 1; g.batch_a[0] = (long long)ms * ms;
+    g.B[0] = w.Am; g.sb_k[0] = 1; g.sb_j[0] = ms; g.batch_b[0] = (long long)ms * ms;   // A_t symmetric: rows as columns
+    g.C = w.Bm; g.ldc = ms; g.batch_c = (long long)ms * ms;
+    g.aux = w.Am; g.ld_aux = ms; g.batch_aux = (long long)ms * ms; g.aux_dtype = dtype;
+    g.epilogue = EPI_POLY; g.pa = ca; g.pb = cb; g.pc = cc; g.symmetric = sym;
+    if ((rc = run_gemm(c, g, engine, "polynomial"))) return rc;
+    // X <- B_t X (wide) or X B_t (tall)
+    g = gemm_desc_zero();
+    g.batch = b; g.in_dtype = dtype; g.b_dtype = dtype; g.out_dtype = dtype;
+    g.M = m; g.N = n;
+    if (wide) {
+      g.K[0] = m;
+      g.A[0] = w.Bm; g.sa_i[0] = m; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * m;
+      g.B[0] = X; g.sb_k[0] = n; g.sb_j[0] = 1; g.batch_b[0] = (long long)m * n;
+    } else {
+      g.K[0] = n;
+      g.A[0] = X; g.sa_i[0] = n; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * n;
+      g.B[0] = w.Bm; g.sb_k[0] = 1; g.sb_j[0] = n; g.batch_b[0] = (long long)n * n;   // B_t symmetric
+    }
+    g.C = Xn; g.ldc = n; g.batch_c = (long long)m * n;
+    g.epilogue = EPI_STORE;
+    if ((rc = run_gemm(c, g, engine, "apply"))) return rc;
+    cur ^= 1;
+  }
+  ctx_stage_mark(c);
+
+  // ---- stage 3: restore (Eq. 3) in ADD mode: out += P W^T ------------------------------------------
+  if (k > 0 && mode == DEFL_RESTORE_ADD) {
+    GemmDesc g = gemm_desc_zero();
+    g.batch = b; g.M = m; g.N = n; g.K[0] = k;
+    g.A[0] = left; g.sa_i[0] = k; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * k; g.in_dtype = F32;
+    g.B[0] = right; g.sb_k[0] = 1; g.sb_j[0] = k; g.batch_b[0] = (long long)n * k; g.b_dtype = F32;
+    g.aux = out; g.ld_aux = n; g.batch_aux = (long long)m * n; g.aux_dtype = dtype;
+    g.C = out; g.ldc = n; g.batch_c = (long long)m * n; g.out_dtype = dtype;
+    g.epilogue = EPI_AUX_PLUS;
+    if ((rc = run_gemm(c, g, DEFL_ENGINE_SIMT, "restore"))) return rc;
+  }
+  ctx_stage_mark(c);
+
+  if (info) {
+    if (info->s && l > 0 &&
+        ctx_fail(c, cudaMemcpyAsync(info->s, w.sv, (size_t)b * l * sizeof(float), cudaMemcpyDeviceToDevice, c->stream), "copy s"))
+      return DEFL_ERR_CUDA;
+    if (info->rho &&
+        ctx_fail(c, cudaMemcpyAsync(info->rho, w.rho, (size_t)b * sizeof(float), cudaMemcpyDeviceToDevice, c->stream), "copy rho"))
+      return DEFL_ERR_CUDA;
+    if (info->status) {
+      // fold the engine's device-wait word into every matrix's status
+      if (ctx_fail(c, or_status_launch(w.status, b, c->wait_status, c->stream, &c->launches), "status"))
+        return DEFL_ERR_CUDA;
+      if (ctx_fail(c, cudaMemcpyAsync(info->status, w.status, (size_t)b * sizeof(int), cudaMemcpyDeviceToDevice, c->stream), "copy status"))
+        return DEFL_ERR_CUDA;
+    }
+  }
+  return DEFL_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,72 @@
+// Shared declarations of the CUDA library: the product descriptor that both engines consume,
+// element-type helpers and the internal kernel-launcher prototypes.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace defl {
+
+enum DType { BF16 = 0, F32 = 1 };
+
+__host__ __device__ inline size_t dtype_size(int dt) { return dt == BF16 ? 2 : 4; }
+
+// What happens to the fp32 accumulator tile acc[i,j] of C = opA(A) opB(B).
+enum Epilogue {
+  EPI_STORE = 0,      // C = alpha * acc
+  EPI_POLY = 1,       // C = pa * [i==j] + pb * aux[i,j] + pc * acc        (B_t = a I + b A_t + c A_t^2, Eq. 2)
+  EPI_AUX_PLUS = 2,   // C = aux_scale * aux[i,j] + alpha * acc            (deflate+normalise, restore, PSD reconstruct)
+  EPI_RESID_NORM = 3  // partial sums of (aux[i,j] - acc)^2, nothing stored (||G - U_k S_k V_k^T||_F^2)
+};
+
+// One batched product. Element (i,kk) of opA is A[i*sa_i + kk*sa_k]; element (kk,j) of opB is
+// B[kk*sb_k + j*sb_j]; C and aux are row-major [M,N] with leading dimension ldc / ld_aux.
+// Up to two K segments are summed into the same accumulator: acc = A0 B0 + A1 B1 (used for the
+// split-precision panels and for the restore step appended to the last filter product).
+struct GemmDesc {
+  int batch, M, N;
+  int nseg;
+  int K[2];
+  const void* A[2]; long long sa_i[2], sa_k[2], batch_a[2];
+  const void* B[2]; long long sb_k[2], sb_j[2], batch_b[2];
+  int in_dtype;                 // type of A (both segments)
+  int b_dtype;                  // type of B (both segments); the tensor engine needs b_dtype == in_dtype
+  void* C; long long ldc, batch_c; int out_dtype;
+  const void* aux; long long ld_aux, batch_aux; int aux_dtype;
+  int epilogue;
+  float alpha, aux_scale, pa, pb, pc;
+  const float* alpha_dev;       // optional per-batch multiplier of alpha (device, [batch])
+  const float* aux_scale_dev;   // optional per-batch multiplier of aux_scale (device, [batch])
+  double* partials;             // EPI_RESID_NORM: [batch, partials_per_batch] written, one slot per CTA-warp
+  int partials_per_batch;
+  int symmetric;                // output is symmetric (M == N): compute upper tiles only and mirror
+};
+
+inline GemmDesc gemm_desc_zero() {
+  GemmDesc g;
+  memset(&g, 0, sizeof(g));
+  g.nseg = 1;
+  g.alpha = 1.f;
+  g.aux_scale = 1.f;
+  return g;
+}
+
+// Engines (each returns cudaGetLastError() of its launch; they never synchronise).
+cudaError_t gemm_simt_launch(const GemmDesc& g, cudaStream_t st, long long* launches);
+int gemm_simt_partials_per_batch(const GemmDesc& g);
+// Tensor-core engine: returns cudaErrorNotSupported when the descriptor cannot be expressed
+// as TMA-tiled tcgen05 products (alignment, type), without launching anything.
+cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word, int num_sms, long long* launches);
+bool gemm_tc_supported(const GemmDesc& g);
+int gemm_tc_partials_per_batch(const GemmDesc& g);
+
+__device__ __forceinline__ float ld_as_float(const void* p, long long idx, int dt) {
+  return dt == BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[idx])
+                    : reinterpret_cast<const float*>(p)[idx];
+}
+__device__ __forceinline__ void st_from_float(void* p, long long idx, int dt, float v) {
+  if (dt == BF16) reinterpret_cast<__nv_bfloat16*>(p)[idx] = __float2bfloat16_rn(v);
+  else reinterpret_cast<float*>(p)[idx] = v;
+}
+
+}  // namespace defl

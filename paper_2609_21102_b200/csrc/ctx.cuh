@@ -1,0 +1,30 @@
+// The context behind the opaque defl_ctx handle, shared by api.cu and psd.cu.
+#pragma once
+#include <cuda_runtime.h>
+#include "common.cuh"
+
+#define DEFL_MAX_MARKS 12
+
+struct defl_ctx {
+  int device;
+  int num_sms;
+  cudaStream_t stream;
+  void* ws;              // scratch memory owned by the context
+  size_t ws_bytes;
+  int* wait_status;      // device word: the tensor engine ORs DEFL_ST_DEVICE_WAIT into it
+  long long launches;    // kernels launched so far
+  bool profiling;
+  int n_marks;
+  cudaEvent_t marks[DEFL_MAX_MARKS];
+  char err[256];
+};
+
+namespace defl {
+size_t align_up(size_t x, size_t a);
+bool ctx_fail(defl_ctx* c, cudaError_t e, const char* where);
+int ctx_reserve(defl_ctx* c, size_t bytes);
+void ctx_stage_mark(defl_ctx* c);
+int run_gemm(defl_ctx* c, const GemmDesc& g, int engine, const char* what);
+int partials_per_batch(const GemmDesc& g, int engine);
+cudaError_t or_status_launch(int* status, int n, const int* word, cudaStream_t st, long long* launches);
+}  // namespace defl

@@ -1,0 +1,570 @@
+// Tensor-core product engine for sm_100a: persistent, warp-specialised tcgen05 kernel.
+//
+//   warp 0      TMA producer: cp.async.bulk.tensor loads of the A and B operand tiles into a ring of
+//               128-byte-swizzled shared-memory stages, signalled through mbarriers
+//   warp 1      allocates tensor memory and issues tcgen05.mma (one elected lane), fp32 accumulators
+//               in tensor memory, two accumulator buffers so that the epilogue of tile i overlaps the
+//               products of tile i+1
+//   warps 2..5  epilogue: tcgen05.ld of the accumulator (each warp its own 32-lane quarter), the
+//               element-wise epilogue (store / polynomial / residual / norm partials), global stores
+//
+// A tile is 128 x BN outputs (BN chosen per call, a multiple of 16 up to 256), K is walked in blocks of
+// 128 bytes (64 bf16 or 32 tf32 values). Either operand may be K-major (K contiguous in global memory)
+// or MN-major; the shared-memory matrix descriptors and the instruction descriptor are built to match.
+// No cluster launch and no multicast: every CTA loads its own operands. Every wait is bounded: when one
+// runs out the kernel raises DEFL_ST_DEVICE_WAIT in the status word, stops waiting and drains.
+#include "common.cuh"
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include <mutex>
+
+namespace defl {
+
+namespace {
+
+constexpr int TILE_M = 128;
+constexpr int KBYTES = 128;                 // bytes of K per stage row (one swizzle span)
+constexpr int NUM_THREADS = 192;
+constexpr int MAX_STAGES = 6;
+constexpr unsigned long long WAIT_NS = 2000000000ull;  // 2 s per wait before giving up
+
+struct TcParams {
+  CUtensorMap tmA[2];
+  CUtensorMap tmB[2];
+  int nseg;
+  int kblocks[2];              // K blocks per segment
+  int M, N, batch;
+  int BN;                      // tile width (UMMA N)
+  int tiles_m, tiles_n;
+  long long total_tiles;
+  int a_mn_major, b_mn_major;  // 0 = K-major, 1 = MN-major
+  int esize;                   // operand element size in bytes (2 bf16, 4 tf32)
+  int stages;
+  uint32_t a_stage_bytes, b_stage_bytes;
+  uint32_t a_boxes, b_boxes;   // TMA boxes per stage per operand
+  uint32_t a_box_bytes, b_box_bytes;
+  uint32_t a_box_rows, b_box_rows;   // MN extent covered by one box (K-major) or 128B/esize (MN-major)
+  uint32_t idesc;
+  // epilogue
+  int epilogue, out_dtype, aux_dtype, symmetric;
+  void* C; long long ldc, batch_c;
+  const void* aux; long long ld_aux, batch_aux;
+  float alpha, aux_scale, pa, pb, pc;
+  const float* alpha_dev; const float* aux_scale_dev;
+  double* partials; int partials_per_batch;
+  int* status;
+};
+
+// ----------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait. `abort_flag` (shared memory) short-circuits every later wait once one has failed.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (*abort_flag) return false;
+  for (int i = 0; i < 4096; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > WAIT_NS) {
+      *abort_flag = 1;
+      if (status) atomicOr(status, 8);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+template <int KIND_TF32>
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  if (KIND_TF32) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  }
+}
+// arrives on the mbarrier once every tcgen05.mma issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (sm_100 format): start address, leading/stride byte offsets (all >> 4),
+// version 1 at bit 46, 128-byte swizzle (layout type 2) at bits 61..63.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+// ----------------------------------------------------------------------------- the kernel
+template <int KIND_TF32>
+__global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_constant__ TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];
+  __shared__ __align__(8) uint64_t acc_full_bar[2];
+  __shared__ __align__(8) uint64_t acc_empty_bar[2];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzled tiles need 1024-byte alignment
+  const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
+  const int total_kblocks = p.kblocks[0] + (p.nseg > 1 ? p.kblocks[1] : 0);
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&acc_full_bar[a]), 1); mbar_init(smem_u32(&acc_empty_bar[a]), 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tmem_base_slot), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      for (long long tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+        const int tn = (int)(tile % p.tiles_n);
+        const int tm = (int)((tile / p.tiles_n) % p.tiles_m);
+        const int bz = (int)(tile / ((long long)p.tiles_n * p.tiles_m));
+        if (p.symmetric && (tn + 1) * p.BN <= tm * TILE_M) continue;   // tile entirely below the diagonal
+        for (int seg = 0; seg < p.nseg; ++seg) {
+          for (int kb = 0; kb < p.kblocks[seg]; ++kb) {
+            mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag, p.status);
+            if (abort_flag) break;
+            const uint32_t fb = smem_u32(&full_bar[stage]);
+            mbar_expect_tx(fb, stage_bytes);
+            const uint32_t sa = smem_base + stage * stage_bytes;
+            const uint32_t sb = sa + p.a_stage_bytes;
+            const int k0 = kb * (KBYTES / p.esize);
+            for (uint32_t bx = 0; bx < p.a_boxes; ++bx) {
+              const int mn0 = tm * TILE_M + (int)(bx * p.a_box_rows);
+              if (p.a_mn_major) tma_load_3d(sa + bx * p.a_box_bytes, &p.tmA[seg], fb, mn0, k0, bz);
+              else tma_load_3d(sa + bx * p.a_box_bytes, &p.tmA[seg], fb, k0, mn0, bz);
+            }
+            for (uint32_t bx = 0; bx < p.b_boxes; ++bx) {
+              const int mn0 = tn * p.BN + (int)(bx * p.b_box_rows);
+              if (p.b_mn_major) tma_load_3d(sb + bx * p.b_box_bytes, &p.tmB[seg], fb, mn0, k0, bz);
+              else tma_load_3d(sb + bx * p.b_box_bytes, &p.tmB[seg], fb, k0, mn0, bz);
+            }
+            if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
+          }
+          if (abort_flag) break;
+        }
+        if (abort_flag) break;
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+      const uint32_t a_kstep = p.a_mn_major ? (uint32_t)(32 / p.esize) * 128u : 32u;   // bytes per UMMA K step
+      const uint32_t b_kstep = p.b_mn_major ? (uint32_t)(32 / p.esize) * 128u : 32u;
+      const uint32_t a_lbo = p.a_mn_major ? p.a_box_bytes : 16u;
+      const uint32_t b_lbo = p.b_mn_major ? p.b_box_bytes : 16u;
+      for (long long tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+        const int tn = (int)(tile % p.tiles_n);
+        const int tm = (int)((tile / p.tiles_n) % p.tiles_m);
+        if (p.symmetric && (tn + 1) * p.BN <= tm * TILE_M) continue;
+        mbar_wait(smem_u32(&acc_empty_bar[acc]), acc_phase ^ 1u, &abort_flag, p.status);
+        if (abort_flag) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * 256u;
+        for (int kb = 0; kb < total_kblocks; ++kb) {
+          mbar_wait(smem_u32(&full_bar[stage]), phase, &abort_flag, p.status);
+          if (abort_flag) break;
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * stage_bytes;
+          const uint32_t sb = sa + p.a_stage_bytes;
+#pragma unroll
+          for (int kk = 0; kk < KBYTES / 32; ++kk) {
+            const uint64_t adesc = make_smem_desc(sa + kk * a_kstep, a_lbo, 1024u);
+            const uint64_t bdesc = make_smem_desc(sb + kk * b_kstep, b_lbo, 1024u);
+            umma<KIND_TF32>(d_tmem, adesc, bdesc, p.idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+          }
+          umma_commit(smem_u32(&empty_bar[stage]));          // frees the stage once these products are done
+          if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
+        }
+        if (abort_flag) break;
+        umma_commit(smem_u32(&acc_full_bar[acc]));           // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps
+    const int q = warp & 3;                 // tensor-memory lane quarter this warp may read
+    uint32_t acc = 0, acc_phase = 0;
+    for (long long tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+      const int tn = (int)(tile % p.tiles_n);
+      const int tm = (int)((tile / p.tiles_n) % p.tiles_m);
+      const int bz = (int)(tile / ((long long)p.tiles_n * p.tiles_m));
+      if (p.symmetric && (tn + 1) * p.BN <= tm * TILE_M) continue;
+      const bool ok = mbar_wait(smem_u32(&acc_full_bar[acc]), acc_phase, &abort_flag, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      const int gi = tm * TILE_M + q * 32 + lane;
+      const bool row_ok = gi < p.M;
+      float alpha = p.alpha, aux_scale = p.aux_scale;
+      if (p.alpha_dev) alpha *= p.alpha_dev[bz];
+      if (p.aux_scale_dev) aux_scale *= p.aux_scale_dev[bz];
+      const long long crow = (long long)bz * p.batch_c + (long long)gi * p.ldc;
+      const long long xrow = (long long)bz * p.batch_aux + (long long)gi * p.ld_aux;
+      double sq = 0.0;
+      for (int c0 = 0; c0 < p.BN; c0 += 16) {
+        uint32_t r[16];
+        __syncwarp();
+        tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256u + (uint32_t)c0, r);
+        tmem_ld_wait();
+        const int gj0 = tn * p.BN + c0;
+        if (gj0 >= p.N) continue;           // warp-uniform
+        float v[16];
+        float sqf = 0.f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int gj = gj0 + j;
+          const float a = __uint_as_float(r[j]);
+          float x = 0.f;
+          const bool in = row_ok && gj < p.N;
+          if (p.epilogue != EPI_STORE && in) x = ld_as_float(p.aux, xrow + gj, p.aux_dtype);
+          float o;
+          if (p.epilogue == EPI_STORE) o = alpha * a;
+          else if (p.epilogue == EPI_POLY) o = p.pb * x + p.pc * a + ((gi == gj) ? p.pa : 0.f);
+          else if (p.epilogue == EPI_AUX_PLUS) o = aux_scale * x + alpha * a;
+          else { o = 0.f; if (in) { const float d = x - a; sqf = fmaf(d, d, sqf); } }
+          v[j] = o;
+        }
+        if (p.epilogue == EPI_RESID_NORM) { sq += (double)sqf; continue; }
+        if (!row_ok) continue;
+        const bool full = (gj0 + 16 <= p.N);
+        if (!p.symmetric) {
+          if (full && p.out_dtype == BF16 && ((crow + gj0) & 7) == 0) {
+            uint4 pk[2];
+            __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(pk);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) h[j] = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.C) + crow + gj0);
+            dst[0] = pk[0]; dst[1] = pk[1];
+          } else if (full && p.out_dtype == F32 && ((crow + gj0) & 3) == 0) {
+            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + crow + gj0);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              if (gj0 + j < p.N) st_from_float(p.C, crow + gj0 + j, p.out_dtype, v[j]);
+          }
+        } else {
+          // symmetric output: write the upper part directly and its mirror image; across the warp the
+          // mirrored stores of one column are contiguous (lanes are consecutive rows)
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int gj = gj0 + j;
+            if (gj >= p.N) continue;
+            if (gj >= gi) st_from_float(p.C, crow + gj, p.out_dtype, v[j]);
+            if (gj > gi) st_from_float(p.C, (long long)bz * p.batch_c + (long long)gj * p.ldc + gi, p.out_dtype, v[j]);
+          }
+        }
+      }
+      // release the accumulator buffer
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&acc_empty_bar[acc]));
+      if (p.epilogue == EPI_RESID_NORM) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sq += __shfl_down_sync(0xffffffffu, sq, o);
+        if (lane == 0)
+          p.partials[(long long)bz * p.partials_per_batch + ((long long)tm * p.tiles_n + tn) * 4 + (warp - 2)] = sq;
+      }
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag && threadIdx.x == 0) {
+    // a wait ran out: give copies that may still be in flight a bounded time to land before the
+    // shared memory is released
+    const unsigned long long t0 = global_ns();
+    while (global_ns() - t0 < 2000000ull) { }
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ----------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  });
+  return fn;
+}
+
+struct OperandPlan {
+  bool mn_major;
+  uint32_t boxes, box_bytes, box_rows, stage_bytes;
+};
+
+// Operand viewed as [batch][MN][K] with element strides s_mn, s_k. One of the strides must be 1.
+bool plan_operand(long long s_mn, long long s_k, int tile_mn, int esize, OperandPlan* pl) {
+  const int span = KBYTES / esize;   // elements per 128 bytes
+  if (s_k == 1) {
+    pl->mn_major = false;
+    pl->boxes = 1;
+    pl->box_rows = tile_mn;
+    pl->box_bytes = (uint32_t)tile_mn * KBYTES;
+    pl->stage_bytes = pl->box_bytes;
+    return true;
+  }
+  if (s_mn == 1) {
+    pl->mn_major = true;
+    pl->boxes = (tile_mn + span - 1) / span;
+    pl->box_rows = span;
+    pl->box_bytes = (uint32_t)span * KBYTES;     // span K-rows of 128 bytes
+    pl->stage_bytes = pl->boxes * pl->box_bytes;
+    return true;
+  }
+  return false;
+}
+
+bool encode_map(CUtensorMap* tm, const void* base, int esize, bool tf32, bool mn_major, long long MN, long long K,
+                long long s_mn, long long s_k, long long batch, long long batch_stride, uint32_t box_rows) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return false;
+  const uint32_t span = KBYTES / esize;
+  cuuint64_t dims[3];
+  cuuint64_t strides[2];
+  cuuint32_t box[3];
+  cuuint32_t estr[3] = {1, 1, 1};
+  if (!mn_major) {          // inner = K
+    dims[0] = (cuuint64_t)K; dims[1] = (cuuint64_t)MN; dims[2] = (cuuint64_t)batch;
+    strides[0] = (cuuint64_t)s_mn * esize; strides[1] = (cuuint64_t)batch_stride * esize;
+    box[0] = span; box[1] = box_rows; box[2] = 1;
+  } else {                  // inner = MN
+    dims[0] = (cuuint64_t)MN; dims[1] = (cuuint64_t)K; dims[2] = (cuuint64_t)batch;
+    strides[0] = (cuuint64_t)s_k * esize; strides[1] = (cuuint64_t)batch_stride * esize;
+    box[0] = span; box[1] = span; box[2] = 1;
+  }
+  if (batch == 1) strides[1] = strides[0] * dims[1];
+  const CUtensorMapDataType dt = (esize == 2) ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                              : (tf32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32);
+  const CUresult r = enc(tm, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int choose_bn(int N) {
+  // widest tile that wastes the fewest padded columns; ties go to the wider tile
+  int best = 16;
+  long long best_cost = -1;
+  for (int bn = 256; bn >= 16; bn -= 16) {
+    const long long tiles = (N + bn - 1) / bn;
+    const long long padded = tiles * bn;
+    // cost: padded columns plus a fixed per-tile overhead that favours fewer, wider tiles
+    const long long cost = padded + tiles * 24;
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
+  }
+  return best;
+}
+
+}  // namespace
+
+bool gemm_tc_supported(const GemmDesc& g) {
+  if (g.batch <= 0 || g.M <= 0 || g.N <= 0) return false;
+  if (g.nseg < 1 || g.nseg > 2) return false;
+  if (g.b_dtype != g.in_dtype) return false;
+  const int esize = (int)dtype_size(g.in_dtype);
+  if (g.symmetric && g.M != g.N) return false;
+  for (int s = 0; s < g.nseg; ++s) {
+    if (g.K[s] <= 0) return false;
+    if (!aligned16(g.A[s]) || !aligned16(g.B[s])) return false;
+    // one unit stride per operand, the other stride and the batch stride multiples of 16 bytes
+    const long long a_other = (g.sa_k[s] == 1) ? g.sa_i[s] : g.sa_k[s];
+    const long long b_other = (g.sb_k[s] == 1) ? g.sb_j[s] : g.sb_k[s];
+    if (g.sa_k[s] != 1 && g.sa_i[s] != 1) return false;
+    if (g.sb_k[s] != 1 && g.sb_j[s] != 1) return false;
+    // tf32 operands are taken K-major only (an MN-major tf32 tile needs a different swizzle atom;
+    // the symmetric fp32 products this engine serves never need it)
+    if (esize == 4 && (g.sa_k[s] != 1 || g.sb_k[s] != 1)) return false;
+    if ((a_other * esize) % 16 || (b_other * esize) % 16) return false;
+    if (g.batch > 1 && ((g.batch_a[s] * esize) % 16 || (g.batch_b[s] * esize) % 16)) return false;
+    // both segments must agree on the operand orientation (one instruction descriptor per launch)
+    if (s > 0) {
+      if ((g.sa_k[s] == 1) != (g.sa_k[0] == 1) || (g.sb_k[s] == 1) != (g.sb_k[0] == 1)) return false;
+    }
+  }
+  return get_encode_fn() != nullptr;
+}
+
+int gemm_tc_partials_per_batch(const GemmDesc& g) {
+  const int bn = choose_bn(g.N);
+  return ((g.M + TILE_M - 1) / TILE_M) * ((g.N + bn - 1) / bn) * 4;
+}
+
+cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word, int num_sms, long long* launches) {
+  if (!gemm_tc_supported(g)) return cudaErrorNotSupported;
+  TcParams p;
+  memset(&p, 0, sizeof(p));
+  const int esize = (int)dtype_size(g.in_dtype);
+  const bool tf32 = (g.in_dtype == F32);
+  p.esize = esize;
+  p.M = g.M; p.N = g.N; p.batch = g.batch;
+  p.BN = choose_bn(g.N);
+  p.tiles_m = (g.M + TILE_M - 1) / TILE_M;
+  p.tiles_n = (g.N + p.BN - 1) / p.BN;
+  p.total_tiles = (long long)p.tiles_m * p.tiles_n * g.batch;
+  p.nseg = g.nseg;
+  OperandPlan pa, pb;
+  // when a dimension has extent 1 both strides may look "unit"; prefer K-major
+  if (!plan_operand(g.sa_i[0], g.sa_k[0], TILE_M, esize, &pa)) return cudaErrorNotSupported;
+  if (!plan_operand(g.sb_j[0], g.sb_k[0], p.BN, esize, &pb)) return cudaErrorNotSupported;
+  p.a_mn_major = pa.mn_major; p.b_mn_major = pb.mn_major;
+  p.a_boxes = pa.boxes; p.a_box_bytes = pa.box_bytes; p.a_box_rows = pa.box_rows; p.a_stage_bytes = pa.stage_bytes;
+  p.b_boxes = pb.boxes; p.b_box_bytes = pb.box_bytes; p.b_box_rows = pb.box_rows; p.b_stage_bytes = pb.stage_bytes;
+  const int span = KBYTES / esize;
+  for (int s = 0; s < g.nseg; ++s) {
+    p.kblocks[s] = (g.K[s] + span - 1) / span;
+    if (!encode_map(&p.tmA[s], g.A[s], esize, tf32, pa.mn_major, g.M, g.K[s], g.sa_i[s], g.sa_k[s], g.batch,
+                    g.batch_a[s], pa.box_rows))
+      return cudaErrorInvalidValue;
+    if (!encode_map(&p.tmB[s], g.B[s], esize, tf32, pb.mn_major, g.N, g.K[s], g.sb_j[s], g.sb_k[s], g.batch,
+                    g.batch_b[s], pb.box_rows))
+      return cudaErrorInvalidValue;
+  }
+  const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
+  const uint32_t smem_budget = 200 * 1024;
+  int stages = (int)(smem_budget / stage_bytes);
+  if (stages > MAX_STAGES) stages = MAX_STAGES;
+  if (stages < 2) return cudaErrorNotSupported;
+  p.stages = stages;
+  // instruction descriptor: fp32 accumulate, operand format, majors, N >> 3 at bit 17, M >> 4 at bit 24
+  const uint32_t fmt = tf32 ? 2u : 1u;
+  p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)p.a_mn_major << 15) | ((uint32_t)p.b_mn_major << 16) |
+            ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+  p.epilogue = g.epilogue; p.out_dtype = g.out_dtype; p.aux_dtype = g.aux_dtype; p.symmetric = g.symmetric;
+  p.C = g.C; p.ldc = g.ldc; p.batch_c = g.batch_c;
+  p.aux = g.aux; p.ld_aux = g.ld_aux; p.batch_aux = g.batch_aux;
+  p.alpha = g.alpha; p.aux_scale = g.aux_scale; p.pa = g.pa; p.pb = g.pb; p.pc = g.pc;
+  p.alpha_dev = g.alpha_dev; p.aux_scale_dev = g.aux_scale_dev;
+  p.partials = g.partials; p.partials_per_batch = g.partials_per_batch;
+  p.status = status_word;
+
+  const size_t smem = (size_t)stages * stage_bytes + 1024;
+  cudaError_t e;
+  if (tf32) e = cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  else e = cudaFuncSetAttribute(gemm_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  long long grid = p.total_tiles < num_sms ? p.total_tiles : num_sms;
+  if (grid < 1) grid = 1;
+  if (tf32) gemm_tc_kernel<1><<<(unsigned)grid, NUM_THREADS, smem, st>>>(p);
+  else gemm_tc_kernel<0><<<(unsigned)grid, NUM_THREADS, smem, st>>>(p);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace defl

@@ -1,0 +1,513 @@
+// Small-panel kernels of the randomized SVD front end (Algorithm 3) and helpers:
+//   * Gram matrices of tall skinny panels (CholeskyQR and the Gram core of the thin SVD)
+//   * l x l Cholesky factorisation + triangular inverse in shared memory (fp64)
+//   * one-sided Jacobi eigensolver of the l x l core in shared memory, one warp per column
+//     pair, rotations through warp shuffles (fp64)
+//   * panel x small-matrix products, column scaling, Frobenius partial sums, scaling,
+//     the counter-based Gaussian fill.
+// All reductions run in a fixed order so that repeated runs are bit-identical.
+#include "common.cuh"
+#include "panel.cuh"
+
+namespace defl {
+
+// ---------------------------------------------------------------------------------------------
+// Gram partials: for panel Y[b, rows, l] (fp32, leading dimension ld), CTA (chunk, batch) writes
+// partial[b, chunk, l, l] = sum over its rows of y_r y_r^T  (fp32 products over 32-row groups,
+// groups added in fp64).
+// ---------------------------------------------------------------------------------------------
+constexpr int GRAM_ROWS = 256;   // rows per CTA
+constexpr int GRAM_SUB = 32;     // rows per fp32 sub-accumulation
+
+__global__ void __launch_bounds__(256) gram_partial_kernel(const float* __restrict__ Y, long long batch_stride,
+                                                           int rows, int l, int ld, int nchunk,
+                                                           double* __restrict__ partial) {
+  __shared__ float tile[GRAM_SUB][MAX_L + 1];
+  const int chunk = blockIdx.x, bz = blockIdx.y, tid = threadIdx.x;
+  const float* Yb = Y + (long long)bz * batch_stride;
+  const int tx = tid % 16, ty = tid / 16;   // 16 x 16 threads, each a 4 x 4 block of the l x l Gram
+  double acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+  const int r_begin = chunk * GRAM_ROWS, r_end = min(rows, r_begin + GRAM_ROWS);
+  for (int r0 = r_begin; r0 < r_end; r0 += GRAM_SUB) {
+    for (int e = tid; e < GRAM_SUB * l; e += 256) {
+      const int rr = e / l, c = e % l;
+      const int gr = r0 + rr;
+      tile[rr][c] = (gr < r_end) ? Yb[(long long)gr * ld + c] : 0.f;
+    }
+    __syncthreads();
+    float f[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) f[i][j] = 0.f;
+    for (int rr = 0; rr < GRAM_SUB; ++rr) {
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = (ty * 4 + i < l) ? tile[rr][ty * 4 + i] : 0.f;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) b[j] = (tx * 4 + j < l) ? tile[rr][tx * 4 + j] : 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) f[i][j] = fmaf(a[i], b[j], f[i][j]);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] += (double)f[i][j];
+    __syncthreads();
+  }
+  double* out = partial + ((long long)bz * nchunk + chunk) * l * l;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int gi = ty * 4 + i, gj = tx * 4 + j;
+      if (gi < l && gj < l) out[gi * l + gj] = acc[i][j];
+    }
+}
+
+int gram_num_chunks(int rows) { return (rows + GRAM_ROWS - 1) / GRAM_ROWS; }
+
+cudaError_t gram_partial_launch(const float* Y, long long batch_stride, int batch, int rows, int l, int ld,
+                                double* partial, cudaStream_t st, long long* launches) {
+  const int nchunk = gram_num_chunks(rows);
+  gram_partial_kernel<<<dim3(nchunk, batch), 256, 0, st>>>(Y, batch_stride, rows, l, ld, nchunk, partial);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Cholesky of W = sum of partials (l x l, fp64, shared memory), W = R^T R, output Rinv = R^-1
+// (upper triangular, fp32, row-major [l,l]). A non-positive pivot restarts with W + shift I and
+// sets DEFL_ST_CHOL_SHIFT (bit 1) in status[b].
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) chol_inv_kernel(const double* __restrict__ partial, int nchunk, int l,
+                                                       float* __restrict__ Rinv, int* __restrict__ status) {
+  extern __shared__ double sm[];
+  double* W = sm;              // [l][l] original Gram
+  double* Lm = sm + l * l;     // [l][l] lower factor, then its inverse
+  __shared__ int bad;
+  const int bz = blockIdx.x, tid = threadIdx.x;
+  const double* pb = partial + (long long)bz * nchunk * l * l;
+  for (int e = tid; e < l * l; e += blockDim.x) {
+    double t = 0.0;
+    for (int c = 0; c < nchunk; ++c) t += pb[(long long)c * l * l + e];
+    W[e] = t;
+  }
+  __syncthreads();
+  // symmetrise exactly
+  for (int e = tid; e < l * l; e += blockDim.x) {
+    const int i = e / l, j = e % l;
+    if (i < j) { const double a = 0.5 * (W[i * l + j] + W[j * l + i]); Lm[i * l + j] = a; Lm[j * l + i] = a; }
+    else if (i == j) Lm[e] = W[e];
+  }
+  __syncthreads();
+  for (int e = tid; e < l * l; e += blockDim.x) W[e] = Lm[e];
+  __syncthreads();
+  double trace = 0.0;
+  for (int i = 0; i < l; ++i) trace += W[i * l + i];
+  double shift = 0.0;
+  for (int attempt = 0; attempt < 6; ++attempt) {
+    for (int e = tid; e < l * l; e += blockDim.x) {
+      const int i = e / l, j = e % l;
+      Lm[e] = W[e] + ((i == j) ? shift : 0.0);
+    }
+    if (tid == 0) bad = 0;
+    __syncthreads();
+    // right-looking Cholesky on the lower triangle
+    for (int j = 0; j < l; ++j) {
+      const double d = Lm[j * l + j];
+      if (!(d > 0.0) || !isfinite(d)) { if (tid == 0) bad = 1; }
+      __syncthreads();
+      if (bad) break;
+      const double sd = sqrt(d);
+      for (int i = j + tid; i < l; i += blockDim.x) Lm[i * l + j] = (i == j) ? sd : Lm[i * l + j] / sd;
+      __syncthreads();
+      const int rem = l - j - 1;
+      for (int e = tid; e < rem * rem; e += blockDim.x) {
+        const int i = j + 1 + e / rem, c = j + 1 + e % rem;
+        if (c <= i) Lm[i * l + c] -= Lm[i * l + j] * Lm[c * l + j];
+      }
+      __syncthreads();
+    }
+    if (!bad) break;
+    // shift as in shifted CholeskyQR: proportional to the trace, growing per attempt
+    shift = (shift == 0.0) ? 1e-10 * (trace > 0.0 ? trace : 1.0) : shift * 100.0;
+    if (tid == 0 && status) atomicOr(&status[bz], 1);
+    __syncthreads();
+  }
+  // Linv by forward substitution, one column per thread: L X = I
+  // X[:,c] for c: x_c = 1/L_cc; x_i = -(sum_{t=c}^{i-1} L_it x_t)/L_ii
+  __syncthreads();
+  double* X = W;   // reuse
+  for (int c = tid; c < l; c += blockDim.x) {
+    for (int i = 0; i < l; ++i) X[i * l + c] = 0.0;
+    if (!bad) {
+      X[c * l + c] = 1.0 / Lm[c * l + c];
+      for (int i = c + 1; i < l; ++i) {
+        double t = 0.0;
+        for (int k2 = c; k2 < i; ++k2) t += Lm[i * l + k2] * X[k2 * l + c];
+        X[i * l + c] = -t / Lm[i * l + i];
+      }
+    } else {
+      X[c * l + c] = 0.0;   // total failure: zero basis, flagged above
+    }
+  }
+  __syncthreads();
+  // Rinv = Linv^T (upper triangular)
+  float* out = Rinv + (long long)bz * l * l;
+  for (int e = tid; e < l * l; e += blockDim.x) {
+    const int i = e / l, j = e % l;
+    out[e] = (float)X[j * l + i];
+  }
+}
+
+cudaError_t chol_inv_launch(const double* partial, int nchunk, int batch, int l, float* Rinv, int* status,
+                            cudaStream_t st, long long* launches) {
+  const size_t smem = 2 * (size_t)l * l * sizeof(double);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * MAX_L * MAX_L * 8);
+    attr_set = true;
+  }
+  chol_inv_kernel<<<batch, 256, smem, st>>>(partial, nchunk, l, Rinv, status);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Out[b, rows, kout] = In[b, rows, l] * Mtx[b, l(, ldm)] (first kout columns of Mtx). In-place safe.
+// ---------------------------------------------------------------------------------------------
+constexpr int PA_ROWS = 64;
+__global__ void __launch_bounds__(256) panel_apply_kernel(const float* In, long long in_bs, int ld_in,
+                                                          const float* __restrict__ Mtx, int ldm, int rows, int l,
+                                                          int kout, float* Out, long long out_bs, int ld_out) {
+  __shared__ float tile[PA_ROWS][MAX_L + 1];
+  __shared__ float mt[MAX_L][MAX_L + 1];
+  const int bz = blockIdx.y, tid = threadIdx.x;
+  const int r0 = blockIdx.x * PA_ROWS;
+  const float* Ib = In + (long long)bz * in_bs;
+  const float* Mb = Mtx + (long long)bz * l * ldm;
+  for (int e = tid; e < l * kout; e += 256) mt[e / kout][e % kout] = Mb[(e / kout) * ldm + (e % kout)];
+  for (int e = tid; e < PA_ROWS * l; e += 256) {
+    const int rr = e / l, c = e % l;
+    tile[rr][c] = (r0 + rr < rows) ? Ib[(long long)(r0 + rr) * ld_in + c] : 0.f;
+  }
+  __syncthreads();
+  float* Ob = Out + (long long)bz * out_bs;
+  for (int e = tid; e < PA_ROWS * kout; e += 256) {
+    const int rr = e / kout, c = e % kout;
+    if (r0 + rr >= rows) continue;
+    float t = 0.f;
+    for (int q = 0; q < l; ++q) t = fmaf(tile[rr][q], mt[q][c], t);
+    Ob[(long long)(r0 + rr) * ld_out + c] = t;
+  }
+}
+
+cudaError_t panel_apply_launch(const float* In, long long in_bs, int ld_in, const float* Mtx, int ldm, int batch,
+                               int rows, int l, int kout, float* Out, long long out_bs, int ld_out, cudaStream_t st,
+                               long long* launches) {
+  if (kout <= 0) return cudaSuccess;
+  panel_apply_kernel<<<dim3((rows + PA_ROWS - 1) / PA_ROWS, batch), 256, 0, st>>>(In, in_bs, ld_in, Mtx, ldm, rows, l,
+                                                                                 kout, Out, out_bs, ld_out);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// One-sided Jacobi eigensolver of the symmetric positive semidefinite core C = sum of partials
+// (l x l). Columns of A = C V are rotated pairwise until mutually orthogonal; then ||a_j|| are the
+// eigenvalues and V the eigenvectors. One warp per column pair (round-robin pairing), lanes over
+// rows, dot products by warp shuffles; fp64 throughout. Outputs (sorted by decreasing eigenvalue):
+//   s[b, l]     = sqrt(eigenvalue)             (singular values of the panel whose Gram this is)
+//   E[b, l, l]  = eigenvectors in columns      (fp32)
+//   Es[b, l, l] = E diag(1/s)                  (fp32; zero column where s is numerically zero)
+// With `signed_input` the matrix is a general symmetric one (Rayleigh quotient of Algorithm 2):
+// eigenvalues keep their sign (lambda_j = v_j^T a_j), sorted by decreasing magnitude, s = lambda.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__global__ void __launch_bounds__(1024) jacobi_eig_kernel(const double* __restrict__ partial, int nchunk, int l,
+                                                          int signed_input, float* __restrict__ s_out,
+                                                          float* __restrict__ E, float* __restrict__ Es,
+                                                          int* __restrict__ status, int max_sweeps) {
+  extern __shared__ double sm[];
+  double* A = sm;             // column-major: A[c * l + r]
+  double* V = sm + l * l;     // column-major
+  __shared__ double lam[MAX_L];
+  __shared__ int order[MAX_L];
+  __shared__ int rotated;
+  const int bz = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const double* pb = partial + (long long)bz * nchunk * l * l;
+  for (int e = tid; e < l * l; e += blockDim.x) {
+    const int r = e / l, c = e % l;
+    double t = 0.0, u = 0.0;
+    for (int ch = 0; ch < nchunk; ++ch) {
+      t += pb[(long long)ch * l * l + r * l + c];
+      u += pb[(long long)ch * l * l + c * l + r];
+    }
+    A[c * l + r] = 0.5 * (t + u);
+    V[c * l + r] = (r == c) ? 1.0 : 0.0;
+  }
+  __syncthreads();
+  const int np = (l + 1) & ~1;        // players, padded to even
+  const int npairs = np / 2;
+  int sweep = 0;
+  for (; sweep < max_sweeps; ++sweep) {
+    if (tid == 0) rotated = 0;
+    __syncthreads();
+    for (int round = 0; round < np - 1; ++round) {
+      if (warp < npairs) {
+        int p, q;
+        if (warp == 0) { p = np - 1; q = round; }
+        else { p = (round + warp) % (np - 1); q = (round - warp + (np - 1)) % (np - 1); }
+        if (p > q) { const int t = p; p = q; q = t; }
+        if (q < l) {
+          double* ap = A + p * l; double* aq = A + q * l;
+          const double x0 = (lane < l) ? ap[lane] : 0.0, x1 = (lane + 32 < l) ? ap[lane + 32] : 0.0;
+          const double y0 = (lane < l) ? aq[lane] : 0.0, y1 = (lane + 32 < l) ? aq[lane + 32] : 0.0;
+          const double alpha = warp_sum(x0 * x0 + x1 * x1);
+          const double beta = warp_sum(y0 * y0 + y1 * y1);
+          const double gamma = warp_sum(x0 * y0 + x1 * y1);
+          if (gamma != 0.0 && fabs(gamma) > 1e-14 * sqrt(alpha * beta)) {
+            if (lane == 0) rotated = 1;
+            const double zeta = (beta - alpha) / (2.0 * gamma);
+            const double t = ((zeta >= 0.0) ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
+            const double c = 1.0 / sqrt(1.0 + t * t), sn = c * t;
+            if (lane < l) { ap[lane] = c * x0 - sn * y0; aq[lane] = sn * x0 + c * y0; }
+            if (lane + 32 < l) { ap[lane + 32] = c * x1 - sn * y1; aq[lane + 32] = sn * x1 + c * y1; }
+            double* vp = V + p * l; double* vq = V + q * l;
+            if (lane < l) { const double a = vp[lane], b = vq[lane]; vp[lane] = c * a - sn * b; vq[lane] = sn * a + c * b; }
+            if (lane + 32 < l) {
+              const double a = vp[lane + 32], b = vq[lane + 32];
+              vp[lane + 32] = c * a - sn * b; vq[lane + 32] = sn * a + c * b;
+            }
+          }
+        }
+      }
+      __syncthreads();
+    }
+    if (!rotated) break;
+    __syncthreads();
+  }
+  if (tid == 0 && sweep >= max_sweeps && status) atomicOr(&status[bz], 2);
+  // eigenvalues
+  if (warp < 32) {
+    for (int j = warp; j < l; j += (blockDim.x >> 5)) {
+      const double* aj = A + j * l; const double* vj = V + j * l;
+      const double a0 = (lane < l) ? aj[lane] : 0.0, a1 = (lane + 32 < l) ? aj[lane + 32] : 0.0;
+      const double v0 = (lane < l) ? vj[lane] : 0.0, v1 = (lane + 32 < l) ? vj[lane + 32] : 0.0;
+      const double nrm = sqrt(warp_sum(a0 * a0 + a1 * a1));
+      const double rq = warp_sum(a0 * v0 + a1 * v1);
+      if (lane == 0) lam[j] = signed_input ? ((rq >= 0.0) ? nrm : -nrm) : nrm;
+    }
+  }
+  __syncthreads();
+  if (tid < l) {
+    const double mine = fabs(lam[tid]);
+    int rank = 0;
+    for (int i = 0; i < l; ++i) {
+      const double o = fabs(lam[i]);
+      if (o > mine || (o == mine && i < tid)) ++rank;
+    }
+    order[rank] = tid;
+  }
+  __syncthreads();
+  for (int e = tid; e < l * l; e += blockDim.x) {
+    const int r = e / l, cc = e % l;
+    const int src = order[cc];
+    const double v = V[src * l + r];
+    const double lm = lam[src];
+    const double sv = signed_input ? lm : sqrt(lm > 0.0 ? lm : 0.0);
+    if (E) E[(long long)bz * l * l + e] = (float)v;
+    if (Es) Es[(long long)bz * l * l + e] = (fabs(sv) > 1e-300) ? (float)(v / sv) : 0.f;
+    if (r == 0 && s_out) s_out[(long long)bz * l + cc] = (float)sv;
+  }
+}
+
+cudaError_t jacobi_eig_launch(const double* partial, int nchunk, int batch, int l, int signed_input, float* s_out,
+                              float* E, float* Es, int* status, cudaStream_t st, long long* launches) {
+  const size_t smem = 2 * (size_t)l * l * sizeof(double);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaFuncSetAttribute(jacobi_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * MAX_L * MAX_L * 8);
+    attr_set = true;
+  }
+  jacobi_eig_kernel<<<batch, 1024, smem, st>>>(partial, nchunk, l, signed_input, s_out, E, Es, status, 40);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Frobenius partial sums of a [b, count] array (bf16 or fp32): partial[b, nblk] in fp64.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) frob_partial_kernel(const void* __restrict__ X, int dtype, long long count,
+                                                           int nblk, double* __restrict__ partial) {
+  __shared__ double red[8];
+  const int bz = blockIdx.y, tid = threadIdx.x;
+  const long long per = (count + nblk - 1) / nblk;
+  const long long lo = (long long)blockIdx.x * per, hi = min(count, lo + per);
+  const long long base = (long long)bz * count;
+  double acc = 0.0;
+  float f = 0.f;
+  int n = 0;
+  for (long long i = lo + tid; i < hi; i += 256) {
+    const float v = ld_as_float(X, base + i, dtype);
+    f = fmaf(v, v, f);
+    if (++n == 16) { acc += (double)f; f = 0.f; n = 0; }
+  }
+  acc += (double)f;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, o);
+  if ((tid & 31) == 0) red[tid >> 5] = acc;
+  __syncthreads();
+  if (tid == 0) {
+    double t = 0.0;
+    for (int w = 0; w < 8; ++w) t += red[w];
+    partial[(long long)bz * nblk + blockIdx.x] = t;
+  }
+}
+
+cudaError_t frob_partial_launch(const void* X, int dtype, int batch, long long count, int nblk, double* partial,
+                                cudaStream_t st, long long* launches) {
+  frob_partial_kernel<<<dim3(nblk, batch), 256, 0, st>>>(X, dtype, count, nblk, partial);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+// rho[b] = sqrt(sum of partials in index order); inv_rho[b] = 1/rho (0 and status bit 4 when rho is 0 or not finite)
+__global__ void rho_finalize_kernel(const double* __restrict__ partial, int nper, int batch, float* __restrict__ rho,
+                                    float* __restrict__ inv_rho, float* __restrict__ inv_rho2,
+                                    int* __restrict__ status) {
+  const int bz = blockIdx.x * blockDim.x + threadIdx.x;
+  if (bz >= batch) return;
+  double t = 0.0;
+  for (int i = 0; i < nper; ++i) t += partial[(long long)bz * nper + i];
+  const double r = sqrt(t);
+  const bool ok = (r > 0.0) && isfinite(r);
+  if (rho) rho[bz] = (float)r;
+  if (inv_rho) inv_rho[bz] = ok ? (float)(1.0 / r) : 0.f;
+  if (inv_rho2) inv_rho2[bz] = ok ? (float)(1.0 / t) : 0.f;
+  if (!ok && status) atomicOr(&status[bz], 4);
+}
+
+cudaError_t rho_finalize_launch(const double* partial, int nper, int batch, float* rho, float* inv_rho,
+                                float* inv_rho2, int* status, cudaStream_t st, long long* launches) {
+  rho_finalize_kernel<<<(batch + 127) / 128, 128, 0, st>>>(partial, nper, batch, rho, inv_rho, inv_rho2, status);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+// Out[b, rows, k] = In[b, rows, (ld_in)] * diag(coef): coef_t = c0 * s[b,t] * (use_inv ? inv_rho[b] : 1) + c1
+__global__ void scale_cols_kernel(const float* __restrict__ In, long long in_bs, int ld_in, int rows, int k,
+                                  const float* __restrict__ s, int ld_s, const float* __restrict__ inv_rho, float c0,
+                                  float c1, float* __restrict__ Out, long long out_bs, int ld_out) {
+  const int bz = blockIdx.y;
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= (long long)rows * k) return;
+  const int r = (int)(e / k), t = (int)(e % k);
+  const float sc = c0 * s[(long long)bz * ld_s + t] * (inv_rho ? inv_rho[bz] : 1.f) + c1;
+  Out[(long long)bz * out_bs + (long long)r * ld_out + t] = In[(long long)bz * in_bs + (long long)r * ld_in + t] * sc;
+}
+
+cudaError_t scale_cols_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int k, const float* s,
+                              int ld_s, const float* inv_rho, float c0, float c1, float* Out, long long out_bs,
+                              int ld_out, cudaStream_t st, long long* launches) {
+  if (k <= 0) return cudaSuccess;
+  const long long tot = (long long)rows * k;
+  scale_cols_kernel<<<dim3((unsigned)((tot + 255) / 256), batch), 256, 0, st>>>(In, in_bs, ld_in, rows, k, s, ld_s,
+                                                                               inv_rho, c0, c1, Out, out_bs, ld_out);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+// Out[b, i] = scale[b] * In[b, i]  (type conversion allowed)
+__global__ void scale_kernel(const void* __restrict__ In, int in_dt, void* __restrict__ Out, int out_dt,
+                             long long count, const float* __restrict__ scale) {
+  const int bz = blockIdx.y;
+  const float sc = scale ? scale[bz] : 1.f;
+  const long long base = (long long)bz * count;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (long long)gridDim.x * blockDim.x)
+    st_from_float(Out, base + i, out_dt, sc * ld_as_float(In, base + i, in_dt));
+}
+
+cudaError_t scale_launch(const void* In, int in_dt, void* Out, int out_dt, int batch, long long count,
+                         const float* scale, cudaStream_t st, long long* launches) {
+  const int nblk = (int)min((long long)1184, (count + 255) / 256);
+  scale_kernel<<<dim3(nblk, batch), 256, 0, st>>>(In, in_dt, Out, out_dt, count, scale);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Counter-based Gaussian fill (the generator documented in the public header).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned long long mix64(unsigned long long x) {
+  x += 0x9E3779B97F4A7C15ull;
+  x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+  x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+  return x ^ (x >> 31);
+}
+
+__global__ void fill_gaussian_kernel(void* __restrict__ dst, long long count, int dtype, unsigned long long seed,
+                                     long long per_stream, unsigned long long seed_stride) {
+  // element e belongs to stream e / per_stream (seed + stream * seed_stride), index e % per_stream
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < count;
+       e += (long long)gridDim.x * blockDim.x) {
+    const unsigned long long stream = per_stream > 0 ? (unsigned long long)(e / per_stream) : 0ull;
+    const unsigned long long idx = per_stream > 0 ? (unsigned long long)(e % per_stream) : (unsigned long long)e;
+    const unsigned long long hs = mix64(seed + stream * seed_stride);
+    const unsigned long long j = idx >> 1;
+    const unsigned long long r1 = mix64(hs ^ (2ull * j)), r2 = mix64(hs ^ (2ull * j + 1ull));
+    const double u1 = ((double)(r1 >> 11) + 1.0) * (1.0 / 9007199254740992.0);
+    const double u2 = (double)(r2 >> 11) * (1.0 / 9007199254740992.0);
+    const double rad = sqrt(-2.0 * log(u1));
+    double sn, cs;
+    sincos(6.283185307179586476925286766559 * u2, &sn, &cs);
+    st_from_float(dst, e, dtype, (float)((idx & 1ull) ? rad * sn : rad * cs));
+  }
+}
+
+cudaError_t fill_gaussian_launch(void* dst, long long count, int dtype, unsigned long long seed, long long per_stream,
+                                 unsigned long long seed_stride, cudaStream_t st, long long* launches) {
+  if (count <= 0) return cudaSuccess;
+  const int nblk = (int)min((long long)2368, (count + 255) / 256);
+  fill_gaussian_kernel<<<nblk, 256, 0, st>>>(dst, count, dtype, seed, per_stream, seed_stride);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+__global__ void fill_int_kernel(int* p, int n, int v) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) p[i] = v;
+}
+cudaError_t fill_int_launch(int* p, int n, int v, cudaStream_t st, long long* launches) {
+  if (n <= 0) return cudaSuccess;
+  fill_int_kernel<<<(n + 255) / 256, 256, 0, st>>>(p, n, v);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace defl
+
+namespace defl {
+__global__ void or_status_kernel(int* status, int n, const int* word) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) status[i] |= *word;
+}
+cudaError_t or_status_launch(int* status, int n, const int* word, cudaStream_t st, long long* launches) {
+  if (n <= 0) return cudaSuccess;
+  or_status_kernel<<<(n + 255) / 256, 256, 0, st>>>(status, n, word);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+}  // namespace defl

@@ -1,0 +1,32 @@
+// Launchers of the small-panel kernels (see panel.cu). None of them synchronises.
+#pragma once
+#include <cuda_runtime.h>
+
+namespace defl {
+
+constexpr int MAX_L = 64;   // widest panel (sketch width / PSD basis width)
+
+int gram_num_chunks(int rows);
+cudaError_t gram_partial_launch(const float* Y, long long batch_stride, int batch, int rows, int l, int ld,
+                                double* partial, cudaStream_t st, long long* launches);
+cudaError_t chol_inv_launch(const double* partial, int nchunk, int batch, int l, float* Rinv, int* status,
+                            cudaStream_t st, long long* launches);
+cudaError_t panel_apply_launch(const float* In, long long in_bs, int ld_in, const float* Mtx, int ldm, int batch,
+                               int rows, int l, int kout, float* Out, long long out_bs, int ld_out, cudaStream_t st,
+                               long long* launches);
+cudaError_t jacobi_eig_launch(const double* partial, int nchunk, int batch, int l, int signed_input, float* s_out,
+                              float* E, float* Es, int* status, cudaStream_t st, long long* launches);
+cudaError_t frob_partial_launch(const void* X, int dtype, int batch, long long count, int nblk, double* partial,
+                                cudaStream_t st, long long* launches);
+cudaError_t rho_finalize_launch(const double* partial, int nper, int batch, float* rho, float* inv_rho,
+                                float* inv_rho2, int* status, cudaStream_t st, long long* launches);
+cudaError_t scale_cols_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int k, const float* s,
+                              int ld_s, const float* inv_rho, float c0, float c1, float* Out, long long out_bs,
+                              int ld_out, cudaStream_t st, long long* launches);
+cudaError_t scale_launch(const void* In, int in_dt, void* Out, int out_dt, int batch, long long count,
+                         const float* scale, cudaStream_t st, long long* launches);
+cudaError_t fill_gaussian_launch(void* dst, long long count, int dtype, unsigned long long seed, long long per_stream,
+                                 unsigned long long seed_stride, cudaStream_t st, long long* launches);
+cudaError_t fill_int_launch(int* p, int n, int v, cudaStream_t st, long long* launches);
+
+}  // namespace defl

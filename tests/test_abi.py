@@ -1,0 +1,54 @@
+"""The C-ABI library builds, loads without a GPU, and exports every function include/defl.h declares."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def libpath():
+    from paper_2609_21102_b200 import build
+    return build.build()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "defl.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(defl_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_declares_the_two_primitives():
+    names = _declared()
+    assert "defl_polar_batched" in names and "defl_psd_project" in names
+    assert len(names) >= 10
+
+
+def test_library_exports_every_declared_symbol(libpath):
+    L = ctypes.CDLL(libpath)
+    for name in _declared():
+        assert hasattr(L, name), name
+
+
+def test_binding_lists_the_same_names(libpath):
+    from paper_2609_21102_b200 import binding
+    assert sorted(binding.EXPORTS) == _declared()
+    binding.lib()
+
+
+def test_status_strings_and_no_device_behaviour(libpath):
+    import torch
+    L = ctypes.CDLL(libpath)
+    L.defl_status_string.restype = ctypes.c_char_p
+    for code in (0, -1, -2, -3, -4):
+        assert len(L.defl_status_string(code)) > 0
+    assert L.defl_polar_workspace_bytes(0, 4, 4, 0, 0, 0) == 0
+    L.defl_polar_workspace_bytes.restype = ctypes.c_size_t
+    assert L.defl_polar_workspace_bytes(2, 128, 256, 0, 4, 4) > 2 * 128 * 256 * 2
+    if not torch.cuda.is_available():
+        h = ctypes.c_void_p()
+        # no CPU fallback: without a device the context cannot even be created
+        assert L.defl_create(ctypes.byref(h), 0) == -3
+        assert not h.value

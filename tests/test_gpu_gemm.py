@@ -1,0 +1,88 @@
+"""The two product engines against a plain PyTorch fp32 product of the same (rounded) inputs."""
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2609_21102_b200 import binding
+    c = binding.Context(0)
+    yield c
+    c.close()
+
+
+def _ref(A, B, ta, tb, alpha=1.0):
+    a = A.float().transpose(1, 2) if ta else A.float()
+    b = B.float().transpose(1, 2) if tb else B.float()
+    return alpha * torch.matmul(a.double(), b.double()).float()
+
+
+def _mk(b, r, c, dtype, seed):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    return torch.randn((b, r, c), generator=g, device="cuda", dtype=torch.float32).to(dtype)
+
+
+SHAPES = [(1, 128, 128, 64), (2, 200, 136, 96), (3, 256, 264, 200), (1, 72, 48, 40), (2, 384, 160, 320)]
+
+
+@pytest.mark.parametrize("b,M,N,K", SHAPES)
+@pytest.mark.parametrize("ta,tb", [(False, True), (False, False), (True, False), (True, True)])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_simt_engine(ctx, b, M, N, K, ta, tb, dtype):
+    from paper_2609_21102_b200 import binding
+    A = _mk(b, K if ta else M, M if ta else K, dtype, 1)
+    B = _mk(b, N if tb else K, K if tb else N, dtype, 2)
+    C = ctx.defl_debug_gemm(A, B, ta, tb, engine=binding.ENGINE_SIMT, out_dtype=torch.float32, alpha=0.5)
+    ref = _ref(A, B, ta, tb, 0.5)
+    assert torch.allclose(C, ref, rtol=1e-4, atol=1e-3)
+
+
+@pytest.mark.parametrize("b,M,N,K", SHAPES)
+@pytest.mark.parametrize("ta,tb", [(False, True), (False, False), (True, False), (True, True)])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_tensor_engine(ctx, b, M, N, K, ta, tb, dtype):
+    from paper_2609_21102_b200 import binding
+    A = _mk(b, K if ta else M, M if ta else K, dtype, 3)
+    B = _mk(b, N if tb else K, K if tb else N, dtype, 4)
+    if dtype == torch.float32 and (ta or not tb):
+        # tf32 tiles are K-major only: the engine must refuse, not compute something else
+        with pytest.raises(binding.DeflError) as e:
+            ctx.defl_debug_gemm(A, B, ta, tb, engine=binding.ENGINE_TENSOR, out_dtype=torch.float32)
+        assert e.value.code == -4
+        return
+    C = ctx.defl_debug_gemm(A, B, ta, tb, engine=binding.ENGINE_TENSOR, out_dtype=torch.float32)
+    torch.cuda.synchronize()
+    ref = _ref(A, B, ta, tb)
+    if dtype == torch.bfloat16:      # exact products of bf16 values, fp32 accumulation
+        assert torch.allclose(C, ref, rtol=1e-4, atol=2e-3)
+    else:                            # tf32 operands: 10-bit mantissas
+        err = (C - ref).norm() / ref.norm()
+        assert err < 2e-3, float(err)
+
+
+def test_tensor_engine_bf16_output_and_large_tiles(ctx):
+    from paper_2609_21102_b200 import binding
+    A = _mk(2, 520, 1600, torch.bfloat16, 5)     # X X^T with a ragged 1600 = 12.5 tiles of 128
+    C = ctx.defl_debug_gemm(A, A, False, True, engine=binding.ENGINE_TENSOR, out_dtype=torch.bfloat16)
+    ref = _ref(A, A, False, True)
+    err = (C.float() - ref).norm() / ref.norm()
+    assert err < 4e-3, float(err)
+    B = _mk(2, 1600, 1608, torch.bfloat16, 6)    # MN-major right operand, N = 1608 ragged
+    A2 = _mk(2, 264, 1600, torch.bfloat16, 7)
+    C2 = ctx.defl_debug_gemm(A2, B, False, False, engine=binding.ENGINE_TENSOR, out_dtype=torch.bfloat16)
+    ref2 = _ref(A2, B, False, False)
+    err2 = (C2.float() - ref2).norm() / ref2.norm()
+    assert err2 < 4e-3, float(err2)
+
+
+@pytest.mark.parametrize("engine_name", ["simt", "tensor"])
+def test_symmetric_mirroring(ctx, engine_name):
+    from paper_2609_21102_b200 import binding
+    engine = binding.ENGINE_SIMT if engine_name == "simt" else binding.ENGINE_TENSOR
+    A = _mk(2, 456, 320, torch.bfloat16, 8)
+    C = ctx.defl_debug_gemm(A, A, False, True, engine=engine, out_dtype=torch.float32, exploit_symmetry=True)
+    ref = _ref(A, A, False, True)
+    assert torch.allclose(C, ref, rtol=1e-4, atol=2e-3)
+    assert torch.equal(C, C.transpose(1, 2))

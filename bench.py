@@ -1,0 +1,295 @@
+#!/usr/bin/env python
+"""Benchmark of the deflated polar filter on synthetic GPT-2-XL-shaped Muon batches.
+
+One step = one pass of the whole hot path (batched randomized SVD, deflate + normalise, five quintic
+Newton-Schulz steps, restore) over one batch: 48 matrices 1600x6400 and 48 matrices 1600x1600 in
+bf16 with the heavy-tailed spectrum sigma_i = max(200/i, 1e-4), k=32, oversampling 16, 2 subspace
+iterations. Prints ONE JSON line (see README / DESIGN for the keys).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--small]
+
+N > 1 is launched under torchrun; every rank runs the same batch on its own GPU (independent
+matrices, no data-path collective) and the line reports the whole-job aggregate.
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "deflated polar-filter TFLOP/s & matrices/s per batch; % bf16 tensor peak"
+MUON = (3.4445, -4.7750, 2.0315)
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+WORKLOADS = {
+    # name: (list of (b, m, n), k, p, J, L)
+    "gpt2_xl": {"groups": [(48, 1600, 6400), (48, 1600, 1600)], "k": 32, "p": 16, "J": 2, "L": 5,
+                "label": "GPT-2-XL Muon shapes, bf16: 48 x 1600x6400 + 48 x 1600x1600, sigma_i=max(200/i,1e-4), "
+                         "k=32, p=16, J=2, 5 Muon quintic steps"},
+    "small": {"groups": [(4, 256, 1024), (4, 256, 256)], "k": 8, "p": 8, "J": 1, "L": 5,
+              "label": "small check: 4 x 256x1024 + 4 x 256x256"},
+}
+
+
+def flops_per_matrix(m, n, k, p, J, L):
+    """Algorithmic flops of one matrix: dense filter count, rSVD products, subtract and restore."""
+    ms, ml = min(m, n), max(m, n)
+    l = min(ms, k + p) if k > 0 else 0
+    filt = L * (4.0 * ms * ms * ml + 2.0 * ms ** 3)
+    rsvd = 2.0 * ml * ms * l * (2 + 2 * J) if k > 0 else 0.0
+    defl = 2.0 * 2.0 * m * n * k          # residual norm pass + X0 pass
+    return filt, rsvd + defl
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    def __init__(self, index):
+        self.index, self.rows, self._stop, self._t = index, [], threading.Event(), None
+
+    def _run(self):
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + q,
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
+                parts = [x.strip() for x in out.strip().split(",")]
+                if len(parts) >= 6:
+                    self.rows.append(parts)
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self._t = threading.Thread(target=self._run, daemon=True)
+        self._t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._t.join(timeout=6)
+
+    def summary(self):
+        if not self.rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        sm = sorted(float(r[0]) for r in self.rows if r[0].replace(".", "").isdigit())
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [nm for i, nm in enumerate(names) if any(r[2 + i].lower().startswith("active") for r in self.rows)]
+        mx = [float(r[1]) for r in self.rows if r[1].replace(".", "").isdigit()]
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(self.rows)}
+
+
+def make_inputs(wl, device):
+    import torch
+    from paper_2609_21102_b200 import inputs
+    groups = []
+    for si, (b, m, n) in enumerate(wl["groups"]):
+        G = inputs.workload_power_law(b, m, n, 4, si, 1.0, 200.0, 1e-4, device=device).to(torch.bfloat16)
+        l = min(min(m, n), wl["k"] + wl["p"])
+        Om = inputs.sketch(b, min(m, n), l, 4, si, device=device)
+        groups.append({"G": G, "Om": Om, "out": torch.empty_like(G)})
+    return groups
+
+
+def run_step(ctx, wl, groups):
+    for g in groups:
+        ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"], sketch=g["Om"],
+                               gamma=1.01)
+
+
+def oracle_sample(wl, seconds_hint=20.0):
+    """Times the fp64 oracle on one matrix of the smallest group (a bounded sample of the workload)."""
+    import numpy as np
+    import oracle
+    from paper_2609_21102_b200 import inputs
+    import torch
+    b, m, n = min(wl["groups"], key=lambda g: g[1] * g[2])
+    si = wl["groups"].index((b, m, n))
+    G = inputs.workload_power_law(1, m, n, 4, si, 1.0, 200.0, 1e-4).to(torch.bfloat16).double().numpy()[0]
+    l = min(min(m, n), wl["k"] + wl["p"])
+    Om = inputs.sketch(1, min(m, n), l, 4, si).double().numpy()[0]
+    t0 = time.perf_counter()
+    oracle.deflated_polar(G, wl["k"], l, Om, wl["J"], oracle.schedule(MUON, wl["L"]), gamma=1.01)
+    dt = time.perf_counter() - t0
+    filt, rest = flops_per_matrix(m, n, wl["k"], wl["p"], wl["J"], wl["L"])
+    return dt, (filt + rest), "1 matrix %dx%d of the batch, full path, fp64" % (m, n)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--small", action="store_true", help="tiny workload for a quick functional check")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl_name = "small" if args.small else "gpt2_xl"
+    wl = WORKLOADS[wl_name]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    config = {"workload": wl["label"], "name": wl_name, "k": wl["k"], "oversample": wl["p"], "power_iters": wl["J"],
+              "filter_steps": wl["L"], "restore": "padded, gamma=1.01",
+              "l2": "inputs (1.2 GB per step) larger than L2; no flush"}
+    tot_f = sum(b * sum(flops_per_matrix(m, n, wl["k"], wl["p"], wl["J"], wl["L"])) for b, m, n in wl["groups"])
+    nmat = sum(b for b, _, _ in wl["groups"])
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        cores = os.cpu_count() or 1
+        times = []
+        for _ in range(max(1, min(args.steps, 3))):
+            dt, fl, sample = oracle_sample(wl)
+            times.append(dt)
+        dt = sum(times) / len(times)
+        val = fl / dt / 1e12
+        line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+                "steps": len(times), "warmup": 0, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
+                "matrices_per_s": 1.0 / dt,
+                "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+                "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return
+
+    import torch
+    from paper_2609_21102_b200 import binding
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    ctx = binding.Context(local_rank)
+    groups = make_inputs(wl, torch.device("cuda", local_rank))
+    ctx.defl_set_profiling(True)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        run_step(ctx, wl, groups)
+    barrier()
+    launches0 = ctx.defl_launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    stage_ms = []
+    with ClockSampler(local_rank) as clk:
+        barrier()
+        ev[0].record()
+        for i in range(args.steps):
+            for g in groups:
+                ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"],
+                                       sketch=g["Om"], gamma=1.01)
+                stage_ms.append(None)      # filled after the timed region (events are already recorded)
+            ev[i + 1].record()
+        barrier()
+    launches = ctx.defl_launch_count() - launches0
+    total_ms = ev[0].elapsed_time(ev[-1])
+    if dist is not None:
+        t = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+
+    # stage split of one more (untimed) step, with the same events the library records on its stream
+    stage_tot = [0.0, 0.0, 0.0, 0.0]
+    filt_flops = 0.0
+    for g, (b, m, n) in zip(groups, wl["groups"]):
+        ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"], sketch=g["Om"],
+                               gamma=1.01)
+        ms = ctx.defl_get_stage_ms()
+        for i in range(min(4, len(ms))):
+            stage_tot[i] += ms[i]
+        filt_flops += b * flops_per_matrix(m, n, wl["k"], wl["p"], wl["J"], wl["L"])[0]
+    plain_ms = 0.0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for g in groups:
+        ctx.defl_polar_batched(g["G"], 0, 0, 0, [list(MUON)] * wl["L"], out=g["out"])
+    e1.record()
+    torch.cuda.synchronize()
+    plain_ms = e0.elapsed_time(e1)
+
+    # end to end through the host-buffer entry point (pinned host tensors, copies inside the timed region)
+    e2e = None
+    if rank == 0 or world > 1:
+        hG = [g["G"].cpu().pin_memory() for g in groups]
+        hO = [torch.empty_like(h).pin_memory() for h in hG]
+        def e2e_step():
+            for h, o, g in zip(hG, hO, groups):
+                ctx.defl_polar_batched_host(h, o, wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], sketch=g["Om"], gamma=1.01)
+        e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        n_e2e = max(1, min(args.steps, 3))
+        for _ in range(n_e2e):
+            e2e_step()
+        torch.cuda.synchronize()
+        e2e_ms = (time.perf_counter() - t0) * 1e3 / n_e2e
+        if dist is not None:
+            t = torch.tensor([e2e_ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        nbytes = sum(h.numel() * h.element_size() for h in hG)
+        e2e = {"value": world * tot_f / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    peaks, peaks_kind = load_peaks()
+    value = world * tot_f / (ms_per_step * 1e-3) / 1e12
+    filt_ms = stage_tot[2]
+    n_filter_launches = 3 * wl["L"] * len(groups)
+    ach = filt_flops / (filt_ms * 1e-3) / 1e12 if filt_ms > 0 else None
+    peak = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
+    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel (filter chain: X X^T, A^2 polynomial, B X)",
+                "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": (ach / peak) if ach else None,
+                "peak_kind": "bf16_tflops_sustained, of %s" % peaks_kind,
+                "frac_of_burst": (ach / float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))) if ach else None,
+                "launches_per_step": n_filter_launches, "avg_launch_ms": filt_ms / n_filter_launches,
+                "flops_per_launch_avg": filt_flops / n_filter_launches, "traffic": None}
+    line = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
+            "matrices_per_s": world * nmat / (ms_per_step * 1e-3),
+            "pct_bf16_peak_sustained": 100.0 * value / world / peak,
+            "stage_ms": {"rsvd": stage_tot[0], "deflate_normalise": stage_tot[1], "filter": stage_tot[2],
+                         "restore": stage_tot[3]},
+            "deflation_overhead_frac": (ms_per_step - plain_ms) / ms_per_step if ms_per_step > 0 else None,
+            "plain_filter_ms": plain_ms,
+            "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clk.summary()}
+    if not args.no_cpu_baseline:
+        dt, fl, sample = oracle_sample(wl)
+        line["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count() or 1,
+                                "kind": "oracle", "sample": sample, "seconds": dt, "matrices_per_s": 1.0 / dt}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

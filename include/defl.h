@@ -113,6 +113,14 @@ int defl_polar_batched(defl_ctx* ctx, const void* G, void* out, int b, int m, in
                        const float* coeff_schedule, int L,
                        const defl_opts* opts, const defl_info* info);
 
+/* The same call for HOST buffers: G_host and out_host are host memory (pinned memory makes the copies
+ * asynchronous and fast). The library copies G to device staging memory it owns, runs defl_polar_batched,
+ * copies the result back and synchronises the stream before returning, so out_host is ready on return.
+ * opts->sketch, if given, is still device memory. Same errors as defl_polar_batched. */
+int defl_polar_batched_host(defl_ctx* ctx, const void* G_host, void* out_host, int b, int m, int n, int dtype,
+                            int k, int oversample, int power_iters,
+                            const float* coeff_schedule, int L, const defl_opts* opts);
+
 /* Batched randomized SVD alone (Algorithm 3) in the caller's orientation:
  *   G ~ P diag(s) W^T with P [b,m,l], s [b,l] descending, W [b,n,l], all fp32; l = min(min(m,n), k+oversample).
  * Any of P, s, W may be NULL. The sketch comes from opts as above. */

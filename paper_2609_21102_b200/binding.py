@@ -25,7 +25,7 @@ CLASSICAL_QUINTIC = (1.875, -1.25, 0.375)
 
 EXPORTS = [
     "defl_create", "defl_destroy", "defl_set_stream", "defl_polar_workspace_bytes", "defl_psd_workspace_bytes",
-    "defl_polar_batched", "defl_brsvd_batched", "defl_psd_project", "defl_fill_gaussian", "defl_debug_gemm",
+    "defl_polar_batched", "defl_polar_batched_host", "defl_brsvd_batched", "defl_psd_project", "defl_fill_gaussian", "defl_debug_gemm",
     "defl_set_profiling", "defl_get_stage_ms", "defl_launch_count", "defl_status_string", "defl_last_error",
 ]
 
@@ -57,6 +57,8 @@ def lib():
         L.defl_psd_workspace_bytes.argtypes = [ctypes.c_int] * 2
         L.defl_polar_batched.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 7 + [
             ctypes.POINTER(ctypes.c_float), ctypes.c_int, ctypes.POINTER(DeflOpts), ctypes.POINTER(DeflInfo)]
+        L.defl_polar_batched_host.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 7 + [
+            ctypes.POINTER(ctypes.c_float), ctypes.c_int, ctypes.POINTER(DeflOpts)]
         L.defl_brsvd_batched.argtypes = [ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 7 + [
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(DeflOpts), ctypes.c_void_p]
         L.defl_psd_project.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
@@ -188,6 +190,23 @@ class Context:
                                       sched, L, ctypes.byref(opts), ctypes.byref(info))
         self._check(rc)
         return (out, extras) if want_info else out
+
+    def defl_polar_batched_host(self, G_host, out_host, k, oversample, power_iters, coeff_schedule, steps=None,
+                                sketch=None, seed=0, restore_mode=RESTORE_PADDED, gamma=0.0, engine=ENGINE_AUTO,
+                                exploit_symmetry=False):
+        """Host-buffer form: G_host/out_host are CPU tensors (pinned for speed); returns when out_host is filled."""
+        if G_host.is_cuda or out_host.is_cuda or not (G_host.is_contiguous() and out_host.is_contiguous()):
+            raise ValueError("G_host and out_host must be contiguous CPU tensors")
+        b, m, n = G_host.shape
+        sched, L = _schedule(coeff_schedule, steps)
+        opts = self._opts(sketch=sketch, seed=seed, restore_mode=restore_mode, gamma=gamma, engine=engine,
+                          exploit_symmetry=exploit_symmetry)
+        self._sync_stream()
+        rc = lib().defl_polar_batched_host(self._h, ctypes.c_void_p(G_host.data_ptr()),
+                                           ctypes.c_void_p(out_host.data_ptr()), b, m, n, _dtype_code(G_host), k,
+                                           oversample, power_iters, sched, L, ctypes.byref(opts))
+        self._check(rc)
+        return out_host
 
     def defl_brsvd_batched(self, G, k, oversample, power_iters, sketch=None, seed=0, engine=ENGINE_AUTO):
         """Algorithm 3 in the caller's orientation: returns (P[b,m,l], s[b,l], W[b,n,l], status[b])."""

@@ -242,6 +242,8 @@ int defl_destroy(defl_ctx* c) {
   cudaSetDevice(c->device);
   cudaDeviceSynchronize();
   if (c->ws) cudaFree(c->ws);
+  if (c->stage_in) cudaFree(c->stage_in);
+  if (c->stage_out) cudaFree(c->stage_out);
   if (c->wait_status) cudaFree(c->wait_status);
   for (int i = 0; i < DEFL_MAX_MARKS; ++i)
     if (c->marks[i]) cudaEventDestroy(c->marks[i]);
@@ -513,6 +515,33 @@ int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int 
         return DEFL_ERR_CUDA;
     }
   }
+  return DEFL_OK;
+}
+
+
+int defl_polar_batched_host(defl_ctx* c, const void* G_host, void* out_host, int b, int m, int n, int dtype, int k,
+                            int oversample, int power_iters, const float* coeff_schedule, int L,
+                            const defl_opts* opts) {
+  if (!c || !G_host || !out_host || b <= 0 || m <= 0 || n <= 0) return DEFL_ERR_ARG;
+  if (dtype != DEFL_BF16 && dtype != DEFL_F32) return DEFL_ERR_ARG;
+  cudaSetDevice(c->device);
+  const size_t bytes = (size_t)b * m * n * dtype_size(dtype);
+  if (bytes > c->stage_bytes) {
+    cudaDeviceSynchronize();
+    if (c->stage_in) cudaFree(c->stage_in);
+    if (c->stage_out) cudaFree(c->stage_out);
+    c->stage_in = c->stage_out = nullptr;
+    c->stage_bytes = 0;
+    if (ctx_fail(c, cudaMalloc(&c->stage_in, bytes), "cudaMalloc(staging)")) return DEFL_ERR_CUDA;
+    if (ctx_fail(c, cudaMalloc(&c->stage_out, bytes), "cudaMalloc(staging)")) return DEFL_ERR_CUDA;
+    c->stage_bytes = bytes;
+  }
+  if (ctx_fail(c, cudaMemcpyAsync(c->stage_in, G_host, bytes, cudaMemcpyHostToDevice, c->stream), "H2D")) return DEFL_ERR_CUDA;
+  const int rc = defl_polar_batched(c, c->stage_in, c->stage_out, b, m, n, dtype, k, oversample, power_iters,
+                                    coeff_schedule, L, opts, nullptr);
+  if (rc) return rc;
+  if (ctx_fail(c, cudaMemcpyAsync(out_host, c->stage_out, bytes, cudaMemcpyDeviceToHost, c->stream), "D2H")) return DEFL_ERR_CUDA;
+  if (ctx_fail(c, cudaStreamSynchronize(c->stream), "synchronize")) return DEFL_ERR_CUDA;
   return DEFL_OK;
 }
 

@@ -11,6 +11,9 @@ struct defl_ctx {
   cudaStream_t stream;
   void* ws;              // scratch memory owned by the context
   size_t ws_bytes;
+  void* stage_in;        // device staging of host inputs/outputs (defl_polar_batched_host)
+  void* stage_out;
+  size_t stage_bytes;
   int* wait_status;      // device word: the tensor engine ORs DEFL_ST_DEVICE_WAIT into it
   long long launches;    // kernels launched so far
   bool profiling;

@@ -146,6 +146,26 @@ int defl_psd_project(defl_ctx* ctx, const void* X, void* P, int n, int k,
  * dst is device memory of `count` elements of dtype (DEFL_BF16 or DEFL_F32). */
 int defl_fill_gaussian(defl_ctx* ctx, void* dst, size_t count, int dtype, uint64_t seed);
 
+/* Batched Frobenius norms without any allocation (no counterpart in the paper; it is the normalisation
+ * scale ||M||_F of Eq. 1 offered on its own). Written for callers that cannot allocate device memory when
+ * they call: code running inside another allocator's critical section or with all device memory already
+ * handed to a pool, and latency-critical loops where cudaMalloc's implicit device synchronisation is not
+ * acceptable. It needs no context and calls no cudaMalloc, cudaFree or allocating library routine: the
+ * partial sums live in a fixed array inside the library (DEFL_NOALLOC_MAX_BATCH x 148 doubles, about
+ * 300 KB, held by every GPU that loads the library until the process exits).
+ *   X      device, [b, count] of dtype (DEFL_BF16 or DEFL_F32), b matrices of `count` elements each
+ *   norms  device, [b] fp32, receives ||X[i]||_F
+ *   cuda_stream  cudaStream_t to enqueue on (NULL = default stream); the call does not synchronise
+ * Works on the CURRENT device. The first call on each device looks up that device's address of the array
+ * (a host-side query, no allocation); make that first call before starting any stream capture.
+ * All calls on a device share the array, so two calls whose kernels may overlap on the GPU (different
+ * streams, no ordering between them) race; calls on one stream are safe. Nothing needs clearing between
+ * calls: every slot that is read has just been written.
+ * Errors: DEFL_ERR_ARG (null pointer, b <= 0, count <= 0, bad dtype), DEFL_ERR_RANK (b > DEFL_NOALLOC_MAX_BATCH;
+ * split the batch), DEFL_ERR_CUDA. */
+#define DEFL_NOALLOC_MAX_BATCH 256
+int defl_frobenius_norms_noalloc(const void* X, int dtype, int b, long long count, float* norms, void* cuda_stream);
+
 /* Diagnostics: one batched product C[b,M,N] = alpha * opA(A) opB(B) through a chosen engine, used by the
  * tests to check the tensor-core tile engine against the fp32 engine (no counterpart in the paper).
  * A element (i,kk) is A[i*sa_i + kk*sa_k], B element (kk,j) is B[kk*sb_k + j*sb_j]; C is row-major [M,N].

@@ -26,7 +26,7 @@ CLASSICAL_QUINTIC = (1.875, -1.25, 0.375)
 EXPORTS = [
     "defl_create", "defl_destroy", "defl_set_stream", "defl_polar_workspace_bytes", "defl_psd_workspace_bytes",
     "defl_polar_batched", "defl_polar_batched_host", "defl_brsvd_batched", "defl_psd_project", "defl_fill_gaussian", "defl_debug_gemm",
-    "defl_set_profiling", "defl_get_stage_ms", "defl_launch_count", "defl_status_string", "defl_last_error",
+    "defl_frobenius_norms_noalloc", "defl_set_profiling", "defl_get_stage_ms", "defl_launch_count", "defl_status_string", "defl_last_error",
 ]
 
 

@@ -511,3 +511,48 @@ cudaError_t or_status_launch(int* status, int n, const int* word, cudaStream_t s
   return cudaGetLastError();
 }
 }  // namespace defl
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free batched Frobenius norm (see defl_frobenius_norms_noalloc in the public header).
+// The partial sums that frob_partial_kernel normally writes into context-owned scratch go into a
+// fixed file-scope device array instead, so the call needs no cudaMalloc at all.
+// ---------------------------------------------------------------------------------------------
+#include "../../include/defl.h"
+#include <mutex>
+
+namespace defl {
+constexpr int NOALLOC_NBLK = 148;   // partial sums per matrix (one per CTA)
+static __device__ __align__(256) double g_noalloc_partials[DEFL_NOALLOC_MAX_BATCH * NOALLOC_NBLK];
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+static double* g_noalloc_ptr[NOALLOC_MAX_DEVICES];   // device address of the array, per device
+static std::mutex g_noalloc_mutex;
+}  // namespace defl
+
+extern "C" int defl_frobenius_norms_noalloc(const void* X, int dtype, int b, long long count, float* norms,
+                                            void* cuda_stream) {
+  using namespace defl;
+  if (!X || !norms || b <= 0 || count <= 0 || (dtype != DEFL_BF16 && dtype != DEFL_F32)) return DEFL_ERR_ARG;
+  if (b > DEFL_NOALLOC_MAX_BATCH) return DEFL_ERR_RANK;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return DEFL_ERR_CUDA;
+  double* scratch = nullptr;
+  {
+    // First call on this device: ask the runtime where this device's copy of the array lives. The
+    // array's name is only a host-side handle here; a kernel must be given the looked-up address.
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_noalloc_partials) != cudaSuccess || !p) return DEFL_ERR_CUDA;
+      g_noalloc_ptr[dev] = reinterpret_cast<double*>(p);
+    }
+    scratch = g_noalloc_ptr[dev];
+  }
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  // every slot read by the second kernel is written by the first, so nothing needs clearing
+  frob_partial_kernel<<<dim3(NOALLOC_NBLK, b), 256, 0, st>>>(X, dtype, count, NOALLOC_NBLK, scratch);
+  if (cudaGetLastError() != cudaSuccess) return DEFL_ERR_CUDA;
+  rho_finalize_kernel<<<(b + 127) / 128, 128, 0, st>>>(scratch, NOALLOC_NBLK, b, norms, nullptr, nullptr, nullptr);
+  if (cudaGetLastError() != cudaSuccess) return DEFL_ERR_CUDA;
+  return DEFL_OK;
+}

@@ -140,9 +140,13 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--small", action="store_true", help="tiny workload for a quick functional check")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the matrices per shape group (profiling captures)")
     args = ap.parse_args()
     wl_name = "small" if args.small else "gpt2_xl"
-    wl = WORKLOADS[wl_name]
+    wl = dict(WORKLOADS[wl_name])
+    if args.batch > 0:
+        wl["groups"] = [(args.batch, m, n) for _, m, n in wl["groups"]]
+        wl["label"] += " [batch overridden to %d per group]" % args.batch
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -17,12 +17,12 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include <mutex>
+#include <cstdlib>
 
 namespace defl {
 
 namespace {
 
-constexpr int TILE_M = 128;
 constexpr int KBYTES = 128;                 // bytes of K per stage row (one swizzle span)
 constexpr int NUM_THREADS = 192;
 constexpr int MAX_STAGES = 6;
@@ -35,6 +35,7 @@ struct TcParams {
   int kblocks[2];              // K blocks per segment
   int M, N, batch;
   int BN;                      // tile width (UMMA N)
+  int tile_m;                  // 128 or 256 rows per tile
   int tiles_m, tiles_n;
   long long total_tiles;
   int a_mn_major, b_mn_major;  // 0 = K-major, 1 = MN-major
@@ -177,6 +178,128 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_
 }
 
 // ----------------------------------------------------------------------------- the kernel
+// Tile geometry. tile_m = 128: one 128-row accumulator per tile, two accumulator buffers (the epilogue
+// of tile i overlaps the products of tile i+1). tile_m = 256: two 128-row halves that share the B tile
+// (half the shared-memory -> tensor-core operand traffic per flop, which is what bounds this kernel: the
+// L2 -> SM path), both halves resident in tensor memory, so a single accumulator buffer.
+struct TileInfo {
+  int tn, tm, bz;
+  int halves;     // bit mask of the 128-row halves this tile computes
+  int n_eff;      // columns actually computed (multiple of 16)
+  bool skip;
+};
+
+__device__ __forceinline__ TileInfo tile_info(const TcParams& p, long long tile) {
+  TileInfo t;
+  t.tn = (int)(tile % p.tiles_n);
+  t.tm = (int)((tile / p.tiles_n) % p.tiles_m);
+  t.bz = (int)(tile / ((long long)p.tiles_n * p.tiles_m));
+  const int row0 = t.tm * p.tile_m, col_end = (t.tn + 1) * p.BN;
+  t.skip = p.symmetric && col_end <= row0;               // entirely below the diagonal
+  t.halves = 1;
+  if (p.tile_m == 256 && p.M - row0 > 128 && !(p.symmetric && col_end <= row0 + 128)) t.halves = 3;
+  int rem = p.N - t.tn * p.BN;
+  rem = (rem + 15) & ~15;
+  t.n_eff = rem < p.BN ? rem : p.BN;
+  return t;
+}
+
+
+// Epilogue of one 128-row half of a tile for the calling warp's 32 rows: read the accumulator from tensor
+// memory 16 columns at a time, apply the element-wise operation, store. The kind is a template parameter
+// so that the per-element code is branch-free.
+template <int EPI>
+__device__ __forceinline__ void epilogue_half(const TcParams& p, uint32_t taddr, int gi, int col0, int n_eff, int bz,
+                                              float alpha, float aux_scale, double& sq) {
+  const bool row_ok = gi < p.M;
+  const bool out_bf16 = (p.out_dtype == BF16), aux_bf16 = (p.aux_dtype == BF16);
+  const size_t crow = (size_t)bz * p.batch_c + (size_t)gi * p.ldc;
+  const size_t xrow = (size_t)bz * p.batch_aux + (size_t)gi * p.ld_aux;
+  const __nv_bfloat16* auxh = reinterpret_cast<const __nv_bfloat16*>(p.aux);
+  const float* auxf = reinterpret_cast<const float*>(p.aux);
+  __nv_bfloat16* outh = reinterpret_cast<__nv_bfloat16*>(p.C);
+  float* outf = reinterpret_cast<float*>(p.C);
+  const bool vec_ok = ((p.ldc & 7) == 0) && ((p.batch_c & 7) == 0) && ((p.ld_aux & 7) == 0 || EPI == EPI_STORE) &&
+                      ((p.batch_aux & 7) == 0 || EPI == EPI_STORE) && !p.symmetric;
+  for (int c0 = 0; c0 < n_eff; c0 += 16) {
+    uint32_t r[16];
+    __syncwarp();
+    tmem_ld16(taddr + (uint32_t)c0, r);
+    tmem_ld_wait();
+    const int gj0 = col0 + c0;
+    if (gj0 >= p.N || !row_ok) continue;
+    const bool full = (gj0 + 16 <= p.N) && vec_ok && ((gj0 & 7) == 0);
+    float x[16];
+    if (EPI != EPI_STORE) {
+      if (full && aux_bf16) {
+        const uint4* src = reinterpret_cast<const uint4*>(auxh + xrow + gj0);
+        uint4 pk[2] = {src[0], src[1]};
+        const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(pk);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { const float2 f = __bfloat1622float2(hh[j]); x[2 * j] = f.x; x[2 * j + 1] = f.y; }
+      } else if (full) {
+        const float4* src = reinterpret_cast<const float4*>(auxf + xrow + gj0);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { const float4 f = src[j]; x[4 * j] = f.x; x[4 * j + 1] = f.y; x[4 * j + 2] = f.z; x[4 * j + 3] = f.w; }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          x[j] = (gj0 + j < p.N) ? (aux_bf16 ? __bfloat162float(auxh[xrow + gj0 + j]) : auxf[xrow + gj0 + j]) : 0.f;
+      }
+    }
+    float v[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const float a = __uint_as_float(r[j]);
+      if (EPI == EPI_STORE) v[j] = alpha * a;
+      else if (EPI == EPI_POLY) v[j] = p.pb * x[j] + p.pc * a + ((gi == gj0 + j) ? p.pa : 0.f);
+      else if (EPI == EPI_AUX_PLUS) v[j] = aux_scale * x[j] + alpha * a;
+      else v[j] = (gj0 + j < p.N) ? (x[j] - a) : 0.f;
+    }
+    if (EPI == EPI_RESID_NORM) {
+      float sqf = 0.f;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) sqf = fmaf(v[j], v[j], sqf);
+      sq += (double)sqf;
+      continue;
+    }
+    if (full) {
+      if (out_bf16) {
+        uint4 pk[2];
+        __nv_bfloat162* hh = reinterpret_cast<__nv_bfloat162*>(pk);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) hh[j] = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+        uint4* dst = reinterpret_cast<uint4*>(outh + crow + gj0);
+        dst[0] = pk[0]; dst[1] = pk[1];
+      } else {
+        float4* dst = reinterpret_cast<float4*>(outf + crow + gj0);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+      }
+    } else if (!p.symmetric) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        if (gj0 + j < p.N) {
+          if (out_bf16) outh[crow + gj0 + j] = __float2bfloat16_rn(v[j]); else outf[crow + gj0 + j] = v[j];
+        }
+    } else {
+      // symmetric output: write the upper part directly and its mirror image; across the warp the
+      // mirrored stores of one column are contiguous (lanes are consecutive rows)
+      const size_t cb = (size_t)bz * p.batch_c;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const int gj = gj0 + j;
+        if (gj >= p.N) continue;
+        if (gj >= gi) { if (out_bf16) outh[crow + gj] = __float2bfloat16_rn(v[j]); else outf[crow + gj] = v[j]; }
+        if (gj > gi) {
+          const size_t m = cb + (size_t)gj * p.ldc + gi;
+          if (out_bf16) outh[m] = __float2bfloat16_rn(v[j]); else outf[m] = v[j];
+        }
+      }
+    }
+  }
+}
+
 template <int KIND_TF32>
 __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -191,6 +314,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzled tiles need 1024-byte alignment
   const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
   const int total_kblocks = p.kblocks[0] + (p.nseg > 1 ? p.kblocks[1] : 0);
+  const uint32_t nacc = (p.tile_m == 256) ? 1u : 2u;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -213,10 +337,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
     if (lane == 0) {
       uint32_t stage = 0, phase = 0;
       for (long long tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
-        const int tn = (int)(tile % p.tiles_n);
-        const int tm = (int)((tile / p.tiles_n) % p.tiles_m);
-        const int bz = (int)(tile / ((long long)p.tiles_n * p.tiles_m));
-        if (p.symmetric && (tn + 1) * p.BN <= tm * TILE_M) continue;   // tile entirely below the diagonal
+        const TileInfo t = tile_info(p, tile);
+        if (t.skip) continue;
         for (int seg = 0; seg < p.nseg; ++seg) {
           for (int kb = 0; kb < p.kblocks[seg]; ++kb) {
             mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag, p.status);
@@ -227,14 +349,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
             const uint32_t sb = sa + p.a_stage_bytes;
             const int k0 = kb * (KBYTES / p.esize);
             for (uint32_t bx = 0; bx < p.a_boxes; ++bx) {
-              const int mn0 = tm * TILE_M + (int)(bx * p.a_box_rows);
-              if (p.a_mn_major) tma_load_3d(sa + bx * p.a_box_bytes, &p.tmA[seg], fb, mn0, k0, bz);
-              else tma_load_3d(sa + bx * p.a_box_bytes, &p.tmA[seg], fb, k0, mn0, bz);
+              const int mn0 = t.tm * p.tile_m + (int)(bx * p.a_box_rows);
+              if (p.a_mn_major) tma_load_3d(sa + bx * p.a_box_bytes, &p.tmA[seg], fb, mn0, k0, t.bz);
+              else tma_load_3d(sa + bx * p.a_box_bytes, &p.tmA[seg], fb, k0, mn0, t.bz);
             }
             for (uint32_t bx = 0; bx < p.b_boxes; ++bx) {
-              const int mn0 = tn * p.BN + (int)(bx * p.b_box_rows);
-              if (p.b_mn_major) tma_load_3d(sb + bx * p.b_box_bytes, &p.tmB[seg], fb, mn0, k0, bz);
-              else tma_load_3d(sb + bx * p.b_box_bytes, &p.tmB[seg], fb, k0, mn0, bz);
+              const int mn0 = t.tn * p.BN + (int)(bx * p.b_box_rows);
+              if (p.b_mn_major) tma_load_3d(sb + bx * p.b_box_bytes, &p.tmB[seg], fb, mn0, k0, t.bz);
+              else tma_load_3d(sb + bx * p.b_box_bytes, &p.tmB[seg], fb, k0, mn0, t.bz);
             }
             if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
           }
@@ -251,14 +373,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       const uint32_t b_kstep = p.b_mn_major ? (uint32_t)(32 / p.esize) * 128u : 32u;
       const uint32_t a_lbo = p.a_mn_major ? p.a_box_bytes : 16u;
       const uint32_t b_lbo = p.b_mn_major ? p.b_box_bytes : 16u;
+      const uint32_t a_half = 128u * KBYTES;   // shared-memory offset of rows 128..255 of the A tile (either major)
       for (long long tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
-        const int tn = (int)(tile % p.tiles_n);
-        const int tm = (int)((tile / p.tiles_n) % p.tiles_m);
-        if (p.symmetric && (tn + 1) * p.BN <= tm * TILE_M) continue;
+        const TileInfo t = tile_info(p, tile);
+        if (t.skip) continue;
         mbar_wait(smem_u32(&acc_empty_bar[acc]), acc_phase ^ 1u, &abort_flag, p.status);
         if (abort_flag) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * 256u;
+        const uint32_t idesc = p.idesc | ((uint32_t)(t.n_eff >> 3) << 17);
+        const uint32_t d0 = tmem_base + ((p.tile_m == 256) ? 0u : acc * 256u);
         for (int kb = 0; kb < total_kblocks; ++kb) {
           mbar_wait(smem_u32(&full_bar[stage]), phase, &abort_flag, p.status);
           if (abort_flag) break;
@@ -267,16 +390,21 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
           const uint32_t sb = sa + p.a_stage_bytes;
 #pragma unroll
           for (int kk = 0; kk < KBYTES / 32; ++kk) {
-            const uint64_t adesc = make_smem_desc(sa + kk * a_kstep, a_lbo, 1024u);
             const uint64_t bdesc = make_smem_desc(sb + kk * b_kstep, b_lbo, 1024u);
-            umma<KIND_TF32>(d_tmem, adesc, bdesc, p.idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+            const uint64_t adesc = make_smem_desc(sa + kk * a_kstep, a_lbo, 1024u);
+            const uint32_t accum = (kb > 0 || kk > 0) ? 1u : 0u;
+            umma<KIND_TF32>(d0, adesc, bdesc, idesc, accum);
+            if (t.halves & 2) {
+              const uint64_t adesc1 = make_smem_desc(sa + a_half + kk * a_kstep, a_lbo, 1024u);
+              umma<KIND_TF32>(d0 + 256u, adesc1, bdesc, idesc, accum);
+            }
           }
           umma_commit(smem_u32(&empty_bar[stage]));          // frees the stage once these products are done
           if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
         }
         if (abort_flag) break;
         umma_commit(smem_u32(&acc_full_bar[acc]));           // accumulator complete
-        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        if (++acc == nacc) { acc = 0; acc_phase ^= 1u; }
       }
     }
   } else {
@@ -284,87 +412,40 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
     const int q = warp & 3;                 // tensor-memory lane quarter this warp may read
     uint32_t acc = 0, acc_phase = 0;
     for (long long tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
-      const int tn = (int)(tile % p.tiles_n);
-      const int tm = (int)((tile / p.tiles_n) % p.tiles_m);
-      const int bz = (int)(tile / ((long long)p.tiles_n * p.tiles_m));
-      if (p.symmetric && (tn + 1) * p.BN <= tm * TILE_M) continue;
+      const TileInfo t = tile_info(p, tile);
+      if (t.skip) continue;
+      const int tn = t.tn, tm = t.tm, bz = t.bz;
       const bool ok = mbar_wait(smem_u32(&acc_full_bar[acc]), acc_phase, &abort_flag, p.status);
       if (!ok) break;
       tc_fence_after();
-      const int gi = tm * TILE_M + q * 32 + lane;
-      const bool row_ok = gi < p.M;
       float alpha = p.alpha, aux_scale = p.aux_scale;
       if (p.alpha_dev) alpha *= p.alpha_dev[bz];
       if (p.aux_scale_dev) aux_scale *= p.aux_scale_dev[bz];
-      const long long crow = (long long)bz * p.batch_c + (long long)gi * p.ldc;
-      const long long xrow = (long long)bz * p.batch_aux + (long long)gi * p.ld_aux;
-      double sq = 0.0;
-      for (int c0 = 0; c0 < p.BN; c0 += 16) {
-        uint32_t r[16];
-        __syncwarp();
-        tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256u + (uint32_t)c0, r);
-        tmem_ld_wait();
-        const int gj0 = tn * p.BN + c0;
-        if (gj0 >= p.N) continue;           // warp-uniform
-        float v[16];
-        float sqf = 0.f;
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const int gj = gj0 + j;
-          const float a = __uint_as_float(r[j]);
-          float x = 0.f;
-          const bool in = row_ok && gj < p.N;
-          if (p.epilogue != EPI_STORE && in) x = ld_as_float(p.aux, xrow + gj, p.aux_dtype);
-          float o;
-          if (p.epilogue == EPI_STORE) o = alpha * a;
-          else if (p.epilogue == EPI_POLY) o = p.pb * x + p.pc * a + ((gi == gj) ? p.pa : 0.f);
-          else if (p.epilogue == EPI_AUX_PLUS) o = aux_scale * x + alpha * a;
-          else { o = 0.f; if (in) { const float d = x - a; sqf = fmaf(d, d, sqf); } }
-          v[j] = o;
+      for (int h = 0; h < (p.tile_m == 256 ? 2 : 1); ++h) {
+        double sq = 0.0;
+        if (t.halves & (1 << h)) {
+          const uint32_t tcol = (p.tile_m == 256) ? (uint32_t)h * 256u : acc * 256u;
+          const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + tcol;
+          const int gi = tm * p.tile_m + h * 128 + q * 32 + lane;
+          switch (p.epilogue) {
+            case EPI_STORE: epilogue_half<EPI_STORE>(p, taddr, gi, tn * p.BN, t.n_eff, bz, alpha, aux_scale, sq); break;
+            case EPI_POLY: epilogue_half<EPI_POLY>(p, taddr, gi, tn * p.BN, t.n_eff, bz, alpha, aux_scale, sq); break;
+            case EPI_AUX_PLUS: epilogue_half<EPI_AUX_PLUS>(p, taddr, gi, tn * p.BN, t.n_eff, bz, alpha, aux_scale, sq); break;
+            default: epilogue_half<EPI_RESID_NORM>(p, taddr, gi, tn * p.BN, t.n_eff, bz, alpha, aux_scale, sq); break;
+          }
         }
-        if (p.epilogue == EPI_RESID_NORM) { sq += (double)sqf; continue; }
-        if (!row_ok) continue;
-        const bool full = (gj0 + 16 <= p.N);
-        if (!p.symmetric) {
-          if (full && p.out_dtype == BF16 && ((crow + gj0) & 7) == 0) {
-            uint4 pk[2];
-            __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(pk);
+        if (p.epilogue == EPI_RESID_NORM) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) h[j] = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
-            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.C) + crow + gj0);
-            dst[0] = pk[0]; dst[1] = pk[1];
-          } else if (full && p.out_dtype == F32 && ((crow + gj0) & 3) == 0) {
-            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + crow + gj0);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-          } else {
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-              if (gj0 + j < p.N) st_from_float(p.C, crow + gj0 + j, p.out_dtype, v[j]);
-          }
-        } else {
-          // symmetric output: write the upper part directly and its mirror image; across the warp the
-          // mirrored stores of one column are contiguous (lanes are consecutive rows)
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int gj = gj0 + j;
-            if (gj >= p.N) continue;
-            if (gj >= gi) st_from_float(p.C, crow + gj, p.out_dtype, v[j]);
-            if (gj > gi) st_from_float(p.C, (long long)bz * p.batch_c + (long long)gj * p.ldc + gi, p.out_dtype, v[j]);
-          }
+          for (int o = 16; o > 0; o >>= 1) sq += __shfl_down_sync(0xffffffffu, sq, o);
+          if (lane == 0)
+            p.partials[(long long)bz * p.partials_per_batch + (((long long)tm * p.tiles_n + tn) * 2 + h) * 4 + (warp - 2)] = sq;
         }
       }
       // release the accumulator buffer
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&acc_empty_bar[acc]));
-      if (p.epilogue == EPI_RESID_NORM) {
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sq += __shfl_down_sync(0xffffffffu, sq, o);
-        if (lane == 0)
-          p.partials[(long long)bz * p.partials_per_batch + ((long long)tm * p.tiles_n + tn) * 4 + (warp - 2)] = sq;
-      }
-      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      if (++acc == nacc) { acc = 0; acc_phase ^= 1u; }
     }
   }
 
@@ -458,18 +539,13 @@ bool encode_map(CUtensorMap* tm, const void* base, int esize, bool tf32, bool mn
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Tuning overrides for experiments (read per launch): DEFL_TC_BN, DEFL_TC_TILE_M, DEFL_TC_STAGES.
 int choose_bn(int N) {
-  // widest tile that wastes the fewest padded columns; ties go to the wider tile
-  int best = 16;
-  long long best_cost = -1;
-  for (int bn = 256; bn >= 16; bn -= 16) {
-    const long long tiles = (N + bn - 1) / bn;
-    const long long padded = tiles * bn;
-    // cost: padded columns plus a fixed per-tile overhead that favours fewer, wider tiles
-    const long long cost = padded + tiles * 24;
-    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
-  }
-  return best;
+  if (const char* e = getenv("DEFL_TC_BN")) { const int v = atoi(e); if (v >= 16 && v <= 256 && v % 16 == 0) return v; }
+  // widest tile; edge tiles only compute the columns that exist (rounded up to 16), so a wide tile wastes
+  // at most 15 columns per tile row
+  const int r = (N + 15) & ~15;
+  return r < 256 ? r : 256;
 }
 
 }  // namespace
@@ -501,9 +577,14 @@ bool gemm_tc_supported(const GemmDesc& g) {
   return get_encode_fn() != nullptr;
 }
 
+int choose_tile_m(int M) {
+  if (const char* e = getenv("DEFL_TC_TILE_M")) { const int v = atoi(e); if (v == 128 || v == 256) return v; }
+  return M > 128 ? 256 : 128;
+}
+
 int gemm_tc_partials_per_batch(const GemmDesc& g) {
-  const int bn = choose_bn(g.N);
-  return ((g.M + TILE_M - 1) / TILE_M) * ((g.N + bn - 1) / bn) * 4;
+  const int bn = choose_bn(g.N), tmh = choose_tile_m(g.M);
+  return ((g.M + tmh - 1) / tmh) * ((g.N + bn - 1) / bn) * 8;
 }
 
 cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word, int num_sms, long long* launches) {
@@ -515,13 +596,14 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   p.esize = esize;
   p.M = g.M; p.N = g.N; p.batch = g.batch;
   p.BN = choose_bn(g.N);
-  p.tiles_m = (g.M + TILE_M - 1) / TILE_M;
+  p.tile_m = choose_tile_m(g.M);
+  p.tiles_m = (g.M + p.tile_m - 1) / p.tile_m;
   p.tiles_n = (g.N + p.BN - 1) / p.BN;
   p.total_tiles = (long long)p.tiles_m * p.tiles_n * g.batch;
   p.nseg = g.nseg;
   OperandPlan pa, pb;
   // when a dimension has extent 1 both strides may look "unit"; prefer K-major
-  if (!plan_operand(g.sa_i[0], g.sa_k[0], TILE_M, esize, &pa)) return cudaErrorNotSupported;
+  if (!plan_operand(g.sa_i[0], g.sa_k[0], p.tile_m, esize, &pa)) return cudaErrorNotSupported;
   if (!plan_operand(g.sb_j[0], g.sb_k[0], p.BN, esize, &pb)) return cudaErrorNotSupported;
   p.a_mn_major = pa.mn_major; p.b_mn_major = pb.mn_major;
   p.a_boxes = pa.boxes; p.a_box_bytes = pa.box_bytes; p.a_box_rows = pa.box_rows; p.a_stage_bytes = pa.stage_bytes;
@@ -537,15 +619,17 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
       return cudaErrorInvalidValue;
   }
   const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
-  const uint32_t smem_budget = 200 * 1024;
+  const uint32_t smem_budget = 224 * 1024;
   int stages = (int)(smem_budget / stage_bytes);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
+  if (const char* e = getenv("DEFL_TC_STAGES")) { const int v = atoi(e); if (v >= 2 && v <= stages) stages = v; }
   if (stages < 2) return cudaErrorNotSupported;
   p.stages = stages;
   // instruction descriptor: fp32 accumulate, operand format, majors, N >> 3 at bit 17, M >> 4 at bit 24
   const uint32_t fmt = tf32 ? 2u : 1u;
+  // (N is filled in per tile by the kernel: edge tiles compute fewer columns)
   p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)p.a_mn_major << 15) | ((uint32_t)p.b_mn_major << 16) |
-            ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+            ((uint32_t)(128 >> 4) << 24);
   p.epilogue = g.epilogue; p.out_dtype = g.out_dtype; p.aux_dtype = g.aux_dtype; p.symmetric = g.symmetric;
   p.C = g.C; p.ldc = g.ldc; p.batch_c = g.batch_c;
   p.aux = g.aux; p.ld_aux = g.ld_aux; p.batch_aux = g.batch_aux;

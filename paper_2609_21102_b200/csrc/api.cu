@@ -93,8 +93,14 @@ struct PolarWs {
   float* rho; float* inv_rho; float* inv_rho2;   // [b]
   int* status;        // [b]
   float* sketch;      // [b,ms,l] when the library draws the sketch
+  // split-precision bf16 copies for the tensor engine (bf16 storage only)
+  __nv_bfloat16* Lhi; __nv_bfloat16* Llo;   // [b,ml,lp]
+  __nv_bfloat16* Shi; __nv_bfloat16* Slo;   // [b,ms,lp]
+  __nv_bfloat16* Pc; __nv_bfloat16* Wc;     // [b,m,3kp], [b,n,3kp]
   size_t bytes;
 };
+
+inline int round_up8(int x) { return (x + 7) & ~7; }
 
 PolarWs carve_polar(void* base, int b, int m, int n, int dtype, int k, int l) {
   const int ms = m < n ? m : n, ml = m < n ? n : m;
@@ -123,19 +129,27 @@ PolarWs carve_polar(void* base, int b, int m, int n, int dtype, int k, int l) {
   w.inv_rho2 = cv.take<float>(b);
   w.status = cv.take<int>(b);
   w.sketch = cv.take<float>((size_t)b * ms * le);
+  const int lp = round_up8(le), kp = round_up8(ke);
+  const bool bf = (dtype == BF16);
+  w.Lhi = cv.take<__nv_bfloat16>(bf ? (size_t)b * ml * lp : 1);
+  w.Llo = cv.take<__nv_bfloat16>(bf ? (size_t)b * ml * lp : 1);
+  w.Shi = cv.take<__nv_bfloat16>(bf ? (size_t)b * ms * lp : 1);
+  w.Slo = cv.take<__nv_bfloat16>(bf ? (size_t)b * ms * lp : 1);
+  w.Pc = cv.take<__nv_bfloat16>(bf ? (size_t)b * m * 3 * kp : 1);
+  w.Wc = cv.take<__nv_bfloat16>(bf ? (size_t)b * n * 3 * kp : 1);
   w.bytes = cv.off;
   return w;
 }
 
 // CholeskyQR2 of the panel P[b, rows, l] in place: twice { W = P^T P; W = R^T R; P <- P R^-1 }.
-int orthonormalise(defl_ctx* c, float* P, int b, int rows, int l, const PolarWs& w, int* status) {
+int orthonormalise(defl_ctx* c, float* P, int b, int rows, int l, double* gram, float* Rinv, int* status) {
   const int nchunk = gram_num_chunks(rows);
   for (int pass = 0; pass < 2; ++pass) {
-    if (ctx_fail(c, gram_partial_launch(P, (long long)rows * l, b, rows, l, l, w.gram, c->stream, &c->launches), "gram"))
+    if (ctx_fail(c, gram_partial_launch(P, (long long)rows * l, b, rows, l, l, gram, c->stream, &c->launches), "gram"))
       return DEFL_ERR_CUDA;
-    if (ctx_fail(c, chol_inv_launch(w.gram, nchunk, b, l, w.Rinv, status, c->stream, &c->launches), "cholesky"))
+    if (ctx_fail(c, chol_inv_launch(gram, nchunk, b, l, Rinv, status, c->stream, &c->launches), "cholesky"))
       return DEFL_ERR_CUDA;
-    if (ctx_fail(c, panel_apply_launch(P, (long long)rows * l, l, w.Rinv, l, b, rows, l, l, P, (long long)rows * l, l,
+    if (ctx_fail(c, panel_apply_launch(P, (long long)rows * l, l, Rinv, l, b, rows, l, l, P, (long long)rows * l, l,
                                        c->stream, &c->launches), "panel apply"))
       return DEFL_ERR_CUDA;
   }
@@ -151,31 +165,42 @@ int run_brsvd(defl_ctx* c, const void* G, int b, int m, int n, int dtype, int l,
   // element (i,j) of A (ml x ms): tall G[i*n+j]; wide G[j*n+i]
   const long long a_si = tall ? n : 1, a_sj = tall ? 1 : n;
   int rc;
-  auto mul_A = [&](const float* Bp, float* Cp) {   // C[ml,l] = A B,  B[ms,l]
+  // Products with G on the tensor engine: the fp32 panel is split into bf16 hi + lo, both multiplied by the
+  // same G tile and accumulated in fp32 (G is bf16 already). Falls back to the fp32 engine when the shape or
+  // type does not fit (fp32 storage, strides not multiples of 16 bytes) or when that engine is requested.
+  const int lp = round_up8(l);
+  auto mul_G = [&](bool transposed, const float* Bp, float* Cp) {   // C = A B (ml x l) or A^T B (ms x l)
+    const int M = transposed ? ms : ml, K = transposed ? ml : ms;
     GemmDesc g = gemm_desc_zero();
-    g.batch = b; g.M = ml; g.N = l; g.K[0] = ms;
-    g.A[0] = G; g.sa_i[0] = a_si; g.sa_k[0] = a_sj; g.batch_a[0] = (long long)m * n; g.in_dtype = dtype;
-    g.B[0] = Bp; g.sb_k[0] = l; g.sb_j[0] = 1; g.batch_b[0] = (long long)ms * l; g.b_dtype = F32;
-    g.C = Cp; g.ldc = l; g.batch_c = (long long)ml * l; g.out_dtype = F32;
+    g.batch = b; g.M = M; g.N = l; g.K[0] = K;
+    g.A[0] = G; g.batch_a[0] = (long long)m * n; g.in_dtype = dtype;
+    g.sa_i[0] = transposed ? a_sj : a_si; g.sa_k[0] = transposed ? a_si : a_sj;
+    g.C = Cp; g.ldc = l; g.batch_c = (long long)M * l; g.out_dtype = F32;
     g.epilogue = EPI_STORE;
-    return run_gemm(c, g, DEFL_ENGINE_SIMT, "A*panel");
+    if (dtype == BF16 && engine != DEFL_ENGINE_SIMT) {
+      __nv_bfloat16* hi = transposed ? w.Lhi : w.Shi;
+      __nv_bfloat16* lo = transposed ? w.Llo : w.Slo;
+      GemmDesc t = g;
+      t.B[0] = hi; t.B[1] = lo; t.b_split = 2; t.b_dtype = BF16;
+      t.sb_k[0] = lp; t.sb_j[0] = 1; t.batch_b[0] = (long long)K * lp;
+      if (gemm_tc_supported(t)) {
+        if (ctx_fail(c, split_panel_launch(Bp, (long long)K * l, l, b, K, l, lp, hi, lo, c->stream, &c->launches), "split panel"))
+          return (int)DEFL_ERR_CUDA;
+        return run_gemm(c, t, DEFL_ENGINE_TENSOR, "G*panel (tensor)");
+      }
+    }
+    g.B[0] = Bp; g.sb_k[0] = l; g.sb_j[0] = 1; g.batch_b[0] = (long long)K * l; g.b_dtype = F32;
+    return run_gemm(c, g, DEFL_ENGINE_SIMT, "G*panel");
   };
-  auto mul_At = [&](const float* Bp, float* Cp) {  // C[ms,l] = A^T B, B[ml,l]
-    GemmDesc g = gemm_desc_zero();
-    g.batch = b; g.M = ms; g.N = l; g.K[0] = ml;
-    g.A[0] = G; g.sa_i[0] = a_sj; g.sa_k[0] = a_si; g.batch_a[0] = (long long)m * n; g.in_dtype = dtype;
-    g.B[0] = Bp; g.sb_k[0] = l; g.sb_j[0] = 1; g.batch_b[0] = (long long)ml * l; g.b_dtype = F32;
-    g.C = Cp; g.ldc = l; g.batch_c = (long long)ms * l; g.out_dtype = F32;
-    g.epilogue = EPI_STORE;
-    return run_gemm(c, g, DEFL_ENGINE_SIMT, "A^T*panel");
-  };
+  auto mul_A = [&](const float* Bp, float* Cp) { return mul_G(false, Bp, Cp); };
+  auto mul_At = [&](const float* Bp, float* Cp) { return mul_G(true, Bp, Cp); };
   if ((rc = mul_A(sketch, w.Lp))) return rc;                               // Y = A Omega
-  if ((rc = orthonormalise(c, w.Lp, b, ml, l, w, w.status))) return rc;    // Q
+  if ((rc = orthonormalise(c, w.Lp, b, ml, l, w.gram, w.Rinv, w.status))) return rc;    // Q
   for (int j = 0; j < J; ++j) {
     if ((rc = mul_At(w.Lp, w.Sp))) return rc;                              // A^T Q
-    if ((rc = orthonormalise(c, w.Sp, b, ms, l, w, w.status))) return rc;
+    if ((rc = orthonormalise(c, w.Sp, b, ms, l, w.gram, w.Rinv, w.status))) return rc;
     if ((rc = mul_A(w.Sp, w.Lp))) return rc;                               // A Y
-    if ((rc = orthonormalise(c, w.Lp, b, ml, l, w, w.status))) return rc;
+    if ((rc = orthonormalise(c, w.Lp, b, ml, l, w.gram, w.Rinv, w.status))) return rc;
   }
   if ((rc = mul_At(w.Lp, w.Sp))) return rc;                                // (Q^T A)^T, [ms, l]
   // thin SVD of Q^T A through the Gram core: (Q^T A)(Q^T A)^T = E diag(s^2) E^T
@@ -405,17 +430,38 @@ int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int 
   const float* left = tall ? w.Uk : w.Vk;     // [b,m,k]
   const float* right = tall ? w.Vk : w.Uk;    // [b,n,k]
   if (k > 0) {
-    // pass 1: norm of the residual, nothing stored
-    if (ctx_fail(c, scale_cols_launch(right, (long long)n * k, k, b, n, k, w.sv, l, nullptr, 1.f, 0.f, w.Ws,
-                                      (long long)n * k, k, c->stream, &c->launches), "W diag(s)"))
-      return DEFL_ERR_CUDA;
+    // R = G - P diag(s) W^T as a rank-k product on the product engine with G read in the epilogue.
+    // bf16 storage: the fp32 factors are split into bf16 hi + lo and the three significant cross terms are
+    // laid side by side along K, [hi|hi|lo] x [hi|lo|hi]^T, one tensor-core product of depth 3k.
+    const int kp = round_up8(k);
     GemmDesc g = gemm_desc_zero();
-    g.batch = b; g.M = m; g.N = n; g.K[0] = k;
-    g.A[0] = left; g.sa_i[0] = k; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * k; g.in_dtype = F32;
-    g.B[0] = w.Ws; g.sb_k[0] = 1; g.sb_j[0] = k; g.batch_b[0] = (long long)n * k; g.b_dtype = F32;
+    g.batch = b; g.M = m; g.N = n;
     g.aux = G; g.ld_aux = n; g.batch_aux = (long long)m * n; g.aux_dtype = dtype;
+    bool tensor_defl = false;
+    if (dtype == BF16 && engine != DEFL_ENGINE_SIMT) {
+      g.K[0] = 3 * kp;
+      g.A[0] = w.Pc; g.sa_i[0] = 3 * kp; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * 3 * kp; g.in_dtype = BF16;
+      g.B[0] = w.Wc; g.sb_k[0] = 1; g.sb_j[0] = 3 * kp; g.batch_b[0] = (long long)n * 3 * kp; g.b_dtype = BF16;
+      tensor_defl = gemm_tc_supported(g);
+    }
+    const int deng = tensor_defl ? DEFL_ENGINE_TENSOR : DEFL_ENGINE_SIMT;
+    if (tensor_defl) {
+      if (ctx_fail(c, split_concat3_launch(left, (long long)m * k, k, b, m, k, kp, nullptr, 0, nullptr, 0.f, 0.f, 0, w.Pc,
+                                           c->stream, &c->launches), "split P"))
+        return DEFL_ERR_CUDA;
+      if (ctx_fail(c, split_concat3_launch(right, (long long)n * k, k, b, n, k, kp, w.sv, l, nullptr, 1.f, 0.f, 1, w.Wc,
+                                           c->stream, &c->launches), "split W diag(s)"))
+        return DEFL_ERR_CUDA;
+    } else {
+      if (ctx_fail(c, scale_cols_launch(right, (long long)n * k, k, b, n, k, w.sv, l, nullptr, 1.f, 0.f, w.Ws,
+                                        (long long)n * k, k, c->stream, &c->launches), "W diag(s)"))
+        return DEFL_ERR_CUDA;
+      g.K[0] = k;
+      g.A[0] = left; g.sa_i[0] = k; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * k; g.in_dtype = F32;
+      g.B[0] = w.Ws; g.sb_k[0] = 1; g.sb_j[0] = k; g.batch_b[0] = (long long)n * k; g.b_dtype = F32;
+    }
+    // pass 1: norm of the residual, nothing stored
     g.epilogue = EPI_RESID_NORM; g.partials = w.npart;
-    const int deng = DEFL_ENGINE_SIMT;   // fp32 panels: exact fp32 products
     g.partials_per_batch = partials_per_batch(g, deng);
     if ((rc = run_gemm(c, g, deng, "residual norm"))) return rc;
     if (ctx_fail(c, rho_finalize_launch(w.npart, g.partials_per_batch, b, w.rho, w.inv_rho, w.inv_rho2, w.status,
@@ -423,9 +469,14 @@ int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int 
       return DEFL_ERR_CUDA;
     // pass 2: X0 = G/rho - P diag(s/rho - 1/gamma) W^T   (ADD mode: without the 1/gamma term)
     const float pad = (mode == DEFL_RESTORE_PADDED) ? 1.f / gamma : 0.f;
-    if (ctx_fail(c, scale_cols_launch(right, (long long)n * k, k, b, n, k, w.sv, l, w.inv_rho, -1.f, pad, w.Ws,
-                                      (long long)n * k, k, c->stream, &c->launches), "W diag(coef)"))
+    if (tensor_defl) {
+      if (ctx_fail(c, split_concat3_launch(right, (long long)n * k, k, b, n, k, kp, w.sv, l, w.inv_rho, -1.f, pad, 1, w.Wc,
+                                           c->stream, &c->launches), "split W diag(coef)"))
+        return DEFL_ERR_CUDA;
+    } else if (ctx_fail(c, scale_cols_launch(right, (long long)n * k, k, b, n, k, w.sv, l, w.inv_rho, -1.f, pad, w.Ws,
+                                             (long long)n * k, k, c->stream, &c->launches), "W diag(coef)")) {
       return DEFL_ERR_CUDA;
+    }
     g.epilogue = EPI_AUX_PLUS; g.partials = nullptr;
     g.aux_scale = 1.f; g.aux_scale_dev = w.inv_rho; g.alpha = 1.f;
     g.C = bufs[cur]; g.ldc = n; g.batch_c = (long long)m * n; g.out_dtype = dtype;
@@ -489,14 +540,31 @@ int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int 
 
   // ---- stage 3: restore (Eq. 3) in ADD mode: out += P W^T ------------------------------------------
   if (k > 0 && mode == DEFL_RESTORE_ADD) {
+    const int kp = round_up8(k);
     GemmDesc g = gemm_desc_zero();
-    g.batch = b; g.M = m; g.N = n; g.K[0] = k;
-    g.A[0] = left; g.sa_i[0] = k; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * k; g.in_dtype = F32;
-    g.B[0] = right; g.sb_k[0] = 1; g.sb_j[0] = k; g.batch_b[0] = (long long)n * k; g.b_dtype = F32;
+    g.batch = b; g.M = m; g.N = n;
     g.aux = out; g.ld_aux = n; g.batch_aux = (long long)m * n; g.aux_dtype = dtype;
     g.C = out; g.ldc = n; g.batch_c = (long long)m * n; g.out_dtype = dtype;
     g.epilogue = EPI_AUX_PLUS;
-    if ((rc = run_gemm(c, g, DEFL_ENGINE_SIMT, "restore"))) return rc;
+    bool tensor_restore = false;
+    if (dtype == BF16 && engine != DEFL_ENGINE_SIMT) {
+      g.K[0] = 3 * kp;
+      g.A[0] = w.Pc; g.sa_i[0] = 3 * kp; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * 3 * kp; g.in_dtype = BF16;
+      g.B[0] = w.Wc; g.sb_k[0] = 1; g.sb_j[0] = 3 * kp; g.batch_b[0] = (long long)n * 3 * kp; g.b_dtype = BF16;
+      tensor_restore = gemm_tc_supported(g);
+    }
+    if (tensor_restore) {
+      // w.Pc still holds the split left factor from the deflation stage; rebuild the right one unscaled
+      if (ctx_fail(c, split_concat3_launch(right, (long long)n * k, k, b, n, k, kp, nullptr, 0, nullptr, 0.f, 0.f, 1, w.Wc,
+                                           c->stream, &c->launches), "split W"))
+        return DEFL_ERR_CUDA;
+      if ((rc = run_gemm(c, g, DEFL_ENGINE_TENSOR, "restore (tensor)"))) return rc;
+    } else {
+      g.K[0] = k;
+      g.A[0] = left; g.sa_i[0] = k; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * k; g.in_dtype = F32;
+      g.B[0] = right; g.sb_k[0] = 1; g.sb_j[0] = k; g.batch_b[0] = (long long)n * k; g.b_dtype = F32;
+      if ((rc = run_gemm(c, g, DEFL_ENGINE_SIMT, "restore"))) return rc;
+    }
   }
   ctx_stage_mark(c);
 

@@ -39,6 +39,8 @@ struct GemmDesc {
   const float* aux_scale_dev;   // optional per-batch multiplier of aux_scale (device, [batch])
   double* partials;             // EPI_RESID_NORM: [batch, partials_per_batch] written, one slot per CTA-warp
   int partials_per_batch;
+  int b_split;                  // 2: opB = B[0] + B[1] (same shape and strides, nseg must be 1); the A tile is loaded once
+  int round_tf32;               // fp32 output rounded to nearest tf32 (it feeds tf32 products, which would truncate)
   int symmetric;                // output is symmetric (M == N): compute upper tiles only and mirror
 };
 
@@ -63,6 +65,11 @@ int gemm_tc_partials_per_batch(const GemmDesc& g);
 __device__ __forceinline__ float ld_as_float(const void* p, long long idx, int dt) {
   return dt == BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[idx])
                     : reinterpret_cast<const float*>(p)[idx];
+}
+__device__ __forceinline__ float round_to_tf32(float x) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+  return __uint_as_float(r);
 }
 __device__ __forceinline__ void st_from_float(void* p, long long idx, int dt, float v) {
   if (dt == BF16) reinterpret_cast<__nv_bfloat16*>(p)[idx] = __float2bfloat16_rn(v);

@@ -29,5 +29,6 @@ int ctx_reserve(defl_ctx* c, size_t bytes);
 void ctx_stage_mark(defl_ctx* c);
 int run_gemm(defl_ctx* c, const GemmDesc& g, int engine, const char* what);
 int partials_per_batch(const GemmDesc& g, int engine);
+int orthonormalise(defl_ctx* c, float* P, int b, int rows, int l, double* gram, float* Rinv, int* status);
 cudaError_t or_status_launch(int* status, int n, const int* word, cudaStream_t st, long long* launches);
 }  // namespace defl

@@ -59,7 +59,11 @@ __global__ void __launch_bounds__(NT) gemm_simt_kernel(const GemmDesc g) {
         if (b_jfast) { kk = e / BN; j = e % BN; } else { j = e / BK; kk = e % BK; }
         const int gj = col0 + j, gk = k0 + kk;
         float v = 0.f;
-        if (gj < g.N && gk < K) v = to_f<TB>(B[(long long)gk * sbk + (long long)gj * sbj]);
+        if (gj < g.N && gk < K) {
+          v = to_f<TB>(B[(long long)gk * sbk + (long long)gj * sbj]);
+          if (g.b_split == 2)
+            v += to_f<TB>((reinterpret_cast<const TB*>(g.B[1]) + (long long)bz * g.batch_b[0])[(long long)gk * sbk + (long long)gj * sbj]);
+        }
         Bs[kk][j] = v;
       }
       __syncthreads();
@@ -109,6 +113,7 @@ __global__ void __launch_bounds__(NT) gemm_simt_kernel(const GemmDesc g) {
           continue;
         }
       }
+      if (g.round_tf32) v = round_to_tf32(v);
       if (g.symmetric) {
         if (gj >= gi) st_from_float(g.C, coff + (long long)gi * g.ldc + gj, g.out_dtype, v);
         if (gj > gi) st_from_float(g.C, coff + (long long)gj * g.ldc + gi, g.out_dtype, v);

@@ -32,6 +32,7 @@ struct TcParams {
   CUtensorMap tmA[2];
   CUtensorMap tmB[2];
   int nseg;
+  int b_split;                 // 2: B is the sum of two operands (tmB[0] + tmB[1]) that share A; else 1
   int kblocks[2];              // K blocks per segment
   int M, N, batch;
   int BN;                      // tile width (UMMA N)
@@ -41,13 +42,14 @@ struct TcParams {
   int a_mn_major, b_mn_major;  // 0 = K-major, 1 = MN-major
   int esize;                   // operand element size in bytes (2 bf16, 4 tf32)
   int stages;
-  uint32_t a_stage_bytes, b_stage_bytes;
+  uint32_t a_stage_bytes, b_stage_bytes;   // b_stage_bytes covers all splits
+  uint32_t b_split_bytes;                  // bytes of one B split within a stage
   uint32_t a_boxes, b_boxes;   // TMA boxes per stage per operand
   uint32_t a_box_bytes, b_box_bytes;
   uint32_t a_box_rows, b_box_rows;   // MN extent covered by one box (K-major) or 128B/esize (MN-major)
   uint32_t idesc;
   // epilogue
-  int epilogue, out_dtype, aux_dtype, symmetric;
+  int epilogue, out_dtype, aux_dtype, symmetric, round_tf32;
   void* C; long long ldc, batch_c;
   const void* aux; long long ld_aux, batch_aux;
   float alpha, aux_scale, pa, pb, pc;
@@ -85,10 +87,12 @@ __device__ __forceinline__ unsigned long long global_ns() {
   return t;
 }
 
-// Bounded wait. `abort_flag` (shared memory) short-circuits every later wait once one has failed.
+// Bounded wait. A short burst of polls first (the common case: the barrier flips within the hardware
+// suspend window of try_wait); after that every poll also checks the CTA's abort flag and a wall-clock
+// budget, so that a protocol error or a lost copy ends in a status bit instead of a hang.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-  if (*abort_flag) return false;
-  for (int i = 0; i < 4096; ++i)
+#pragma unroll 1
+  for (int i = 0; i < 64; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   while (true) {
@@ -177,6 +181,11 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_
   return d;
 }
 
+// constant upper part of a descriptor; the 14-bit start-address field (address >> 4) is added per product
+__device__ __forceinline__ uint64_t smem_desc_hi(uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return make_smem_desc(0, lbo_bytes, sbo_bytes);
+}
+
 // ----------------------------------------------------------------------------- the kernel
 // Tile geometry. tile_m = 128: one 128-row accumulator per tile, two accumulator buffers (the epilogue
 // of tile i overlaps the products of tile i+1). tile_m = 256: two 128-row halves that share the B tile
@@ -256,6 +265,10 @@ __device__ __forceinline__ void epilogue_half(const TcParams& p, uint32_t taddr,
       else if (EPI == EPI_AUX_PLUS) v[j] = aux_scale * x[j] + alpha * a;
       else v[j] = (gj0 + j < p.N) ? (x[j] - a) : 0.f;
     }
+    if (p.round_tf32) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) v[j] = round_to_tf32(v[j]);
+    }
     if (EPI == EPI_RESID_NORM) {
       float sqf = 0.f;
 #pragma unroll
@@ -300,7 +313,7 @@ __device__ __forceinline__ void epilogue_half(const TcParams& p, uint32_t taddr,
   }
 }
 
-template <int KIND_TF32>
+template <int KIND_TF32, int BSPLIT>
 __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
@@ -341,8 +354,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
         if (t.skip) continue;
         for (int seg = 0; seg < p.nseg; ++seg) {
           for (int kb = 0; kb < p.kblocks[seg]; ++kb) {
-            mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag, p.status);
-            if (abort_flag) break;
+            if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag, p.status)) break;
             const uint32_t fb = smem_u32(&full_bar[stage]);
             mbar_expect_tx(fb, stage_bytes);
             const uint32_t sa = smem_base + stage * stage_bytes;
@@ -353,10 +365,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
               if (p.a_mn_major) tma_load_3d(sa + bx * p.a_box_bytes, &p.tmA[seg], fb, mn0, k0, t.bz);
               else tma_load_3d(sa + bx * p.a_box_bytes, &p.tmA[seg], fb, k0, mn0, t.bz);
             }
-            for (uint32_t bx = 0; bx < p.b_boxes; ++bx) {
-              const int mn0 = t.tn * p.BN + (int)(bx * p.b_box_rows);
-              if (p.b_mn_major) tma_load_3d(sb + bx * p.b_box_bytes, &p.tmB[seg], fb, mn0, k0, t.bz);
-              else tma_load_3d(sb + bx * p.b_box_bytes, &p.tmB[seg], fb, k0, mn0, t.bz);
+#pragma unroll
+            for (int sp = 0; sp < BSPLIT; ++sp) {
+              const CUtensorMap* tmb = &p.tmB[BSPLIT > 1 ? sp : seg];
+              const uint32_t sbs = sb + (uint32_t)sp * p.b_split_bytes;
+              for (uint32_t bx = 0; bx < p.b_boxes; ++bx) {
+                const int mn0 = t.tn * p.BN + (int)(bx * p.b_box_rows);
+                if (p.b_mn_major) tma_load_3d(sbs + bx * p.b_box_bytes, tmb, fb, mn0, k0, t.bz);
+                else tma_load_3d(sbs + bx * p.b_box_bytes, tmb, fb, k0, mn0, t.bz);
+              }
             }
             if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
           }
@@ -369,40 +386,44 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
-      const uint32_t a_kstep = p.a_mn_major ? (uint32_t)(32 / p.esize) * 128u : 32u;   // bytes per UMMA K step
-      const uint32_t b_kstep = p.b_mn_major ? (uint32_t)(32 / p.esize) * 128u : 32u;
-      const uint32_t a_lbo = p.a_mn_major ? p.a_box_bytes : 16u;
-      const uint32_t b_lbo = p.b_mn_major ? p.b_box_bytes : 16u;
-      const uint32_t a_half = 128u * KBYTES;   // shared-memory offset of rows 128..255 of the A tile (either major)
+      // descriptor start addresses advance in units of 16 bytes
+      const uint32_t a_kstep16 = (p.a_mn_major ? (uint32_t)(32 / p.esize) * 128u : 32u) >> 4;   // per UMMA K step
+      const uint32_t b_kstep16 = (p.b_mn_major ? (uint32_t)(32 / p.esize) * 128u : 32u) >> 4;
+      const uint64_t a_hi = smem_desc_hi(p.a_mn_major ? p.a_box_bytes : 16u, 1024u);
+      const uint64_t b_hi = smem_desc_hi(p.b_mn_major ? p.b_box_bytes : 16u, 1024u);
+      const uint32_t a_half16 = (128u * KBYTES) >> 4;   // rows 128..255 of the A tile (either major)
+      const uint32_t split16 = p.b_split_bytes >> 4;
+      const uint32_t stage16 = stage_bytes >> 4, a_stage16 = p.a_stage_bytes >> 4, base16 = smem_base >> 4;
       for (long long tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
         const TileInfo t = tile_info(p, tile);
         if (t.skip) continue;
-        mbar_wait(smem_u32(&acc_empty_bar[acc]), acc_phase ^ 1u, &abort_flag, p.status);
-        if (abort_flag) break;
+        if (!mbar_wait(smem_u32(&acc_empty_bar[acc]), acc_phase ^ 1u, &abort_flag, p.status)) break;
         tc_fence_after();
         const uint32_t idesc = p.idesc | ((uint32_t)(t.n_eff >> 3) << 17);
         const uint32_t d0 = tmem_base + ((p.tile_m == 256) ? 0u : acc * 256u);
+        const bool two = (t.halves & 2) != 0;
+        bool ok = true;
         for (int kb = 0; kb < total_kblocks; ++kb) {
-          mbar_wait(smem_u32(&full_bar[stage]), phase, &abort_flag, p.status);
-          if (abort_flag) break;
+          if (!mbar_wait(smem_u32(&full_bar[stage]), phase, &abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = smem_base + stage * stage_bytes;
-          const uint32_t sb = sa + p.a_stage_bytes;
+          const uint32_t sa16 = base16 + stage * stage16;
+          const uint32_t sb16 = sa16 + a_stage16;
 #pragma unroll
           for (int kk = 0; kk < KBYTES / 32; ++kk) {
-            const uint64_t bdesc = make_smem_desc(sb + kk * b_kstep, b_lbo, 1024u);
-            const uint64_t adesc = make_smem_desc(sa + kk * a_kstep, a_lbo, 1024u);
+            const uint64_t adesc = a_hi | (uint64_t)(sa16 + kk * a_kstep16);
+            const uint64_t bdesc = b_hi | (uint64_t)(sb16 + kk * b_kstep16);
             const uint32_t accum = (kb > 0 || kk > 0) ? 1u : 0u;
             umma<KIND_TF32>(d0, adesc, bdesc, idesc, accum);
-            if (t.halves & 2) {
-              const uint64_t adesc1 = make_smem_desc(sa + a_half + kk * a_kstep, a_lbo, 1024u);
-              umma<KIND_TF32>(d0 + 256u, adesc1, bdesc, idesc, accum);
+            if (two) umma<KIND_TF32>(d0 + 256u, adesc + a_half16, bdesc, idesc, accum);
+            if (BSPLIT == 2) {
+              umma<KIND_TF32>(d0, adesc, bdesc + split16, idesc, 1u);
+              if (two) umma<KIND_TF32>(d0 + 256u, adesc + a_half16, bdesc + split16, idesc, 1u);
             }
           }
           umma_commit(smem_u32(&empty_bar[stage]));          // frees the stage once these products are done
           if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
         }
-        if (abort_flag) break;
+        if (!ok) break;
         umma_commit(smem_u32(&acc_full_bar[acc]));           // accumulator complete
         if (++acc == nacc) { acc = 0; acc_phase ^= 1u; }
       }
@@ -438,7 +459,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) sq += __shfl_down_sync(0xffffffffu, sq, o);
           if (lane == 0)
-            p.partials[(long long)bz * p.partials_per_batch + (((long long)tm * p.tiles_n + tn) * 2 + h) * 4 + (warp - 2)] = sq;
+            p.partials[(long long)bz * p.partials_per_batch + (((long long)tm * p.tiles_n + tn) * (p.tile_m == 256 ? 2 : 1) + h) * 4 + (warp - 2)] = sq;
         }
       }
       // release the accumulator buffer
@@ -553,6 +574,7 @@ int choose_bn(int N) {
 bool gemm_tc_supported(const GemmDesc& g) {
   if (g.batch <= 0 || g.M <= 0 || g.N <= 0) return false;
   if (g.nseg < 1 || g.nseg > 2) return false;
+  if (g.b_split == 2 && (g.nseg != 1 || !aligned16(g.B[1]))) return false;
   if (g.b_dtype != g.in_dtype) return false;
   const int esize = (int)dtype_size(g.in_dtype);
   if (g.symmetric && g.M != g.N) return false;
@@ -584,7 +606,7 @@ int choose_tile_m(int M) {
 
 int gemm_tc_partials_per_batch(const GemmDesc& g) {
   const int bn = choose_bn(g.N), tmh = choose_tile_m(g.M);
-  return ((g.M + tmh - 1) / tmh) * ((g.N + bn - 1) / bn) * 8;
+  return ((g.M + tmh - 1) / tmh) * ((g.N + bn - 1) / bn) * (tmh == 256 ? 8 : 4);
 }
 
 cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word, int num_sms, long long* launches) {
@@ -607,8 +629,15 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   if (!plan_operand(g.sb_j[0], g.sb_k[0], p.BN, esize, &pb)) return cudaErrorNotSupported;
   p.a_mn_major = pa.mn_major; p.b_mn_major = pb.mn_major;
   p.a_boxes = pa.boxes; p.a_box_bytes = pa.box_bytes; p.a_box_rows = pa.box_rows; p.a_stage_bytes = pa.stage_bytes;
-  p.b_boxes = pb.boxes; p.b_box_bytes = pb.box_bytes; p.b_box_rows = pb.box_rows; p.b_stage_bytes = pb.stage_bytes;
+  p.b_split = (g.b_split == 2) ? 2 : 1;
+  p.b_boxes = pb.boxes; p.b_box_bytes = pb.box_bytes; p.b_box_rows = pb.box_rows;
+  p.b_split_bytes = pb.stage_bytes; p.b_stage_bytes = pb.stage_bytes * p.b_split;
   const int span = KBYTES / esize;
+  if (p.b_split == 2) {
+    if (!encode_map(&p.tmB[1], g.B[1], esize, tf32, pb.mn_major, g.N, g.K[0], g.sb_j[0], g.sb_k[0], g.batch,
+                    g.batch_b[0], pb.box_rows))
+      return cudaErrorInvalidValue;
+  }
   for (int s = 0; s < g.nseg; ++s) {
     p.kblocks[s] = (g.K[s] + span - 1) / span;
     if (!encode_map(&p.tmA[s], g.A[s], esize, tf32, pa.mn_major, g.M, g.K[s], g.sa_i[s], g.sa_k[s], g.batch,
@@ -630,7 +659,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   // (N is filled in per tile by the kernel: edge tiles compute fewer columns)
   p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)p.a_mn_major << 15) | ((uint32_t)p.b_mn_major << 16) |
             ((uint32_t)(128 >> 4) << 24);
-  p.epilogue = g.epilogue; p.out_dtype = g.out_dtype; p.aux_dtype = g.aux_dtype; p.symmetric = g.symmetric;
+  p.epilogue = g.epilogue; p.out_dtype = g.out_dtype; p.aux_dtype = g.aux_dtype; p.symmetric = g.symmetric; p.round_tf32 = g.round_tf32;
   p.C = g.C; p.ldc = g.ldc; p.batch_c = g.batch_c;
   p.aux = g.aux; p.ld_aux = g.ld_aux; p.batch_aux = g.batch_aux;
   p.alpha = g.alpha; p.aux_scale = g.aux_scale; p.pa = g.pa; p.pb = g.pb; p.pc = g.pc;
@@ -640,13 +669,13 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
 
   const size_t smem = (size_t)stages * stage_bytes + 1024;
   cudaError_t e;
-  if (tf32) e = cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  else e = cudaFuncSetAttribute(gemm_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  auto kern = tf32 ? (p.b_split == 2 ? gemm_tc_kernel<1, 2> : gemm_tc_kernel<1, 1>)
+                   : (p.b_split == 2 ? gemm_tc_kernel<0, 2> : gemm_tc_kernel<0, 1>);
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   long long grid = p.total_tiles < num_sms ? p.total_tiles : num_sms;
   if (grid < 1) grid = 1;
-  if (tf32) gemm_tc_kernel<1><<<(unsigned)grid, NUM_THREADS, smem, st>>>(p);
-  else gemm_tc_kernel<0><<<(unsigned)grid, NUM_THREADS, smem, st>>>(p);
+  kern<<<(unsigned)grid, NUM_THREADS, smem, st>>>(p);
   if (launches) ++*launches;
   return cudaGetLastError();
 }

@@ -19,12 +19,14 @@ namespace defl {
 constexpr int GRAM_ROWS = 256;   // rows per CTA
 constexpr int GRAM_SUB = 32;     // rows per fp32 sub-accumulation
 
-__global__ void __launch_bounds__(256) gram_partial_kernel(const float* __restrict__ Y, long long batch_stride,
-                                                           int rows, int l, int ld, int nchunk,
+__global__ void __launch_bounds__(256) gram_partial_kernel(const float* __restrict__ Y, const float* __restrict__ Y2,
+                                                           long long batch_stride, int rows, int l, int ld, int nchunk,
                                                            double* __restrict__ partial) {
   __shared__ float tile[GRAM_SUB][MAX_L + 1];
+  __shared__ float tile2[GRAM_SUB][MAX_L + 1];
   const int chunk = blockIdx.x, bz = blockIdx.y, tid = threadIdx.x;
   const float* Yb = Y + (long long)bz * batch_stride;
+  const float* Y2b = Y2 ? Y2 + (long long)bz * batch_stride : nullptr;
   const int tx = tid % 16, ty = tid / 16;   // 16 x 16 threads, each a 4 x 4 block of the l x l Gram
   double acc[4][4];
 #pragma unroll
@@ -37,6 +39,7 @@ __global__ void __launch_bounds__(256) gram_partial_kernel(const float* __restri
       const int rr = e / l, c = e % l;
       const int gr = r0 + rr;
       tile[rr][c] = (gr < r_end) ? Yb[(long long)gr * ld + c] : 0.f;
+      tile2[rr][c] = Y2b ? ((gr < r_end) ? Y2b[(long long)gr * ld + c] : 0.f) : tile[rr][c];
     }
     __syncthreads();
     float f[4][4];
@@ -49,7 +52,7 @@ __global__ void __launch_bounds__(256) gram_partial_kernel(const float* __restri
 #pragma unroll
       for (int i = 0; i < 4; ++i) a[i] = (ty * 4 + i < l) ? tile[rr][ty * 4 + i] : 0.f;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) b[j] = (tx * 4 + j < l) ? tile[rr][tx * 4 + j] : 0.f;
+      for (int j = 0; j < 4; ++j) b[j] = (tx * 4 + j < l) ? tile2[rr][tx * 4 + j] : 0.f;
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -74,9 +77,9 @@ __global__ void __launch_bounds__(256) gram_partial_kernel(const float* __restri
 int gram_num_chunks(int rows) { return (rows + GRAM_ROWS - 1) / GRAM_ROWS; }
 
 cudaError_t gram_partial_launch(const float* Y, long long batch_stride, int batch, int rows, int l, int ld,
-                                double* partial, cudaStream_t st, long long* launches) {
+                                double* partial, cudaStream_t st, long long* launches, const float* Y2) {
   const int nchunk = gram_num_chunks(rows);
-  gram_partial_kernel<<<dim3(nchunk, batch), 256, 0, st>>>(Y, batch_stride, rows, l, ld, nchunk, partial);
+  gram_partial_kernel<<<dim3(nchunk, batch), 256, 0, st>>>(Y, Y2, batch_stride, rows, l, ld, nchunk, partial);
   if (launches) ++*launches;
   return cudaGetLastError();
 }
@@ -384,14 +387,18 @@ cudaError_t frob_partial_launch(const void* X, int dtype, int batch, long long c
   return cudaGetLastError();
 }
 
-// rho[b] = sqrt(sum of partials in index order); inv_rho[b] = 1/rho (0 and status bit 4 when rho is 0 or not finite)
+// rho[b] = sqrt(sum of partials); one warp per matrix, lane-strided sums then a shuffle tree (fixed order);
+// inv_rho[b] = 1/rho (0 and status bit 4 when rho is 0 or not finite)
 __global__ void rho_finalize_kernel(const double* __restrict__ partial, int nper, int batch, float* __restrict__ rho,
                                     float* __restrict__ inv_rho, float* __restrict__ inv_rho2,
                                     int* __restrict__ status) {
-  const int bz = blockIdx.x * blockDim.x + threadIdx.x;
+  const int bz = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (bz >= batch) return;
   double t = 0.0;
-  for (int i = 0; i < nper; ++i) t += partial[(long long)bz * nper + i];
+  for (int i = lane; i < nper; i += 32) t += partial[(long long)bz * nper + i];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+  if (lane != 0) return;
   const double r = sqrt(t);
   const bool ok = (r > 0.0) && isfinite(r);
   if (rho) rho[bz] = (float)r;
@@ -402,7 +409,7 @@ __global__ void rho_finalize_kernel(const double* __restrict__ partial, int nper
 
 cudaError_t rho_finalize_launch(const double* partial, int nper, int batch, float* rho, float* inv_rho,
                                 float* inv_rho2, int* status, cudaStream_t st, long long* launches) {
-  rho_finalize_kernel<<<(batch + 127) / 128, 128, 0, st>>>(partial, nper, batch, rho, inv_rho, inv_rho2, status);
+  rho_finalize_kernel<<<(batch + 3) / 4, 128, 0, st>>>(partial, nper, batch, rho, inv_rho, inv_rho2, status);
   if (launches) ++*launches;
   return cudaGetLastError();
 }
@@ -432,18 +439,22 @@ cudaError_t scale_cols_launch(const float* In, long long in_bs, int ld_in, int b
 
 // Out[b, i] = scale[b] * In[b, i]  (type conversion allowed)
 __global__ void scale_kernel(const void* __restrict__ In, int in_dt, void* __restrict__ Out, int out_dt,
-                             long long count, const float* __restrict__ scale) {
+                             long long count, const float* __restrict__ scale, int round_tf32) {
   const int bz = blockIdx.y;
   const float sc = scale ? scale[bz] : 1.f;
   const long long base = (long long)bz * count;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (long long)gridDim.x * blockDim.x)
-    st_from_float(Out, base + i, out_dt, sc * ld_as_float(In, base + i, in_dt));
+  {
+    float v = sc * ld_as_float(In, base + i, in_dt);
+    if (round_tf32) v = round_to_tf32(v);
+    st_from_float(Out, base + i, out_dt, v);
+  }
 }
 
 cudaError_t scale_launch(const void* In, int in_dt, void* Out, int out_dt, int batch, long long count,
-                         const float* scale, cudaStream_t st, long long* launches) {
+                         const float* scale, cudaStream_t st, long long* launches, int round_tf32) {
   const int nblk = (int)min((long long)1184, (count + 255) / 256);
-  scale_kernel<<<dim3(nblk, batch), 256, 0, st>>>(In, in_dt, Out, out_dt, count, scale);
+  scale_kernel<<<dim3(nblk, batch), 256, 0, st>>>(In, in_dt, Out, out_dt, count, scale, round_tf32);
   if (launches) ++*launches;
   return cudaGetLastError();
 }
@@ -552,7 +563,71 @@ extern "C" int defl_frobenius_norms_noalloc(const void* X, int dtype, int b, lon
   // every slot read by the second kernel is written by the first, so nothing needs clearing
   frob_partial_kernel<<<dim3(NOALLOC_NBLK, b), 256, 0, st>>>(X, dtype, count, NOALLOC_NBLK, scratch);
   if (cudaGetLastError() != cudaSuccess) return DEFL_ERR_CUDA;
-  rho_finalize_kernel<<<(b + 127) / 128, 128, 0, st>>>(scratch, NOALLOC_NBLK, b, norms, nullptr, nullptr, nullptr);
+  rho_finalize_kernel<<<(b + 3) / 4, 128, 0, st>>>(scratch, NOALLOC_NBLK, b, norms, nullptr, nullptr, nullptr);
   if (cudaGetLastError() != cudaSuccess) return DEFL_ERR_CUDA;
   return DEFL_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Split-precision copies of fp32 panels for the tensor engine: x = hi + lo with hi = bf16(x),
+// lo = bf16(x - hi) (about 16 significant bits together).
+// ---------------------------------------------------------------------------------------------
+namespace defl {
+
+// hi, lo [b, rows, lp] from In [b, rows, l] (leading dimension ld_in); columns l..lp-1 are zero.
+__global__ void split_panel_kernel(const float* __restrict__ In, long long in_bs, int ld_in, int rows, int l, int lp,
+                                   __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  const int bz = blockIdx.y;
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= (long long)rows * lp) return;
+  const int r = (int)(e / lp), c = (int)(e % lp);
+  const float x = (c < l) ? In[(long long)bz * in_bs + (long long)r * ld_in + c] : 0.f;
+  const __nv_bfloat16 h = __float2bfloat16_rn(x);
+  const long long o = (long long)bz * rows * lp + e;
+  hi[o] = h;
+  lo[o] = __float2bfloat16_rn(x - __bfloat162float(h));
+}
+
+cudaError_t split_panel_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int l, int lp,
+                               __nv_bfloat16* hi, __nv_bfloat16* lo, cudaStream_t st, long long* launches) {
+  const long long tot = (long long)rows * lp;
+  split_panel_kernel<<<dim3((unsigned)((tot + 255) / 256), batch), 256, 0, st>>>(In, in_bs, ld_in, rows, l, lp, hi, lo);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+// Out [b, rows, 3*kp] bf16 = three column blocks of the (optionally column-scaled) panel In [b, rows, k]:
+//   pattern 0: [hi | hi | lo]      pattern 1: [hi | lo | hi]
+// so that  Out0 * Out1^T = hi hi^T + hi lo^T + lo hi^T  (the product of the two fp32 panels up to the lo*lo term).
+// Column t is scaled by  c0 * s[b,t] * (inv_rho ? inv_rho[b] : 1) + c1  when s is given.
+__global__ void split_concat3_kernel(const float* __restrict__ In, long long in_bs, int ld_in, int rows, int k, int kp,
+                                     const float* __restrict__ s, int ld_s, const float* __restrict__ inv_rho, float c0,
+                                     float c1, int pattern, __nv_bfloat16* __restrict__ Out) {
+  const int bz = blockIdx.y;
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= (long long)rows * kp) return;
+  const int r = (int)(e / kp), t = (int)(e % kp);
+  float x = 0.f;
+  if (t < k) {
+    x = In[(long long)bz * in_bs + (long long)r * ld_in + t];
+    if (s) x *= c0 * s[(long long)bz * ld_s + t] * (inv_rho ? inv_rho[bz] : 1.f) + c1;
+  }
+  const __nv_bfloat16 h = __float2bfloat16_rn(x);
+  const __nv_bfloat16 lw = __float2bfloat16_rn(x - __bfloat162float(h));
+  __nv_bfloat16* o = Out + ((long long)bz * rows + r) * (3LL * kp);
+  o[t] = h;
+  o[kp + t] = pattern ? lw : h;
+  o[2 * kp + t] = pattern ? h : lw;
+}
+
+cudaError_t split_concat3_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int k, int kp,
+                                 const float* s, int ld_s, const float* inv_rho, float c0, float c1, int pattern,
+                                 __nv_bfloat16* Out, cudaStream_t st, long long* launches) {
+  const long long tot = (long long)rows * kp;
+  split_concat3_kernel<<<dim3((unsigned)((tot + 255) / 256), batch), 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s,
+                                                                                  inv_rho, c0, c1, pattern, Out);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace defl

@@ -7,8 +7,9 @@ namespace defl {
 constexpr int MAX_L = 64;   // widest panel (sketch width / PSD basis width)
 
 int gram_num_chunks(int rows);
+// partial Gram blocks of Y^T Y2 (Y2 = nullptr: Y^T Y)
 cudaError_t gram_partial_launch(const float* Y, long long batch_stride, int batch, int rows, int l, int ld,
-                                double* partial, cudaStream_t st, long long* launches);
+                                double* partial, cudaStream_t st, long long* launches, const float* Y2 = nullptr);
 cudaError_t chol_inv_launch(const double* partial, int nchunk, int batch, int l, float* Rinv, int* status,
                             cudaStream_t st, long long* launches);
 cudaError_t panel_apply_launch(const float* In, long long in_bs, int ld_in, const float* Mtx, int ldm, int batch,
@@ -24,9 +25,18 @@ cudaError_t scale_cols_launch(const float* In, long long in_bs, int ld_in, int b
                               int ld_s, const float* inv_rho, float c0, float c1, float* Out, long long out_bs,
                               int ld_out, cudaStream_t st, long long* launches);
 cudaError_t scale_launch(const void* In, int in_dt, void* Out, int out_dt, int batch, long long count,
-                         const float* scale, cudaStream_t st, long long* launches);
+                         const float* scale, cudaStream_t st, long long* launches, int round_tf32 = 0);
 cudaError_t fill_gaussian_launch(void* dst, long long count, int dtype, unsigned long long seed, long long per_stream,
                                  unsigned long long seed_stride, cudaStream_t st, long long* launches);
 cudaError_t fill_int_launch(int* p, int n, int v, cudaStream_t st, long long* launches);
 
+}  // namespace defl
+
+#include <cuda_bf16.h>
+namespace defl {
+cudaError_t split_panel_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int l, int lp,
+                               __nv_bfloat16* hi, __nv_bfloat16* lo, cudaStream_t st, long long* launches);
+cudaError_t split_concat3_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int k, int kp,
+                                 const float* s, int ld_s, const float* inv_rho, float c0, float c1, int pattern,
+                                 __nv_bfloat16* Out, cudaStream_t st, long long* launches);
 }  // namespace defl

@@ -1,12 +1,486 @@
-// Deflated PSD projection (Algorithm 2). Placeholder translation unit until the kernels land.
+// Deflated PSD projection (Algorithm 2) of one symmetric fp32 matrix, as kernel launches on one stream:
+//   block step Z~ = Z V, Rayleigh-Ritz on V^T Z~ (one-sided Jacobi core), Ritz vectors U = V E,
+//   R = Z - sum_I lambda_i u_i u_i^T, Lanczos upper estimate of ||R||_2 (App. D.1),
+//   X0 = R/theta + (1/gamma) sum_I sign(lambda_i) u_i u_i^T, the composite odd filter g (tf32 tensor
+//   cores, every product symmetric), P = (R + R g(X0))/2 + sum_{lambda_i > 0} lambda_i u_i u_i^T,
+//   P <- (P + P^T)/2, V <- CholeskyQR2(Z~).
+// The basis V is orthonormalised on entry, so a Gaussian start block is accepted.
 #include "../../include/defl.h"
+#include "common.cuh"
+#include "panel.cuh"
 #include "ctx.cuh"
 
+#include <cstdio>
+#include <cstring>
+
+using namespace defl;
+
+namespace defl {
+
+// ---------------------------------------------------------------------------------------------
+// y = A x for a dense row-major fp32 matrix: one warp per row, float4 loads, fixed-order reduction.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) symv_kernel(const float* __restrict__ A, const float* __restrict__ x,
+                                                   float* __restrict__ y, int n, const int* __restrict__ skip) {
+  if (skip && *skip) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const bool vec = (n & 3) == 0;
+  for (int r = blockIdx.x * 8 + warp; r < n; r += gridDim.x * 8) {
+    const float* row = A + (long long)r * n;
+    float acc = 0.f;
+    if (vec) {
+      const float4* r4 = reinterpret_cast<const float4*>(row);
+      const float4* x4 = reinterpret_cast<const float4*>(x);
+      for (int i = lane; i < n / 4; i += 32) {
+        const float4 a = r4[i], b = __ldg(&x4[i]);
+        acc = fmaf(a.x, b.x, acc); acc = fmaf(a.y, b.y, acc); acc = fmaf(a.z, b.z, acc); acc = fmaf(a.w, b.w, acc);
+      }
+    } else {
+      for (int i = lane; i < n; i += 32) acc = fmaf(row[i], __ldg(&x[i]), acc);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) y[r] = acc;
+  }
+}
+
+static cudaError_t symv_launch(const float* A, const float* x, float* y, int n, const int* skip, cudaStream_t st,
+                               long long* launches) {
+  int grid = (n + 7) / 8;
+  if (grid > 148 * 8) grid = 148 * 8;
+  symv_kernel<<<grid, 256, 0, st>>>(A, x, y, n, skip);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Lanczos on R^2 with full reorthogonalisation (App. D.1). One CTA does the vector work of a step:
+//   alpha_j = q_j . w;  w -= Q_j (Q_j^T w) twice;  beta_j = ||w||;  q_{j+1} = w / beta_j
+// State in device memory: Q[steps, n], T[steps, steps] (dense tridiagonal, fp64), done flag.
+// ---------------------------------------------------------------------------------------------
+struct LanczosState {
+  float* Q;        // [steps, n]
+  double* T;       // [steps, steps]
+  float* w;        // [n] work vector (R R q_j)
+  float* t;        // [n] work vector (R q_j)
+  int* done;       // set when the recurrence broke down (beta ~ 0); later steps become no-ops
+  double* beta_prev;
+};
+
+__device__ double block_sum(double v, double* red) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  double t = 0.0;
+  for (int i = 0; i < nw; ++i) t += red[i];
+  return t;
+}
+
+__global__ void __launch_bounds__(1024) lanczos_init_kernel(const float* __restrict__ v0, int n, int steps, LanczosState s) {
+  __shared__ double red[32];
+  double a = 0.0;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) a += (double)v0[i] * (double)v0[i];
+  const double nv = sqrt(block_sum(a, red));
+  for (int i = threadIdx.x; i < n; i += blockDim.x) s.Q[i] = (nv > 0.0) ? (float)((double)v0[i] / nv) : 0.f;
+  for (int i = threadIdx.x; i < steps * steps; i += blockDim.x) s.T[i] = 0.0;
+  if (threadIdx.x == 0) { *s.done = (nv > 0.0) ? 0 : 1; *s.beta_prev = 0.0; }
+}
+
+__global__ void __launch_bounds__(1024) lanczos_step_kernel(int j, int n, int steps, LanczosState s) {
+  __shared__ double red[32];
+  __shared__ double coef[DEFL_LANCZOS_STEPS];
+  if (*s.done) return;
+  const float* q = s.Q + (long long)j * n;
+  double a = 0.0;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) a += (double)q[i] * (double)s.w[i];
+  a = block_sum(a, red);
+  if (threadIdx.x == 0) s.T[j * steps + j] = a;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  for (int pass = 0; pass < 2; ++pass) {
+    // c = Q_j^T w, one warp per basis vector, then w -= Q_j c
+    for (int p = warp; p <= j; p += nw) {
+      const float* qp = s.Q + (long long)p * n;
+      double d = 0.0;
+      for (int i = lane; i < n; i += 32) d += (double)qp[i] * (double)s.w[i];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+      if (lane == 0) coef[p] = d;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+      double wi = (double)s.w[i];
+      for (int p = 0; p <= j; ++p) wi -= coef[p] * (double)s.Q[(long long)p * n + i];
+      s.w[i] = (float)wi;
+    }
+    __syncthreads();
+  }
+  double b = 0.0;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) b += (double)s.w[i] * (double)s.w[i];
+  b = sqrt(block_sum(b, red));
+  if (j + 1 == steps) return;
+  const double a0 = s.T[0];
+  if (!(b > 1e-12 * fabs(a0))) {
+    __syncthreads();
+    if (threadIdx.x == 0) *s.done = 1;
+    return;
+  }
+  if (threadIdx.x == 0) { s.T[j * steps + j + 1] = b; s.T[(j + 1) * steps + j] = b; }
+  float* qn = s.Q + (long long)(j + 1) * n;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) qn[i] = (float)((double)s.w[i] / b);
+}
+
+// v = sum_p E[p][0] q_p (the Ritz vector of the largest Ritz value); E is [steps, steps] row-major fp32
+__global__ void lanczos_ritz_kernel(int n, int steps, const float* __restrict__ Q, const float* __restrict__ E,
+                                    float* __restrict__ v) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  double a = 0.0;
+  for (int p = 0; p < steps; ++p) a += (double)E[p * steps] * (double)Q[(long long)p * n + i];
+  v[i] = (float)a;
+}
+
+// theta = sqrt(max(rho, 0) + ||w - rho v||), inv_theta = 1/theta (0 + status bit when theta is not a positive number)
+__global__ void __launch_bounds__(1024) lanczos_theta_kernel(int n, const float* __restrict__ rho_p,
+                                                             const float* __restrict__ v, const float* __restrict__ w,
+                                                             float* theta, float* inv_theta, int* status) {
+  __shared__ double red[32];
+  const double rho = (double)rho_p[0];
+  double a = 0.0;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const double d = (double)w[i] - rho * (double)v[i];
+    a += d * d;
+  }
+  a = sqrt(block_sum(a, red));
+  if (threadIdx.x == 0) {
+    const double th = sqrt((rho > 0.0 ? rho : 0.0) + a);
+    const bool ok = th > 0.0 && isfinite(th);
+    theta[0] = (float)th;
+    inv_theta[0] = ok ? (float)(1.0 / th) : 0.f;
+    if (!ok && status) atomicOr(status, 4);
+  }
+}
+
+// P <- (P + P^T)/2 in place, 32 x 32 tiles through shared memory; tile pair (bi <= bj) per CTA
+__global__ void __launch_bounds__(256) symmetrise_kernel(float* __restrict__ P, int n) {
+  __shared__ float ta[32][33], tb[32][33];
+  const int bi = blockIdx.y, bj = blockIdx.x;
+  if (bj < bi) return;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int r = ty; r < 32; r += 8) {
+    const int i = bi * 32 + r, j = bj * 32 + tx;
+    ta[r][tx] = (i < n && j < n) ? P[(long long)i * n + j] : 0.f;
+    const int i2 = bj * 32 + r, j2 = bi * 32 + tx;
+    tb[r][tx] = (i2 < n && j2 < n) ? P[(long long)i2 * n + j2] : 0.f;
+  }
+  __syncthreads();
+  for (int r = ty; r < 32; r += 8) {
+    const int i = bi * 32 + r, j = bj * 32 + tx;
+    if (i < n && j < n) P[(long long)i * n + j] = 0.5f * (ta[r][tx] + tb[tx][r]);
+    const int i2 = bj * 32 + r, j2 = bi * 32 + tx;
+    if (bi != bj && i2 < n && j2 < n) P[(long long)i2 * n + j2] = 0.5f * (tb[r][tx] + ta[tx][r]);
+  }
+}
+
+// hi = tf32(x) (round to nearest), lo = tf32(x - hi)
+__global__ void split_tf32_kernel(const float* __restrict__ X, float* __restrict__ hi, float* __restrict__ lo, long long count) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (long long)gridDim.x * blockDim.x) {
+    const float x = X[i];
+    const float h = round_to_tf32(x);
+    hi[i] = h;
+    lo[i] = round_to_tf32(x - h);
+  }
+}
+
+// out[t] = f(lam[t]) per column scale helpers: mode 0: lambda, 1: sign(lambda)/gamma, 2: max(lambda, 0); negated if neg
+__global__ void ritz_scale_kernel(const float* __restrict__ lam, int k, int mode, float gamma, int neg, float* __restrict__ out) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= k) return;
+  const float l = lam[t];
+  float v = l;
+  if (mode == 1) v = (l > 0.f ? 1.f : (l < 0.f ? -1.f : 0.f)) / gamma;
+  else if (mode == 2) v = l > 0.f ? l : 0.f;
+  out[t] = neg ? -v : v;
+}
+
+struct PsdWs {
+  float* R; float* Xa; float* Xb; float* W; float* Tt;   // [n,n]
+  float* Zt;        // [n,K]  Z V
+  float* Vo;        // [n,K]  orthonormalised incoming basis
+  float* U;         // [n,K]  Ritz vectors (leading k used)
+  float* Us;        // [n,K]  scaled copy
+  double* gram;     // [nchunk, K, K]
+  float* Rinv; float* E; float* Es; float* lam; float* coef;   // [K,K] x3, [K], [K]
+  float* Q; double* T; float* lw; float* lt; float* lv; float* lE; float* lrho;   // Lanczos state
+  int* done; double* beta_prev;
+  double* npart; float* theta; float* inv_theta; float* dummy;
+  int* status;
+  float* start;     // [n] generated Lanczos start vector
+  size_t bytes;
+};
+
+struct Carver2 {
+  char* base; size_t off;
+  explicit Carver2(void* p) : base(reinterpret_cast<char*>(p)), off(0) {}
+  template <typename T> T* take(size_t count) {
+    T* r = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off = align_up(off + count * sizeof(T), 256);
+    return r;
+  }
+};
+
+static PsdWs carve_psd(void* base, int n, int K) {
+  Carver2 cv(base);
+  PsdWs w;
+  const size_t nn = (size_t)n * n;
+  const int Ke = K > 0 ? K : 1;
+  const int S = DEFL_LANCZOS_STEPS;
+  w.R = cv.take<float>(nn); w.Xa = cv.take<float>(nn); w.Xb = cv.take<float>(nn);
+  w.W = cv.take<float>(nn); w.Tt = cv.take<float>(nn);
+  w.Zt = cv.take<float>((size_t)n * Ke); w.Vo = cv.take<float>((size_t)n * Ke);
+  w.U = cv.take<float>((size_t)n * Ke); w.Us = cv.take<float>((size_t)n * Ke);
+  w.gram = cv.take<double>((size_t)gram_num_chunks(n) * Ke * Ke);
+  w.Rinv = cv.take<float>((size_t)Ke * Ke); w.E = cv.take<float>((size_t)Ke * Ke); w.Es = cv.take<float>((size_t)Ke * Ke);
+  w.lam = cv.take<float>(Ke); w.coef = cv.take<float>(Ke);
+  w.Q = cv.take<float>((size_t)S * n); w.T = cv.take<double>(S * S);
+  w.lw = cv.take<float>(n); w.lt = cv.take<float>(n); w.lv = cv.take<float>(n);
+  w.lE = cv.take<float>(S * S); w.lrho = cv.take<float>(S);
+  w.done = cv.take<int>(1); w.beta_prev = cv.take<double>(1);
+  w.npart = cv.take<double>(1184);
+  w.theta = cv.take<float>(1); w.inv_theta = cv.take<float>(1); w.dummy = cv.take<float>(S * S);
+  w.status = cv.take<int>(1);
+  w.start = cv.take<float>(n);
+  w.bytes = cv.off;
+  return w;
+}
+
+// Scale estimate of the symmetric matrix A (n x n): theta, inv_theta in device memory.
+static int estimate_scale(defl_ctx* c, const float* A, int n, int norm_mode, const float* start, const PsdWs& w) {
+  if (norm_mode == DEFL_NORM_FROBENIUS) {
+    const int nblk = 296;
+    if (ctx_fail(c, frob_partial_launch(A, F32, 1, (long long)n * n, nblk, w.npart, c->stream, &c->launches), "frobenius"))
+      return DEFL_ERR_CUDA;
+    if (ctx_fail(c, rho_finalize_launch(w.npart, nblk, 1, w.theta, w.inv_theta, nullptr, w.status, c->stream, &c->launches), "theta"))
+      return DEFL_ERR_CUDA;
+    return DEFL_OK;
+  }
+  int steps = DEFL_LANCZOS_STEPS;
+  if (steps > n) steps = n;
+  LanczosState s;
+  s.Q = w.Q; s.T = w.T; s.w = w.lw; s.t = w.lt; s.done = w.done; s.beta_prev = w.beta_prev;
+  lanczos_init_kernel<<<1, 1024, 0, c->stream>>>(start, n, steps, s);
+  ++c->launches;
+  if (ctx_fail(c, cudaGetLastError(), "lanczos init")) return DEFL_ERR_CUDA;
+  for (int j = 0; j < steps; ++j) {
+    if (ctx_fail(c, symv_launch(A, w.Q + (size_t)j * n, w.lt, n, w.done, c->stream, &c->launches), "symv")) return DEFL_ERR_CUDA;
+    if (ctx_fail(c, symv_launch(A, w.lt, w.lw, n, w.done, c->stream, &c->launches), "symv")) return DEFL_ERR_CUDA;
+    lanczos_step_kernel<<<1, 1024, 0, c->stream>>>(j, n, steps, s);
+    ++c->launches;
+    if (ctx_fail(c, cudaGetLastError(), "lanczos step")) return DEFL_ERR_CUDA;
+  }
+  // largest Ritz pair of the (zero-padded) tridiagonal matrix through the Jacobi core
+  if (ctx_fail(c, jacobi_eig_launch(w.T, 1, 1, steps, 1, w.lrho, w.lE, nullptr, w.status, c->stream, &c->launches), "ritz"))
+    return DEFL_ERR_CUDA;
+  lanczos_ritz_kernel<<<(n + 255) / 256, 256, 0, c->stream>>>(n, steps, w.Q, w.lE, w.lv);
+  ++c->launches;
+  if (ctx_fail(c, cudaGetLastError(), "ritz vector")) return DEFL_ERR_CUDA;
+  if (ctx_fail(c, symv_launch(A, w.lv, w.lt, n, nullptr, c->stream, &c->launches), "symv")) return DEFL_ERR_CUDA;
+  if (ctx_fail(c, symv_launch(A, w.lt, w.lw, n, nullptr, c->stream, &c->launches), "symv")) return DEFL_ERR_CUDA;
+  lanczos_theta_kernel<<<1, 1024, 0, c->stream>>>(n, w.lrho, w.lv, w.lw, w.theta, w.inv_theta, w.status);
+  ++c->launches;
+  if (ctx_fail(c, cudaGetLastError(), "theta")) return DEFL_ERR_CUDA;
+  return DEFL_OK;
+}
+
+// C = aux_scale * aux + alpha * U diag(coef) U^T  (rank-k symmetric update, exact fp32 products)
+static int rank_update(defl_ctx* c, const PsdWs& w, int n, int K, int k, int coef_mode, float gamma, int neg,
+                       const float* aux, float aux_scale, const float* aux_scale_dev, float* C, int round_tf32 = 0) {
+  ritz_scale_kernel<<<1, 64, 0, c->stream>>>(w.lam, k, coef_mode, gamma, neg, w.coef);
+  ++c->launches;
+  if (ctx_fail(c, cudaGetLastError(), "ritz scale")) return DEFL_ERR_CUDA;
+  if (ctx_fail(c, scale_cols_launch(w.U, 0, K, 1, n, k, w.coef, K, nullptr, 1.f, 0.f, w.Us, 0, K, c->stream, &c->launches), "U diag"))
+    return DEFL_ERR_CUDA;
+  GemmDesc g = gemm_desc_zero();
+  g.batch = 1; g.M = n; g.N = n; g.K[0] = k;
+  g.A[0] = w.U; g.sa_i[0] = K; g.sa_k[0] = 1; g.in_dtype = F32;
+  g.B[0] = w.Us; g.sb_k[0] = 1; g.sb_j[0] = K; g.b_dtype = F32;
+  g.aux = aux; g.ld_aux = n; g.aux_dtype = F32;
+  g.C = C; g.ldc = n; g.out_dtype = F32;
+  g.epilogue = EPI_AUX_PLUS; g.aux_scale = aux_scale; g.aux_scale_dev = aux_scale_dev; g.alpha = 1.f;
+  g.round_tf32 = round_tf32;
+  return run_gemm(c, g, DEFL_ENGINE_SIMT, "rank-k update");
+}
+
+}  // namespace defl
+
 extern "C" {
-size_t defl_psd_workspace_bytes(int n, int K) { (void)n; (void)K; return 0; }
-int defl_psd_project(defl_ctx* ctx, const void* X, void* P, int n, int k, float* warm_basis, int K,
+
+size_t defl_psd_workspace_bytes(int n, int K) {
+  if (n <= 0 || K < 0) return 0;
+  return carve_psd(nullptr, n, K).bytes;
+}
+
+int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float* warm_basis, int K,
                      const float* coeff_schedule, int T, const defl_opts* opts, const defl_info* info) {
-  (void)ctx; (void)X; (void)P; (void)n; (void)k; (void)warm_basis; (void)K; (void)coeff_schedule; (void)T; (void)opts; (void)info;
-  return DEFL_ERR_UNSUPPORTED;
+  if (!c || !Xv || !Pv || n <= 0 || k < 0 || K < 0 || T < 0) return DEFL_ERR_ARG;
+  if (K > 0 && !warm_basis) return DEFL_ERR_ARG;
+  if (T > 0 && !coeff_schedule) return DEFL_ERR_ARG;
+  if (k > K || K > DEFL_MAX_L || K >= n || T > DEFL_MAX_STEPS) return DEFL_ERR_RANK;
+  const float* Z = reinterpret_cast<const float*>(Xv);
+  float* P = reinterpret_cast<float*>(Pv);
+  {
+    const char* z0 = reinterpret_cast<const char*>(Xv);
+    const char* p0 = reinterpret_cast<const char*>(Pv);
+    const size_t bytes = (size_t)n * n * sizeof(float);
+    if (z0 < p0 + bytes && p0 < z0 + bytes) return DEFL_ERR_ARG;
+  }
+  const int norm_mode = opts ? opts->norm_mode : DEFL_NORM_LANCZOS;
+  if (norm_mode != DEFL_NORM_LANCZOS && norm_mode != DEFL_NORM_FROBENIUS) return DEFL_ERR_ARG;
+  const float gamma = (opts && opts->gamma > 0.f) ? opts->gamma : 1.1f;
+  const int engine_opt = opts ? opts->engine : DEFL_ENGINE_AUTO;
+  if (engine_opt < 0 || engine_opt > 2) return DEFL_ERR_ARG;
+  // the filter products run on the tensor cores (tf32) unless the fp32 engine is requested
+  const int engine = (engine_opt == DEFL_ENGINE_SIMT) ? DEFL_ENGINE_SIMT : DEFL_ENGINE_TENSOR;
+  const int sym = (opts && opts->exploit_symmetry) ? 1 : 0;
+  const bool deflate = (k > 0) && !(opts && opts->warmup);
+  // iterates that feed tf32 products are stored already rounded to nearest tf32: the tensor core would
+  // otherwise truncate them, which biases every product towards zero
+  const int tf32_round = (engine == DEFL_ENGINE_TENSOR) ? 1 : 0;
+
+  cudaSetDevice(c->device);
+  int rc = ctx_reserve(c, carve_psd(nullptr, n, K).bytes);
+  if (rc) return rc;
+  PsdWs w = carve_psd(c->ws, n, K);
+  c->n_marks = 0;
+  c->err[0] = 0;
+  ctx_stage_mark(c);
+  if (ctx_fail(c, fill_int_launch(w.status, 1, 0, c->stream, &c->launches), "status")) return DEFL_ERR_CUDA;
+
+  // ---- stage 0: block step and Rayleigh-Ritz (lines 1-2) -------------------------------------------
+  if (K > 0) {
+    if (ctx_fail(c, cudaMemcpyAsync(w.Vo, warm_basis, (size_t)n * K * sizeof(float), cudaMemcpyDeviceToDevice, c->stream), "copy V"))
+      return DEFL_ERR_CUDA;
+    if ((rc = orthonormalise(c, w.Vo, 1, n, K, w.gram, w.Rinv, w.status))) return rc;
+    GemmDesc g = gemm_desc_zero();
+    g.batch = 1; g.M = n; g.N = K; g.K[0] = n;
+    g.A[0] = Z; g.sa_i[0] = n; g.sa_k[0] = 1; g.in_dtype = F32;
+    g.B[0] = w.Vo; g.sb_k[0] = K; g.sb_j[0] = 1; g.b_dtype = F32;
+    g.C = w.Zt; g.ldc = K; g.out_dtype = F32; g.epilogue = EPI_STORE;
+    if ((rc = run_gemm(c, g, DEFL_ENGINE_SIMT, "Z V"))) return rc;
+    // H = V^T Z~ (symmetrised inside the eigensolver), H = E diag(lambda) E^T, sorted by |lambda|
+    if (ctx_fail(c, gram_partial_launch(w.Vo, 0, 1, n, K, K, w.gram, c->stream, &c->launches, w.Zt), "V^T Z V")) return DEFL_ERR_CUDA;
+    if (ctx_fail(c, jacobi_eig_launch(w.gram, gram_num_chunks(n), 1, K, 1, w.lam, w.E, nullptr, w.status, c->stream, &c->launches), "ritz"))
+      return DEFL_ERR_CUDA;
+    if (ctx_fail(c, panel_apply_launch(w.Vo, 0, K, w.E, K, 1, n, K, K, w.U, 0, K, c->stream, &c->launches), "U = V E"))
+      return DEFL_ERR_CUDA;
+  }
+  ctx_stage_mark(c);
+
+  // ---- stage 1: R = Z - sum_I lambda_i u_i u_i^T (line 5) -------------------------------------------
+  const float* Rm = Z;
+  if (deflate) {
+    if ((rc = rank_update(c, w, n, K, k, 0, gamma, 1, Z, 1.f, nullptr, w.R))) return rc;
+    Rm = w.R;
+  }
+  ctx_stage_mark(c);
+
+  // ---- stage 2: scale (line 6 / line 9) --------------------------------------------------------------
+  const float* start = (opts && opts->lanczos_start) ? opts->lanczos_start : w.start;
+  if (norm_mode == DEFL_NORM_LANCZOS && !(opts && opts->lanczos_start)) {
+    if (ctx_fail(c, fill_gaussian_launch(w.start, n, F32, opts ? opts->seed : 0ull, 0, 0ull, c->stream, &c->launches), "start vector"))
+      return DEFL_ERR_CUDA;
+  }
+  if ((rc = estimate_scale(c, Rm, n, norm_mode, start, w))) return rc;
+  ctx_stage_mark(c);
+
+  // ---- stage 3: X0 = R/theta + (1/gamma) sum_I sign(lambda_i) u_i u_i^T (line 7) ---------------------
+  float* bufs[2] = {w.Xa, w.Xb};
+  int cur = 0;
+  if (deflate) {
+    if ((rc = rank_update(c, w, n, K, k, 1, gamma, 0, Rm, 1.f, w.inv_theta, bufs[cur], tf32_round))) return rc;
+  } else {
+    if (ctx_fail(c, scale_launch(Rm, F32, bufs[cur], F32, 1, (long long)n * n, w.inv_theta, c->stream, &c->launches, tf32_round), "normalise"))
+      return DEFL_ERR_CUDA;
+  }
+  ctx_stage_mark(c);
+
+  // ---- stage 4: g = p_T o ... o p_1 on the symmetric X0: W = X^2, Tt = a I + b W + c W^2, X <- X Tt ------
+  for (int t = 0; t < T; ++t) {
+    const float ca = coeff_schedule[3 * t], cb = coeff_schedule[3 * t + 1], cc = coeff_schedule[3 * t + 2];
+    const float* X = bufs[cur];
+    float* Xn = bufs[cur ^ 1];
+    GemmDesc g = gemm_desc_zero();
+    g.batch = 1; g.in_dtype = F32; g.b_dtype = F32; g.out_dtype = F32;
+    g.M = n; g.N = n; g.K[0] = n;
+    g.A[0] = X; g.sa_i[0] = n; g.sa_k[0] = 1;
+    g.B[0] = X; g.sb_k[0] = 1; g.sb_j[0] = n;          // X symmetric: rows as columns
+    g.C = w.W; g.ldc = n; g.epilogue = EPI_STORE; g.symmetric = sym; g.round_tf32 = tf32_round;
+    if ((rc = run_gemm(c, g, gemm_tc_supported(g) ? engine : DEFL_ENGINE_SIMT, "X^2"))) return rc;
+    g.A[0] = w.W; g.B[0] = w.W; g.C = w.Tt;
+    g.aux = w.W; g.ld_aux = n; g.aux_dtype = F32;
+    g.epilogue = EPI_POLY; g.pa = ca; g.pb = cb; g.pc = cc;
+    if ((rc = run_gemm(c, g, gemm_tc_supported(g) ? engine : DEFL_ENGINE_SIMT, "polynomial"))) return rc;
+    g.A[0] = X; g.B[0] = w.Tt; g.C = Xn; g.aux = nullptr;
+    g.epilogue = EPI_STORE; g.symmetric = 0;            // X Tt is symmetric only up to rounding: compute all of it
+    if ((rc = run_gemm(c, g, gemm_tc_supported(g) ? engine : DEFL_ENGINE_SIMT, "apply"))) return rc;
+    cur ^= 1;
+  }
+  ctx_stage_mark(c);
+
+  // ---- stage 5: P = (R + R g(X0))/2 + sum_{lambda_i > 0} lambda_i u_i u_i^T, symmetrised (lines 8, 12) ----
+  {
+    GemmDesc g = gemm_desc_zero();
+    g.batch = 1; g.in_dtype = F32; g.b_dtype = F32; g.out_dtype = F32;
+    g.M = n; g.N = n; g.K[0] = n;
+    g.A[0] = Rm; g.sa_i[0] = n; g.sa_k[0] = 1;
+    g.B[0] = bufs[cur]; g.sb_k[0] = 1; g.sb_j[0] = n;   // g(X0) symmetric up to rounding
+    if (tf32_round && gemm_tc_supported(g)) {
+      // R carries the large entries of this product: feed it as two tf32 terms R = R_hi + R_lo (two K
+      // segments against the same g) so that the tensor core does not truncate it
+      split_tf32_kernel<<<1184, 256, 0, c->stream>>>(Rm, w.W, w.Tt, (long long)n * n);
+      ++c->launches;
+      if (ctx_fail(c, cudaGetLastError(), "split R")) return DEFL_ERR_CUDA;
+      g.nseg = 2; g.K[1] = n;
+      g.A[0] = w.W; g.A[1] = w.Tt; g.sa_i[1] = n; g.sa_k[1] = 1;
+      g.B[1] = bufs[cur]; g.sb_k[1] = 1; g.sb_j[1] = n;
+    }
+    g.aux = Rm; g.ld_aux = n; g.aux_dtype = F32;
+    g.C = P; g.ldc = n;
+    g.epilogue = EPI_AUX_PLUS; g.aux_scale = 0.5f; g.alpha = 0.5f;
+    if ((rc = run_gemm(c, g, gemm_tc_supported(g) ? engine : DEFL_ENGINE_SIMT, "R g(X0)"))) return rc;
+    if (deflate) {
+      if ((rc = rank_update(c, w, n, K, k, 2, gamma, 0, P, 1.f, nullptr, P))) return rc;
+    }
+    symmetrise_kernel<<<dim3((n + 31) / 32, (n + 31) / 32), 256, 0, c->stream>>>(P, n);
+    ++c->launches;
+    if (ctx_fail(c, cudaGetLastError(), "symmetrise")) return DEFL_ERR_CUDA;
+  }
+  ctx_stage_mark(c);
+
+  // ---- stage 6: V <- CholeskyQR(Z~) (line 11) ----------------------------------------------------------
+  if (K > 0) {
+    if ((rc = orthonormalise(c, w.Zt, 1, n, K, w.gram, w.Rinv, w.status))) return rc;
+    if (ctx_fail(c, cudaMemcpyAsync(warm_basis, w.Zt, (size_t)n * K * sizeof(float), cudaMemcpyDeviceToDevice, c->stream), "copy V"))
+      return DEFL_ERR_CUDA;
+  }
+  ctx_stage_mark(c);
+
+  if (info) {
+    if (info->s && K > 0 &&
+        ctx_fail(c, cudaMemcpyAsync(info->s, w.lam, (size_t)K * sizeof(float), cudaMemcpyDeviceToDevice, c->stream), "copy lambda"))
+      return DEFL_ERR_CUDA;
+    if (info->rho &&
+        ctx_fail(c, cudaMemcpyAsync(info->rho, w.theta, sizeof(float), cudaMemcpyDeviceToDevice, c->stream), "copy theta"))
+      return DEFL_ERR_CUDA;
+    if (info->status) {
+      if (ctx_fail(c, or_status_launch(w.status, 1, c->wait_status, c->stream, &c->launches), "status")) return DEFL_ERR_CUDA;
+      if (ctx_fail(c, cudaMemcpyAsync(info->status, w.status, sizeof(int), cudaMemcpyDeviceToDevice, c->stream), "copy status"))
+        return DEFL_ERR_CUDA;
+    }
+  }
+  return DEFL_OK;
 }
-}
+
+}  // extern "C"

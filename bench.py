@@ -47,6 +47,26 @@ def flops_per_matrix(m, n, k, p, J, L):
     return filt, rsvd + defl
 
 
+# Average DRAM bytes per filter-product launch (dram__bytes_read + dram__bytes_write from the ncu capture
+# summarised in profiles/gemm_tc_kernel_filter_gpt2_xl_batch8.md, 8 matrices per group, scaled by 48/8).
+FILTER_TRAFFIC_BYTES_PER_LAUNCH = 1131e6
+
+
+def max_over_ranks(value, dist=None, device="cpu"):
+    """Largest `value` over all ranks (a time: the job is as slow as its slowest rank)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(units_per_rank, world, ms_max):
+    """Whole-job rate when every rank processes `units_per_rank` in `ms_max` milliseconds (weak scaling)."""
+    return world * units_per_rank / (ms_max * 1e-3)
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -210,11 +230,7 @@ def main():
             ev[i + 1].record()
         barrier()
     launches = ctx.defl_launch_count() - launches0
-    total_ms = ev[0].elapsed_time(ev[-1])
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(ev[0].elapsed_time(ev[-1]), dist, "cuda")
     ms_per_step = total_ms / args.steps
 
     # stage split of one more (untimed) step, with the same events the library records on its stream
@@ -251,13 +267,9 @@ def main():
         for _ in range(n_e2e):
             e2e_step()
         torch.cuda.synchronize()
-        e2e_ms = (time.perf_counter() - t0) * 1e3 / n_e2e
-        if dist is not None:
-            t = torch.tensor([e2e_ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3 / n_e2e, dist, "cuda")
         nbytes = sum(h.numel() * h.element_size() for h in hG)
-        e2e = {"value": world * tot_f / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+        e2e = {"value": aggregate_throughput(tot_f, world, e2e_ms) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes}
 
     if rank != 0:
@@ -265,7 +277,7 @@ def main():
             dist.destroy_process_group()
         return
     peaks, peaks_kind = load_peaks()
-    value = world * tot_f / (ms_per_step * 1e-3) / 1e12
+    value = aggregate_throughput(tot_f, world, ms_per_step) / 1e12
     filt_ms = stage_tot[2]
     n_filter_launches = 3 * wl["L"] * len(groups)
     ach = filt_flops / (filt_ms * 1e-3) / 1e12 if filt_ms > 0 else None
@@ -275,7 +287,9 @@ def main():
                 "peak_kind": "bf16_tflops_sustained, of %s" % peaks_kind,
                 "frac_of_burst": (ach / float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))) if ach else None,
                 "launches_per_step": n_filter_launches, "avg_launch_ms": filt_ms / n_filter_launches,
-                "flops_per_launch_avg": filt_flops / n_filter_launches, "traffic": None}
+                "flops_per_launch_avg": filt_flops / n_filter_launches,
+                "traffic": FILTER_TRAFFIC_BYTES_PER_LAUNCH if (wl_name == "gpt2_xl" and args.batch == 0) else None,
+                "traffic_unit": "bytes per launch (ncu, 8-matrix capture scaled to the batch)"}
     line = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,

@@ -128,10 +128,27 @@ def make_inputs(wl, device):
     return groups
 
 
-def run_step(ctx, wl, groups):
-    for g in groups:
-        ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"], sketch=g["Om"],
-                               gamma=1.01)
+def run_step(ctx, wl, groups, lanes=None):
+    """One step = every shape group through defl_polar_batched. With `lanes` (one (context, stream) pair per
+    group) the independent groups are enqueued on their own streams, forked from and joined to the current
+    stream, so that the small latency-bound kernels of one group overlap the other group's work."""
+    import torch
+    if not lanes:
+        for g in groups:
+            ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"],
+                                   sketch=g["Om"], gamma=1.01)
+        return
+    main = torch.cuda.current_stream()
+    fork = torch.cuda.Event()
+    fork.record(main)
+    for g, (c, s) in zip(groups, lanes):
+        s.wait_event(fork)
+        with torch.cuda.stream(s):
+            c.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"],
+                                 sketch=g["Om"], gamma=1.01)
+            done = torch.cuda.Event()
+            done.record(s)
+        main.wait_event(done)
 
 
 def oracle_sample(wl, seconds_hint=20.0):
@@ -160,6 +177,7 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--small", action="store_true", help="tiny workload for a quick functional check")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--streams", type=int, default=2, help="2: one stream + context per shape group; 1: one stream")
     ap.add_argument("--batch", type=int, default=0, help="override the matrices per shape group (profiling captures)")
     args = ap.parse_args()
     wl_name = "small" if args.small else "gpt2_xl"
@@ -213,23 +231,27 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    lanes = None
+    if args.streams > 1:
+        lanes = [(binding.Context(local_rank), torch.cuda.Stream()) for _ in groups]
+    config["streams"] = len(lanes) if lanes else 1
+
+    def launch_total():
+        return ctx.defl_launch_count() + (sum(c.defl_launch_count() for c, _ in lanes) if lanes else 0)
+
     for _ in range(max(args.warmup, 3)):
-        run_step(ctx, wl, groups)
+        run_step(ctx, wl, groups, lanes)
     barrier()
-    launches0 = ctx.defl_launch_count()
+    launches0 = launch_total()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    stage_ms = []
     with ClockSampler(local_rank) as clk:
         barrier()
         ev[0].record()
         for i in range(args.steps):
-            for g in groups:
-                ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"],
-                                       sketch=g["Om"], gamma=1.01)
-                stage_ms.append(None)      # filled after the timed region (events are already recorded)
+            run_step(ctx, wl, groups, lanes)
             ev[i + 1].record()
         barrier()
-    launches = ctx.defl_launch_count() - launches0
+    launches = launch_total() - launches0
     total_ms = max_over_ranks(ev[0].elapsed_time(ev[-1]), dist, "cuda")
     ms_per_step = total_ms / args.steps
 

@@ -142,17 +142,28 @@ PolarWs carve_polar(void* base, int b, int m, int n, int dtype, int k, int l) {
 }
 
 // CholeskyQR2 of the panel P[b, rows, l] in place: twice { W = P^T P; W = R^T R; P <- P R^-1 }.
-int orthonormalise(defl_ctx* c, float* P, int b, int rows, int l, double* gram, float* Rinv, int* status) {
-  const int nchunk = gram_num_chunks(rows);
-  for (int pass = 0; pass < 2; ++pass) {
-    if (ctx_fail(c, gram_partial_launch(P, (long long)rows * l, b, rows, l, l, gram, c->stream, &c->launches), "gram"))
+int orthonormalise(defl_ctx* c, float* P, int b, int rows, int l, double* gram, float* Rinv, int* status,
+                   __nv_bfloat16* hi, __nv_bfloat16* lo, int lp, int passes) {
+  // CholeskyQR: Gram(P); R = chol; P <- P R^-1. With passes = 2 (CholeskyQR2) the second Gram is taken in the
+  // same panel pass as the first solve. The last pass can also write P as bf16 hi + lo for the next
+  // tensor-core product.
+  const int nchunk = fused_num_chunks(rows);
+  const long long bs = (long long)rows * l;
+  if (ctx_fail(c, panel_fused_launch(P, bs, l, b, rows, l, nullptr, 0, l, nullptr, 0, 0, nullptr, nullptr, 0, gram,
+                                     c->stream, &c->launches), "gram"))
+    return DEFL_ERR_CUDA;
+  if (ctx_fail(c, chol_inv_launch(gram, nchunk, b, l, Rinv, status, c->stream, &c->launches), "cholesky"))
+    return DEFL_ERR_CUDA;
+  if (passes >= 2) {
+    if (ctx_fail(c, panel_fused_launch(P, bs, l, b, rows, l, Rinv, l, l, P, bs, l, nullptr, nullptr, 0, gram, c->stream,
+                                       &c->launches), "apply + gram"))
       return DEFL_ERR_CUDA;
     if (ctx_fail(c, chol_inv_launch(gram, nchunk, b, l, Rinv, status, c->stream, &c->launches), "cholesky"))
       return DEFL_ERR_CUDA;
-    if (ctx_fail(c, panel_apply_launch(P, (long long)rows * l, l, Rinv, l, b, rows, l, l, P, (long long)rows * l, l,
-                                       c->stream, &c->launches), "panel apply"))
-      return DEFL_ERR_CUDA;
   }
+  if (ctx_fail(c, panel_fused_launch(P, bs, l, b, rows, l, Rinv, l, l, P, bs, l, hi, lo, lp, nullptr, c->stream,
+                                     &c->launches), "apply"))
+    return DEFL_ERR_CUDA;
   return DEFL_OK;
 }
 
@@ -169,7 +180,7 @@ int run_brsvd(defl_ctx* c, const void* G, int b, int m, int n, int dtype, int l,
   // same G tile and accumulated in fp32 (G is bf16 already). Falls back to the fp32 engine when the shape or
   // type does not fit (fp32 storage, strides not multiples of 16 bytes) or when that engine is requested.
   const int lp = round_up8(l);
-  auto mul_G = [&](bool transposed, const float* Bp, float* Cp) {   // C = A B (ml x l) or A^T B (ms x l)
+  auto mul_G = [&](bool transposed, const float* Bp, float* Cp, bool presplit) {   // C = A B (ml x l) or A^T B (ms x l)
     const int M = transposed ? ms : ml, K = transposed ? ml : ms;
     GemmDesc g = gemm_desc_zero();
     g.batch = b; g.M = M; g.N = l; g.K[0] = K;
@@ -184,7 +195,8 @@ int run_brsvd(defl_ctx* c, const void* G, int b, int m, int n, int dtype, int l,
       t.B[0] = hi; t.B[1] = lo; t.b_split = 2; t.b_dtype = BF16;
       t.sb_k[0] = lp; t.sb_j[0] = 1; t.batch_b[0] = (long long)K * lp;
       if (gemm_tc_supported(t)) {
-        if (ctx_fail(c, split_panel_launch(Bp, (long long)K * l, l, b, K, l, lp, hi, lo, c->stream, &c->launches), "split panel"))
+        if (!presplit &&
+            ctx_fail(c, split_panel_launch(Bp, (long long)K * l, l, b, K, l, lp, hi, lo, c->stream, &c->launches), "split panel"))
           return (int)DEFL_ERR_CUDA;
         return run_gemm(c, t, DEFL_ENGINE_TENSOR, "G*panel (tensor)");
       }
@@ -192,30 +204,44 @@ int run_brsvd(defl_ctx* c, const void* G, int b, int m, int n, int dtype, int l,
     g.B[0] = Bp; g.sb_k[0] = l; g.sb_j[0] = 1; g.batch_b[0] = (long long)K * l; g.b_dtype = F32;
     return run_gemm(c, g, DEFL_ENGINE_SIMT, "G*panel");
   };
-  auto mul_A = [&](const float* Bp, float* Cp) { return mul_G(false, Bp, Cp); };
-  auto mul_At = [&](const float* Bp, float* Cp) { return mul_G(true, Bp, Cp); };
-  if ((rc = mul_A(sketch, w.Lp))) return rc;                               // Y = A Omega
-  if ((rc = orthonormalise(c, w.Lp, b, ml, l, w.gram, w.Rinv, w.status))) return rc;    // Q
+  // after an orthonormalisation the panel's bf16 split already exists (written by its last pass)
+  const bool split_out = (dtype == BF16 && engine != DEFL_ENGINE_SIMT);
+  auto mul_A = [&](const float* Bp, float* Cp, bool presplit) { return mul_G(false, Bp, Cp, presplit); };
+  auto mul_At = [&](const float* Bp, float* Cp, bool presplit) { return mul_G(true, Bp, Cp, presplit); };
+  // The basis that defines B = Q^T A gets CholeskyQR2; the intermediate bases of the subspace iteration only
+  // need to stay well conditioned, so one CholeskyQR pass (as Algorithm 3 prints it) is enough there: any
+  // basis of the same span gives the same triplets.
+  auto orth_long = [&](int passes) {
+    return orthonormalise(c, w.Lp, b, ml, l, w.gram, w.Rinv, w.status, split_out ? w.Lhi : nullptr,
+                          split_out ? w.Llo : nullptr, lp, passes);
+  };
+  auto orth_short = [&](int passes) {
+    return orthonormalise(c, w.Sp, b, ms, l, w.gram, w.Rinv, w.status, split_out ? w.Shi : nullptr,
+                          split_out ? w.Slo : nullptr, lp, passes);
+  };
+  if ((rc = mul_A(sketch, w.Lp, false))) return rc;                        // Y = A Omega
+  if ((rc = orth_long(J == 0 ? 2 : 1))) return rc;                          // Q
   for (int j = 0; j < J; ++j) {
-    if ((rc = mul_At(w.Lp, w.Sp))) return rc;                              // A^T Q
-    if ((rc = orthonormalise(c, w.Sp, b, ms, l, w.gram, w.Rinv, w.status))) return rc;
-    if ((rc = mul_A(w.Sp, w.Lp))) return rc;                               // A Y
-    if ((rc = orthonormalise(c, w.Lp, b, ml, l, w.gram, w.Rinv, w.status))) return rc;
+    if ((rc = mul_At(w.Lp, w.Sp, split_out))) return rc;                   // A^T Q
+    if ((rc = orth_short(1))) return rc;
+    if ((rc = mul_A(w.Sp, w.Lp, split_out))) return rc;                    // A Y
+    if ((rc = orth_long(j + 1 == J ? 2 : 1))) return rc;
   }
-  if ((rc = mul_At(w.Lp, w.Sp))) return rc;                                // (Q^T A)^T, [ms, l]
+  if ((rc = mul_At(w.Lp, w.Sp, split_out))) return rc;                     // (Q^T A)^T, [ms, l]
   // thin SVD of Q^T A through the Gram core: (Q^T A)(Q^T A)^T = E diag(s^2) E^T
-  if (ctx_fail(c, gram_partial_launch(w.Sp, (long long)ms * l, b, ms, l, l, w.gram, c->stream, &c->launches), "gram core"))
+  if (ctx_fail(c, panel_fused_launch(w.Sp, (long long)ms * l, l, b, ms, l, nullptr, 0, l, nullptr, 0, 0, nullptr, nullptr, 0,
+                                     w.gram, c->stream, &c->launches), "gram core"))
     return DEFL_ERR_CUDA;
-  if (ctx_fail(c, jacobi_eig_launch(w.gram, gram_num_chunks(ms), b, l, 0, w.sv, w.E, w.Es, w.status, c->stream,
+  if (ctx_fail(c, jacobi_eig_launch(w.gram, fused_num_chunks(ms), b, l, 0, w.sv, w.E, w.Es, w.status, c->stream,
                                     &c->launches), "jacobi"))
     return DEFL_ERR_CUDA;
   if (k_keep > 0) {
     // U = Q E (long side), V = (Q^T A)^T E diag(1/s) (short side); keep the leading k_keep columns
-    if (ctx_fail(c, panel_apply_launch(w.Lp, (long long)ml * l, l, w.E, l, b, ml, l, k_keep, w.Uk, (long long)ml * k_keep,
-                                       k_keep, c->stream, &c->launches), "U = Q E"))
+    if (ctx_fail(c, panel_fused_launch(w.Lp, (long long)ml * l, l, b, ml, l, w.E, l, k_keep, w.Uk, (long long)ml * k_keep,
+                                       k_keep, nullptr, nullptr, 0, nullptr, c->stream, &c->launches), "U = Q E"))
       return DEFL_ERR_CUDA;
-    if (ctx_fail(c, panel_apply_launch(w.Sp, (long long)ms * l, l, w.Es, l, b, ms, l, k_keep, w.Vk, (long long)ms * k_keep,
-                                       k_keep, c->stream, &c->launches), "V = B^T E / s"))
+    if (ctx_fail(c, panel_fused_launch(w.Sp, (long long)ms * l, l, b, ms, l, w.Es, l, k_keep, w.Vk, (long long)ms * k_keep,
+                                       k_keep, nullptr, nullptr, 0, nullptr, c->stream, &c->launches), "V = B^T E / s"))
       return DEFL_ERR_CUDA;
   }
   return DEFL_OK;

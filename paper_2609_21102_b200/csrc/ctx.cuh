@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include "common.cuh"
+#include <cuda_bf16.h>
 
 #define DEFL_MAX_MARKS 12
 
@@ -29,6 +30,7 @@ int ctx_reserve(defl_ctx* c, size_t bytes);
 void ctx_stage_mark(defl_ctx* c);
 int run_gemm(defl_ctx* c, const GemmDesc& g, int engine, const char* what);
 int partials_per_batch(const GemmDesc& g, int engine);
-int orthonormalise(defl_ctx* c, float* P, int b, int rows, int l, double* gram, float* Rinv, int* status);
+int orthonormalise(defl_ctx* c, float* P, int b, int rows, int l, double* gram, float* Rinv, int* status,
+                   __nv_bfloat16* hi = nullptr, __nv_bfloat16* lo = nullptr, int lp = 0, int passes = 2);
 cudaError_t or_status_launch(int* status, int n, const int* word, cudaStream_t st, long long* launches);
 }  // namespace defl

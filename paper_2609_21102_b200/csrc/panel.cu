@@ -89,16 +89,18 @@ cudaError_t gram_partial_launch(const float* Y, long long batch_stride, int batc
 // (upper triangular, fp32, row-major [l,l]). A non-positive pivot restarts with W + shift I and
 // sets DEFL_ST_CHOL_SHIFT (bit 1) in status[b].
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) chol_inv_kernel(const double* __restrict__ partial, int nchunk, int l,
+__global__ void __launch_bounds__(512) chol_inv_kernel(const double* __restrict__ partial, int nchunk, int l,
                                                        float* __restrict__ Rinv, int* __restrict__ status) {
   extern __shared__ double sm[];
   double* W = sm;              // [l][l] original Gram
   double* Lm = sm + l * l;     // [l][l] lower factor, then its inverse
   __shared__ int bad;
+  __shared__ double rdiag[MAX_L];
   const int bz = blockIdx.x, tid = threadIdx.x;
   const double* pb = partial + (long long)bz * nchunk * l * l;
   for (int e = tid; e < l * l; e += blockDim.x) {
     double t = 0.0;
+#pragma unroll 8
     for (int c = 0; c < nchunk; ++c) t += pb[(long long)c * l * l + e];
     W[e] = t;
   }
@@ -128,8 +130,8 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const double* __restrict_
       if (!(d > 0.0) || !isfinite(d)) { if (tid == 0) bad = 1; }
       __syncthreads();
       if (bad) break;
-      const double sd = sqrt(d);
-      for (int i = j + tid; i < l; i += blockDim.x) Lm[i * l + j] = (i == j) ? sd : Lm[i * l + j] / sd;
+      const double sd = sqrt(d), isd = 1.0 / sd;
+      for (int i = j + tid; i < l; i += blockDim.x) Lm[i * l + j] = (i == j) ? sd : Lm[i * l + j] * isd;
       __syncthreads();
       const int rem = l - j - 1;
       for (int e = tid; e < rem * rem; e += blockDim.x) {
@@ -148,17 +150,24 @@ __global__ void __launch_bounds__(256) chol_inv_kernel(const double* __restrict_
   // X[:,c] for c: x_c = 1/L_cc; x_i = -(sum_{t=c}^{i-1} L_it x_t)/L_ii
   __syncthreads();
   double* X = W;   // reuse
-  for (int c = tid; c < l; c += blockDim.x) {
-    for (int i = 0; i < l; ++i) X[i * l + c] = 0.0;
-    if (!bad) {
-      X[c * l + c] = 1.0 / Lm[c * l + c];
-      for (int i = c + 1; i < l; ++i) {
+  for (int e = tid; e < l * l; e += blockDim.x) X[e] = 0.0;
+  if (tid < l) rdiag[tid] = bad ? 0.0 : 1.0 / Lm[tid * l + tid];
+  __syncthreads();
+  if (!bad) {
+    // eight lanes per column share each row's dot product; a column never leaves its warp, so rows are
+    // ordered by __syncwarp only
+    const int sub = tid & 7;
+    for (int c = tid >> 3; c < ((l + 3) & ~3); c += blockDim.x >> 3) {
+      for (int i = 0; i < l; ++i) {
         double t = 0.0;
-        for (int k2 = c; k2 < i; ++k2) t += Lm[i * l + k2] * X[k2 * l + c];
-        X[i * l + c] = -t / Lm[i * l + i];
+        if (c < l && i > c)
+          for (int k2 = c + sub; k2 < i; k2 += 8) t += Lm[i * l + k2] * X[k2 * l + c];
+        t += __shfl_xor_sync(0xffffffffu, t, 1);
+        t += __shfl_xor_sync(0xffffffffu, t, 2);
+        t += __shfl_xor_sync(0xffffffffu, t, 4);
+        if (sub == 0 && c < l && i >= c) X[i * l + c] = ((i == c) ? 1.0 - t : -t) * rdiag[i];
+        __syncwarp();
       }
-    } else {
-      X[c * l + c] = 0.0;   // total failure: zero basis, flagged above
     }
   }
   __syncthreads();
@@ -178,7 +187,7 @@ cudaError_t chol_inv_launch(const double* partial, int nchunk, int batch, int l,
     cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * MAX_L * MAX_L * 8);
     attr_set = true;
   }
-  chol_inv_kernel<<<batch, 256, smem, st>>>(partial, nchunk, l, Rinv, status);
+  chol_inv_kernel<<<batch, 512, smem, st>>>(partial, nchunk, l, Rinv, status);
   if (launches) ++*launches;
   return cudaGetLastError();
 }
@@ -626,6 +635,175 @@ cudaError_t split_concat3_launch(const float* In, long long in_bs, int ld_in, in
   const long long tot = (long long)rows * kp;
   split_concat3_kernel<<<dim3((unsigned)((tot + 255) / 256), batch), 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s,
                                                                                   inv_rho, c0, c1, pattern, Out);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace defl
+
+// ---------------------------------------------------------------------------------------------
+// Fused panel pass for CholeskyQR2 and the triplet products: for panel In[b, rows, l]
+//   Out = In * Mtx[:, :kout]   (Mtx null: Out = In), written as fp32 and/or as bf16 hi + lo,
+//   and/or the Gram partials of Out (fp32 products over 128-row tiles, tiles added in fp64).
+// One CTA walks a chunk of FUSED_CHUNK rows in 128-row tiles; register-blocked 4 x 8 outputs per thread.
+// In-place (Out == In) is safe: a tile is read completely before it is written.
+// ---------------------------------------------------------------------------------------------
+namespace defl {
+
+constexpr int FUSED_TILE = 128;
+constexpr int FUSED_CHUNK = 512;
+constexpr int FUSED_TS = MAX_L + 4;
+
+int fused_num_chunks(int rows) { return (rows + FUSED_CHUNK - 1) / FUSED_CHUNK; }
+
+__global__ void __launch_bounds__(256) panel_fused_kernel(const float* In, long long in_bs, int ld_in, int rows, int l,
+                                                          const float* __restrict__ Mtx, int ldm, int kout,
+                                                          float* Out, long long out_bs, int ld_out,
+                                                          __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                                                          int lp, double* __restrict__ partial, int nchunk) {
+  extern __shared__ __align__(16) float fsm[];
+  // row stride 68 floats: rows stay 16-byte aligned, so register blocks are fetched with 128-bit loads
+  float (*tile)[FUSED_TS] = reinterpret_cast<float (*)[FUSED_TS]>(fsm);                          // [128][68]
+  float (*ms)[FUSED_TS] = reinterpret_cast<float (*)[FUSED_TS]>(fsm + FUSED_TILE * FUSED_TS);    // [64][68]
+  const int chunk = blockIdx.x, bz = blockIdx.y, tid = threadIdx.x;
+  const float* Ib = In + (long long)bz * in_bs;
+  const int wout = Mtx ? kout : l;      // width of Out
+  if (Mtx) {
+    const float* Mb = Mtx + (long long)bz * l * ldm;
+    for (int e = tid; e < MAX_L * MAX_L; e += 256) {
+      const int r = e / MAX_L, cc = e % MAX_L;
+      ms[r][cc] = (r < l && cc < kout) ? Mb[r * ldm + cc] : 0.f;
+    }
+  }
+  const int ty = tid >> 3, tx = tid & 7;        // product: rows ty*4.., cols tx*8..
+  const int gy = tid >> 4, gx = tid & 15;       // Gram: block (gy*4.., gx*4..)
+  double gacc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) gacc[i][j] = 0.0;
+  const int r_begin = chunk * FUSED_CHUNK, r_end = min(rows, r_begin + FUSED_CHUNK);
+  for (int r0 = r_begin; r0 < r_end; r0 += FUSED_TILE) {
+    __syncthreads();
+    if (ld_in == l && (l & 3) == 0 && ((reinterpret_cast<uintptr_t>(Ib) & 15) == 0)) {
+      // contiguous tile: all loads of a thread are issued before the first use (8 x 16 bytes in flight)
+      const float4* src = reinterpret_cast<const float4*>(Ib + (long long)r0 * l);
+      const int cnt4 = FUSED_TILE * l / 4;
+      float4 buf[FUSED_TILE * MAX_L / 4 / 256];
+#pragma unroll
+      for (int it = 0; it < FUSED_TILE * MAX_L / 4 / 256; ++it) {
+        const int f4 = tid + it * 256;
+        const int rr = (f4 * 4) / l;
+        buf[it] = (f4 < cnt4 && r0 + rr < r_end) ? src[f4] : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int it = 0; it < FUSED_TILE * MAX_L / 4 / 256; ++it) {
+        const int f4 = tid + it * 256;
+        if (f4 < cnt4) {
+          const int rr = (f4 * 4) / l, c = (f4 * 4) % l;
+          tile[rr][c] = buf[it].x; tile[rr][c + 1] = buf[it].y; tile[rr][c + 2] = buf[it].z; tile[rr][c + 3] = buf[it].w;
+        }
+      }
+    } else {
+      const int lr = (l + 3) & ~3;      // columns l..lr-1 are zeroed: the product walks the row in blocks of four
+      for (int e = tid; e < FUSED_TILE * lr; e += 256) {
+        const int rr = e / lr, c = e % lr;
+        tile[rr][c] = (c < l && r0 + rr < r_end) ? Ib[(long long)(r0 + rr) * ld_in + c] : 0.f;
+      }
+    }
+    __syncthreads();
+    if (Mtx) {
+      float acc[4][8];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+      // Mtx rows beyond l and columns beyond kout were zeroed when it was staged, so blocks of four are safe
+      for (int q = 0; q < l; q += 4) {
+        float4 a4[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) a4[i] = *reinterpret_cast<const float4*>(&tile[ty * 4 + i][q]);
+#pragma unroll
+        for (int qq = 0; qq < 4; ++qq) {
+          const float4 b0 = *reinterpret_cast<const float4*>(&ms[q + qq][tx * 8]);
+          const float4 b1 = *reinterpret_cast<const float4*>(&ms[q + qq][tx * 8 + 4]);
+          const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float av = (qq == 0) ? a4[i].x : (qq == 1) ? a4[i].y : (qq == 2) ? a4[i].z : a4[i].w;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(av, b[j], acc[i][j]);
+          }
+        }
+      }
+      __syncthreads();
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (tx * 8 + j < wout) tile[ty * 4 + i][tx * 8 + j] = acc[i][j];
+      __syncthreads();
+    }
+    if (Out) {
+      float* Ob = Out + (long long)bz * out_bs;
+      for (int e = tid; e < FUSED_TILE * wout; e += 256) {
+        const int rr = e / wout, c = e % wout;
+        if (r0 + rr < r_end) Ob[(long long)(r0 + rr) * ld_out + c] = tile[rr][c];
+      }
+    }
+    if (hi) {
+      for (int e = tid; e < FUSED_TILE * lp; e += 256) {
+        const int rr = e / lp, c = e % lp;
+        if (r0 + rr >= r_end) continue;
+        const float x = (c < wout) ? tile[rr][c] : 0.f;
+        const __nv_bfloat16 h = __float2bfloat16_rn(x);
+        const long long o = ((long long)bz * rows + r0 + rr) * lp + c;
+        hi[o] = h;
+        lo[o] = __float2bfloat16_rn(x - __bfloat162float(h));
+      }
+    }
+    if (partial) {
+      float f[4][4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) f[i][j] = 0.f;
+      const int nr = min(FUSED_TILE, r_end - r0);
+      for (int rr = 0; rr < nr; ++rr) {
+        const float4 a4 = *reinterpret_cast<const float4*>(&tile[rr][gy * 4]);
+        const float4 b4 = *reinterpret_cast<const float4*>(&tile[rr][gx * 4]);
+        const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) f[i][j] = fmaf(a[i], b[j], f[i][j]);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) gacc[i][j] += (double)f[i][j];
+    }
+  }
+  if (partial) {
+    double* out = partial + ((long long)bz * nchunk + chunk) * wout * wout;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int gi = gy * 4 + i, gj = gx * 4 + j;
+        if (gi < wout && gj < wout) out[gi * wout + gj] = gacc[i][j];
+      }
+  }
+}
+
+cudaError_t panel_fused_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int l, const float* Mtx,
+                               int ldm, int kout, float* Out, long long out_bs, int ld_out, __nv_bfloat16* hi,
+                               __nv_bfloat16* lo, int lp, double* partial, cudaStream_t st, long long* launches) {
+  const size_t smem = (size_t)(FUSED_TILE + MAX_L) * FUSED_TS * sizeof(float);
+  cudaFuncSetAttribute(panel_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const int nchunk = fused_num_chunks(rows);
+  panel_fused_kernel<<<dim3(nchunk, batch), 256, smem, st>>>(In, in_bs, ld_in, rows, l, Mtx, ldm, kout, Out, out_bs, ld_out,
+                                                            hi, lo, lp, partial, nchunk);
   if (launches) ++*launches;
   return cudaGetLastError();
 }

@@ -5,8 +5,8 @@
 //   warp 1      allocates tensor memory and issues tcgen05.mma (one elected lane), fp32 accumulators
 //               in tensor memory, two accumulator buffers so that the epilogue of tile i overlaps the
 //               products of tile i+1
-//   warps 2..5  epilogue: tcgen05.ld of the accumulator (each warp its own 32-lane quarter), the
-//               element-wise epilogue (store / polynomial / residual / norm partials), global stores
+//   warps 2..9  epilogue: tcgen05.ld of the accumulator (two warps per 32-lane quarter, alternating 32-column
+//               blocks), the element-wise epilogue (store / polynomial / residual / norm partials), global stores
 //
 // A tile is 128 x BN outputs (BN chosen per call, a multiple of 16 up to 256), K is walked in blocks of
 // 128 bytes (64 bf16 or 32 tf32 values). Either operand may be K-major (K contiguous in global memory)
@@ -24,7 +24,8 @@ namespace defl {
 namespace {
 
 constexpr int KBYTES = 128;                 // bytes of K per stage row (one swizzle span)
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 320;            // producer warp, MMA warp, eight epilogue warps
+constexpr int EPI_WARPS = 8;
 constexpr int MAX_STAGES = 6;
 constexpr unsigned long long WAIT_NS = 2000000000ull;  // 2 s per wait before giving up
 
@@ -38,6 +39,7 @@ struct TcParams {
   int BN;                      // tile width (UMMA N)
   int tile_m;                  // 128 or 256 rows per tile
   int tiles_m, tiles_n;
+  int tiles_per_matrix;        // tiles enumerated per matrix (fewer than tiles_m * tiles_n for symmetric output)
   long long total_tiles;
   int a_mn_major, b_mn_major;  // 0 = K-major, 1 = MN-major
   int esize;                   // operand element size in bytes (2 bf16, 4 tf32)
@@ -200,9 +202,24 @@ struct TileInfo {
 
 __device__ __forceinline__ TileInfo tile_info(const TcParams& p, long long tile) {
   TileInfo t;
-  t.tn = (int)(tile % p.tiles_n);
-  t.tm = (int)((tile / p.tiles_n) % p.tiles_m);
-  t.bz = (int)(tile / ((long long)p.tiles_n * p.tiles_m));
+  if (p.symmetric) {
+    // only tiles that reach the diagonal or lie right of it are enumerated, so that every CTA gets the same
+    // share of real work: tile row tm starts at column tile (tm * tile_m) / BN
+    t.bz = (int)(tile / p.tiles_per_matrix);
+    int idx = (int)(tile % p.tiles_per_matrix);
+    int tm = 0;
+    for (; tm < p.tiles_m; ++tm) {
+      const int first = (tm * p.tile_m) / p.BN;
+      const int cnt = p.tiles_n - first;
+      if (idx < cnt) { t.tn = first + idx; break; }
+      idx -= cnt;
+    }
+    t.tm = tm;
+  } else {
+    t.tn = (int)(tile % p.tiles_n);
+    t.tm = (int)((tile / p.tiles_n) % p.tiles_m);
+    t.bz = (int)(tile / ((long long)p.tiles_n * p.tiles_m));
+  }
   const int row0 = t.tm * p.tile_m, col_end = (t.tn + 1) * p.BN;
   t.skip = p.symmetric && col_end <= row0;               // entirely below the diagonal
   t.halves = 1;
@@ -214,102 +231,131 @@ __device__ __forceinline__ TileInfo tile_info(const TcParams& p, long long tile)
 }
 
 
-// Epilogue of one 128-row half of a tile for the calling warp's 32 rows: read the accumulator from tensor
-// memory 16 columns at a time, apply the element-wise operation, store. The kind is a template parameter
-// so that the per-element code is branch-free.
+// Epilogue of one 128-row half of a tile for the calling warp's 32 rows (one row per lane). The two warps
+// that share a tensor-memory lane quarter take alternate 32-column blocks. Per block: two 16-column
+// tensor-memory loads and (when the operation reads `aux`) the global loads of both chunks are issued before
+// anything is consumed, so that several requests per warp are in flight; then the element-wise operation and
+// 16-byte stores. The kind is a template parameter so that the per-element code is branch-free.
 template <int EPI>
-__device__ __forceinline__ void epilogue_half(const TcParams& p, uint32_t taddr, int gi, int col0, int n_eff, int bz,
-                                              float alpha, float aux_scale, double& sq) {
-  const bool row_ok = gi < p.M;
-  const bool out_bf16 = (p.out_dtype == BF16), aux_bf16 = (p.aux_dtype == BF16);
-  const size_t crow = (size_t)bz * p.batch_c + (size_t)gi * p.ldc;
-  const size_t xrow = (size_t)bz * p.batch_aux + (size_t)gi * p.ld_aux;
+__device__ __forceinline__ void load_aux16(const TcParams& p, bool take, bool vec, bool aux_bf16, size_t xoff, int gj0,
+                                           float* x) {
+  if (EPI == EPI_STORE) return;
   const __nv_bfloat16* auxh = reinterpret_cast<const __nv_bfloat16*>(p.aux);
   const float* auxf = reinterpret_cast<const float*>(p.aux);
+  if (!take) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) x[j] = 0.f;
+  } else if (vec && aux_bf16) {
+    const uint4* src = reinterpret_cast<const uint4*>(auxh + xoff);
+    uint4 pk[2] = {src[0], src[1]};
+    const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(pk);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { const float2 f = __bfloat1622float2(hh[j]); x[2 * j] = f.x; x[2 * j + 1] = f.y; }
+  } else if (vec) {
+    const float4* src = reinterpret_cast<const float4*>(auxf + xoff);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { const float4 f = src[j]; x[4 * j] = f.x; x[4 * j + 1] = f.y; x[4 * j + 2] = f.z; x[4 * j + 3] = f.w; }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      x[j] = (gj0 + j < p.N) ? (aux_bf16 ? __bfloat162float(auxh[xoff + j]) : auxf[xoff + j]) : 0.f;
+  }
+}
+
+template <int EPI>
+__device__ __forceinline__ void finish16(const TcParams& p, const uint32_t* r, const float* x, int gi, int gi_warp0,
+                                         int gj0, bool row_ok, bool vec, size_t crow, size_t cbatch, float alpha,
+                                         float aux_scale, double& sq) {
+  if (gj0 >= p.N) return;
+  const bool out_bf16 = (p.out_dtype == BF16);
   __nv_bfloat16* outh = reinterpret_cast<__nv_bfloat16*>(p.C);
   float* outf = reinterpret_cast<float*>(p.C);
-  const bool vec_ok = ((p.ldc & 7) == 0) && ((p.batch_c & 7) == 0) && ((p.ld_aux & 7) == 0 || EPI == EPI_STORE) &&
-                      ((p.batch_aux & 7) == 0 || EPI == EPI_STORE) && !p.symmetric;
-  for (int c0 = 0; c0 < n_eff; c0 += 16) {
-    uint32_t r[16];
-    __syncwarp();
-    tmem_ld16(taddr + (uint32_t)c0, r);
-    tmem_ld_wait();
-    const int gj0 = col0 + c0;
-    if (gj0 >= p.N || !row_ok) continue;
-    const bool full = (gj0 + 16 <= p.N) && vec_ok && ((gj0 & 7) == 0);
-    float x[16];
-    if (EPI != EPI_STORE) {
-      if (full && aux_bf16) {
-        const uint4* src = reinterpret_cast<const uint4*>(auxh + xrow + gj0);
-        uint4 pk[2] = {src[0], src[1]};
-        const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(pk);
+  float v[16];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { const float2 f = __bfloat1622float2(hh[j]); x[2 * j] = f.x; x[2 * j + 1] = f.y; }
-      } else if (full) {
-        const float4* src = reinterpret_cast<const float4*>(auxf + xrow + gj0);
+  for (int j = 0; j < 16; ++j) {
+    const float a = __uint_as_float(r[j]);
+    if (EPI == EPI_STORE) v[j] = alpha * a;
+    else if (EPI == EPI_POLY) v[j] = p.pb * x[j] + p.pc * a + ((gi == gj0 + j) ? p.pa : 0.f);
+    else if (EPI == EPI_AUX_PLUS) v[j] = aux_scale * x[j] + alpha * a;
+    else v[j] = (row_ok && gj0 + j < p.N) ? (x[j] - a) : 0.f;
+  }
+  if (p.round_tf32) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) { const float4 f = src[j]; x[4 * j] = f.x; x[4 * j + 1] = f.y; x[4 * j + 2] = f.z; x[4 * j + 3] = f.w; }
-      } else {
+    for (int j = 0; j < 16; ++j) v[j] = round_to_tf32(v[j]);
+  }
+  if (EPI == EPI_RESID_NORM) {
+    float sqf = 0.f;
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-          x[j] = (gj0 + j < p.N) ? (aux_bf16 ? __bfloat162float(auxh[xrow + gj0 + j]) : auxf[xrow + gj0 + j]) : 0.f;
-      }
+    for (int j = 0; j < 16; ++j) sqf = fmaf(v[j], v[j], sqf);
+    sq += (double)sqf;
+    return;
+  }
+  if (!row_ok) return;
+  // symmetric output: chunks entirely right of the warp's rows are stored like any other chunk and mirrored;
+  // chunks that touch the diagonal go element by element; chunks left of it are skipped by the caller
+  const bool mirror_all = p.symmetric && gj0 > gi_warp0 + 31;
+  if (vec && (!p.symmetric || mirror_all)) {
+    if (out_bf16) {
+      uint4 pk[2];
+      __nv_bfloat162* hh = reinterpret_cast<__nv_bfloat162*>(pk);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) hh[j] = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+      uint4* dst = reinterpret_cast<uint4*>(outh + crow + gj0);
+      dst[0] = pk[0]; dst[1] = pk[1];
+    } else {
+      float4* dst = reinterpret_cast<float4*>(outf + crow + gj0);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
     }
-    float v[16];
+  } else {
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-      const float a = __uint_as_float(r[j]);
-      if (EPI == EPI_STORE) v[j] = alpha * a;
-      else if (EPI == EPI_POLY) v[j] = p.pb * x[j] + p.pc * a + ((gi == gj0 + j) ? p.pa : 0.f);
-      else if (EPI == EPI_AUX_PLUS) v[j] = aux_scale * x[j] + alpha * a;
-      else v[j] = (gj0 + j < p.N) ? (x[j] - a) : 0.f;
-    }
-    if (p.round_tf32) {
-#pragma unroll
-      for (int j = 0; j < 16; ++j) v[j] = round_to_tf32(v[j]);
-    }
-    if (EPI == EPI_RESID_NORM) {
-      float sqf = 0.f;
-#pragma unroll
-      for (int j = 0; j < 16; ++j) sqf = fmaf(v[j], v[j], sqf);
-      sq += (double)sqf;
-      continue;
-    }
-    if (full) {
-      if (out_bf16) {
-        uint4 pk[2];
-        __nv_bfloat162* hh = reinterpret_cast<__nv_bfloat162*>(pk);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) hh[j] = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
-        uint4* dst = reinterpret_cast<uint4*>(outh + crow + gj0);
-        dst[0] = pk[0]; dst[1] = pk[1];
-      } else {
-        float4* dst = reinterpret_cast<float4*>(outf + crow + gj0);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-      }
-    } else if (!p.symmetric) {
-#pragma unroll
-      for (int j = 0; j < 16; ++j)
-        if (gj0 + j < p.N) {
-          if (out_bf16) outh[crow + gj0 + j] = __float2bfloat16_rn(v[j]); else outf[crow + gj0 + j] = v[j];
-        }
-    } else {
-      // symmetric output: write the upper part directly and its mirror image; across the warp the
-      // mirrored stores of one column are contiguous (lanes are consecutive rows)
-      const size_t cb = (size_t)bz * p.batch_c;
-#pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const int gj = gj0 + j;
-        if (gj >= p.N) continue;
-        if (gj >= gi) { if (out_bf16) outh[crow + gj] = __float2bfloat16_rn(v[j]); else outf[crow + gj] = v[j]; }
-        if (gj > gi) {
-          const size_t m = cb + (size_t)gj * p.ldc + gi;
-          if (out_bf16) outh[m] = __float2bfloat16_rn(v[j]); else outf[m] = v[j];
-        }
+      const int gj = gj0 + j;
+      if (gj < p.N && (!p.symmetric || gj >= gi)) {
+        if (out_bf16) outh[crow + gj] = __float2bfloat16_rn(v[j]); else outf[crow + gj] = v[j];
       }
     }
+  }
+  if (p.symmetric) {
+    // mirror image: for a fixed column the 32 lanes are 32 consecutive rows, i.e. one contiguous run
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const int gj = gj0 + j;
+      if (gj < p.N && gj > gi) {
+        const size_t m = cbatch + (size_t)gj * p.ldc + gi;
+        if (out_bf16) outh[m] = __float2bfloat16_rn(v[j]); else outf[m] = v[j];
+      }
+    }
+  }
+}
+
+template <int EPI>
+__device__ __forceinline__ void epilogue_half(const TcParams& p, uint32_t taddr, int gi, int gi_warp0, int col0, int n_eff,
+                                              int bz, int wsel, float alpha, float aux_scale, double& sq) {
+  const bool row_ok = gi < p.M;
+  const bool aux_bf16 = (p.aux_dtype == BF16);
+  const size_t cbatch = (size_t)bz * p.batch_c;
+  const size_t crow = cbatch + (size_t)gi * p.ldc;
+  const size_t xrow = (size_t)bz * p.batch_aux + (size_t)gi * p.ld_aux;
+  const bool vec_ok = ((p.ldc & 7) == 0) && ((p.batch_c & 7) == 0) && ((p.ld_aux & 7) == 0 || EPI == EPI_STORE) &&
+                      ((p.batch_aux & 7) == 0 || EPI == EPI_STORE);
+  for (int c0 = wsel * 32; c0 < n_eff; c0 += 64) {
+    const int gj0 = col0 + c0, gj1 = gj0 + 16;
+    // symmetric output: nothing to do for a block entirely left of the warp's rows (warp-uniform)
+    if (p.symmetric && gj0 + 31 < gi_warp0) continue;
+    const bool second = (c0 + 16 < n_eff);
+    uint32_t r0[16], r1[16];
+    __syncwarp();
+    tmem_ld16(taddr + (uint32_t)c0, r0);
+    if (second) tmem_ld16(taddr + (uint32_t)c0 + 16u, r1);
+    const bool vec0 = vec_ok && (gj0 + 16 <= p.N) && ((gj0 & 7) == 0);
+    const bool vec1 = vec_ok && (gj1 + 16 <= p.N) && ((gj1 & 7) == 0);
+    float x0[16], x1[16];
+    load_aux16<EPI>(p, row_ok && gj0 < p.N, vec0, aux_bf16, xrow + gj0, gj0, x0);
+    load_aux16<EPI>(p, second && row_ok && gj1 < p.N, vec1, aux_bf16, xrow + gj1, gj1, x1);
+    tmem_ld_wait();
+    finish16<EPI>(p, r0, x0, gi, gi_warp0, gj0, row_ok, vec0, crow, cbatch, alpha, aux_scale, sq);
+    if (second) finish16<EPI>(p, r1, x1, gi, gi_warp0, gj1, row_ok, vec1, crow, cbatch, alpha, aux_scale, sq);
   }
 }
 
@@ -332,7 +378,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&acc_full_bar[a]), 1); mbar_init(smem_u32(&acc_empty_bar[a]), 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&acc_full_bar[a]), 1); mbar_init(smem_u32(&acc_empty_bar[a]), EPI_WARPS); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -431,6 +477,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   } else {
     // ------------------------------------------------------------------ epilogue warps
     const int q = warp & 3;                 // tensor-memory lane quarter this warp may read
+    const int wsel = (warp - 2) >> 2;       // which of the two warps of that quarter: alternate 32-column blocks
     uint32_t acc = 0, acc_phase = 0;
     for (long long tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
       const TileInfo t = tile_info(p, tile);
@@ -447,19 +494,19 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
         if (t.halves & (1 << h)) {
           const uint32_t tcol = (p.tile_m == 256) ? (uint32_t)h * 256u : acc * 256u;
           const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + tcol;
-          const int gi = tm * p.tile_m + h * 128 + q * 32 + lane;
+          const int gi0 = tm * p.tile_m + h * 128 + q * 32, gi = gi0 + lane;
           switch (p.epilogue) {
-            case EPI_STORE: epilogue_half<EPI_STORE>(p, taddr, gi, tn * p.BN, t.n_eff, bz, alpha, aux_scale, sq); break;
-            case EPI_POLY: epilogue_half<EPI_POLY>(p, taddr, gi, tn * p.BN, t.n_eff, bz, alpha, aux_scale, sq); break;
-            case EPI_AUX_PLUS: epilogue_half<EPI_AUX_PLUS>(p, taddr, gi, tn * p.BN, t.n_eff, bz, alpha, aux_scale, sq); break;
-            default: epilogue_half<EPI_RESID_NORM>(p, taddr, gi, tn * p.BN, t.n_eff, bz, alpha, aux_scale, sq); break;
+            case EPI_STORE: epilogue_half<EPI_STORE>(p, taddr, gi, gi0, tn * p.BN, t.n_eff, bz, wsel, alpha, aux_scale, sq); break;
+            case EPI_POLY: epilogue_half<EPI_POLY>(p, taddr, gi, gi0, tn * p.BN, t.n_eff, bz, wsel, alpha, aux_scale, sq); break;
+            case EPI_AUX_PLUS: epilogue_half<EPI_AUX_PLUS>(p, taddr, gi, gi0, tn * p.BN, t.n_eff, bz, wsel, alpha, aux_scale, sq); break;
+            default: epilogue_half<EPI_RESID_NORM>(p, taddr, gi, gi0, tn * p.BN, t.n_eff, bz, wsel, alpha, aux_scale, sq); break;
           }
         }
         if (p.epilogue == EPI_RESID_NORM) {
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) sq += __shfl_down_sync(0xffffffffu, sq, o);
           if (lane == 0)
-            p.partials[(long long)bz * p.partials_per_batch + (((long long)tm * p.tiles_n + tn) * (p.tile_m == 256 ? 2 : 1) + h) * 4 + (warp - 2)] = sq;
+            p.partials[(long long)bz * p.partials_per_batch + (((long long)tm * p.tiles_n + tn) * (p.tile_m == 256 ? 2 : 1) + h) * EPI_WARPS + (warp - 2)] = sq;
         }
       }
       // release the accumulator buffer
@@ -606,7 +653,7 @@ int choose_tile_m(int M) {
 
 int gemm_tc_partials_per_batch(const GemmDesc& g) {
   const int bn = choose_bn(g.N), tmh = choose_tile_m(g.M);
-  return ((g.M + tmh - 1) / tmh) * ((g.N + bn - 1) / bn) * (tmh == 256 ? 8 : 4);
+  return ((g.M + tmh - 1) / tmh) * ((g.N + bn - 1) / bn) * (tmh == 256 ? 2 : 1) * EPI_WARPS;
 }
 
 cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word, int num_sms, long long* launches) {
@@ -621,7 +668,15 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   p.tile_m = choose_tile_m(g.M);
   p.tiles_m = (g.M + p.tile_m - 1) / p.tile_m;
   p.tiles_n = (g.N + p.BN - 1) / p.BN;
-  p.total_tiles = (long long)p.tiles_m * p.tiles_n * g.batch;
+  p.tiles_per_matrix = p.tiles_m * p.tiles_n;
+  if (g.symmetric) {
+    p.tiles_per_matrix = 0;
+    for (int tm = 0; tm < p.tiles_m; ++tm) {
+      const int first = (tm * p.tile_m) / p.BN;
+      if (first < p.tiles_n) p.tiles_per_matrix += p.tiles_n - first;
+    }
+  }
+  p.total_tiles = (long long)p.tiles_per_matrix * g.batch;
   p.nseg = g.nseg;
   OperandPlan pa, pb;
   // when a dimension has extent 1 both strides may look "unit"; prefer K-major

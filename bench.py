@@ -25,6 +25,7 @@ sys.path.insert(0, ROOT)
 
 METRIC = "deflated polar-filter TFLOP/s & matrices/s per batch; % bf16 tensor peak"
 MUON = (3.4445, -4.7750, 2.0315)
+SYM = True   # compute X X^T and A A on the tiles that reach the diagonal and mirror them (--no-symmetry turns it off)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 WORKLOADS = {
@@ -65,6 +66,29 @@ def max_over_ranks(value, dist=None, device="cpu"):
 def aggregate_throughput(units_per_rank, world, ms_max):
     """Whole-job rate when every rank processes `units_per_rank` in `ms_max` milliseconds (weak scaling)."""
     return world * units_per_rank / (ms_max * 1e-3)
+
+
+def executed_filter_flops(m, n, L, symmetric, tile=256):
+    """Flops the tensor engine executes for the L filter steps of one matrix. It works on 256 x 256 output
+    tiles made of two 128-row halves; edge tiles compute only the rows (in halves) and columns (in sixteens)
+    that exist; with `symmetric` the two symmetric products skip every half-tile left of the diagonal."""
+    ms, ml = min(m, n), max(m, n)
+
+    def product(M, N, K, sym):
+        total = 0.0
+        for r0 in range(0, M, tile):
+            for c0 in range(0, N, tile):
+                cols = min(tile, ((N - c0 + 15) // 16) * 16)
+                for h0 in (r0, r0 + 128):
+                    if h0 >= M:
+                        continue
+                    if sym and c0 + tile <= h0:
+                        continue
+                    total += 2.0 * 128 * cols * K
+        return total
+
+    return L * (product(ms, ms, ml, symmetric) + product(ms, ms, ms, symmetric) +
+                (product(m, n, m, False) if m <= n else product(m, n, n, False)))
 
 
 def load_peaks():
@@ -136,7 +160,7 @@ def run_step(ctx, wl, groups, lanes=None):
     if not lanes:
         for g in groups:
             ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"],
-                                   sketch=g["Om"], gamma=1.01)
+                                   sketch=g["Om"], gamma=1.01, exploit_symmetry=SYM)
         return
     main = torch.cuda.current_stream()
     fork = torch.cuda.Event()
@@ -145,7 +169,7 @@ def run_step(ctx, wl, groups, lanes=None):
         s.wait_event(fork)
         with torch.cuda.stream(s):
             c.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"],
-                                 sketch=g["Om"], gamma=1.01)
+                                 sketch=g["Om"], gamma=1.01, exploit_symmetry=SYM)
             done = torch.cuda.Event()
             done.record(s)
         main.wait_event(done)
@@ -177,9 +201,12 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--small", action="store_true", help="tiny workload for a quick functional check")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-symmetry", action="store_true", help="compute the symmetric products in full")
     ap.add_argument("--streams", type=int, default=2, help="2: one stream + context per shape group; 1: one stream")
     ap.add_argument("--batch", type=int, default=0, help="override the matrices per shape group (profiling captures)")
     args = ap.parse_args()
+    global SYM
+    SYM = not args.no_symmetry
     wl_name = "small" if args.small else "gpt2_xl"
     wl = dict(WORKLOADS[wl_name])
     if args.batch > 0:
@@ -189,7 +216,7 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     config = {"workload": wl["label"], "name": wl_name, "k": wl["k"], "oversample": wl["p"], "power_iters": wl["J"],
-              "filter_steps": wl["L"], "restore": "padded, gamma=1.01",
+              "filter_steps": wl["L"], "restore": "padded, gamma=1.01", "exploit_symmetry": SYM,
               "l2": "inputs (1.2 GB per step) larger than L2; no flush"}
     tot_f = sum(b * sum(flops_per_matrix(m, n, wl["k"], wl["p"], wl["J"], wl["L"])) for b, m, n in wl["groups"])
     nmat = sum(b for b, _, _ in wl["groups"])
@@ -257,19 +284,21 @@ def main():
 
     # stage split of one more (untimed) step, with the same events the library records on its stream
     stage_tot = [0.0, 0.0, 0.0, 0.0]
-    filt_flops = 0.0
+    filt_flops = 0.0        # dense count of the filter products
+    filt_executed = 0.0     # flops the tensor cores actually execute (tiles below the diagonal are skipped)
     for g, (b, m, n) in zip(groups, wl["groups"]):
         ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"], sketch=g["Om"],
-                               gamma=1.01)
+                               gamma=1.01, exploit_symmetry=SYM)
         ms = ctx.defl_get_stage_ms()
         for i in range(min(4, len(ms))):
             stage_tot[i] += ms[i]
         filt_flops += b * flops_per_matrix(m, n, wl["k"], wl["p"], wl["J"], wl["L"])[0]
+        filt_executed += b * executed_filter_flops(m, n, wl["L"], SYM)
     plain_ms = 0.0
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for g in groups:
-        ctx.defl_polar_batched(g["G"], 0, 0, 0, [list(MUON)] * wl["L"], out=g["out"])
+        ctx.defl_polar_batched(g["G"], 0, 0, 0, [list(MUON)] * wl["L"], out=g["out"], exploit_symmetry=SYM)
     e1.record()
     torch.cuda.synchronize()
     plain_ms = e0.elapsed_time(e1)
@@ -281,7 +310,8 @@ def main():
         hO = [torch.empty_like(h).pin_memory() for h in hG]
         def e2e_step():
             for h, o, g in zip(hG, hO, groups):
-                ctx.defl_polar_batched_host(h, o, wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], sketch=g["Om"], gamma=1.01)
+                ctx.defl_polar_batched_host(h, o, wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], sketch=g["Om"], gamma=1.01,
+                                            exploit_symmetry=SYM)
         e2e_step()
         barrier()
         t0 = time.perf_counter()
@@ -302,14 +332,17 @@ def main():
     value = aggregate_throughput(tot_f, world, ms_per_step) / 1e12
     filt_ms = stage_tot[2]
     n_filter_launches = 3 * wl["L"] * len(groups)
-    ach = filt_flops / (filt_ms * 1e-3) / 1e12 if filt_ms > 0 else None
+    # achieved = flops the kernel really executes / its time (no credit for skipped symmetric tiles)
+    ach = filt_executed / (filt_ms * 1e-3) / 1e12 if filt_ms > 0 else None
+    ach_dense = filt_flops / (filt_ms * 1e-3) / 1e12 if filt_ms > 0 else None
     peak = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
     roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel (filter chain: X X^T, A^2 polynomial, B X)",
                 "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": (ach / peak) if ach else None,
                 "peak_kind": "bf16_tflops_sustained, of %s" % peaks_kind,
                 "frac_of_burst": (ach / float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))) if ach else None,
                 "launches_per_step": n_filter_launches, "avg_launch_ms": filt_ms / n_filter_launches,
-                "flops_per_launch_avg": filt_flops / n_filter_launches,
+                "flops_per_launch_avg": filt_executed / n_filter_launches,
+                "dense_equivalent_tflops": ach_dense,
                 "traffic": FILTER_TRAFFIC_BYTES_PER_LAUNCH if (wl_name == "gpt2_xl" and args.batch == 0) else None,
                 "traffic_unit": "bytes per launch (ncu, 8-matrix capture scaled to the batch)"}
     line = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,

@@ -32,6 +32,8 @@ constexpr unsigned long long WAIT_NS = 2000000000ull;  // 2 s per wait before gi
 struct TcParams {
   CUtensorMap tmA[2];
   CUtensorMap tmB[2];
+  CUtensorMap tmAux;           // [batch, M, N] view of `aux`, used only to prefetch the epilogue's tile into L2
+  int aux_prefetch;
   int nseg;
   int b_split;                 // 2: B is the sum of two operands (tmB[0] + tmB[1]) that share A; else 1
   int kblocks[2];              // K blocks per segment
@@ -113,6 +115,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
+}
+
+// asks the memory system to bring one tile of a tensor into L2 (no shared memory, no completion to wait for)
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* tm, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+               ::"l"(tm), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
 }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
@@ -398,6 +407,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       for (long long tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
         const TileInfo t = tile_info(p, tile);
         if (t.skip) continue;
+        // the epilogue of this tile will read the matching tile of `aux` with plain loads: start moving it
+        // from HBM into L2 now, a whole main loop ahead
+        if (p.aux_prefetch) tma_prefetch_3d(&p.tmAux, t.tn * p.BN, t.tm * p.tile_m, t.bz);
         for (int seg = 0; seg < p.nseg; ++seg) {
           for (int kb = 0; kb < p.kblocks[seg]; ++kb) {
             if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag, p.status)) break;
@@ -720,6 +732,23 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   p.alpha = g.alpha; p.aux_scale = g.aux_scale; p.pa = g.pa; p.pb = g.pb; p.pc = g.pc;
   p.alpha_dev = g.alpha_dev; p.aux_scale_dev = g.aux_scale_dev;
   p.partials = g.partials; p.partials_per_batch = g.partials_per_batch;
+  p.aux_prefetch = 0;
+  if (g.aux && g.epilogue != EPI_STORE && aligned16(g.aux)) {
+    const int aes = (int)dtype_size(g.aux_dtype);
+    if ((g.ld_aux * aes) % 16 == 0 && (g.batch == 1 || (g.batch_aux * aes) % 16 == 0)) {
+      EncodeTiledFn enc = get_encode_fn();
+      cuuint64_t dims[3] = {(cuuint64_t)g.N, (cuuint64_t)g.M, (cuuint64_t)g.batch};
+      cuuint64_t strides[2] = {(cuuint64_t)g.ld_aux * aes, (cuuint64_t)(g.batch == 1 ? g.ld_aux * (long long)g.M : g.batch_aux) * aes};
+      // 16-bit types: a full 256-column tile per box; 32-bit types: box columns are capped at 256 elements too
+      cuuint32_t box[3] = {(cuuint32_t)(p.BN < 256 ? p.BN : 256), (cuuint32_t)p.tile_m, 1};
+      cuuint32_t estr[3] = {1, 1, 1};
+      const CUtensorMapDataType dt = (aes == 2) ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+      if (enc && enc(&p.tmAux, dt, 3, const_cast<void*>(g.aux), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+        p.aux_prefetch = 1;
+    }
+  }
   p.status = status_word;
 
   const size_t smem = (size_t)stages * stage_bytes + 1024;

@@ -79,6 +79,10 @@ typedef struct defl_opts {
                             advance the basis (the paper keeps the gate off while the basis stabilises) */
   int engine;            /* DEFL_ENGINE_* */
   int exploit_symmetry;  /* non-zero: compute only the upper tiles of X X^T and of A^2 and mirror them */
+  float tau;             /* deflation gate of Algorithms 1 and 2. <= 0 (default): deflate exactly k components.
+                            > 0: with s the k estimated magnitudes, deflate only if s_k < tau * s_1, and then the
+                            components with s_i > tau * s_1 (PSD: among all K Ritz values); otherwise the call
+                            reduces to the undeflated filter for that matrix. Decided per matrix on the device. */
 } defl_opts;
 
 typedef struct defl_info {
@@ -86,6 +90,7 @@ typedef struct defl_info {
                     decreasing magnitude); may be NULL */
   float* rho;    /* device, [b]: ||R||_F used for normalisation (PSD: [1], the scale theta-hat); may be NULL */
   int* status;   /* device, [b]: DEFL_ST_* bits (PSD: [1]); may be NULL */
+  int* k_used;   /* device, [b]: number of components actually deflated (PSD: [1]); may be NULL */
 } defl_info;
 
 /* Context. `device` is a CUDA ordinal. defl_create makes no assumption about the current device

@@ -33,11 +33,13 @@ EXPORTS = [
 class DeflOpts(ctypes.Structure):
     _fields_ = [("sketch", ctypes.c_void_p), ("seed", ctypes.c_uint64), ("restore_mode", ctypes.c_int),
                 ("gamma", ctypes.c_float), ("norm_mode", ctypes.c_int), ("lanczos_start", ctypes.c_void_p),
-                ("warmup", ctypes.c_int), ("engine", ctypes.c_int), ("exploit_symmetry", ctypes.c_int)]
+                ("warmup", ctypes.c_int), ("engine", ctypes.c_int), ("exploit_symmetry", ctypes.c_int),
+                ("tau", ctypes.c_float)]
 
 
 class DeflInfo(ctypes.Structure):
-    _fields_ = [("s", ctypes.c_void_p), ("rho", ctypes.c_void_p), ("status", ctypes.c_void_p)]
+    _fields_ = [("s", ctypes.c_void_p), ("rho", ctypes.c_void_p), ("status", ctypes.c_void_p),
+                ("k_used", ctypes.c_void_p)]
 
 
 _lib = None
@@ -146,7 +148,7 @@ class Context:
             raise DeflError(rc, lib().defl_last_error(self._h).decode())
 
     def _opts(self, sketch=None, seed=0, restore_mode=RESTORE_PADDED, gamma=0.0, norm_mode=NORM_LANCZOS,
-              lanczos_start=None, warmup=False, engine=ENGINE_AUTO, exploit_symmetry=False):
+              lanczos_start=None, warmup=False, engine=ENGINE_AUTO, exploit_symmetry=False, tau=0.0):
         o = DeflOpts()
         o.sketch = sketch.data_ptr() if sketch is not None else None
         o.seed = seed
@@ -157,12 +159,13 @@ class Context:
         o.warmup = int(bool(warmup))
         o.engine = engine
         o.exploit_symmetry = int(bool(exploit_symmetry))
+        o.tau = tau
         return o
 
     # ------------------------------------------------------------------------------------------
     def defl_polar_batched(self, G, k, oversample, power_iters, coeff_schedule, steps=None, out=None, sketch=None,
                            seed=0, restore_mode=RESTORE_PADDED, gamma=0.0, engine=ENGINE_AUTO,
-                           exploit_symmetry=False, want_info=False):
+                           exploit_symmetry=False, want_info=False, tau=0.0):
         """out[b,m,n] = deflated polar factor of every G[b] (Algorithm 3 + Algorithm 1)."""
         _dev(G, "G")
         if G.ndim != 3:
@@ -175,7 +178,7 @@ class Context:
             if sketch.dtype != torch.float32:
                 raise TypeError("sketch must be float32")
         opts = self._opts(sketch=sketch, seed=seed, restore_mode=restore_mode, gamma=gamma, engine=engine,
-                          exploit_symmetry=exploit_symmetry)
+                          exploit_symmetry=exploit_symmetry, tau=tau)
         info = DeflInfo()
         extras = None
         if want_info:
@@ -183,8 +186,10 @@ class Context:
             s = torch.zeros((b, max(l, 1)), dtype=torch.float32, device=G.device)
             rho = torch.zeros((b,), dtype=torch.float32, device=G.device)
             status = torch.zeros((b,), dtype=torch.int32, device=G.device)
+            k_used = torch.zeros((b,), dtype=torch.int32, device=G.device)
             info.s, info.rho, info.status = s.data_ptr(), rho.data_ptr(), status.data_ptr()
-            extras = {"s": s[:, :l], "rho": rho, "status": status}
+            info.k_used = k_used.data_ptr()
+            extras = {"s": s[:, :l], "rho": rho, "status": status, "k_used": k_used}
         self._sync_stream()
         rc = lib().defl_polar_batched(self._h, _ptr(G), _ptr(out), b, m, n, _dtype_code(G), k, oversample, power_iters,
                                       sched, L, ctypes.byref(opts), ctypes.byref(info))
@@ -226,7 +231,7 @@ class Context:
 
     def defl_psd_project(self, X, k, warm_basis, coeff_schedule, steps=None, out=None, gamma=0.0,
                          norm_mode=NORM_LANCZOS, lanczos_start=None, seed=0, warmup=False, engine=ENGINE_AUTO,
-                         exploit_symmetry=False, want_info=False):
+                         exploit_symmetry=False, want_info=False, tau=0.0):
         """P = deflated PSD projection of the symmetric X[n,n] (Algorithm 2); warm_basis[n,K] is updated in place."""
         _dev(X, "X")
         n = X.shape[0]
@@ -239,15 +244,17 @@ class Context:
         out = torch.empty_like(X) if out is None else _dev(out, "out")
         sched, T = _schedule(coeff_schedule, steps)
         opts = self._opts(gamma=gamma, norm_mode=norm_mode, lanczos_start=lanczos_start, seed=seed, warmup=warmup,
-                          engine=engine, exploit_symmetry=exploit_symmetry)
+                          engine=engine, exploit_symmetry=exploit_symmetry, tau=tau)
         info = DeflInfo()
         extras = None
         if want_info:
             lam = torch.zeros((max(K, 1),), dtype=torch.float32, device=X.device)
             theta = torch.zeros((1,), dtype=torch.float32, device=X.device)
             status = torch.zeros((1,), dtype=torch.int32, device=X.device)
+            k_used = torch.zeros((1,), dtype=torch.int32, device=X.device)
             info.s, info.rho, info.status = lam.data_ptr(), theta.data_ptr(), status.data_ptr()
-            extras = {"lam": lam[:K], "theta": theta, "status": status}
+            info.k_used = k_used.data_ptr()
+            extras = {"lam": lam[:K], "theta": theta, "status": status, "k_used": k_used}
         self._sync_stream()
         rc = lib().defl_psd_project(self._h, _ptr(X), _ptr(out), n, k, _ptr(warm_basis), K, sched, T,
                                     ctypes.byref(opts), ctypes.byref(info))

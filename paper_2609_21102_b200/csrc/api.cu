@@ -92,6 +92,7 @@ struct PolarWs {
   double* npart;      // [b,nper] Frobenius partial sums
   float* rho; float* inv_rho; float* inv_rho2;   // [b]
   int* status;        // [b]
+  int* keff;          // [b] components deflated per matrix (gate)
   float* sketch;      // [b,ms,l] when the library draws the sketch
   // split-precision bf16 copies for the tensor engine (bf16 storage only)
   __nv_bfloat16* Lhi; __nv_bfloat16* Llo;   // [b,ml,lp]
@@ -128,6 +129,7 @@ PolarWs carve_polar(void* base, int b, int m, int n, int dtype, int k, int l) {
   w.inv_rho = cv.take<float>(b);
   w.inv_rho2 = cv.take<float>(b);
   w.status = cv.take<int>(b);
+  w.keff = cv.take<int>(b);
   w.sketch = cv.take<float>((size_t)b * ms * le);
   const int lp = round_up8(le), kp = round_up8(ke);
   const bool bf = (dtype == BF16);
@@ -430,6 +432,7 @@ int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int 
   if (engine < 0 || engine > 2) return DEFL_ERR_ARG;
   const float gamma = (opts && opts->gamma > 0.f) ? opts->gamma : 1.01f;
   const int sym = (opts && opts->exploit_symmetry) ? 1 : 0;
+  const float tau = opts ? opts->tau : 0.f;
 
   cudaSetDevice(c->device);
   int rc = ctx_reserve(c, carve_polar(nullptr, b, m, n, dtype, k, l).bytes);
@@ -460,6 +463,9 @@ int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int 
     // bf16 storage: the fp32 factors are split into bf16 hi + lo and the three significant cross terms are
     // laid side by side along K, [hi|hi|lo] x [hi|lo|hi]^T, one tensor-core product of depth 3k.
     const int kp = round_up8(k);
+    // gate (Algorithm 1, lines 1-2): per matrix, how many of the k triplets are deflated; the columns beyond
+    // that count are zeroed in the scaled right factor, which removes them from every product below
+    if (ctx_fail(c, gate_launch(w.sv, l, b, k, k, tau, w.keff, c->stream, &c->launches), "gate")) return DEFL_ERR_CUDA;
     GemmDesc g = gemm_desc_zero();
     g.batch = b; g.M = m; g.N = n;
     g.aux = G; g.ld_aux = n; g.batch_aux = (long long)m * n; g.aux_dtype = dtype;
@@ -476,11 +482,11 @@ int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int 
                                            c->stream, &c->launches), "split P"))
         return DEFL_ERR_CUDA;
       if (ctx_fail(c, split_concat3_launch(right, (long long)n * k, k, b, n, k, kp, w.sv, l, nullptr, 1.f, 0.f, 1, w.Wc,
-                                           c->stream, &c->launches), "split W diag(s)"))
+                                           c->stream, &c->launches, w.keff), "split W diag(s)"))
         return DEFL_ERR_CUDA;
     } else {
       if (ctx_fail(c, scale_cols_launch(right, (long long)n * k, k, b, n, k, w.sv, l, nullptr, 1.f, 0.f, w.Ws,
-                                        (long long)n * k, k, c->stream, &c->launches), "W diag(s)"))
+                                        (long long)n * k, k, c->stream, &c->launches, w.keff), "W diag(s)"))
         return DEFL_ERR_CUDA;
       g.K[0] = k;
       g.A[0] = left; g.sa_i[0] = k; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * k; g.in_dtype = F32;
@@ -497,10 +503,10 @@ int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int 
     const float pad = (mode == DEFL_RESTORE_PADDED) ? 1.f / gamma : 0.f;
     if (tensor_defl) {
       if (ctx_fail(c, split_concat3_launch(right, (long long)n * k, k, b, n, k, kp, w.sv, l, w.inv_rho, -1.f, pad, 1, w.Wc,
-                                           c->stream, &c->launches), "split W diag(coef)"))
+                                           c->stream, &c->launches, w.keff), "split W diag(coef)"))
         return DEFL_ERR_CUDA;
     } else if (ctx_fail(c, scale_cols_launch(right, (long long)n * k, k, b, n, k, w.sv, l, w.inv_rho, -1.f, pad, w.Ws,
-                                             (long long)n * k, k, c->stream, &c->launches), "W diag(coef)")) {
+                                             (long long)n * k, k, c->stream, &c->launches, w.keff), "W diag(coef)")) {
       return DEFL_ERR_CUDA;
     }
     g.epilogue = EPI_AUX_PLUS; g.partials = nullptr;
@@ -582,13 +588,16 @@ int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int 
     if (tensor_restore) {
       // w.Pc still holds the split left factor from the deflation stage; rebuild the right one unscaled
       if (ctx_fail(c, split_concat3_launch(right, (long long)n * k, k, b, n, k, kp, nullptr, 0, nullptr, 0.f, 0.f, 1, w.Wc,
-                                           c->stream, &c->launches), "split W"))
+                                           c->stream, &c->launches, w.keff), "split W"))
         return DEFL_ERR_CUDA;
       if ((rc = run_gemm(c, g, DEFL_ENGINE_TENSOR, "restore (tensor)"))) return rc;
     } else {
+      if (ctx_fail(c, scale_cols_launch(right, (long long)n * k, k, b, n, k, w.sv, l, nullptr, 0.f, 1.f, w.Ws,
+                                        (long long)n * k, k, c->stream, &c->launches, w.keff), "W (gated)"))
+        return DEFL_ERR_CUDA;
       g.K[0] = k;
       g.A[0] = left; g.sa_i[0] = k; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * k; g.in_dtype = F32;
-      g.B[0] = right; g.sb_k[0] = 1; g.sb_j[0] = k; g.batch_b[0] = (long long)n * k; g.b_dtype = F32;
+      g.B[0] = w.Ws; g.sb_k[0] = 1; g.sb_j[0] = k; g.batch_b[0] = (long long)n * k; g.b_dtype = F32;
       if ((rc = run_gemm(c, g, DEFL_ENGINE_SIMT, "restore"))) return rc;
     }
   }
@@ -601,6 +610,11 @@ int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int 
     if (info->rho &&
         ctx_fail(c, cudaMemcpyAsync(info->rho, w.rho, (size_t)b * sizeof(float), cudaMemcpyDeviceToDevice, c->stream), "copy rho"))
       return DEFL_ERR_CUDA;
+    if (info->k_used) {
+      if (k == 0 && ctx_fail(c, fill_int_launch(w.keff, b, 0, c->stream, &c->launches), "k_used")) return DEFL_ERR_CUDA;
+      if (ctx_fail(c, cudaMemcpyAsync(info->k_used, w.keff, (size_t)b * sizeof(int), cudaMemcpyDeviceToDevice, c->stream), "copy k_used"))
+        return DEFL_ERR_CUDA;
+    }
     if (info->status) {
       // fold the engine's device-wait word into every matrix's status
       if (ctx_fail(c, or_status_launch(w.status, b, c->wait_status, c->stream, &c->launches), "status"))

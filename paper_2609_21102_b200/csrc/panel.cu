@@ -426,22 +426,24 @@ cudaError_t rho_finalize_launch(const double* partial, int nper, int batch, floa
 // Out[b, rows, k] = In[b, rows, (ld_in)] * diag(coef): coef_t = c0 * s[b,t] * (use_inv ? inv_rho[b] : 1) + c1
 __global__ void scale_cols_kernel(const float* __restrict__ In, long long in_bs, int ld_in, int rows, int k,
                                   const float* __restrict__ s, int ld_s, const float* __restrict__ inv_rho, float c0,
-                                  float c1, float* __restrict__ Out, long long out_bs, int ld_out) {
+                                  float c1, float* __restrict__ Out, long long out_bs, int ld_out,
+                                  const int* __restrict__ keff) {
   const int bz = blockIdx.y;
   const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= (long long)rows * k) return;
   const int r = (int)(e / k), t = (int)(e % k);
-  const float sc = c0 * s[(long long)bz * ld_s + t] * (inv_rho ? inv_rho[bz] : 1.f) + c1;
+  float sc = c0 * s[(long long)bz * ld_s + t] * (inv_rho ? inv_rho[bz] : 1.f) + c1;
+  if (keff && t >= keff[bz]) sc = 0.f;     // column not deflated for this matrix (gate)
   Out[(long long)bz * out_bs + (long long)r * ld_out + t] = In[(long long)bz * in_bs + (long long)r * ld_in + t] * sc;
 }
 
 cudaError_t scale_cols_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int k, const float* s,
                               int ld_s, const float* inv_rho, float c0, float c1, float* Out, long long out_bs,
-                              int ld_out, cudaStream_t st, long long* launches) {
+                              int ld_out, cudaStream_t st, long long* launches, const int* keff) {
   if (k <= 0) return cudaSuccess;
   const long long tot = (long long)rows * k;
   scale_cols_kernel<<<dim3((unsigned)((tot + 255) / 256), batch), 256, 0, st>>>(In, in_bs, ld_in, rows, k, s, ld_s,
-                                                                               inv_rho, c0, c1, Out, out_bs, ld_out);
+                                                                               inv_rho, c0, c1, Out, out_bs, ld_out, keff);
   if (launches) ++*launches;
   return cudaGetLastError();
 }
@@ -611,13 +613,14 @@ cudaError_t split_panel_launch(const float* In, long long in_bs, int ld_in, int 
 // Column t is scaled by  c0 * s[b,t] * (inv_rho ? inv_rho[b] : 1) + c1  when s is given.
 __global__ void split_concat3_kernel(const float* __restrict__ In, long long in_bs, int ld_in, int rows, int k, int kp,
                                      const float* __restrict__ s, int ld_s, const float* __restrict__ inv_rho, float c0,
-                                     float c1, int pattern, __nv_bfloat16* __restrict__ Out) {
+                                     float c1, int pattern, __nv_bfloat16* __restrict__ Out,
+                                     const int* __restrict__ keff) {
   const int bz = blockIdx.y;
   const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= (long long)rows * kp) return;
   const int r = (int)(e / kp), t = (int)(e % kp);
   float x = 0.f;
-  if (t < k) {
+  if (t < k && !(keff && t >= keff[bz])) {
     x = In[(long long)bz * in_bs + (long long)r * ld_in + t];
     if (s) x *= c0 * s[(long long)bz * ld_s + t] * (inv_rho ? inv_rho[bz] : 1.f) + c1;
   }
@@ -631,10 +634,35 @@ __global__ void split_concat3_kernel(const float* __restrict__ In, long long in_
 
 cudaError_t split_concat3_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int k, int kp,
                                  const float* s, int ld_s, const float* inv_rho, float c0, float c1, int pattern,
-                                 __nv_bfloat16* Out, cudaStream_t st, long long* launches) {
+                                 __nv_bfloat16* Out, cudaStream_t st, long long* launches, const int* keff) {
   const long long tot = (long long)rows * kp;
   split_concat3_kernel<<<dim3((unsigned)((tot + 255) / 256), batch), 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s,
-                                                                                  inv_rho, c0, c1, pattern, Out);
+                                                                                  inv_rho, c0, c1, pattern, Out, keff);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+// The deflation gate of Algorithms 1 and 2 on the estimated magnitudes s[b, 0..] (descending in magnitude):
+//   tau <= 0: keff = window (deflate exactly the requested number);
+//   tau > 0 : if |s_window| < tau |s_1| then keff = #{i < kmax : |s_i| > tau |s_1|}, else keff = 0.
+__global__ void gate_kernel(const float* __restrict__ s, int ld_s, int batch, int window, int kmax, float tau,
+                            int* __restrict__ keff) {
+  const int bz = blockIdx.x * blockDim.x + threadIdx.x;
+  if (bz >= batch) return;
+  const float* sb = s + (long long)bz * ld_s;
+  int k = window;
+  if (tau > 0.f && window > 0) {
+    const float s1 = fabsf(sb[0]);
+    k = 0;
+    if (fabsf(sb[window - 1]) < tau * s1)
+      for (int i = 0; i < kmax; ++i) if (fabsf(sb[i]) > tau * s1) k = i + 1;
+  }
+  keff[bz] = k;
+}
+
+cudaError_t gate_launch(const float* s, int ld_s, int batch, int window, int kmax, float tau, int* keff, cudaStream_t st,
+                        long long* launches) {
+  gate_kernel<<<(batch + 127) / 128, 128, 0, st>>>(s, ld_s, batch, window, kmax, tau, keff);
   if (launches) ++*launches;
   return cudaGetLastError();
 }

@@ -23,7 +23,7 @@ cudaError_t rho_finalize_launch(const double* partial, int nper, int batch, floa
                                 float* inv_rho2, int* status, cudaStream_t st, long long* launches);
 cudaError_t scale_cols_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int k, const float* s,
                               int ld_s, const float* inv_rho, float c0, float c1, float* Out, long long out_bs,
-                              int ld_out, cudaStream_t st, long long* launches);
+                              int ld_out, cudaStream_t st, long long* launches, const int* keff = nullptr);
 cudaError_t scale_launch(const void* In, int in_dt, void* Out, int out_dt, int batch, long long count,
                          const float* scale, cudaStream_t st, long long* launches, int round_tf32 = 0);
 cudaError_t fill_gaussian_launch(void* dst, long long count, int dtype, unsigned long long seed, long long per_stream,
@@ -38,7 +38,9 @@ cudaError_t split_panel_launch(const float* In, long long in_bs, int ld_in, int 
                                __nv_bfloat16* hi, __nv_bfloat16* lo, cudaStream_t st, long long* launches);
 cudaError_t split_concat3_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int k, int kp,
                                  const float* s, int ld_s, const float* inv_rho, float c0, float c1, int pattern,
-                                 __nv_bfloat16* Out, cudaStream_t st, long long* launches);
+                                 __nv_bfloat16* Out, cudaStream_t st, long long* launches, const int* keff = nullptr);
+cudaError_t gate_launch(const float* s, int ld_s, int batch, int window, int kmax, float tau, int* keff, cudaStream_t st,
+                        long long* launches);
 }  // namespace defl
 
 namespace defl {

@@ -195,9 +195,11 @@ __global__ void split_tf32_kernel(const float* __restrict__ X, float* __restrict
 }
 
 // out[t] = f(lam[t]) per column scale helpers: mode 0: lambda, 1: sign(lambda)/gamma, 2: max(lambda, 0); negated if neg
-__global__ void ritz_scale_kernel(const float* __restrict__ lam, int k, int mode, float gamma, int neg, float* __restrict__ out) {
+__global__ void ritz_scale_kernel(const float* __restrict__ lam, int k, int mode, float gamma, int neg, float* __restrict__ out,
+                                  const int* __restrict__ keff) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= k) return;
+  if (t >= keff[0]) { out[t] = 0.f; return; }     // not in the deflated set (gate)
   const float l = lam[t];
   float v = l;
   if (mode == 1) v = (l > 0.f ? 1.f : (l < 0.f ? -1.f : 0.f)) / gamma;
@@ -217,6 +219,7 @@ struct PsdWs {
   int* done; double* beta_prev;
   double* npart; float* theta; float* inv_theta; float* dummy;
   int* status;
+  int* keff;        // [1] size of the deflated set (gate)
   float* start;     // [n] generated Lanczos start vector
   size_t bytes;
 };
@@ -251,6 +254,7 @@ static PsdWs carve_psd(void* base, int n, int K) {
   w.npart = cv.take<double>(1184);
   w.theta = cv.take<float>(1); w.inv_theta = cv.take<float>(1); w.dummy = cv.take<float>(S * S);
   w.status = cv.take<int>(1);
+  w.keff = cv.take<int>(1);
   w.start = cv.take<float>(n);
   w.bytes = cv.off;
   return w;
@@ -297,7 +301,7 @@ static int estimate_scale(defl_ctx* c, const float* A, int n, int norm_mode, con
 // C = aux_scale * aux + alpha * U diag(coef) U^T  (rank-k symmetric update, exact fp32 products)
 static int rank_update(defl_ctx* c, const PsdWs& w, int n, int K, int k, int coef_mode, float gamma, int neg,
                        const float* aux, float aux_scale, const float* aux_scale_dev, float* C, int round_tf32 = 0) {
-  ritz_scale_kernel<<<1, 64, 0, c->stream>>>(w.lam, k, coef_mode, gamma, neg, w.coef);
+  ritz_scale_kernel<<<1, 64, 0, c->stream>>>(w.lam, k, coef_mode, gamma, neg, w.coef, w.keff);
   ++c->launches;
   if (ctx_fail(c, cudaGetLastError(), "ritz scale")) return DEFL_ERR_CUDA;
   if (ctx_fail(c, scale_cols_launch(w.U, 0, K, 1, n, k, w.coef, K, nullptr, 1.f, 0.f, w.Us, 0, K, c->stream, &c->launches), "U diag"))
@@ -345,6 +349,9 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
   const int engine = (engine_opt == DEFL_ENGINE_SIMT) ? DEFL_ENGINE_SIMT : DEFL_ENGINE_TENSOR;
   const int sym = (opts && opts->exploit_symmetry) ? 1 : 0;
   const bool deflate = (k > 0) && !(opts && opts->warmup);
+  const float tau = opts ? opts->tau : 0.f;
+  // with the gate the deflated set is {i : |lambda_i| > tau |lambda_1|} among all K Ritz values; without it, the first k
+  const int kcols = (deflate && tau > 0.f) ? K : k;
   // iterates that feed tf32 products are stored already rounded to nearest tf32: the tensor core would
   // otherwise truncate them, which biases every product towards zero
   const int tf32_round = (engine == DEFL_ENGINE_TENSOR) ? 1 : 0;
@@ -381,7 +388,8 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
   // ---- stage 1: R = Z - sum_I lambda_i u_i u_i^T (line 5) -------------------------------------------
   const float* Rm = Z;
   if (deflate) {
-    if ((rc = rank_update(c, w, n, K, k, 0, gamma, 1, Z, 1.f, nullptr, w.R))) return rc;
+    if (ctx_fail(c, gate_launch(w.lam, K, 1, k, K, tau, w.keff, c->stream, &c->launches), "gate")) return DEFL_ERR_CUDA;
+    if ((rc = rank_update(c, w, n, K, kcols, 0, gamma, 1, Z, 1.f, nullptr, w.R))) return rc;
     Rm = w.R;
   }
   ctx_stage_mark(c);
@@ -399,7 +407,7 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
   float* bufs[2] = {w.Xa, w.Xb};
   int cur = 0;
   if (deflate) {
-    if ((rc = rank_update(c, w, n, K, k, 1, gamma, 0, Rm, 1.f, w.inv_theta, bufs[cur], tf32_round))) return rc;
+    if ((rc = rank_update(c, w, n, K, kcols, 1, gamma, 0, Rm, 1.f, w.inv_theta, bufs[cur], tf32_round))) return rc;
   } else {
     if (ctx_fail(c, scale_launch(Rm, F32, bufs[cur], F32, 1, (long long)n * n, w.inv_theta, c->stream, &c->launches, tf32_round), "normalise"))
       return DEFL_ERR_CUDA;
@@ -451,7 +459,7 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
     g.epilogue = EPI_AUX_PLUS; g.aux_scale = 0.5f; g.alpha = 0.5f;
     if ((rc = run_gemm(c, g, gemm_tc_supported(g) ? engine : DEFL_ENGINE_SIMT, "R g(X0)"))) return rc;
     if (deflate) {
-      if ((rc = rank_update(c, w, n, K, k, 2, gamma, 0, P, 1.f, nullptr, P))) return rc;
+      if ((rc = rank_update(c, w, n, K, kcols, 2, gamma, 0, P, 1.f, nullptr, P))) return rc;
     }
     symmetrise_kernel<<<dim3((n + 31) / 32, (n + 31) / 32), 256, 0, c->stream>>>(P, n);
     ++c->launches;
@@ -474,6 +482,11 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
     if (info->rho &&
         ctx_fail(c, cudaMemcpyAsync(info->rho, w.theta, sizeof(float), cudaMemcpyDeviceToDevice, c->stream), "copy theta"))
       return DEFL_ERR_CUDA;
+    if (info->k_used) {
+      if (!deflate && ctx_fail(c, fill_int_launch(w.keff, 1, 0, c->stream, &c->launches), "k_used")) return DEFL_ERR_CUDA;
+      if (ctx_fail(c, cudaMemcpyAsync(info->k_used, w.keff, sizeof(int), cudaMemcpyDeviceToDevice, c->stream), "copy k_used"))
+        return DEFL_ERR_CUDA;
+    }
     if (info->status) {
       if (ctx_fail(c, or_status_launch(w.status, 1, c->wait_status, c->stream, &c->launches), "status")) return DEFL_ERR_CUDA;
       if (ctx_fail(c, cudaMemcpyAsync(info->status, w.status, sizeof(int), cudaMemcpyDeviceToDevice, c->stream), "copy status"))

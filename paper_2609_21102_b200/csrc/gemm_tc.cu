@@ -3,21 +3,31 @@
 //   warp 0      TMA producer: cp.async.bulk.tensor loads of the A and B operand tiles into a ring of
 //               128-byte-swizzled shared-memory stages, signalled through mbarriers
 //   warp 1      allocates tensor memory and issues tcgen05.mma (one elected lane), fp32 accumulators
-//               in tensor memory, two accumulator buffers so that the epilogue of tile i overlaps the
-//               products of tile i+1
+//               in tensor memory
 //   warps 2..9  epilogue: tcgen05.ld of the accumulator (two warps per 32-lane quarter, alternating 32-column
-//               blocks), the element-wise epilogue (store / polynomial / residual / norm partials), global stores
+//               blocks), the element-wise epilogue (store / polynomial / residual / norm partials), global
+//               accesses coalesced through a per-warp staging buffer in shared memory
 //
-// A tile is 128 x BN outputs (BN chosen per call, a multiple of 16 up to 256), K is walked in blocks of
-// 128 bytes (64 bf16 or 32 tf32 values). Either operand may be K-major (K contiguous in global memory)
-// or MN-major; the shared-memory matrix descriptors and the instruction descriptor are built to match.
-// No cluster launch and no multicast: every CTA loads its own operands. Every wait is bounded: when one
-// runs out the kernel raises DEFL_ST_DEVICE_WAIT in the status word, stops waiting and drains.
+// Tile forms (BN = tile width, a multiple of 16 up to 256; K is walked in blocks of 128 bytes = 64 bf16 or
+// 32 tf32 values):
+//   M <= 128    one CTA, 128 x BN tile, two accumulator buffers (epilogue of tile i overlaps tile i+1)
+//   M >  128    a cluster of two CTAs per 256 x BN tile (tcgen05 cta_group::2): each CTA stages 128 rows of A
+//               and half of the B columns, the leader CTA issues one 256-row product for both, each CTA holds
+//               its 128 accumulator rows in its own tensor memory, two accumulator buffers. A pipeline stage
+//               covers two K blocks: the cost of one step of the two issuing threads (barrier wait, four
+//               products at ~75 cycles of issue each, commit) otherwise exceeds the 512 cycles the tensor
+//               pipe needs per K block. DEFL_TC_PAIR=0 selects the older single-CTA form of the 256-row tile
+//               (two 128-row halves sharing the B tile, one accumulator buffer).
+// Either operand may be K-major (K contiguous in global memory) or MN-major; the shared-memory matrix
+// descriptors and the instruction descriptor are built to match. No multicast copies: every CTA loads its own
+// operands. Every wait is bounded: when one runs out the kernel raises DEFL_ST_DEVICE_WAIT in the status word,
+// stops waiting and drains.
 #include "common.cuh"
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include <mutex>
 #include <cstdlib>
+#include <cstdio>
 
 namespace defl {
 
@@ -38,10 +48,12 @@ struct TcParams {
   int aux_prefetch;
   int nseg;
   int b_split;                 // 2: B is the sum of two operands (tmB[0] + tmB[1]) that share A; else 1
-  int kblocks[2];              // K blocks per segment
+  int kblocks[2];              // pipeline steps per segment (a step covers `ksub` K blocks of 128 bytes)
+  int ksub;                    // K blocks per pipeline stage (1 or 2)
   int M, N, batch;
   int BN;                      // tile width (UMMA N)
   int tile_m;                  // 128 or 256 rows per tile
+  int pair;                    // 1: a cluster of two CTAs per 256-row tile (tcgen05 cta_group::2), each CTA 128 rows
   int tiles_m, tiles_n;
   int tiles_per_matrix;        // tiles enumerated per matrix (fewer than tiles_m * tiles_n for symmetric output)
   long long total_tiles;
@@ -119,6 +131,34 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
       : "memory");
 }
 
+// Pair mode (two CTAs of a cluster drive one tcgen05.mma.cta_group::2): the copy lands in the executing CTA's
+// shared memory, its completion is counted on an mbarrier that may live in the peer CTA (a shared::cluster
+// address). No multicast: every CTA fetches its own operand halves.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* tm, uint32_t bar_cluster, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // asks the memory system to bring one tile of a tensor into L2 (no shared memory, no completion to wait for)
 __device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* tm, int c0, int c1, int c2) {
   asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
@@ -134,6 +174,15 @@ __device__ __forceinline__ void tmem_relinquish() {
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -153,6 +202,30 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t adesc, uint64_t b
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
   }
+}
+// 256-row product of a CTA pair: each CTA supplies 128 rows of A and half of the B columns from its own shared
+// memory (same offsets in both), and receives its 128 rows of the accumulator in its own tensor memory
+template <int KIND_TF32>
+__device__ __forceinline__ void umma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  if (KIND_TF32) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  }
+}
+// pair mode: arrives on the mbarrier at this shared-memory offset in BOTH CTAs of the pair
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
 }
 // arrives on the mbarrier once every tcgen05.mma issued so far by this thread has completed
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -236,7 +309,7 @@ __device__ __forceinline__ TileInfo tile_info(const TcParams& p, long long tile)
   t.halves = 1;
   if (p.tile_m == 256 && p.M - row0 > 128 && !(p.symmetric && col_end <= row0 + 128)) t.halves = 3;
   int rem = p.N - t.tn * p.BN;
-  rem = (rem + 15) & ~15;
+  rem = p.pair ? ((rem + 31) & ~31) : ((rem + 15) & ~15);    // a pair splits the columns in two halves of 16k
   t.n_eff = rem < p.BN ? rem : p.BN;
   return t;
 }
@@ -493,7 +566,7 @@ __device__ __forceinline__ void epilogue_half(const TcParams& p, uint32_t taddr,
   }
 }
 
-template <int KIND_TF32, int BSPLIT>
+template <int KIND_TF32, int BSPLIT, int PAIR>
 __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
@@ -505,23 +578,34 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzled tiles need 1024-byte alignment
-  const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
+  const uint32_t sub_bytes = p.a_stage_bytes + p.b_stage_bytes;      // one K block of A and B
+  const uint32_t stage_bytes = sub_bytes * (uint32_t)p.ksub;
   const int total_kblocks = p.kblocks[0] + (p.nseg > 1 ? p.kblocks[1] : 0);
-  const uint32_t nacc = (p.tile_m == 256) ? 1u : 2u;
+  // Pair mode: CTA 0 of the cluster (the leader) issues the products for both CTAs and owns the barriers that
+  // gate them (full_bar, acc_empty_bar); empty_bar and acc_full_bar exist in both CTAs and are signalled in both
+  // by one commit. Every CTA loads, and writes out, its own 128 rows.
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+  const long long tile0 = PAIR ? (long long)(blockIdx.x >> 1) : (long long)blockIdx.x;
+  const long long tile_step = PAIR ? (long long)(gridDim.x >> 1) : (long long)gridDim.x;
+  const uint32_t nacc = (!PAIR && p.tile_m == 256) ? 1u : 2u;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&acc_full_bar[a]), 1); mbar_init(smem_u32(&acc_empty_bar[a]), EPI_WARPS); }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(smem_u32(&acc_full_bar[a]), 1);
+      mbar_init(smem_u32(&acc_empty_bar[a]), PAIR ? 2 * EPI_WARPS : EPI_WARPS);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(&tmem_base_slot), 512);
-    tmem_relinquish();
+    if (PAIR) { tmem_alloc_pair(smem_u32(&tmem_base_slot), 512); tmem_relinquish_pair(); }
+    else { tmem_alloc(smem_u32(&tmem_base_slot), 512); tmem_relinquish(); }
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();      // the peer's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
 
@@ -529,50 +613,88 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       uint32_t stage = 0, phase = 0;
-      for (long long tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+      // everything the inner loop needs sits in registers: this one thread's issue rate bounds the whole pipeline
+      // when a K block is short (a parameter re-read or an integer division per copy costs more than the copy)
+      const int arow = PAIR ? (int)rank * 128 : 0;              // this CTA's rows within the tile
+      const int kstep = KBYTES / p.esize;
+      const bool a_mn = p.a_mn_major != 0, b_mn = p.b_mn_major != 0;
+      const uint32_t a_boxes = p.a_boxes, b_boxes = p.b_boxes;
+      const uint32_t a_box_bytes = p.a_box_bytes, b_box_bytes = p.b_box_bytes;
+      const int a_box_rows = (int)p.a_box_rows, b_box_rows = (int)p.b_box_rows;
+      const uint32_t a_stage_bytes = p.a_stage_bytes, b_split_bytes = p.b_split_bytes;
+      const uint32_t nstages = (uint32_t)p.stages;
+      const int ksub = p.ksub;
+      const uint32_t tx_bytes = PAIR ? 2u * stage_bytes : stage_bytes;   // a pair counts both CTAs' copies on the leader's barrier
+      const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
+      const uint32_t full0_sig = PAIR ? map_to_cta(full0, 0) : full0;    // the barrier the copies signal
+      const int BN = p.BN, tile_m = p.tile_m, nseg = p.nseg;
+      const bool aux_prefetch = p.aux_prefetch != 0;
+      for (long long tile = tile0; tile < p.total_tiles; tile += tile_step) {
         const TileInfo t = tile_info(p, tile);
         if (t.skip) continue;
         // the epilogues read the matching tile of `aux` with plain loads: start moving it from HBM into L2
         // well ahead (AUX_AHEAD tiles of this CTA; short main loops leave no time otherwise)
-        if (p.aux_prefetch) {
-          if (tile == (long long)blockIdx.x) {
+        if (aux_prefetch) {
+          if (tile == tile0) {
             for (int d = 0; d < AUX_AHEAD; ++d) {
-              const long long tp = tile + (long long)d * gridDim.x;
+              const long long tp = tile + (long long)d * tile_step;
               if (tp >= p.total_tiles) break;
               const TileInfo u = tile_info(p, tp);
-              if (!u.skip) tma_prefetch_3d(&p.tmAux, u.tn * p.BN, u.tm * p.tile_m, u.bz);
+              if (!u.skip) tma_prefetch_3d(&p.tmAux, u.tn * BN, u.tm * tile_m + arow, u.bz);
             }
           }
-          const long long tp = tile + (long long)AUX_AHEAD * gridDim.x;
+          const long long tp = tile + (long long)AUX_AHEAD * tile_step;
           if (tp < p.total_tiles) {
             const TileInfo u = tile_info(p, tp);
-            if (!u.skip) tma_prefetch_3d(&p.tmAux, u.tn * p.BN, u.tm * p.tile_m, u.bz);
+            if (!u.skip) tma_prefetch_3d(&p.tmAux, u.tn * BN, u.tm * tile_m + arow, u.bz);
           }
         }
-        for (int seg = 0; seg < p.nseg; ++seg) {
-          for (int kb = 0; kb < p.kblocks[seg]; ++kb) {
-            if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, &abort_flag, p.status)) break;
-            const uint32_t fb = smem_u32(&full_bar[stage]);
-            mbar_expect_tx(fb, stage_bytes);
-            const uint32_t sa = smem_base + stage * stage_bytes;
-            const uint32_t sb = sa + p.a_stage_bytes;
-            const int k0 = kb * (KBYTES / p.esize);
-            for (uint32_t bx = 0; bx < p.a_boxes; ++bx) {
-              const int mn0 = t.tm * p.tile_m + (int)(bx * p.a_box_rows);
-              if (p.a_mn_major) tma_load_3d(sa + bx * p.a_box_bytes, &p.tmA[seg], fb, mn0, k0, t.bz);
-              else tma_load_3d(sa + bx * p.a_box_bytes, &p.tmA[seg], fb, k0, mn0, t.bz);
-            }
+        const int a_mn0 = t.tm * tile_m + arow;
+        const int b_mn0 = t.tn * BN + (PAIR ? (int)rank * (t.n_eff >> 1) : 0);   // a pair: this CTA's half of the columns
+        const int bz = t.bz;
+        for (int seg = 0; seg < nseg; ++seg) {
+          const CUtensorMap* tma = &p.tmA[seg];
+          const CUtensorMap* tmb0 = &p.tmB[BSPLIT > 1 ? 0 : seg];
+          const CUtensorMap* tmb1 = &p.tmB[1];
+          const int nkb = p.kblocks[seg];
+          int k0 = 0;
+          for (int kb = 0; kb < nkb; ++kb) {
+            if (!mbar_wait(empty0 + 8u * stage, phase ^ 1u, &abort_flag, p.status)) break;
+            if (!PAIR || rank == 0) mbar_expect_tx(full0 + 8u * stage, tx_bytes);
+            const uint32_t fb = full0_sig + 8u * stage;
+            // (a K block past the end of K is filled with zeros by the copy engine and adds nothing)
+            for (int sub = 0; sub < ksub; ++sub, k0 += kstep) {
+              const uint32_t sa = smem_base + stage * stage_bytes + (uint32_t)sub * sub_bytes;
+              const uint32_t sb = sa + a_stage_bytes;
+              for (uint32_t bx = 0; bx < a_boxes; ++bx) {
+                const int mn0 = a_mn0 + (int)bx * a_box_rows;
+                const uint32_t dst = sa + bx * a_box_bytes;
+                if (PAIR) {
+                  if (a_mn) tma_load_3d_pair(dst, tma, fb, mn0, k0, bz);
+                  else tma_load_3d_pair(dst, tma, fb, k0, mn0, bz);
+                } else {
+                  if (a_mn) tma_load_3d(dst, tma, fb, mn0, k0, bz);
+                  else tma_load_3d(dst, tma, fb, k0, mn0, bz);
+                }
+              }
 #pragma unroll
-            for (int sp = 0; sp < BSPLIT; ++sp) {
-              const CUtensorMap* tmb = &p.tmB[BSPLIT > 1 ? sp : seg];
-              const uint32_t sbs = sb + (uint32_t)sp * p.b_split_bytes;
-              for (uint32_t bx = 0; bx < p.b_boxes; ++bx) {
-                const int mn0 = t.tn * p.BN + (int)(bx * p.b_box_rows);
-                if (p.b_mn_major) tma_load_3d(sbs + bx * p.b_box_bytes, tmb, fb, mn0, k0, t.bz);
-                else tma_load_3d(sbs + bx * p.b_box_bytes, tmb, fb, k0, mn0, t.bz);
+              for (int sp = 0; sp < BSPLIT; ++sp) {
+                const CUtensorMap* tmb = sp ? tmb1 : tmb0;
+                const uint32_t sbs = sb + (uint32_t)sp * b_split_bytes;
+                for (uint32_t bx = 0; bx < b_boxes; ++bx) {
+                  const int mn0 = b_mn0 + (int)bx * b_box_rows;
+                  const uint32_t dst = sbs + bx * b_box_bytes;
+                  if (PAIR) {
+                    if (b_mn) tma_load_3d_pair(dst, tmb, fb, mn0, k0, bz);
+                    else tma_load_3d_pair(dst, tmb, fb, k0, mn0, bz);
+                  } else {
+                    if (b_mn) tma_load_3d(dst, tmb, fb, mn0, k0, bz);
+                    else tma_load_3d(dst, tmb, fb, k0, mn0, bz);
+                  }
+                }
               }
             }
-            if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
+            if (++stage == nstages) { stage = 0; phase ^= 1u; }
           }
           if (abort_flag) break;
         }
@@ -581,7 +703,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
       uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
       // descriptor start addresses advance in units of 16 bytes
       const uint32_t a_kstep16 = (p.a_mn_major ? (uint32_t)(32 / p.esize) * 128u : 32u) >> 4;   // per UMMA K step
@@ -590,38 +712,52 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       const uint64_t b_hi = smem_desc_hi(p.b_mn_major ? p.b_box_bytes : 16u, 1024u);
       const uint32_t a_half16 = (128u * KBYTES) >> 4;   // rows 128..255 of the A tile (either major)
       const uint32_t split16 = p.b_split_bytes >> 4;
-      const uint32_t stage16 = stage_bytes >> 4, a_stage16 = p.a_stage_bytes >> 4, base16 = smem_base >> 4;
-      for (long long tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+      const uint32_t stage16 = stage_bytes >> 4, sub16 = sub_bytes >> 4, a_stage16 = p.a_stage_bytes >> 4, base16 = smem_base >> 4;
+      const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
+      const uint32_t nstages = (uint32_t)p.stages;
+      const int ksub = p.ksub;
+      const uint32_t idesc0 = p.idesc;
+      const bool tall = !PAIR && p.tile_m == 256;
+      for (long long tile = tile0; tile < p.total_tiles; tile += tile_step) {
         const TileInfo t = tile_info(p, tile);
         if (t.skip) continue;
         if (!mbar_wait(smem_u32(&acc_empty_bar[acc]), acc_phase ^ 1u, &abort_flag, p.status)) break;
         tc_fence_after();
-        const uint32_t idesc = p.idesc | ((uint32_t)(t.n_eff >> 3) << 17);
-        const uint32_t d0 = tmem_base + ((p.tile_m == 256) ? 0u : acc * 256u);
-        const bool two = (t.halves & 2) != 0;
+        const uint32_t idesc = idesc0 | ((uint32_t)(t.n_eff >> 3) << 17);
+        const uint32_t d0 = tmem_base + (tall ? 0u : acc * 256u);
+        const bool two = !PAIR && (t.halves & 2) != 0;
         bool ok = true;
+        uint32_t accum = 0;                                   // the first product of a tile overwrites the accumulator
         for (int kb = 0; kb < total_kblocks; ++kb) {
-          if (!mbar_wait(smem_u32(&full_bar[stage]), phase, &abort_flag, p.status)) { ok = false; break; }
+          if (!mbar_wait(full0 + 8u * stage, phase, &abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa16 = base16 + stage * stage16;
-          const uint32_t sb16 = sa16 + a_stage16;
+          for (int sub = 0; sub < ksub; ++sub) {
+            const uint32_t sa16 = base16 + stage * stage16 + (uint32_t)sub * sub16;
+            const uint32_t sb16 = sa16 + a_stage16;
 #pragma unroll
-          for (int kk = 0; kk < KBYTES / 32; ++kk) {
-            const uint64_t adesc = a_hi | (uint64_t)(sa16 + kk * a_kstep16);
-            const uint64_t bdesc = b_hi | (uint64_t)(sb16 + kk * b_kstep16);
-            const uint32_t accum = (kb > 0 || kk > 0) ? 1u : 0u;
-            umma<KIND_TF32>(d0, adesc, bdesc, idesc, accum);
-            if (two) umma<KIND_TF32>(d0 + 256u, adesc + a_half16, bdesc, idesc, accum);
-            if (BSPLIT == 2) {
-              umma<KIND_TF32>(d0, adesc, bdesc + split16, idesc, 1u);
-              if (two) umma<KIND_TF32>(d0 + 256u, adesc + a_half16, bdesc + split16, idesc, 1u);
+            for (int kk = 0; kk < KBYTES / 32; ++kk) {
+              const uint64_t adesc = a_hi | (uint64_t)(sa16 + kk * a_kstep16);
+              const uint64_t bdesc = b_hi | (uint64_t)(sb16 + kk * b_kstep16);
+              if (PAIR) {
+                umma_pair<KIND_TF32>(d0, adesc, bdesc, idesc, accum);
+                if (BSPLIT == 2) umma_pair<KIND_TF32>(d0, adesc, bdesc + split16, idesc, 1u);
+              } else {
+                umma<KIND_TF32>(d0, adesc, bdesc, idesc, accum);
+                if (two) umma<KIND_TF32>(d0 + 256u, adesc + a_half16, bdesc, idesc, accum);
+                if (BSPLIT == 2) {
+                  umma<KIND_TF32>(d0, adesc, bdesc + split16, idesc, 1u);
+                  if (two) umma<KIND_TF32>(d0 + 256u, adesc + a_half16, bdesc + split16, idesc, 1u);
+                }
+              }
+              accum = 1u;
             }
           }
-          umma_commit(smem_u32(&empty_bar[stage]));          // frees the stage once these products are done
-          if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
+          // frees the stage (in both CTAs of a pair) once these products are done
+          if (PAIR) umma_commit_pair(empty0 + 8u * stage); else umma_commit(empty0 + 8u * stage);
+          if (++stage == nstages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        umma_commit(smem_u32(&acc_full_bar[acc]));           // accumulator complete
+        if (PAIR) umma_commit_pair(smem_u32(&acc_full_bar[acc])); else umma_commit(smem_u32(&acc_full_bar[acc]));   // accumulator complete
         if (++acc == nacc) { acc = 0; acc_phase ^= 1u; }
       }
     }
@@ -631,7 +767,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
     const int wsel = (warp - 2) >> 2;       // which of the two warps of that quarter: alternate 32-column blocks
     uint8_t* stg = smem_raw + (smem_base - smem_u32(smem_raw)) + (uint32_t)p.stages * stage_bytes + (uint32_t)(warp - 2) * STAGING_BYTES;
     uint32_t acc = 0, acc_phase = 0;
-    for (long long tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+    const int h_first = PAIR ? (int)rank : 0;
+    const int h_last = PAIR ? (int)rank : ((p.tile_m == 256) ? 1 : 0);
+    for (long long tile = tile0; tile < p.total_tiles; tile += tile_step) {
       const TileInfo t = tile_info(p, tile);
       if (t.skip) continue;
       const int tn = t.tn, tm = t.tm, bz = t.bz;
@@ -641,10 +779,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       float alpha = p.alpha, aux_scale = p.aux_scale;
       if (p.alpha_dev) alpha *= p.alpha_dev[bz];
       if (p.aux_scale_dev) aux_scale *= p.aux_scale_dev[bz];
-      for (int h = 0; h < (p.tile_m == 256 ? 2 : 1); ++h) {
+      for (int h = h_first; h <= h_last; ++h) {
         double sq = 0.0;
         if (t.halves & (1 << h)) {
-          const uint32_t tcol = (p.tile_m == 256) ? (uint32_t)h * 256u : acc * 256u;
+          const uint32_t tcol = (!PAIR && p.tile_m == 256) ? (uint32_t)h * 256u : acc * 256u;
           const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + tcol;
           const int gi0 = tm * p.tile_m + h * 128 + q * 32, gi = gi0 + lane;
           switch (p.epilogue) {
@@ -664,7 +802,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       // release the accumulator buffer
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&acc_empty_bar[acc]));
+      if (lane == 0) {
+        if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty_bar[acc]), 0));
+        else mbar_arrive(smem_u32(&acc_empty_bar[acc]));
+      }
       if (++acc == nacc) { acc = 0; acc_phase ^= 1u; }
     }
   }
@@ -679,9 +820,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
     while (global_ns() - t0 < 2000000ull) { }
   }
   __syncthreads();
+  if (PAIR) cluster_sync_all();      // nothing of this CTA is released while the peer may still signal or read it
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, 512);
+    if (PAIR) tmem_dealloc_pair(tmem_base, 512); else tmem_dealloc(tmem_base, 512);
   }
 }
 
@@ -760,12 +902,26 @@ bool encode_map(CUtensorMap* tm, const void* base, int esize, bool tf32, bool mn
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Tuning overrides for experiments (read per launch): DEFL_TC_BN, DEFL_TC_TILE_M, DEFL_TC_STAGES.
-int choose_bn(int N) {
-  if (const char* e = getenv("DEFL_TC_BN")) { const int v = atoi(e); if (v >= 16 && v <= 256 && v % 16 == 0) return v; }
-  // widest tile; edge tiles only compute the columns that exist (rounded up to 16), so a wide tile wastes
-  // at most 15 columns per tile row
-  const int r = (N + 15) & ~15;
+int choose_bn(int N, bool pair) {
+  const int q = pair ? 32 : 16;
+  if (const char* e = getenv("DEFL_TC_BN")) { const int v = atoi(e); if (v >= q && v <= 256 && v % q == 0) return v; }
+  // widest tile; edge tiles only compute the columns that exist (rounded up to 16, or 32 for a CTA pair), so
+  // a wide tile wastes at most q - 1 columns per tile row
+  const int r = (N + q - 1) & ~(q - 1);
   return r < 256 ? r : 256;
+}
+
+int choose_tile_m_impl(int M) {
+  if (const char* e = getenv("DEFL_TC_TILE_M")) { const int v = atoi(e); if (v == 128 || v == 256) return v; }
+  return M > 128 ? 256 : 128;
+}
+
+// 256-row tiles are computed by a cluster of two CTAs (tcgen05 cta_group::2) unless DEFL_TC_PAIR=0 asks for
+// the single-CTA form (two 128-row halves in one CTA)
+bool choose_pair(int M) {
+  if (choose_tile_m_impl(M) != 256) return false;
+  if (const char* e = getenv("DEFL_TC_PAIR")) return atoi(e) != 0;
+  return true;
 }
 
 }  // namespace
@@ -798,13 +954,10 @@ bool gemm_tc_supported(const GemmDesc& g) {
   return get_encode_fn() != nullptr;
 }
 
-int choose_tile_m(int M) {
-  if (const char* e = getenv("DEFL_TC_TILE_M")) { const int v = atoi(e); if (v == 128 || v == 256) return v; }
-  return M > 128 ? 256 : 128;
-}
+int choose_tile_m(int M) { return choose_tile_m_impl(M); }
 
 int gemm_tc_partials_per_batch(const GemmDesc& g) {
-  const int bn = choose_bn(g.N), tmh = choose_tile_m(g.M);
+  const int bn = choose_bn(g.N, choose_pair(g.M)), tmh = choose_tile_m(g.M);
   return ((g.M + tmh - 1) / tmh) * ((g.N + bn - 1) / bn) * (tmh == 256 ? 2 : 1) * EPI_WARPS;
 }
 
@@ -816,8 +969,9 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   const bool tf32 = (g.in_dtype == F32);
   p.esize = esize;
   p.M = g.M; p.N = g.N; p.batch = g.batch;
-  p.BN = choose_bn(g.N);
   p.tile_m = choose_tile_m(g.M);
+  p.pair = choose_pair(g.M) ? 1 : 0;
+  p.BN = choose_bn(g.N, p.pair != 0);
   p.tiles_m = (g.M + p.tile_m - 1) / p.tile_m;
   p.tiles_n = (g.N + p.BN - 1) / p.BN;
   p.tiles_per_matrix = p.tiles_m * p.tiles_n;
@@ -832,8 +986,9 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   p.nseg = g.nseg;
   OperandPlan pa, pb;
   // when a dimension has extent 1 both strides may look "unit"; prefer K-major
-  if (!plan_operand(g.sa_i[0], g.sa_k[0], p.tile_m, esize, &pa)) return cudaErrorNotSupported;
-  if (!plan_operand(g.sb_j[0], g.sb_k[0], p.BN, esize, &pb)) return cudaErrorNotSupported;
+  // (per CTA: in pair mode each CTA stages 128 rows of A and half of the tile's B columns)
+  if (!plan_operand(g.sa_i[0], g.sa_k[0], p.pair ? 128 : p.tile_m, esize, &pa)) return cudaErrorNotSupported;
+  if (!plan_operand(g.sb_j[0], g.sb_k[0], p.pair ? p.BN / 2 : p.BN, esize, &pb)) return cudaErrorNotSupported;
   p.a_mn_major = pa.mn_major; p.b_mn_major = pb.mn_major;
   p.a_boxes = pa.boxes; p.a_box_bytes = pa.box_bytes; p.a_box_rows = pa.box_rows; p.a_stage_bytes = pa.stage_bytes;
   p.b_split = (g.b_split == 2) ? 2 : 1;
@@ -845,8 +1000,14 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
                     g.batch_b[0], pb.box_rows))
       return cudaErrorInvalidValue;
   }
+  // a pair's K block is half the work per CTA of the single-CTA form, too short to hide the per-step cost of the
+  // two issuing threads (barrier wait, commit): its pipeline steps cover two K blocks when three such stages fit
+  const uint32_t smem_budget = 224 * 1024 - EPI_WARPS * STAGING_BYTES;
+  const uint32_t sub_bytes = p.a_stage_bytes + p.b_stage_bytes;
+  p.ksub = (p.pair && 3u * 2u * sub_bytes <= smem_budget) ? 2 : 1;
+  if (const char* e = getenv("DEFL_TC_KSUB")) { const int v = atoi(e); if ((v == 1 || v == 2) && (uint32_t)v * sub_bytes * 2u <= smem_budget) p.ksub = v; }
   for (int s = 0; s < g.nseg; ++s) {
-    p.kblocks[s] = (g.K[s] + span - 1) / span;
+    p.kblocks[s] = ((g.K[s] + span - 1) / span + p.ksub - 1) / p.ksub;
     if (!encode_map(&p.tmA[s], g.A[s], esize, tf32, pa.mn_major, g.M, g.K[s], g.sa_i[s], g.sa_k[s], g.batch,
                     g.batch_a[s], pa.box_rows))
       return cudaErrorInvalidValue;
@@ -854,8 +1015,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
                     g.batch_b[s], pb.box_rows))
       return cudaErrorInvalidValue;
   }
-  const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
-  const uint32_t smem_budget = 224 * 1024 - EPI_WARPS * STAGING_BYTES;
+  const uint32_t stage_bytes = sub_bytes * (uint32_t)p.ksub;
   int stages = (int)(smem_budget / stage_bytes);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (const char* e = getenv("DEFL_TC_STAGES")) { const int v = atoi(e); if (v >= 2 && v <= stages) stages = v; }
@@ -865,7 +1025,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   const uint32_t fmt = tf32 ? 2u : 1u;
   // (N is filled in per tile by the kernel: edge tiles compute fewer columns)
   p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)p.a_mn_major << 15) | ((uint32_t)p.b_mn_major << 16) |
-            ((uint32_t)(128 >> 4) << 24);
+            ((uint32_t)((p.pair ? 256 : 128) >> 4) << 24);
   p.epilogue = g.epilogue; p.out_dtype = g.out_dtype; p.aux_dtype = g.aux_dtype; p.symmetric = g.symmetric; p.round_tf32 = g.round_tf32;
   p.C = g.C; p.ldc = g.ldc; p.batch_c = g.batch_c;
   p.aux = g.aux; p.ld_aux = g.ld_aux; p.batch_aux = g.batch_aux;
@@ -880,7 +1040,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
       cuuint64_t dims[3] = {(cuuint64_t)g.N, (cuuint64_t)g.M, (cuuint64_t)g.batch};
       cuuint64_t strides[2] = {(cuuint64_t)g.ld_aux * aes, (cuuint64_t)(g.batch == 1 ? g.ld_aux * (long long)g.M : g.batch_aux) * aes};
       // 16-bit types: a full 256-column tile per box; 32-bit types: box columns are capped at 256 elements too
-      cuuint32_t box[3] = {(cuuint32_t)(p.BN < 256 ? p.BN : 256), (cuuint32_t)p.tile_m, 1};
+      cuuint32_t box[3] = {(cuuint32_t)(p.BN < 256 ? p.BN : 256), (cuuint32_t)(p.pair ? 128 : p.tile_m), 1};
       cuuint32_t estr[3] = {1, 1, 1};
       const CUtensorMapDataType dt = (aes == 2) ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
       if (enc && enc(&p.tmAux, dt, 3, const_cast<void*>(g.aux), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -893,8 +1053,46 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
 
   const size_t smem = (size_t)stages * stage_bytes + 1024 + EPI_WARPS * STAGING_BYTES;
   cudaError_t e;
-  auto kern = tf32 ? (p.b_split == 2 ? gemm_tc_kernel<1, 2> : gemm_tc_kernel<1, 1>)
-                   : (p.b_split == 2 ? gemm_tc_kernel<0, 2> : gemm_tc_kernel<0, 1>);
+  if (p.pair) {
+    auto kern = tf32 ? (p.b_split == 2 ? gemm_tc_kernel<1, 2, 1> : gemm_tc_kernel<1, 1, 1>)
+                     : (p.b_split == 2 ? gemm_tc_kernel<0, 2, 1> : gemm_tc_kernel<0, 1, 1>);
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    // how many CTA pairs the device can hold at once (a GPC with an odd number of free SMs leaves one out)
+    static int max_pairs[4][64];   // per kernel variant and device; 0 = not asked yet
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const int variant = (tf32 ? 2 : 0) + (p.b_split == 2 ? 1 : 0);
+    int pairs = (dev >= 0 && dev < 64) ? max_pairs[variant][dev] : 0;
+    if (pairs <= 0) {
+      cfg.gridDim = dim3((unsigned)(num_sms & ~1), 1, 1);
+      int n = 0;
+      e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+      if (e != cudaSuccess) return e;
+      pairs = n > 0 ? n : 1;
+      if (pairs > num_sms / 2) pairs = num_sms / 2;
+      if (dev >= 0 && dev < 64) max_pairs[variant][dev] = pairs;
+      if (getenv("DEFL_TC_DEBUG")) fprintf(stderr, "gemm_tc: %d CTA pairs resident (occupancy query %d), %d stages\n", pairs, n, stages);
+    }
+    long long npairs = p.total_tiles < pairs ? p.total_tiles : pairs;
+    if (npairs < 1) npairs = 1;
+    cfg.gridDim = dim3((unsigned)(2 * npairs), 1, 1);
+    e = cudaLaunchKernelEx(&cfg, kern, p);
+    if (launches) ++*launches;
+    return e != cudaSuccess ? e : cudaGetLastError();
+  }
+  auto kern = tf32 ? (p.b_split == 2 ? gemm_tc_kernel<1, 2, 0> : gemm_tc_kernel<1, 1, 0>)
+                   : (p.b_split == 2 ? gemm_tc_kernel<0, 2, 0> : gemm_tc_kernel<0, 1, 0>);
   e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   long long grid = p.total_tiles < num_sms ? p.total_tiles : num_sms;

@@ -151,8 +151,10 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
   return r;
 }
+// (default semantics, release at CTA scope: what the arrival orders is the tensor-memory read-out, which the
+// tcgen05 fences cover; a cluster-scope release would also wait for every global store of the thread to drain)
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
@@ -425,101 +427,134 @@ __device__ __forceinline__ uint32_t stage_off(int row, int piece, int rowb, int 
   return (uint32_t)(row * rowb + ((piece ^ key) << 4));
 }
 
-template <int EPI, int AES, int OES>
+// Coalesced fetch of one 32 x 32 block of `aux` (rows gi_warp0.., columns gj0..) into a staging buffer, 16 bytes per
+// lane and instruction, whole 64- or 128-byte row segments per warp instruction. The asynchronous form
+// (cp.async) needs no registers for the data, so that the fetch of a warp's next block can be in flight while
+// the current one is processed; rows past M are filled with zeros.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+template <int ES>
+__device__ __forceinline__ void aux_fetch_async(const TcParams& p, int lane, int gi_warp0, int gj0, int bz, uint8_t* stg) {
+  constexpr int rowb = 32 * ES, pp = rowb >> 4, rpi = 32 / pp;     // rpi = rows covered by one warp instruction
+  const uint8_t* abase = reinterpret_cast<const uint8_t*>(p.aux) +
+                         ((size_t)bz * p.batch_aux + (size_t)gi_warp0 * p.ld_aux + gj0) * ES;
+  const int prow = lane / pp, piece = lane % pp;
+  const uint32_t sbase = smem_u32(stg);
+#pragma unroll
+  for (int i = 0; i < pp; ++i) {
+    const int row = prow + rpi * i;
+    const bool ok = gi_warp0 + row < p.M;
+    cp_async16(sbase + stage_off(row, piece, rowb, pp), abase + (size_t)(ok ? row : 0) * p.ld_aux * ES + piece * 16, ok ? 16u : 0u);
+  }
+  cp_async_commit();
+}
+
+// One complete 32 x 32 block whose `aux` values already sit (or are about to land) in `stg`. ES = element size of
+// `aux` and of the output (the same type). Each lane turns its row of the staged block into results 16 bytes at
+// a time, in place; the block then leaves with coalesced 16-byte stores. `pending` = number of cp.async groups
+// that may still be in flight after this block's own (0 or 1).
+template <int EPI, int ES, int PENDING>
 __device__ __forceinline__ void epilogue_block_fast(const TcParams& p, uint32_t taddr, uint8_t* stg, int lane, int gi_warp0,
                                                     int gj0, int bz, float alpha, float aux_scale, double& sq) {
+  constexpr int rowb = 32 * ES, pp = rowb >> 4, rpi = 32 / pp, epp = 16 / ES;   // epp = elements per 16-byte piece
+  const int prow = lane / pp, piece = lane % pp;
   uint32_t r[32];
-  __syncwarp();
   tmem_ld16(taddr, r);
   tmem_ld16(taddr + 16u, r + 16);
-  float x[32];
   if (EPI != EPI_STORE) {
-    constexpr int aes = AES;
-    constexpr int rowb = 32 * aes, pp = rowb >> 4, rpi = 32 / pp;     // rows covered by one warp instruction
-    const uint8_t* abase = reinterpret_cast<const uint8_t*>(p.aux) +
-                           ((size_t)bz * p.batch_aux + (size_t)gi_warp0 * p.ld_aux + gj0) * aes;
-    const int prow = lane / pp, piece = lane % pp;
-    uint4 t[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      if (i < pp) {
-        const int row = prow + rpi * i;
-        t[i] = (gi_warp0 + row < p.M)
-                   ? *reinterpret_cast<const uint4*>(abase + (size_t)row * p.ld_aux * aes + piece * 16)
-                   : make_uint4(0u, 0u, 0u, 0u);
-      }
-    }
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-      if (i < pp) *reinterpret_cast<uint4*>(stg + stage_off(prow + rpi * i, piece, rowb, pp)) = t[i];
-    __syncwarp();
-#pragma unroll
-    for (int pc = 0; pc < 8; ++pc) {
-      if (pc < pp) {
-        const uint4 q = *reinterpret_cast<const uint4*>(stg + stage_off(lane, pc, rowb, pp));
-        if (aes == 2) {
-          const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(&q);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) { const float2 f = __bfloat1622float2(hh[j]); x[(pc & 3) * 8 + 2 * j] = f.x; x[(pc & 3) * 8 + 2 * j + 1] = f.y; }
-        } else {
-          x[pc * 4] = __uint_as_float(q.x); x[pc * 4 + 1] = __uint_as_float(q.y);
-          x[pc * 4 + 2] = __uint_as_float(q.z); x[pc * 4 + 3] = __uint_as_float(q.w);
-        }
-      }
-    }
+    cp_async_wait<PENDING>();
     __syncwarp();
   }
   tmem_ld_wait();
   const int gi = gi_warp0 + lane;
-  float v[32];
+  const bool row_ok = gi < p.M;
+  float sqf = 0.f;
 #pragma unroll
-  for (int j = 0; j < 32; ++j) {
-    const float a = __uint_as_float(r[j]);
-    if (EPI == EPI_STORE) v[j] = alpha * a;
-    else if (EPI == EPI_POLY) v[j] = p.pb * x[j] + p.pc * a + ((gi == gj0 + j) ? p.pa : 0.f);
-    else if (EPI == EPI_AUX_PLUS) v[j] = aux_scale * x[j] + alpha * a;
-    else v[j] = (gi < p.M) ? (x[j] - a) : 0.f;
-  }
-  if (p.round_tf32) {
+  for (int pc = 0; pc < pp; ++pc) {
+    uint4* slot = reinterpret_cast<uint4*>(stg + stage_off(lane, pc, rowb, pp));
+    float x[epp], v[epp];
+    if (EPI != EPI_STORE) {
+      const uint4 q = *slot;
+      if (ES == 2) {
+        const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(&q);
 #pragma unroll
-    for (int j = 0; j < 32; ++j) v[j] = round_to_tf32(v[j]);
-  }
-  if (EPI == EPI_RESID_NORM) {
-    float sqf = 0.f;
+        for (int j = 0; j < epp / 2; ++j) { const float2 f = __bfloat1622float2(hh[j]); x[2 * j] = f.x; x[2 * j + 1] = f.y; }
+      } else {
+        x[0] = __uint_as_float(q.x); x[1] = __uint_as_float(q.y); x[2 % epp] = __uint_as_float(q.z); x[3 % epp] = __uint_as_float(q.w);
+      }
+    }
 #pragma unroll
-    for (int j = 0; j < 32; ++j) sqf = fmaf(v[j], v[j], sqf);
-    sq += (double)sqf;
-    return;
-  }
-  constexpr int oes = OES;
-  constexpr int rowb = 32 * oes, pp = rowb >> 4, rpi = 32 / pp;
-#pragma unroll
-  for (int pc = 0; pc < 8; ++pc) {
-    if (pc < pp) {
+    for (int j = 0; j < epp; ++j) {
+      const int c = pc * epp + j;
+      const float a = __uint_as_float(r[c]);
+      if (EPI == EPI_STORE) v[j] = alpha * a;
+      else if (EPI == EPI_POLY) v[j] = p.pb * x[j] + p.pc * a + ((gi == gj0 + c) ? p.pa : 0.f);
+      else if (EPI == EPI_AUX_PLUS) v[j] = aux_scale * x[j] + alpha * a;
+      else v[j] = row_ok ? (x[j] - a) : 0.f;
+      if (p.round_tf32) v[j] = round_to_tf32(v[j]);
+      if (EPI == EPI_RESID_NORM) sqf = fmaf(v[j], v[j], sqf);
+    }
+    if (EPI != EPI_RESID_NORM) {
       uint4 q;
-      if (oes == 2) {
+      if (ES == 2) {
         __nv_bfloat162* hh = reinterpret_cast<__nv_bfloat162*>(&q);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) hh[j] = __floats2bfloat162_rn(v[(pc & 3) * 8 + 2 * j], v[(pc & 3) * 8 + 2 * j + 1]);
+        for (int j = 0; j < epp / 2; ++j) hh[j] = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
       } else {
-        q = make_uint4(__float_as_uint(v[pc * 4]), __float_as_uint(v[pc * 4 + 1]), __float_as_uint(v[pc * 4 + 2]),
-                       __float_as_uint(v[pc * 4 + 3]));
+        q = make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2 % epp]), __float_as_uint(v[3 % epp]));
       }
-      *reinterpret_cast<uint4*>(stg + stage_off(lane, pc, rowb, pp)) = q;
+      *slot = q;
     }
   }
+  if (EPI == EPI_RESID_NORM) {
+    sq += (double)sqf;
+    __syncwarp();
+    return;
+  }
   __syncwarp();
-  uint8_t* cbase = reinterpret_cast<uint8_t*>(p.C) + ((size_t)bz * p.batch_c + (size_t)gi_warp0 * p.ldc + gj0) * oes;
-  const int prow = lane / pp, piece = lane % pp;
+  uint8_t* cbase = reinterpret_cast<uint8_t*>(p.C) + ((size_t)bz * p.batch_c + (size_t)gi_warp0 * p.ldc + gj0) * ES;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    if (i < pp) {
-      const int row = prow + rpi * i;
-      const uint4 q = *reinterpret_cast<const uint4*>(stg + stage_off(row, piece, rowb, pp));
-      if (gi_warp0 + row < p.M) *reinterpret_cast<uint4*>(cbase + (size_t)row * p.ldc * oes + piece * 16) = q;
-    }
+  for (int i = 0; i < pp; ++i) {
+    const int row = prow + rpi * i;
+    const uint4 q = *reinterpret_cast<const uint4*>(stg + stage_off(row, piece, rowb, pp));
+    if (gi_warp0 + row < p.M) *reinterpret_cast<uint4*>(cbase + (size_t)row * p.ldc * ES + piece * 16) = q;
   }
   __syncwarp();
+}
+
+// the warp's complete 32-column blocks c0, c0 + 64, ... below `lim`; returns the first block not done. Two-byte
+// types: the 4 KB staging buffer holds two blocks, and the fetch of block i+1 is issued before block i is
+// processed. Four-byte types: one block at a time.
+template <int EPI, int ES>
+__device__ __forceinline__ int epilogue_fast_blocks(const TcParams& p, uint32_t taddr, uint8_t* stg, int lane, int gi_warp0,
+                                                    int col0, int c0, int lim, int bz, float alpha, float aux_scale,
+                                                    double& sq) {
+  constexpr bool AHEAD = (ES == 2) && (EPI != EPI_STORE);
+  int half = 0;
+  __syncwarp();
+  if (AHEAD && c0 + 32 <= lim) aux_fetch_async<ES>(p, lane, gi_warp0, col0 + c0, bz, stg);
+#pragma unroll 1
+  for (; c0 + 32 <= lim; c0 += 64) {
+    uint8_t* cur = stg + (AHEAD ? half * (STAGING_BYTES / 2) : 0);
+    if (AHEAD) {
+      if (c0 + 96 <= lim) {
+        aux_fetch_async<ES>(p, lane, gi_warp0, col0 + c0 + 64, bz, stg + (half ^ 1) * (STAGING_BYTES / 2));
+        epilogue_block_fast<EPI, ES, 1>(p, taddr + (uint32_t)c0, cur, lane, gi_warp0, col0 + c0, bz, alpha, aux_scale, sq);
+      } else {
+        epilogue_block_fast<EPI, ES, 0>(p, taddr + (uint32_t)c0, cur, lane, gi_warp0, col0 + c0, bz, alpha, aux_scale, sq);
+      }
+      half ^= 1;
+    } else {
+      if (EPI != EPI_STORE) aux_fetch_async<ES>(p, lane, gi_warp0, col0 + c0, bz, cur);
+      epilogue_block_fast<EPI, ES, 0>(p, taddr + (uint32_t)c0, cur, lane, gi_warp0, col0 + c0, bz, alpha, aux_scale, sq);
+    }
+  }
+  return c0;
 }
 
 template <int EPI>
@@ -533,23 +568,22 @@ __device__ __forceinline__ void epilogue_half(const TcParams& p, uint32_t taddr,
   const size_t xrow = (size_t)bz * p.batch_aux + (size_t)gi * p.ld_aux;
   const bool vec_ok = ((p.ldc & 7) == 0) && ((p.batch_c & 7) == 0) && ((p.ld_aux & 7) == 0 || EPI == EPI_STORE) &&
                       ((p.batch_aux & 7) == 0 || EPI == EPI_STORE);
-  for (int c0 = wsel * 32; c0 < n_eff; c0 += 64) {
+  const bool a2 = (p.aux_dtype == BF16), o2 = (p.out_dtype == BF16);
+  // the coalesced path wants `aux` and the output in the same type (true of every product the library makes)
+  const bool fast_ok = !p.symmetric && vec_ok && (EPI == EPI_STORE || EPI == EPI_RESID_NORM || a2 == o2);
+  int c0 = wsel * 32;
+  if (fast_ok) {
+    // the complete 32-column blocks come first; whatever is left (a ragged edge) takes the general path below
+    int lim = p.N - col0;
+    if (lim > n_eff) lim = n_eff;
+    const bool two = (EPI == EPI_STORE) ? o2 : a2;
+    if (two) c0 = epilogue_fast_blocks<EPI, 2>(p, taddr, stg, lane, gi_warp0, col0, c0, lim, bz, alpha, aux_scale, sq);
+    else c0 = epilogue_fast_blocks<EPI, 4>(p, taddr, stg, lane, gi_warp0, col0, c0, lim, bz, alpha, aux_scale, sq);
+  }
+  for (; c0 < n_eff; c0 += 64) {
     const int gj0 = col0 + c0, gj1 = gj0 + 16;
     // symmetric output: nothing to do for a block entirely left of the warp's rows (warp-uniform)
     if (p.symmetric && gj0 + 31 < gi_warp0) continue;
-    if (!p.symmetric && vec_ok && gj0 + 32 <= p.N && c0 + 32 <= n_eff) {      // warp-uniform
-      const uint32_t ta = taddr + (uint32_t)c0;
-      const bool a2 = (p.aux_dtype == BF16), o2 = (p.out_dtype == BF16);
-      if (EPI == EPI_STORE || EPI == EPI_RESID_NORM) {      // only one of the two types matters
-        const bool two = (EPI == EPI_STORE) ? o2 : a2;
-        if (two) epilogue_block_fast<EPI, 2, 2>(p, ta, stg, lane, gi_warp0, gj0, bz, alpha, aux_scale, sq);
-        else epilogue_block_fast<EPI, 4, 4>(p, ta, stg, lane, gi_warp0, gj0, bz, alpha, aux_scale, sq);
-      } else if (a2 && o2) epilogue_block_fast<EPI, 2, 2>(p, ta, stg, lane, gi_warp0, gj0, bz, alpha, aux_scale, sq);
-      else if (!a2 && !o2) epilogue_block_fast<EPI, 4, 4>(p, ta, stg, lane, gi_warp0, gj0, bz, alpha, aux_scale, sq);
-      else if (a2) epilogue_block_fast<EPI, 2, 4>(p, ta, stg, lane, gi_warp0, gj0, bz, alpha, aux_scale, sq);
-      else epilogue_block_fast<EPI, 4, 2>(p, ta, stg, lane, gi_warp0, gj0, bz, alpha, aux_scale, sq);
-      continue;
-    }
     const bool second = (c0 + 16 < n_eff);
     uint32_t r0[16], r1[16];
     __syncwarp();
@@ -918,10 +952,14 @@ int choose_tile_m_impl(int M) {
 
 // 256-row tiles are computed by a cluster of two CTAs (tcgen05 cta_group::2) unless DEFL_TC_PAIR=0 asks for
 // the single-CTA form (two 128-row halves in one CTA)
-bool choose_pair(int M) {
+bool choose_pair(int M, int N) {
   if (choose_tile_m_impl(M) != 256) return false;
   if (const char* e = getenv("DEFL_TC_PAIR")) return atoi(e) != 0;
-  return true;
+  // narrow outputs (the range-finder's panels) stream A from HBM with next to no arithmetic per byte: the
+  // pair's issue cost per product is then the bound, and the single-CTA form is faster
+  int min_n = 128;
+  if (const char* e = getenv("DEFL_TC_PAIR_MIN_N")) min_n = atoi(e);
+  return N >= min_n;
 }
 
 }  // namespace
@@ -957,7 +995,7 @@ bool gemm_tc_supported(const GemmDesc& g) {
 int choose_tile_m(int M) { return choose_tile_m_impl(M); }
 
 int gemm_tc_partials_per_batch(const GemmDesc& g) {
-  const int bn = choose_bn(g.N, choose_pair(g.M)), tmh = choose_tile_m(g.M);
+  const int bn = choose_bn(g.N, choose_pair(g.M, g.N)), tmh = choose_tile_m(g.M);
   return ((g.M + tmh - 1) / tmh) * ((g.N + bn - 1) / bn) * (tmh == 256 ? 2 : 1) * EPI_WARPS;
 }
 
@@ -970,7 +1008,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   p.esize = esize;
   p.M = g.M; p.N = g.N; p.batch = g.batch;
   p.tile_m = choose_tile_m(g.M);
-  p.pair = choose_pair(g.M) ? 1 : 0;
+  p.pair = choose_pair(g.M, g.N) ? 1 : 0;
   p.BN = choose_bn(g.N, p.pair != 0);
   p.tiles_m = (g.M + p.tile_m - 1) / p.tile_m;
   p.tiles_n = (g.N + p.BN - 1) / p.BN;

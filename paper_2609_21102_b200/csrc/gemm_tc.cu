@@ -50,6 +50,7 @@ struct TcParams {
   int b_split;                 // 2: B is the sum of two operands (tmB[0] + tmB[1]) that share A; else 1
   int kblocks[2];              // pipeline steps per segment (a step covers `ksub` K blocks of 128 bytes)
   int ksub;                    // K blocks per pipeline stage (1 or 2)
+  int kreal[2];                // K blocks of 128 bytes per segment (the last step of a segment may hold fewer than ksub)
   int M, N, batch;
   int BN;                      // tile width (UMMA N)
   int tile_m;                  // 128 or 256 rows per tile
@@ -659,6 +660,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       const uint32_t nstages = (uint32_t)p.stages;
       const int ksub = p.ksub;
       const uint32_t tx_bytes = PAIR ? 2u * stage_bytes : stage_bytes;   // a pair counts both CTAs' copies on the leader's barrier
+      const uint32_t tx_sub_bytes = PAIR ? 2u * sub_bytes : sub_bytes;
       const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
       const uint32_t full0_sig = PAIR ? map_to_cta(full0, 0) : full0;    // the barrier the copies signal
       const int BN = p.BN, tile_m = p.tile_m, nseg = p.nseg;
@@ -691,13 +693,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
           const CUtensorMap* tmb0 = &p.tmB[BSPLIT > 1 ? 0 : seg];
           const CUtensorMap* tmb1 = &p.tmB[1];
           const int nkb = p.kblocks[seg];
+          int left = p.kreal[seg];                            // K blocks of the segment not yet requested
           int k0 = 0;
-          for (int kb = 0; kb < nkb; ++kb) {
+          for (int kb = 0; kb < nkb; ++kb, left -= ksub) {
             if (!mbar_wait(empty0 + 8u * stage, phase ^ 1u, &abort_flag, p.status)) break;
-            if (!PAIR || rank == 0) mbar_expect_tx(full0 + 8u * stage, tx_bytes);
+            const int nsub = left < ksub ? left : ksub;       // the last step of a segment may be short
+            if (!PAIR || rank == 0) mbar_expect_tx(full0 + 8u * stage, nsub == ksub ? tx_bytes : tx_sub_bytes * (uint32_t)nsub);
             const uint32_t fb = full0_sig + 8u * stage;
-            // (a K block past the end of K is filled with zeros by the copy engine and adds nothing)
-            for (int sub = 0; sub < ksub; ++sub, k0 += kstep) {
+            // (the part of a K block past the end of K is filled with zeros by the copy engine and adds nothing)
+            for (int sub = 0; sub < nsub; ++sub, k0 += kstep) {
               const uint32_t sa = smem_base + stage * stage_bytes + (uint32_t)sub * sub_bytes;
               const uint32_t sb = sa + a_stage_bytes;
               for (uint32_t bx = 0; bx < a_boxes; ++bx) {
@@ -750,6 +754,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
       const uint32_t nstages = (uint32_t)p.stages;
       const int ksub = p.ksub;
+      const int kreal0 = p.kreal[0], kreal1 = p.kreal[1], steps0 = p.kblocks[0];
       const uint32_t idesc0 = p.idesc;
       const bool tall = !PAIR && p.tile_m == 256;
       for (long long tile = tile0; tile < p.total_tiles; tile += tile_step) {
@@ -762,10 +767,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
         const bool two = !PAIR && (t.halves & 2) != 0;
         bool ok = true;
         uint32_t accum = 0;                                   // the first product of a tile overwrites the accumulator
-        for (int kb = 0; kb < total_kblocks; ++kb) {
+        int left = kreal0;                                    // K blocks not yet multiplied in the current segment
+        for (int kb = 0; kb < total_kblocks; ++kb, left -= ksub) {
+          if (kb == steps0) left = kreal1;
           if (!mbar_wait(full0 + 8u * stage, phase, &abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
-          for (int sub = 0; sub < ksub; ++sub) {
+          const int nsub = left < ksub ? left : ksub;
+          for (int sub = 0; sub < nsub; ++sub) {
             const uint32_t sa16 = base16 + stage * stage16 + (uint32_t)sub * sub16;
             const uint32_t sb16 = sa16 + a_stage16;
 #pragma unroll
@@ -1045,7 +1053,8 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   p.ksub = (p.pair && 3u * 2u * sub_bytes <= smem_budget) ? 2 : 1;
   if (const char* e = getenv("DEFL_TC_KSUB")) { const int v = atoi(e); if ((v == 1 || v == 2) && (uint32_t)v * sub_bytes * 2u <= smem_budget) p.ksub = v; }
   for (int s = 0; s < g.nseg; ++s) {
-    p.kblocks[s] = ((g.K[s] + span - 1) / span + p.ksub - 1) / p.ksub;
+    p.kreal[s] = (g.K[s] + span - 1) / span;
+    p.kblocks[s] = (p.kreal[s] + p.ksub - 1) / p.ksub;
     if (!encode_map(&p.tmA[s], g.A[s], esize, tf32, pa.mn_major, g.M, g.K[s], g.sa_i[s], g.sa_k[s], g.batch,
                     g.batch_a[s], pa.box_rows))
       return cudaErrorInvalidValue;

@@ -100,6 +100,18 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "memory");
   return ok;
 }
+// non-blocking probe of a barrier phase
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -646,17 +658,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    // The whole warp runs the loop: lane 0 waits for the stage and posts the expected byte count, then every lane
+    // issues ONE of the step's copies (operand, K block, box, split fixed per lane), so that the copies of a step
+    // leave in one warp instruction instead of one thread instruction each (a thread-serial issue of 4-6 copies
+    // took longer than the tensor pipe needs for the step). Everything the loop needs sits in registers.
+    {
       uint32_t stage = 0, phase = 0;
-      // everything the inner loop needs sits in registers: this one thread's issue rate bounds the whole pipeline
-      // when a K block is short (a parameter re-read or an integer division per copy costs more than the copy)
       const int arow = PAIR ? (int)rank * 128 : 0;              // this CTA's rows within the tile
       const int kstep = KBYTES / p.esize;
-      const bool a_mn = p.a_mn_major != 0, b_mn = p.b_mn_major != 0;
-      const uint32_t a_boxes = p.a_boxes, b_boxes = p.b_boxes;
-      const uint32_t a_box_bytes = p.a_box_bytes, b_box_bytes = p.b_box_bytes;
-      const int a_box_rows = (int)p.a_box_rows, b_box_rows = (int)p.b_box_rows;
-      const uint32_t a_stage_bytes = p.a_stage_bytes, b_split_bytes = p.b_split_bytes;
+      const int a_boxes = (int)p.a_boxes, b_boxes = (int)p.b_boxes;
       const uint32_t nstages = (uint32_t)p.stages;
       const int ksub = p.ksub;
       const uint32_t tx_bytes = PAIR ? 2u * stage_bytes : stage_bytes;   // a pair counts both CTAs' copies on the leader's barrier
@@ -665,12 +675,31 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       const uint32_t full0_sig = PAIR ? map_to_cta(full0, 0) : full0;    // the barrier the copies signal
       const int BN = p.BN, tile_m = p.tile_m, nseg = p.nseg;
       const bool aux_prefetch = p.aux_prefetch != 0;
-      for (long long tile = tile0; tile < p.total_tiles; tile += tile_step) {
+      // this lane's copy within a step (the host guarantees at most 32 copies per step), fixed for the launch
+      const int per_sub = a_boxes + BSPLIT * b_boxes;
+      const int ops = ksub * per_sub;
+      const int my_sub = lane / per_sub;
+      int my_r = lane - my_sub * per_sub;
+      const bool my_on = lane < ops;
+      const bool my_a = my_r < a_boxes;
+      int my_sp = 0;
+      if (!my_a) { my_r -= a_boxes; my_sp = my_r / b_boxes; my_r -= my_sp * b_boxes; }
+      const int my_mn_off = my_r * (int)(my_a ? p.a_box_rows : p.b_box_rows);
+      const uint32_t my_dst_off = (uint32_t)my_sub * sub_bytes +
+                                  (my_a ? (uint32_t)my_r * p.a_box_bytes
+                                        : p.a_stage_bytes + (uint32_t)my_sp * p.b_split_bytes + (uint32_t)my_r * p.b_box_bytes);
+      const bool my_mn_major = (my_a ? p.a_mn_major : p.b_mn_major) != 0;
+      const int my_k_off = my_sub * kstep;
+      const CUtensorMap* my_tm0 = my_a ? &p.tmA[0] : &p.tmB[BSPLIT > 1 ? my_sp : 0];
+      const CUtensorMap* my_tm1 = my_a ? &p.tmA[1] : &p.tmB[BSPLIT > 1 ? my_sp : 1];
+      const int kblocks0 = p.kblocks[0], kblocks1 = p.kblocks[1], kreal0 = p.kreal[0], kreal1 = p.kreal[1];
+      const long long total_tiles = p.total_tiles;
+      for (long long tile = tile0; tile < total_tiles; tile += tile_step) {
         const TileInfo t = tile_info(p, tile);
         if (t.skip) continue;
-        // the epilogues read the matching tile of `aux` with plain loads: start moving it from HBM into L2
-        // well ahead (AUX_AHEAD tiles of this CTA; short main loops leave no time otherwise)
-        if (aux_prefetch) {
+        // the epilogues read the matching tile of `aux`: start moving it from HBM into L2 well ahead
+        // (AUX_AHEAD tiles of this CTA; short main loops leave no time otherwise)
+        if (aux_prefetch && lane == 0) {
           if (tile == tile0) {
             for (int d = 0; d < AUX_AHEAD; ++d) {
               const long long tp = tile + (long long)d * tile_step;
@@ -688,55 +717,34 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
         const int a_mn0 = t.tm * tile_m + arow;
         const int b_mn0 = t.tn * BN + (PAIR ? (int)rank * (t.n_eff >> 1) : 0);   // a pair: this CTA's half of the columns
         const int bz = t.bz;
-        for (int seg = 0; seg < nseg; ++seg) {
-          const CUtensorMap* tma = &p.tmA[seg];
-          const CUtensorMap* tmb0 = &p.tmB[BSPLIT > 1 ? 0 : seg];
-          const CUtensorMap* tmb1 = &p.tmB[1];
-          const int nkb = p.kblocks[seg];
-          int left = p.kreal[seg];                            // K blocks of the segment not yet requested
-          int k0 = 0;
-          for (int kb = 0; kb < nkb; ++kb, left -= ksub) {
-            if (!mbar_wait(empty0 + 8u * stage, phase ^ 1u, &abort_flag, p.status)) break;
+        const int my_mn = (my_a ? a_mn0 : b_mn0) + my_mn_off;
+        bool live = true;
+        for (int seg = 0; seg < nseg && live; ++seg) {
+          const int nkb = seg ? kblocks1 : kblocks0;
+          int left = seg ? kreal1 : kreal0;                   // K blocks of the segment not yet requested
+          const CUtensorMap* tm = seg ? my_tm1 : my_tm0;
+          int kc = my_k_off;
+          for (int kb = 0; kb < nkb; ++kb, left -= ksub, kc += ksub * kstep) {
+            int ok = 1;
+            if (lane == 0) ok = mbar_wait(empty0 + 8u * stage, phase ^ 1u, &abort_flag, p.status) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) { live = false; break; }
             const int nsub = left < ksub ? left : ksub;       // the last step of a segment may be short
-            if (!PAIR || rank == 0) mbar_expect_tx(full0 + 8u * stage, nsub == ksub ? tx_bytes : tx_sub_bytes * (uint32_t)nsub);
-            const uint32_t fb = full0_sig + 8u * stage;
+            if (lane == 0 && (!PAIR || rank == 0))
+              mbar_expect_tx(full0 + 8u * stage, nsub == ksub ? tx_bytes : tx_sub_bytes * (uint32_t)nsub);
             // (the part of a K block past the end of K is filled with zeros by the copy engine and adds nothing)
-            for (int sub = 0; sub < nsub; ++sub, k0 += kstep) {
-              const uint32_t sa = smem_base + stage * stage_bytes + (uint32_t)sub * sub_bytes;
-              const uint32_t sb = sa + a_stage_bytes;
-              for (uint32_t bx = 0; bx < a_boxes; ++bx) {
-                const int mn0 = a_mn0 + (int)bx * a_box_rows;
-                const uint32_t dst = sa + bx * a_box_bytes;
-                if (PAIR) {
-                  if (a_mn) tma_load_3d_pair(dst, tma, fb, mn0, k0, bz);
-                  else tma_load_3d_pair(dst, tma, fb, k0, mn0, bz);
-                } else {
-                  if (a_mn) tma_load_3d(dst, tma, fb, mn0, k0, bz);
-                  else tma_load_3d(dst, tma, fb, k0, mn0, bz);
-                }
-              }
-#pragma unroll
-              for (int sp = 0; sp < BSPLIT; ++sp) {
-                const CUtensorMap* tmb = sp ? tmb1 : tmb0;
-                const uint32_t sbs = sb + (uint32_t)sp * b_split_bytes;
-                for (uint32_t bx = 0; bx < b_boxes; ++bx) {
-                  const int mn0 = b_mn0 + (int)bx * b_box_rows;
-                  const uint32_t dst = sbs + bx * b_box_bytes;
-                  if (PAIR) {
-                    if (b_mn) tma_load_3d_pair(dst, tmb, fb, mn0, k0, bz);
-                    else tma_load_3d_pair(dst, tmb, fb, k0, mn0, bz);
-                  } else {
-                    if (b_mn) tma_load_3d(dst, tmb, fb, mn0, k0, bz);
-                    else tma_load_3d(dst, tmb, fb, k0, mn0, bz);
-                  }
-                }
-              }
+            if (my_on && my_sub < nsub) {
+              const uint32_t fb = full0_sig + 8u * stage;
+              const uint32_t dst = smem_base + stage * stage_bytes + my_dst_off;
+              const int c0 = my_mn_major ? my_mn : kc, c1 = my_mn_major ? kc : my_mn;
+              if (PAIR) tma_load_3d_pair(dst, tm, fb, c0, c1, bz);
+              else tma_load_3d(dst, tm, fb, c0, c1, bz);
             }
+            __syncwarp();
             if (++stage == nstages) { stage = 0; phase ^= 1u; }
           }
-          if (abort_flag) break;
         }
-        if (abort_flag) break;
+        if (!live) break;
       }
     }
   } else if (warp == 1) {
@@ -768,10 +776,16 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
         bool ok = true;
         uint32_t accum = 0;                                   // the first product of a tile overwrites the accumulator
         int left = kreal0;                                    // K blocks not yet multiplied in the current segment
+        uint32_t ready = 0;                                   // the next stage was seen full while this one was issued
         for (int kb = 0; kb < total_kblocks; ++kb, left -= ksub) {
           if (kb == steps0) left = kreal1;
-          if (!mbar_wait(full0 + 8u * stage, phase, &abort_flag, p.status)) { ok = false; break; }
+          if (!ready && !mbar_wait(full0 + 8u * stage, phase, &abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
+          {
+            // probe the following stage now: the answer arrives while this stage's products are issued
+            const uint32_t ns = (stage + 1 == nstages) ? 0u : stage + 1;
+            ready = (kb + 1 < total_kblocks) ? mbar_test(full0 + 8u * ns, ns == 0u ? phase ^ 1u : phase) : 0u;
+          }
           const int nsub = left < ksub ? left : ksub;
           for (int sub = 0; sub < nsub; ++sub) {
             const uint32_t sa16 = base16 + stage * stage16 + (uint32_t)sub * sub16;
@@ -1062,6 +1076,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
                     g.batch_b[s], pb.box_rows))
       return cudaErrorInvalidValue;
   }
+  if ((uint32_t)p.ksub * (p.a_boxes + (uint32_t)p.b_split * p.b_boxes) > 32u) return cudaErrorNotSupported;   // one copy per producer lane
   const uint32_t stage_bytes = sub_bytes * (uint32_t)p.ksub;
   int stages = (int)(smem_budget / stage_bytes);
   if (stages > MAX_STAGES) stages = MAX_STAGES;

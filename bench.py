@@ -286,14 +286,17 @@ def main():
     stage_tot = [0.0, 0.0, 0.0, 0.0]
     filt_flops = 0.0        # dense count of the filter products
     filt_executed = 0.0     # flops the tensor cores actually execute (tiles below the diagonal are skipped)
-    for g, (b, m, n) in zip(groups, wl["groups"]):
-        ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"], sketch=g["Om"],
-                               gamma=1.01, exploit_symmetry=SYM)
-        ms = ctx.defl_get_stage_ms()
-        for i in range(min(4, len(ms))):
-            stage_tot[i] += ms[i]
-        filt_flops += b * flops_per_matrix(m, n, wl["k"], wl["p"], wl["J"], wl["L"])[0]
-        filt_executed += b * executed_filter_flops(m, n, wl["L"], SYM)
+    STAGE_REPS = 3          # averaged: a single step's split moves by several percent with the power state
+    for rep in range(STAGE_REPS):
+        for g, (b, m, n) in zip(groups, wl["groups"]):
+            ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"], sketch=g["Om"],
+                                   gamma=1.01, exploit_symmetry=SYM)
+            ms = ctx.defl_get_stage_ms()
+            for i in range(min(4, len(ms))):
+                stage_tot[i] += ms[i] / STAGE_REPS
+            if rep == 0:
+                filt_flops += b * flops_per_matrix(m, n, wl["k"], wl["p"], wl["J"], wl["L"])[0]
+                filt_executed += b * executed_filter_flops(m, n, wl["L"], SYM)
     plain_ms = 0.0
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()

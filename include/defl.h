@@ -120,8 +120,11 @@ int defl_polar_batched(defl_ctx* ctx, const void* G, void* out, int b, int m, in
 
 /* The same call for HOST buffers: G_host and out_host are host memory (pinned memory makes the copies
  * asynchronous and fast). The library copies G to device staging memory it owns, runs defl_polar_batched,
- * copies the result back and synchronises the stream before returning, so out_host is ready on return.
- * opts->sketch, if given, is still device memory. Same errors as defl_polar_batched. */
+ * copies the result back and synchronises before returning, so out_host is ready on return. The batch goes
+ * through in a few chunks of whole matrices, the copies of one chunk overlapping the computation of another on
+ * streams the context owns; every matrix gets the result (and the sketch) it would get from one
+ * defl_polar_batched call on the whole batch. opts->sketch, if given, is still device memory. Same errors as
+ * defl_polar_batched. */
 int defl_polar_batched_host(defl_ctx* ctx, const void* G_host, void* out_host, int b, int m, int n, int dtype,
                             int k, int oversample, int power_iters,
                             const float* coeff_schedule, int L, const defl_opts* opts);

@@ -5,6 +5,7 @@
 #include "common.cuh"
 #include "panel.cuh"
 #include "ctx.cuh"
+#include <cstdlib>
 
 #include <cstdio>
 #include <cstring>
@@ -297,6 +298,11 @@ int defl_destroy(defl_ctx* c) {
   if (c->ws) cudaFree(c->ws);
   if (c->stage_in) cudaFree(c->stage_in);
   if (c->stage_out) cudaFree(c->stage_out);
+  if (c->copy_ready) {
+    cudaStreamDestroy(c->copy_in);
+    cudaStreamDestroy(c->copy_out);
+    for (int i = 0; i < DEFL_HOST_MAX_CHUNKS; ++i) { cudaEventDestroy(c->chunk_in[i]); cudaEventDestroy(c->chunk_done[i]); }
+  }
   if (c->wait_status) cudaFree(c->wait_status);
   for (int i = 0; i < DEFL_MAX_MARKS; ++i)
     if (c->marks[i]) cudaEventDestroy(c->marks[i]);
@@ -644,12 +650,61 @@ int defl_polar_batched_host(defl_ctx* c, const void* G_host, void* out_host, int
     if (ctx_fail(c, cudaMalloc(&c->stage_out, bytes), "cudaMalloc(staging)")) return DEFL_ERR_CUDA;
     c->stage_bytes = bytes;
   }
-  if (ctx_fail(c, cudaMemcpyAsync(c->stage_in, G_host, bytes, cudaMemcpyHostToDevice, c->stream), "H2D")) return DEFL_ERR_CUDA;
-  const int rc = defl_polar_batched(c, c->stage_in, c->stage_out, b, m, n, dtype, k, oversample, power_iters,
-                                    coeff_schedule, L, opts, nullptr);
+  // The batch is independent matrices: it goes through in chunks, the copy of chunk i+1 to the device and of
+  // chunk i-1 back to the host running (on streams of their own) while chunk i is computed. Few chunks: the small
+  // kernels of the range finder take about the same time for 12 matrices as for 48.
+  int chunks = b >= 24 ? 3 : (b >= 8 ? 2 : 1);
+  if (const char* e = getenv("DEFL_HOST_CHUNKS")) { const int v = atoi(e); if (v >= 1) chunks = v; }
+  if (chunks > DEFL_HOST_MAX_CHUNKS) chunks = DEFL_HOST_MAX_CHUNKS;
+  if (chunks > b) chunks = b;
+  if (!c->copy_ready) {
+    bool ok = cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; ok && i < DEFL_HOST_MAX_CHUNKS; ++i)
+      ok = cudaEventCreateWithFlags(&c->chunk_in[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&c->chunk_done[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { ctx_fail(c, cudaErrorUnknown, "streams for the host-buffer path"); return DEFL_ERR_CUDA; }
+    c->copy_ready = 1;
+  }
+  const size_t per_matrix = (size_t)m * n * dtype_size(dtype);
+  const int per = (b + chunks - 1) / chunks;
+  const int ms = m < n ? m : n;
+  int l = k > 0 ? k + oversample : 0;
+  if (l > ms) l = ms;
+  // the staging buffers may still be read by work the caller queued on the compute stream before this call
+  if (ctx_fail(c, cudaEventRecord(c->chunk_done[0], c->stream), "record")) return DEFL_ERR_CUDA;
+  if (ctx_fail(c, cudaStreamWaitEvent(c->copy_in, c->chunk_done[0], 0), "wait")) return DEFL_ERR_CUDA;
+  for (int i = 0; i < chunks; ++i) {
+    const int b0 = i * per, bc = (b - b0 < per) ? b - b0 : per;
+    if (bc <= 0) { chunks = i; break; }
+    const size_t off = (size_t)b0 * per_matrix;
+    if (ctx_fail(c, cudaMemcpyAsync((char*)c->stage_in + off, (const char*)G_host + off, (size_t)bc * per_matrix,
+                                    cudaMemcpyHostToDevice, c->copy_in), "H2D")) return DEFL_ERR_CUDA;
+    if (ctx_fail(c, cudaEventRecord(c->chunk_in[i], c->copy_in), "record")) return DEFL_ERR_CUDA;
+  }
+  int rc = DEFL_OK;
+  for (int i = 0; i < chunks && rc == DEFL_OK; ++i) {
+    const int b0 = i * per, bc = (b - b0 < per) ? b - b0 : per;
+    const size_t off = (size_t)b0 * per_matrix;
+    defl_opts o;
+    if (opts) o = *opts; else memset(&o, 0, sizeof(o));
+    // matrix b0 + j of the batch keeps the sketch it would get in one call: its slice of Omega, or stream b0 + j
+    if (o.sketch) o.sketch += (size_t)b0 * ms * l; else o.seed += (uint64_t)b0;
+    if (ctx_fail(c, cudaStreamWaitEvent(c->stream, c->chunk_in[i], 0), "wait")) { rc = DEFL_ERR_CUDA; break; }
+    rc = defl_polar_batched(c, (char*)c->stage_in + off, (char*)c->stage_out + off, bc, m, n, dtype, k, oversample,
+                            power_iters, coeff_schedule, L, &o, nullptr);
+    if (rc) break;
+    if (ctx_fail(c, cudaEventRecord(c->chunk_done[i], c->stream), "record") ||
+        ctx_fail(c, cudaStreamWaitEvent(c->copy_out, c->chunk_done[i], 0), "wait") ||
+        ctx_fail(c, cudaMemcpyAsync((char*)out_host + off, (char*)c->stage_out + off, (size_t)bc * per_matrix,
+                                    cudaMemcpyDeviceToHost, c->copy_out), "D2H"))
+      rc = DEFL_ERR_CUDA;
+  }
+  // everything queued so far finishes before the call returns, also after an error
+  const cudaError_t e1 = cudaStreamSynchronize(c->copy_in), e2 = cudaStreamSynchronize(c->stream),
+                    e3 = cudaStreamSynchronize(c->copy_out);
   if (rc) return rc;
-  if (ctx_fail(c, cudaMemcpyAsync(out_host, c->stage_out, bytes, cudaMemcpyDeviceToHost, c->stream), "D2H")) return DEFL_ERR_CUDA;
-  if (ctx_fail(c, cudaStreamSynchronize(c->stream), "synchronize")) return DEFL_ERR_CUDA;
+  if (ctx_fail(c, e1, "synchronize") || ctx_fail(c, e2, "synchronize") || ctx_fail(c, e3, "synchronize")) return DEFL_ERR_CUDA;
   return DEFL_OK;
 }
 

@@ -6,6 +6,8 @@
 
 #define DEFL_MAX_MARKS 12
 
+#define DEFL_HOST_MAX_CHUNKS 8
+
 struct defl_ctx {
   int device;
   int num_sms;
@@ -15,6 +17,9 @@ struct defl_ctx {
   void* stage_in;        // device staging of host inputs/outputs (defl_polar_batched_host)
   void* stage_out;
   size_t stage_bytes;
+  cudaStream_t copy_in, copy_out;          // host-buffer entry point: copies overlap the compute stream
+  cudaEvent_t chunk_in[DEFL_HOST_MAX_CHUNKS], chunk_done[DEFL_HOST_MAX_CHUNKS];
+  int copy_ready;                           // streams and events above exist
   int* wait_status;      // device word: the tensor engine ORs DEFL_ST_DEVICE_WAIT into it
   long long launches;    // kernels launched so far
   bool profiling;

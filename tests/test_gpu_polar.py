@@ -182,3 +182,19 @@ def test_zero_matrix_is_flagged_not_trapped(ctx):
     torch.cuda.synchronize()
     assert torch.count_nonzero(out) == 0
     assert int(info["status"][0]) & binding.ST_ZERO_RESIDUAL
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("given_sketch", [False, True])
+def test_host_buffer_path_matches_device_path(ctx, given_sketch):
+    """The host-buffer entry point splits the batch into chunks and overlaps copies with computation; every
+    matrix must come out bit-identical to one device call on the whole batch (same sketch per matrix)."""
+    from paper_2609_21102_b200 import binding
+    b, m, n, k, p = 10, 192, 320, 4, 4
+    G = inputs.workload_spiked(b, m, n, 7, spikes=k).to(torch.bfloat16)
+    Gd = G.cuda()
+    sk = inputs.sketch(b, min(m, n), k + p, 2, shape_index=7).cuda() if given_sketch else None
+    ref = ctx.defl_polar_batched(Gd, k, p, 1, _sched(binding.MUON_QUINTIC, 5), sketch=sk, seed=77).cpu()
+    out = torch.empty_like(G).pin_memory()
+    ctx.defl_polar_batched_host(G.pin_memory(), out, k, p, 1, _sched(binding.MUON_QUINTIC, 5), sketch=sk, seed=77)
+    assert torch.equal(out, ref)

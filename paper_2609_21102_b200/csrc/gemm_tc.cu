@@ -537,6 +537,33 @@ __device__ __forceinline__ void epilogue_block_fast(const TcParams& p, uint32_t 
     const uint4 q = *reinterpret_cast<const uint4*>(stg + stage_off(row, piece, rowb, pp));
     if (gi_warp0 + row < p.M) *reinterpret_cast<uint4*>(cbase + (size_t)row * p.ldc * ES + piece * 16) = q;
   }
+  if (p.symmetric && gj0 > gi_warp0) {
+    // mirror image of a block above the diagonal (the caller guarantees 32 complete rows): transposed row c of the
+    // block is 32 values = pp pieces of 16 bytes; pp consecutive lanes write one such row, each lane gathering its
+    // epp values from one column of the staged block
+    uint8_t* mbase = reinterpret_cast<uint8_t*>(p.C) + ((size_t)bz * p.batch_c + (size_t)gj0 * p.ldc + gi_warp0) * ES;
+#pragma unroll
+    for (int i = 0; i < pp; ++i) {
+      const int c = rpi * i + prow;                 // column of the block = row of the mirror image
+      const int cp = c / epp, ce = (c % epp) * ES;  // its piece and byte offset within a staged row
+      uint4 q;
+      if (ES == 2) {
+        uint16_t h[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          h[e] = *reinterpret_cast<const uint16_t*>(stg + stage_off(piece * epp + e, cp, rowb, pp) + ce);
+        q = make_uint4((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16),
+                       (uint32_t)h[4] | ((uint32_t)h[5] << 16), (uint32_t)h[6] | ((uint32_t)h[7] << 16));
+      } else {
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          w[e] = *reinterpret_cast<const uint32_t*>(stg + stage_off(piece * epp + e, cp, rowb, pp) + ce);
+        q = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+      *reinterpret_cast<uint4*>(mbase + (size_t)c * p.ldc * ES + piece * 16) = q;
+    }
+  }
   __syncwarp();
 }
 
@@ -549,6 +576,8 @@ __device__ __forceinline__ int epilogue_fast_blocks(const TcParams& p, uint32_t 
                                                     double& sq) {
   constexpr bool AHEAD = (ES == 2) && (EPI != EPI_STORE);
   int half = 0;
+  // symmetric output: nothing to do for blocks entirely left of the warp's rows (they are written as mirror images)
+  if (p.symmetric) while (c0 + 32 <= lim && col0 + c0 + 31 < gi_warp0) c0 += 64;
   __syncwarp();
   if (AHEAD && c0 + 32 <= lim) aux_fetch_async<ES>(p, lane, gi_warp0, col0 + c0, bz, stg);
 #pragma unroll 1
@@ -583,7 +612,9 @@ __device__ __forceinline__ void epilogue_half(const TcParams& p, uint32_t taddr,
                       ((p.batch_aux & 7) == 0 || EPI == EPI_STORE);
   const bool a2 = (p.aux_dtype == BF16), o2 = (p.out_dtype == BF16);
   // the coalesced path wants `aux` and the output in the same type (true of every product the library makes)
-  const bool fast_ok = !p.symmetric && vec_ok && (EPI == EPI_STORE || EPI == EPI_RESID_NORM || a2 == o2);
+  // (symmetric output: the mirror stores of the coalesced path assume 32 complete rows)
+  const bool fast_ok = vec_ok && (EPI == EPI_STORE || EPI == EPI_RESID_NORM || a2 == o2) &&
+                       (!p.symmetric || (gi_warp0 + 32 <= p.M && EPI != EPI_RESID_NORM));
   int c0 = wsel * 32;
   if (fast_ok) {
     // the complete 32-column blocks come first; whatever is left (a ragged edge) takes the general path below

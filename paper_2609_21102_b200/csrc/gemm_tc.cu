@@ -998,15 +998,17 @@ int choose_bn(int N, bool pair) {
   return r < 256 ? r : 256;
 }
 
-int choose_tile_m_impl(int M) {
+int choose_tile_m_impl(int M, int N, int batch) {
+  (void)N; (void)batch;
   if (const char* e = getenv("DEFL_TC_TILE_M")) { const int v = atoi(e); if (v == 128 || v == 256) return v; }
+  // (128-row tiles for narrow outputs whose 256-row tiles fill the last wave of CTAs badly were measured: slower)
   return M > 128 ? 256 : 128;
 }
 
 // 256-row tiles are computed by a cluster of two CTAs (tcgen05 cta_group::2) unless DEFL_TC_PAIR=0 asks for
 // the single-CTA form (two 128-row halves in one CTA)
-bool choose_pair(int M, int N) {
-  if (choose_tile_m_impl(M) != 256) return false;
+bool choose_pair(int M, int N, int batch) {
+  if (choose_tile_m_impl(M, N, batch) != 256) return false;
   if (const char* e = getenv("DEFL_TC_PAIR")) return atoi(e) != 0;
   // narrow outputs (the range-finder's panels) stream A from HBM with next to no arithmetic per byte: the
   // pair's issue cost per product is then the bound, and the single-CTA form is faster
@@ -1045,10 +1047,9 @@ bool gemm_tc_supported(const GemmDesc& g) {
   return get_encode_fn() != nullptr;
 }
 
-int choose_tile_m(int M) { return choose_tile_m_impl(M); }
 
 int gemm_tc_partials_per_batch(const GemmDesc& g) {
-  const int bn = choose_bn(g.N, choose_pair(g.M, g.N)), tmh = choose_tile_m(g.M);
+  const int bn = choose_bn(g.N, choose_pair(g.M, g.N, g.batch)), tmh = choose_tile_m_impl(g.M, g.N, g.batch);
   return ((g.M + tmh - 1) / tmh) * ((g.N + bn - 1) / bn) * (tmh == 256 ? 2 : 1) * EPI_WARPS;
 }
 
@@ -1060,8 +1061,8 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   const bool tf32 = (g.in_dtype == F32);
   p.esize = esize;
   p.M = g.M; p.N = g.N; p.batch = g.batch;
-  p.tile_m = choose_tile_m(g.M);
-  p.pair = choose_pair(g.M, g.N) ? 1 : 0;
+  p.tile_m = choose_tile_m_impl(g.M, g.N, g.batch);
+  p.pair = choose_pair(g.M, g.N, g.batch) ? 1 : 0;
   p.BN = choose_bn(g.N, p.pair != 0);
   p.tiles_m = (g.M + p.tile_m - 1) / p.tile_m;
   p.tiles_n = (g.N + p.BN - 1) / p.BN;

@@ -48,9 +48,10 @@ def flops_per_matrix(m, n, k, p, J, L):
     return filt, rsvd + defl
 
 
-# Average DRAM bytes per filter-product launch (dram__bytes_read + dram__bytes_write from the ncu capture
-# summarised in profiles/gemm_tc_kernel_filter_gpt2_xl_batch8.md, 8 matrices per group, scaled by 48/8).
-FILTER_TRAFFIC_BYTES_PER_LAUNCH = 1131e6
+# Average DRAM bytes per filter-product launch: dram__bytes_read + dram__bytes_write of the six kinds of filter
+# launch (X X^T, A^2 polynomial, B X for each shape group) from the ncu captures summarised in
+# profiles/gemm_tc_kernel_filter_gpt2_xl_batch8.md (8 matrices per group: 132.3 MB on average), scaled by 48/8.
+FILTER_TRAFFIC_BYTES_PER_LAUNCH = 794e6
 
 
 def max_over_ranks(value, dist=None, device="cpu"):
@@ -101,33 +102,54 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs: one nvidia-smi process in loop
+    mode (50 ms period), started ahead of the region; only samples that arrive between mark_start() and
+    mark_end() are kept."""
 
     def __init__(self, index):
-        self.index, self.rows, self._stop, self._t = index, [], threading.Event(), None
+        self.index, self.rows, self._all, self._t, self._p = index, [], [], None, None
+        self.t0 = self.t1 = None
 
     def _run(self):
-        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
-        while not self._stop.is_set():
-            try:
-                out = subprocess.run(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + q,
-                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
-                parts = [x.strip() for x in out.strip().split(",")]
-                if len(parts) >= 6:
-                    self.rows.append(parts)
-            except Exception:
-                pass
-            self._stop.wait(0.1)
+        for line in self._p.stdout:
+            parts = [x.strip() for x in line.strip().split(",")]
+            if len(parts) >= 6:
+                self._all.append((time.time(), parts))
 
     def __enter__(self):
-        self._t = threading.Thread(target=self._run, daemon=True)
-        self._t.start()
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        try:
+            self._p = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + q,
+                                        "--format=csv,noheader,nounits", "-lms", "50"], stdout=subprocess.PIPE,
+                                       stderr=subprocess.DEVNULL, text=True, bufsize=1)
+            self._t = threading.Thread(target=self._run, daemon=True)
+            self._t.start()
+            time.sleep(0.3)      # let the first samples arrive before the region starts
+        except Exception:
+            self._p = None
         return self
 
+    def mark_start(self):
+        self.t0 = time.time()
+
+    def mark_end(self):
+        self.t1 = time.time()
+
     def __exit__(self, *a):
-        self._stop.set()
-        self._t.join(timeout=6)
+        if self._p is not None:
+            self._p.terminate()          # the one process this object started
+            try:
+                self._p.wait(timeout=5)
+            except Exception:
+                self._p.kill()
+            self._t.join(timeout=5)
+        t0 = self.t0 if self.t0 is not None else 0.0
+        t1 = self.t1 if self.t1 is not None else float("inf")
+        self.rows = [r for (t, r) in self._all if t0 <= t <= t1]
+        if not self.rows and self._all:      # a region shorter than the period: the nearest sample
+            mid = 0.5 * (t0 + min(t1, time.time()))
+            self.rows = [min(self._all, key=lambda tr: abs(tr[0] - mid))[1]]
 
     def summary(self):
         if not self.rows:
@@ -196,7 +218,7 @@ def oracle_sample(wl, seconds_hint=20.0):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--small", action="store_true", help="tiny workload for a quick functional check")
@@ -273,11 +295,13 @@ def main():
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     with ClockSampler(local_rank) as clk:
         barrier()
+        clk.mark_start()
         ev[0].record()
         for i in range(args.steps):
             run_step(ctx, wl, groups, lanes)
             ev[i + 1].record()
         barrier()
+        clk.mark_end()
     launches = launch_total() - launches0
     total_ms = max_over_ranks(ev[0].elapsed_time(ev[-1]), dist, "cuda")
     ms_per_step = total_ms / args.steps

@@ -16,8 +16,9 @@
 //               its 128 accumulator rows in its own tensor memory, two accumulator buffers. A pipeline stage
 //               covers two K blocks: the cost of one step of the two issuing threads (barrier wait, four
 //               products at ~75 cycles of issue each, commit) otherwise exceeds the 512 cycles the tensor
-//               pipe needs per K block. DEFL_TC_PAIR=0 selects the older single-CTA form of the 256-row tile
-//               (two 128-row halves sharing the B tile, one accumulator buffer).
+//               pipe needs per K block (one K block per stage when two would not leave three stages).
+//               DEFL_TC_PAIR=0 selects the older single-CTA form of the 256-row tile (two 128-row halves
+//               sharing the B tile, one accumulator buffer).
 // Either operand may be K-major (K contiguous in global memory) or MN-major; the shared-memory matrix
 // descriptors and the instruction descriptor are built to match. No multicast copies: every CTA loads its own
 // operands. Every wait is bounded: when one runs out the kernel raises DEFL_ST_DEVICE_WAIT in the status word,
@@ -1010,9 +1011,9 @@ int choose_tile_m_impl(int M, int N, int batch) {
 bool choose_pair(int M, int N, int batch) {
   if (choose_tile_m_impl(M, N, batch) != 256) return false;
   if (const char* e = getenv("DEFL_TC_PAIR")) return atoi(e) != 0;
-  // narrow outputs (the range-finder's panels) stream A from HBM with next to no arithmetic per byte: the
-  // pair's issue cost per product is then the bound, and the single-CTA form is faster
-  int min_n = 128;
+  // (DEFL_TC_PAIR_MIN_N: outputs narrower than this take the single-CTA form; measured on the range finder's
+  // 48-column panels the pair streams A faster, 4.9-5.1 against 4.3-4.6 TB/s, so the default keeps every width)
+  int min_n = 0;
   if (const char* e = getenv("DEFL_TC_PAIR_MIN_N")) min_n = atoi(e);
   return N >= min_n;
 }

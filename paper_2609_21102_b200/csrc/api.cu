@@ -150,7 +150,7 @@ int orthonormalise(defl_ctx* c, float* P, int b, int rows, int l, double* gram, 
   // CholeskyQR: Gram(P); R = chol; P <- P R^-1. With passes = 2 (CholeskyQR2) the second Gram is taken in the
   // same panel pass as the first solve. The last pass can also write P as bf16 hi + lo for the next
   // tensor-core product.
-  const int nchunk = fused_num_chunks(rows);
+  const int nchunk = fused_num_chunks(rows, b);
   const long long bs = (long long)rows * l;
   if (ctx_fail(c, panel_fused_launch(P, bs, l, b, rows, l, nullptr, 0, l, nullptr, 0, 0, nullptr, nullptr, 0, gram,
                                      c->stream, &c->launches), "gram"))
@@ -235,7 +235,7 @@ int run_brsvd(defl_ctx* c, const void* G, int b, int m, int n, int dtype, int l,
   if (ctx_fail(c, panel_fused_launch(w.Sp, (long long)ms * l, l, b, ms, l, nullptr, 0, l, nullptr, 0, 0, nullptr, nullptr, 0,
                                      w.gram, c->stream, &c->launches), "gram core"))
     return DEFL_ERR_CUDA;
-  if (ctx_fail(c, jacobi_eig_launch(w.gram, fused_num_chunks(ms), b, l, 0, w.sv, w.E, w.Es, w.status, c->stream,
+  if (ctx_fail(c, jacobi_eig_launch(w.gram, fused_num_chunks(ms, b), b, l, 0, w.sv, w.E, w.Es, w.status, c->stream,
                                     &c->launches), "jacobi"))
     return DEFL_ERR_CUDA;
   if (k_keep > 0) {

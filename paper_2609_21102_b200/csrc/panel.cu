@@ -673,16 +673,31 @@ cudaError_t gate_launch(const float* s, int ld_s, int batch, int window, int kma
 // Fused panel pass for CholeskyQR2 and the triplet products: for panel In[b, rows, l]
 //   Out = In * Mtx[:, :kout]   (Mtx null: Out = In), written as fp32 and/or as bf16 hi + lo,
 //   and/or the Gram partials of Out (fp32 products over 128-row tiles, tiles added in fp64).
-// One CTA walks a chunk of FUSED_CHUNK rows in 128-row tiles; register-blocked 4 x 8 outputs per thread.
+// One CTA walks its share of the rows in 128-row tiles; register-blocked 4 x 8 outputs per thread.
 // In-place (Out == In) is safe: a tile is read completely before it is written.
 // ---------------------------------------------------------------------------------------------
 namespace defl {
 
 constexpr int FUSED_TILE = 128;
-constexpr int FUSED_CHUNK = 512;
 constexpr int FUSED_TS = MAX_L + 4;
 
-int fused_num_chunks(int rows) { return (rows + FUSED_CHUNK - 1) / FUSED_CHUNK; }
+// Rows are split over CTAs in whole 128-row tiles. The split is chosen so that all CTAs of the launch are resident
+// at once (four per SM with this kernel's shared memory): a fixed 512-row split gave 624 CTAs for 592 places on
+// the 48 x 6400-row panels, i.e. a second wave for 32 CTAs, and left two thirds of the GPU idle on 1600-row panels.
+// At least two tiles per CTA, so the count never exceeds gram_num_chunks(rows), which sizes the partials buffer.
+int fused_num_chunks(int rows, int batch) {
+  static int sms = 0;
+  if (sms <= 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+      sms = 148;
+  }
+  const int places = sms * 4;
+  const int tiles = (rows + FUSED_TILE - 1) / FUSED_TILE;
+  int t = 2;
+  while (t < tiles && (long long)((tiles + t - 1) / t) * batch > places) ++t;
+  return (tiles + t - 1) / t;
+}
 
 __global__ void __launch_bounds__(256) panel_fused_kernel(const float* In, long long in_bs, int ld_in, int rows, int l,
                                                           const float* __restrict__ Mtx, int ldm, int kout,
@@ -710,27 +725,26 @@ __global__ void __launch_bounds__(256) panel_fused_kernel(const float* In, long 
   for (int i = 0; i < 4; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) gacc[i][j] = 0.0;
-  const int r_begin = chunk * FUSED_CHUNK, r_end = min(rows, r_begin + FUSED_CHUNK);
+  const int tiles = (rows + FUSED_TILE - 1) / FUSED_TILE;
+  const int chunk_rows = ((tiles + nchunk - 1) / nchunk) * FUSED_TILE;
+  const int r_begin = chunk * chunk_rows, r_end = min(rows, r_begin + chunk_rows);
   for (int r0 = r_begin; r0 < r_end; r0 += FUSED_TILE) {
     __syncthreads();
-    if (ld_in == l && (l & 3) == 0 && ((reinterpret_cast<uintptr_t>(Ib) & 15) == 0)) {
-      // contiguous tile: all loads of a thread are issued before the first use (8 x 16 bytes in flight)
-      const float4* src = reinterpret_cast<const float4*>(Ib + (long long)r0 * l);
-      const int cnt4 = FUSED_TILE * l / 4;
-      float4 buf[FUSED_TILE * MAX_L / 4 / 256];
+    if ((ld_in & 3) == 0 && (l & 3) == 0 && ((reinterpret_cast<uintptr_t>(Ib) & 15) == 0)) {
+      // 16 threads per row (one float4 each, up to 64 columns), 16 rows per pass: no index division, and all
+      // eight loads of a thread are issued before the first use
+      const int c4 = tid & 15, rr0 = tid >> 4;
+      const bool col_ok = c4 * 4 < l;
+      float4 buf[FUSED_TILE / 16];
 #pragma unroll
-      for (int it = 0; it < FUSED_TILE * MAX_L / 4 / 256; ++it) {
-        const int f4 = tid + it * 256;
-        const int rr = (f4 * 4) / l;
-        buf[it] = (f4 < cnt4 && r0 + rr < r_end) ? src[f4] : make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int it = 0; it < FUSED_TILE / 16; ++it) {
+        const int rr = rr0 + it * 16;
+        buf[it] = (col_ok && r0 + rr < r_end) ? *reinterpret_cast<const float4*>(Ib + (long long)(r0 + rr) * ld_in + c4 * 4)
+                                              : make_float4(0.f, 0.f, 0.f, 0.f);
       }
+      if (col_ok) {
 #pragma unroll
-      for (int it = 0; it < FUSED_TILE * MAX_L / 4 / 256; ++it) {
-        const int f4 = tid + it * 256;
-        if (f4 < cnt4) {
-          const int rr = (f4 * 4) / l, c = (f4 * 4) % l;
-          tile[rr][c] = buf[it].x; tile[rr][c + 1] = buf[it].y; tile[rr][c + 2] = buf[it].z; tile[rr][c + 3] = buf[it].w;
-        }
+        for (int it = 0; it < FUSED_TILE / 16; ++it) *reinterpret_cast<float4*>(&tile[rr0 + it * 16][c4 * 4]) = buf[it];
       }
     } else {
       const int lr = (l + 3) & ~3;      // columns l..lr-1 are zeroed: the product walks the row in blocks of four
@@ -765,29 +779,72 @@ __global__ void __launch_bounds__(256) panel_fused_kernel(const float* In, long 
         }
       }
       __syncthreads();
+      // (columns wout.. of the tile receive zeros: the staged matrix has zero columns there)
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-          if (tx * 8 + j < wout) tile[ty * 4 + i][tx * 8 + j] = acc[i][j];
+      for (int i = 0; i < 4; ++i) {
+        *reinterpret_cast<float4*>(&tile[ty * 4 + i][tx * 8]) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+        *reinterpret_cast<float4*>(&tile[ty * 4 + i][tx * 8 + 4]) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
+      }
       __syncthreads();
     }
     if (Out) {
       float* Ob = Out + (long long)bz * out_bs;
-      for (int e = tid; e < FUSED_TILE * wout; e += 256) {
-        const int rr = e / wout, c = e % wout;
-        if (r0 + rr < r_end) Ob[(long long)(r0 + rr) * ld_out + c] = tile[rr][c];
+      if ((wout & 3) == 0 && (ld_out & 3) == 0 && ((reinterpret_cast<uintptr_t>(Ob) & 15) == 0)) {
+        const int c4 = tid & 15, rr0 = tid >> 4;
+        if (c4 * 4 < wout) {
+#pragma unroll
+          for (int it = 0; it < FUSED_TILE / 16; ++it) {
+            const int rr = rr0 + it * 16;
+            if (r0 + rr < r_end)
+              *reinterpret_cast<float4*>(Ob + (long long)(r0 + rr) * ld_out + c4 * 4) = *reinterpret_cast<const float4*>(&tile[rr][c4 * 4]);
+          }
+        }
+      } else {
+        for (int e = tid; e < FUSED_TILE * wout; e += 256) {
+          const int rr = e / wout, c = e % wout;
+          if (r0 + rr < r_end) Ob[(long long)(r0 + rr) * ld_out + c] = tile[rr][c];
+        }
       }
     }
     if (hi) {
-      for (int e = tid; e < FUSED_TILE * lp; e += 256) {
-        const int rr = e / lp, c = e % lp;
-        if (r0 + rr >= r_end) continue;
-        const float x = (c < wout) ? tile[rr][c] : 0.f;
-        const __nv_bfloat16 h = __float2bfloat16_rn(x);
-        const long long o = ((long long)bz * rows + r0 + rr) * lp + c;
-        hi[o] = h;
-        lo[o] = __float2bfloat16_rn(x - __bfloat162float(h));
+      if ((lp & 3) == 0 && lp <= 64 && ((reinterpret_cast<uintptr_t>(hi) | reinterpret_cast<uintptr_t>(lo)) & 7) == 0) {
+        // four values per thread: 8-byte stores of the hi and lo halves (tile columns wout..lp-1 may hold
+        // leftovers of the input, so they are masked here)
+        const int c4 = tid & 15, rr0 = tid >> 4;
+        if (c4 * 4 < lp) {
+#pragma unroll
+          for (int it = 0; it < FUSED_TILE / 16; ++it) {
+            const int rr = rr0 + it * 16;
+            if (r0 + rr >= r_end) continue;
+            const float4 x4 = *reinterpret_cast<const float4*>(&tile[rr][c4 * 4]);
+            float x[4] = {x4.x, x4.y, x4.z, x4.w};
+            __nv_bfloat16 h[4], lw[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              if (c4 * 4 + j >= wout) x[j] = 0.f;
+              h[j] = __float2bfloat16_rn(x[j]);
+              lw[j] = __float2bfloat16_rn(x[j] - __bfloat162float(h[j]));
+            }
+            const long long o = ((long long)bz * rows + r0 + rr) * lp + c4 * 4;
+            uint2 hv, lv;
+            hv.x = (uint32_t)__bfloat16_as_ushort(h[0]) | ((uint32_t)__bfloat16_as_ushort(h[1]) << 16);
+            hv.y = (uint32_t)__bfloat16_as_ushort(h[2]) | ((uint32_t)__bfloat16_as_ushort(h[3]) << 16);
+            lv.x = (uint32_t)__bfloat16_as_ushort(lw[0]) | ((uint32_t)__bfloat16_as_ushort(lw[1]) << 16);
+            lv.y = (uint32_t)__bfloat16_as_ushort(lw[2]) | ((uint32_t)__bfloat16_as_ushort(lw[3]) << 16);
+            *reinterpret_cast<uint2*>(hi + o) = hv;
+            *reinterpret_cast<uint2*>(lo + o) = lv;
+          }
+        }
+      } else {
+        for (int e = tid; e < FUSED_TILE * lp; e += 256) {
+          const int rr = e / lp, c = e % lp;
+          if (r0 + rr >= r_end) continue;
+          const float x = (c < wout) ? tile[rr][c] : 0.f;
+          const __nv_bfloat16 h = __float2bfloat16_rn(x);
+          const long long o = ((long long)bz * rows + r0 + rr) * lp + c;
+          hi[o] = h;
+          lo[o] = __float2bfloat16_rn(x - __bfloat162float(h));
+        }
       }
     }
     if (partial) {
@@ -829,7 +886,7 @@ cudaError_t panel_fused_launch(const float* In, long long in_bs, int ld_in, int 
                                __nv_bfloat16* lo, int lp, double* partial, cudaStream_t st, long long* launches) {
   const size_t smem = (size_t)(FUSED_TILE + MAX_L) * FUSED_TS * sizeof(float);
   cudaFuncSetAttribute(panel_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  const int nchunk = fused_num_chunks(rows);
+  const int nchunk = fused_num_chunks(rows, batch);
   panel_fused_kernel<<<dim3(nchunk, batch), 256, smem, st>>>(In, in_bs, ld_in, rows, l, Mtx, ldm, kout, Out, out_bs, ld_out,
                                                             hi, lo, lp, partial, nchunk);
   if (launches) ++*launches;

@@ -44,9 +44,9 @@ cudaError_t gate_launch(const float* s, int ld_s, int batch, int window, int kma
 }  // namespace defl
 
 namespace defl {
-int fused_num_chunks(int rows);
+int fused_num_chunks(int rows, int batch);
 // Out = In * Mtx[:, :kout] (Mtx null: identity), optional fp32 / bf16 hi+lo outputs, optional Gram partials of Out
-// ([b, fused_num_chunks(rows), w, w] fp64 with w = width of Out)
+// ([b, fused_num_chunks(rows, b), w, w] fp64 with w = width of Out)
 cudaError_t panel_fused_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int l, const float* Mtx,
                                int ldm, int kout, float* Out, long long out_bs, int ld_out, __nv_bfloat16* hi,
                                __nv_bfloat16* lo, int lp, double* partial, cudaStream_t st, long long* launches);

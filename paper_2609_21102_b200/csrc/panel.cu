@@ -682,7 +682,7 @@ constexpr int FUSED_TILE = 128;
 constexpr int FUSED_TS = MAX_L + 4;
 
 // Rows are split over CTAs in whole 128-row tiles. The split is chosen so that all CTAs of the launch are resident
-// at once (four per SM with this kernel's shared memory): a fixed 512-row split gave 624 CTAs for 592 places on
+// at once (two per SM with this kernel's registers): a fixed 512-row split gave 624 CTAs for 592 places on
 // the 48 x 6400-row panels, i.e. a second wave for 32 CTAs, and left two thirds of the GPU idle on 1600-row panels.
 // At least two tiles per CTA, so the count never exceeds gram_num_chunks(rows), which sizes the partials buffer.
 int fused_num_chunks(int rows, int batch) {
@@ -692,14 +692,14 @@ int fused_num_chunks(int rows, int batch) {
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
       sms = 148;
   }
-  const int places = sms * 4;
+  const int places = sms * 2;
   const int tiles = (rows + FUSED_TILE - 1) / FUSED_TILE;
   int t = 2;
   while (t < tiles && (long long)((tiles + t - 1) / t) * batch > places) ++t;
   return (tiles + t - 1) / t;
 }
 
-__global__ void __launch_bounds__(256) panel_fused_kernel(const float* In, long long in_bs, int ld_in, int rows, int l,
+__global__ void __launch_bounds__(256, 2) panel_fused_kernel(const float* In, long long in_bs, int ld_in, int rows, int l,
                                                           const float* __restrict__ Mtx, int ldm, int kout,
                                                           float* Out, long long out_bs, int ld_out,
                                                           __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
@@ -719,12 +719,26 @@ __global__ void __launch_bounds__(256) panel_fused_kernel(const float* In, long 
     }
   }
   const int ty = tid >> 3, tx = tid & 7;        // product: rows ty*4.., cols tx*8..
-  const int gy = tid >> 4, gx = tid & 15;       // Gram: block (gy*4.., gx*4..)
-  double gacc[4][4];
+  // Gram: the upper block triangle of W = In^T In (or Out^T Out) in blocks of 4 rows x 8 columns; the threads form
+  // `ngrp` groups of `nblk` (one block each), group g takes the rows g, g + ngrp, ... of every tile. fp32 sums
+  // per thread (at most rows-per-CTA / ngrp terms), added up over the groups in fp64 at the end, in a fixed order.
+  const int nb4 = (wout + 3) >> 2, nb8 = (wout + 7) >> 3;
+  int nblk = 0;
+  for (int j = 0; j < nb8; ++j) nblk += min(nb4, 2 * j + 2);
+  const int ngrp = min(16, 256 / nblk);
+  const int grp = tid / nblk;
+  const bool gram_on = partial != nullptr && grp < ngrp;
+  int bi = 0, bj = 0;          // this thread's block: rows 4 bi.., columns 8 bj.. of W
+  {
+    int rem = tid - grp * nblk;
+    while (bj < nb8 - 1 && rem >= min(nb4, 2 * bj + 2)) { rem -= min(nb4, 2 * bj + 2); ++bj; }
+    bi = rem;
+  }
+  float g8[4][8];
 #pragma unroll
   for (int i = 0; i < 4; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) gacc[i][j] = 0.0;
+    for (int j = 0; j < 8; ++j) g8[i][j] = 0.f;
   const int tiles = (rows + FUSED_TILE - 1) / FUSED_TILE;
   const int chunk_rows = ((tiles + nchunk - 1) / nchunk) * FUSED_TILE;
   const int r_begin = chunk * chunk_rows, r_end = min(rows, r_begin + chunk_rows);
@@ -847,37 +861,45 @@ __global__ void __launch_bounds__(256) panel_fused_kernel(const float* In, long 
         }
       }
     }
-    if (partial) {
-      float f[4][4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) f[i][j] = 0.f;
+    if (gram_on) {
       const int nr = min(FUSED_TILE, r_end - r0);
-      for (int rr = 0; rr < nr; ++rr) {
-        const float4 a4 = *reinterpret_cast<const float4*>(&tile[rr][gy * 4]);
-        const float4 b4 = *reinterpret_cast<const float4*>(&tile[rr][gx * 4]);
-        const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
+      for (int rr = grp; rr < nr; rr += ngrp) {
+        const float4 a0 = *reinterpret_cast<const float4*>(&tile[rr][bi * 4]);
+        const float4 b0 = *reinterpret_cast<const float4*>(&tile[rr][bj * 8]);
+        const float4 b1 = *reinterpret_cast<const float4*>(&tile[rr][bj * 8 + 4]);
+        const float a[4] = {a0.x, a0.y, a0.z, a0.w};
+        const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i)
 #pragma unroll
-          for (int j = 0; j < 4; ++j) f[i][j] = fmaf(a[i], b[j], f[i][j]);
+          for (int j = 0; j < 8; ++j) g8[i][j] = fmaf(a[i], b[j], g8[i][j]);
       }
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) gacc[i][j] += (double)f[i][j];
     }
   }
   if (partial) {
-    double* out = partial + ((long long)bz * nchunk + chunk) * wout * wout;
+    // sum over the groups in fp64 (group order fixed: the result does not depend on timing), in the tile's memory
+    double* red = reinterpret_cast<double*>(fsm);        // [wout][wout], upper blocks only
+    __syncthreads();
+    for (int e = tid; e < wout * wout; e += 256) red[e] = 0.0;
+    __syncthreads();
+    for (int g = 0; g < ngrp; ++g) {
+      if (gram_on && grp == g) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+        for (int i = 0; i < 4; ++i)
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int gi = gy * 4 + i, gj = gx * 4 + j;
-        if (gi < wout && gj < wout) out[gi * wout + gj] = gacc[i][j];
+          for (int j = 0; j < 8; ++j) {
+            const int gi = bi * 4 + i, gj = bj * 8 + j;
+            if (gi < wout && gj < wout) red[gi * wout + gj] += (double)g8[i][j];
+          }
       }
+      __syncthreads();
+    }
+    double* out = partial + ((long long)bz * nchunk + chunk) * wout * wout;
+    for (int e = tid; e < wout * wout; e += 256) {
+      const int gi = e / wout, gj = e - gi * wout;
+      // blocks below the block diagonal were not computed: take the mirror image
+      out[e] = ((gi >> 3) <= (gj >> 3)) ? red[e] : red[gj * wout + gi];
+    }
   }
 }
 

@@ -122,24 +122,34 @@ __global__ void __launch_bounds__(512) chol_inv_kernel(const double* __restrict_
       const int i = e / l, j = e % l;
       Lm[e] = W[e] + ((i == j) ? shift : 0.0);
     }
-    if (tid == 0) bad = 0;
     __syncthreads();
-    // right-looking Cholesky on the lower triangle
+    // Right-looking Cholesky on the lower triangle, one barrier per column: in phase j every thread reads the
+    // pivot d_j itself (so a bad pivot is seen by all alike), the trailing block is updated from the UNSCALED
+    // column j times 1/d_j, and column j-1 (which nobody reads any more) is scaled in passing.
+    // (one reciprocal square root per column and thread: 1/d = rsqrt(d)^2, sqrt(d) = d rsqrt(d); a division and a
+    // square root in fp64 cost several hundred cycles of latency each, more than the rest of the column)
+    bool failed = false;
+    double sd_prev = 1.0, isd_prev = 1.0;
+    const int ti = tid >> 6, tc = tid & 63;        // 8 rows x 64 columns of the trailing block per pass
     for (int j = 0; j < l; ++j) {
       const double d = Lm[j * l + j];
-      if (!(d > 0.0) || !isfinite(d)) { if (tid == 0) bad = 1; }
-      __syncthreads();
-      if (bad) break;
-      const double sd = sqrt(d), isd = 1.0 / sd;
-      for (int i = j + tid; i < l; i += blockDim.x) Lm[i * l + j] = (i == j) ? sd : Lm[i * l + j] * isd;
-      __syncthreads();
-      const int rem = l - j - 1;
-      for (int e = tid; e < rem * rem; e += blockDim.x) {
-        const int i = j + 1 + e / rem, c = j + 1 + e % rem;
-        if (c <= i) Lm[i * l + c] -= Lm[i * l + j] * Lm[c * l + j];
+      if (!(d > 0.0) || !isfinite(d)) { failed = true; break; }
+      const double isd = rsqrt(d), inv_d = isd * isd;
+      if (j > 0) {
+        for (int i = j - 1 + tid; i < l; i += blockDim.x) Lm[i * l + j - 1] = (i == j - 1) ? sd_prev : Lm[i * l + j - 1] * isd_prev;
       }
+      const int c = j + 1 + tc;
+      if (c < l) {
+        const double lc = Lm[c * l + j] * inv_d;
+        for (int i = j + 1 + ti; i < l; i += 8)
+          if (c <= i) Lm[i * l + c] -= Lm[i * l + j] * lc;
+      }
+      sd_prev = d * isd; isd_prev = isd;
       __syncthreads();
     }
+    if (!failed && tid == 0) Lm[(l - 1) * l + l - 1] = sd_prev;
+    if (tid == 0) bad = failed ? 1 : 0;
+    __syncthreads();
     if (!bad) break;
     // shift as in shifted CholeskyQR: proportional to the trace, growing per attempt
     shift = (shift == 0.0) ? 1e-10 * (trace > 0.0 ? trace : 1.0) : shift * 100.0;

@@ -300,11 +300,18 @@ __global__ void __launch_bounds__(1024) jacobi_eig_kernel(const double* __restri
           const double alpha = warp_sum(x0 * x0 + x1 * x1);
           const double beta = warp_sum(y0 * y0 + y1 * y1);
           const double gamma = warp_sum(x0 * y0 + x1 * y1);
-          if (gamma != 0.0 && fabs(gamma) > 1e-14 * sqrt(alpha * beta)) {
+          // rotate when |gamma| > 1e-14 sqrt(alpha beta) (compared in squares). The rotation is built from one
+          // division and two reciprocal square roots: fp64 divisions and square roots are long instruction
+          // sequences, and this chain is the latency of a round.
+          if (gamma != 0.0 && gamma * gamma > 1e-28 * (alpha * beta)) {
             if (lane == 0) rotated = 1;
             const double zeta = (beta - alpha) / (2.0 * gamma);
-            const double t = ((zeta >= 0.0) ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
-            const double c = 1.0 / sqrt(1.0 + t * t), sn = c * t;
+            const double w = 1.0 + zeta * zeta;
+            const double root = w * rsqrt(w);                          // sqrt(1 + zeta^2)
+            // t = sign(zeta) / (|zeta| + root) = sign(zeta) (root - |zeta|)   [(root - |zeta|)(root + |zeta|) = 1],
+            // evaluated in the stable form for large |zeta|: 1 / (|zeta| + root) = rsqrt-free via one more division
+            const double t = ((zeta >= 0.0) ? 1.0 : -1.0) / (fabs(zeta) + root);
+            const double c = rsqrt(1.0 + t * t), sn = c * t;
             if (lane < l) { ap[lane] = c * x0 - sn * y0; aq[lane] = sn * x0 + c * y0; }
             if (lane + 32 < l) { ap[lane + 32] = c * x1 - sn * y1; aq[lane + 32] = sn * x1 + c * y1; }
             double* vp = V + p * l; double* vq = V + q * l;

@@ -86,3 +86,25 @@ def test_symmetric_mirroring(ctx, engine_name):
     ref = _ref(A, A, False, True)
     assert torch.allclose(C, ref, rtol=1e-4, atol=2e-3)
     assert torch.equal(C, C.transpose(1, 2))
+
+
+@pytest.mark.parametrize("knobs", [{"DEFL_TC_PAIR": "0"}, {"DEFL_TC_KSUB": "1"}, {"DEFL_TC_TILE_M": "128"},
+                                   {"DEFL_TC_STAGES": "2"}])
+@pytest.mark.parametrize("sym", [False, True])
+def test_tensor_engine_other_tile_forms(ctx, monkeypatch, knobs, sym):
+    """The tile forms the default rules do not pick for these shapes (single-CTA 256-row tile, one K block per
+    stage, 128-row tiles, the shallowest pipeline) stay correct: the knobs are read per launch."""
+    from paper_2609_21102_b200 import binding
+    for k, v in knobs.items():
+        monkeypatch.setenv(k, v)
+    A = _mk(2, 712, 1096, torch.bfloat16, 9)          # ragged in M (712 = 2 x 256 + 200), K = 17.1 blocks
+    if sym:
+        C = ctx.defl_debug_gemm(A, A, False, True, engine=binding.ENGINE_TENSOR, out_dtype=torch.float32,
+                                exploit_symmetry=True)
+        ref = _ref(A, A, False, True)
+        assert torch.equal(C, C.transpose(1, 2))
+    else:
+        B = _mk(2, 1096, 328, torch.bfloat16, 10)     # MN-major right operand, ragged N
+        C = ctx.defl_debug_gemm(A, B, False, False, engine=binding.ENGINE_TENSOR, out_dtype=torch.float32)
+        ref = _ref(A, B, False, False)
+    assert torch.allclose(C, ref, rtol=1e-4, atol=4e-3)

@@ -335,10 +335,28 @@ def main():
     if rank == 0 or world > 1:
         hG = [g["G"].cpu().pin_memory() for g in groups]
         hO = [torch.empty_like(h).pin_memory() for h in hG]
+        def e2e_group(c, h, o, g, stream=None):
+            if stream is None:
+                c.defl_polar_batched_host(h, o, wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], sketch=g["Om"], gamma=1.01,
+                                          exploit_symmetry=SYM)
+            else:
+                torch.cuda.set_device(local_rank)
+                with torch.cuda.stream(stream):
+                    c.defl_polar_batched_host(h, o, wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], sketch=g["Om"],
+                                              gamma=1.01, exploit_symmetry=SYM)
+
         def e2e_step():
-            for h, o, g in zip(hG, hO, groups):
-                ctx.defl_polar_batched_host(h, o, wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], sketch=g["Om"], gamma=1.01,
-                                            exploit_symmetry=SYM)
+            # the call blocks until its output sits in host memory; with one context per shape group the groups
+            # run from host threads of their own, so that one group's copies overlap the other's computation
+            if not lanes:
+                for h, o, g in zip(hG, hO, groups):
+                    e2e_group(ctx, h, o, g)
+                return
+            ts = [threading.Thread(target=e2e_group, args=(c, h, o, g, s)) for (c, s), h, o, g in zip(lanes, hG, hO, groups)]
+            for t in ts:
+                t.start()
+            for t in ts:
+                t.join()
         e2e_step()
         barrier()
         t0 = time.perf_counter()

@@ -129,6 +129,27 @@ int defl_polar_batched_host(defl_ctx* ctx, const void* G_host, void* out_host, i
                             int k, int oversample, int power_iters,
                             const float* coeff_schedule, int L, const defl_opts* opts);
 
+/* One Deflated Muon step for a group of same-shape matrices (Section 3, "Muon with deflation": the polar-factor
+ * routine inside Muon is replaced by Algorithm 3 + Algorithm 1, once per shape group; Section 1, "Two
+ * applications": W <- W - lambda polar(M) with M the momentum matrix). In this order, all on the context's stream:
+ *   Mom <- mu * Mom + Grad              (skipped when Grad is NULL: Mom is then taken as it is)
+ *   D    = Mom, or Grad + mu * Mom when `nesterov` is non-zero (Mom here is the new momentum as stored)
+ *   W   <- (1 - lr * weight_decay) * W - lr * scale * F(D)
+ * where F is exactly what defl_polar_batched computes (same k, oversample, power_iters, schedule, opts, info).
+ * The weight update is the epilogue of the last filter product (and of the restore product in ADD mode): F(D) is
+ * never written to memory. The paper fixes only the last line with lr = lambda, scale = 1, weight_decay = 0; the
+ * momentum rule, Nesterov form, decoupled weight decay and `scale` are the usual Muon conventions, stated here
+ * because the paper takes them from the Muon references.
+ *   W    device, [b,m,n] row-major, type w_dtype (DEFL_BF16 | DEFL_F32), updated in place
+ *   Mom  device, [b,m,n], type dtype, updated in place;  Grad  device, [b,m,n], type dtype, not modified, or NULL
+ * L >= 1 is required (the update rides on the last product). Scratch: the context's workspace plus two buffers of
+ * b*m*n elements of `dtype` that it keeps. Errors as defl_polar_batched; DEFL_ERR_ARG also for nesterov without
+ * Grad. */
+int defl_muon_step_batched(defl_ctx* ctx, void* W, int w_dtype, void* Mom, const void* Grad, int b, int m, int n,
+                           int dtype, float lr, float mu, int nesterov, float weight_decay, float scale,
+                           int k, int oversample, int power_iters, const float* coeff_schedule, int L,
+                           const defl_opts* opts, const defl_info* info);
+
 /* Batched randomized SVD alone (Algorithm 3) in the caller's orientation:
  *   G ~ P diag(s) W^T with P [b,m,l], s [b,l] descending, W [b,n,l], all fp32; l = min(min(m,n), k+oversample).
  * Any of P, s, W may be NULL. The sketch comes from opts as above. */

@@ -150,6 +150,39 @@ def deflated_polar(G, k, l, Omega, J, coeffs, tau=0.0, gamma=1.01, mode=PADDED):
     return out, s[:l], int(info[0]), float(info[1])
 
 
+def round_to_storage(x, storage):
+    """Values as a `storage` buffer holds them: None or 'f64' = unchanged, 'f32', or 'bf16' (round to nearest, ties to
+    even, on the float32 bit pattern: keep the upper 16 bits after adding 0x7FFF plus the lowest kept bit)."""
+    if storage in (None, "f64"):
+        return np.array(x, dtype=np.float64)
+    x32 = np.ascontiguousarray(np.asarray(x, dtype=np.float64).astype(np.float32))
+    if storage == "f32":
+        return x32.astype(np.float64)
+    if storage != "bf16":
+        raise ValueError(storage)
+    bits = x32.view(np.uint32).astype(np.uint64)
+    bits = ((bits + 0x7FFF + ((bits >> 16) & 1)) >> 16) << 16
+    return bits.astype(np.uint32).view(np.float32).reshape(x32.shape).astype(np.float64)
+
+
+def muon_step(W, Mom, Grad, lr, mu, k, l, Omega, J, coeffs, nesterov=False, weight_decay=0.0, scale=1.0,
+              storage=None, tau=0.0, gamma=1.01, mode=PADDED):
+    """One Deflated Muon step on one matrix (Section 1, "Two applications": W <- W - lambda polar(M), M the momentum
+    matrix; Section 3, "Muon with deflation": polar is Algorithm 3 + Algorithm 1). The momentum rule, Nesterov form,
+    decoupled weight decay and `scale` follow the usual Muon conventions (the paper takes them from its Muon
+    references): Mom' = mu Mom + Grad, kept in `storage`; D = Mom' or Grad + mu Mom'; W' = (1 - lr wd) W - lr scale F(D).
+    Returns (W', Mom')."""
+    W, Mom = _f64(W), _f64(Mom)
+    if Grad is None:
+        Mom1 = Mom.copy()
+    else:
+        Grad = _f64(Grad)
+        Mom1 = round_to_storage(mu * Mom + Grad, storage)
+    D = (Grad + mu * Mom1) if nesterov else Mom1
+    F = deflated_polar(D, k, l, Omega, J, coeffs, tau=tau, gamma=gamma, mode=mode)[0]
+    return (1.0 - lr * weight_decay) * W - lr * scale * F, Mom1
+
+
 def lanczos_upper(Z, v0, steps=20):
     Z, v0 = _f64(Z), _f64(v0)
     return float(lib().orc_lanczos_upper(_L(Z.shape[0]), _p(Z), _I(steps), _p(v0)))

@@ -25,7 +25,7 @@ CLASSICAL_QUINTIC = (1.875, -1.25, 0.375)
 
 EXPORTS = [
     "defl_create", "defl_destroy", "defl_set_stream", "defl_polar_workspace_bytes", "defl_psd_workspace_bytes",
-    "defl_polar_batched", "defl_polar_batched_host", "defl_brsvd_batched", "defl_psd_project", "defl_fill_gaussian", "defl_debug_gemm",
+    "defl_polar_batched", "defl_polar_batched_host", "defl_muon_step_batched", "defl_brsvd_batched", "defl_psd_project", "defl_fill_gaussian", "defl_debug_gemm",
     "defl_frobenius_norms_noalloc", "defl_set_profiling", "defl_get_stage_ms", "defl_launch_count", "defl_status_string", "defl_last_error",
 ]
 
@@ -61,6 +61,9 @@ def lib():
             ctypes.POINTER(ctypes.c_float), ctypes.c_int, ctypes.POINTER(DeflOpts), ctypes.POINTER(DeflInfo)]
         L.defl_polar_batched_host.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 7 + [
             ctypes.POINTER(ctypes.c_float), ctypes.c_int, ctypes.POINTER(DeflOpts)]
+        L.defl_muon_step_batched.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p] + [
+            ctypes.c_int] * 4 + [ctypes.c_float, ctypes.c_float, ctypes.c_int, ctypes.c_float, ctypes.c_float] + [
+            ctypes.c_int] * 3 + [ctypes.POINTER(ctypes.c_float), ctypes.c_int, ctypes.POINTER(DeflOpts), ctypes.POINTER(DeflInfo)]
         L.defl_brsvd_batched.argtypes = [ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 7 + [
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(DeflOpts), ctypes.c_void_p]
         L.defl_psd_project.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
@@ -195,6 +198,34 @@ class Context:
                                       sched, L, ctypes.byref(opts), ctypes.byref(info))
         self._check(rc)
         return (out, extras) if want_info else out
+
+    def defl_muon_step_batched(self, W, Mom, Grad, lr, mu, k, oversample, power_iters, coeff_schedule, steps=None,
+                               nesterov=False, weight_decay=0.0, scale=1.0, sketch=None, seed=0,
+                               restore_mode=RESTORE_PADDED, gamma=0.0, engine=ENGINE_AUTO, exploit_symmetry=False,
+                               tau=0.0):
+        """One Deflated Muon step on a shape group, in place: Mom <- mu Mom + Grad (Grad may be None),
+        W <- (1 - lr wd) W - lr scale F(Mom or its Nesterov look-ahead), F = defl_polar_batched's map."""
+        _dev(W, "W"), _dev(Mom, "Mom")
+        if Mom.ndim != 3 or W.shape != Mom.shape:
+            raise ValueError("W and Mom must be [b, m, n] of the same shape")
+        if Grad is not None:
+            _dev(Grad, "Grad")
+            if Grad.shape != Mom.shape or Grad.dtype != Mom.dtype:
+                raise ValueError("Grad must match Mom in shape and type")
+        b, m, n = Mom.shape
+        sched, L = _schedule(coeff_schedule, steps)
+        if sketch is not None:
+            _dev(sketch, "sketch")
+            if sketch.dtype != torch.float32:
+                raise TypeError("sketch must be float32")
+        opts = self._opts(sketch=sketch, seed=seed, restore_mode=restore_mode, gamma=gamma, engine=engine,
+                          exploit_symmetry=exploit_symmetry, tau=tau)
+        self._sync_stream()
+        rc = lib().defl_muon_step_batched(self._h, _ptr(W), _dtype_code(W), _ptr(Mom), _ptr(Grad) if Grad is not None else None,
+                                          b, m, n, _dtype_code(Mom), lr, mu, int(bool(nesterov)), weight_decay, scale,
+                                          k, oversample, power_iters, sched, L, ctypes.byref(opts), None)
+        self._check(rc)
+        return W
 
     def defl_polar_batched_host(self, G_host, out_host, k, oversample, power_iters, coeff_schedule, steps=None,
                                 sketch=None, seed=0, restore_mode=RESTORE_PADDED, gamma=0.0, engine=ENGINE_AUTO,

@@ -412,13 +412,21 @@ int defl_brsvd_batched(defl_ctx* c, const void* G, int b, int m, int n, int dtyp
   return DEFL_OK;
 }
 
-int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int n, int dtype, int k, int oversample,
-                       int power_iters, const float* coeff_schedule, int L, const defl_opts* opts,
-                       const defl_info* info) {
+// Weight update fused into the last product of the chain: W <- keep * W + step * (result of Algorithm 1)
+struct WeightUpdate {
+  void* W;
+  int w_dtype;
+  float keep, step;
+};
+
+static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n, int dtype, int k, int oversample,
+                      int power_iters, const float* coeff_schedule, int L, const defl_opts* opts,
+                      const defl_info* info, const WeightUpdate* upd) {
   if (!c || !G || !out || b <= 0 || m <= 0 || n <= 0 || k < 0 || oversample < 0 || power_iters < 0 || L < 0)
     return DEFL_ERR_ARG;
   if (dtype != DEFL_BF16 && dtype != DEFL_F32) return DEFL_ERR_ARG;
   if (L > 0 && !coeff_schedule) return DEFL_ERR_ARG;
+  if (upd && (L < 1 || !upd->W)) return DEFL_ERR_ARG;      // the update rides on the last filter product
   const size_t es = dtype_size(dtype);
   const size_t gbytes = (size_t)b * m * n * es;
   {
@@ -571,6 +579,12 @@ int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int 
     }
     g.C = Xn; g.ldc = n; g.batch_c = (long long)m * n;
     g.epilogue = EPI_STORE;
+    if (upd && t == L - 1) {
+      // last step of a Muon update: W <- keep W + step (B_L X) instead of storing the iterate
+      g.C = upd->W; g.out_dtype = upd->w_dtype;
+      g.aux = upd->W; g.ld_aux = n; g.batch_aux = (long long)m * n; g.aux_dtype = upd->w_dtype;
+      g.epilogue = EPI_AUX_PLUS; g.alpha = upd->step; g.aux_scale = upd->keep;
+    }
     if ((rc = run_gemm(c, g, engine, "apply"))) return rc;
     cur ^= 1;
   }
@@ -584,6 +598,10 @@ int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int 
     g.aux = out; g.ld_aux = n; g.batch_aux = (long long)m * n; g.aux_dtype = dtype;
     g.C = out; g.ldc = n; g.batch_c = (long long)m * n; g.out_dtype = dtype;
     g.epilogue = EPI_AUX_PLUS;
+    if (upd) {      // Muon update: the head joins the weights with the same step, W <- W + step P W^T
+      g.aux = upd->W; g.aux_dtype = upd->w_dtype; g.C = upd->W; g.out_dtype = upd->w_dtype;
+      g.alpha = upd->step; g.aux_scale = 1.f;
+    }
     bool tensor_restore = false;
     if (dtype == BF16 && engine != DEFL_ENGINE_SIMT) {
       g.K[0] = 3 * kp;
@@ -633,6 +651,50 @@ int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int 
 }
 
 
+int defl_polar_batched(defl_ctx* c, const void* G, void* out, int b, int m, int n, int dtype, int k, int oversample,
+                       int power_iters, const float* coeff_schedule, int L, const defl_opts* opts,
+                       const defl_info* info) {
+  return polar_core(c, G, out, b, m, n, dtype, k, oversample, power_iters, coeff_schedule, L, opts, info, nullptr);
+}
+
+static int ensure_staging(defl_ctx* c, size_t bytes) {
+  if (bytes <= c->stage_bytes) return DEFL_OK;
+  cudaDeviceSynchronize();
+  if (c->stage_in) cudaFree(c->stage_in);
+  if (c->stage_out) cudaFree(c->stage_out);
+  c->stage_in = c->stage_out = nullptr;
+  c->stage_bytes = 0;
+  if (ctx_fail(c, cudaMalloc(&c->stage_in, bytes), "cudaMalloc(staging)")) return DEFL_ERR_CUDA;
+  if (ctx_fail(c, cudaMalloc(&c->stage_out, bytes), "cudaMalloc(staging)")) return DEFL_ERR_CUDA;
+  c->stage_bytes = bytes;
+  return DEFL_OK;
+}
+
+int defl_muon_step_batched(defl_ctx* c, void* W, int w_dtype, void* Mom, const void* Grad, int b, int m, int n,
+                           int dtype, float lr, float mu, int nesterov, float weight_decay, float scale, int k,
+                           int oversample, int power_iters, const float* coeff_schedule, int L,
+                           const defl_opts* opts, const defl_info* info) {
+  if (!c || !W || !Mom || b <= 0 || m <= 0 || n <= 0) return DEFL_ERR_ARG;
+  if ((dtype != DEFL_BF16 && dtype != DEFL_F32) || (w_dtype != DEFL_BF16 && w_dtype != DEFL_F32)) return DEFL_ERR_ARG;
+  if (L < 1 || !coeff_schedule) return DEFL_ERR_ARG;
+  if (nesterov && !Grad) return DEFL_ERR_ARG;
+  cudaSetDevice(c->device);
+  const size_t count = (size_t)b * m * n;
+  int rc = ensure_staging(c, count * dtype_size(dtype));
+  if (rc) return rc;
+  // momentum, then the matrix whose polar factor is taken: the stored momentum itself, or the Nesterov look-ahead
+  const void* D = Mom;
+  if (Grad) {
+    void* look = nesterov ? c->stage_in : nullptr;
+    if (ctx_fail(c, momentum_launch(Mom, Grad, look, dtype, (long long)count, mu, c->stream, &c->launches), "momentum"))
+      return DEFL_ERR_CUDA;
+    if (nesterov) D = look;
+  }
+  WeightUpdate upd;
+  upd.W = W; upd.w_dtype = w_dtype; upd.keep = 1.f - lr * weight_decay; upd.step = -lr * scale;
+  return polar_core(c, D, c->stage_out, b, m, n, dtype, k, oversample, power_iters, coeff_schedule, L, opts, info, &upd);
+}
+
 int defl_polar_batched_host(defl_ctx* c, const void* G_host, void* out_host, int b, int m, int n, int dtype, int k,
                             int oversample, int power_iters, const float* coeff_schedule, int L,
                             const defl_opts* opts) {
@@ -640,16 +702,7 @@ int defl_polar_batched_host(defl_ctx* c, const void* G_host, void* out_host, int
   if (dtype != DEFL_BF16 && dtype != DEFL_F32) return DEFL_ERR_ARG;
   cudaSetDevice(c->device);
   const size_t bytes = (size_t)b * m * n * dtype_size(dtype);
-  if (bytes > c->stage_bytes) {
-    cudaDeviceSynchronize();
-    if (c->stage_in) cudaFree(c->stage_in);
-    if (c->stage_out) cudaFree(c->stage_out);
-    c->stage_in = c->stage_out = nullptr;
-    c->stage_bytes = 0;
-    if (ctx_fail(c, cudaMalloc(&c->stage_in, bytes), "cudaMalloc(staging)")) return DEFL_ERR_CUDA;
-    if (ctx_fail(c, cudaMalloc(&c->stage_out, bytes), "cudaMalloc(staging)")) return DEFL_ERR_CUDA;
-    c->stage_bytes = bytes;
-  }
+  if (ensure_staging(c, bytes)) return DEFL_ERR_CUDA;
   // The batch is independent matrices: it goes through in chunks, the copy of chunk i+1 to the device and of
   // chunk i-1 back to the host running (on streams of their own) while chunk i is computed. Few chunks: the small
   // kernels of the range finder take about the same time for 12 matrices as for 48.

@@ -932,4 +932,59 @@ cudaError_t panel_fused_launch(const float* In, long long in_bs, int ld_in, int 
   return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------------
+// Momentum of a Muon step, element-wise in fp32: Mom <- mu Mom + Grad, stored in the momentum's type; when `look`
+// is given it receives Grad + mu Mom' with Mom' the STORED (rounded) new momentum, i.e. the Nesterov look-ahead
+// is a function of the optimizer state as it is kept in memory.
+// ---------------------------------------------------------------------------------------------
+template <typename T, int V>
+__global__ void __launch_bounds__(256) momentum_vec_kernel(T* Mom, const T* __restrict__ Grad, T* look, long long nvec, float mu) {
+  // V elements (16 bytes) per thread and trip
+  struct alignas(16) Pack { T v[V]; };
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
+    const Pack g = reinterpret_cast<const Pack*>(Grad)[i];
+    Pack m = reinterpret_cast<const Pack*>(Mom)[i];
+    Pack l;
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      const float gf = (float)g.v[j];
+      m.v[j] = (T)fmaf(mu, (float)m.v[j], gf);
+      l.v[j] = (T)fmaf(mu, (float)m.v[j], gf);          // from the momentum as stored
+    }
+    reinterpret_cast<Pack*>(Mom)[i] = m;
+    if (look) reinterpret_cast<Pack*>(look)[i] = l;
+  }
+}
+
+__global__ void __launch_bounds__(256) momentum_kernel(void* Mom, const void* __restrict__ Grad, void* look, int dtype,
+                                                       long long first, long long count, float mu) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = first + (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += stride) {
+    const float g = ld_as_float(Grad, i, dtype);
+    st_from_float(Mom, i, dtype, fmaf(mu, ld_as_float(Mom, i, dtype), g));
+    if (look) st_from_float(look, i, dtype, fmaf(mu, ld_as_float(Mom, i, dtype), g));
+  }
+}
+cudaError_t momentum_launch(void* Mom, const void* Grad, void* look, int dtype, long long count, float mu, cudaStream_t st,
+                            long long* launches) {
+  if (count <= 0) return cudaSuccess;
+  const bool aligned = ((reinterpret_cast<uintptr_t>(Mom) | reinterpret_cast<uintptr_t>(Grad) | reinterpret_cast<uintptr_t>(look)) & 15) == 0;
+  const int per = (dtype == BF16) ? 8 : 4;
+  const long long nvec = aligned ? count / per : 0;
+  if (nvec > 0) {
+    const int nblk = (int)min((long long)148 * 16, (nvec + 255) / 256);
+    if (dtype == BF16)
+      momentum_vec_kernel<__nv_bfloat16, 8><<<nblk, 256, 0, st>>>((__nv_bfloat16*)Mom, (const __nv_bfloat16*)Grad, (__nv_bfloat16*)look, nvec, mu);
+    else
+      momentum_vec_kernel<float, 4><<<nblk, 256, 0, st>>>((float*)Mom, (const float*)Grad, (float*)look, nvec, mu);
+    if (launches) ++*launches;
+  }
+  if (nvec * per < count) {      // the unaligned or leftover part
+    momentum_kernel<<<1, 256, 0, st>>>(Mom, Grad, look, dtype, nvec * per, count, mu);
+    if (launches) ++*launches;
+  }
+  return cudaGetLastError();
+}
+
 }  // namespace defl

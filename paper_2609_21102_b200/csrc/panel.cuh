@@ -50,4 +50,8 @@ int fused_num_chunks(int rows, int batch);
 cudaError_t panel_fused_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int l, const float* Mtx,
                                int ldm, int kout, float* Out, long long out_bs, int ld_out, __nv_bfloat16* hi,
                                __nv_bfloat16* lo, int lp, double* partial, cudaStream_t st, long long* launches);
+// Muon momentum: Mom <- mu Mom + Grad (stored type `dtype`); look (may be null) <- Grad + mu Mom_stored
+cudaError_t momentum_launch(void* Mom, const void* Grad, void* look, int dtype, long long count, float mu, cudaStream_t st,
+                            long long* launches);
+
 }  // namespace defl

@@ -52,3 +52,19 @@ def test_status_strings_and_no_device_behaviour(libpath):
         # no CPU fallback: without a device the context cannot even be created
         assert L.defl_create(ctypes.byref(h), 0) == -3
         assert not h.value
+
+
+def test_shape_groups_and_stacking():
+    """Host-side grouping of a parameter list by stored shape (no GPU, no arithmetic)."""
+    import torch
+    from paper_2609_21102_b200 import grouping
+    shapes = [(8, 4), (4, 8), (8, 4), (3,), (8, 4), (4, 8), (2, 2, 2)]
+    g = grouping.shape_groups(shapes)
+    assert list(g.items()) == [((8, 4), [0, 2, 4]), ((4, 8), [1, 5])]
+    ts = [torch.full(s, float(i)) for i, s in enumerate(shapes)]
+    buf, views = grouping.stack_group(ts, g[(8, 4)])
+    assert buf.shape == (3, 8, 4) and [float(v[0, 0]) for v in views] == [0.0, 2.0, 4.0]
+    views[1].add_(1.0)                      # a view writes through to the stacked buffer
+    assert float(buf[1, 3, 3]) == 3.0
+    with pytest.raises(ValueError):
+        grouping.stack_group(ts, [0, 1])

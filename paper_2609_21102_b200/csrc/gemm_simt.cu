@@ -88,6 +88,36 @@ __global__ void __launch_bounds__(NT) gemm_simt_kernel(const GemmDesc g) {
   if (g.aux_scale_dev) aux_scale *= g.aux_scale_dev[bz];
   const long long coff = (long long)bz * g.batch_c, xoff = (long long)bz * g.batch_aux;
   double sq = 0.0;
+  // fp32 rows that a thread can take 16 bytes at a time (the rank-k updates of n x n matrices are pure epilogue)
+  const bool vec4 = TN == 4 && !g.symmetric && g.out_dtype == F32 && (g.epilogue == EPI_STORE || g.aux_dtype == F32) &&
+                    g.epilogue != EPI_RESID_NORM && col0 + BN <= g.N && (g.ldc & 3) == 0 && (g.batch_c & 3) == 0 &&
+                    (reinterpret_cast<uintptr_t>(g.C) & 15) == 0 &&
+                    (g.epilogue == EPI_STORE || ((g.ld_aux & 3) == 0 && (g.batch_aux & 3) == 0 &&
+                                                 (reinterpret_cast<uintptr_t>(g.aux) & 15) == 0));
+  if (vec4) {
+#pragma unroll
+    for (int i = 0; i < TM; ++i) {
+      const int gi = row0 + ty * TM + i;
+      if (gi >= g.M) continue;
+      const int gj = col0 + tx * TN;
+      float x[4] = {0.f, 0.f, 0.f, 0.f};
+      if (g.epilogue != EPI_STORE) {
+        const float4 x4 = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.aux) + xoff + (long long)gi * g.ld_aux + gj);
+        x[0] = x4.x; x[1] = x4.y; x[2] = x4.z; x[3] = x4.w;
+      }
+      float v[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float a = acc[i][j];
+        if (g.epilogue == EPI_STORE) v[j] = alpha * a;
+        else if (g.epilogue == EPI_POLY) v[j] = g.pb * x[j] + g.pc * a + ((gi == gj + j) ? g.pa : 0.f);
+        else v[j] = aux_scale * x[j] + alpha * a;
+        if (g.round_tf32) v[j] = round_to_tf32(v[j]);
+      }
+      *reinterpret_cast<float4*>(reinterpret_cast<float*>(g.C) + coff + (long long)gi * g.ldc + gj) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+    return;
+  }
 #pragma unroll
   for (int i = 0; i < TM; ++i) {
     const int gi = row0 + ty * TM + i;

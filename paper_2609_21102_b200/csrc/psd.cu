@@ -31,10 +31,23 @@ __global__ void __launch_bounds__(256) symv_kernel(const float* __restrict__ A, 
     if (vec) {
       const float4* r4 = reinterpret_cast<const float4*>(row);
       const float4* x4 = reinterpret_cast<const float4*>(x);
-      for (int i = lane; i < n / 4; i += 32) {
-        const float4 a = r4[i], b = __ldg(&x4[i]);
-        acc = fmaf(a.x, b.x, acc); acc = fmaf(a.y, b.y, acc); acc = fmaf(a.z, b.z, acc); acc = fmaf(a.w, b.w, acc);
+      // four independent partial sums and loads in flight per lane; combined in a fixed order
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+      const int n4 = n / 4;
+      int i = lane;
+      for (; i + 96 < n4; i += 128) {
+        const float4 p0 = r4[i], p1 = r4[i + 32], p2 = r4[i + 64], p3 = r4[i + 96];
+        const float4 q0 = __ldg(&x4[i]), q1 = __ldg(&x4[i + 32]), q2 = __ldg(&x4[i + 64]), q3 = __ldg(&x4[i + 96]);
+        a0 = fmaf(p0.x, q0.x, a0); a0 = fmaf(p0.y, q0.y, a0); a0 = fmaf(p0.z, q0.z, a0); a0 = fmaf(p0.w, q0.w, a0);
+        a1 = fmaf(p1.x, q1.x, a1); a1 = fmaf(p1.y, q1.y, a1); a1 = fmaf(p1.z, q1.z, a1); a1 = fmaf(p1.w, q1.w, a1);
+        a2 = fmaf(p2.x, q2.x, a2); a2 = fmaf(p2.y, q2.y, a2); a2 = fmaf(p2.z, q2.z, a2); a2 = fmaf(p2.w, q2.w, a2);
+        a3 = fmaf(p3.x, q3.x, a3); a3 = fmaf(p3.y, q3.y, a3); a3 = fmaf(p3.z, q3.z, a3); a3 = fmaf(p3.w, q3.w, a3);
       }
+      for (; i < n4; i += 32) {
+        const float4 a = r4[i], b = __ldg(&x4[i]);
+        a0 = fmaf(a.x, b.x, a0); a0 = fmaf(a.y, b.y, a0); a0 = fmaf(a.z, b.z, a0); a0 = fmaf(a.w, b.w, a0);
+      }
+      acc = (a0 + a1) + (a2 + a3);
     } else {
       for (int i = lane; i < n; i += 32) acc = fmaf(row[i], __ldg(&x[i]), acc);
     }
@@ -42,6 +55,22 @@ __global__ void __launch_bounds__(256) symv_kernel(const float* __restrict__ A, 
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
     if (lane == 0) y[r] = acc;
   }
+}
+
+// out[i] = sum over s of part[s * count + i], s in ascending order (fixed order: reproducible)
+__global__ void __launch_bounds__(256) sum_slices_kernel(const float* __restrict__ part, int slices, long long count,
+                                                         float* __restrict__ out) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  float t = 0.f;
+  for (int s2 = 0; s2 < slices; ++s2) t += part[(long long)s2 * count + i];
+  out[i] = t;
+}
+static cudaError_t sum_slices_launch(const float* part, int slices, long long count, float* out, cudaStream_t st,
+                                     long long* launches) {
+  sum_slices_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(part, slices, count, out);
+  if (launches) ++*launches;
+  return cudaGetLastError();
 }
 
 static cudaError_t symv_launch(const float* A, const float* x, float* y, int n, const int* skip, cudaStream_t st,
@@ -130,6 +159,66 @@ __global__ void __launch_bounds__(1024) lanczos_step_kernel(int j, int n, int st
   if (threadIdx.x == 0) { s.T[j * steps + j + 1] = b; s.T[(j + 1) * steps + j] = b; }
   float* qn = s.Q + (long long)(j + 1) * n;
   for (int i = threadIdx.x; i < n; i += blockDim.x) qn[i] = (float)((double)s.w[i] / b);
+}
+
+// The same step with the work vector in registers (n <= 1024 * EPT): all j + 1 projections of a pass are reduced
+// together (warp shuffles, then one pass over the per-warp partial sums in warp order), two block barriers per pass
+// instead of a dependent chain of loops over global memory. alpha_j is the j-th projection of the first pass.
+template <int EPT>
+__global__ void __launch_bounds__(1024) lanczos_step_reg_kernel(int j, int n, int steps, LanczosState s) {
+  __shared__ double part[32][DEFL_LANCZOS_STEPS];
+  __shared__ double coef[DEFL_LANCZOS_STEPS];
+  __shared__ double red[32];
+  if (*s.done) return;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  double wv[EPT];
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; wv[e] = (i < n) ? (double)s.w[i] : 0.0; }
+  for (int pass = 0; pass < 2; ++pass) {
+    for (int p = 0; p <= j; ++p) {
+      const float* qp = s.Q + (long long)p * n;
+      double d = 0.0;
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; if (i < n) d += (double)qp[i] * wv[e]; }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+      if (lane == 0) part[warp][p] = d;
+    }
+    __syncthreads();
+    if (tid <= j) {
+      double t = 0.0;
+      for (int w2 = 0; w2 < 32; ++w2) t += part[w2][tid];
+      coef[tid] = t;
+      if (pass == 0 && tid == j) s.T[j * steps + j] = t;
+    }
+    __syncthreads();
+    for (int p = 0; p <= j; ++p) {
+      const float* qp = s.Q + (long long)p * n;
+      const double cp = coef[p];
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; if (i < n) wv[e] -= cp * (double)qp[i]; }
+    }
+    // (the work vector goes through fp32 between the passes, as it does when it lives in memory)
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) wv[e] = (double)(float)wv[e];
+  }
+  double b = 0.0;
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) b += wv[e] * wv[e];
+  b = sqrt(block_sum(b, red));
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; if (i < n) s.w[i] = (float)wv[e]; }
+  if (j + 1 == steps) return;
+  const double a0 = s.T[0];
+  if (!(b > 1e-12 * fabs(a0))) {
+    __syncthreads();
+    if (tid == 0) *s.done = 1;
+    return;
+  }
+  if (tid == 0) { s.T[j * steps + j + 1] = b; s.T[(j + 1) * steps + j] = b; }
+  float* qn = s.Q + (long long)(j + 1) * n;
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; if (i < n) qn[i] = (float)(wv[e] / b); }
 }
 
 // v = sum_p E[p][0] q_p (the Ritz vector of the largest Ritz value); E is [steps, steps] row-major fp32
@@ -280,7 +369,9 @@ static int estimate_scale(defl_ctx* c, const float* A, int n, int norm_mode, con
   for (int j = 0; j < steps; ++j) {
     if (ctx_fail(c, symv_launch(A, w.Q + (size_t)j * n, w.lt, n, w.done, c->stream, &c->launches), "symv")) return DEFL_ERR_CUDA;
     if (ctx_fail(c, symv_launch(A, w.lt, w.lw, n, w.done, c->stream, &c->launches), "symv")) return DEFL_ERR_CUDA;
-    lanczos_step_kernel<<<1, 1024, 0, c->stream>>>(j, n, steps, s);
+    if (n <= 4096) lanczos_step_reg_kernel<4><<<1, 1024, 0, c->stream>>>(j, n, steps, s);
+    else if (n <= 8192) lanczos_step_reg_kernel<8><<<1, 1024, 0, c->stream>>>(j, n, steps, s);
+    else lanczos_step_kernel<<<1, 1024, 0, c->stream>>>(j, n, steps, s);
     ++c->launches;
     if (ctx_fail(c, cudaGetLastError(), "lanczos step")) return DEFL_ERR_CUDA;
   }
@@ -375,7 +466,21 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
     g.A[0] = Z; g.sa_i[0] = n; g.sa_k[0] = 1; g.in_dtype = F32;
     g.B[0] = w.Vo; g.sb_k[0] = K; g.sb_j[0] = 1; g.b_dtype = F32;
     g.C = w.Zt; g.ldc = K; g.out_dtype = F32; g.epilogue = EPI_STORE;
+    // a tall product with a narrow output has few tiles (n/64): the inner dimension is cut into `cuts` slices,
+    // taken as a batch into partial products (in the n x n scratch the filter uses later) and summed in slice order
+    int cuts = 1;
+    while (cuts < 16 && n % (2 * cuts * 16) == 0 && (long long)(n / 64 + 1) * cuts < 4LL * c->num_sms && 2LL * cuts * K <= n) cuts *= 2;
+    if (cuts > 1) {
+      const int kc = n / cuts;
+      g.batch = cuts; g.K[0] = kc;
+      g.batch_a[0] = kc;                       // slice s of Z: columns s kc ..
+      g.batch_b[0] = (long long)kc * K;        // slice s of V: rows s kc ..
+      g.C = w.W; g.batch_c = (long long)n * K;
+    }
     if ((rc = run_gemm(c, g, DEFL_ENGINE_SIMT, "Z V"))) return rc;
+    if (cuts > 1 &&
+        ctx_fail(c, sum_slices_launch(w.W, cuts, (long long)n * K, w.Zt, c->stream, &c->launches), "sum slices"))
+      return DEFL_ERR_CUDA;
     // H = V^T Z~ (symmetrised inside the eigensolver), H = E diag(lambda) E^T, sorted by |lambda|
     if (ctx_fail(c, gram_partial_launch(w.Vo, 0, 1, n, K, K, w.gram, c->stream, &c->launches, w.Zt), "V^T Z V")) return DEFL_ERR_CUDA;
     if (ctx_fail(c, jacobi_eig_launch(w.gram, gram_num_chunks(n), 1, K, 1, w.lam, w.E, nullptr, w.status, c->stream, &c->launches), "ritz"))

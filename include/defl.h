@@ -168,6 +168,28 @@ int defl_psd_project(defl_ctx* ctx, const void* X, void* P, int n, int k,
                      const float* coeff_schedule, int T,
                      const defl_opts* opts, const defl_info* info);
 
+/* Three-block ADMM for a standard-form SDP whose constraints are diag(X) = b (max-cut type):
+ *   min <C, X>  s.t.  diag(X) = b, X PSD;   A(X) = diag(X), A*(y) = Diag(y), A A* = I.
+ * One iteration (Appendix C.1, the ADMM iteration; the S-update is Algorithm 2 through defl_psd_project):
+ *   y <- b / sigma - diag(X / sigma + S - C)
+ *   Z  = C - Diag(y) - X / sigma;        S <- projection of Z on the PSD cone (deflated, basis carried along)
+ *   X <- X + sigma (S + Diag(y) - C)
+ * After every iteration the three eigenvalue-free KKT terms of Appendix C.4 are evaluated on the device:
+ *   residuals[3 it + 0] = ||diag(X) - b||_2 / (1 + ||b||_2)
+ *   residuals[3 it + 1] = ||Diag(y) + S - C||_F / (1 + ||C||_F)
+ *   residuals[3 it + 2] = |<C, X> - b^T y| / (1 + |<C, X>| + |b^T y|)
+ *   C  device, [n,n] fp32 symmetric, not modified;  b  device, [n] fp32;  n a multiple of 4
+ *   X, S  device, [n,n] fp32, IN/OUT: the iterates (zeros for a cold start);  y  device, [n] fp32, OUT
+ *   warm_basis, K, k, coeff_schedule, T, opts: as defl_psd_project; the first `warmup_iters` iterations run with
+ *   the gate off (opts->warmup), as the paper does while the basis settles
+ *   residuals  HOST, [iters][3] fp32, written before the call returns (may be NULL); the call synchronises the
+ *   stream twice (norms of b and C at the start, the residual history at the end)
+ * Scratch besides the projection's workspace: two buffers of n*n fp32 the context keeps. Errors as
+ * defl_psd_project; DEFL_ERR_ARG also for n not a multiple of 4 or sigma <= 0. */
+int defl_admm_diag_sdp(defl_ctx* ctx, const void* C, const float* b, int n, float sigma, int iters, int warmup_iters,
+                       void* X, void* S, float* y, int k, float* warm_basis, int K,
+                       const float* coeff_schedule, int T, const defl_opts* opts, float* residuals);
+
 /* Counter-based standard-normal fill (the sketch of Algorithm 3 when none is passed):
  *   h(x): x += 0x9E3779B97F4A7C15; x = (x ^ x>>30) * 0xBF58476D1CE4E5B9; x = (x ^ x>>27) * 0x94D049BB133111EB; x ^ x>>31
  *   j = idx/2; r1 = h(h(seed) ^ 2j); r2 = h(h(seed) ^ (2j+1)); u1 = ((r1>>11)+1) 2^-53; u2 = (r2>>11) 2^-53

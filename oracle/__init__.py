@@ -204,6 +204,28 @@ def psd_project(Z, Vb, k, coeffs, tau=0.0, gamma=1.1, warmup=False, norm_mode=NO
     return P, Vn[:, :K], lam[:K], int(info[0]), float(info[1])
 
 
+def admm_diag_sdp(C, b, sigma, iters, X, S, project, warmup_iters=0):
+    """Three-block ADMM of Appendix C.1 for  min <C,X>  s.t.  diag(X) = b, X PSD  (A = diag, A* = Diag, A A* = I),
+    `iters` iterations from the iterates (X, S). `project(Z, warmup)` returns the S-update, e.g. a closure over
+    psd_project that carries the basis along, or an exact eigenvalue projection. Returns (X, S, y, res[iters,3])
+    with the three eigenvalue-free KKT terms of Appendix C.4 after every iteration."""
+    C, X, S, b = _f64(C), _f64(X).copy(), _f64(S).copy(), _f64(b)
+    n = C.shape[0]
+    y = np.zeros(n)
+    res = np.zeros((iters, 3))
+    nb, nc = np.linalg.norm(b), np.linalg.norm(C)
+    for it in range(iters):
+        y = b / sigma - np.diag(X / sigma + S - C)
+        Z = C - np.diag(y) - X / sigma
+        S = project(Z, it < warmup_iters)
+        X = X + sigma * (S + np.diag(y) - C)
+        obj, dual = float(np.sum(C * X)), float(b @ y)
+        res[it, 0] = np.linalg.norm(np.diag(X) - b) / (1.0 + nb)
+        res[it, 1] = np.linalg.norm(np.diag(y) + S - C) / (1.0 + nc)
+        res[it, 2] = abs(obj - dual) / (1.0 + abs(obj) + abs(dual))
+    return X, S, y, res
+
+
 def fill_gaussian(count, seed):
     out = np.empty(count)
     lib().orc_fill_gaussian(_p(out), _L(count), ctypes.c_uint64(seed))

@@ -25,7 +25,7 @@ CLASSICAL_QUINTIC = (1.875, -1.25, 0.375)
 
 EXPORTS = [
     "defl_create", "defl_destroy", "defl_set_stream", "defl_polar_workspace_bytes", "defl_psd_workspace_bytes",
-    "defl_polar_batched", "defl_polar_batched_host", "defl_muon_step_batched", "defl_brsvd_batched", "defl_psd_project", "defl_fill_gaussian", "defl_debug_gemm",
+    "defl_polar_batched", "defl_polar_batched_host", "defl_muon_step_batched", "defl_brsvd_batched", "defl_psd_project", "defl_admm_diag_sdp", "defl_fill_gaussian", "defl_debug_gemm",
     "defl_frobenius_norms_noalloc", "defl_set_profiling", "defl_get_stage_ms", "defl_launch_count", "defl_status_string", "defl_last_error",
 ]
 
@@ -69,6 +69,10 @@ def lib():
         L.defl_psd_project.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
                                        ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_float), ctypes.c_int,
                                        ctypes.POINTER(DeflOpts), ctypes.POINTER(DeflInfo)]
+        L.defl_admm_diag_sdp.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_float,
+                                         ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                         ctypes.c_int, ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_float),
+                                         ctypes.c_int, ctypes.POINTER(DeflOpts), ctypes.POINTER(ctypes.c_float)]
         L.defl_fill_gaussian.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint64]
         L.defl_debug_gemm.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                       ctypes.c_void_p, ctypes.c_longlong, ctypes.c_longlong, ctypes.c_longlong,
@@ -291,6 +295,33 @@ class Context:
                                     ctypes.byref(opts), ctypes.byref(info))
         self._check(rc)
         return (out, extras) if want_info else out
+
+    def defl_admm_diag_sdp(self, C, b, sigma, iters, X, S, k, warm_basis, coeff_schedule, steps=None, warmup_iters=0,
+                           gamma=0.0, norm_mode=NORM_LANCZOS, lanczos_start=None, seed=0, engine=ENGINE_AUTO,
+                           exploit_symmetry=False, tau=0.0):
+        """`iters` ADMM iterations for min <C,X> s.t. diag(X) = b, X PSD (Appendix C.1), X and S updated in place.
+        Returns (y[n], residuals[iters,3]) with the three eigenvalue-free KKT terms per iteration."""
+        _dev(C, "C"), _dev(b, "b"), _dev(X, "X"), _dev(S, "S")
+        n = C.shape[0]
+        for t, nm in ((C, "C"), (X, "X"), (S, "S")):
+            if t.dtype != torch.float32 or tuple(t.shape) != (n, n):
+                raise ValueError(nm + " must be a float32 [n, n] matrix")
+        if b.dtype != torch.float32 or tuple(b.shape) != (n,):
+            raise ValueError("b must be a float32 [n] vector")
+        K = 0
+        if warm_basis is not None:
+            _dev(warm_basis, "warm_basis")
+            K = warm_basis.shape[1]
+        sched, T = _schedule(coeff_schedule, steps)
+        opts = self._opts(gamma=gamma, norm_mode=norm_mode, lanczos_start=lanczos_start, seed=seed, engine=engine,
+                          exploit_symmetry=exploit_symmetry, tau=tau)
+        y = torch.zeros((n,), dtype=torch.float32, device=C.device)
+        res = (ctypes.c_float * max(3 * iters, 1))()
+        self._sync_stream()
+        rc = lib().defl_admm_diag_sdp(self._h, _ptr(C), _ptr(b), n, sigma, iters, warmup_iters, _ptr(X), _ptr(S), _ptr(y),
+                                      k, _ptr(warm_basis), K, sched, T, ctypes.byref(opts), res)
+        self._check(rc)
+        return y, torch.tensor(list(res)[:3 * iters], dtype=torch.float32).reshape(iters, 3)
 
     def defl_fill_gaussian(self, dst, seed):
         _dev(dst, "dst")

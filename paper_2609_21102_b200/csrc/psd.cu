@@ -408,6 +408,101 @@ static int rank_update(defl_ctx* c, const PsdWs& w, int n, int K, int k, int coe
   return run_gemm(c, g, DEFL_ENGINE_SIMT, "rank-k update");
 }
 
+// ---------------------------------------------------------------------------------------------
+// Three-block ADMM for SDPs with the constraints diag(X) = b (App. C.1): element-wise kernels around
+// the projection. A(X) = diag(X), A*(y) = Diag(y), A A* = I.
+// ---------------------------------------------------------------------------------------------
+// y_i = b_i / sigma - (X_ii / sigma + S_ii - C_ii)
+__global__ void admm_y_kernel(const float* __restrict__ C, const float* __restrict__ X, const float* __restrict__ S,
+                              const float* __restrict__ b, float* __restrict__ y, int n, float inv_sigma) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const long long d = (long long)i * n + i;
+  y[i] = b[i] * inv_sigma - (X[d] * inv_sigma + S[d] - C[d]);
+}
+
+// Z = C - Diag(y) - X / sigma
+__global__ void __launch_bounds__(256) admm_z_kernel(const float* __restrict__ C, const float* __restrict__ X,
+                                                     const float* __restrict__ y, float* __restrict__ Z, int n,
+                                                     float inv_sigma) {
+  const long long total4 = (long long)n * n / 4;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < total4; q += stride) {
+    const float4 c4 = reinterpret_cast<const float4*>(C)[q], x4 = reinterpret_cast<const float4*>(X)[q];
+    const long long e = q * 4;
+    const int i = (int)(e / n), j = (int)(e - (long long)i * n);
+    float z[4] = {c4.x - x4.x * inv_sigma, c4.y - x4.y * inv_sigma, c4.z - x4.z * inv_sigma, c4.w - x4.w * inv_sigma};
+    if (i >= j && i < j + 4) z[i - j] -= y[i];
+    reinterpret_cast<float4*>(Z)[q] = make_float4(z[0], z[1], z[2], z[3]);
+  }
+}
+
+// X <- X + sigma (S + Diag(y) - C), and per-CTA partial sums (fp64, fixed order) of
+//   [0] ||Diag(y) + S - C||_F^2   [1] <C, X_new>   [2] sum_i (X_new_ii - b_i)^2
+__global__ void __launch_bounds__(256) admm_x_kernel(const float* __restrict__ C, const float* __restrict__ S,
+                                                     const float* __restrict__ y, const float* __restrict__ b,
+                                                     float* __restrict__ X, int n, float sigma,
+                                                     double* __restrict__ partial) {
+  __shared__ double red[3][8];
+  const long long total4 = (long long)n * n / 4;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  double dres = 0.0, obj = 0.0, pres = 0.0;
+  for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < total4; q += stride) {
+    const float4 c4 = reinterpret_cast<const float4*>(C)[q], s4 = reinterpret_cast<const float4*>(S)[q];
+    float4 x4 = reinterpret_cast<float4*>(X)[q];
+    const long long e = q * 4;
+    const int i = (int)(e / n), j = (int)(e - (long long)i * n);
+    float r[4] = {s4.x - c4.x, s4.y - c4.y, s4.z - c4.z, s4.w - c4.w};
+    const bool has_diag = (i >= j && i < j + 4);
+    if (has_diag) r[i - j] += y[i];
+    float xn[4] = {x4.x + sigma * r[0], x4.y + sigma * r[1], x4.z + sigma * r[2], x4.w + sigma * r[3]};
+    const float cc[4] = {c4.x, c4.y, c4.z, c4.w};
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      dres += (double)r[t] * (double)r[t];
+      obj += (double)cc[t] * (double)xn[t];
+    }
+    if (has_diag) { const double d = (double)xn[i - j] - (double)b[i]; pres += d * d; }
+    reinterpret_cast<float4*>(X)[q] = make_float4(xn[0], xn[1], xn[2], xn[3]);
+  }
+  double v[3] = {dres, obj, pres};
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int t = 0; t < 3; ++t) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v[t] += __shfl_down_sync(0xffffffffu, v[t], o);
+    if (lane == 0) red[t][warp] = v[t];
+  }
+  __syncthreads();
+  if (threadIdx.x < 3) {
+    double t = 0.0;
+    for (int w2 = 0; w2 < 8; ++w2) t += red[threadIdx.x][w2];
+    partial[(long long)blockIdx.x * 3 + threadIdx.x] = t;
+  }
+}
+
+// the three eigenvalue-free KKT terms of the iteration (App. C.4), from the partial sums and b^T y, ||b||, ||C||_F
+__global__ void admm_residual_kernel(const double* __restrict__ partial, int nblk, const float* __restrict__ b,
+                                     const float* __restrict__ y, int n, double norm_b, double norm_c,
+                                     float* __restrict__ out3) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  double dres = 0.0, obj = 0.0, pres = 0.0, by = 0.0;
+  for (int i = 0; i < nblk; ++i) { dres += partial[3 * i]; obj += partial[3 * i + 1]; pres += partial[3 * i + 2]; }
+  for (int i = 0; i < n; ++i) by += (double)b[i] * (double)y[i];
+  out3[0] = (float)(sqrt(pres) / (1.0 + norm_b));
+  out3[1] = (float)(sqrt(dres) / (1.0 + norm_c));
+  out3[2] = (float)(fabs(obj - by) / (1.0 + fabs(obj) + fabs(by)));
+}
+
+// sum of squares of a float array in one CTA (norms of b and C, once per call)
+__global__ void __launch_bounds__(1024) sumsq_kernel(const float* __restrict__ x, long long count, double* out) {
+  __shared__ double red[32];
+  double a = 0.0;
+  for (long long i = threadIdx.x; i < count; i += blockDim.x) a += (double)x[i] * (double)x[i];
+  a = block_sum(a, red);
+  if (threadIdx.x == 0) *out = a;
+}
+
 }  // namespace defl
 
 extern "C" {
@@ -536,7 +631,12 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
     g.epilogue = EPI_POLY; g.pa = ca; g.pb = cb; g.pc = cc;
     if ((rc = run_gemm(c, g, gemm_tc_supported(g) ? engine : DEFL_ENGINE_SIMT, "polynomial"))) return rc;
     g.A[0] = X; g.B[0] = w.Tt; g.C = Xn; g.aux = nullptr;
-    g.epilogue = EPI_STORE; g.symmetric = 0;            // X Tt is symmetric only up to rounding: compute all of it
+    // X Tt is symmetric only up to rounding, and the iterate must be EXACTLY symmetric: the products above take
+    // X^T for X (rows as columns), which is the Gram X X^T, and an antisymmetric error N that anticommutes with
+    // sign(X) then comes back as 2N after every step (X' = S + 3N/2 - S N S / 2). So the upper tiles are computed
+    // and mirrored, whatever exploit_symmetry says; the skew part of the rounding turns into a symmetric error of
+    // the same size, which the iteration does not amplify.
+    g.epilogue = EPI_STORE; g.symmetric = 1;
     if ((rc = run_gemm(c, g, gemm_tc_supported(g) ? engine : DEFL_ENGINE_SIMT, "apply"))) return rc;
     cur ^= 1;
   }
@@ -597,6 +697,72 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
       if (ctx_fail(c, cudaMemcpyAsync(info->status, w.status, sizeof(int), cudaMemcpyDeviceToDevice, c->stream), "copy status"))
         return DEFL_ERR_CUDA;
     }
+  }
+  return DEFL_OK;
+}
+
+
+int defl_admm_diag_sdp(defl_ctx* c, const void* Cv, const float* b, int n, float sigma, int iters, int warmup_iters,
+                       void* Xv, void* Sv, float* y, int k, float* warm_basis, int K, const float* coeff_schedule,
+                       int T, const defl_opts* opts, float* residuals) {
+  if (!c || !Cv || !b || !Xv || !Sv || !y || n <= 0 || (n & 3) || iters < 0 || !(sigma > 0.f)) return DEFL_ERR_ARG;
+  cudaSetDevice(c->device);
+  const float* C = reinterpret_cast<const float*>(Cv);
+  float* X = reinterpret_cast<float*>(Xv);
+  float* S = reinterpret_cast<float*>(Sv);
+  // scratch of this loop: Z [n,n], partial sums, residual history on the device; the context keeps it with the
+  // staging buffers of the host-buffer entry point (the projection uses the workspace proper)
+  const int nblk = c->num_sms * 4;
+  const size_t zbytes = (size_t)n * n * sizeof(float);
+  const size_t extra = align_up((size_t)nblk * 3 * sizeof(double), 256) + align_up((size_t)(iters > 0 ? iters : 1) * 3 * sizeof(float), 256) + 256;
+  const size_t need = zbytes > extra ? zbytes : extra;
+  {
+    const size_t bytes = need;
+    if (bytes > c->stage_bytes) {
+      cudaDeviceSynchronize();
+      if (c->stage_in) cudaFree(c->stage_in);
+      if (c->stage_out) cudaFree(c->stage_out);
+      c->stage_in = c->stage_out = nullptr;
+      c->stage_bytes = 0;
+      if (ctx_fail(c, cudaMalloc(&c->stage_in, bytes), "cudaMalloc(ADMM scratch)")) return DEFL_ERR_CUDA;
+      if (ctx_fail(c, cudaMalloc(&c->stage_out, bytes), "cudaMalloc(ADMM scratch)")) return DEFL_ERR_CUDA;
+      c->stage_bytes = bytes;
+    }
+  }
+  float* Z = reinterpret_cast<float*>(c->stage_in);
+  char* aux = reinterpret_cast<char*>(c->stage_out);
+  double* partial = reinterpret_cast<double*>(aux);
+  float* hist = reinterpret_cast<float*>(aux + align_up((size_t)nblk * 3 * sizeof(double), 256));
+  double* norms = reinterpret_cast<double*>(aux + align_up((size_t)nblk * 3 * sizeof(double), 256) +
+                                            align_up((size_t)(iters > 0 ? iters : 1) * 3 * sizeof(float), 256));
+  sumsq_kernel<<<1, 1024, 0, c->stream>>>(b, n, norms);
+  sumsq_kernel<<<1, 1024, 0, c->stream>>>(C, (long long)n * n, norms + 1);
+  c->launches += 2;
+  double hn[2] = {0.0, 0.0};
+  if (ctx_fail(c, cudaMemcpyAsync(hn, norms, sizeof(hn), cudaMemcpyDeviceToHost, c->stream), "norms") ||
+      ctx_fail(c, cudaStreamSynchronize(c->stream), "synchronize"))
+    return DEFL_ERR_CUDA;
+  const double norm_b = sqrt(hn[0]), norm_c = sqrt(hn[1]);
+  const float inv_sigma = 1.f / sigma;
+  defl_opts o;
+  if (opts) o = *opts; else memset(&o, 0, sizeof(o));
+  for (int it = 0; it < iters; ++it) {
+    admm_y_kernel<<<(n + 255) / 256, 256, 0, c->stream>>>(C, X, S, b, y, n, inv_sigma);
+    admm_z_kernel<<<nblk, 256, 0, c->stream>>>(C, X, y, Z, n, inv_sigma);
+    c->launches += 2;
+    if (ctx_fail(c, cudaGetLastError(), "ADMM y, Z")) return DEFL_ERR_CUDA;
+    o.warmup = (it < warmup_iters) ? 1 : (opts ? opts->warmup : 0);
+    const int rc = defl_psd_project(c, Z, S, n, k, warm_basis, K, coeff_schedule, T, &o, nullptr);
+    if (rc) return rc;
+    admm_x_kernel<<<nblk, 256, 0, c->stream>>>(C, S, y, b, X, n, sigma, partial);
+    admm_residual_kernel<<<1, 32, 0, c->stream>>>(partial, nblk, b, y, n, norm_b, norm_c, hist + 3 * it);
+    c->launches += 2;
+    if (ctx_fail(c, cudaGetLastError(), "ADMM X")) return DEFL_ERR_CUDA;
+  }
+  if (residuals && iters > 0) {
+    if (ctx_fail(c, cudaMemcpyAsync(residuals, hist, (size_t)iters * 3 * sizeof(float), cudaMemcpyDeviceToHost, c->stream), "residuals") ||
+        ctx_fail(c, cudaStreamSynchronize(c->stream), "synchronize"))
+      return DEFL_ERR_CUDA;
   }
   return DEFL_OK;
 }

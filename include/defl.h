@@ -34,6 +34,7 @@ extern "C" {
 /* storage types of G / out */
 #define DEFL_BF16 0 /* bf16 storage, bf16 tensor-core products, fp32 accumulation */
 #define DEFL_F32 1  /* fp32 storage; polar path: fp32 FMA products; PSD filter: tf32 tensor-core products */
+#define DEFL_F16 2  /* IEEE half: the FP16 filter of the PSD projection (opts->half_filter) and defl_debug_gemm only */
 
 /* where the head is restored (polar) */
 #define DEFL_RESTORE_PADDED 0 /* Algorithm 1: X0 = R/||R||_F + U_k V_k^T / gamma, out = N^L(X0) */
@@ -83,6 +84,10 @@ typedef struct defl_opts {
                             > 0: with s the k estimated magnitudes, deflate only if s_k < tau * s_1, and then the
                             components with s_i > tau * s_1 (PSD: among all K Ritz values); otherwise the call
                             reduces to the undeflated filter for that matrix. Decided per matrix on the device. */
+  int half_filter;       /* PSD only, non-zero: the T filter steps run in IEEE half precision (iterates stored in
+                            half, tensor-core products with fp32 accumulation), the precision the paper's SDP runs
+                            use for the filter (Appendix C.2). Everything around the filter stays fp32/tf32.
+                            Needs n a multiple of 8 and the tensor engine. */
 } defl_opts;
 
 typedef struct defl_info {

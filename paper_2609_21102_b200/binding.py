@@ -13,7 +13,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libdeflpolar.so")
 
-BF16, F32 = 0, 1
+BF16, F32, F16 = 0, 1, 2
 RESTORE_PADDED, RESTORE_ADD = 0, 1
 NORM_LANCZOS, NORM_FROBENIUS = 0, 1
 ENGINE_AUTO, ENGINE_SIMT, ENGINE_TENSOR = 0, 1, 2
@@ -34,7 +34,7 @@ class DeflOpts(ctypes.Structure):
     _fields_ = [("sketch", ctypes.c_void_p), ("seed", ctypes.c_uint64), ("restore_mode", ctypes.c_int),
                 ("gamma", ctypes.c_float), ("norm_mode", ctypes.c_int), ("lanczos_start", ctypes.c_void_p),
                 ("warmup", ctypes.c_int), ("engine", ctypes.c_int), ("exploit_symmetry", ctypes.c_int),
-                ("tau", ctypes.c_float)]
+                ("tau", ctypes.c_float), ("half_filter", ctypes.c_int)]
 
 
 class DeflInfo(ctypes.Structure):
@@ -102,7 +102,9 @@ def _dtype_code(t):
         return BF16
     if t.dtype == torch.float32:
         return F32
-    raise TypeError("only bfloat16 and float32 tensors are supported")
+    if t.dtype == torch.float16:
+        return F16
+    raise TypeError("only bfloat16, float16 and float32 tensors are supported")
 
 
 def _ptr(t):
@@ -155,7 +157,7 @@ class Context:
             raise DeflError(rc, lib().defl_last_error(self._h).decode())
 
     def _opts(self, sketch=None, seed=0, restore_mode=RESTORE_PADDED, gamma=0.0, norm_mode=NORM_LANCZOS,
-              lanczos_start=None, warmup=False, engine=ENGINE_AUTO, exploit_symmetry=False, tau=0.0):
+              lanczos_start=None, warmup=False, engine=ENGINE_AUTO, exploit_symmetry=False, tau=0.0, half_filter=False):
         o = DeflOpts()
         o.sketch = sketch.data_ptr() if sketch is not None else None
         o.seed = seed
@@ -167,6 +169,7 @@ class Context:
         o.engine = engine
         o.exploit_symmetry = int(bool(exploit_symmetry))
         o.tau = tau
+        o.half_filter = int(bool(half_filter))
         return o
 
     # ------------------------------------------------------------------------------------------
@@ -266,7 +269,7 @@ class Context:
 
     def defl_psd_project(self, X, k, warm_basis, coeff_schedule, steps=None, out=None, gamma=0.0,
                          norm_mode=NORM_LANCZOS, lanczos_start=None, seed=0, warmup=False, engine=ENGINE_AUTO,
-                         exploit_symmetry=False, want_info=False, tau=0.0):
+                         exploit_symmetry=False, want_info=False, tau=0.0, half_filter=False):
         """P = deflated PSD projection of the symmetric X[n,n] (Algorithm 2); warm_basis[n,K] is updated in place."""
         _dev(X, "X")
         n = X.shape[0]
@@ -279,7 +282,7 @@ class Context:
         out = torch.empty_like(X) if out is None else _dev(out, "out")
         sched, T = _schedule(coeff_schedule, steps)
         opts = self._opts(gamma=gamma, norm_mode=norm_mode, lanczos_start=lanczos_start, seed=seed, warmup=warmup,
-                          engine=engine, exploit_symmetry=exploit_symmetry, tau=tau)
+                          engine=engine, exploit_symmetry=exploit_symmetry, tau=tau, half_filter=half_filter)
         info = DeflInfo()
         extras = None
         if want_info:
@@ -298,7 +301,7 @@ class Context:
 
     def defl_admm_diag_sdp(self, C, b, sigma, iters, X, S, k, warm_basis, coeff_schedule, steps=None, warmup_iters=0,
                            gamma=0.0, norm_mode=NORM_LANCZOS, lanczos_start=None, seed=0, engine=ENGINE_AUTO,
-                           exploit_symmetry=False, tau=0.0):
+                           exploit_symmetry=False, tau=0.0, half_filter=False):
         """`iters` ADMM iterations for min <C,X> s.t. diag(X) = b, X PSD (Appendix C.1), X and S updated in place.
         Returns (y[n], residuals[iters,3]) with the three eigenvalue-free KKT terms per iteration."""
         _dev(C, "C"), _dev(b, "b"), _dev(X, "X"), _dev(S, "S")
@@ -314,7 +317,7 @@ class Context:
             K = warm_basis.shape[1]
         sched, T = _schedule(coeff_schedule, steps)
         opts = self._opts(gamma=gamma, norm_mode=norm_mode, lanczos_start=lanczos_start, seed=seed, engine=engine,
-                          exploit_symmetry=exploit_symmetry, tau=tau)
+                          exploit_symmetry=exploit_symmetry, tau=tau, half_filter=half_filter)
         y = torch.zeros((n,), dtype=torch.float32, device=C.device)
         res = (ctypes.c_float * max(3 * iters, 1))()
         self._sync_stream()
@@ -351,7 +354,7 @@ class Context:
         self._sync_stream()
         rc = lib().defl_debug_gemm(self._h, engine, b, M, N, K, _ptr(A), sa_i, sa_k, A.shape[1] * A.shape[2],
                                    _ptr(B), sb_k, sb_j, B.shape[1] * B.shape[2], _ptr(C), _dtype_code(A),
-                                   BF16 if out_dtype == torch.bfloat16 else F32, alpha, int(exploit_symmetry))
+                                   {torch.bfloat16: BF16, torch.float16: F16}.get(out_dtype, F32), alpha, int(exploit_symmetry))
         self._check(rc)
         return C
 

@@ -47,7 +47,7 @@ void ctx_stage_mark(defl_ctx* c) {
 // products on exact fp32 FMA; ENGINE_TENSOR also sends fp32 products there (as tf32).
 bool use_tensor_engine(const GemmDesc& g, int engine) {
   if (engine == DEFL_ENGINE_SIMT) return false;
-  if (engine == DEFL_ENGINE_AUTO && g.in_dtype != BF16) return false;
+  if (engine == DEFL_ENGINE_AUTO && g.in_dtype == F32) return false;
   return gemm_tc_supported(g);
 }
 
@@ -60,7 +60,11 @@ int run_gemm(defl_ctx* c, const GemmDesc& g, int engine, const char* what) {
   }
   cudaError_t e;
   if (tc) e = gemm_tc_launch(g, c->stream, c->wait_status, c->num_sms, &c->launches);
-  else e = gemm_simt_launch(g, c->stream, &c->launches);
+  else if (g.in_dtype == F16 || g.b_dtype == F16) {
+    // IEEE half operands exist for the tensor cores only (the FP16 projection filter)
+    snprintf(c->err, sizeof(c->err), "%s: half-precision operands need the tensor engine", what);
+    return DEFL_ERR_UNSUPPORTED;
+  } else e = gemm_simt_launch(g, c->stream, &c->launches);
   if (ctx_fail(c, e, what)) return DEFL_ERR_CUDA;
   return DEFL_OK;
 }

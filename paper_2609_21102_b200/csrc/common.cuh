@@ -3,13 +3,14 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 
 namespace defl {
 
-enum DType { BF16 = 0, F32 = 1 };
+enum DType { BF16 = 0, F32 = 1, F16 = 2 };      // F16: IEEE half (operands and iterates of the FP16 projection filter)
 
-__host__ __device__ inline size_t dtype_size(int dt) { return dt == BF16 ? 2 : 4; }
+__host__ __device__ inline size_t dtype_size(int dt) { return dt == F32 ? 4 : 2; }
 
 // What happens to the fp32 accumulator tile acc[i,j] of C = opA(A) opB(B).
 enum Epilogue {
@@ -64,7 +65,8 @@ int gemm_tc_partials_per_batch(const GemmDesc& g);
 
 __device__ __forceinline__ float ld_as_float(const void* p, long long idx, int dt) {
   return dt == BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[idx])
-                    : reinterpret_cast<const float*>(p)[idx];
+         : dt == F16 ? __half2float(reinterpret_cast<const __half*>(p)[idx])
+                     : reinterpret_cast<const float*>(p)[idx];
 }
 __device__ __forceinline__ float round_to_tf32(float x) {
   uint32_t r;
@@ -73,7 +75,20 @@ __device__ __forceinline__ float round_to_tf32(float x) {
 }
 __device__ __forceinline__ void st_from_float(void* p, long long idx, int dt, float v) {
   if (dt == BF16) reinterpret_cast<__nv_bfloat16*>(p)[idx] = __float2bfloat16_rn(v);
+  else if (dt == F16) reinterpret_cast<__half*>(p)[idx] = __float2half_rn(v);
   else reinterpret_cast<float*>(p)[idx] = v;
+}
+
+// two packed 16-bit values (bf16 or, with `f16`, IEEE half) <-> two floats
+__device__ __forceinline__ float2 unpack16x2(uint32_t w, bool f16) {
+  if (f16) return __half22float2(*reinterpret_cast<const __half2*>(&w));
+  return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w));
+}
+__device__ __forceinline__ uint32_t pack16x2(float a, float b, bool f16) {
+  uint32_t w;
+  if (f16) { const __half2 h = __floats2half2_rn(a, b); w = *reinterpret_cast<const uint32_t*>(&h); }
+  else { const __nv_bfloat162 h = __floats2bfloat162_rn(a, b); w = *reinterpret_cast<const uint32_t*>(&h); }
+  return w;
 }
 
 }  // namespace defl

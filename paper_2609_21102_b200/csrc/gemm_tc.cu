@@ -70,6 +70,7 @@ struct TcParams {
   uint32_t idesc;
   // epilogue
   int epilogue, out_dtype, aux_dtype, symmetric, round_tf32;
+  int half_f16;                // 16-bit operands, aux and output are IEEE half (else bf16)
   void* C; long long ldc, batch_c;
   const void* aux; long long ld_aux, batch_aux;
   float alpha, aux_scale, pa, pb, pc;
@@ -340,17 +341,18 @@ template <int EPI>
 __device__ __forceinline__ void load_aux16(const TcParams& p, bool take, bool vec, bool aux_bf16, size_t xoff, int gj0,
                                            float* x) {
   if (EPI == EPI_STORE) return;
-  const __nv_bfloat16* auxh = reinterpret_cast<const __nv_bfloat16*>(p.aux);
+  const uint16_t* auxh = reinterpret_cast<const uint16_t*>(p.aux);
   const float* auxf = reinterpret_cast<const float*>(p.aux);
+  const bool f16 = p.half_f16 != 0;
   if (!take) {
 #pragma unroll
     for (int j = 0; j < 16; ++j) x[j] = 0.f;
   } else if (vec && aux_bf16) {
     const uint4* src = reinterpret_cast<const uint4*>(auxh + xoff);
     uint4 pk[2] = {src[0], src[1]};
-    const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(pk);
+    const uint32_t* hh = reinterpret_cast<const uint32_t*>(pk);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) { const float2 f = __bfloat1622float2(hh[j]); x[2 * j] = f.x; x[2 * j + 1] = f.y; }
+    for (int j = 0; j < 8; ++j) { const float2 f = unpack16x2(hh[j], f16); x[2 * j] = f.x; x[2 * j + 1] = f.y; }
   } else if (vec) {
     const float4* src = reinterpret_cast<const float4*>(auxf + xoff);
 #pragma unroll
@@ -358,7 +360,7 @@ __device__ __forceinline__ void load_aux16(const TcParams& p, bool take, bool ve
   } else {
 #pragma unroll
     for (int j = 0; j < 16; ++j)
-      x[j] = (gj0 + j < p.N) ? (aux_bf16 ? __bfloat162float(auxh[xoff + j]) : auxf[xoff + j]) : 0.f;
+      x[j] = (gj0 + j < p.N) ? (aux_bf16 ? unpack16x2((uint32_t)auxh[xoff + j], f16).x : auxf[xoff + j]) : 0.f;
   }
 }
 
@@ -367,8 +369,9 @@ __device__ __forceinline__ void finish16(const TcParams& p, const uint32_t* r, c
                                          int gj0, bool row_ok, bool vec, size_t crow, size_t cbatch, float alpha,
                                          float aux_scale, double& sq) {
   if (gj0 >= p.N) return;
-  const bool out_bf16 = (p.out_dtype == BF16);
-  __nv_bfloat16* outh = reinterpret_cast<__nv_bfloat16*>(p.C);
+  const bool out_bf16 = (p.out_dtype != F32);       // a 16-bit output type
+  const bool f16 = p.half_f16 != 0;
+  uint16_t* outh = reinterpret_cast<uint16_t*>(p.C);
   float* outf = reinterpret_cast<float*>(p.C);
   float v[16];
 #pragma unroll
@@ -397,9 +400,9 @@ __device__ __forceinline__ void finish16(const TcParams& p, const uint32_t* r, c
   if (vec && (!p.symmetric || mirror_all)) {
     if (out_bf16) {
       uint4 pk[2];
-      __nv_bfloat162* hh = reinterpret_cast<__nv_bfloat162*>(pk);
+      uint32_t* hh = reinterpret_cast<uint32_t*>(pk);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) hh[j] = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+      for (int j = 0; j < 8; ++j) hh[j] = pack16x2(v[2 * j], v[2 * j + 1], f16);
       uint4* dst = reinterpret_cast<uint4*>(outh + crow + gj0);
       dst[0] = pk[0]; dst[1] = pk[1];
     } else {
@@ -412,7 +415,7 @@ __device__ __forceinline__ void finish16(const TcParams& p, const uint32_t* r, c
     for (int j = 0; j < 16; ++j) {
       const int gj = gj0 + j;
       if (gj < p.N && (!p.symmetric || gj >= gi)) {
-        if (out_bf16) outh[crow + gj] = __float2bfloat16_rn(v[j]); else outf[crow + gj] = v[j];
+        if (out_bf16) outh[crow + gj] = (uint16_t)pack16x2(v[j], 0.f, f16); else outf[crow + gj] = v[j];
       }
     }
   }
@@ -423,7 +426,7 @@ __device__ __forceinline__ void finish16(const TcParams& p, const uint32_t* r, c
       const int gj = gj0 + j;
       if (gj < p.N && gj > gi) {
         const size_t m = cbatch + (size_t)gj * p.ldc + gi;
-        if (out_bf16) outh[m] = __float2bfloat16_rn(v[j]); else outf[m] = v[j];
+        if (out_bf16) outh[m] = (uint16_t)pack16x2(v[j], 0.f, f16); else outf[m] = v[j];
       }
     }
   }
@@ -487,6 +490,7 @@ __device__ __forceinline__ void epilogue_block_fast(const TcParams& p, uint32_t 
   tmem_ld_wait();
   const int gi = gi_warp0 + lane;
   const bool row_ok = gi < p.M;
+  const bool f16 = p.half_f16 != 0;
   float sqf = 0.f;
 #pragma unroll
   for (int pc = 0; pc < pp; ++pc) {
@@ -495,9 +499,9 @@ __device__ __forceinline__ void epilogue_block_fast(const TcParams& p, uint32_t 
     if (EPI != EPI_STORE) {
       const uint4 q = *slot;
       if (ES == 2) {
-        const __nv_bfloat162* hh = reinterpret_cast<const __nv_bfloat162*>(&q);
+        const uint32_t* hh = reinterpret_cast<const uint32_t*>(&q);
 #pragma unroll
-        for (int j = 0; j < epp / 2; ++j) { const float2 f = __bfloat1622float2(hh[j]); x[2 * j] = f.x; x[2 * j + 1] = f.y; }
+        for (int j = 0; j < epp / 2; ++j) { const float2 f = unpack16x2(hh[j], f16); x[2 * j] = f.x; x[2 * j + 1] = f.y; }
       } else {
         x[0] = __uint_as_float(q.x); x[1] = __uint_as_float(q.y); x[2 % epp] = __uint_as_float(q.z); x[3 % epp] = __uint_as_float(q.w);
       }
@@ -516,9 +520,9 @@ __device__ __forceinline__ void epilogue_block_fast(const TcParams& p, uint32_t 
     if (EPI != EPI_RESID_NORM) {
       uint4 q;
       if (ES == 2) {
-        __nv_bfloat162* hh = reinterpret_cast<__nv_bfloat162*>(&q);
+        uint32_t* hh = reinterpret_cast<uint32_t*>(&q);
 #pragma unroll
-        for (int j = 0; j < epp / 2; ++j) hh[j] = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+        for (int j = 0; j < epp / 2; ++j) hh[j] = pack16x2(v[2 * j], v[2 * j + 1], f16);
       } else {
         q = make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2 % epp]), __float_as_uint(v[3 % epp]));
       }
@@ -605,13 +609,13 @@ __device__ __forceinline__ void epilogue_half(const TcParams& p, uint32_t taddr,
                                               int bz, int wsel, float alpha, float aux_scale, double& sq, uint8_t* stg,
                                               int lane) {
   const bool row_ok = gi < p.M;
-  const bool aux_bf16 = (p.aux_dtype == BF16);
+  const bool aux_bf16 = (p.aux_dtype != F32);       // a 16-bit aux type
   const size_t cbatch = (size_t)bz * p.batch_c;
   const size_t crow = cbatch + (size_t)gi * p.ldc;
   const size_t xrow = (size_t)bz * p.batch_aux + (size_t)gi * p.ld_aux;
   const bool vec_ok = ((p.ldc & 7) == 0) && ((p.batch_c & 7) == 0) && ((p.ld_aux & 7) == 0 || EPI == EPI_STORE) &&
                       ((p.batch_aux & 7) == 0 || EPI == EPI_STORE);
-  const bool a2 = (p.aux_dtype == BF16), o2 = (p.out_dtype == BF16);
+  const bool a2 = (p.aux_dtype != F32), o2 = (p.out_dtype != F32);
   // the coalesced path wants `aux` and the output in the same type (true of every product the library makes)
   // (symmetric output: the mirror stores of the coalesced path assume 32 complete rows)
   const bool fast_ok = vec_ok && (EPI == EPI_STORE || EPI == EPI_RESID_NORM || a2 == o2) &&
@@ -979,6 +983,7 @@ bool encode_map(CUtensorMap* tm, const void* base, int esize, bool tf32, bool mn
     box[0] = span; box[1] = span; box[2] = 1;
   }
   if (batch == 1) strides[1] = strides[0] * dims[1];
+  // (16-bit operands: the copy engine only needs the element size; bf16 and IEEE half tiles move alike)
   const CUtensorMapDataType dt = (esize == 2) ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
                                               : (tf32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32);
   const CUresult r = enc(tm, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -1025,6 +1030,13 @@ bool gemm_tc_supported(const GemmDesc& g) {
   if (g.nseg < 1 || g.nseg > 2) return false;
   if (g.b_split == 2 && (g.nseg != 1 || !aligned16(g.B[1]))) return false;
   if (g.b_dtype != g.in_dtype) return false;
+  // one 16-bit kind per launch: the epilogue converts aux and output with the operands' kind
+  {
+    const int kinds[3] = {g.in_dtype, g.epilogue == EPI_STORE ? F32 : g.aux_dtype, g.epilogue == EPI_RESID_NORM ? F32 : g.out_dtype};
+    bool bf = false, hf = false;
+    for (int i = 0; i < 3; ++i) { bf |= kinds[i] == BF16; hf |= kinds[i] == F16; }
+    if (bf && hf) return false;
+  }
   const int esize = (int)dtype_size(g.in_dtype);
   if (g.symmetric && g.M != g.N) return false;
   for (int s = 0; s < g.nseg; ++s) {
@@ -1117,11 +1129,12 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   if (stages < 2) return cudaErrorNotSupported;
   p.stages = stages;
   // instruction descriptor: fp32 accumulate, operand format, majors, N >> 3 at bit 17, M >> 4 at bit 24
-  const uint32_t fmt = tf32 ? 2u : 1u;
+  const uint32_t fmt = tf32 ? 2u : (g.in_dtype == F16 ? 0u : 1u);      // kind::tf32: TF32 = 2; kind::f16: F16 = 0, BF16 = 1
   // (N is filled in per tile by the kernel: edge tiles compute fewer columns)
   p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)p.a_mn_major << 15) | ((uint32_t)p.b_mn_major << 16) |
             ((uint32_t)((p.pair ? 256 : 128) >> 4) << 24);
   p.epilogue = g.epilogue; p.out_dtype = g.out_dtype; p.aux_dtype = g.aux_dtype; p.symmetric = g.symmetric; p.round_tf32 = g.round_tf32;
+  p.half_f16 = (g.in_dtype == F16 || (g.epilogue != EPI_STORE && g.aux_dtype == F16) || g.out_dtype == F16) ? 1 : 0;
   p.C = g.C; p.ldc = g.ldc; p.batch_c = g.batch_c;
   p.aux = g.aux; p.ld_aux = g.ld_aux; p.batch_aux = g.batch_aux;
   p.alpha = g.alpha; p.aux_scale = g.aux_scale; p.pa = g.pa; p.pb = g.pb; p.pc = g.pc;

@@ -7,6 +7,7 @@
 // The basis V is orthonormalised on entry, so a Gaussian start block is accepted.
 #include "../../include/defl.h"
 #include "common.cuh"
+#include <cuda_fp16.h>
 #include "panel.cuh"
 #include "ctx.cuh"
 
@@ -541,6 +542,9 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
   // iterates that feed tf32 products are stored already rounded to nearest tf32: the tensor core would
   // otherwise truncate them, which biases every product towards zero
   const int tf32_round = (engine == DEFL_ENGINE_TENSOR) ? 1 : 0;
+  // FP16 filter (Appendix C.2: the filter is used in half precision): iterates in IEEE half, kind::f16 products
+  const bool half = opts && opts->half_filter;
+  if (half && (engine != DEFL_ENGINE_TENSOR || (n & 7))) return DEFL_ERR_UNSUPPORTED;
 
   cudaSetDevice(c->device);
   int rc = ctx_reserve(c, carve_psd(nullptr, n, K).bytes);
@@ -615,7 +619,38 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
   ctx_stage_mark(c);
 
   // ---- stage 4: g = p_T o ... o p_1 on the symmetric X0: W = X^2, Tt = a I + b W + c W^2, X <- X Tt ------
-  for (int t = 0; t < T; ++t) {
+  if (half && T > 0) {
+    // half-precision buffers inside the fp32 scratch that is free here: the two iterates share the other iterate
+    // buffer, W and Tt share the fp32 W; the result returns to fp32 (rounded to tf32) for the reconstruction
+    const size_t nn = (size_t)n * n;
+    __half* H[2] = {reinterpret_cast<__half*>(bufs[cur ^ 1]), reinterpret_cast<__half*>(bufs[cur ^ 1]) + nn};
+    __half* HW = reinterpret_cast<__half*>(w.W);
+    __half* HT = HW + nn;
+    if (ctx_fail(c, scale_launch(bufs[cur], F32, H[0], F16, 1, (long long)nn, nullptr, c->stream, &c->launches, 0), "to half"))
+      return DEFL_ERR_CUDA;
+    int hc = 0;
+    for (int t = 0; t < T; ++t) {
+      const float ca = coeff_schedule[3 * t], cb = coeff_schedule[3 * t + 1], cc = coeff_schedule[3 * t + 2];
+      GemmDesc g = gemm_desc_zero();
+      g.batch = 1; g.in_dtype = F16; g.b_dtype = F16; g.out_dtype = F16;
+      g.M = n; g.N = n; g.K[0] = n;
+      g.A[0] = H[hc]; g.sa_i[0] = n; g.sa_k[0] = 1;
+      g.B[0] = H[hc]; g.sb_k[0] = 1; g.sb_j[0] = n;          // X symmetric: rows as columns
+      g.C = HW; g.ldc = n; g.epilogue = EPI_STORE; g.symmetric = 1;
+      if ((rc = run_gemm(c, g, DEFL_ENGINE_TENSOR, "X^2 (half)"))) return rc;
+      g.A[0] = HW; g.B[0] = HW; g.C = HT;
+      g.aux = HW; g.ld_aux = n; g.aux_dtype = F16;
+      g.epilogue = EPI_POLY; g.pa = ca; g.pb = cb; g.pc = cc;
+      if ((rc = run_gemm(c, g, DEFL_ENGINE_TENSOR, "polynomial (half)"))) return rc;
+      g.A[0] = H[hc]; g.B[0] = HT; g.C = H[hc ^ 1]; g.aux = nullptr;
+      g.epilogue = EPI_STORE; g.symmetric = 1;              // the iterate stays exactly symmetric (see below)
+      if ((rc = run_gemm(c, g, DEFL_ENGINE_TENSOR, "apply (half)"))) return rc;
+      hc ^= 1;
+    }
+    if (ctx_fail(c, scale_launch(H[hc], F16, bufs[cur], F32, 1, (long long)nn, nullptr, c->stream, &c->launches, tf32_round), "from half"))
+      return DEFL_ERR_CUDA;
+  }
+  for (int t = 0; t < (half ? 0 : T); ++t) {
     const float ca = coeff_schedule[3 * t], cb = coeff_schedule[3 * t + 1], cc = coeff_schedule[3 * t + 2];
     const float* X = bufs[cur];
     float* Xn = bufs[cur ^ 1];

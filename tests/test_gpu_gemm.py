@@ -108,3 +108,26 @@ def test_tensor_engine_other_tile_forms(ctx, monkeypatch, knobs, sym):
         C = ctx.defl_debug_gemm(A, B, False, False, engine=binding.ENGINE_TENSOR, out_dtype=torch.float32)
         ref = _ref(A, B, False, False)
     assert torch.allclose(C, ref, rtol=1e-4, atol=4e-3)
+
+
+@pytest.mark.parametrize("ta,tb", [(False, True), (False, False), (True, False)])
+@pytest.mark.parametrize("out_dtype", [torch.float16, torch.float32])
+def test_tensor_engine_ieee_half(ctx, ta, tb, out_dtype):
+    """IEEE half operands (the FP16 projection filter's type): exact products, fp32 accumulation."""
+    from paper_2609_21102_b200 import binding
+    b, M, N, K = 2, 328, 264, 200
+    A = _mk(b, K if ta else M, M if ta else K, torch.float16, 21)
+    B = _mk(b, N if tb else K, K if tb else N, torch.float16, 22)
+    C = ctx.defl_debug_gemm(A, B, ta, tb, engine=binding.ENGINE_TENSOR, out_dtype=out_dtype)
+    ref = _ref(A, B, ta, tb)
+    if out_dtype == torch.float32:
+        assert torch.allclose(C, ref, rtol=1e-4, atol=2e-3)
+    else:
+        assert torch.allclose(C.float(), ref, rtol=2.0 ** -10, atol=2e-3)      # one rounding to half on store
+    As = _mk(b, 456, 320, torch.float16, 23)
+    Cs = ctx.defl_debug_gemm(As, As, False, True, engine=binding.ENGINE_TENSOR, out_dtype=out_dtype, exploit_symmetry=True)
+    assert torch.equal(Cs, Cs.transpose(1, 2))
+    assert torch.allclose(Cs.float(), _ref(As, As, False, True), rtol=2.0 ** -10, atol=2e-3)
+    with pytest.raises(binding.DeflError) as e:
+        ctx.defl_debug_gemm(A, B, ta, tb, engine=binding.ENGINE_SIMT)
+    assert e.value.code == -4

@@ -45,10 +45,13 @@ SCHED7 = [[1.875, -1.25, 0.375]] * 7
 
 
 @pytest.mark.parametrize("n,K,k", [(256, 8, 4), (200, 6, 3), (384, 16, 8)])
-@pytest.mark.parametrize("engine_name", ["tensor", "simt"])
+@pytest.mark.parametrize("engine_name", ["tensor", "simt", "half"])
 def test_psd_matches_oracle_with_tracked_basis(ctx, n, K, k, engine_name):
+    """engine "half": the filter steps in IEEE half precision (the paper's SDP runs use the filter in half
+    precision, Appendix C.2), everything around them unchanged; same oracle, same tolerance."""
     from paper_2609_21102_b200 import binding
-    engine = binding.ENGINE_AUTO if engine_name == "tensor" else binding.ENGINE_SIMT
+    engine = binding.ENGINE_SIMT if engine_name == "simt" else binding.ENGINE_AUTO
+    half = engine_name == "half"
     X64, lam, q = _sdp_like(n, k, 50.0, 600 + n)
     X = X64.float().cuda()
     V0 = inputs.randn((n, K), 77 + n).float()
@@ -57,14 +60,15 @@ def test_psd_matches_oracle_with_tracked_basis(ctx, n, K, k, engine_name):
     Vo = _orth(V0.double().numpy())
     Xo = X.double().cpu().numpy()
     for it in range(3):          # three block steps on a static matrix: the basis converges on both sides
-        P, info = ctx.defl_psd_project(X, k, Vg, SCHED7, gamma=1.1, lanczos_start=v0, engine=engine, want_info=True)
+        P, info = ctx.defl_psd_project(X, k, Vg, SCHED7, gamma=1.1, lanczos_start=v0, engine=engine, want_info=True,
+                                       half_filter=half)
         torch.cuda.synchronize()
         Po, Vo_next, lam_o, ndef, theta_o = oracle.psd_project(Xo, Vo, k, oracle.schedule(SCHED7), gamma=1.1,
                                                                lanczos_v0=v0.double().cpu().numpy())
         assert int(info["status"][0]) == 0
         Pg = P.double().cpu().numpy()
         assert np.array_equal(Pg, Pg.T)
-        tol = TOL_TF32_UNDEFLATED if (it == 0 and engine_name == "tensor") else TOL
+        tol = TOL_TF32_UNDEFLATED if (it == 0 and engine_name != "simt") else TOL
         assert _rel(Pg, Po) <= tol, (it, _rel(Pg, Po))
         assert abs(float(info["theta"][0]) - theta_o) <= 1e-3 * theta_o
         lg = info["lam"].double().cpu().numpy()
@@ -183,3 +187,14 @@ def test_psd_with_the_stage_one_minimax_schedule(ctx):
     bulk = lambda M: np.linalg.norm((M - head) - (exact - head)) / np.linalg.norm(exact - head)
     assert bulk(Po) <= 1e-3          # the oracle with this filter is the projection up to eigenvalues below eps theta
     assert bulk(Pg) <= 2e-2          # tf32 against the exact projection, bulk only (measured 1.0e-2)
+
+
+def test_half_filter_needs_the_tensor_engine_and_aligned_rows(ctx):
+    from paper_2609_21102_b200 import binding
+    X = torch.eye(200, device="cuda")
+    with pytest.raises(binding.DeflError) as e:
+        ctx.defl_psd_project(X, 0, None, SCHED7, engine=binding.ENGINE_SIMT, half_filter=True)
+    assert e.value.code == -4
+    with pytest.raises(binding.DeflError) as e:
+        ctx.defl_psd_project(torch.eye(204, device="cuda"), 0, None, SCHED7, half_filter=True)     # 204 = 8 * 25.5
+    assert e.value.code == -4

@@ -26,6 +26,7 @@ sys.path.insert(0, ROOT)
 METRIC = "deflated polar-filter TFLOP/s & matrices/s per batch; % bf16 tensor peak"
 MUON = (3.4445, -4.7750, 2.0315)
 SYM = True   # compute X X^T and A A on the tiles that reach the diagonal and mirror them (--no-symmetry turns it off)
+BF16_ITERATES = False   # --bf16-iterates: keep the filter's iterates in bf16 instead of scaled IEEE half
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 WORKLOADS = {
@@ -182,7 +183,7 @@ def run_step(ctx, wl, groups, lanes=None):
     if not lanes:
         for g in groups:
             ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"],
-                                   sketch=g["Om"], gamma=1.01, exploit_symmetry=SYM)
+                                   sketch=g["Om"], gamma=1.01, exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
         return
     main = torch.cuda.current_stream()
     fork = torch.cuda.Event()
@@ -191,7 +192,7 @@ def run_step(ctx, wl, groups, lanes=None):
         s.wait_event(fork)
         with torch.cuda.stream(s):
             c.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"],
-                                 sketch=g["Om"], gamma=1.01, exploit_symmetry=SYM)
+                                 sketch=g["Om"], gamma=1.01, exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
             done = torch.cuda.Event()
             done.record(s)
         main.wait_event(done)
@@ -224,11 +225,13 @@ def main():
     ap.add_argument("--small", action="store_true", help="tiny workload for a quick functional check")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-symmetry", action="store_true", help="compute the symmetric products in full")
+    ap.add_argument("--bf16-iterates", action="store_true", help="filter iterates stored in bf16 (default: scaled IEEE half)")
     ap.add_argument("--streams", type=int, default=2, help="2: one stream + context per shape group; 1: one stream")
     ap.add_argument("--batch", type=int, default=0, help="override the matrices per shape group (profiling captures)")
     args = ap.parse_args()
-    global SYM
+    global SYM, BF16_ITERATES
     SYM = not args.no_symmetry
+    BF16_ITERATES = bool(args.bf16_iterates)
     wl_name = "small" if args.small else "gpt2_xl"
     wl = dict(WORKLOADS[wl_name])
     if args.batch > 0:
@@ -239,6 +242,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     config = {"workload": wl["label"], "name": wl_name, "k": wl["k"], "oversample": wl["p"], "power_iters": wl["J"],
               "filter_steps": wl["L"], "restore": "padded, gamma=1.01", "exploit_symmetry": SYM,
+              "storage": "input and output bf16; filter iterates " + ("bf16" if BF16_ITERATES else "IEEE half scaled by 32 (same tensor rate)"),
               "l2": "inputs (1.2 GB per step) larger than L2; no flush"}
     tot_f = sum(b * sum(flops_per_matrix(m, n, wl["k"], wl["p"], wl["J"], wl["L"])) for b, m, n in wl["groups"])
     nmat = sum(b for b, _, _ in wl["groups"])
@@ -314,7 +318,7 @@ def main():
     for rep in range(STAGE_REPS):
         for g, (b, m, n) in zip(groups, wl["groups"]):
             ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"], sketch=g["Om"],
-                                   gamma=1.01, exploit_symmetry=SYM)
+                                   gamma=1.01, exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
             ms = ctx.defl_get_stage_ms()
             for i in range(min(4, len(ms))):
                 stage_tot[i] += ms[i] / STAGE_REPS
@@ -325,7 +329,7 @@ def main():
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for g in groups:
-        ctx.defl_polar_batched(g["G"], 0, 0, 0, [list(MUON)] * wl["L"], out=g["out"], exploit_symmetry=SYM)
+        ctx.defl_polar_batched(g["G"], 0, 0, 0, [list(MUON)] * wl["L"], out=g["out"], exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
     e1.record()
     torch.cuda.synchronize()
     plain_ms = e0.elapsed_time(e1)

@@ -34,7 +34,7 @@ class DeflOpts(ctypes.Structure):
     _fields_ = [("sketch", ctypes.c_void_p), ("seed", ctypes.c_uint64), ("restore_mode", ctypes.c_int),
                 ("gamma", ctypes.c_float), ("norm_mode", ctypes.c_int), ("lanczos_start", ctypes.c_void_p),
                 ("warmup", ctypes.c_int), ("engine", ctypes.c_int), ("exploit_symmetry", ctypes.c_int),
-                ("tau", ctypes.c_float), ("half_filter", ctypes.c_int)]
+                ("tau", ctypes.c_float), ("half_filter", ctypes.c_int), ("bf16_iterates", ctypes.c_int)]
 
 
 class DeflInfo(ctypes.Structure):
@@ -157,7 +157,7 @@ class Context:
             raise DeflError(rc, lib().defl_last_error(self._h).decode())
 
     def _opts(self, sketch=None, seed=0, restore_mode=RESTORE_PADDED, gamma=0.0, norm_mode=NORM_LANCZOS,
-              lanczos_start=None, warmup=False, engine=ENGINE_AUTO, exploit_symmetry=False, tau=0.0, half_filter=False):
+              lanczos_start=None, warmup=False, engine=ENGINE_AUTO, exploit_symmetry=False, tau=0.0, half_filter=False, bf16_iterates=False):
         o = DeflOpts()
         o.sketch = sketch.data_ptr() if sketch is not None else None
         o.seed = seed
@@ -170,12 +170,13 @@ class Context:
         o.exploit_symmetry = int(bool(exploit_symmetry))
         o.tau = tau
         o.half_filter = int(bool(half_filter))
+        o.bf16_iterates = int(bool(bf16_iterates))
         return o
 
     # ------------------------------------------------------------------------------------------
     def defl_polar_batched(self, G, k, oversample, power_iters, coeff_schedule, steps=None, out=None, sketch=None,
                            seed=0, restore_mode=RESTORE_PADDED, gamma=0.0, engine=ENGINE_AUTO,
-                           exploit_symmetry=False, want_info=False, tau=0.0):
+                           exploit_symmetry=False, want_info=False, tau=0.0, bf16_iterates=False):
         """out[b,m,n] = deflated polar factor of every G[b] (Algorithm 3 + Algorithm 1)."""
         _dev(G, "G")
         if G.ndim != 3:
@@ -188,7 +189,7 @@ class Context:
             if sketch.dtype != torch.float32:
                 raise TypeError("sketch must be float32")
         opts = self._opts(sketch=sketch, seed=seed, restore_mode=restore_mode, gamma=gamma, engine=engine,
-                          exploit_symmetry=exploit_symmetry, tau=tau)
+                          exploit_symmetry=exploit_symmetry, tau=tau, bf16_iterates=bf16_iterates)
         info = DeflInfo()
         extras = None
         if want_info:

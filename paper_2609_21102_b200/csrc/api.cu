@@ -451,6 +451,19 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
   const float gamma = (opts && opts->gamma > 0.f) ? opts->gamma : 1.01f;
   const int sym = (opts && opts->exploit_symmetry) ? 1 : 0;
   const float tau = opts ? opts->tau : 0.f;
+  // Iterate type of the filter. bf16 inputs: X_t, A_t, B_t are kept in IEEE half, scaled by 32 (Y = 32 X, so
+  // A' = Y Y^T = 1024 A and the step's coefficients become a, b/2^10, c/2^20; the last product scales back by 1/32).
+  // Same tensor-core rate as bf16, three more mantissa bits: the rounding of the stored iterate is what limits
+  // the bf16 path's accuracy on wide matrices with slowly decaying spectra. The power-of-two scale keeps small
+  // entries (1/sqrt(mn) of a normalised residual, off-diagonal Gram entries) out of half's subnormal range, and
+  // overflow would need a singular value above 8. opts->bf16_iterates keeps everything in bf16; shapes the tensor
+  // engine cannot take (rows not a multiple of 8 elements, unaligned buffers) do too, since the fp32 FMA engine
+  // has no half path.
+  const bool half_iter = dtype == DEFL_BF16 && engine != DEFL_ENGINE_SIMT && L > 0 && !(opts && opts->bf16_iterates) &&
+                         (m % 8 == 0) && (n % 8 == 0) && ((reinterpret_cast<uintptr_t>(out) & 15) == 0) &&
+                         ((reinterpret_cast<uintptr_t>(G) & 15) == 0) && (!upd || (reinterpret_cast<uintptr_t>(upd->W) & 15) == 0);
+  const int it_dtype = half_iter ? (int)F16 : dtype;
+  const float ys = half_iter ? 32.f : 1.f;
 
   cudaSetDevice(c->device);
   int rc = ctx_reserve(c, carve_polar(nullptr, b, m, n, dtype, k, l).bytes);
@@ -528,8 +541,8 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
       return DEFL_ERR_CUDA;
     }
     g.epilogue = EPI_AUX_PLUS; g.partials = nullptr;
-    g.aux_scale = 1.f; g.aux_scale_dev = w.inv_rho; g.alpha = 1.f;
-    g.C = bufs[cur]; g.ldc = n; g.batch_c = (long long)m * n; g.out_dtype = dtype;
+    g.aux_scale = ys; g.aux_scale_dev = w.inv_rho; g.alpha = ys;
+    g.C = bufs[cur]; g.ldc = n; g.batch_c = (long long)m * n; g.out_dtype = it_dtype;
     if ((rc = run_gemm(c, g, deng, "deflate+normalise"))) return rc;
   } else {
     const int nblk = 296;
@@ -538,7 +551,7 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
     if (ctx_fail(c, rho_finalize_launch(w.npart, nblk, b, w.rho, w.inv_rho, w.inv_rho2, w.status, c->stream,
                                         &c->launches), "rho"))
       return DEFL_ERR_CUDA;
-    if (ctx_fail(c, scale_launch(G, dtype, bufs[cur], dtype, b, (long long)m * n, w.inv_rho, c->stream, &c->launches), "normalise"))
+    if (ctx_fail(c, scale_launch(G, dtype, bufs[cur], it_dtype, b, (long long)m * n, w.inv_rho, c->stream, &c->launches, 0, ys), "normalise"))
       return DEFL_ERR_CUDA;
   }
   ctx_stage_mark(c);
@@ -549,7 +562,7 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
     const void* X = bufs[cur];
     void* Xn = bufs[cur ^ 1];
     GemmDesc g = gemm_desc_zero();
-    g.batch = b; g.in_dtype = dtype; g.b_dtype = dtype; g.out_dtype = dtype;
+    g.batch = b; g.in_dtype = it_dtype; g.b_dtype = it_dtype; g.out_dtype = it_dtype;
     // A_t = X X^T (wide) or X^T X (tall), ms x ms, symmetric
     g.M = ms; g.N = ms; g.K[0] = ml;
     g.A[0] = X; g.B[0] = X; g.batch_a[0] = g.batch_b[0] = (long long)m * n;
@@ -560,17 +573,18 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
     if ((rc = run_gemm(c, g, engine, "gram"))) return rc;
     // B_t = a I + b A_t + c A_t A_t
     g = gemm_desc_zero();
-    g.batch = b; g.in_dtype = dtype; g.b_dtype = dtype; g.out_dtype = dtype;
+    g.batch = b; g.in_dtype = it_dtype; g.b_dtype = it_dtype; g.out_dtype = it_dtype;
     g.M = ms; g.N = ms; g.K[0] = ms;
     g.A[0] = w.Am; g.sa_i[0] = ms; g.sa_k[0] = 1; g.batch_a[0] = (long long)ms * ms;
     g.B[0] = w.Am; g.sb_k[0] = 1; g.sb_j[0] = ms; g.batch_b[0] = (long long)ms * ms;   // A_t symmetric: rows as columns
     g.C = w.Bm; g.ldc = ms; g.batch_c = (long long)ms * ms;
-    g.aux = w.Am; g.ld_aux = ms; g.batch_aux = (long long)ms * ms; g.aux_dtype = dtype;
-    g.epilogue = EPI_POLY; g.pa = ca; g.pb = cb; g.pc = cc; g.symmetric = sym;
+    g.aux = w.Am; g.ld_aux = ms; g.batch_aux = (long long)ms * ms; g.aux_dtype = it_dtype;
+    // (with scaled iterates the stored Gram is ys^2 A_t: the coefficients absorb the powers)
+    g.epilogue = EPI_POLY; g.pa = ca; g.pb = cb / (ys * ys); g.pc = cc / (ys * ys * ys * ys); g.symmetric = sym;
     if ((rc = run_gemm(c, g, engine, "polynomial"))) return rc;
     // X <- B_t X (wide) or X B_t (tall)
     g = gemm_desc_zero();
-    g.batch = b; g.in_dtype = dtype; g.b_dtype = dtype; g.out_dtype = dtype;
+    g.batch = b; g.in_dtype = it_dtype; g.b_dtype = it_dtype; g.out_dtype = it_dtype;
     g.M = m; g.N = n;
     if (wide) {
       g.K[0] = m;
@@ -583,11 +597,12 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
     }
     g.C = Xn; g.ldc = n; g.batch_c = (long long)m * n;
     g.epilogue = EPI_STORE;
+    if (t == L - 1) { g.out_dtype = dtype; g.alpha = 1.f / ys; }      // the result leaves in the caller's type and scale
     if (upd && t == L - 1) {
       // last step of a Muon update: W <- keep W + step (B_L X) instead of storing the iterate
       g.C = upd->W; g.out_dtype = upd->w_dtype;
       g.aux = upd->W; g.ld_aux = n; g.batch_aux = (long long)m * n; g.aux_dtype = upd->w_dtype;
-      g.epilogue = EPI_AUX_PLUS; g.alpha = upd->step; g.aux_scale = upd->keep;
+      g.epilogue = EPI_AUX_PLUS; g.alpha = upd->step / ys; g.aux_scale = upd->keep;
     }
     if ((rc = run_gemm(c, g, engine, "apply"))) return rc;
     cur ^= 1;

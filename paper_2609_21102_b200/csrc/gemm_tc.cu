@@ -70,7 +70,7 @@ struct TcParams {
   uint32_t idesc;
   // epilogue
   int epilogue, out_dtype, aux_dtype, symmetric, round_tf32;
-  int half_f16;                // 16-bit operands, aux and output are IEEE half (else bf16)
+  int aux_f16, out_f16;        // a 16-bit aux / output is IEEE half (else bf16); the operands' kind is in idesc
   void* C; long long ldc, batch_c;
   const void* aux; long long ld_aux, batch_aux;
   float alpha, aux_scale, pa, pb, pc;
@@ -343,7 +343,7 @@ __device__ __forceinline__ void load_aux16(const TcParams& p, bool take, bool ve
   if (EPI == EPI_STORE) return;
   const uint16_t* auxh = reinterpret_cast<const uint16_t*>(p.aux);
   const float* auxf = reinterpret_cast<const float*>(p.aux);
-  const bool f16 = p.half_f16 != 0;
+  const bool f16 = p.aux_f16 != 0;
   if (!take) {
 #pragma unroll
     for (int j = 0; j < 16; ++j) x[j] = 0.f;
@@ -370,7 +370,7 @@ __device__ __forceinline__ void finish16(const TcParams& p, const uint32_t* r, c
                                          float aux_scale, double& sq) {
   if (gj0 >= p.N) return;
   const bool out_bf16 = (p.out_dtype != F32);       // a 16-bit output type
-  const bool f16 = p.half_f16 != 0;
+  const bool f16 = p.out_f16 != 0;
   uint16_t* outh = reinterpret_cast<uint16_t*>(p.C);
   float* outf = reinterpret_cast<float*>(p.C);
   float v[16];
@@ -490,7 +490,7 @@ __device__ __forceinline__ void epilogue_block_fast(const TcParams& p, uint32_t 
   tmem_ld_wait();
   const int gi = gi_warp0 + lane;
   const bool row_ok = gi < p.M;
-  const bool f16 = p.half_f16 != 0;
+  const bool f16 = p.aux_f16 != 0, o16 = p.out_f16 != 0;
   float sqf = 0.f;
 #pragma unroll
   for (int pc = 0; pc < pp; ++pc) {
@@ -522,7 +522,7 @@ __device__ __forceinline__ void epilogue_block_fast(const TcParams& p, uint32_t 
       if (ES == 2) {
         uint32_t* hh = reinterpret_cast<uint32_t*>(&q);
 #pragma unroll
-        for (int j = 0; j < epp / 2; ++j) hh[j] = pack16x2(v[2 * j], v[2 * j + 1], f16);
+        for (int j = 0; j < epp / 2; ++j) hh[j] = pack16x2(v[2 * j], v[2 * j + 1], o16);
       } else {
         q = make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2 % epp]), __float_as_uint(v[3 % epp]));
       }
@@ -1030,13 +1030,6 @@ bool gemm_tc_supported(const GemmDesc& g) {
   if (g.nseg < 1 || g.nseg > 2) return false;
   if (g.b_split == 2 && (g.nseg != 1 || !aligned16(g.B[1]))) return false;
   if (g.b_dtype != g.in_dtype) return false;
-  // one 16-bit kind per launch: the epilogue converts aux and output with the operands' kind
-  {
-    const int kinds[3] = {g.in_dtype, g.epilogue == EPI_STORE ? F32 : g.aux_dtype, g.epilogue == EPI_RESID_NORM ? F32 : g.out_dtype};
-    bool bf = false, hf = false;
-    for (int i = 0; i < 3; ++i) { bf |= kinds[i] == BF16; hf |= kinds[i] == F16; }
-    if (bf && hf) return false;
-  }
   const int esize = (int)dtype_size(g.in_dtype);
   if (g.symmetric && g.M != g.N) return false;
   for (int s = 0; s < g.nseg; ++s) {
@@ -1134,7 +1127,8 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)p.a_mn_major << 15) | ((uint32_t)p.b_mn_major << 16) |
             ((uint32_t)((p.pair ? 256 : 128) >> 4) << 24);
   p.epilogue = g.epilogue; p.out_dtype = g.out_dtype; p.aux_dtype = g.aux_dtype; p.symmetric = g.symmetric; p.round_tf32 = g.round_tf32;
-  p.half_f16 = (g.in_dtype == F16 || (g.epilogue != EPI_STORE && g.aux_dtype == F16) || g.out_dtype == F16) ? 1 : 0;
+  p.aux_f16 = (g.epilogue != EPI_STORE && g.aux_dtype == F16) ? 1 : 0;
+  p.out_f16 = (g.out_dtype == F16) ? 1 : 0;
   p.C = g.C; p.ldc = g.ldc; p.batch_c = g.batch_c;
   p.aux = g.aux; p.ld_aux = g.ld_aux; p.batch_aux = g.batch_aux;
   p.alpha = g.alpha; p.aux_scale = g.aux_scale; p.pa = g.pa; p.pb = g.pb; p.pc = g.pc;

@@ -467,9 +467,9 @@ cudaError_t scale_cols_launch(const float* In, long long in_bs, int ld_in, int b
 
 // Out[b, i] = scale[b] * In[b, i]  (type conversion allowed)
 __global__ void scale_kernel(const void* __restrict__ In, int in_dt, void* __restrict__ Out, int out_dt,
-                             long long count, const float* __restrict__ scale, int round_tf32) {
+                             long long count, const float* __restrict__ scale, int round_tf32, float mult) {
   const int bz = blockIdx.y;
-  const float sc = scale ? scale[bz] : 1.f;
+  const float sc = (scale ? scale[bz] : 1.f) * mult;
   const long long base = (long long)bz * count;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (long long)gridDim.x * blockDim.x)
   {
@@ -480,9 +480,9 @@ __global__ void scale_kernel(const void* __restrict__ In, int in_dt, void* __res
 }
 
 cudaError_t scale_launch(const void* In, int in_dt, void* Out, int out_dt, int batch, long long count,
-                         const float* scale, cudaStream_t st, long long* launches, int round_tf32) {
+                         const float* scale, cudaStream_t st, long long* launches, int round_tf32, float mult) {
   const int nblk = (int)min((long long)1184, (count + 255) / 256);
-  scale_kernel<<<dim3(nblk, batch), 256, 0, st>>>(In, in_dt, Out, out_dt, count, scale, round_tf32);
+  scale_kernel<<<dim3(nblk, batch), 256, 0, st>>>(In, in_dt, Out, out_dt, count, scale, round_tf32, mult);
   if (launches) ++*launches;
   return cudaGetLastError();
 }

@@ -25,7 +25,7 @@ cudaError_t scale_cols_launch(const float* In, long long in_bs, int ld_in, int b
                               int ld_s, const float* inv_rho, float c0, float c1, float* Out, long long out_bs,
                               int ld_out, cudaStream_t st, long long* launches, const int* keff = nullptr);
 cudaError_t scale_launch(const void* In, int in_dt, void* Out, int out_dt, int batch, long long count,
-                         const float* scale, cudaStream_t st, long long* launches, int round_tf32 = 0);
+                         const float* scale, cudaStream_t st, long long* launches, int round_tf32 = 0, float mult = 1.f);
 cudaError_t fill_gaussian_launch(void* dst, long long count, int dtype, unsigned long long seed, long long per_stream,
                                  unsigned long long seed_stride, cudaStream_t st, long long* launches);
 cudaError_t fill_int_launch(int* p, int n, int v, cudaStream_t st, long long* launches);

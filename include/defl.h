@@ -32,7 +32,7 @@ extern "C" {
 #endif
 
 /* storage types of G / out */
-#define DEFL_BF16 0 /* bf16 storage, bf16 tensor-core products, fp32 accumulation */
+#define DEFL_BF16 0 /* bf16 storage of inputs and outputs, 16-bit tensor-core products, fp32 accumulation */
 #define DEFL_F32 1  /* fp32 storage; polar path: fp32 FMA products; PSD filter: tf32 tensor-core products */
 #define DEFL_F16 2  /* IEEE half: the FP16 filter of the PSD projection (opts->half_filter) and defl_debug_gemm only */
 

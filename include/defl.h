@@ -90,8 +90,7 @@ typedef struct defl_opts {
                             Needs n a multiple of 8 and the tensor engine. */
   int bf16_iterates;     /* polar path with bf16 input, non-zero: keep the filter's iterates X_t, A_t, B_t in bf16.
                             Default (0): they are kept in IEEE half scaled by 32 (same tensor-core rate, three more
-                            mantissa bits; input, output and every other stage are unchanged), whenever the shape
-                            allows the tensor engine throughout (m, n multiples of 8, 16-byte aligned buffers). */
+                            mantissa bits; input, output and every other stage are unchanged). */
 } defl_opts;
 
 typedef struct defl_info {

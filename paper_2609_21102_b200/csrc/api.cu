@@ -60,11 +60,7 @@ int run_gemm(defl_ctx* c, const GemmDesc& g, int engine, const char* what) {
   }
   cudaError_t e;
   if (tc) e = gemm_tc_launch(g, c->stream, c->wait_status, c->num_sms, &c->launches);
-  else if (g.in_dtype == F16 || g.b_dtype == F16) {
-    // IEEE half operands exist for the tensor cores only (the FP16 projection filter)
-    snprintf(c->err, sizeof(c->err), "%s: half-precision operands need the tensor engine", what);
-    return DEFL_ERR_UNSUPPORTED;
-  } else e = gemm_simt_launch(g, c->stream, &c->launches);
+  else e = gemm_simt_launch(g, c->stream, &c->launches);
   if (ctx_fail(c, e, what)) return DEFL_ERR_CUDA;
   return DEFL_OK;
 }
@@ -456,12 +452,8 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
   // Same tensor-core rate as bf16, three more mantissa bits: the rounding of the stored iterate is what limits
   // the bf16 path's accuracy on wide matrices with slowly decaying spectra. The power-of-two scale keeps small
   // entries (1/sqrt(mn) of a normalised residual, off-diagonal Gram entries) out of half's subnormal range, and
-  // overflow would need a singular value above 8. opts->bf16_iterates keeps everything in bf16; shapes the tensor
-  // engine cannot take (rows not a multiple of 8 elements, unaligned buffers) do too, since the fp32 FMA engine
-  // has no half path.
-  const bool half_iter = dtype == DEFL_BF16 && engine != DEFL_ENGINE_SIMT && L > 0 && !(opts && opts->bf16_iterates) &&
-                         (m % 8 == 0) && (n % 8 == 0) && ((reinterpret_cast<uintptr_t>(out) & 15) == 0) &&
-                         ((reinterpret_cast<uintptr_t>(G) & 15) == 0) && (!upd || (reinterpret_cast<uintptr_t>(upd->W) & 15) == 0);
+  // overflow would need a singular value above 8. opts->bf16_iterates keeps everything in bf16.
+  const bool half_iter = dtype == DEFL_BF16 && L > 0 && !(opts && opts->bf16_iterates);
   const int it_dtype = half_iter ? (int)F16 : dtype;
   const float ys = half_iter ? 32.f : 1.f;
 

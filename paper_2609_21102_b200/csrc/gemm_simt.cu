@@ -1,4 +1,4 @@
-// fp32-FMA product engine: C = epilogue(opA(A) opB(B)) for arbitrary strides and bf16/fp32 inputs.
+// fp32-FMA product engine: C = epilogue(opA(A) opB(B)) for arbitrary strides and bf16/half/fp32 inputs.
 // It is the library's own reference engine (every shape, exact fp32 products) and the engine of
 // the fp32 polar path; the large bf16 products normally run on the tensor-core engine instead.
 #include "common.cuh"
@@ -15,6 +15,8 @@ template <>
 __device__ __forceinline__ float to_f<float>(float v) { return v; }
 template <>
 __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <>
+__device__ __forceinline__ float to_f<__half>(__half v) { return __half2float(v); }
 
 template <typename TIn, typename TB>
 __global__ void __launch_bounds__(NT) gemm_simt_kernel(const GemmDesc g) {
@@ -175,7 +177,11 @@ int gemm_simt_partials_per_batch(const GemmDesc& g) {
 cudaError_t gemm_simt_launch(const GemmDesc& g, cudaStream_t st, long long* launches) {
   if (g.batch <= 0 || g.M <= 0 || g.N <= 0) return cudaSuccess;
   dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.batch);
-  if (g.in_dtype == BF16 && g.b_dtype == BF16) gemm_simt_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, NT, 0, st>>>(g);
+  if (g.in_dtype == F16 || g.b_dtype == F16) {
+    // IEEE half operands (iterates of the bf16 path on shapes the tensor engine cannot take): both or neither
+    if (g.in_dtype != F16 || g.b_dtype != F16) return cudaErrorNotSupported;
+    gemm_simt_kernel<__half, __half><<<grid, NT, 0, st>>>(g);
+  } else if (g.in_dtype == BF16 && g.b_dtype == BF16) gemm_simt_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, NT, 0, st>>>(g);
   else if (g.in_dtype == BF16) gemm_simt_kernel<__nv_bfloat16, float><<<grid, NT, 0, st>>>(g);
   else if (g.b_dtype == BF16) gemm_simt_kernel<float, __nv_bfloat16><<<grid, NT, 0, st>>>(g);
   else gemm_simt_kernel<float, float><<<grid, NT, 0, st>>>(g);

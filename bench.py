@@ -27,6 +27,10 @@ METRIC = "deflated polar-filter TFLOP/s & matrices/s per batch; % bf16 tensor pe
 MUON = (3.4445, -4.7750, 2.0315)
 SYM = True   # compute X X^T and A A on the tiles that reach the diagonal and mirror them (--no-symmetry turns it off)
 BF16_ITERATES = False   # --bf16-iterates: keep the filter's iterates in bf16 instead of scaled IEEE half
+GAMMA = 1.01            # padding of the restored head (1.1 with the minimax schedule, the value the paper uses with it)
+SCHEDULE = "muon"       # --schedule minimax: per-step minimax quintics (the Polar-Express-style mapping)
+SCHEDULE_NOTE = "Muon quintic (3.4445, -4.7750, 2.0315) every step"
+_MINIMAX = {}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 WORKLOADS = {
@@ -37,6 +41,18 @@ WORKLOADS = {
     "small": {"groups": [(4, 256, 1024), (4, 256, 256)], "k": 8, "p": 8, "J": 1, "L": 5,
               "label": "small check: 4 x 256x1024 + 4 x 256x256"},
 }
+
+
+def sched_of(wl):
+    """The [L][3] coefficient schedule of the run: Muon's quintic repeated, or per-step minimax quintics built by
+    greedy Remez exchange from [1e-3, 1] (first step rescaled by 1.01); same products per step either way."""
+    L = wl["L"]
+    if SCHEDULE == "muon":
+        return [list(MUON)] * L
+    if L not in _MINIMAX:
+        from paper_2609_21102_b200 import schedules
+        _MINIMAX[L] = [list(c) for c in schedules.remez_sign_schedule(1e-3, L, margin=0.01)[0]]
+    return _MINIMAX[L]
 
 
 def flops_per_matrix(m, n, k, p, J, L):
@@ -182,8 +198,8 @@ def run_step(ctx, wl, groups, lanes=None):
     import torch
     if not lanes:
         for g in groups:
-            ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"],
-                                   sketch=g["Om"], gamma=1.01, exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
+            ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], sched_of(wl), out=g["out"],
+                                   sketch=g["Om"], gamma=GAMMA, exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
         return
     main = torch.cuda.current_stream()
     fork = torch.cuda.Event()
@@ -191,8 +207,8 @@ def run_step(ctx, wl, groups, lanes=None):
     for g, (c, s) in zip(groups, lanes):
         s.wait_event(fork)
         with torch.cuda.stream(s):
-            c.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"],
-                                 sketch=g["Om"], gamma=1.01, exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
+            c.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], sched_of(wl), out=g["out"],
+                                 sketch=g["Om"], gamma=GAMMA, exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
             done = torch.cuda.Event()
             done.record(s)
         main.wait_event(done)
@@ -210,7 +226,7 @@ def oracle_sample(wl, seconds_hint=20.0):
     l = min(min(m, n), wl["k"] + wl["p"])
     Om = inputs.sketch(1, min(m, n), l, 4, si).double().numpy()[0]
     t0 = time.perf_counter()
-    oracle.deflated_polar(G, wl["k"], l, Om, wl["J"], oracle.schedule(MUON, wl["L"]), gamma=1.01)
+    oracle.deflated_polar(G, wl["k"], l, Om, wl["J"], oracle.schedule(sched_of(wl)), gamma=GAMMA)
     dt = time.perf_counter() - t0
     filt, rest = flops_per_matrix(m, n, wl["k"], wl["p"], wl["J"], wl["L"])
     return dt, (filt + rest), "1 matrix %dx%d of the batch, full path, fp64" % (m, n)
@@ -226,10 +242,17 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-symmetry", action="store_true", help="compute the symmetric products in full")
     ap.add_argument("--bf16-iterates", action="store_true", help="filter iterates stored in bf16 (default: scaled IEEE half)")
+    ap.add_argument("--schedule", choices=["muon", "minimax"], default="muon",
+                    help="muon: Muon's quintic every step; minimax: per-step minimax quintics (Polar-Express-style)")
     ap.add_argument("--streams", type=int, default=2, help="2: one stream + context per shape group; 1: one stream")
     ap.add_argument("--batch", type=int, default=0, help="override the matrices per shape group (profiling captures)")
     args = ap.parse_args()
-    global SYM, BF16_ITERATES
+    global SYM, BF16_ITERATES, SCHEDULE, SCHEDULE_NOTE, GAMMA
+    SCHEDULE = args.schedule
+    if SCHEDULE == "minimax":
+        GAMMA = 1.1
+        SCHEDULE_NOTE = ("per-step minimax quintics (greedy Remez from [1e-3, 1], first step / 1.01): the "
+                         "Polar-Express-style mapping, coefficients computed by schedules.remez_sign_schedule")
     SYM = not args.no_symmetry
     BF16_ITERATES = bool(args.bf16_iterates)
     wl_name = "small" if args.small else "gpt2_xl"
@@ -237,11 +260,13 @@ def main():
     if args.batch > 0:
         wl["groups"] = [(args.batch, m, n) for _, m, n in wl["groups"]]
         wl["label"] += " [batch overridden to %d per group]" % args.batch
+    if SCHEDULE == "minimax":
+        wl["label"] = wl["label"].replace("5 Muon quintic steps", "5 per-step minimax quintic steps (Polar-Express-style)")
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     config = {"workload": wl["label"], "name": wl_name, "k": wl["k"], "oversample": wl["p"], "power_iters": wl["J"],
-              "filter_steps": wl["L"], "restore": "padded, gamma=1.01", "exploit_symmetry": SYM,
+              "filter_steps": wl["L"], "restore": "padded, gamma=%g" % GAMMA, "schedule": SCHEDULE_NOTE, "exploit_symmetry": SYM,
               "storage": "input and output bf16; filter iterates " + ("bf16" if BF16_ITERATES else "IEEE half scaled by 32 (same tensor rate)"),
               "l2": "inputs (1.2 GB per step) larger than L2; no flush"}
     tot_f = sum(b * sum(flops_per_matrix(m, n, wl["k"], wl["p"], wl["J"], wl["L"])) for b, m, n in wl["groups"])
@@ -317,8 +342,8 @@ def main():
     STAGE_REPS = 3          # averaged: a single step's split moves by several percent with the power state
     for rep in range(STAGE_REPS):
         for g, (b, m, n) in zip(groups, wl["groups"]):
-            ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], out=g["out"], sketch=g["Om"],
-                                   gamma=1.01, exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
+            ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], sched_of(wl), out=g["out"], sketch=g["Om"],
+                                   gamma=GAMMA, exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
             ms = ctx.defl_get_stage_ms()
             for i in range(min(4, len(ms))):
                 stage_tot[i] += ms[i] / STAGE_REPS
@@ -329,7 +354,7 @@ def main():
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for g in groups:
-        ctx.defl_polar_batched(g["G"], 0, 0, 0, [list(MUON)] * wl["L"], out=g["out"], exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
+        ctx.defl_polar_batched(g["G"], 0, 0, 0, sched_of(wl), out=g["out"], exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
     e1.record()
     torch.cuda.synchronize()
     plain_ms = e0.elapsed_time(e1)
@@ -341,13 +366,13 @@ def main():
         hO = [torch.empty_like(h).pin_memory() for h in hG]
         def e2e_group(c, h, o, g, stream=None):
             if stream is None:
-                c.defl_polar_batched_host(h, o, wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], sketch=g["Om"], gamma=1.01,
+                c.defl_polar_batched_host(h, o, wl["k"], wl["p"], wl["J"], sched_of(wl), sketch=g["Om"], gamma=GAMMA,
                                           exploit_symmetry=SYM)
             else:
                 torch.cuda.set_device(local_rank)
                 with torch.cuda.stream(stream):
-                    c.defl_polar_batched_host(h, o, wl["k"], wl["p"], wl["J"], [list(MUON)] * wl["L"], sketch=g["Om"],
-                                              gamma=1.01, exploit_symmetry=SYM)
+                    c.defl_polar_batched_host(h, o, wl["k"], wl["p"], wl["J"], sched_of(wl), sketch=g["Om"],
+                                              gamma=GAMMA, exploit_symmetry=SYM)
 
         def e2e_step():
             # the call blocks until its output sits in host memory; with one context per shape group the groups

@@ -301,13 +301,14 @@ struct TileInfo {
   bool skip;
 };
 
-__device__ __forceinline__ TileInfo tile_info(const TcParams& p, long long tile) {
+__device__ __forceinline__ TileInfo tile_info(const TcParams& p, long long tile64) {
   TileInfo t;
+  const int tile = (int)tile64;          // the host refuses launches with 2^31 tiles or more: 32-bit divisions
   if (p.symmetric) {
     // only tiles that reach the diagonal or lie right of it are enumerated, so that every CTA gets the same
     // share of real work: tile row tm starts at column tile (tm * tile_m) / BN
-    t.bz = (int)(tile / p.tiles_per_matrix);
-    int idx = (int)(tile % p.tiles_per_matrix);
+    t.bz = tile / p.tiles_per_matrix;
+    int idx = tile - t.bz * p.tiles_per_matrix;
     int tm = 0;
     for (; tm < p.tiles_m; ++tm) {
       const int first = (tm * p.tile_m) / p.BN;
@@ -317,9 +318,10 @@ __device__ __forceinline__ TileInfo tile_info(const TcParams& p, long long tile)
     }
     t.tm = tm;
   } else {
-    t.tn = (int)(tile % p.tiles_n);
-    t.tm = (int)((tile / p.tiles_n) % p.tiles_m);
-    t.bz = (int)(tile / ((long long)p.tiles_n * p.tiles_m));
+    t.bz = tile / p.tiles_per_matrix;
+    const int idx = tile - t.bz * p.tiles_per_matrix;
+    t.tm = idx / p.tiles_n;
+    t.tn = idx - t.tm * p.tiles_n;
   }
   const int row0 = t.tm * p.tile_m, col_end = (t.tn + 1) * p.BN;
   t.skip = p.symmetric && col_end <= row0;               // entirely below the diagonal
@@ -1081,6 +1083,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
     }
   }
   p.total_tiles = (long long)p.tiles_per_matrix * g.batch;
+  if (p.total_tiles >= (1ll << 31)) return cudaErrorNotSupported;      // the kernel's tile arithmetic is 32-bit
   p.nseg = g.nseg;
   OperandPlan pa, pb;
   // when a dimension has extent 1 both strides may look "unit"; prefer K-major

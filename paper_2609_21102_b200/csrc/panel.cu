@@ -258,14 +258,27 @@ __device__ __forceinline__ double warp_sum(double v) {
   return v;
 }
 
-__global__ void __launch_bounds__(1024) jacobi_eig_kernel(const double* __restrict__ partial, int nchunk, int l,
-                                                          int signed_input, float* __restrict__ s_out,
-                                                          float* __restrict__ E, float* __restrict__ Es,
-                                                          int* __restrict__ status, int max_sweeps) {
+// eight lanes of a warp add up their values (the lanes sub = 0..7 of one column pair)
+__device__ __forceinline__ double group8_sum(double v) {
+  v += __shfl_xor_sync(0xffffffffu, v, 1);
+  v += __shfl_xor_sync(0xffffffffu, v, 2);
+  v += __shfl_xor_sync(0xffffffffu, v, 4);
+  return v;
+}
+
+constexpr int JAC_THREADS = 256;        // 32 column pairs x 8 lanes
+constexpr int JAC_NR = MAX_L / 8;       // rows per lane
+
+__global__ void __launch_bounds__(JAC_THREADS) jacobi_eig_kernel(const double* __restrict__ partial, int nchunk, int l,
+                                                                 int signed_input, float* __restrict__ s_out,
+                                                                 float* __restrict__ E, float* __restrict__ Es,
+                                                                 int* __restrict__ status, int max_sweeps) {
   extern __shared__ double sm[];
-  double* A = sm;             // column-major: A[c * l + r]
-  double* V = sm + l * l;     // column-major
+  const int ls = l | 1;       // column stride (odd: the four pairs of a warp start in different banks)
+  double* A = sm;             // column-major: A[c * ls + r]
+  double* V = sm + MAX_L * (MAX_L + 1);     // column-major
   __shared__ double lam[MAX_L];
+  __shared__ double nrm2[MAX_L];      // squared column norms of A, carried along by the rotations
   __shared__ int order[MAX_L];
   __shared__ int rotated;
   const int bz = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -277,48 +290,112 @@ __global__ void __launch_bounds__(1024) jacobi_eig_kernel(const double* __restri
       t += pb[(long long)ch * l * l + r * l + c];
       u += pb[(long long)ch * l * l + c * l + r];
     }
-    A[c * l + r] = 0.5 * (t + u);
-    V[c * l + r] = (r == c) ? 1.0 : 0.0;
+    A[c * ls + r] = 0.5 * (t + u);
+    V[c * ls + r] = (r == c) ? 1.0 : 0.0;
   }
   __syncthreads();
   const int np = (l + 1) & ~1;        // players, padded to even
   const int npairs = np / 2;
+  // Eight lanes per column pair, four pairs per warp: the three dot products of a pair take three shuffle steps
+  // each instead of five, and a round issues a sixth of the shuffles of the one-warp-per-pair form (whose
+  // shuffle traffic, not its arithmetic, filled the round).
+  const int grp = tid >> 3, sub = tid & 7;
+  const int nr = (l + 7) >> 3;        // rows per lane actually present
+  // The eigenvector accumulation V is needed only for a signed spectrum (to tell the sign of an eigenvalue). For
+  // a Gram matrix the columns of A converge to lambda_j v_j with lambda_j >= 0, so the eigenvectors are the
+  // normalised columns: the rotations skip V, a third of the fp64 work (fp64 issue is what bounds this kernel).
+  const bool track_v = signed_input != 0;
   int sweep = 0;
   for (; sweep < max_sweeps; ++sweep) {
     if (tid == 0) rotated = 0;
+    // Squared column norms, exact at the start of every sweep. Within the sweep a rotation by tan t moves
+    // t gamma from one column's squared norm to the other's (alpha' = alpha - t gamma, beta' = beta + t gamma), so
+    // a round computes one dot product per pair instead of three; the sweep that finds nothing to rotate, which
+    // ends the iteration, has tested every pair against exact norms.
+    for (int j0 = 0; j0 < l; j0 += JAC_THREADS / 8) {      // (the same trip count for every lane: shuffles inside)
+      const int j = j0 + grp;
+      double acc = 0.0;
+#pragma unroll
+      for (int i = 0; i < JAC_NR; ++i) {
+        const int r = sub + 8 * i;
+        if (i < nr && r < l && j < l) { const double v = A[j * ls + r]; acc = fma(v, v, acc); }
+      }
+      acc = group8_sum(acc);
+      if (sub == 0 && j < l) nrm2[j] = acc;
+    }
     __syncthreads();
     for (int round = 0; round < np - 1; ++round) {
-      if (warp < npairs) {
-        int p, q;
-        if (warp == 0) { p = np - 1; q = round; }
-        else { p = (round + warp) % (np - 1); q = (round - warp + (np - 1)) % (np - 1); }
+      int p = 0, q = l;
+      if (grp < npairs) {
+        if (grp == 0) { p = np - 1; q = round; }
+        else {
+          // (round + grp) and (round - grp) modulo np - 1: both lie within one period of the range
+          p = round + grp; if (p >= np - 1) p -= np - 1;
+          q = round - grp; if (q < 0) q += np - 1;
+        }
         if (p > q) { const int t = p; p = q; q = t; }
-        if (q < l) {
-          double* ap = A + p * l; double* aq = A + q * l;
-          const double x0 = (lane < l) ? ap[lane] : 0.0, x1 = (lane + 32 < l) ? ap[lane + 32] : 0.0;
-          const double y0 = (lane < l) ? aq[lane] : 0.0, y1 = (lane + 32 < l) ? aq[lane + 32] : 0.0;
-          const double alpha = warp_sum(x0 * x0 + x1 * x1);
-          const double beta = warp_sum(y0 * y0 + y1 * y1);
-          const double gamma = warp_sum(x0 * y0 + x1 * y1);
-          // rotate when |gamma| > 1e-14 sqrt(alpha beta) (compared in squares). The rotation is built from one
-          // division and two reciprocal square roots: fp64 divisions and square roots are long instruction
-          // sequences, and this chain is the latency of a round.
-          if (gamma != 0.0 && gamma * gamma > 1e-28 * (alpha * beta)) {
-            if (lane == 0) rotated = 1;
-            const double zeta = (beta - alpha) / (2.0 * gamma);
-            const double w = 1.0 + zeta * zeta;
-            const double root = w * rsqrt(w);                          // sqrt(1 + zeta^2)
-            // t = sign(zeta) / (|zeta| + root) = sign(zeta) (root - |zeta|)   [(root - |zeta|)(root + |zeta|) = 1],
-            // evaluated in the stable form for large |zeta|: 1 / (|zeta| + root) = rsqrt-free via one more division
-            const double t = ((zeta >= 0.0) ? 1.0 : -1.0) / (fabs(zeta) + root);
-            const double c = rsqrt(1.0 + t * t), sn = c * t;
-            if (lane < l) { ap[lane] = c * x0 - sn * y0; aq[lane] = sn * x0 + c * y0; }
-            if (lane + 32 < l) { ap[lane + 32] = c * x1 - sn * y1; aq[lane + 32] = sn * x1 + c * y1; }
-            double* vp = V + p * l; double* vq = V + q * l;
-            if (lane < l) { const double a = vp[lane], b = vq[lane]; vp[lane] = c * a - sn * b; vq[lane] = sn * a + c * b; }
-            if (lane + 32 < l) {
-              const double a = vp[lane + 32], b = vq[lane + 32];
-              vp[lane + 32] = c * a - sn * b; vq[lane + 32] = sn * a + c * b;
+      }
+      const bool live = q < l;            // (a pair with the padding player, or a group beyond the pairs, idles)
+      double* ap = A + p * ls; double* aq = A + (live ? q : p) * ls;
+      double x[JAC_NR], y[JAC_NR];
+      double pg = 0.0;
+#pragma unroll
+      for (int i = 0; i < JAC_NR; ++i) {
+        if (i < nr) {
+          const int r = sub + 8 * i;
+          const bool in = live && r < l;
+          x[i] = in ? ap[r] : 0.0;
+          y[i] = in ? aq[r] : 0.0;
+          pg = fma(x[i], y[i], pg);
+        }
+      }
+      const double gamma = group8_sum(pg);
+      const double alpha = live ? nrm2[p] : 0.0, beta = live ? nrm2[q] : 0.0;
+      // rotate when |gamma| > 1e-11 sqrt(alpha beta) (compared in squares): the eigenvalues are then good to about
+      // 1e-22 and the vectors to 1e-11 over the relative gap, far beyond the fp32 outputs
+      if (live && gamma != 0.0 && gamma * gamma > 1e-22 * (alpha * beta)) {
+        if (sub == 0) rotated = 1;
+        // The rotation angle only steers the iteration (any exact rotation keeps V orthogonal and the invariants
+        // intact), so tan is computed in fp32 from the exponent-scaled pair (beta - alpha, 2 gamma); cos comes
+        // from an fp32 reciprocal square root refined by two Newton steps in fp64, which makes c^2 + s^2 = 1 hold
+        // to fp64 rounding. A rotation then leaves 1e-7 of the inner product instead of none, and the pair's
+        // next visit removes that. The chain of dependent fp64 operations, which is the latency of a round,
+        // shrinks to a third. Out-of-range exponents take the fp64 formula.
+        const double d = beta - alpha, g2 = 2.0 * gamma;
+        const double big = fmax(fabs(d), fabs(g2));
+        const int ex = (int)((__double_as_longlong(big) >> 52) & 0x7ff);
+        const double sc = __longlong_as_double((long long)(2046 - ex) << 52);       // 2^(1023 - ex)
+        const float df = (float)(d * sc), gf = (float)(g2 * sc);
+        double c, sn, tg;
+        if (ex >= 1 && ex <= 2045 && fabsf(gf) > 1e-30f) {
+          const float zf = df / gf, az = fabsf(zf);
+          // t = sign(zeta) / (|zeta| + sqrt(1 + zeta^2)): the root of t^2 + 2 zeta t - 1 = 0 of smaller magnitude
+          const float tf = (az > 1e15f) ? 0.5f / zf : copysignf(1.0f / (az + sqrtf(fmaf(zf, zf, 1.0f))), zf);
+          const double t = (double)tf;
+          const double w = fma(t, t, 1.0), h = 0.5 * w;            // w in [1, 2]
+          double yv = (double)rsqrtf((float)w);
+          yv = yv * fma(-h * yv, yv, 1.5);
+          yv = yv * fma(-h * yv, yv, 1.5);
+          c = yv; sn = yv * t;
+          tg = t * gamma;
+        } else {
+          const double zeta = d / g2;
+          const double w = 1.0 + zeta * zeta;
+          const double root = w * rsqrt(w);                          // sqrt(1 + zeta^2)
+          const double t = ((zeta >= 0.0) ? 1.0 : -1.0) / (fabs(zeta) + root);
+          c = rsqrt(1.0 + t * t); sn = c * t;
+          tg = t * gamma;
+        }
+        if (sub == 0) { nrm2[p] = alpha - tg; nrm2[q] = beta + tg; }
+        double* vp = V + p * ls; double* vq = V + q * ls;
+#pragma unroll
+        for (int i = 0; i < JAC_NR; ++i) {
+          const int r = sub + 8 * i;
+          if (i < nr && r < l) {
+            ap[r] = c * x[i] - sn * y[i]; aq[r] = sn * x[i] + c * y[i];
+            if (track_v) {
+              const double a = vp[r], b = vq[r];
+              vp[r] = c * a - sn * b; vq[r] = sn * a + c * b;
             }
           }
         }
@@ -332,12 +409,21 @@ __global__ void __launch_bounds__(1024) jacobi_eig_kernel(const double* __restri
   // eigenvalues
   if (warp < 32) {
     for (int j = warp; j < l; j += (blockDim.x >> 5)) {
-      const double* aj = A + j * l; const double* vj = V + j * l;
+      const double* aj = A + j * ls; const double* vj = V + j * ls;
       const double a0 = (lane < l) ? aj[lane] : 0.0, a1 = (lane + 32 < l) ? aj[lane + 32] : 0.0;
       const double v0 = (lane < l) ? vj[lane] : 0.0, v1 = (lane + 32 < l) ? vj[lane + 32] : 0.0;
       const double nrm = sqrt(warp_sum(a0 * a0 + a1 * a1));
       const double rq = warp_sum(a0 * v0 + a1 * v1);
       if (lane == 0) lam[j] = signed_input ? ((rq >= 0.0) ? nrm : -nrm) : nrm;
+      if (!track_v) {
+        // v_j = a_j / lambda_j; a column that vanished (rank-deficient input) keeps its unit vector, which only
+        // ever meets a zero singular value
+        const double inv = (nrm > 1e-150) ? 1.0 / nrm : 0.0;
+        if (nrm > 1e-150) {
+          if (lane < l) V[j * ls + lane] = a0 * inv;
+          if (lane + 32 < l) V[j * ls + lane + 32] = a1 * inv;
+        }
+      }
     }
   }
   __syncthreads();
@@ -354,7 +440,7 @@ __global__ void __launch_bounds__(1024) jacobi_eig_kernel(const double* __restri
   for (int e = tid; e < l * l; e += blockDim.x) {
     const int r = e / l, cc = e % l;
     const int src = order[cc];
-    const double v = V[src * l + r];
+    const double v = V[src * ls + r];
     const double lm = lam[src];
     const double sv = signed_input ? lm : sqrt(lm > 0.0 ? lm : 0.0);
     if (E) E[(long long)bz * l * l + e] = (float)v;
@@ -365,13 +451,13 @@ __global__ void __launch_bounds__(1024) jacobi_eig_kernel(const double* __restri
 
 cudaError_t jacobi_eig_launch(const double* partial, int nchunk, int batch, int l, int signed_input, float* s_out,
                               float* E, float* Es, int* status, cudaStream_t st, long long* launches) {
-  const size_t smem = 2 * (size_t)l * l * sizeof(double);
+  const size_t smem = 2 * (size_t)MAX_L * (MAX_L + 1) * sizeof(double);
   static bool attr_set = false;
   if (!attr_set) {
-    cudaFuncSetAttribute(jacobi_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * MAX_L * MAX_L * 8);
+    cudaFuncSetAttribute(jacobi_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     attr_set = true;
   }
-  jacobi_eig_kernel<<<batch, 1024, smem, st>>>(partial, nchunk, l, signed_input, s_out, E, Es, status, 40);
+  jacobi_eig_kernel<<<batch, JAC_THREADS, smem, st>>>(partial, nchunk, l, signed_input, s_out, E, Es, status, 40);
   if (launches) ++*launches;
   return cudaGetLastError();
 }

@@ -228,7 +228,9 @@ int defl_frobenius_norms_noalloc(const void* X, int dtype, int b, long long coun
 /* Diagnostics: one batched product C[b,M,N] = alpha * opA(A) opB(B) through a chosen engine, used by the
  * tests to check the tensor-core tile engine against the fp32 engine (no counterpart in the paper).
  * A element (i,kk) is A[i*sa_i + kk*sa_k], B element (kk,j) is B[kk*sb_k + j*sb_j]; C is row-major [M,N].
- * in_dtype / out_dtype are DEFL_BF16 or DEFL_F32; strides in elements. */
+ * in_dtype / out_dtype are DEFL_BF16 or DEFL_F32; strides in elements. exploit_symmetry: bit 0 = the product is
+ * symmetric (upper tiles computed and mirrored); bit 1 = the product is written transposed, C row-major [N,M]
+ * (tensor engine only; DEFL_ERR_UNSUPPORTED otherwise). */
 int defl_debug_gemm(defl_ctx* ctx, int engine, int batch, int M, int N, int K,
                     const void* A, long long sa_i, long long sa_k, long long batch_a,
                     const void* B, long long sb_k, long long sb_j, long long batch_b,

@@ -334,8 +334,9 @@ class Context:
         return dst
 
     def defl_debug_gemm(self, A, B, trans_a=False, trans_b=False, engine=ENGINE_AUTO, out_dtype=None, alpha=1.0,
-                        exploit_symmetry=False):
-        """C[b] = alpha * op(A[b]) op(B[b]); op = transpose of the stored matrix when the flag is set."""
+                        exploit_symmetry=False, transpose_out=False):
+        """C[b] = alpha * op(A[b]) op(B[b]); op = transpose of the stored matrix when the flag is set. With
+        transpose_out the engine writes the product transposed: the result has shape [b, N, M]."""
         _dev(A, "A"), _dev(B, "B")
         b = A.shape[0]
         if trans_a:
@@ -351,11 +352,12 @@ class Context:
             N = B.shape[2]
             sb_k, sb_j = N, 1
         out_dtype = out_dtype or A.dtype
-        C = torch.empty((b, M, N), dtype=out_dtype, device=A.device)
+        C = torch.empty((b, N, M) if transpose_out else (b, M, N), dtype=out_dtype, device=A.device)
         self._sync_stream()
         rc = lib().defl_debug_gemm(self._h, engine, b, M, N, K, _ptr(A), sa_i, sa_k, A.shape[1] * A.shape[2],
                                    _ptr(B), sb_k, sb_j, B.shape[1] * B.shape[2], _ptr(C), _dtype_code(A),
-                                   {torch.bfloat16: BF16, torch.float16: F16}.get(out_dtype, F32), alpha, int(exploit_symmetry))
+                                   {torch.bfloat16: BF16, torch.float16: F16}.get(out_dtype, F32), alpha,
+                                   int(bool(exploit_symmetry)) | (2 if transpose_out else 0))
         self._check(rc)
         return C
 

@@ -54,7 +54,7 @@ bool use_tensor_engine(const GemmDesc& g, int engine) {
 // Run one product on the engine the options ask for. Returns a DEFL_* code.
 int run_gemm(defl_ctx* c, const GemmDesc& g, int engine, const char* what) {
   const bool tc = use_tensor_engine(g, engine);
-  if (engine == DEFL_ENGINE_TENSOR && !tc) {
+  if ((engine == DEFL_ENGINE_TENSOR || g.transpose_out) && !tc) {
     snprintf(c->err, sizeof(c->err), "%s: shape/type not supported by the tensor engine", what);
     return DEFL_ERR_UNSUPPORTED;
   }
@@ -374,7 +374,8 @@ int defl_debug_gemm(defl_ctx* c, int engine, int batch, int M, int N, int K, con
   g.B[0] = B; g.sb_k[0] = sb_k; g.sb_j[0] = sb_j; g.batch_b[0] = batch_b;
   g.in_dtype = in_dtype; g.b_dtype = in_dtype;
   g.C = C; g.ldc = N; g.batch_c = (long long)M * N; g.out_dtype = out_dtype;
-  g.epilogue = EPI_STORE; g.alpha = alpha; g.symmetric = exploit_symmetry ? 1 : 0;
+  g.epilogue = EPI_STORE; g.alpha = alpha; g.symmetric = (exploit_symmetry & 1) ? 1 : 0;
+  if (exploit_symmetry & 2) { g.transpose_out = 1; g.ldc = M; }
   return run_gemm(c, g, engine, "debug gemm");
 }
 
@@ -590,6 +591,19 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
     g.C = Xn; g.ldc = n; g.batch_c = (long long)m * n;
     g.epilogue = EPI_STORE;
     if (t == L - 1) { g.out_dtype = dtype; g.alpha = 1.f / ys; }      // the result leaves in the caller's type and scale
+    if (wide && !(upd && t == L - 1)) {
+      // The tensor engine pads the product's rows to whole 256-row tiles, its columns only to 32: for a wide X
+      // whose short side is not a multiple of 256 (1600 = 6.25 tiles) it is cheaper to compute (B X)^T = X^T B
+      // (rows = the long side) and let the epilogue write the tile transposed, which is the same memory.
+      GemmDesc gt = g;
+      gt.M = n; gt.N = m;
+      gt.A[0] = X; gt.sa_i[0] = 1; gt.sa_k[0] = n; gt.batch_a[0] = (long long)m * n;
+      gt.B[0] = w.Bm; gt.sb_j[0] = m; gt.sb_k[0] = 1; gt.batch_b[0] = (long long)m * m;    // B_t symmetric
+      gt.transpose_out = 1;
+      const long long pad_rows = (long long)((m + 255) / 256) * 256 * ((n + 31) / 32 * 32);
+      const long long pad_rows_t = (long long)((n + 255) / 256) * 256 * ((m + 31) / 32 * 32);
+      if (m > 128 && pad_rows_t < pad_rows && use_tensor_engine(gt, engine) && !getenv("DEFL_NO_TRANSPOSED_APPLY")) g = gt;
+    }
     if (upd && t == L - 1) {
       // last step of a Muon update: W <- keep W + step (B_L X) instead of storing the iterate
       g.C = upd->W; g.out_dtype = upd->w_dtype;

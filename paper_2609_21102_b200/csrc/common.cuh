@@ -43,6 +43,7 @@ struct GemmDesc {
   int b_split;                  // 2: opB = B[0] + B[1] (same shape and strides, nseg must be 1); the A tile is loaded once
   int round_tf32;               // fp32 output rounded to nearest tf32 (it feeds tf32 products, which would truncate)
   int symmetric;                // output is symmetric (M == N): compute upper tiles only and mirror
+  int transpose_out;            // element (i, j) of the product is stored at C[j * ldc + i] (tensor engine, EPI_STORE only)
 };
 
 inline GemmDesc gemm_desc_zero() {

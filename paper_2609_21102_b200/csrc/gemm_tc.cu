@@ -70,6 +70,7 @@ struct TcParams {
   uint32_t idesc;
   // epilogue
   int epilogue, out_dtype, aux_dtype, symmetric, round_tf32;
+  int transposed;              // EPI_STORE: the tile is written transposed, element (i, j) at C[j * ldc + i]
   int aux_f16, out_f16;        // a 16-bit aux / output is IEEE half (else bf16); the operands' kind is in idesc
   void* C; long long ldc, batch_c;
   const void* aux; long long ld_aux, batch_aux;
@@ -396,6 +397,18 @@ __device__ __forceinline__ void finish16(const TcParams& p, const uint32_t* r, c
     return;
   }
   if (!row_ok) return;
+  if (p.transposed) {
+    // for a fixed column the 32 lanes are 32 consecutive rows of the product, one contiguous run of C
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const int gj = gj0 + j;
+      if (gj < p.N) {
+        const size_t m = cbatch + (size_t)gj * p.ldc + gi;
+        if (out_bf16) outh[m] = (uint16_t)pack16x2(v[j], 0.f, f16); else outf[m] = v[j];
+      }
+    }
+    return;
+  }
   // symmetric output: chunks entirely right of the warp's rows are stored like any other chunk and mirrored;
   // chunks that touch the diagonal go element by element; chunks left of it are skipped by the caller
   const bool mirror_all = p.symmetric && gj0 > gi_warp0 + 31;
@@ -537,14 +550,17 @@ __device__ __forceinline__ void epilogue_block_fast(const TcParams& p, uint32_t 
     return;
   }
   __syncwarp();
-  uint8_t* cbase = reinterpret_cast<uint8_t*>(p.C) + ((size_t)bz * p.batch_c + (size_t)gi_warp0 * p.ldc + gj0) * ES;
+  if (!p.transposed) {
+    uint8_t* cbase = reinterpret_cast<uint8_t*>(p.C) + ((size_t)bz * p.batch_c + (size_t)gi_warp0 * p.ldc + gj0) * ES;
 #pragma unroll
-  for (int i = 0; i < pp; ++i) {
-    const int row = prow + rpi * i;
-    const uint4 q = *reinterpret_cast<const uint4*>(stg + stage_off(row, piece, rowb, pp));
-    if (gi_warp0 + row < p.M) *reinterpret_cast<uint4*>(cbase + (size_t)row * p.ldc * ES + piece * 16) = q;
+    for (int i = 0; i < pp; ++i) {
+      const int row = prow + rpi * i;
+      const uint4 q = *reinterpret_cast<const uint4*>(stg + stage_off(row, piece, rowb, pp));
+      if (gi_warp0 + row < p.M) *reinterpret_cast<uint4*>(cbase + (size_t)row * p.ldc * ES + piece * 16) = q;
+    }
   }
-  if (p.symmetric && gj0 > gi_warp0) {
+  // (a transposed output is written the way a symmetric one is mirrored)
+  if (p.transposed || (p.symmetric && gj0 > gi_warp0)) {
     // mirror image of a block above the diagonal (the caller guarantees 32 complete rows): transposed row c of the
     // block is 32 values = pp pieces of 16 bytes; pp consecutive lanes write one such row, each lane gathering its
     // epp values from one column of the staged block
@@ -621,7 +637,8 @@ __device__ __forceinline__ void epilogue_half(const TcParams& p, uint32_t taddr,
   // the coalesced path wants `aux` and the output in the same type (true of every product the library makes)
   // (symmetric output: the mirror stores of the coalesced path assume 32 complete rows)
   const bool fast_ok = vec_ok && (EPI == EPI_STORE || EPI == EPI_RESID_NORM || a2 == o2) &&
-                       (!p.symmetric || (gi_warp0 + 32 <= p.M && EPI != EPI_RESID_NORM));
+                       (!p.symmetric || (gi_warp0 + 32 <= p.M && EPI != EPI_RESID_NORM)) &&
+                       (!p.transposed || gi_warp0 + 32 <= p.M);
   int c0 = wsel * 32;
   if (fast_ok) {
     // the complete 32-column blocks come first; whatever is left (a ragged edge) takes the general path below
@@ -1034,6 +1051,7 @@ bool gemm_tc_supported(const GemmDesc& g) {
   if (g.b_dtype != g.in_dtype) return false;
   const int esize = (int)dtype_size(g.in_dtype);
   if (g.symmetric && g.M != g.N) return false;
+  if (g.transpose_out && (g.epilogue != EPI_STORE || g.symmetric)) return false;
   for (int s = 0; s < g.nseg; ++s) {
     if (g.K[s] <= 0) return false;
     if (!aligned16(g.A[s]) || !aligned16(g.B[s])) return false;
@@ -1130,6 +1148,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)p.a_mn_major << 15) | ((uint32_t)p.b_mn_major << 16) |
             ((uint32_t)((p.pair ? 256 : 128) >> 4) << 24);
   p.epilogue = g.epilogue; p.out_dtype = g.out_dtype; p.aux_dtype = g.aux_dtype; p.symmetric = g.symmetric; p.round_tf32 = g.round_tf32;
+  p.transposed = g.transpose_out ? 1 : 0;
   p.aux_f16 = (g.epilogue != EPI_STORE && g.aux_dtype == F16) ? 1 : 0;
   p.out_f16 = (g.out_dtype == F16) ? 1 : 0;
   p.C = g.C; p.ldc = g.ldc; p.batch_c = g.batch_c;

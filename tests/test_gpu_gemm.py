@@ -77,6 +77,28 @@ def test_tensor_engine_bf16_output_and_large_tiles(ctx):
     assert err2 < 4e-3, float(err2)
 
 
+@pytest.mark.parametrize("b,M,N,K", [(2, 640, 200, 200), (1, 392, 136, 96), (2, 264, 72, 320), (1, 1600, 1600, 64)])
+@pytest.mark.parametrize("ta,tb", [(True, True), (False, True), (True, False)])
+@pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
+def test_tensor_engine_transposed_output(ctx, b, M, N, K, ta, tb, out_dtype):
+    """The product written transposed (the form the filter uses for X <- B X on a wide X): complete blocks take
+    the coalesced path, ragged rows and columns the general one."""
+    from paper_2609_21102_b200 import binding
+    A = _mk(b, K if ta else M, M if ta else K, torch.bfloat16, 21)
+    B = _mk(b, N if tb else K, K if tb else N, torch.bfloat16, 22)
+    C = ctx.defl_debug_gemm(A, B, ta, tb, engine=binding.ENGINE_TENSOR, out_dtype=out_dtype, alpha=0.25, transpose_out=True)
+    torch.cuda.synchronize()
+    assert C.shape == (b, N, M)
+    ref = _ref(A, B, ta, tb, 0.25).transpose(1, 2)
+    if out_dtype == torch.float32:
+        assert torch.allclose(C, ref, rtol=1e-4, atol=2e-3)
+    else:
+        assert torch.equal(C, ref.to(torch.bfloat16)) or float((C.float() - ref).norm() / ref.norm()) < 3e-3
+    with pytest.raises(binding.DeflError) as e:      # the fp32 engine does not write transposed: refused, not ignored
+        ctx.defl_debug_gemm(A, B, ta, tb, engine=binding.ENGINE_SIMT, out_dtype=out_dtype, transpose_out=True)
+    assert e.value.code == -4
+
+
 @pytest.mark.parametrize("engine_name", ["simt", "tensor"])
 def test_symmetric_mirroring(ctx, engine_name):
     from paper_2609_21102_b200 import binding

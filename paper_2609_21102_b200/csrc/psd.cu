@@ -165,6 +165,9 @@ __global__ void __launch_bounds__(1024) lanczos_step_kernel(int j, int n, int st
 // The same step with the work vector in registers (n <= 1024 * EPT): all j + 1 projections of a pass are reduced
 // together (warp shuffles, then one pass over the per-warp partial sums in warp order), two block barriers per pass
 // instead of a dependent chain of loops over global memory. alpha_j is the j-th projection of the first pass.
+// The vectors and the per-warp sums are fp32 (the vectors are stored in fp32 anyway); fp64 is kept for adding up
+// the 32 per-warp sums, the tridiagonal entries and the norm. With fp64 products and shuffles throughout, one CTA
+// spent 22 us per step on fp64 instruction issue alone.
 template <int EPT>
 __global__ void __launch_bounds__(1024) lanczos_step_reg_kernel(int j, int n, int steps, LanczosState s) {
   __shared__ double part[32][DEFL_LANCZOS_STEPS];
@@ -172,18 +175,18 @@ __global__ void __launch_bounds__(1024) lanczos_step_reg_kernel(int j, int n, in
   __shared__ double red[32];
   if (*s.done) return;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  double wv[EPT];
+  float wv[EPT];
 #pragma unroll
-  for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; wv[e] = (i < n) ? (double)s.w[i] : 0.0; }
+  for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; wv[e] = (i < n) ? s.w[i] : 0.f; }
   for (int pass = 0; pass < 2; ++pass) {
     for (int p = 0; p <= j; ++p) {
       const float* qp = s.Q + (long long)p * n;
-      double d = 0.0;
+      float d = 0.f;
 #pragma unroll
-      for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; if (i < n) d += (double)qp[i] * wv[e]; }
+      for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; if (i < n) d = fmaf(qp[i], wv[e], d); }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
-      if (lane == 0) part[warp][p] = d;
+      if (lane == 0) part[warp][p] = (double)d;
     }
     __syncthreads();
     if (tid <= j) {
@@ -195,20 +198,17 @@ __global__ void __launch_bounds__(1024) lanczos_step_reg_kernel(int j, int n, in
     __syncthreads();
     for (int p = 0; p <= j; ++p) {
       const float* qp = s.Q + (long long)p * n;
-      const double cp = coef[p];
+      const float cp = (float)coef[p];
 #pragma unroll
-      for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; if (i < n) wv[e] -= cp * (double)qp[i]; }
+      for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; if (i < n) wv[e] = fmaf(-cp, qp[i], wv[e]); }
     }
-    // (the work vector goes through fp32 between the passes, as it does when it lives in memory)
-#pragma unroll
-    for (int e = 0; e < EPT; ++e) wv[e] = (double)(float)wv[e];
   }
-  double b = 0.0;
+  float bf = 0.f;
 #pragma unroll
-  for (int e = 0; e < EPT; ++e) b += wv[e] * wv[e];
-  b = sqrt(block_sum(b, red));
+  for (int e = 0; e < EPT; ++e) bf = fmaf(wv[e], wv[e], bf);
+  const double b = sqrt(block_sum((double)bf, red));
 #pragma unroll
-  for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; if (i < n) s.w[i] = (float)wv[e]; }
+  for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; if (i < n) s.w[i] = wv[e]; }
   if (j + 1 == steps) return;
   const double a0 = s.T[0];
   if (!(b > 1e-12 * fabs(a0))) {
@@ -218,8 +218,9 @@ __global__ void __launch_bounds__(1024) lanczos_step_reg_kernel(int j, int n, in
   }
   if (tid == 0) { s.T[j * steps + j + 1] = b; s.T[(j + 1) * steps + j] = b; }
   float* qn = s.Q + (long long)(j + 1) * n;
+  const float inv_b = (float)(1.0 / b);
 #pragma unroll
-  for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; if (i < n) qn[i] = (float)(wv[e] / b); }
+  for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; if (i < n) qn[i] = wv[e] * inv_b; }
 }
 
 // v = sum_p E[p][0] q_p (the Ritz vector of the largest Ritz value); E is [steps, steps] row-major fp32

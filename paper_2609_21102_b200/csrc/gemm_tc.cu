@@ -489,6 +489,57 @@ __device__ __forceinline__ void aux_fetch_async(const TcParams& p, int lane, int
   cp_async_commit();
 }
 
+// The calling lane's row of one staged 32 x 32 block, 16 bytes at a time and in place: `aux` values in, results out
+// (nothing is written for the residual norm, whose partial sum of squares is returned). The formats of two-byte
+// values (F16A: `aux` is IEEE half, F16O: the output is; else bf16) and whether the block meets the diagonal (DIAG,
+// the polynomial's identity term) are template parameters, so that the loop has no per-element tests. Rows past M
+// need no test either: their `aux` was filled with zeros and so was their part of the A operand.
+template <int EPI, int ES, bool F16A, bool F16O, bool DIAG>
+__device__ __forceinline__ float transform_row(const TcParams& p, const uint32_t* r, uint8_t* stg, int lane, int gi, int gj0,
+                                               float alpha, float aux_scale) {
+  constexpr int rowb = 32 * ES, pp = rowb >> 4, epp = 16 / ES;   // epp = elements per 16-byte piece
+  const bool rnd = (ES == 4) && p.round_tf32 != 0;
+  float sqf = 0.f;
+#pragma unroll
+  for (int pc = 0; pc < pp; ++pc) {
+    uint4* slot = reinterpret_cast<uint4*>(stg + stage_off(lane, pc, rowb, pp));
+    float x[epp], v[epp];
+    if (EPI != EPI_STORE) {
+      const uint4 q = *slot;
+      if (ES == 2) {
+        const uint32_t* hh = reinterpret_cast<const uint32_t*>(&q);
+#pragma unroll
+        for (int j = 0; j < epp / 2; ++j) { const float2 f = unpack16x2(hh[j], F16A); x[2 * j] = f.x; x[2 * j + 1] = f.y; }
+      } else {
+        x[0] = __uint_as_float(q.x); x[1] = __uint_as_float(q.y); x[2 % epp] = __uint_as_float(q.z); x[3 % epp] = __uint_as_float(q.w);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < epp; ++j) {
+      const int c = pc * epp + j;
+      const float a = __uint_as_float(r[c]);
+      if (EPI == EPI_STORE) v[j] = alpha * a;
+      else if (EPI == EPI_POLY) v[j] = p.pb * x[j] + p.pc * a + ((DIAG && gi == gj0 + c) ? p.pa : 0.f);
+      else if (EPI == EPI_AUX_PLUS) v[j] = aux_scale * x[j] + alpha * a;
+      else v[j] = x[j] - a;
+      if (rnd) v[j] = round_to_tf32(v[j]);
+      if (EPI == EPI_RESID_NORM) sqf = fmaf(v[j], v[j], sqf);
+    }
+    if (EPI != EPI_RESID_NORM) {
+      uint4 q;
+      if (ES == 2) {
+        uint32_t* hh = reinterpret_cast<uint32_t*>(&q);
+#pragma unroll
+        for (int j = 0; j < epp / 2; ++j) hh[j] = pack16x2(v[2 * j], v[2 * j + 1], F16O);
+      } else {
+        q = make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2 % epp]), __float_as_uint(v[3 % epp]));
+      }
+      *slot = q;
+    }
+  }
+  return sqf;
+}
+
 // One complete 32 x 32 block whose `aux` values already sit (or are about to land) in `stg`. ES = element size of
 // `aux` and of the output (the same type). Each lane turns its row of the staged block into results 16 bytes at
 // a time, in place; the block then leaves with coalesced 16-byte stores. `pending` = number of cp.async groups
@@ -507,45 +558,21 @@ __device__ __forceinline__ void epilogue_block_fast(const TcParams& p, uint32_t 
   }
   tmem_ld_wait();
   const int gi = gi_warp0 + lane;
-  const bool row_ok = gi < p.M;
-  const bool f16 = p.aux_f16 != 0, o16 = p.out_f16 != 0;
-  float sqf = 0.f;
-#pragma unroll
-  for (int pc = 0; pc < pp; ++pc) {
-    uint4* slot = reinterpret_cast<uint4*>(stg + stage_off(lane, pc, rowb, pp));
-    float x[epp], v[epp];
-    if (EPI != EPI_STORE) {
-      const uint4 q = *slot;
-      if (ES == 2) {
-        const uint32_t* hh = reinterpret_cast<const uint32_t*>(&q);
-#pragma unroll
-        for (int j = 0; j < epp / 2; ++j) { const float2 f = unpack16x2(hh[j], f16); x[2 * j] = f.x; x[2 * j + 1] = f.y; }
-      } else {
-        x[0] = __uint_as_float(q.x); x[1] = __uint_as_float(q.y); x[2 % epp] = __uint_as_float(q.z); x[3 % epp] = __uint_as_float(q.w);
-      }
-    }
-#pragma unroll
-    for (int j = 0; j < epp; ++j) {
-      const int c = pc * epp + j;
-      const float a = __uint_as_float(r[c]);
-      if (EPI == EPI_STORE) v[j] = alpha * a;
-      else if (EPI == EPI_POLY) v[j] = p.pb * x[j] + p.pc * a + ((gi == gj0 + c) ? p.pa : 0.f);
-      else if (EPI == EPI_AUX_PLUS) v[j] = aux_scale * x[j] + alpha * a;
-      else v[j] = row_ok ? (x[j] - a) : 0.f;
-      if (p.round_tf32) v[j] = round_to_tf32(v[j]);
-      if (EPI == EPI_RESID_NORM) sqf = fmaf(v[j], v[j], sqf);
-    }
-    if (EPI != EPI_RESID_NORM) {
-      uint4 q;
-      if (ES == 2) {
-        uint32_t* hh = reinterpret_cast<uint32_t*>(&q);
-#pragma unroll
-        for (int j = 0; j < epp / 2; ++j) hh[j] = pack16x2(v[2 * j], v[2 * j + 1], o16);
-      } else {
-        q = make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2 % epp]), __float_as_uint(v[3 % epp]));
-      }
-      *slot = q;
-    }
+  // the formats of the two-byte types and the position of the diagonal are the same for the whole warp: one
+  // branch per block selects a row loop without per-element tests
+  const bool diag = (EPI == EPI_POLY) && gj0 < gi_warp0 + 32 && gj0 + 32 > gi_warp0;
+  const int fmt = (ES == 2 ? ((EPI != EPI_STORE && p.aux_f16) ? 1 : 0) | ((EPI != EPI_RESID_NORM && p.out_f16) ? 2 : 0) : 0) |
+                  (diag ? 4 : 0);
+  float sqf;
+  switch (fmt) {
+    case 0: sqf = transform_row<EPI, ES, false, false, false>(p, r, stg, lane, gi, gj0, alpha, aux_scale); break;
+    case 1: sqf = transform_row<EPI, ES, true, false, false>(p, r, stg, lane, gi, gj0, alpha, aux_scale); break;
+    case 2: sqf = transform_row<EPI, ES, false, true, false>(p, r, stg, lane, gi, gj0, alpha, aux_scale); break;
+    case 3: sqf = transform_row<EPI, ES, true, true, false>(p, r, stg, lane, gi, gj0, alpha, aux_scale); break;
+    case 4: sqf = transform_row<EPI, ES, false, false, true>(p, r, stg, lane, gi, gj0, alpha, aux_scale); break;
+    case 5: sqf = transform_row<EPI, ES, true, false, true>(p, r, stg, lane, gi, gj0, alpha, aux_scale); break;
+    case 6: sqf = transform_row<EPI, ES, false, true, true>(p, r, stg, lane, gi, gj0, alpha, aux_scale); break;
+    default: sqf = transform_row<EPI, ES, true, true, true>(p, r, stg, lane, gi, gj0, alpha, aux_scale); break;
   }
   if (EPI == EPI_RESID_NORM) {
     sq += (double)sqf;

@@ -373,7 +373,7 @@ __device__ __forceinline__ void load_aux16(const TcParams& p, bool take, bool ve
 template <int EPI>
 __device__ __forceinline__ void finish16(const TcParams& p, const uint32_t* r, const float* x, int gi, int gi_warp0,
                                          int gj0, bool row_ok, bool vec, size_t crow, size_t cbatch, float alpha,
-                                         float aux_scale, double& sq) {
+                                         float aux_scale, float& sq) {
   if (gj0 >= p.N) return;
   const bool out_bf16 = (p.out_dtype != F32);       // a 16-bit output type
   const bool f16 = p.out_f16 != 0;
@@ -396,7 +396,7 @@ __device__ __forceinline__ void finish16(const TcParams& p, const uint32_t* r, c
     float sqf = 0.f;
 #pragma unroll
     for (int j = 0; j < 16; ++j) sqf = fmaf(v[j], v[j], sqf);
-    sq += (double)sqf;
+    sq += sqf;
     return;
   }
   if (!row_ok) return;
@@ -546,7 +546,7 @@ __device__ __forceinline__ float transform_row(const TcParams& p, const uint32_t
 // that may still be in flight after this block's own (0 or 1).
 template <int EPI, int ES, int PENDING>
 __device__ __forceinline__ void epilogue_block_fast(const TcParams& p, uint32_t taddr, uint8_t* stg, int lane, int gi_warp0,
-                                                    int gj0, int bz, float alpha, float aux_scale, double& sq) {
+                                                    int gj0, int bz, float alpha, float aux_scale, float& sq) {
   constexpr int rowb = 32 * ES, pp = rowb >> 4, rpi = 32 / pp, epp = 16 / ES;   // epp = elements per 16-byte piece
   const int prow = lane / pp, piece = lane % pp;
   uint32_t r[32];
@@ -575,7 +575,7 @@ __device__ __forceinline__ void epilogue_block_fast(const TcParams& p, uint32_t 
     default: sqf = transform_row<EPI, ES, true, true, true>(p, r, stg, lane, gi, gj0, alpha, aux_scale); break;
   }
   if (EPI == EPI_RESID_NORM) {
-    sq += (double)sqf;
+    sq += sqf;
     __syncwarp();
     return;
   }
@@ -626,7 +626,7 @@ __device__ __forceinline__ void epilogue_block_fast(const TcParams& p, uint32_t 
 template <int EPI, int ES>
 __device__ __forceinline__ int epilogue_fast_blocks(const TcParams& p, uint32_t taddr, uint8_t* stg, int lane, int gi_warp0,
                                                     int col0, int c0, int lim, int bz, float alpha, float aux_scale,
-                                                    double& sq) {
+                                                    float& sq) {
   constexpr bool AHEAD = (ES == 2) && (EPI != EPI_STORE);
   int half = 0;
   // symmetric output: nothing to do for blocks entirely left of the warp's rows (they are written as mirror images)
@@ -654,7 +654,7 @@ __device__ __forceinline__ int epilogue_fast_blocks(const TcParams& p, uint32_t 
 
 template <int EPI>
 __device__ __forceinline__ void epilogue_half(const TcParams& p, uint32_t taddr, int gi, int gi_warp0, int col0, int n_eff,
-                                              int bz, int wsel, float alpha, float aux_scale, double& sq, uint8_t* stg,
+                                              int bz, int wsel, float alpha, float aux_scale, float& sq, uint8_t* stg,
                                               int lane) {
   const bool row_ok = gi < p.M;
   const bool aux_bf16 = (p.aux_dtype != F32);       // a 16-bit aux type
@@ -921,7 +921,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       if (p.alpha_dev) alpha *= p.alpha_dev[bz];
       if (p.aux_scale_dev) aux_scale *= p.aux_scale_dev[bz];
       for (int h = h_first; h <= h_last; ++h) {
-        double sq = 0.0;
+        float sq = 0.f;      // the warp's sum of squares over this tile half (at most 32 x 256 values), fp32
         if (t.halves & (1 << h)) {
           const uint32_t tcol = (!PAIR && p.tile_m == 256) ? (uint32_t)h * 256u : acc * 256u;
           const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + tcol;

@@ -1187,7 +1187,9 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   p.alpha_dev = g.alpha_dev; p.aux_scale_dev = g.aux_scale_dev;
   p.partials = g.partials; p.partials_per_batch = g.partials_per_batch;
   p.aux_prefetch = 0;
-  if (g.aux && g.epilogue != EPI_STORE && aligned16(g.aux)) {
+  // (Off unless DEFL_TC_AUX_PREFETCH is set: with the epilogue's own fetch one block ahead the extra L2 prefetch
+  // made the deflation passes 6 % slower and raised their DRAM reads to 1.6x the matrix, measured.)
+  if (g.aux && g.epilogue != EPI_STORE && aligned16(g.aux) && getenv("DEFL_TC_AUX_PREFETCH")) {
     const int aes = (int)dtype_size(g.aux_dtype);
     if ((g.ld_aux * aes) % 16 == 0 && (g.batch == 1 || (g.batch_aux * aes) % 16 == 0)) {
       EncodeTiledFn enc = get_encode_fn();

@@ -279,8 +279,8 @@ int defl_create(defl_ctx** out, int device) {
   c->device = device;
   cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device);
   int ok = 1;
-  if (cudaMalloc(&c->wait_status, sizeof(int)) != cudaSuccess) ok = 0;
-  if (ok) cudaMemset(c->wait_status, 0, sizeof(int));
+  if (cudaMalloc(&c->wait_status, 2 * sizeof(int)) != cudaSuccess) ok = 0;      // status word, tile counter
+  if (ok) cudaMemset(c->wait_status, 0, 2 * sizeof(int));
   for (int i = 0; ok && i < DEFL_MAX_MARKS; ++i)
     if (cudaEventCreate(&c->marks[i]) != cudaSuccess) ok = 0;
   cudaSetDevice(prev);

@@ -20,7 +20,7 @@ struct defl_ctx {
   cudaStream_t copy_in, copy_out;          // host-buffer entry point: copies overlap the compute stream
   cudaEvent_t chunk_in[DEFL_HOST_MAX_CHUNKS], chunk_done[DEFL_HOST_MAX_CHUNKS];
   int copy_ready;                           // streams and events above exist
-  int* wait_status;      // device word: the tensor engine ORs DEFL_ST_DEVICE_WAIT into it
+  int* wait_status;      // device words: [0] the tensor engine ORs DEFL_ST_DEVICE_WAIT into it, [1] its tile counter
   long long launches;    // kernels launched so far
   bool profiling;
   int n_marks;

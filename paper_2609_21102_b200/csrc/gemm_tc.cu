@@ -40,6 +40,7 @@ constexpr int EPI_WARPS = 8;
 constexpr int STAGING_BYTES = 4096;         // per epilogue warp: one 32 x 32 block of 4-byte values
 constexpr int AUX_AHEAD = 3;                // tiles (per CTA) by which the aux prefetch runs ahead
 constexpr int MAX_STAGES = 6;
+constexpr int SCHED_SLOTS = 8;              // tile numbers published ahead of the slowest reader (pair form)
 constexpr unsigned long long WAIT_NS = 2000000000ull;  // 2 s per wait before giving up
 
 struct TcParams {
@@ -78,6 +79,7 @@ struct TcParams {
   const float* alpha_dev; const float* aux_scale_dev;
   double* partials; int partials_per_batch;
   int* status;
+  unsigned int* tile_counter;  // pair form: tiles beyond each pair's first are handed out through this counter (null: fixed stride)
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -174,6 +176,12 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
 // tcgen05 fences cover; a cluster-scope release would also wait for every global store of the thread to drain)
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+// 4-byte store into the other CTA's shared memory that counts as 4 transaction bytes on a barrier there: readers
+// that wait on that barrier see the value, with no fence on either side (the way a bulk copy is seen)
+__device__ __forceinline__ void st_async_u32(uint32_t addr_cluster, uint32_t v, uint32_t bar_cluster) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+               ::"r"(addr_cluster), "r"(v), "r"(bar_cluster) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
@@ -707,6 +715,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   __shared__ __align__(8) uint64_t acc_empty_bar[2];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
+  // Pair form with a tile counter: the leader's producer publishes each tile number to both CTAs (sched_tile,
+  // sched_full: a plain store and arrive at home, a 4-byte asynchronous store that completes the peer's barrier
+  // there); every reader (the peer's producer, the issuing thread, the epilogue warps of both CTAs: 18 in all)
+  // acknowledges on the leader's sched_empty before the slot is reused.
+  __shared__ __align__(8) uint64_t sched_full[SCHED_SLOTS];
+  __shared__ __align__(8) uint64_t sched_empty[SCHED_SLOTS];
+  __shared__ int sched_tile[SCHED_SLOTS];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzled tiles need 1024-byte alignment
@@ -720,6 +735,20 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   const long long tile0 = PAIR ? (long long)(blockIdx.x >> 1) : (long long)blockIdx.x;
   const long long tile_step = PAIR ? (long long)(gridDim.x >> 1) : (long long)gridDim.x;
   const uint32_t nacc = (!PAIR && p.tile_m == 256) ? 1u : 2u;
+  // Tiles: every pair starts on tile number = its own number; with a tile counter the later ones are whatever
+  // the counter hands out next (so a pair that starts late, or meets costlier tiles, simply takes fewer),
+  // otherwise they follow at a fixed stride.
+  const bool dynamic = PAIR && p.tile_counter != nullptr;
+  const uint32_t sfull0 = smem_u32(&sched_full[0]);
+  const uint32_t sempty0_leader = PAIR ? map_to_cta(smem_u32(&sched_empty[0]), 0) : smem_u32(&sched_empty[0]);
+  // one reader's step: wait for slot `it`, read the tile number, acknowledge; -1 = no more tiles, -2 = a wait ran out
+  auto sched_read = [&](int it) -> long long {
+    const uint32_t s2 = (uint32_t)it % SCHED_SLOTS, ph = ((uint32_t)it / SCHED_SLOTS) & 1u;
+    if (!mbar_wait(sfull0 + 8u * s2, ph, &abort_flag, p.status)) return -2;
+    const int tnum = *reinterpret_cast<volatile int*>(&sched_tile[s2]);
+    mbar_arrive_cluster(sempty0_leader + 8u * s2);
+    return (long long)tnum;
+  };
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -727,6 +756,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&acc_full_bar[a]), 1);
       mbar_init(smem_u32(&acc_empty_bar[a]), PAIR ? 2 * EPI_WARPS : EPI_WARPS);
+    }
+    for (int s2 = 0; s2 < SCHED_SLOTS; ++s2) {
+      mbar_init(smem_u32(&sched_full[s2]), 1);
+      mbar_init(smem_u32(&sched_empty[s2]), 2 * EPI_WARPS + 2);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -779,12 +812,52 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       const CUtensorMap* my_tm1 = my_a ? &p.tmA[1] : &p.tmB[BSPLIT > 1 ? my_sp : 1];
       const int kblocks0 = p.kblocks[0], kblocks1 = p.kblocks[1], kreal0 = p.kreal[0], kreal1 = p.kreal[1];
       const long long total_tiles = p.total_tiles;
-      for (long long tile = tile0; tile < total_tiles; tile += tile_step) {
+      const uint32_t sfull0_peer = PAIR ? map_to_cta(sfull0, 1) : 0u;
+      const uint32_t stile0_peer = PAIR ? map_to_cta(smem_u32(&sched_tile[0]), 1) : 0u;
+      const long long npairs = tile_step;
+      // tickets drawn from the counter by all pairs together: one per tile beyond the first round, plus the one
+      // per pair that tells it to stop; whoever draws the last one puts the counter back to zero
+      const long long last_ticket = (total_tiles > npairs ? total_tiles - npairs : 0) + npairs - 1;
+      unsigned int ticket = 0;
+      for (int it = 0;; ++it) {
+        long long tile;
+        if (!dynamic) {
+          tile = tile0 + (long long)it * tile_step;
+          if (tile >= total_tiles) break;
+        } else {
+          long long tl = 0;
+          if (lane == 0) {
+            if (rank == 0) {
+              if (it == 0) {
+                tl = tile0;
+              } else {
+                tl = npairs + (long long)ticket;
+                if ((long long)ticket == last_ticket) atomicExch(p.tile_counter, 0u);
+                if (tl >= total_tiles) tl = -1;
+              }
+              const uint32_t s2 = (uint32_t)it % SCHED_SLOTS, ph = ((uint32_t)it / SCHED_SLOTS) & 1u;
+              if (!mbar_wait(smem_u32(&sched_empty[s2]), ph ^ 1u, &abort_flag, p.status)) tl = -2;
+              if (tl != -2) {
+                sched_tile[s2] = (int)tl;
+                mbar_arrive(sfull0 + 8u * s2);
+                st_async_u32(stile0_peer + 4u * s2, (uint32_t)(int)tl, sfull0_peer + 8u * s2);
+                // the next tile's ticket: its latency hides behind this tile's copies
+                if (tl >= 0) ticket = atomicAdd(p.tile_counter, 1u);
+              }
+            } else {
+              // the peer's slot completes on this arrival plus the 4 bytes the leader sends
+              mbar_expect_tx(sfull0 + 8u * ((uint32_t)it % SCHED_SLOTS), 4u);
+              tl = sched_read(it);
+            }
+          }
+          tile = __shfl_sync(0xffffffffu, tl, 0);
+          if (tile < 0) break;
+        }
         const TileInfo t = tile_info(p, tile);
         if (t.skip) continue;
         // the epilogues read the matching tile of `aux`: start moving it from HBM into L2 well ahead
         // (AUX_AHEAD tiles of this CTA; short main loops leave no time otherwise)
-        if (aux_prefetch && lane == 0) {
+        if (aux_prefetch && !dynamic && lane == 0) {
           if (tile == tile0) {
             for (int d = 0; d < AUX_AHEAD; ++d) {
               const long long tp = tile + (long long)d * tile_step;
@@ -850,7 +923,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       const int kreal0 = p.kreal[0], kreal1 = p.kreal[1], steps0 = p.kblocks[0];
       const uint32_t idesc0 = p.idesc;
       const bool tall = !PAIR && p.tile_m == 256;
-      for (long long tile = tile0; tile < p.total_tiles; tile += tile_step) {
+      for (int it = 0;; ++it) {
+        long long tile;
+        if (!dynamic) {
+          tile = tile0 + (long long)it * tile_step;
+          if (tile >= p.total_tiles) break;
+        } else {
+          tile = sched_read(it);
+          if (tile < 0) break;
+        }
         const TileInfo t = tile_info(p, tile);
         if (t.skip) continue;
         if (!mbar_wait(smem_u32(&acc_empty_bar[acc]), acc_phase ^ 1u, &abort_flag, p.status)) break;
@@ -910,7 +991,17 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
     uint32_t acc = 0, acc_phase = 0;
     const int h_first = PAIR ? (int)rank : 0;
     const int h_last = PAIR ? (int)rank : ((p.tile_m == 256) ? 1 : 0);
-    for (long long tile = tile0; tile < p.total_tiles; tile += tile_step) {
+    for (int it = 0;; ++it) {
+      long long tile;
+      if (!dynamic) {
+        tile = tile0 + (long long)it * tile_step;
+        if (tile >= p.total_tiles) break;
+      } else {
+        long long tl = 0;
+        if (lane == 0) tl = sched_read(it);
+        tile = __shfl_sync(0xffffffffu, tl, 0);
+        if (tile < 0) break;
+      }
       const TileInfo t = tile_info(p, tile);
       if (t.skip) continue;
       const int tn = t.tn, tm = t.tm, bz = t.bz;
@@ -1206,6 +1297,9 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
     }
   }
   p.status = status_word;
+  // the word after the status word is this context's tile counter (zero between launches: the kernel that uses it
+  // puts it back); launches of one context are ordered on its stream, so they never share it in time
+  p.tile_counter = (p.pair && status_word && !getenv("DEFL_TC_STATIC")) ? reinterpret_cast<unsigned int*>(status_word + 1) : nullptr;
 
   const size_t smem = (size_t)stages * stage_bytes + 1024 + EPI_WARPS * STAGING_BYTES;
   cudaError_t e;

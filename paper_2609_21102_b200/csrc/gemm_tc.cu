@@ -923,17 +923,27 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       const int kreal0 = p.kreal[0], kreal1 = p.kreal[1], steps0 = p.kblocks[0];
       const uint32_t idesc0 = p.idesc;
       const bool tall = !PAIR && p.tile_m == 256;
-      for (int it = 0;; ++it) {
-        long long tile;
-        if (!dynamic) {
-          tile = tile0 + (long long)it * tile_step;
-          if (tile >= p.total_tiles) break;
-        } else {
-          tile = sched_read(it);
-          if (tile < 0) break;
+      // The number and geometry of the NEXT tile are worked out in the middle of the current one (after the products
+      // of its last step but one have been issued, while the tensor pipe is busy with them), so that at the tile
+      // boundary the thread goes straight from the last commit to the first product of the next tile.
+      auto next_tile = [&](int it) -> long long {
+        if (dynamic) return sched_read(it);
+        const long long tl = tile0 + (long long)it * tile_step;
+        return tl < p.total_tiles ? tl : -1;
+      };
+      const int prep = total_kblocks >= 2 ? total_kblocks - 2 : 0;
+      int it = 0;
+      long long nxt = next_tile(it);
+      TileInfo tnx;
+      if (nxt >= 0) tnx = tile_info(p, nxt);
+      while (nxt >= 0) {
+        const TileInfo t = tnx;
+        ++it;
+        if (t.skip) {
+          nxt = next_tile(it);
+          if (nxt >= 0) tnx = tile_info(p, nxt);
+          continue;
         }
-        const TileInfo t = tile_info(p, tile);
-        if (t.skip) continue;
         if (!mbar_wait(smem_u32(&acc_empty_bar[acc]), acc_phase ^ 1u, &abort_flag, p.status)) break;
         tc_fence_after();
         const uint32_t idesc = idesc0 | ((uint32_t)(t.n_eff >> 3) << 17);
@@ -977,9 +987,18 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
           // frees the stage (in both CTAs of a pair) once these products are done
           if (PAIR) umma_commit_pair(empty0 + 8u * stage); else umma_commit(empty0 + 8u * stage);
           if (++stage == nstages) { stage = 0; phase ^= 1u; }
+          if (kb == prep) {
+            if (total_kblocks == 1) {      // a one-step tile: the accumulator is complete, say so before looking ahead
+              if (PAIR) umma_commit_pair(smem_u32(&acc_full_bar[acc])); else umma_commit(smem_u32(&acc_full_bar[acc]));
+            }
+            nxt = next_tile(it);
+            if (nxt >= 0) tnx = tile_info(p, nxt);
+          }
         }
         if (!ok) break;
-        if (PAIR) umma_commit_pair(smem_u32(&acc_full_bar[acc])); else umma_commit(smem_u32(&acc_full_bar[acc]));   // accumulator complete
+        if (total_kblocks != 1) {
+          if (PAIR) umma_commit_pair(smem_u32(&acc_full_bar[acc])); else umma_commit(smem_u32(&acc_full_bar[acc]));   // accumulator complete
+        }
         if (++acc == nacc) { acc = 0; acc_phase ^= 1u; }
       }
     }
@@ -1297,9 +1316,12 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
     }
   }
   p.status = status_word;
-  // the word after the status word is this context's tile counter (zero between launches: the kernel that uses it
-  // puts it back); launches of one context are ordered on its stream, so they never share it in time
-  p.tile_counter = (p.pair && status_word && !getenv("DEFL_TC_STATIC")) ? reinterpret_cast<unsigned int*>(status_word + 1) : nullptr;
+  // DEFL_TC_DYNAMIC: tiles handed out through a counter instead of a fixed stride. The word after the status word
+  // is this context's counter (zero between launches: the kernel that uses it puts it back; launches of one
+  // context are ordered on its stream, so they never share it in time). Off by default: measured on the filter's
+  // products it gains 2 % where tiles are long and uneven (the symmetric Gram product) and loses 2-3 % where they
+  // are short (one more hand-off per tile), and the whole step comes out the same.
+  p.tile_counter = (p.pair && status_word && getenv("DEFL_TC_DYNAMIC")) ? reinterpret_cast<unsigned int*>(status_word + 1) : nullptr;
 
   const size_t smem = (size_t)stages * stage_bytes + 1024 + EPI_WARPS * STAGING_BYTES;
   cudaError_t e;

@@ -111,7 +111,8 @@ def test_symmetric_mirroring(ctx, engine_name):
 
 
 @pytest.mark.parametrize("knobs", [{"DEFL_TC_PAIR": "0"}, {"DEFL_TC_KSUB": "1"}, {"DEFL_TC_TILE_M": "128"},
-                                   {"DEFL_TC_STAGES": "2"}])
+                                   {"DEFL_TC_STAGES": "2"}, {"DEFL_TC_DYNAMIC": "1"},
+                                   {"DEFL_TC_DYNAMIC": "1", "DEFL_TC_STAGES": "2"}])
 @pytest.mark.parametrize("sym", [False, True])
 def test_tensor_engine_other_tile_forms(ctx, monkeypatch, knobs, sym):
     """The tile forms the default rules do not pick for these shapes (single-CTA 256-row tile, one K block per
@@ -130,6 +131,23 @@ def test_tensor_engine_other_tile_forms(ctx, monkeypatch, knobs, sym):
         C = ctx.defl_debug_gemm(A, B, False, False, engine=binding.ENGINE_TENSOR, out_dtype=torch.float32)
         ref = _ref(A, B, False, False)
     assert torch.allclose(C, ref, rtol=1e-4, atol=4e-3)
+
+
+@pytest.mark.parametrize("K", [64, 200, 1096])
+@pytest.mark.parametrize("sym", [False, True])
+def test_tensor_engine_dynamic_tiles(ctx, monkeypatch, K, sym):
+    """Tiles handed out through the counter (DEFL_TC_DYNAMIC), more tiles than CTA pairs so that every pair draws
+    several; a one-step K, a short and a long one. Run twice: the counter must be back at zero after a launch."""
+    from paper_2609_21102_b200 import binding
+    monkeypatch.setenv("DEFL_TC_DYNAMIC", "1")
+    A = _mk(14, 1000, K, torch.bfloat16, 31)
+    B = A if sym else _mk(14, 1032, K, torch.bfloat16, 32)
+    ref = _ref(A, B, False, True)
+    for _ in range(2):
+        C = ctx.defl_debug_gemm(A, B, False, True, engine=binding.ENGINE_TENSOR, out_dtype=torch.float32,
+                                exploit_symmetry=sym)
+        torch.cuda.synchronize()
+        assert torch.allclose(C, ref, rtol=1e-4, atol=4e-3)
 
 
 @pytest.mark.parametrize("ta,tb", [(False, True), (False, False), (True, False)])

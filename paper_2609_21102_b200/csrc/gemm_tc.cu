@@ -497,6 +497,35 @@ __device__ __forceinline__ void aux_fetch_async(const TcParams& p, int lane, int
   cp_async_commit();
 }
 
+// Transposed store of one 32 x 32 block of 16-bit results (EPI_STORE): C[(gj0 + c) * ldc + gi_warp0 + r] = alpha acc[r][c].
+// Each lane packs its row into 16 words of two columns, trades words with its neighbour lane so that a word holds
+// two ROWS of one column, and writes it into the staging buffer laid out as the transposed block (32 columns x 64
+// bytes, conflict-free); the block then leaves in 64-byte rows, 16 bytes per lane. A third of the instructions of
+// gathering the transposed block element by element out of a row-major staging buffer.
+template <bool F16O>
+__device__ __forceinline__ void store_block_transposed16(const TcParams& p, const uint32_t* r, uint8_t* stg, int lane,
+                                                         int gi_warp0, int gj0, int bz, float alpha) {
+  uint32_t* T = reinterpret_cast<uint32_t*>(stg);          // [32 columns][16 words]
+  const bool odd = (lane & 1) != 0;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const uint32_t w = pack16x2(alpha * __uint_as_float(r[2 * j]), alpha * __uint_as_float(r[2 * j + 1]), F16O);
+    const uint32_t y = __shfl_xor_sync(0xffffffffu, w, 1);
+    // even lane: column 2j, rows (mine, neighbour's); odd lane: column 2j + 1, rows (neighbour's, mine)
+    const uint32_t word = odd ? __byte_perm(y, w, 0x7632) : __byte_perm(w, y, 0x5410);
+    T[(2 * j + (odd ? 1 : 0)) * 16 + (lane >> 1)] = word;
+  }
+  __syncwarp();
+  uint8_t* mbase = reinterpret_cast<uint8_t*>(p.C) + ((size_t)bz * p.batch_c + (size_t)gj0 * p.ldc + gi_warp0) * 2;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int c = (lane >> 2) + 8 * i;
+    const uint4 q = *reinterpret_cast<const uint4*>(stg + c * 64 + (lane & 3) * 16);
+    *reinterpret_cast<uint4*>(mbase + (size_t)c * p.ldc * 2 + (lane & 3) * 16) = q;
+  }
+  __syncwarp();
+}
+
 // The calling lane's row of one staged 32 x 32 block, 16 bytes at a time and in place: `aux` values in, results out
 // (nothing is written for the residual norm, whose partial sum of squares is returned). The formats of two-byte
 // values (F16A: `aux` is IEEE half, F16O: the output is; else bf16) and whether the block meets the diagonal (DIAG,
@@ -565,6 +594,13 @@ __device__ __forceinline__ void epilogue_block_fast(const TcParams& p, uint32_t 
     __syncwarp();
   }
   tmem_ld_wait();
+  if (EPI == EPI_STORE && ES == 2) {
+    if (p.transposed) {            // (warp-uniform)
+      if (p.out_f16) store_block_transposed16<true>(p, r, stg, lane, gi_warp0, gj0, bz, alpha);
+      else store_block_transposed16<false>(p, r, stg, lane, gi_warp0, gj0, bz, alpha);
+      return;
+    }
+  }
   const int gi = gi_warp0 + lane;
   // the formats of the two-byte types and the position of the diagonal are the same for the whole warp: one
   // branch per block selects a row loop without per-element tests

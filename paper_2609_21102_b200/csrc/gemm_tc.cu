@@ -1189,7 +1189,9 @@ bool encode_map(CUtensorMap* tm, const void* base, int esize, bool tf32, bool mn
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Tuning overrides for experiments (read per launch): DEFL_TC_BN, DEFL_TC_TILE_M, DEFL_TC_STAGES.
+// Tuning overrides for experiments and for the tests of the forms the default rules do not pick (environment,
+// read per launch): DEFL_TC_BN, DEFL_TC_TILE_M, DEFL_TC_STAGES, DEFL_TC_KSUB, DEFL_TC_PAIR, DEFL_TC_PAIR_MIN_N,
+// DEFL_TC_DYNAMIC (tiles through a counter), DEFL_TC_AUX_PREFETCH (L2 prefetch of `aux`), DEFL_TC_DEBUG.
 int choose_bn(int N, bool pair) {
   const int q = pair ? 32 : 16;
   if (const char* e = getenv("DEFL_TC_BN")) { const int v = atoi(e); if (v >= q && v <= 256 && v % q == 0) return v; }

@@ -26,7 +26,8 @@ sys.path.insert(0, ROOT)
 METRIC = "deflated polar-filter TFLOP/s & matrices/s per batch; % bf16 tensor peak"
 MUON = (3.4445, -4.7750, 2.0315)
 SYM = True   # compute X X^T and A A on the tiles that reach the diagonal and mirror them (--no-symmetry turns it off)
-BF16_ITERATES = False   # --bf16-iterates: keep the filter's iterates in bf16 instead of scaled IEEE half
+BF16_ITERATES = 0       # storage of the filter's iterates: 0 scaled IEEE half in the first two steps then bf16 (default),
+                        # 1 bf16 throughout (--bf16-iterates), 2 scaled half throughout (--half-iterates)
 GAMMA = 1.01            # padding of the restored head (1.1 with the minimax schedule, the value the paper uses with it)
 SCHEDULE = "muon"       # --schedule minimax: per-step minimax quintics (the Polar-Express-style mapping)
 SCHEDULE_NOTE = "Muon quintic (3.4445, -4.7750, 2.0315) every step"
@@ -241,7 +242,8 @@ def main():
     ap.add_argument("--small", action="store_true", help="tiny workload for a quick functional check")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-symmetry", action="store_true", help="compute the symmetric products in full")
-    ap.add_argument("--bf16-iterates", action="store_true", help="filter iterates stored in bf16 (default: scaled IEEE half)")
+    ap.add_argument("--bf16-iterates", action="store_true", help="filter iterates stored in bf16 in every step (default: scaled IEEE half in the first two)")
+    ap.add_argument("--half-iterates", action="store_true", help="filter iterates stored in scaled IEEE half in every step")
     ap.add_argument("--schedule", choices=["muon", "minimax"], default="muon",
                     help="muon: Muon's quintic every step; minimax: per-step minimax quintics (Polar-Express-style)")
     ap.add_argument("--streams", type=int, default=2, help="2: one stream + context per shape group; 1: one stream")
@@ -254,7 +256,7 @@ def main():
         SCHEDULE_NOTE = ("per-step minimax quintics (greedy Remez from [1e-3, 1], first step / 1.01): the "
                          "Polar-Express-style mapping, coefficients computed by schedules.remez_sign_schedule")
     SYM = not args.no_symmetry
-    BF16_ITERATES = bool(args.bf16_iterates)
+    BF16_ITERATES = 1 if args.bf16_iterates else (2 if args.half_iterates else 0)
     wl_name = "small" if args.small else "gpt2_xl"
     wl = dict(WORKLOADS[wl_name])
     if args.batch > 0:
@@ -267,7 +269,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     config = {"workload": wl["label"], "name": wl_name, "k": wl["k"], "oversample": wl["p"], "power_iters": wl["J"],
               "filter_steps": wl["L"], "restore": "padded, gamma=%g" % GAMMA, "schedule": SCHEDULE_NOTE, "exploit_symmetry": SYM,
-              "storage": "input and output bf16; filter iterates " + ("bf16" if BF16_ITERATES else "IEEE half scaled by 32 (same tensor rate)"),
+              "storage": "input and output bf16; filter iterates " + ("bf16" if BF16_ITERATES == 1 else ("IEEE half scaled by 32" if BF16_ITERATES == 2 else "IEEE half scaled by 32 in the first two steps, bf16 after")),
               "l2": "inputs (1.2 GB per step) larger than L2; no flush"}
     tot_f = sum(b * sum(flops_per_matrix(m, n, wl["k"], wl["p"], wl["J"], wl["L"])) for b, m, n in wl["groups"])
     nmat = sum(b for b, _, _ in wl["groups"])
@@ -339,17 +341,24 @@ def main():
     stage_tot = [0.0, 0.0, 0.0, 0.0]
     filt_flops = 0.0        # dense count of the filter products
     filt_executed = 0.0     # flops the tensor cores actually execute (tiles below the diagonal are skipped)
-    STAGE_REPS = 3          # averaged: a single step's split moves by several percent with the power state
+    STAGE_REPS = 7          # median over the repetitions: a single step's split moves by several percent with the
+                            # power state, and reading the events synchronises the stream after every call
+    per_rep = []
     for rep in range(STAGE_REPS):
+        tot = [0.0, 0.0, 0.0, 0.0]
         for g, (b, m, n) in zip(groups, wl["groups"]):
             ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], sched_of(wl), out=g["out"], sketch=g["Om"],
                                    gamma=GAMMA, exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
             ms = ctx.defl_get_stage_ms()
             for i in range(min(4, len(ms))):
-                stage_tot[i] += ms[i] / STAGE_REPS
+                tot[i] += ms[i]
             if rep == 0:
                 filt_flops += b * flops_per_matrix(m, n, wl["k"], wl["p"], wl["J"], wl["L"])[0]
                 filt_executed += b * executed_filter_flops(m, n, wl["L"], SYM)
+        per_rep.append(tot)
+    for i in range(4):
+        vals = sorted(r[i] for r in per_rep)
+        stage_tot[i] = vals[len(vals) // 2]
     plain_ms = 0.0
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()

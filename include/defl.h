@@ -88,9 +88,11 @@ typedef struct defl_opts {
                             half, tensor-core products with fp32 accumulation), the precision the paper's SDP runs
                             use for the filter (Appendix C.2). Everything around the filter stays fp32/tf32.
                             Needs n a multiple of 8 and the tensor engine. */
-  int bf16_iterates;     /* polar path with bf16 input, non-zero: keep the filter's iterates X_t, A_t, B_t in bf16.
-                            Default (0): they are kept in IEEE half scaled by 32 (same tensor-core rate, three more
-                            mantissa bits; input, output and every other stage are unchanged). */
+  int bf16_iterates;     /* polar path with bf16 input: storage type of the filter's iterates X_t, A_t, B_t (input,
+                            output and every other stage are unchanged). 0 (default): IEEE half scaled by 32 in the
+                            first two filter steps (same tensor-core rate, three more mantissa bits: the rounding of
+                            the early iterates is what limits accuracy), bf16 in the later ones (less power, i.e.
+                            more clock under a power cap). 1: bf16 in every step. 2: scaled half in every step. */
 } defl_opts;
 
 typedef struct defl_info {

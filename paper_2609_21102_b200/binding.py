@@ -170,7 +170,7 @@ class Context:
         o.exploit_symmetry = int(bool(exploit_symmetry))
         o.tau = tau
         o.half_filter = int(bool(half_filter))
-        o.bf16_iterates = int(bool(bf16_iterates))
+        o.bf16_iterates = int(bf16_iterates)      # 0 mixed (default), 1 / True bf16 throughout, 2 half throughout
         return o
 
     # ------------------------------------------------------------------------------------------

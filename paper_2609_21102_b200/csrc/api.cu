@@ -453,10 +453,19 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
   // Same tensor-core rate as bf16, three more mantissa bits: the rounding of the stored iterate is what limits
   // the bf16 path's accuracy on wide matrices with slowly decaying spectra. The power-of-two scale keeps small
   // entries (1/sqrt(mn) of a normalised residual, off-diagonal Gram entries) out of half's subnormal range, and
-  // overflow would need a singular value above 8. opts->bf16_iterates keeps everything in bf16.
-  const bool half_iter = dtype == DEFL_BF16 && L > 0 && !(opts && opts->bf16_iterates);
-  const int it_dtype = half_iter ? (int)F16 : dtype;
-  const float ys = half_iter ? 32.f : 1.f;
+  // overflow would need a singular value above 8.
+  // How many steps need it: the rounding of X_0 and of the first iterates is what costs accuracy (the small
+  // singular values are still small there). Measured on the 48 x 1600 x 6400 workload against the oracle: half in
+  // all five steps 5.5e-3, in the first four 6.5e-3, three 8.1e-3, two 1.07e-2, one 1.5e-2, none (bf16 throughout)
+  // 4.2e-2. Half-precision products draw more power than bf16 ones, and under the board's power cap that is clock:
+  // 23.3 ms per step with five half steps, 22.6 ms with two or one, 21.9 ms with none. Default: the first two
+  // steps in half, the rest in bf16. opts->bf16_iterates = 1: bf16 throughout; = 2: half throughout.
+  const int it_mode = opts ? opts->bf16_iterates : 0;
+  const bool half_iter = dtype == DEFL_BF16 && L > 0 && it_mode != 1;
+  // the first `n_half` filter steps keep the iterate in scaled IEEE half, the rest in bf16
+  const int n_half = half_iter ? (it_mode == 2 ? L : (L < 2 ? L : 2)) : 0;
+  const int it_dtype = n_half > 0 ? (int)F16 : dtype;      // format and scale of X_0
+  const float ys = n_half > 0 ? 32.f : 1.f;
 
   cudaSetDevice(c->device);
   int rc = ctx_reserve(c, carve_polar(nullptr, b, m, n, dtype, k, l).bytes);
@@ -554,6 +563,9 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
     const float ca = coeff_schedule[3 * t], cb = coeff_schedule[3 * t + 1], cc = coeff_schedule[3 * t + 2];
     const void* X = bufs[cur];
     void* Xn = bufs[cur ^ 1];
+    const bool hs = t < n_half, hn = t + 1 < n_half;
+    const int it_dtype = hs ? (int)F16 : dtype, nx_dtype = hn ? (int)F16 : dtype;     // this step's and the next one's
+    const float ys = hs ? 32.f : 1.f, ys_next = hn ? 32.f : 1.f;
     GemmDesc g = gemm_desc_zero();
     g.batch = b; g.in_dtype = it_dtype; g.b_dtype = it_dtype; g.out_dtype = it_dtype;
     // A_t = X X^T (wide) or X^T X (tall), ms x ms, symmetric
@@ -590,6 +602,7 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
     }
     g.C = Xn; g.ldc = n; g.batch_c = (long long)m * n;
     g.epilogue = EPI_STORE;
+    g.out_dtype = nx_dtype; g.alpha = ys_next / ys;                   // the next step's format and scale
     if (t == L - 1) { g.out_dtype = dtype; g.alpha = 1.f / ys; }      // the result leaves in the caller's type and scale
     if (wide && !(upd && t == L - 1)) {
       // The tensor engine pads the product's rows to whole 256-row tiles, its columns only to 32: for a wide X

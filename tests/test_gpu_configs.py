@@ -72,20 +72,22 @@ def test_workload3_power_law_per_step_schedule(ctx, shape_index, n):
     _check_samples(ctx, G, Om, 16, 8, 1, _minimax_schedule(), 1.1, [23], 1e-2)
 
 
-# With the filter's iterates in bf16 (opts->bf16_iterates) the 1600 x 6400 group of workload 4 sits at 4.2e-2
-# against the fp64 oracle, not 3e-2. The cause is the bf16 storage of the iterate X_t alone: the figure is the same
-# to four digits on the exact-fp32-product engine, with A_t and B_t held in fp32, and it drops to 1e-5 with fp32
-# storage (measured). Rounding X_t (relative 2^-9 per entry) tilts each small singular direction by about
-# 1e-3 * ||X_t||_F / (sqrt(m) sigma_i), which this spectrum (sigma_i = 200/i, floor 3.6e-3 after deflation) and the
-# 4:1 aspect make large. The default keeps the iterates in IEEE half scaled by 32 (three more mantissa bits, same
-# tensor-core rate): 5.5e-3 on this group, 3.9e-3 on the square one, against 1.7e-3 for the bf16 rounding of the
-# exact result alone. The bf16-iterate option is still checked, at the looser bound.
+# Storage of the filter's iterates on workload 4 (error against the fp64 oracle, 1600 x 6400 group / square group):
+# bf16 in every step 4.2e-2 / 2.8e-2; scaled IEEE half in the first step only 1.5e-2 / 1.1e-2; in the first two
+# (the default) 1.07e-2 / 8.2e-3; in all five 5.5e-3 / 3.9e-3; the bf16 rounding of the exact result alone is 1.7e-3.
+# The cause is the storage rounding of X_t alone: the bf16 figure is the same to four digits on the
+# exact-fp32-product engine with A_t and B_t held in fp32, and it drops to 1e-5 with fp32 storage (measured).
+# Rounding X_t (relative 2^-9 per entry in bf16) tilts each small singular direction by about
+# 1e-3 * ||X_t||_F / (sqrt(m) sigma_i), large for this spectrum (sigma_i = 200/i, floor 3.6e-3 after deflation) and
+# the 4:1 aspect while sigma_i is still small, i.e. in the first steps: later steps can afford bf16.
+TOL_DEFAULT_XL = 1.5e-2              # two half steps, then bf16 (spec tolerance for the bf16 path: 3e-2)
+TOL_HALF_ITERATES_XL = 1e-2
 TOL_BF16_ITERATES_XL_WIDE = 5e-2
 
 
 def test_workload4_gpt2_xl_both_groups(ctx):
     dev = torch.device("cuda")
-    for shape_index, (m, n), samples, tol in ((1, (1600, 1600), [0, 47], 1e-2), (0, (1600, 6400), [5], 1e-2)):
+    for shape_index, (m, n), samples, tol in ((1, (1600, 1600), [0, 47], TOL_DEFAULT_XL), (0, (1600, 6400), [5], TOL_DEFAULT_XL)):
         G = inputs.workload_power_law(48, m, n, 4, shape_index, 1.0, 200.0, 1e-4, device=dev).to(torch.bfloat16)
         Om = inputs.sketch(48, 1600, 48, 4, shape_index, device=dev)
         _check_samples(ctx, G, Om, 32, 16, 2, [MUON] * 5, 1.01, samples, tol)
@@ -98,9 +100,13 @@ def test_workload4_gpt2_xl_both_groups(ctx):
                                             oracle.schedule([MUON] * 5), gamma=1.01)
             assert _rel(out32[2].double().cpu().numpy(), ref) <= 2e-3
             outb = ctx.defl_polar_batched(G[:4].contiguous(), 32, 16, 2, [MUON] * 5, sketch=Om[:4].contiguous(), gamma=1.01,
-                                          exploit_symmetry=True, bf16_iterates=True)
+                                          exploit_symmetry=True, bf16_iterates=1)
             eb = _rel(outb[2].double().cpu().numpy(), ref)
-            assert 1e-2 < eb <= TOL_BF16_ITERATES_XL_WIDE, eb       # the option does switch the storage type
+            assert 2e-2 < eb <= TOL_BF16_ITERATES_XL_WIDE, eb       # the option does switch the storage type
+            outh = ctx.defl_polar_batched(G[:4].contiguous(), 32, 16, 2, [MUON] * 5, sketch=Om[:4].contiguous(), gamma=1.01,
+                                          exploit_symmetry=True, bf16_iterates=2)
+            eh = _rel(outh[2].double().cpu().numpy(), ref)
+            assert eh <= TOL_HALF_ITERATES_XL, eh
         del G, Om
         torch.cuda.empty_cache()
 
@@ -109,7 +115,7 @@ def test_workload4_add_mode_and_tall_orientation(ctx):
     dev = torch.device("cuda")
     G = inputs.workload_power_law(4, 6400, 1600, 4, 0, 1.0, 200.0, 1e-4, device=dev).to(torch.bfloat16)
     Om = inputs.sketch(4, 1600, 48, 4, 0, device=dev)
-    _check_samples(ctx, G, Om, 32, 16, 2, [MUON] * 5, 1.01, [3], 1e-2, mode=1)
+    _check_samples(ctx, G, Om, 32, 16, 2, [MUON] * 5, 1.01, [3], TOL_DEFAULT_XL, mode=1)
 
 
 def test_workload5_sdp_sequence(ctx):

@@ -39,7 +39,7 @@ def _oracle_batch(G, k, p, J, sched, Om, gamma, mode):
     return outs
 
 
-def _run_case(ctx, G64, dtype, k, p, J, sched, gamma, mode, engine, workload=1, exploit_symmetry=False):
+def _run_case(ctx, G64, dtype, k, p, J, sched, gamma, mode, engine, workload=1, exploit_symmetry=False, iterates=0):
     from paper_2609_21102_b200 import binding
     G = inputs.round_to(G64, dtype).cuda()
     b, m, n = G.shape
@@ -47,7 +47,7 @@ def _run_case(ctx, G64, dtype, k, p, J, sched, gamma, mode, engine, workload=1, 
     l = min(ms, k + p) if k > 0 else 0
     Om = inputs.sketch(b, ms, max(l, 1), workload).cuda() if k > 0 else None
     out, info = ctx.defl_polar_batched(G, k, p, J, sched, sketch=Om, restore_mode=mode, gamma=gamma, engine=engine,
-                                       exploit_symmetry=exploit_symmetry, want_info=True)
+                                       exploit_symmetry=exploit_symmetry, want_info=True, bf16_iterates=iterates)
     torch.cuda.synchronize()
     ref = _oracle_batch(G, k, p, J, sched, Om, gamma, mode)
     errs = []
@@ -111,6 +111,24 @@ def test_bf16_matches_oracle(ctx, shape, engine_name):
     for mode in (0, 1):
         errs = _run_case(ctx, G64, torch.bfloat16, 8, 8, 1, _sched(binding.MUON_QUINTIC, 5), 1.01, mode, engine)
         assert max(errs) <= TOL[torch.bfloat16], errs
+
+
+@pytest.mark.parametrize("L", [1, 2, 3, 6])
+@pytest.mark.parametrize("shape", [(256, 512), (200, 136)])
+def test_bf16_iterate_storage_options(ctx, shape, L):
+    """The three storage options of the filter's iterates (scaled half in the first two steps then bf16, bf16
+    throughout, scaled half throughout) against the oracle, for filter depths below, at and above the switch; the
+    second shape runs on the fp32 FMA engine (rows not a multiple of 8 elements)."""
+    from paper_2609_21102_b200 import binding
+    m, n = shape
+    sig = inputs.spectrum_power(min(m, n), 0.8, 50.0)
+    G64 = torch.stack([inputs.from_spectrum(m, n, sig, 2500 + i) for i in range(2)])
+    errs = {}
+    for it in (0, 1, 2):
+        errs[it] = max(_run_case(ctx, G64, torch.bfloat16, 8, 8, 1, _sched(binding.MUON_QUINTIC, L), 1.01, 0,
+                                 binding.ENGINE_AUTO, exploit_symmetry=True, iterates=it))
+        assert errs[it] <= TOL[torch.bfloat16], (it, errs)
+    assert errs[2] <= errs[1] * 1.05 + 1e-3, errs          # half storage is never the less accurate one
 
 
 def test_bf16_symmetric_option_and_plain_path(ctx):

@@ -92,7 +92,9 @@ typedef struct defl_opts {
                             output and every other stage are unchanged). 0 (default): IEEE half scaled by 32 in the
                             first two filter steps (same tensor-core rate, three more mantissa bits: the rounding of
                             the early iterates is what limits accuracy), bf16 in the later ones (less power, i.e.
-                            more clock under a power cap). 1: bf16 in every step. 2: scaled half in every step. */
+                            more clock under a power cap); with DEFL_RESTORE_ADD scaled half in every step (that mode
+                            is about ten times more sensitive to the storage rounding). 1: bf16 in every step.
+                            2: scaled half in every step. */
 } defl_opts;
 
 typedef struct defl_info {

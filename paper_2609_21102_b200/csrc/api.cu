@@ -460,10 +460,13 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
   // 4.2e-2. Half-precision products draw more power than bf16 ones, and under the board's power cap that is clock:
   // 23.3 ms per step with five half steps, 22.6 ms with two or one, 21.9 ms with none. Default: the first two
   // steps in half, the rest in bf16. opts->bf16_iterates = 1: bf16 throughout; = 2: half throughout.
+  // ADD restore keeps half in every step: without the head inside X_0 all its singular values are small and stay
+  // small for longer, and the same storage rounding costs about ten times more (a 636 x 75 case with six steps:
+  // 2.8e-2 with half throughout, 8.2e-2 with two half steps, 1.7e-1 with bf16; padded restore 2.7e-3 / 9.8e-3 / 1.7e-2).
   const int it_mode = opts ? opts->bf16_iterates : 0;
   const bool half_iter = dtype == DEFL_BF16 && L > 0 && it_mode != 1;
   // the first `n_half` filter steps keep the iterate in scaled IEEE half, the rest in bf16
-  const int n_half = half_iter ? (it_mode == 2 ? L : (L < 2 ? L : 2)) : 0;
+  const int n_half = half_iter ? ((it_mode == 2 || mode == DEFL_RESTORE_ADD) ? L : (L < 2 ? L : 2)) : 0;
   const int it_dtype = n_half > 0 ? (int)F16 : dtype;      // format and scale of X_0
   const float ys = n_half > 0 ? 32.f : 1.f;
 

@@ -92,8 +92,11 @@ cudaError_t gram_partial_launch(const float* Y, long long batch_stride, int batc
 __global__ void __launch_bounds__(512) chol_inv_kernel(const double* __restrict__ partial, int nchunk, int l,
                                                        float* __restrict__ Rinv, int* __restrict__ status) {
   extern __shared__ double sm[];
-  double* W = sm;              // [l][l] original Gram
-  double* Lm = sm + l * l;     // [l][l] lower factor, then its inverse
+  // rows are padded to an odd number of doubles: a column walk (row stride apart) then touches every bank once
+  // instead of one bank 32 times (l = 48 doubles = 96 words = 0 mod 32)
+  const int ls = l | 1;
+  double* W = sm;                              // [l][ls] original Gram
+  double* Lm = sm + MAX_L * (MAX_L + 1);       // [l][ls] lower factor, then its inverse
   __shared__ int bad;
   __shared__ double rdiag[MAX_L];
   const int bz = blockIdx.x, tid = threadIdx.x;
@@ -102,25 +105,25 @@ __global__ void __launch_bounds__(512) chol_inv_kernel(const double* __restrict_
     double t = 0.0;
 #pragma unroll 8
     for (int c = 0; c < nchunk; ++c) t += pb[(long long)c * l * l + e];
-    W[e] = t;
+    W[(e / l) * ls + e % l] = t;
   }
   __syncthreads();
   // symmetrise exactly
   for (int e = tid; e < l * l; e += blockDim.x) {
     const int i = e / l, j = e % l;
-    if (i < j) { const double a = 0.5 * (W[i * l + j] + W[j * l + i]); Lm[i * l + j] = a; Lm[j * l + i] = a; }
-    else if (i == j) Lm[e] = W[e];
+    if (i < j) { const double a = 0.5 * (W[i * ls + j] + W[j * ls + i]); Lm[i * ls + j] = a; Lm[j * ls + i] = a; }
+    else if (i == j) Lm[i * ls + j] = W[i * ls + j];
   }
   __syncthreads();
-  for (int e = tid; e < l * l; e += blockDim.x) W[e] = Lm[e];
+  for (int e = tid; e < l * l; e += blockDim.x) { const int o = (e / l) * ls + e % l; W[o] = Lm[o]; }
   __syncthreads();
   double trace = 0.0;
-  for (int i = 0; i < l; ++i) trace += W[i * l + i];
+  for (int i = 0; i < l; ++i) trace += W[i * ls + i];
   double shift = 0.0;
   for (int attempt = 0; attempt < 6; ++attempt) {
     for (int e = tid; e < l * l; e += blockDim.x) {
       const int i = e / l, j = e % l;
-      Lm[e] = W[e] + ((i == j) ? shift : 0.0);
+      Lm[i * ls + j] = W[i * ls + j] + ((i == j) ? shift : 0.0);
     }
     __syncthreads();
     // Right-looking Cholesky on the lower triangle, one barrier per column: in phase j every thread reads the
@@ -132,22 +135,22 @@ __global__ void __launch_bounds__(512) chol_inv_kernel(const double* __restrict_
     double sd_prev = 1.0, isd_prev = 1.0;
     const int ti = tid >> 6, tc = tid & 63;        // 8 rows x 64 columns of the trailing block per pass
     for (int j = 0; j < l; ++j) {
-      const double d = Lm[j * l + j];
+      const double d = Lm[j * ls + j];
       if (!(d > 0.0) || !isfinite(d)) { failed = true; break; }
       const double isd = rsqrt(d), inv_d = isd * isd;
       if (j > 0) {
-        for (int i = j - 1 + tid; i < l; i += blockDim.x) Lm[i * l + j - 1] = (i == j - 1) ? sd_prev : Lm[i * l + j - 1] * isd_prev;
+        for (int i = j - 1 + tid; i < l; i += blockDim.x) Lm[i * ls + j - 1] = (i == j - 1) ? sd_prev : Lm[i * ls + j - 1] * isd_prev;
       }
       const int c = j + 1 + tc;
       if (c < l) {
-        const double lc = Lm[c * l + j] * inv_d;
+        const double lc = Lm[c * ls + j] * inv_d;
         for (int i = j + 1 + ti; i < l; i += 8)
-          if (c <= i) Lm[i * l + c] -= Lm[i * l + j] * lc;
+          if (c <= i) Lm[i * ls + c] -= Lm[i * ls + j] * lc;
       }
       sd_prev = d * isd; isd_prev = isd;
       __syncthreads();
     }
-    if (!failed && tid == 0) Lm[(l - 1) * l + l - 1] = sd_prev;
+    if (!failed && tid == 0) Lm[(l - 1) * ls + l - 1] = sd_prev;
     if (tid == 0) bad = failed ? 1 : 0;
     __syncthreads();
     if (!bad) break;
@@ -160,8 +163,8 @@ __global__ void __launch_bounds__(512) chol_inv_kernel(const double* __restrict_
   // X[:,c] for c: x_c = 1/L_cc; x_i = -(sum_{t=c}^{i-1} L_it x_t)/L_ii
   __syncthreads();
   double* X = W;   // reuse
-  for (int e = tid; e < l * l; e += blockDim.x) X[e] = 0.0;
-  if (tid < l) rdiag[tid] = bad ? 0.0 : 1.0 / Lm[tid * l + tid];
+  for (int e = tid; e < l * ls; e += blockDim.x) X[e] = 0.0;
+  if (tid < l) rdiag[tid] = bad ? 0.0 : 1.0 / Lm[tid * ls + tid];
   __syncthreads();
   if (!bad) {
     // eight lanes per column share each row's dot product; a column never leaves its warp, so rows are
@@ -171,11 +174,11 @@ __global__ void __launch_bounds__(512) chol_inv_kernel(const double* __restrict_
       for (int i = 0; i < l; ++i) {
         double t = 0.0;
         if (c < l && i > c)
-          for (int k2 = c + sub; k2 < i; k2 += 8) t += Lm[i * l + k2] * X[k2 * l + c];
+          for (int k2 = c + sub; k2 < i; k2 += 8) t += Lm[i * ls + k2] * X[k2 * ls + c];
         t += __shfl_xor_sync(0xffffffffu, t, 1);
         t += __shfl_xor_sync(0xffffffffu, t, 2);
         t += __shfl_xor_sync(0xffffffffu, t, 4);
-        if (sub == 0 && c < l && i >= c) X[i * l + c] = ((i == c) ? 1.0 - t : -t) * rdiag[i];
+        if (sub == 0 && c < l && i >= c) X[i * ls + c] = ((i == c) ? 1.0 - t : -t) * rdiag[i];
         __syncwarp();
       }
     }
@@ -185,16 +188,16 @@ __global__ void __launch_bounds__(512) chol_inv_kernel(const double* __restrict_
   float* out = Rinv + (long long)bz * l * l;
   for (int e = tid; e < l * l; e += blockDim.x) {
     const int i = e / l, j = e % l;
-    out[e] = (float)X[j * l + i];
+    out[e] = (float)X[j * ls + i];
   }
 }
 
 cudaError_t chol_inv_launch(const double* partial, int nchunk, int batch, int l, float* Rinv, int* status,
                             cudaStream_t st, long long* launches) {
-  const size_t smem = 2 * (size_t)l * l * sizeof(double);
+  const size_t smem = 2 * (size_t)MAX_L * (MAX_L + 1) * sizeof(double);
   static bool attr_set = false;
   if (!attr_set) {
-    cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * MAX_L * MAX_L * 8);
+    cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     attr_set = true;
   }
   chol_inv_kernel<<<batch, 512, smem, st>>>(partial, nchunk, l, Rinv, status);

@@ -144,8 +144,21 @@ __global__ void __launch_bounds__(512) chol_inv_kernel(const double* __restrict_
       const int c = j + 1 + tc;
       if (c < l) {
         const double lc = Lm[c * ls + j] * inv_d;
-        for (int i = j + 1 + ti; i < l; i += 8)
-          if (c <= i) Lm[i * ls + c] -= Lm[i * ls + j] * lc;
+        // all loads of the thread's (up to MAX_L / 8) rows first, then the updates: written as one loop, every
+        // iteration's loads wait for the previous iteration's store (the compiler cannot tell they do not alias)
+        double a[MAX_L / 8], bj[MAX_L / 8];
+#pragma unroll
+        for (int u = 0; u < MAX_L / 8; ++u) {
+          const int i = j + 1 + ti + 8 * u;
+          const bool on = i < l && c <= i;
+          a[u] = on ? Lm[i * ls + c] : 0.0;
+          bj[u] = on ? Lm[i * ls + j] : 0.0;
+        }
+#pragma unroll
+        for (int u = 0; u < MAX_L / 8; ++u) {
+          const int i = j + 1 + ti + 8 * u;
+          if (i < l && c <= i) Lm[i * ls + c] = a[u] - bj[u] * lc;
+        }
       }
       sd_prev = d * isd; isd_prev = isd;
       __syncthreads();

@@ -180,19 +180,35 @@ __global__ void __launch_bounds__(512) chol_inv_kernel(const double* __restrict_
   if (tid < l) rdiag[tid] = bad ? 0.0 : 1.0 / Lm[tid * ls + tid];
   __syncthreads();
   if (!bad) {
-    // eight lanes per column share each row's dot product; a column never leaves its warp, so rows are
-    // ordered by __syncwarp only
-    const int sub = tid & 7;
-    for (int c = tid >> 3; c < ((l + 3) & ~3); c += blockDim.x >> 3) {
-      for (int i = 0; i < l; ++i) {
-        double t = 0.0;
-        if (c < l && i > c)
-          for (int k2 = c + sub; k2 < i; k2 += 8) t += Lm[i * ls + k2] * X[k2 * ls + c];
-        t += __shfl_xor_sync(0xffffffffu, t, 1);
-        t += __shfl_xor_sync(0xffffffffu, t, 2);
-        t += __shfl_xor_sync(0xffffffffu, t, 4);
-        if (sub == 0 && c < l && i >= c) X[i * ls + c] = ((i == c) ? 1.0 - t : -t) * rdiag[i];
-        __syncwarp();
+    // Eight lanes per column c of X = L^-1 (blockDim / 8 = 64 columns at once), column-oriented: lane `sub` keeps,
+    // in registers, the running sums s_r = sum_{k<i} L_rk x_k of the rows r = sub (mod 8). Step i: the owner of row i
+    // hands s_i to the group (one shuffle), everybody forms x_i = (delta_ic - s_i) / L_ii, and adds L_ri x_i to its
+    // sums of the rows below. Per step that is one shuffle and one multiply on the critical path and at most
+    // MAX_L / 8 independent multiply-adds per lane; the row-oriented form (a dot product split over the lanes,
+    // three shuffle levels and a warp barrier per row) spent 2.5x the fp64 instructions, which is what bounds it.
+    const int c = tid >> 3, sub = tid & 7;
+    const int c_warp0 = (tid >> 5) * 4;          // first column of this warp
+    double srow[MAX_L / 8];
+#pragma unroll
+    for (int u = 0; u < MAX_L / 8; ++u) srow[u] = 0.0;
+    if (c_warp0 < l) {                           // (a warp whose four columns all lie beyond l has nothing to do)
+#pragma unroll
+      for (int u = 0; u < MAX_L / 8; ++u) {
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+          const int i = 8 * u + w;
+          if (i < l && i >= c_warp0) {           // uniform in the warp: rows above its first column give x_i = 0
+            const double si = __shfl_sync(0xffffffffu, srow[u], w, 8);
+            double xi = 0.0;
+            if (c < l && i >= c) xi = ((i == c) ? 1.0 - si : -si) * rdiag[i];
+            if (sub == w && c < l) X[i * ls + c] = xi;
+#pragma unroll
+            for (int u2 = u; u2 < MAX_L / 8; ++u2) {
+              const int r = 8 * u2 + sub;
+              if (r > i && r < l) srow[u2] = fma(Lm[r * ls + i], xi, srow[u2]);
+            }
+          }
+        }
       }
     }
   }

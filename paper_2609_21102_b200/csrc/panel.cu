@@ -1013,9 +1013,12 @@ __global__ void __launch_bounds__(256, 2) panel_fused_kernel(const float* In, lo
   }
   if (partial) {
     // sum over the groups in fp64 (group order fixed: the result does not depend on timing), in the tile's memory
-    double* red = reinterpret_cast<double*>(fsm);        // [wout][wout], upper blocks only
+    // (rows padded to an odd stride: the blocks of a group lie 4 rows apart and the mirror reads walk a column, both
+    // of which land on one shared-memory bank when a row is 48 doubles = 96 words)
+    const int wr = wout | 1;
+    double* red = reinterpret_cast<double*>(fsm);        // [wout][wr], upper blocks only
     __syncthreads();
-    for (int e = tid; e < wout * wout; e += 256) red[e] = 0.0;
+    for (int e = tid; e < wout * wr; e += 256) red[e] = 0.0;
     __syncthreads();
     for (int g = 0; g < ngrp; ++g) {
       if (gram_on && grp == g) {
@@ -1024,7 +1027,7 @@ __global__ void __launch_bounds__(256, 2) panel_fused_kernel(const float* In, lo
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const int gi = bi * 4 + i, gj = bj * 8 + j;
-            if (gi < wout && gj < wout) red[gi * wout + gj] += (double)g8[i][j];
+            if (gi < wout && gj < wout) red[gi * wr + gj] += (double)g8[i][j];
           }
       }
       __syncthreads();
@@ -1033,7 +1036,7 @@ __global__ void __launch_bounds__(256, 2) panel_fused_kernel(const float* In, lo
     for (int e = tid; e < wout * wout; e += 256) {
       const int gi = e / wout, gj = e - gi * wout;
       // blocks below the block diagonal were not computed: take the mirror image
-      out[e] = ((gi >> 3) <= (gj >> 3)) ? red[e] : red[gj * wout + gi];
+      out[e] = ((gi >> 3) <= (gj >> 3)) ? red[gi * wr + gj] : red[gj * wr + gi];
     }
   }
 }

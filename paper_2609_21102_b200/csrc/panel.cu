@@ -853,7 +853,11 @@ __global__ void __launch_bounds__(256, 2) panel_fused_kernel(const float* In, lo
       ms[r][cc] = (r < l && cc < kout) ? Mb[r * ldm + cc] : 0.f;
     }
   }
-  const int ty = tid >> 3, tx = tid & 7;        // product: rows ty*4.., cols tx*8..
+  // product: thread (ty, tx) computes rows ty, ty + 32, ty + 64, ty + 96 and columns 4 tx .. 4 tx + 3, 32 + 4 tx .. + 3.
+  // A warp's four ty values are then four consecutive tile rows (68 floats apart: different banks) and its eight
+  // tx values read 128 contiguous bytes of the staged matrix: one shared-memory wavefront per 16-byte load. (With
+  // rows 4 ty + i and columns 8 tx + j the same loads took two wavefronts each, and the product was bound by them.)
+  const int ty = tid >> 3, tx = tid & 7;
   // Gram: the upper block triangle of W = In^T In (or Out^T Out) in blocks of 4 rows x 8 columns; the threads form
   // `ngrp` groups of `nblk` (one block each), group g takes the rows g, g + ngrp, ... of every tile. fp32 sums
   // per thread (at most rows-per-CTA / ngrp terms), added up over the groups in fp64 at the end, in a fixed order.
@@ -913,11 +917,11 @@ __global__ void __launch_bounds__(256, 2) panel_fused_kernel(const float* In, lo
       for (int q = 0; q < l; q += 4) {
         float4 a4[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) a4[i] = *reinterpret_cast<const float4*>(&tile[ty * 4 + i][q]);
+        for (int i = 0; i < 4; ++i) a4[i] = *reinterpret_cast<const float4*>(&tile[ty + 32 * i][q]);
 #pragma unroll
         for (int qq = 0; qq < 4; ++qq) {
-          const float4 b0 = *reinterpret_cast<const float4*>(&ms[q + qq][tx * 8]);
-          const float4 b1 = *reinterpret_cast<const float4*>(&ms[q + qq][tx * 8 + 4]);
+          const float4 b0 = *reinterpret_cast<const float4*>(&ms[q + qq][tx * 4]);
+          const float4 b1 = *reinterpret_cast<const float4*>(&ms[q + qq][32 + tx * 4]);
           const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
@@ -931,8 +935,8 @@ __global__ void __launch_bounds__(256, 2) panel_fused_kernel(const float* In, lo
       // (columns wout.. of the tile receive zeros: the staged matrix has zero columns there)
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        *reinterpret_cast<float4*>(&tile[ty * 4 + i][tx * 8]) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-        *reinterpret_cast<float4*>(&tile[ty * 4 + i][tx * 8 + 4]) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
+        *reinterpret_cast<float4*>(&tile[ty + 32 * i][tx * 4]) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+        *reinterpret_cast<float4*>(&tile[ty + 32 * i][32 + tx * 4]) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
       }
       __syncthreads();
     }

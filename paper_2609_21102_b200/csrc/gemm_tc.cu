@@ -465,8 +465,10 @@ __device__ __forceinline__ void finish16(const TcParams& p, const uint32_t* r, c
 // shared memory with an XOR swizzle: `aux` is fetched with coalesced loads, written to the buffer, and each lane
 // reads back its row; the results take the same way in the other direction.
 __device__ __forceinline__ uint32_t stage_off(int row, int piece, int rowb, int pp) {
-  // rowb = bytes per row (64 or 128), pp = 16-byte pieces per row (4 or 8); rows of 64 bytes share a 128-byte line
-  const int key = (rowb == 64) ? ((row >> 1) & 3) : (row & 7);
+  // rowb = bytes per row (64 or 128), pp = 16-byte pieces per row (4 or 8); rows of 64 bytes share a 128-byte line.
+  // The key of a 64-byte row also takes in row >> 3: the transposed gather of a mirrored block reads, in one
+  // instruction, the same column of rows 8 apart, which the key (row >> 1) & 3 alone left on one bank.
+  const int key = (rowb == 64) ? (((row >> 1) ^ (row >> 3)) & 3) : (row & 7);
   return (uint32_t)(row * rowb + ((piece ^ key) << 4));
 }
 

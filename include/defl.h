@@ -41,7 +41,7 @@ extern "C" {
 #define DEFL_RESTORE_ADD 1    /* Eq. 3:       X0 = R/||R||_F,                   out = N^L(X0) + U_k V_k^T */
 
 /* normalisation scale of the symmetric residual (PSD) */
-#define DEFL_NORM_LANCZOS 0   /* App. D.1: 20-step Lanczos upper estimate of ||R||_2 */
+#define DEFL_NORM_LANCZOS 0   /* Appendix E.1, "Normalization scale": 20-step Lanczos upper estimate of ||R||_2 */
 #define DEFL_NORM_FROBENIUS 1 /* ||R||_F, a looser valid upper bound */
 
 /* which product engine runs the large matrix products */
@@ -86,15 +86,18 @@ typedef struct defl_opts {
                             reduces to the undeflated filter for that matrix. Decided per matrix on the device. */
   int half_filter;       /* PSD only, non-zero: the T filter steps run in IEEE half precision (iterates stored in
                             half, tensor-core products with fp32 accumulation), the precision the paper's SDP runs
-                            use for the filter (Appendix C.2). Everything around the filter stays fp32/tf32.
+                            use for the filter (Appendix E.2, "Composite Minimax Filter"). Everything around the filter stays fp32/tf32.
                             Needs n a multiple of 8 and the tensor engine. */
   int bf16_iterates;     /* polar path with bf16 input: storage type of the filter's iterates X_t, A_t, B_t (input,
                             output and every other stage are unchanged). 0 (default): IEEE half scaled by 32 in the
                             first two filter steps (same tensor-core rate, three more mantissa bits: the rounding of
                             the early iterates is what limits accuracy), bf16 in the later ones (less power, i.e.
                             more clock under a power cap); with DEFL_RESTORE_ADD scaled half in every step (that mode
-                            is about ten times more sensitive to the storage rounding). 1: bf16 in every step.
-                            2: scaled half in every step. */
+                            is about ten times more sensitive to the storage rounding). 1: bf16 in every step, the
+                            storage the paper's training runs use; NOT within the library's 3e-2 accuracy bar on wide
+                            matrices with slowly decaying spectra (1600 x 6400, sigma_i = 200/i, k = 32: 4.2e-2 relative
+                            Frobenius error against an fp64 evaluation of the same algorithm; square and faster
+                            decaying cases stay below 3e-2). 2: scaled half in every step. */
 } defl_opts;
 
 typedef struct defl_info {
@@ -182,11 +185,11 @@ int defl_psd_project(defl_ctx* ctx, const void* X, void* P, int n, int k,
 
 /* Three-block ADMM for a standard-form SDP whose constraints are diag(X) = b (max-cut type):
  *   min <C, X>  s.t.  diag(X) = b, X PSD;   A(X) = diag(X), A*(y) = Diag(y), A A* = I.
- * One iteration (Appendix C.1, the ADMM iteration; the S-update is Algorithm 2 through defl_psd_project):
+ * One iteration (Appendix E.1, "ADMM for Standard-Form SDP": the ADMM iteration; the S-update is Algorithm 2 through defl_psd_project):
  *   y <- b / sigma - diag(X / sigma + S - C)
  *   Z  = C - Diag(y) - X / sigma;        S <- projection of Z on the PSD cone (deflated, basis carried along)
  *   X <- X + sigma (S + Diag(y) - C)
- * After every iteration the three eigenvalue-free KKT terms of Appendix C.4 are evaluated on the device:
+ * After every iteration the three eigenvalue-free KKT terms of Appendix E.4, "Experimental Details" are evaluated on the device:
  *   residuals[3 it + 0] = ||diag(X) - b||_2 / (1 + ||b||_2)
  *   residuals[3 it + 1] = ||Diag(y) + S - C||_F / (1 + ||C||_F)
  *   residuals[3 it + 2] = |<C, X> - b^T y| / (1 + |<C, X>| + |b^T y|)

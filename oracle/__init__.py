@@ -205,10 +205,10 @@ def psd_project(Z, Vb, k, coeffs, tau=0.0, gamma=1.1, warmup=False, norm_mode=NO
 
 
 def admm_diag_sdp(C, b, sigma, iters, X, S, project, warmup_iters=0):
-    """Three-block ADMM of Appendix C.1 for  min <C,X>  s.t.  diag(X) = b, X PSD  (A = diag, A* = Diag, A A* = I),
+    """Three-block ADMM of Appendix E.1, "ADMM for Standard-Form SDP" for  min <C,X>  s.t.  diag(X) = b, X PSD  (A = diag, A* = Diag, A A* = I),
     `iters` iterations from the iterates (X, S). `project(Z, warmup)` returns the S-update, e.g. a closure over
     psd_project that carries the basis along, or an exact eigenvalue projection. Returns (X, S, y, res[iters,3])
-    with the three eigenvalue-free KKT terms of Appendix C.4 after every iteration."""
+    with the three eigenvalue-free KKT terms of Appendix E.4, "Experimental Details" after every iteration."""
     C, X, S, b = _f64(C), _f64(X).copy(), _f64(S).copy(), _f64(b)
     n = C.shape[0]
     y = np.zeros(n)

@@ -11,13 +11,13 @@
 //   Eq. 1          fixed-depth filter  X0 = A/theta, X_t = p_t(X_{t-1})
 //   Eq. 2          quintic Newton-Schulz map  N(X) = aX + b(XX^T)X + c(XX^T)^2 X
 //   Eq. 3          decomposition identities used by "restore"
-//   Eq. 5 + App. A Bjorck-Bowie coefficients of the degree-(2d+1) family
+//   Eq. 5 + Appendix B (proof of Theorem 1): Bjorck-Bowie coefficients of the degree-(2d+1) family
 //   Algorithm 1    deflated polar factor (gate, subtract, normalise, padded init, filter)
 //   Algorithm 2    deflated PSD projection (Rayleigh-Ritz, gate on |lambda|, padded init,
 //                  reconstruction, symmetrisation, basis update)
 //   Algorithm 3    batched randomized SVD (sketch, orthonormalise, J subspace iterations,
 //                  thin SVD of Q^T A, truncate)
-//   App. D.1       20-step Lanczos upper estimate theta = sqrt(rho + ||Z^2 v - rho v||)
+//   Appendix E.1, "Normalization scale"       20-step Lanczos upper estimate theta = sqrt(rho + ||Z^2 v - rho v||)
 //   Eq. 6, Eq. 7   PSD projection through the sign function, and the undeflated baseline
 //
 // Pinned (tests/test_oracle_*.py): Example 1's printed values, the Bjorck-Bowie closed form,
@@ -208,7 +208,7 @@ static void jacobi_eig(long n, const double* H, double* lam, double* E) {
 }
 
 // ------------------------------------------------------------------------------------------
-// Eq. 5 / App. A: Bjorck-Bowie coefficients a_i = (-1)^i sum_{j=i..d} 4^-j C(2j,j) C(j,i)
+// Eq. 5 / Appendix B (proof of Theorem 1): Bjorck-Bowie coefficients a_i = (-1)^i sum_{j=i..d} 4^-j C(2j,j) C(j,i)
 // ------------------------------------------------------------------------------------------
 static double binom(int n, int k) {
   double r = 1.0;
@@ -356,7 +356,7 @@ extern "C" void orc_deflated_polar(long m, long n, const double* G, long k, long
 }
 
 // ------------------------------------------------------------------------------------------
-// App. D.1: Lanczos on Z^2 (applied as Z(Zv), never formed), `steps` steps with full
+// Appendix E.1, "Normalization scale": Lanczos on Z^2 (applied as Z(Zv), never formed), `steps` steps with full
 // reorthogonalisation from the start vector v0; (rho, v) = largest Ritz pair;
 // theta = sqrt(rho + ||Z^2 v - rho v||_2).
 // ------------------------------------------------------------------------------------------
@@ -423,7 +423,7 @@ extern "C" double orc_lanczos_upper(long n, const double* Z, int steps, const do
 //            tau > 0 the paper's gate on the leading k magnitudes: if s_k < tau s_1 deflate
 //            {i : |lambda_i| > tau s_1}, else nothing.
 //   k = 0 or warmup != 0 : the undeflated baseline P = Z (I + g(Z/theta)) / 2  (Eq. 7).
-//   norm_mode 0 : Lanczos upper estimate (App. D.1) with start vector lanczos_v0[n];
+//   norm_mode 0 : Lanczos upper estimate (Appendix E.1, "Normalization scale") with start vector lanczos_v0[n];
 //             1 : Frobenius norm;  2 : the value theta_given.
 //   g = p_T o ... o p_1 with quintics coeffs[T][3].
 // Outputs: P[n,n] (exactly symmetric), Vnext[n,K] = orth(Z Vb), lam[K] Ritz values in the order

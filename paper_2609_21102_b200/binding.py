@@ -303,7 +303,7 @@ class Context:
     def defl_admm_diag_sdp(self, C, b, sigma, iters, X, S, k, warm_basis, coeff_schedule, steps=None, warmup_iters=0,
                            gamma=0.0, norm_mode=NORM_LANCZOS, lanczos_start=None, seed=0, engine=ENGINE_AUTO,
                            exploit_symmetry=False, tau=0.0, half_filter=False):
-        """`iters` ADMM iterations for min <C,X> s.t. diag(X) = b, X PSD (Appendix C.1), X and S updated in place.
+        """`iters` ADMM iterations for min <C,X> s.t. diag(X) = b, X PSD (Appendix E.1, "ADMM for Standard-Form SDP"), X and S updated in place.
         Returns (y[n], residuals[iters,3]) with the three eigenvalue-free KKT terms per iteration."""
         _dev(C, "C"), _dev(b, "b"), _dev(X, "X"), _dev(S, "S")
         n = C.shape[0]

@@ -1,6 +1,6 @@
 // Deflated PSD projection (Algorithm 2) of one symmetric fp32 matrix, as kernel launches on one stream:
 //   block step Z~ = Z V, Rayleigh-Ritz on V^T Z~ (one-sided Jacobi core), Ritz vectors U = V E,
-//   R = Z - sum_I lambda_i u_i u_i^T, Lanczos upper estimate of ||R||_2 (App. D.1),
+//   R = Z - sum_I lambda_i u_i u_i^T, Lanczos upper estimate of ||R||_2 (Appendix E.1, "Normalization scale"),
 //   X0 = R/theta + (1/gamma) sum_I sign(lambda_i) u_i u_i^T, the composite odd filter g (tf32 tensor
 //   cores, every product symmetric), P = (R + R g(X0))/2 + sum_{lambda_i > 0} lambda_i u_i u_i^T,
 //   P <- (P + P^T)/2, V <- CholeskyQR2(Z~).
@@ -84,7 +84,7 @@ static cudaError_t symv_launch(const float* A, const float* x, float* y, int n, 
 }
 
 // ---------------------------------------------------------------------------------------------
-// Lanczos on R^2 with full reorthogonalisation (App. D.1). One CTA does the vector work of a step:
+// Lanczos on R^2 with full reorthogonalisation (Appendix E.1, "Normalization scale"). One CTA does the vector work of a step:
 //   alpha_j = q_j . w;  w -= Q_j (Q_j^T w) twice;  beta_j = ||w||;  q_{j+1} = w / beta_j
 // State in device memory: Q[steps, n], T[steps, steps] (dense tridiagonal, fp64), done flag.
 // ---------------------------------------------------------------------------------------------
@@ -411,7 +411,7 @@ static int rank_update(defl_ctx* c, const PsdWs& w, int n, int K, int k, int coe
 }
 
 // ---------------------------------------------------------------------------------------------
-// Three-block ADMM for SDPs with the constraints diag(X) = b (App. C.1): element-wise kernels around
+// Three-block ADMM for SDPs with the constraints diag(X) = b (Appendix E.1, "ADMM for Standard-Form SDP"): element-wise kernels around
 // the projection. A(X) = diag(X), A*(y) = Diag(y), A A* = I.
 // ---------------------------------------------------------------------------------------------
 // y_i = b_i / sigma - (X_ii / sigma + S_ii - C_ii)
@@ -483,7 +483,7 @@ __global__ void __launch_bounds__(256) admm_x_kernel(const float* __restrict__ C
   }
 }
 
-// the three eigenvalue-free KKT terms of the iteration (App. C.4), from the partial sums and b^T y, ||b||, ||C||_F
+// the three eigenvalue-free KKT terms of the iteration (Appendix E.4, "Experimental Details"), from the partial sums and b^T y, ||b||, ||C||_F
 __global__ void admm_residual_kernel(const double* __restrict__ partial, int nblk, const float* __restrict__ b,
                                      const float* __restrict__ y, int n, double norm_b, double norm_c,
                                      float* __restrict__ out3) {
@@ -543,7 +543,7 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
   // iterates that feed tf32 products are stored already rounded to nearest tf32: the tensor core would
   // otherwise truncate them, which biases every product towards zero
   const int tf32_round = (engine == DEFL_ENGINE_TENSOR) ? 1 : 0;
-  // FP16 filter (Appendix C.2: the filter is used in half precision): iterates in IEEE half, kind::f16 products
+  // FP16 filter (Appendix E.2, "Composite Minimax Filter": the filter is used in half precision): iterates in IEEE half, kind::f16 products
   const bool half = opts && opts->half_filter;
   if (half && (engine != DEFL_ENGINE_TENSOR || (n & 7))) return DEFL_ERR_UNSUPPORTED;
 

@@ -1,4 +1,4 @@
-"""Shape groups of a Deflated Muon step (Appendix "Grouping": matrices of one shape are stacked into one batch and
+"""Shape groups of a Deflated Muon step (Appendix D, "Grouping": matrices of one shape are stacked into one batch and
 the batched range finder runs once per group per optimizer step).
 
 Host-side bookkeeping only, no arithmetic. The library takes wide matrices as they are stored

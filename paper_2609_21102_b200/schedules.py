@@ -1,8 +1,8 @@
 """Coefficient schedules for the fixed polynomial filter (host side, fp64, numpy only; no GPU, no oracle).
 
-* `bjorck_bowie(d)`: the classical Newton-Schulz map N_d of Eq. 2 (Appendix A closed form), as odd-power
+* `bjorck_bowie(d)`: the classical Newton-Schulz map N_d of Eq. 2 (closed form in Appendix B, the proof of Theorem 1), as odd-power
   coefficients; d = 2 gives (15/8, -5/4, 3/8).
-* `remez_sign_schedule(eps, T)`: stage one of the composite minimax sign filter (Appendix C.2): T odd quintics
+* `remez_sign_schedule(eps, T)`: stage one of the composite minimax sign filter (Appendix E.2, "Composite Minimax Filter"): T odd quintics
   g_t(x) = a x + b x^3 + c x^5, g_t the best uniform approximation of 1 on [a_t, b_t], [a_1, b_1] = [eps, 1],
   [a_{t+1}, b_{t+1}] = g_t([a_t, b_t]). The composition g_T o ... o g_1 approximates sign(x) on
   [-1, -eps] u [eps, 1]. (Stage two, the joint gradient refinement for the ReLU error, is not implemented.)
@@ -72,10 +72,10 @@ def minimax_odd_quintic(lo, hi, iters=100):
 
 
 def remez_sign_schedule(eps=1e-3, T=7, margin=0.0):
-    """Stage one of Appendix C.2: [(a_t, b_t, c_t)] for t = 1..T and the per-stage errors max |g_t - 1| on [a_t, b_t].
+    """Stage one of Appendix E.2, "Composite Minimax Filter": [(a_t, b_t, c_t)] for t = 1..T and the per-stage errors max |g_t - 1| on [a_t, b_t].
 
     Unlike the classical map, these polynomials are only meant for |x| <= 1: an input eigenvalue slightly above 1
-    (the Lanczos scale of Appendix D.1 is a heuristic upper estimate) leaves the next stage's interval and the
+    (the Lanczos scale of Appendix E.1, "Normalization scale" is a heuristic upper estimate) leaves the next stage's interval and the
     composition diverges. `margin` > 0 composes the first stage with x / (1 + margin), i.e. the schedule then
     covers [-(1 + margin), 1 + margin] and approximates the sign function from eps (1 + margin) on."""
     lo, hi = float(eps), 1.0

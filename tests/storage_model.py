@@ -1,0 +1,83 @@
+"""Sensitivity of the filter to the storage format of its iterate, evaluated with the oracle (test infrastructure).
+
+The library keeps the filter's iterate X_t in a narrow format between steps (IEEE half scaled by 32, bf16, or fp32
+rounded to tf32); the oracle keeps it in fp64. How far that rounding alone moves the result depends on the input
+(its singular values below the filter's knee are multiplied by the first slope at every step) and on the restore
+mode, not on any kernel. The functions here measure it on the oracle's side: the oracle's own filter step is applied
+step by step and the iterate is rounded between steps the way the storage format demands. The distance between that
+result and the oracle's unrounded result is the error the storage format explains; a parity test whose tolerance is
+tied to it asserts that the kernels add nothing of that size on top.
+
+Only numpy roundings and calls of the oracle; nothing here touches the CUDA library.
+"""
+import numpy as np
+
+import oracle
+
+
+def round_half_scaled(x, scale=32.0):
+    """Values as an IEEE half buffer holding scale * x keeps them (round to nearest even, gradual underflow)."""
+    with np.errstate(over="ignore"):
+        return (np.asarray(x, dtype=np.float64) * scale).astype(np.float16).astype(np.float64) / scale
+
+
+def round_bf16(x):
+    return oracle.round_to_storage(x, "bf16")
+
+
+def round_tf32(x):
+    """fp32 values rounded to nearest (ties away from zero, as cvt.rna does) on 10 explicit mantissa bits."""
+    x32 = np.ascontiguousarray(np.asarray(x, dtype=np.float64).astype(np.float32))
+    bits = x32.view(np.uint32).astype(np.uint64)
+    bits = ((bits + 0x1000) >> 13) << 13
+    return bits.astype(np.uint32).view(np.float32).reshape(x32.shape).astype(np.float64)
+
+
+ROUNDERS = {"half": round_half_scaled, "bf16": round_bf16, "tf32": round_tf32, "none": lambda x: np.asarray(x, dtype=np.float64)}
+
+
+def filter_with_storage(X0, sched, formats):
+    """p_L o ... o p_1 applied to X0 by the oracle's filter, one step per call, with the iterate rounded to
+    formats[t] before step t+1 reads it (formats[0] is the storage of X0 itself); the last result is not rounded."""
+    X = np.asarray(X0, dtype=np.float64)
+    for t, c in enumerate(sched):
+        X = ROUNDERS[formats[t]](X)
+        X = oracle.filter_quintic(X, [list(c)])
+    return X
+
+
+def polar_formats(L, add_mode, option=0):
+    """Iterate storage of the bf16 polar path per step: option 0 = scaled half in the first two steps (every step in
+    ADD mode), bf16 after; 1 = bf16 throughout; 2 = half throughout."""
+    if option == 1:
+        return ["bf16"] * L
+    n_half = L if (option == 2 or add_mode) else min(L, 2)
+    return ["half"] * n_half + ["bf16"] * (L - n_half)
+
+
+def polar_entry(G, k, l, Omega, J, gamma, add_mode):
+    """The oracle's filter input X0 for one matrix (Algorithm 3 then lines 3-4 of Algorithm 1), the head U_k V_k^T
+    that ADD mode adds back, in the caller's orientation."""
+    G = np.asarray(G, dtype=np.float64)
+    m, n = G.shape
+    tall = m >= n
+    A = G if tall else G.T
+    none = np.zeros((0, 3))
+    if k == 0:
+        out0, _, _ = oracle.alg1(A, None, None, None, none)
+        return (out0 if tall else out0.T), np.zeros_like(G)
+    U, s, V = oracle.brsvd(A, Omega, J)
+    U, s, V = U[:, :k], s[:k], V[:, :k]
+    head = U @ V.T
+    out0, _, _ = oracle.alg1(A, U, s, V, none, gamma=gamma, mode=oracle.ADD if add_mode else oracle.PADDED)
+    X0 = out0 - head if add_mode else out0        # with no filter steps ADD mode returns X0 + head
+    return (X0 if tall else X0.T), (head if tall else head.T)
+
+
+def polar_storage_error(G, k, l, Omega, J, sched, gamma, add_mode, option=0):
+    """Relative Frobenius distance between the oracle's result with the iterate rounded to the path's storage
+    formats and its result in fp64 throughout: what the storage format alone explains for this input."""
+    X0, head = polar_entry(G, k, l, Omega, J, gamma, add_mode)
+    exact = oracle.filter_quintic(X0, sched) + (head if add_mode else 0.0)
+    stored = filter_with_storage(X0, sched, polar_formats(len(sched), add_mode, option)) + (head if add_mode else 0.0)
+    return float(np.linalg.norm(stored - exact) / np.linalg.norm(exact))

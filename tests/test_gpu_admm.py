@@ -1,4 +1,4 @@
-"""defl_admm_diag_sdp on the GPU against the fp64 oracle loop (Appendix C.1), iteration by iteration."""
+"""defl_admm_diag_sdp on the GPU against the fp64 oracle loop (Appendix E.1, "ADMM for Standard-Form SDP"), iteration by iteration."""
 import numpy as np
 import pytest
 import torch

@@ -33,27 +33,57 @@ def _minimax_schedule(L=5):
     return [list(c) for c in sched]
 
 
-def _check_samples(ctx, G, Om, k, p, J, sched, gamma, samples, tol, mode=0, band=(0.05, 1.6)):
+def _scalar_band(sched, x_lo, x_hi, grid=4001):
+    """Image of [x_lo, x_hi] under the composite scalar map p_L o ... o p_1, p_t(x) = a x + b x^3 + c x^5."""
+    x = np.linspace(x_lo, x_hi, grid)
+    for a, b, c in sched:
+        x = a * x + b * x ** 3 + c * x ** 5
+    return float(x.min()), float(x.max())
+
+
+def _check_every_matrix(out, G, rho, sched, gamma, sigma_floor, slack):
+    """Properties that hold for every matrix of the batch at any size, evaluated on the device in fp32/fp64:
+    (1) out and G share their singular vectors (the filter acts on singular values only), so out G^T (short side) is
+        symmetric positive semidefinite: a result that belongs to another matrix, or a transposed or permuted one, fails;
+    (2) every singular value of out lies in the image of [sigma_floor / rho, 1] under the scalar composite map (after
+        Frobenius normalisation the residual's singular values are at most 1, and the padded head sits at 1 / gamma)."""
+    b, m, n = G.shape
+    o, g = out.float(), G.float()
+    S = o @ g.transpose(1, 2) if m <= n else o.transpose(1, 2) @ g
+    skew = (S - S.transpose(1, 2)).flatten(1).norm(dim=1) / S.flatten(1).norm(dim=1)
+    # (a result that belongs to another matrix gives a ratio near sqrt(2); storage rounding of the iterates leaves
+    # 1e-2 to 5e-2, most with the steep first step of the per-step minimax schedule)
+    assert float(skew.max()) <= 0.1, ("out G^T not symmetric", float(skew.max()))
+    ev = torch.linalg.eigvalsh(0.5 * (S + S.transpose(1, 2)).double())
+    assert float((ev.min(dim=1).values / ev.max(dim=1).values).min()) >= -slack, "out G^T not positive semidefinite"
+    gram = (o @ o.transpose(1, 2) if m <= n else o.transpose(1, 2) @ o).double()
+    sv = torch.linalg.eigvalsh(gram).clamp(min=0).sqrt()
+    for i in range(b):
+        lo, hi = _scalar_band(sched, sigma_floor / float(rho[i]), 1.0)
+        assert float(sv[i].min()) >= lo - slack and float(sv[i].max()) <= hi + slack, (i, float(sv[i].min()), float(sv[i].max()), lo, hi)
+
+
+def _check_samples(ctx, G, Om, k, p, J, sched, gamma, samples, tol, mode=0, sigma_floor=0.0, slack=4e-2):
     b, m, n = G.shape
     l = min(min(m, n), k + p)
     out, info = ctx.defl_polar_batched(G, k, p, J, sched, sketch=Om, gamma=gamma, restore_mode=mode,
                                        exploit_symmetry=True, want_info=True)
     torch.cuda.synchronize()
     assert int(info["status"].max()) == 0
+    worst = 0.0
     for i in samples:
         ref, s, kk, rho = oracle.deflated_polar(G[i].double().cpu().numpy(), k, l, Om[i].double().cpu().numpy(), J,
                                                 oracle.schedule(sched), gamma=gamma, mode=mode)
         err = _rel(out[i].double().cpu().numpy(), ref)
+        worst = max(worst, err)
         assert err <= tol, (i, err)
         assert abs(float(info["rho"][i]) - rho) <= 2e-3 * rho
         assert np.allclose(info["s"][i].double().cpu().numpy()[:k], s[:k], rtol=5e-3)
-    # every matrix: finite, and its squared Frobenius norm is that of a matrix whose min(m,n) singular values
-    # all lie in the band the quintic maps [0,1] into after a few steps (roughly [0.3, 1.25])
-    o = out.float()
-    assert bool(torch.isfinite(o).all())
-    fro2 = (o * o).sum(dim=(1, 2)) / min(m, n)
-    assert float(fro2.min()) > band[0] and float(fro2.max()) < band[1]
-    return out
+    print("parity %dx%dx%d k=%d mode=%d samples=%s worst=%.3e (tol %.1e)" % (b, m, n, k, mode, samples, worst, tol))
+    assert bool(torch.isfinite(out.float()).all())
+    if mode == 0:
+        _check_every_matrix(out, G, info["rho"].cpu(), sched, gamma, sigma_floor, slack)
+    return out, worst
 
 
 @pytest.mark.parametrize("shape_index,m,n", [(0, 768, 768), (1, 768, 3072)])
@@ -61,7 +91,7 @@ def test_workload2_gpt2_small_spiked(ctx, shape_index, m, n):
     dev = torch.device("cuda")
     G = inputs.workload_spiked(12, m, n, shape_index, device=dev).to(torch.bfloat16)
     Om = inputs.sketch(12, min(m, n), 16, 2, shape_index, device=dev)
-    _check_samples(ctx, G, Om, 8, 8, 1, [MUON] * 5, 1.01, [0, 11], 3e-2)
+    _check_samples(ctx, G, Om, 8, 8, 1, [MUON] * 5, 1.01, [0, 3, 7, 11], 3e-2)
 
 
 @pytest.mark.parametrize("shape_index,n", [(0, 1024), (1, 3072), (2, 4096)])
@@ -69,7 +99,7 @@ def test_workload3_power_law_per_step_schedule(ctx, shape_index, n):
     dev = torch.device("cuda")
     G = inputs.workload_power_law(24, 1024, n, 3, shape_index, 0.8, 50.0, device=dev).to(torch.bfloat16)
     Om = inputs.sketch(24, 1024, 24, 3, shape_index, device=dev)
-    _check_samples(ctx, G, Om, 16, 8, 1, _minimax_schedule(), 1.1, [23], 1e-2)
+    _check_samples(ctx, G, Om, 16, 8, 1, _minimax_schedule(), 1.1, [0, 8, 16, 23], 1e-2, sigma_floor=50.0 * 1024 ** -0.8)
 
 
 # Storage of the filter's iterates on workload 4 (error against the fp64 oracle, 1600 x 6400 group / square group):
@@ -80,18 +110,20 @@ def test_workload3_power_law_per_step_schedule(ctx, shape_index, n):
 # Rounding X_t (relative 2^-9 per entry in bf16) tilts each small singular direction by about
 # 1e-3 * ||X_t||_F / (sqrt(m) sigma_i), large for this spectrum (sigma_i = 200/i, floor 3.6e-3 after deflation) and
 # the 4:1 aspect while sigma_i is still small, i.e. in the first steps: later steps can afford bf16.
-TOL_DEFAULT_XL = 1.5e-2              # two half steps, then bf16 (spec tolerance for the bf16 path: 3e-2)
+TOL_DEFAULT_XL = 1.5e-2              # two half steps, then bf16 (the bf16 path's bar is 3e-2)
 TOL_HALF_ITERATES_XL = 1e-2
 TOL_BF16_ITERATES_XL_WIDE = 5e-2
+# SDP workload, deflated calls: error of P against the oracle relative to the bulk of P alone (tf32 filter)
+TOL_SDP_BULK = 2e-3
 
 
 def test_workload4_gpt2_xl_both_groups(ctx):
     dev = torch.device("cuda")
-    for shape_index, (m, n), samples, tol in ((1, (1600, 1600), [0, 47], TOL_DEFAULT_XL), (0, (1600, 6400), [5], TOL_DEFAULT_XL)):
+    for shape_index, (m, n), samples, tol in ((1, (1600, 1600), [0, 15, 31, 47], TOL_DEFAULT_XL), (0, (1600, 6400), [5, 17, 29, 41], TOL_DEFAULT_XL)):
         G = inputs.workload_power_law(48, m, n, 4, shape_index, 1.0, 200.0, 1e-4, device=dev).to(torch.bfloat16)
         Om = inputs.sketch(48, 1600, 48, 4, shape_index, device=dev)
-        _check_samples(ctx, G, Om, 32, 16, 2, [MUON] * 5, 1.01, samples, tol)
-        _check_samples(ctx, G, Om, 32, 16, 2, _minimax_schedule(), 1.1, samples[:1], tol, band=(0.6, 1.3))
+        _check_samples(ctx, G, Om, 32, 16, 2, [MUON] * 5, 1.01, samples, tol, sigma_floor=0.125)
+        _check_samples(ctx, G, Om, 32, 16, 2, _minimax_schedule(), 1.1, samples[:2], tol, sigma_floor=0.125)
         if n == 6400:
             # same matrices with fp32 storage on the exact engine (4 of them): the kernels themselves are exact
             out32 = ctx.defl_polar_batched(G[:4].float().contiguous(), 32, 16, 2, [MUON] * 5, sketch=Om[:4].contiguous(),
@@ -118,35 +150,56 @@ def test_workload4_add_mode_and_tall_orientation(ctx):
     _check_samples(ctx, G, Om, 32, 16, 2, [MUON] * 5, 1.01, [3], TOL_DEFAULT_XL, mode=1)
 
 
+def _bulk_norm(P, lam, n_deflated):
+    """Frobenius norm of P without its restored positive head: the head's eigenvalues (about 1e3) carry almost all of
+    ||P||_F (about 2e3 against 26 for the bulk), so an error is also judged against the bulk alone. The restored part
+    is sum lambda_i u_i u_i^T over the deflated Ritz pairs with lambda_i > 0, orthogonal to the rest up to the
+    Ritz residual: ||bulk||_F^2 = ||P||_F^2 - sum lambda_i^2."""
+    head2 = float(sum(l * l for l in lam[:n_deflated] if l > 0))
+    return float(np.sqrt(max(np.linalg.norm(P) ** 2 - head2, 0.0)))
+
+
 def test_workload5_sdp_sequence(ctx):
-    """Oracle parity at n = 1024 on a drifting sequence (warm-up, then deflated calls); at n = 4096, where one
-    fp64 oracle projection costs 3 TFLOP, the deflated projection is checked against a brute-force fp64
-    eigendecomposition (torch.linalg.eigh on the GPU) instead."""
-    from paper_2609_21102_b200 import binding
+    """The drifting SDP sequence (two warm-up calls, then deflated calls) against the oracle: every call at n = 1024;
+    at n = 4096, where one fp64 oracle projection costs 3 TFLOP, the first deflated call (both sides start it from
+    the same basis, the one the library produced during its warm-up calls). The error is judged on P as a whole and
+    on the bulk alone; the last projection is also compared with an fp64 eigendecomposition."""
     dev = torch.device("cuda")
     sched = [[1.875, -1.25, 0.375]] * 7
-    for n, oracle_checked in ((1024, True), (4096, False)):
+    for n, oracle_calls in ((1024, (0, 1, 2, 3)), (4096, (2,))):
         K, k = 16, 8
         x, lam = inputs.sdp_first(n, heads=k, head_mag=1.0e3, device=dev)
         V = inputs.randn((n, K), inputs.seed_for(5, 0, inputs.PURPOSE_BASIS), dev).float()
         v0 = inputs.gaussian_vector(n, 5, inputs.PURPOSE_LANCZOS, device=dev)
-        Vo = None
-        if oracle_checked:
-            q, r = np.linalg.qr(V.double().cpu().numpy())
-            Vo = q * np.sign(np.diag(r))[None, :]
         for t in range(4):
             X = x.float()
             warm = t < 2
+            V_in = V.double().cpu().numpy()
+            if t == 0:      # the library orthonormalises the Gaussian start block itself; the oracle wants it done
+                q, r = np.linalg.qr(V_in)
+                V_in = q * np.sign(np.diag(r))[None, :]
             P, info = ctx.defl_psd_project(X, k, V, sched, gamma=1.1, lanczos_start=v0, warmup=warm,
                                            exploit_symmetry=True, want_info=True)
             torch.cuda.synchronize()
             assert int(info["status"][0]) == 0
             assert torch.equal(P, P.T)
-            if oracle_checked:
-                Po, Vo, lam_o, ndef, th = oracle.psd_project(X.double().cpu().numpy(), Vo, k, oracle.schedule(sched),
+            if t in oracle_calls:
+                Po, Vo, lam_o, ndef, th = oracle.psd_project(X.double().cpu().numpy(), V_in, k, oracle.schedule(sched),
                                                              gamma=1.1, warmup=warm, lanczos_v0=v0.double().cpu().numpy())
-                assert _rel(P.double().cpu().numpy(), Po) <= (4e-3 if warm else 2e-3), (n, t)
+                Pg = P.double().cpu().numpy()
+                assert _rel(Pg, Po) <= 2e-3, (n, t, _rel(Pg, Po))
                 assert abs(float(info["theta"][0]) - th) <= 2e-3 * th
+                if not warm:
+                    assert ndef == k and int(info["k_used"][0]) == k
+                    bulk = _bulk_norm(Po, lam_o, ndef)
+                    assert 0.2 * np.sqrt(n) < bulk < np.sqrt(n)        # ||max(U(-1,1), 0)||_F is about sqrt(n / 6)
+                    err_bulk = float(np.linalg.norm(Pg - Po)) / bulk
+                    print("sdp n=%d call %d: whole %.3e bulk-only %.3e (bulk norm %.1f)" % (n, t, _rel(Pg, Po), err_bulk, bulk))
+                    assert err_bulk <= TOL_SDP_BULK, (n, t, err_bulk)
+                    # the updated bases span the same subspace
+                    Vg = V.double().cpu().numpy()
+                    assert _rel(Vg @ Vg.T, Vo @ Vo.T) <= 1e-3
+                del Po, Pg
             x = inputs.sdp_next(x, t + 1)
         # last (deflated) projection against the exact projection
         w, v = torch.linalg.eigh(X.double())

@@ -48,7 +48,7 @@ SCHED7 = [[1.875, -1.25, 0.375]] * 7
 @pytest.mark.parametrize("engine_name", ["tensor", "simt", "half"])
 def test_psd_matches_oracle_with_tracked_basis(ctx, n, K, k, engine_name):
     """engine "half": the filter steps in IEEE half precision (the paper's SDP runs use the filter in half
-    precision, Appendix C.2), everything around them unchanged; same oracle, same tolerance."""
+    precision, Appendix E.2, "Composite Minimax Filter"), everything around them unchanged; same oracle, same tolerance."""
     from paper_2609_21102_b200 import binding
     engine = binding.ENGINE_SIMT if engine_name == "simt" else binding.ENGINE_AUTO
     half = engine_name == "half"
@@ -159,7 +159,7 @@ def test_psd_argument_errors(ctx):
 
 
 def test_psd_with_the_stage_one_minimax_schedule(ctx):
-    """Appendix C.2's composite sign filter (stage one, eps = 1e-3, T = 7) as the schedule: parity with the oracle on
+    """Appendix E.2, "Composite Minimax Filter"'s composite sign filter (stage one, eps = 1e-3, T = 7) as the schedule: parity with the oracle on
     the same schedule, and — because this filter reaches the sign function on [eps, 1] — closeness to the exact
     projection from LAPACK."""
     from paper_2609_21102_b200 import binding, schedules

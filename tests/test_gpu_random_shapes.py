@@ -1,12 +1,18 @@
 """Seeded random shapes and options through defl_polar_batched against the oracle: ragged and aligned sizes, tall and
-wide, k = 0 and k > 0, J = 0..2, L = 1..6, both storage types, symmetric tiles on and off. PADDED restore only:
-Eq. 3's post-add (ADD mode) amplifies the difference between two inexact sets of triplets by a^L, which is a
-property of that mode (the paper pads for this reason), not of an implementation."""
+wide, k = 0 and k > 0, J = 0..2, L = 1..6, both storage types, symmetric tiles on and off, both restore modes.
+
+PADDED restore (Algorithm 1) is held to the library's bars: 3e-2 with bf16 storage, 2e-3 with fp32 storage.
+ADD restore (Eq. 3) is held to 2e-3 with fp32 storage. With bf16 storage its iterates live in IEEE half, and without
+the head inside X_0 every singular value of X_0 is small, so the rounding of the stored iterate is multiplied by the
+filter's first slope at every step (3.44^6 for six Muon steps): there the bar is what that rounding alone explains,
+measured on the oracle's side (storage_model.polar_storage_error: the oracle's own steps with the iterate rounded to
+the storage format between them), doubled, and never below 3e-2."""
 import numpy as np
 import pytest
 import torch
 
 import oracle
+import storage_model
 from paper_2609_21102_b200 import inputs
 
 pytestmark = pytest.mark.gpu
@@ -51,3 +57,51 @@ def test_random_configurations(ctx, seed):
                                             oracle.schedule([mu] * L), gamma=1.05)
             err = float(np.linalg.norm(out[i].double().cpu().numpy() - ref) / np.linalg.norm(ref))
             assert err <= tol, (case, i, err)
+
+
+def _add_cases(seed, trials):
+    rng = np.random.default_rng(seed)
+    for trial in range(trials):
+        b = int(rng.integers(1, 4))
+        m, n = int(rng.integers(40, 720)), int(rng.integers(40, 720))
+        if rng.random() < 0.5:
+            m, n = (m // 8) * 8 + 8, (n // 8) * 8 + 8
+        ms = min(m, n)
+        k = int(rng.integers(1, min(12, ms // 3)))
+        p = int(rng.integers(1, 9))
+        J, L, sym = int(rng.integers(0, 3)), int(rng.integers(1, 7)), bool(rng.integers(0, 2))
+        l = min(ms, k + p)
+        sigma = np.concatenate([np.sort(rng.uniform(5, 60, k))[::-1], rng.uniform(0.05, 1.0, ms - k)])
+        G = torch.stack([inputs.from_spectrum(m, n, sigma, 9000 * seed + 10 * trial + i) for i in range(b)])
+        Om = torch.tensor(rng.standard_normal((b, ms, l)), dtype=torch.float32)
+        yield trial, b, m, n, k, p, l, J, L, sym, G, Om
+
+
+@pytest.mark.parametrize("seed", [21, 22])
+def test_random_configurations_add_restore(ctx, seed):
+    """Eq. 3's post-add on ragged shapes. The same values go through in fp32 storage (exact products: the restore
+    mode on its own) and in bf16 storage (tensor engine, half iterates), each against the oracle run on the values
+    that storage holds."""
+    from paper_2609_21102_b200 import binding
+    mu = list(binding.MUON_QUINTIC)
+    worst = {"f32": 0.0, "bf16": 0.0}
+    for trial, b, m, n, k, p, l, J, L, sym, G, Om in _add_cases(seed, 10):
+        sched = [mu] * L
+        for dt, name in ((torch.float32, "f32"), (torch.bfloat16, "bf16")):
+            Gs = G.to(dt)
+            out, info = ctx.defl_polar_batched(Gs.cuda(), k, p, J, sched, sketch=Om.cuda(), gamma=1.05,
+                                               restore_mode=binding.RESTORE_ADD, exploit_symmetry=sym, want_info=True)
+            torch.cuda.synchronize()
+            case = (seed, trial, b, m, n, k, p, J, L, sym, name)
+            assert int(info["status"].max()) == 0, case
+            for i in range(b):
+                Gi, Oi = Gs[i].double().numpy(), Om[i].double().numpy()
+                ref, *_ = oracle.deflated_polar(Gi, k, l, Oi, J, oracle.schedule(sched), gamma=1.05, mode=oracle.ADD)
+                err = float(np.linalg.norm(out[i].double().cpu().numpy() - ref) / np.linalg.norm(ref))
+                if name == "f32":
+                    tol = 2e-3
+                else:
+                    tol = max(3e-2, 2.0 * storage_model.polar_storage_error(Gi, k, l, Oi, J, sched, 1.05, True))
+                worst[name] = max(worst[name], err / tol)
+                assert err <= tol, (case, i, err, tol)
+    print("ADD restore, seed %d: worst error / tolerance" % seed, worst)

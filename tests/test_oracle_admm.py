@@ -1,4 +1,4 @@
-"""Pins for the oracle's ADMM loop (Appendix C.1 iteration, Appendix C.4 residual terms): an analytically built KKT
+"""Pins for the oracle's ADMM loop (Appendix E.1 "ADMM for Standard-Form SDP" iteration, Appendix E.4, "Experimental Details" residual terms): an analytically built KKT
 point must be a fixed point, a 2 x 2 instance has a closed-form optimum, and on small max-cut instances the loop with
 LAPACK's exact projection must drive the optimality conditions of the SDP pair to zero. Nothing expected here comes
 from the oracle."""
@@ -55,7 +55,7 @@ def test_small_maxcut_reaches_the_optimality_conditions():
     assert abs(np.sum(C * X) - b @ y) < 1e-5
     assert np.linalg.eigvalsh(X).min() > -1e-8 and np.linalg.eigvalsh(S).min() > -1e-8
     assert abs(np.sum(X * S)) < 1e-5
-    # the residual terms reported are those quantities, normalised as in Appendix C.4
+    # the residual terms reported are those quantities, normalised as in Appendix E.4, "Experimental Details"
     assert np.isclose(res[-1, 0], np.linalg.norm(np.diag(X) - b) / (1 + np.linalg.norm(b)), atol=1e-12)
     assert res[-1].max() < 1e-6 and res[0].max() > 1e-2
     # the value is bounded by the trivial cut bounds: every edge cut gives -|E|, and the SDP relaxes max-cut

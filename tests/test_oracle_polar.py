@@ -45,7 +45,7 @@ def _p_quintic(x, coeffs, L):
 
 
 # ---------------------------------------------------------------------------------------------
-# Coefficients: Eq. 2's printed triple and the closed form of App. A
+# Coefficients: Eq. 2's printed triple and the closed form of Appendix B (proof of Theorem 1)
 # ---------------------------------------------------------------------------------------------
 def test_bjorck_bowie_reproduces_printed_quintic():
     g = _golden("classical_quintic.txt")
@@ -239,7 +239,7 @@ def test_brsvd_invariants_and_sandwich_bound():
     res = A - (U * s) @ V.T
     assert np.isclose(np.linalg.norm(res) ** 2, np.linalg.norm(A) ** 2 - (s ** 2).sum(), rtol=1e-10)
     assert np.allclose(U.T @ A, (V * s).T, atol=1e-11)
-    # sandwich bound on the singular values with the actual sketch (App. B, subspace-iteration bounds)
+    # sandwich bound on the singular values with the actual sketch (Appendix D, "Bounds for randomized subspace iteration")
     Om1 = Vex[:, :k].T @ Om
     Om2 = Vex[:, k:].T @ Om
     c = np.linalg.norm(Om2 @ np.linalg.pinv(Om1), 2)

@@ -1,4 +1,4 @@
-"""Pins for the schedule tools (Eq. 2 / Appendix A closed form; Appendix C.2 stage one): the printed classical
+"""Pins for the schedule tools (Eq. 2 / closed form in Appendix B, the proof of Theorem 1; Appendix E.2, "Composite Minimax Filter" stage one): the printed classical
 coefficients, the equioscillation that characterises a best uniform approximation, an independent linear-programming
 solution of the same minimax problem, and the limits the construction must reach."""
 import os

@@ -1,0 +1,47 @@
+"""The storage-sensitivity helpers used by the GPU parity tests: the roundings are the formats' roundings, and
+the step-by-step evaluation, with no rounding, is the oracle's own whole-path result."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import storage_model as sm
+from paper_2609_21102_b200 import inputs
+
+MUON = list(oracle.MUON_QUINTIC)
+
+
+def test_roundings_match_the_formats():
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal(4096) * np.exp(rng.uniform(-6, 2, 4096))
+    for name, unit, ref in (("half", 2.0 ** -11, None), ("bf16", 2.0 ** -8, torch.bfloat16), ("tf32", 2.0 ** -11, None)):
+        r = sm.ROUNDERS[name](x)
+        assert np.array_equal(sm.ROUNDERS[name](r), r)                       # idempotent
+        normal = np.abs(x) * 32.0 >= 2.0 ** -14 if name == "half" else np.ones_like(x, dtype=bool)     # half: below that, gradual underflow
+        assert float(np.max(np.abs(r - x)[normal] / np.abs(x)[normal])) <= unit * (1 + 1e-6)
+        if ref is not None:
+            assert np.array_equal(r, torch.tensor(x, dtype=torch.float32).to(ref).double().numpy())
+    # half: values as torch's float16 keeps 32 x
+    assert np.array_equal(sm.round_half_scaled(x), (torch.tensor(x * 32.0, dtype=torch.float64).to(torch.float16).double() / 32.0).numpy())
+    # tf32 keeps 10 explicit mantissa bits: the low 13 bits of the fp32 pattern are zero
+    bits = sm.round_tf32(x).astype(np.float32).view(np.uint32)
+    assert int(np.bitwise_and(bits, 0x1FFF).max()) == 0
+
+
+@pytest.mark.parametrize("m,n", [(96, 40), (40, 96)])
+@pytest.mark.parametrize("add_mode", [False, True])
+def test_stepwise_evaluation_is_the_oracle_path(m, n, add_mode):
+    k, l, J, gamma, L = 4, 8, 1, 1.05, 4
+    sigma = np.concatenate([[30.0, 20.0, 12.0, 8.0], np.linspace(1.0, 0.05, 36)])
+    G = inputs.from_spectrum(m, n, sigma, 4242).numpy()
+    Om = np.random.default_rng(3).standard_normal((min(m, n), l))
+    ref, *_ = oracle.deflated_polar(G, k, l, Om, J, oracle.schedule([MUON] * L), gamma=gamma,
+                                    mode=oracle.ADD if add_mode else oracle.PADDED)
+    X0, head = sm.polar_entry(G, k, l, Om, J, gamma, add_mode)
+    got = sm.filter_with_storage(X0, [MUON] * L, ["none"] * L) + (head if add_mode else 0.0)
+    assert np.linalg.norm(got - ref) <= 1e-11 * np.linalg.norm(ref)
+    assert sm.polar_storage_error(G, k, l, Om, J, [MUON] * L, gamma, add_mode, option=2) > 0.0
+    # bf16 storage moves the result more than half storage does
+    e_half = sm.polar_storage_error(G, k, l, Om, J, [MUON] * L, gamma, add_mode, option=2)
+    e_bf16 = sm.polar_storage_error(G, k, l, Om, J, [MUON] * L, gamma, add_mode, option=1)
+    assert e_bf16 > 2.0 * e_half

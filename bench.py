@@ -6,15 +6,22 @@ Newton-Schulz steps, restore) over one batch: 48 matrices 1600x6400 and 48 matri
 bf16 with the heavy-tailed spectrum sigma_i = max(200/i, 1e-4), k=32, oversampling 16, 2 subspace
 iterations. Prints ONE JSON line (see README / DESIGN for the keys).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--small]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--small] [--no-extras]
 
-N > 1 is launched under torchrun; every rank runs the same batch on its own GPU (independent
-matrices, no data-path collective) and the line reports the whole-job aggregate.
+`value` counts the flops the method needs (symmetric products once when the symmetric tiles are on); the
+dense-equivalent figure is a separate key. Besides the timed K steps the run reports a sustained leg (the step
+repeated for at least 3 s, with its clock record), and under `extras` the other workloads: the GPT-2-small and
+medium/large shape batches, the XL batch with the per-step minimax schedule and with the additive restore, and
+the 20-call SDP projection sequence at n = 4096 with its stage split.
+
+N > 1: every rank runs the same batch on its own GPU (independent matrices, no data-path collective) and the line
+reports the whole-job aggregate; without an outer torchrun the script starts its N ranks itself.
 `--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
 """
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import threading
@@ -25,30 +32,34 @@ sys.path.insert(0, ROOT)
 
 METRIC = "deflated polar-filter TFLOP/s & matrices/s per batch; % bf16 tensor peak"
 MUON = (3.4445, -4.7750, 2.0315)
-SYM = True   # compute X X^T and A A on the tiles that reach the diagonal and mirror them (--no-symmetry turns it off)
-BF16_ITERATES = 0       # storage of the filter's iterates: 0 scaled IEEE half in the first two steps then bf16 (default),
-                        # 1 bf16 throughout (--bf16-iterates), 2 scaled half throughout (--half-iterates)
-GAMMA = 1.01            # padding of the restored head (1.1 with the minimax schedule, the value the paper uses with it)
-SCHEDULE = "muon"       # --schedule minimax: per-step minimax quintics (the Polar-Express-style mapping)
-SCHEDULE_NOTE = "Muon quintic (3.4445, -4.7750, 2.0315) every step"
-_MINIMAX = {}
+CLASSICAL = (1.875, -1.25, 0.375)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+_MINIMAX = {}
 
+# name: shape groups (b, m, n), k, p, J, L, schedule, gamma, input recipe
 WORKLOADS = {
-    # name: (list of (b, m, n), k, p, J, L)
-    "gpt2_xl": {"groups": [(48, 1600, 6400), (48, 1600, 1600)], "k": 32, "p": 16, "J": 2, "L": 5,
+    "gpt2_xl": {"groups": [(48, 1600, 6400), (48, 1600, 1600)], "k": 32, "p": 16, "J": 2, "L": 5, "schedule": "muon",
+                "gamma": 1.01, "workload": 4, "recipe": ("power", 1.0, 200.0, 1e-4),
                 "label": "GPT-2-XL Muon shapes, bf16: 48 x 1600x6400 + 48 x 1600x1600, sigma_i=max(200/i,1e-4), "
                          "k=32, p=16, J=2, 5 Muon quintic steps"},
-    "small": {"groups": [(4, 256, 1024), (4, 256, 256)], "k": 8, "p": 8, "J": 1, "L": 5,
+    "gpt2_small": {"groups": [(12, 768, 768), (12, 768, 3072)], "k": 8, "p": 8, "J": 1, "L": 5, "schedule": "muon",
+                   "gamma": 1.01, "workload": 2, "recipe": ("spiked",),
+                   "label": "GPT-2-small Muon shapes, bf16: 12 x 768x768 + 12 x 768x3072, N(0,1) bulk + 8 spikes, "
+                            "k=8, p=8, J=1, 5 Muon quintic steps"},
+    "gpt2_medium_large": {"groups": [(24, 1024, 1024), (24, 1024, 3072), (24, 1024, 4096)], "k": 16, "p": 8, "J": 1,
+                          "L": 5, "schedule": "minimax", "gamma": 1.1, "workload": 3, "recipe": ("power", 0.8, 50.0, 0.0),
+                          "label": "GPT-2-medium/large Muon shapes, bf16: 24 x 1024x{1024,3072,4096}, sigma_i=50 i^-0.8, "
+                                   "k=16, p=8, J=1, 5 per-step minimax quintic steps (Polar-Express-style)"},
+    "small": {"groups": [(4, 256, 1024), (4, 256, 256)], "k": 8, "p": 8, "J": 1, "L": 5, "schedule": "muon",
+              "gamma": 1.01, "workload": 4, "recipe": ("power", 1.0, 200.0, 1e-4),
               "label": "small check: 4 x 256x1024 + 4 x 256x256"},
 }
 
 
-def sched_of(wl):
-    """The [L][3] coefficient schedule of the run: Muon's quintic repeated, or per-step minimax quintics built by
-    greedy Remez exchange from [1e-3, 1] (first step rescaled by 1.01); same products per step either way."""
-    L = wl["L"]
-    if SCHEDULE == "muon":
+def schedule_of(name, L):
+    """[L][3] coefficients: Muon's quintic repeated, or per-step minimax quintics built by greedy Remez exchange from
+    [1e-3, 1] (first step rescaled by 1.01): the Polar-Express-style mapping. Same products per step either way."""
+    if name == "muon":
         return [list(MUON)] * L
     if L not in _MINIMAX:
         from paper_2609_21102_b200 import schedules
@@ -56,14 +67,24 @@ def sched_of(wl):
     return _MINIMAX[L]
 
 
-def flops_per_matrix(m, n, k, p, J, L):
-    """Algorithmic flops of one matrix: dense filter count, rSVD products, subtract and restore."""
+def algorithmic_flops(m, n, k, p, J, L, symmetric, add_restore=False):
+    """Flops the method needs for one matrix: (filter, front end). Filter per step: the Gram matrix and its square
+    (each counted once per symmetric pair when the symmetric tiles are on, else in full) and the apply product;
+    front end: the (2 + 2J) products of the randomized SVD with the l-column panel, the rank-k subtraction and, with
+    the additive restore, the rank-k add."""
     ms, ml = min(m, n), max(m, n)
     l = min(ms, k + p) if k > 0 else 0
-    filt = L * (4.0 * ms * ms * ml + 2.0 * ms ** 3)
-    rsvd = 2.0 * ml * ms * l * (2 + 2 * J) if k > 0 else 0.0
-    defl = 2.0 * 2.0 * m * n * k          # residual norm pass + X0 pass
-    return filt, rsvd + defl
+    if symmetric:
+        filt = L * (ms * (ms + 1.0) * ml + ms * ms * (ms + 1.0) + 2.0 * ms * ms * ml)
+    else:
+        filt = L * (4.0 * ms * ms * ml + 2.0 * ms ** 3)
+    front = (2.0 * ml * ms * l * (2 + 2 * J) + 2.0 * m * n * k * (2 if add_restore else 1)) if k > 0 else 0.0
+    return filt, front
+
+
+def dense_filter_flops(m, n, L):
+    ms, ml = min(m, n), max(m, n)
+    return L * (4.0 * ms * ms * ml + 2.0 * ms ** 3)
 
 
 # Average DRAM bytes per filter-product launch: dram__bytes_read + dram__bytes_write of the six kinds of filter
@@ -87,29 +108,6 @@ def aggregate_throughput(units_per_rank, world, ms_max):
     return world * units_per_rank / (ms_max * 1e-3)
 
 
-def executed_filter_flops(m, n, L, symmetric, tile=256):
-    """Flops the tensor engine executes for the L filter steps of one matrix. It works on 256 x 256 output
-    tiles made of two 128-row halves; edge tiles compute only the rows (in halves) and columns (in sixteens)
-    that exist; with `symmetric` the two symmetric products skip every half-tile left of the diagonal."""
-    ms, ml = min(m, n), max(m, n)
-
-    def product(M, N, K, sym):
-        total = 0.0
-        for r0 in range(0, M, tile):
-            for c0 in range(0, N, tile):
-                cols = min(tile, ((N - c0 + 15) // 16) * 16)
-                for h0 in (r0, r0 + 128):
-                    if h0 >= M:
-                        continue
-                    if sym and c0 + tile <= h0:
-                        continue
-                    total += 2.0 * 128 * cols * K
-        return total
-
-    return L * (product(ms, ms, ml, symmetric) + product(ms, ms, ms, symmetric) +
-                (product(m, n, m, False) if m <= n else product(m, n, n, False)))
-
-
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -120,64 +118,75 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs: one nvidia-smi process in loop
-    mode (50 ms period), started ahead of the region; only samples that arrive between mark_start() and
-    mark_end() are kept."""
+    """SM clock, power and throttle reasons of one GPU while a timed region runs: NVML polled every 10 ms from a
+    thread (read-only queries), nvidia-smi in loop mode as the fallback. Regions are cut out afterwards by time."""
+
+    REASONS = (("hw_slowdown", 0x8), ("hw_thermal_slowdown", 0x40), ("sw_thermal_slowdown", 0x20), ("sw_power_cap", 0x4))
 
     def __init__(self, index):
-        self.index, self.rows, self._all, self._t, self._p = index, [], [], None, None
-        self.t0 = self.t1 = None
+        self.index, self.rows, self._stop, self._t, self._p, self.max_mhz = index, [], False, None, None, None
 
-    def _run(self):
+    def _nvml(self):
+        import pynvml
+        pynvml.nvmlInit()
+        h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+        self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+        reasons = getattr(pynvml, "nvmlDeviceGetCurrentClocksEventReasons", None) or pynvml.nvmlDeviceGetCurrentClocksThrottleReasons
+        while not self._stop:
+            try:
+                self.rows.append((time.time(), float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)),
+                                  pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0, int(reasons(h))))
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def _smi(self):
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        self._p = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + q, "--format=csv,noheader,nounits",
+                                    "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True, bufsize=1)
         for line in self._p.stdout:
             parts = [x.strip() for x in line.strip().split(",")]
-            if len(parts) >= 6:
-                self._all.append((time.time(), parts))
+            if len(parts) >= 7 and parts[0].replace(".", "").isdigit():
+                mask = sum(bit for (nm, bit), v in zip(self.REASONS, parts[3:7]) if v.lower().startswith("active"))
+                self.max_mhz = float(parts[1])
+                self.rows.append((time.time(), float(parts[0]), float(parts[2]) if parts[2].replace(".", "").isdigit() else 0.0, mask))
 
     def __enter__(self):
-        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
         try:
-            self._p = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + q,
-                                        "--format=csv,noheader,nounits", "-lms", "50"], stdout=subprocess.PIPE,
-                                       stderr=subprocess.DEVNULL, text=True, bufsize=1)
-            self._t = threading.Thread(target=self._run, daemon=True)
-            self._t.start()
-            time.sleep(0.3)      # let the first samples arrive before the region starts
+            import pynvml  # noqa: F401
+            target = self._nvml
         except Exception:
-            self._p = None
+            target = self._smi
+        self._t = threading.Thread(target=target, daemon=True)
+        self._t.start()
+        time.sleep(0.2)
         return self
 
-    def mark_start(self):
-        self.t0 = time.time()
-
-    def mark_end(self):
-        self.t1 = time.time()
-
     def __exit__(self, *a):
+        self._stop = True
         if self._p is not None:
             self._p.terminate()          # the one process this object started
             try:
                 self._p.wait(timeout=5)
             except Exception:
                 self._p.kill()
-            self._t.join(timeout=5)
-        t0 = self.t0 if self.t0 is not None else 0.0
-        t1 = self.t1 if self.t1 is not None else float("inf")
-        self.rows = [r for (t, r) in self._all if t0 <= t <= t1]
-        if not self.rows and self._all:      # a region shorter than the period: the nearest sample
-            mid = 0.5 * (t0 + min(t1, time.time()))
-            self.rows = [min(self._all, key=lambda tr: abs(tr[0] - mid))[1]]
+        self._t.join(timeout=5)
 
-    def summary(self):
-        if not self.rows:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
-        sm = sorted(float(r[0]) for r in self.rows if r[0].replace(".", "").isdigit())
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [nm for i, nm in enumerate(names) if any(r[2 + i].lower().startswith("active") for r in self.rows)]
-        mx = [float(r[1]) for r in self.rows if r[1].replace(".", "").isdigit()]
-        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(self.rows)}
+    def summary(self, t0, t1):
+        rows = [r for r in self.rows if t0 <= r[0] <= t1]
+        if not rows and self.rows:      # a region shorter than the period: the nearest sample
+            mid = 0.5 * (t0 + t1)
+            rows = [min(self.rows, key=lambda r: abs(r[0] - mid))]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unsampled"], "samples": 0}
+        sm = sorted(r[1] for r in rows)
+        pw = sorted(r[2] for r in rows)
+        mask = 0
+        for r in rows:
+            mask |= r[3]
+        return {"sm_mhz": sm[len(sm) // 2], "sm_min_mhz": sm[0], "sm_max_mhz": self.max_mhz,
+                "power_w": pw[len(pw) // 2], "reasons": [nm for nm, bit in self.REASONS if mask & bit], "samples": len(rows)}
 
 
 def make_inputs(wl, device):
@@ -185,22 +194,27 @@ def make_inputs(wl, device):
     from paper_2609_21102_b200 import inputs
     groups = []
     for si, (b, m, n) in enumerate(wl["groups"]):
-        G = inputs.workload_power_law(b, m, n, 4, si, 1.0, 200.0, 1e-4, device=device).to(torch.bfloat16)
+        if wl["recipe"][0] == "spiked":
+            G = inputs.workload_spiked(b, m, n, si, device=device)
+        else:
+            _, expo, top, floor = wl["recipe"]
+            G = inputs.workload_power_law(b, m, n, wl["workload"], si, expo, top, floor, device=device)
+        G = G.to(torch.bfloat16)
         l = min(min(m, n), wl["k"] + wl["p"])
-        Om = inputs.sketch(b, min(m, n), l, 4, si, device=device)
+        Om = inputs.sketch(b, min(m, n), l, wl["workload"], si, device=device)
         groups.append({"G": G, "Om": Om, "out": torch.empty_like(G)})
     return groups
 
 
-def run_step(ctx, wl, groups, lanes=None):
+def run_step(ctx, wl, groups, opts, lanes=None):
     """One step = every shape group through defl_polar_batched. With `lanes` (one (context, stream) pair per
-    group) the independent groups are enqueued on their own streams, forked from and joined to the current
-    stream, so that the small latency-bound kernels of one group overlap the other group's work."""
+    group) the independent groups are enqueued on their own streams, forked from and joined to the current stream."""
     import torch
+    sched = schedule_of(wl["schedule"], wl["L"])
+    kw = dict(gamma=wl["gamma"], exploit_symmetry=opts["sym"], bf16_iterates=opts["iterates"], restore_mode=opts["mode"])
     if not lanes:
         for g in groups:
-            ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], sched_of(wl), out=g["out"],
-                                   sketch=g["Om"], gamma=GAMMA, exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
+            ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], sched, out=g["out"], sketch=g["Om"], **kw)
         return
     main = torch.cuda.current_stream()
     fork = torch.cuda.Event()
@@ -208,29 +222,171 @@ def run_step(ctx, wl, groups, lanes=None):
     for g, (c, s) in zip(groups, lanes):
         s.wait_event(fork)
         with torch.cuda.stream(s):
-            c.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], sched_of(wl), out=g["out"],
-                                 sketch=g["Om"], gamma=GAMMA, exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
+            c.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], sched, out=g["out"], sketch=g["Om"], **kw)
             done = torch.cuda.Event()
             done.record(s)
         main.wait_event(done)
 
 
-def oracle_sample(wl, seconds_hint=20.0):
-    """Times the fp64 oracle on one matrix of the smallest group (a bounded sample of the workload)."""
-    import numpy as np
-    import oracle
-    from paper_2609_21102_b200 import inputs
+def time_steps(fn, steps, sync):
+    """ms per step of `steps` back-to-back calls of fn, by CUDA events on the current stream."""
     import torch
-    b, m, n = min(wl["groups"], key=lambda g: g[1] * g[2])
-    si = wl["groups"].index((b, m, n))
-    G = inputs.workload_power_law(1, m, n, 4, si, 1.0, 200.0, 1e-4).to(torch.bfloat16).double().numpy()[0]
-    l = min(min(m, n), wl["k"] + wl["p"])
-    Om = inputs.sketch(1, min(m, n), l, 4, si).double().numpy()[0]
-    t0 = time.perf_counter()
-    oracle.deflated_polar(G, wl["k"], l, Om, wl["J"], oracle.schedule(sched_of(wl)), gamma=GAMMA)
-    dt = time.perf_counter() - t0
-    filt, rest = flops_per_matrix(m, n, wl["k"], wl["p"], wl["J"], wl["L"])
-    return dt, (filt + rest), "1 matrix %dx%d of the batch, full path, fp64" % (m, n)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync()
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    sync()
+    return e0.elapsed_time(e1) / steps
+
+
+def workload_flops(wl, sym, add=False):
+    filt = sum(b * algorithmic_flops(m, n, wl["k"], wl["p"], wl["J"], wl["L"], sym, add)[0] for b, m, n in wl["groups"])
+    front = sum(b * algorithmic_flops(m, n, wl["k"], wl["p"], wl["J"], wl["L"], sym, add)[1] for b, m, n in wl["groups"])
+    return filt, front
+
+
+def oracle_sample(wl):
+    """Times the fp64 oracle, as it stands, on ONE matrix of EACH shape group of the workload (a bounded sample);
+    returns (seconds per group sample, flops per group sample, description)."""
+    import oracle
+    import torch
+    from paper_2609_21102_b200 import inputs
+    secs, fl = [], []
+    sched = oracle.schedule(schedule_of(wl["schedule"], wl["L"]))
+    for si, (b, m, n) in enumerate(wl["groups"]):
+        _, expo, top, floor = wl["recipe"]
+        G = inputs.workload_power_law(1, m, n, wl["workload"], si, expo, top, floor).to(torch.bfloat16).double().numpy()[0]
+        l = min(min(m, n), wl["k"] + wl["p"])
+        Om = inputs.sketch(1, min(m, n), l, wl["workload"], si).double().numpy()[0]
+        t0 = time.perf_counter()
+        oracle.deflated_polar(G, wl["k"], l, Om, wl["J"], sched, gamma=wl["gamma"])
+        secs.append(time.perf_counter() - t0)
+        # the oracle evaluates every product in full (no symmetric shortcut)
+        fl.append(sum(algorithmic_flops(m, n, wl["k"], wl["p"], wl["J"], wl["L"], False)))
+    what = " + ".join("1 of %d matrices %dx%d" % g for g in wl["groups"])
+    return secs, fl, what + ", full path, fp64"
+
+
+def reference_arm(args, wl, config):
+    """The oracle as the reference arm: each step runs it on one matrix of each shape group."""
+    cores = os.cpu_count() or 1
+    for _ in range(max(0, args.warmup)):
+        oracle_sample(wl)
+    times, fl, sample = [], None, ""
+    for _ in range(max(1, args.steps)):
+        secs, fl, sample = oracle_sample(wl)
+        times.append(sum(secs))
+    dt = sum(times) / len(times)
+    val = sum(fl) / dt / 1e12
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": len(times), "warmup": max(0, args.warmup), "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
+            "matrices_per_s": len(wl["groups"]) / dt,
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def measure_tf32_peak():
+    """Dense tf32 product rate of this GPU the way the bf16 peak was taken: torch.matmul 8192^3 with tf32 allowed,
+    best of 10 (the denominator of the SDP filter's roofline fraction; a library product, outside every timed path)."""
+    import torch
+    prev = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = True
+    try:
+        a = torch.randn((8192, 8192), device="cuda")
+        b = torch.randn((8192, 8192), device="cuda")
+        for _ in range(3):
+            torch.matmul(a, b)
+        best = 1e9
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            torch.matmul(a, b)
+            e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        return 2.0 * 8192 ** 3 / (best * 1e-3) / 1e12
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = prev
+
+
+def extra_polar(ctx, name, opts, device, steps=10, label=None):
+    """ms per batch, TFLOP/s (flops the method needs), matrices/s and launches of one more workload."""
+    import torch
+    wl = WORKLOADS[name]
+    groups = make_inputs(wl, device)
+    for _ in range(3):
+        run_step(ctx, wl, groups, opts)
+    l0 = ctx.defl_launch_count()
+    ms = time_steps(lambda: run_step(ctx, wl, groups, opts), steps, torch.cuda.synchronize)
+    launches = (ctx.defl_launch_count() - l0) // steps
+    st = ctx.defl_get_stage_ms(min(64, steps * len(groups)))
+    per = min(64, steps * len(groups)) / len(groups)
+    filt, front = workload_flops(wl, opts["sym"], opts["mode"] == 1)
+    out = {"workload": label or wl["label"], "ms_per_batch": ms, "tflops": (filt + front) / (ms * 1e-3) / 1e12,
+           "matrices_per_s": sum(b for b, _, _ in wl["groups"]) / (ms * 1e-3), "launches_per_batch": int(launches),
+           "stage_ms": {"rsvd": st[0] / per, "deflate_normalise": st[1] / per, "filter": st[2] / per, "restore": st[3] / per}}
+    del groups
+    torch.cuda.empty_cache()
+    return out
+
+
+def extra_sdp(ctx, peaks, device, n=4096, calls=20, warm=2):
+    """The SDP projection sequence at n = 4096 (tf32 filter): ms per projection over the deflated calls, the seven-stage
+    split, the filter + reconstruction products against a measured tf32 peak, and the Lanczos passes against HBM."""
+    import torch
+    from paper_2609_21102_b200 import inputs
+    K, k, T = 16, 8, 7
+    sched = [list(CLASSICAL)] * T
+    x, _ = inputs.sdp_first(n, heads=k, head_mag=1.0e3, device=device)
+    V = inputs.randn((n, K), inputs.seed_for(5, 0, inputs.PURPOSE_BASIS), device).float()
+    v0 = inputs.gaussian_vector(n, 5, inputs.PURPOSE_LANCZOS, device=device)
+    P = torch.empty((n, n), dtype=torch.float32, device=device)
+    times, warm_times = [], []
+    for t in range(calls):
+        X = x.float()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.defl_psd_project(X, k, V, sched, out=P, gamma=1.1, lanczos_start=v0, warmup=t < warm, exploit_symmetry=True)
+        e1.record()
+        torch.cuda.synchronize()
+        (warm_times if t < warm else times).append(e0.elapsed_time(e1))
+        x = inputs.sdp_next(x, t + 1)
+    nd = len(times)
+    st = [s / nd for s in ctx.defl_get_stage_ms(nd)]
+    names = ["block_step_rayleigh_ritz", "deflate", "lanczos_scale", "initialise", "filter", "reconstruct", "basis_update"]
+    tf32_peak = measure_tf32_peak()
+    flops = T * 3.0 * n * n * (n + 1.0) + 2.0 * n ** 3          # symmetric products once, R g(X0) in full
+    prod_ms = st[4] + st[5]
+    symv_bytes = 42.0 * 4.0 * n * n
+    times.sort()
+    return {"workload": "SDP PSD projection, fp32 storage / tf32 filter: 20 drifting symmetric %dx%d matrices, 8 eigenvalues "
+                        "+-1e3 over U(-1,1), k=8, K=16, 7 classical quintic steps, 2 warm-up calls" % (n, n),
+            "ms_per_projection": sum(times) / nd, "ms_per_projection_median": times[nd // 2],
+            "ms_per_warmup_call": sum(warm_times) / max(1, len(warm_times)),
+            "stage_ms": dict(zip(names, st)),
+            "roofline_filter": {"bound": "tensor", "kernel": "gemm_tc_kernel (tf32: X^2, W^2 polynomial, X T_t, R g(X0))",
+                                "achieved": flops / (prod_ms * 1e-3) / 1e12, "peak": tf32_peak, "unit": "TFLOP/s",
+                                "frac": flops / (prod_ms * 1e-3) / 1e12 / tf32_peak,
+                                "peak_kind": "torch.matmul 8192^3 with tf32 allowed, best of 10, this run"},
+            "roofline_lanczos": {"bound": "hbm", "kernel": "symv_kernel (42 passes over R) + lanczos_step_kernel",
+                                 "achieved": symv_bytes / (st[2] * 1e-3) / 1e9, "peak": float(peaks.get("hbm_gbs", 6650.0)),
+                                 "unit": "GB/s", "frac": symv_bytes / (st[2] * 1e-3) / 1e9 / float(peaks.get("hbm_gbs", 6650.0)),
+                                 "note": "R (67 MB) fits the 126 MB L2: passes after the first are served from it"}}
+
+
+def spawn_ranks(args):
+    """--gpus N without an outer launcher: start the N ranks here (weak-scaling replicas, one batch per rank)."""
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
@@ -241,73 +397,63 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--small", action="store_true", help="tiny workload for a quick functional check")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the other workloads, the sustained leg and the end-to-end leg")
     ap.add_argument("--no-symmetry", action="store_true", help="compute the symmetric products in full")
     ap.add_argument("--bf16-iterates", action="store_true", help="filter iterates stored in bf16 in every step (default: scaled IEEE half in the first two)")
     ap.add_argument("--half-iterates", action="store_true", help="filter iterates stored in scaled IEEE half in every step")
     ap.add_argument("--schedule", choices=["muon", "minimax"], default="muon",
                     help="muon: Muon's quintic every step; minimax: per-step minimax quintics (Polar-Express-style)")
-    ap.add_argument("--streams", type=int, default=2, help="2: one stream + context per shape group; 1: one stream")
+    ap.add_argument("--add-restore", action="store_true", help="Eq. 3's post-add (fused into the last filter product) instead of the padded entry")
+    ap.add_argument("--streams", type=int, default=2, help="2: one stream + context per shape group (the groups are independent); 1: one stream")
     ap.add_argument("--batch", type=int, default=0, help="override the matrices per shape group (profiling captures)")
     args = ap.parse_args()
-    global SYM, BF16_ITERATES, SCHEDULE, SCHEDULE_NOTE, GAMMA
-    SCHEDULE = args.schedule
-    if SCHEDULE == "minimax":
-        GAMMA = 1.1
-        SCHEDULE_NOTE = ("per-step minimax quintics (greedy Remez from [1e-3, 1], first step / 1.01): the "
-                         "Polar-Express-style mapping, coefficients computed by schedules.remez_sign_schedule")
-    SYM = not args.no_symmetry
-    BF16_ITERATES = 1 if args.bf16_iterates else (2 if args.half_iterates else 0)
+
     wl_name = "small" if args.small else "gpt2_xl"
     wl = dict(WORKLOADS[wl_name])
+    if args.schedule == "minimax":
+        wl["schedule"], wl["gamma"] = "minimax", 1.1
+        wl["label"] = wl["label"].replace("5 Muon quintic steps", "5 per-step minimax quintic steps (Polar-Express-style)")
     if args.batch > 0:
         wl["groups"] = [(args.batch, m, n) for _, m, n in wl["groups"]]
         wl["label"] += " [batch overridden to %d per group]" % args.batch
-    if SCHEDULE == "minimax":
-        wl["label"] = wl["label"].replace("5 Muon quintic steps", "5 per-step minimax quintic steps (Polar-Express-style)")
+    opts = {"sym": not args.no_symmetry, "iterates": 1 if args.bf16_iterates else (2 if args.half_iterates else 0),
+            "mode": 1 if args.add_restore else 0}
+    storage = ("bf16" if opts["iterates"] == 1 else "IEEE half scaled by 32" if (opts["iterates"] == 2 or opts["mode"] == 1)
+               else "IEEE half scaled by 32 in the first two steps, bf16 after")
+    sched_note = ("Muon quintic (3.4445, -4.7750, 2.0315) every step" if wl["schedule"] == "muon" else
+                  "per-step minimax quintics (greedy Remez from [1e-3, 1], first step / 1.01): the Polar-Express-style "
+                  "mapping, coefficients computed by schedules.remez_sign_schedule")
+    config = {"workload": wl["label"], "name": wl_name, "k": wl["k"], "oversample": wl["p"], "power_iters": wl["J"],
+              "filter_steps": wl["L"], "restore": ("additive (Eq. 3), in the last filter product" if opts["mode"] else "padded, gamma=%g" % wl["gamma"]),
+              "schedule": sched_note, "exploit_symmetry": opts["sym"],
+              "storage": "input and output bf16; filter iterates " + storage,
+              "l2": "inputs (1.2 GB per step) larger than L2; no flush"}
+
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) == 0:
+            reference_arm(args, wl, config)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
+
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    config = {"workload": wl["label"], "name": wl_name, "k": wl["k"], "oversample": wl["p"], "power_iters": wl["J"],
-              "filter_steps": wl["L"], "restore": "padded, gamma=%g" % GAMMA, "schedule": SCHEDULE_NOTE, "exploit_symmetry": SYM,
-              "storage": "input and output bf16; filter iterates " + ("bf16" if BF16_ITERATES == 1 else ("IEEE half scaled by 32" if BF16_ITERATES == 2 else "IEEE half scaled by 32 in the first two steps, bf16 after")),
-              "l2": "inputs (1.2 GB per step) larger than L2; no flush"}
-    tot_f = sum(b * sum(flops_per_matrix(m, n, wl["k"], wl["p"], wl["J"], wl["L"])) for b, m, n in wl["groups"])
-    nmat = sum(b for b, _, _ in wl["groups"])
-
-    if args.impl == "reference":
-        if rank != 0:
-            return
-        cores = os.cpu_count() or 1
-        # W untimed and K timed steps, each the oracle's full path on one 1600x1600 matrix of the batch (about 1.5 s)
-        for _ in range(max(0, args.warmup)):
-            oracle_sample(wl)
-        times = []
-        for _ in range(max(1, args.steps)):
-            dt, fl, sample = oracle_sample(wl)
-            times.append(dt)
-        dt = sum(times) / len(times)
-        val = fl / dt / 1e12
-        line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
-                "steps": len(times), "warmup": max(0, args.warmup), "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
-                "matrices_per_s": 1.0 / dt,
-                "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
-                "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
-        print(json.dumps(line))
-        return
 
     import torch
     from paper_2609_21102_b200 import binding
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
     dist = None
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.init_process_group("nccl", device_id=device)
     ctx = binding.Context(local_rank)
-    groups = make_inputs(wl, torch.device("cuda", local_rank))
     ctx.defl_set_profiling(True)
+    groups = make_inputs(wl, device)
+    ngroups = len(groups)
 
     def barrier():
         if dist is not None:
@@ -322,78 +468,100 @@ def main():
     def launch_total():
         return ctx.defl_launch_count() + (sum(c.defl_launch_count() for c, _ in lanes) if lanes else 0)
 
-    for _ in range(max(args.warmup, 3)):
-        run_step(ctx, wl, groups, lanes)
-    barrier()
-    launches0 = launch_total()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    step = lambda: run_step(ctx, wl, groups, opts, lanes)
+    filt_f, front_f = workload_flops(wl, opts["sym"], opts["mode"] == 1)
+    tot_f = filt_f + front_f
+    dense_f = sum(b * dense_filter_flops(m, n, wl["L"]) for b, m, n in wl["groups"]) + front_f
+    nmat = sum(b for b, _, _ in wl["groups"])
+
     with ClockSampler(local_rank) as clk:
+        for _ in range(max(args.warmup, 3)):
+            step()
         barrier()
-        clk.mark_start()
+        launches0 = launch_total()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        barrier()
+        t_start = time.time()
         ev[0].record()
         for i in range(args.steps):
-            run_step(ctx, wl, groups, lanes)
-            ev[i + 1].record()
+            step()
+        ev[1].record()
         barrier()
-        clk.mark_end()
-    launches = launch_total() - launches0
-    total_ms = max_over_ranks(ev[0].elapsed_time(ev[-1]), dist, "cuda")
-    ms_per_step = total_ms / args.steps
+        t_end = time.time()
+        launches = launch_total() - launches0
+        total_ms = max_over_ranks(ev[0].elapsed_time(ev[1]), dist, "cuda")
+        ms_per_step = total_ms / args.steps
+        clocks = clk.summary(t_start, t_end)
 
-    # stage split of one more (untimed) step, with the same events the library records on its stream
-    stage_tot = [0.0, 0.0, 0.0, 0.0]
-    filt_flops = 0.0        # dense count of the filter products
-    filt_executed = 0.0     # flops the tensor cores actually execute (tiles below the diagonal are skipped)
-    STAGE_REPS = 7          # median over the repetitions: a single step's split moves by several percent with the
-                            # power state, and reading the events synchronises the stream after every call
-    per_rep = []
-    for rep in range(STAGE_REPS):
-        tot = [0.0, 0.0, 0.0, 0.0]
-        for g, (b, m, n) in zip(groups, wl["groups"]):
-            ctx.defl_polar_batched(g["G"], wl["k"], wl["p"], wl["J"], sched_of(wl), out=g["out"], sketch=g["Om"],
-                                   gamma=GAMMA, exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
-            ms = ctx.defl_get_stage_ms()
-            for i in range(min(4, len(ms))):
-                tot[i] += ms[i]
-            if rep == 0:
-                filt_flops += b * flops_per_matrix(m, n, wl["k"], wl["p"], wl["J"], wl["L"])[0]
-                filt_executed += b * executed_filter_flops(m, n, wl["L"], SYM)
-        per_rep.append(tot)
-    for i in range(4):
-        vals = sorted(r[i] for r in per_rep)
-        stage_tot[i] = vals[len(vals) // 2]
-    plain_ms = 0.0
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for g in groups:
-        ctx.defl_polar_batched(g["G"], 0, 0, 0, sched_of(wl), out=g["out"], exploit_symmetry=SYM, bf16_iterates=BF16_ITERATES)
-    e1.record()
-    torch.cuda.synchronize()
-    plain_ms = e0.elapsed_time(e1)
+        # Stage split and the dominant kernel's time: a second timed region of the same K steps on ONE stream, where the
+        # events the library records between the stages of every call bracket exactly that stage's kernels (with one
+        # stream per shape group the stages of the two groups interleave and a per-stage time is not defined).
+        if lanes:
+            for _ in range(2):
+                run_step(ctx, wl, groups, opts, None)
+            barrier()
+            es = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+            es[0].record()
+            for i in range(args.steps):
+                run_step(ctx, wl, groups, opts, None)
+            es[1].record()
+            barrier()
+            one_stream_ms = max_over_ranks(es[0].elapsed_time(es[1]), dist, "cuda") / args.steps
+        else:
+            one_stream_ms = ms_per_step
+        ncalls = min(64, args.steps * ngroups) // ngroups * ngroups
+        st = ctx.defl_get_stage_ms(ncalls)
+        stage_ms = [s / (ncalls / ngroups) for s in st[:4]]
+        stage_src = ("CUDA events recorded by the library on its stream inside a timed region of %d steps on one stream "
+                     "(%.3f ms per step there)" % (ncalls // ngroups, one_stream_ms))
+
+        sustained = None
+        plain_ms = None
+        if not args.no_extras:
+            # sustained leg: the same step back to back for at least 3 s (the board settles at its power cap)
+            barrier()
+            s0 = time.time()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            n_sus = 0
+            while True:
+                for _ in range(10):
+                    step()
+                n_sus += 10
+                torch.cuda.synchronize()
+                if time.time() - s0 >= 3.0:
+                    break
+            e1.record()
+            barrier()
+            s1 = time.time()
+            sus_ms = max_over_ranks(e0.elapsed_time(e1) / n_sus, dist, "cuda")
+            sustained = {"ms_per_step": sus_ms, "steps": n_sus, "tflops": aggregate_throughput(tot_f, world, sus_ms) / 1e12,
+                         "clocks": clk.summary(s0 + 0.5, s1)}
+        # the plain (undeflated) filter of the same batch, for the deflation overhead
+        plain = lambda: [ctx.defl_polar_batched(g["G"], 0, 0, 0, schedule_of(wl["schedule"], wl["L"]), out=g["out"],
+                                                exploit_symmetry=opts["sym"], bf16_iterates=opts["iterates"]) for g in groups]
+        plain()
+        plain_ms = time_steps(plain, 5, torch.cuda.synchronize)
 
     # end to end through the host-buffer entry point (pinned host tensors, copies inside the timed region)
     e2e = None
-    if rank == 0 or world > 1:
+    if not args.no_extras:
+        sched = schedule_of(wl["schedule"], wl["L"])
         hG = [g["G"].cpu().pin_memory() for g in groups]
         hO = [torch.empty_like(h).pin_memory() for h in hG]
-        def e2e_group(c, h, o, g, stream=None):
-            if stream is None:
-                c.defl_polar_batched_host(h, o, wl["k"], wl["p"], wl["J"], sched_of(wl), sketch=g["Om"], gamma=GAMMA,
-                                          exploit_symmetry=SYM)
-            else:
-                torch.cuda.set_device(local_rank)
-                with torch.cuda.stream(stream):
-                    c.defl_polar_batched_host(h, o, wl["k"], wl["p"], wl["J"], sched_of(wl), sketch=g["Om"],
-                                              gamma=GAMMA, exploit_symmetry=SYM)
+        e2e_ctx = [binding.Context(local_rank) for _ in groups]
+        e2e_streams = [torch.cuda.Stream() for _ in groups]
+
+        def e2e_group(c, s, h, o, g):
+            torch.cuda.set_device(local_rank)
+            with torch.cuda.stream(s):
+                c.defl_polar_batched_host(h, o, wl["k"], wl["p"], wl["J"], sched, sketch=g["Om"], gamma=wl["gamma"],
+                                          exploit_symmetry=opts["sym"], restore_mode=opts["mode"])
 
         def e2e_step():
-            # the call blocks until its output sits in host memory; with one context per shape group the groups
-            # run from host threads of their own, so that one group's copies overlap the other's computation
-            if not lanes:
-                for h, o, g in zip(hG, hO, groups):
-                    e2e_group(ctx, h, o, g)
-                return
-            ts = [threading.Thread(target=e2e_group, args=(c, h, o, g, s)) for (c, s), h, o, g in zip(lanes, hG, hO, groups)]
+            # the call blocks until its output sits in host memory; the shape groups run from host threads of their
+            # own (one context each), so that one group's copies overlap the other's computation
+            ts = [threading.Thread(target=e2e_group, args=(c, s, h, o, g)) for c, s, h, o, g in zip(e2e_ctx, e2e_streams, hG, hO, groups)]
             for t in ts:
                 t.start()
             for t in ts:
@@ -409,42 +577,77 @@ def main():
         nbytes = sum(h.numel() * h.element_size() for h in hG)
         e2e = {"value": aggregate_throughput(tot_f, world, e2e_ms) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes}
+        del hG, hO, e2e_ctx
 
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
+
     peaks, peaks_kind = load_peaks()
+    burst = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
+    sust = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
     value = aggregate_throughput(tot_f, world, ms_per_step) / 1e12
-    filt_ms = stage_tot[2]
-    n_filter_launches = 3 * wl["L"] * len(groups)
-    # achieved = flops the kernel really executes / its time (no credit for skipped symmetric tiles)
-    ach = filt_executed / (filt_ms * 1e-3) / 1e12 if filt_ms > 0 else None
-    ach_dense = filt_flops / (filt_ms * 1e-3) / 1e12 if filt_ms > 0 else None
-    peak = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
+    filt_ms = stage_ms[2]
+    n_filter_launches = 3 * wl["L"] * ngroups
+    ach = filt_f / (filt_ms * 1e-3) / 1e12 if filt_ms > 0 else None
+    sm_mhz = clocks.get("sm_mhz") or 0.0
+    # a short timed region runs near the maximum clock (compare with the burst peak), a long one at the power cap
+    # (compare with the sustained peak): both fractions are given, and time x clock so that runs at different clocks compare
     roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel (filter chain: X X^T, A^2 polynomial, B X)",
-                "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": (ach / peak) if ach else None,
-                "peak_kind": "bf16_tflops_sustained, of %s" % peaks_kind,
-                "frac_of_burst": (ach / float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))) if ach else None,
+                "achieved": ach, "peak": burst, "unit": "TFLOP/s", "frac": (ach / burst) if ach else None,
+                "peak_kind": "bf16_tflops (burst), of %s" % peaks_kind,
+                "frac_of_sustained_peak": (ach / sust) if ach else None,
+                "flops": "flops the method needs (symmetric products once); per launch: %.4g" % (filt_f / n_filter_launches),
                 "launches_per_step": n_filter_launches, "avg_launch_ms": filt_ms / n_filter_launches,
-                "flops_per_launch_avg": filt_executed / n_filter_launches,
-                "dense_equivalent_tflops": ach_dense,
+                "stage_source": stage_src,
+                "ms_x_mhz": filt_ms * sm_mhz,
+                "dense_equivalent_tflops": sum(b * dense_filter_flops(m, n, wl["L"]) for b, m, n in wl["groups"]) / (filt_ms * 1e-3) / 1e12,
                 "traffic": FILTER_TRAFFIC_BYTES_PER_LAUNCH if (wl_name == "gpt2_xl" and args.batch == 0) else None,
                 "traffic_unit": "bytes per launch (ncu, 8-matrix capture scaled to the batch)"}
+    front_ms = stage_ms[0] + stage_ms[1] + stage_ms[3]
     line = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
+            "flops_convention": "value = flops the method needs / time (symmetric products counted once); dense_equivalent_tflops counts them in full",
+            "dense_equivalent_tflops": aggregate_throughput(dense_f, world, ms_per_step) / 1e12,
             "matrices_per_s": world * nmat / (ms_per_step * 1e-3),
-            "pct_bf16_peak_sustained": 100.0 * value / world / peak,
-            "stage_ms": {"rsvd": stage_tot[0], "deflate_normalise": stage_tot[1], "filter": stage_tot[2],
-                         "restore": stage_tot[3]},
-            "deflation_overhead_frac": (ms_per_step - plain_ms) / ms_per_step if ms_per_step > 0 else None,
+            "pct_bf16_peak": {"burst": 100.0 * value / world / burst, "sustained": 100.0 * value / world / sust},
+            "stage_ms": {"rsvd": stage_ms[0], "deflate_normalise": stage_ms[1], "filter": stage_ms[2], "restore": stage_ms[3],
+                         "one_stream_ms_per_step": one_stream_ms},
+            "deflation_overhead_frac": (ms_per_step - plain_ms) / ms_per_step if plain_ms else None,
+            "front_end_frac_of_step": front_ms / sum(stage_ms) if sum(stage_ms) > 0 else None,
             "plain_filter_ms": plain_ms,
-            "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clk.summary()}
+            "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "sustained": sustained}
+
+    if not args.no_extras and wl_name == "gpt2_xl" and args.batch == 0:
+        extras = {}
+        try:
+            extras["gpt2_small"] = extra_polar(ctx, "gpt2_small", opts, device, steps=20)
+            extras["gpt2_medium_large"] = extra_polar(ctx, "gpt2_medium_large", opts, device, steps=10)
+            del groups
+            torch.cuda.empty_cache()
+            xl_minimax = dict(WORKLOADS["gpt2_xl"], schedule="minimax", gamma=1.1)
+            WORKLOADS["_xl_minimax"] = xl_minimax
+            extras["gpt2_xl_minimax_schedule"] = extra_polar(ctx, "_xl_minimax", opts, device, steps=10,
+                                                             label="GPT-2-XL batch, per-step minimax schedule, gamma=1.1")
+            extras["gpt2_xl_add_restore"] = extra_polar(ctx, "gpt2_xl", dict(opts, mode=1), device, steps=10,
+                                                        label="GPT-2-XL batch, additive restore (Eq. 3) in the last filter product")
+            extras["sdp_4096"] = extra_sdp(ctx, peaks, device)
+        except Exception as e:      # an extra that fails must not take the headline with it
+            extras["error"] = repr(e)
+        line["extras"] = extras
+
     if not args.no_cpu_baseline:
-        dt, fl, sample = oracle_sample(wl)
-        line["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count() or 1,
-                                "kind": "oracle", "sample": sample, "seconds": dt, "matrices_per_s": 1.0 / dt}
+        secs, fl, sample = oracle_sample(wl)
+        # whole batch at the oracle's measured seconds per matrix of each shape (every matrix of a shape costs the same)
+        batch_s = sum(b * s for (b, _, _), s in zip(wl["groups"], secs))
+        batch_f = sum(b * f for (b, _, _), f in zip(wl["groups"], fl))
+        line["cpu_baseline"] = {"value": batch_f / batch_s / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count() or 1,
+                                "kind": "oracle", "sample": sample,
+                                "seconds_per_matrix": {"%dx%d" % (m, n): s for (_, m, n), s in zip(wl["groups"], secs)},
+                                "extrapolated": "batch figure = measured seconds per matrix of each shape x matrices of that shape",
+                                "batch_seconds_extrapolated": batch_s, "matrices_per_s": nmat / batch_s}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

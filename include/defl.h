@@ -16,8 +16,8 @@
  *   - All work is enqueued on the context's stream and the call returns without synchronising
  *     (the only exception: growing the scratch memory synchronises the device).
  *   - Return value: 0 = OK, < 0 = caller error, nothing was launched (see defl_status_string).
- *     Numerical events (Cholesky breakdown, Jacobi sweep cap, zero residual, a device-side wait
- *     that ran out) are reported per matrix in defl_info.status, never by a trap.
+ *     Numerical events (Cholesky breakdown, Jacobi sweep cap, zero residual, a non-finite result, a
+ *     device-side wait that ran out) are reported per matrix in defl_info.status, never by a trap.
  *   - There is no CPU fallback: without a CUDA device every compute entry point returns
  *     DEFL_ERR_CUDA.
  */
@@ -59,8 +59,12 @@ extern "C" {
 /* per-matrix status bits in defl_info.status */
 #define DEFL_ST_CHOL_SHIFT 1   /* a Cholesky pivot was not positive; factorised with a diagonal shift */
 #define DEFL_ST_JACOBI_CAP 2   /* the Jacobi eigensolver hit its sweep cap */
-#define DEFL_ST_ZERO_RESIDUAL 4 /* ||R||_F was zero or not finite: residual treated as zero */
+#define DEFL_ST_ZERO_RESIDUAL 4 /* ||R||_F was zero, not finite, or (bf16 storage, where it is taken as
+                                  sqrt(||G||_F^2 - sum s_i^2)) below 1e-3 ||G||_F: residual treated as zero */
 #define DEFL_ST_DEVICE_WAIT 8  /* a bounded device-side wait ran out; the output is not valid */
+#define DEFL_ST_NONFINITE 16   /* the result of this matrix holds Inf or NaN: its input did, or an iterate left the range
+                                  of its storage format (scaled IEEE half iterates overflow beyond about 2e3, which a
+                                  normalised input reaches only with a schedule that diverges); polar calls only */
 
 #define DEFL_MAX_L 64 /* largest sketch width k + oversample (and PSD basis width K) */
 #define DEFL_MAX_STEPS 32 /* largest filter depth L (or T) */
@@ -109,7 +113,11 @@ typedef struct defl_info {
 } defl_info;
 
 /* Context. `device` is a CUDA ordinal. defl_create makes no assumption about the current device
- * and restores it. Not thread safe: one context per host thread or external locking. */
+ * and restores it. Not thread safe: one context per host thread or external locking.
+ * Environment overrides are read here, once, and never on the call path: DEFL_TC_BN, DEFL_TC_TILE_M, DEFL_TC_STAGES,
+ * DEFL_TC_KSUB, DEFL_TC_PAIR, DEFL_TC_PAIR_MIN_N, DEFL_TC_DYNAMIC, DEFL_TC_AUX_PREFETCH, DEFL_TC_DEBUG (tile forms of
+ * the tensor engine, for experiments and tests), DEFL_TC_WAIT_MS (limit of the device-side waits, default 2000),
+ * DEFL_NO_TRANSPOSED_APPLY, DEFL_HOST_CHUNKS, DEFL_JACOBI_SWEEPS (sweep cap of the Jacobi core, default 40). */
 int defl_create(defl_ctx** out, int device);
 int defl_destroy(defl_ctx* ctx);
 int defl_set_stream(defl_ctx* ctx, void* cuda_stream); /* cudaStream_t; NULL = default stream */
@@ -117,6 +125,16 @@ int defl_set_stream(defl_ctx* ctx, void* cuda_stream); /* cudaStream_t; NULL = d
 /* Bytes of context scratch a polar / PSD call of this shape needs (what the context will hold). */
 size_t defl_polar_workspace_bytes(int b, int m, int n, int dtype, int k, int oversample);
 size_t defl_psd_workspace_bytes(int n, int K);
+
+/* The paper gives the estimation window and the oversampling as ratios of the short side (Algorithm 3, line 1:
+ * r = ceil(w m), r' = min{m, r + ceil(delta m)}; Algorithm 2: r = ceil(w n), K = ceil(w' n)). These two calls turn
+ * the ratios into the counts the compute calls take: *k = r, *oversample = r' - r (polar, m the short side of an
+ * m x n matrix; r is capped at m - 1), and *k = r, *K = ceil(w' n) (PSD; r is capped at K). Host arithmetic only.
+ * With opts->tau > 0 the window is what the gate looks at and k_used reports how many of the r were deflated.
+ * Returns DEFL_ERR_RANK when the widths exceed DEFL_MAX_L (the counts are still written), DEFL_ERR_ARG for negative
+ * ratios, non-positive sizes or null pointers. */
+int defl_polar_window(int m, int n, float w, float delta, int* k, int* oversample);
+int defl_psd_window(int n, float w, float w_prime, int* k, int* K);
 
 /* Deflated polar factor of a batch (Algorithm 3 then Algorithm 1, fixed-k reading).
  *   G    [b,m,n] dtype, not modified.         out [b,m,n] dtype, must not overlap G.
@@ -237,7 +255,9 @@ int defl_frobenius_norms_noalloc(const void* X, int dtype, int b, long long coun
  * A element (i,kk) is A[i*sa_i + kk*sa_k], B element (kk,j) is B[kk*sb_k + j*sb_j]; C is row-major [M,N].
  * in_dtype / out_dtype are DEFL_BF16 or DEFL_F32; strides in elements. exploit_symmetry: bit 0 = the product is
  * symmetric (upper tiles computed and mirrored); bit 1 = the product is written transposed, C row-major [N,M]
- * (tensor engine only; DEFL_ERR_UNSUPPORTED otherwise). */
+ * (tensor engine only; DEFL_ERR_UNSUPPORTED otherwise); bit 2 = test of the bounded waits (tensor engine, outputs
+ * of at most 128 rows): the first pipeline step of every CTA's first tile is never copied, so the wait for it runs
+ * out after the context's wait limit, C is not written and defl_device_wait_status reports DEFL_ST_DEVICE_WAIT. */
 int defl_debug_gemm(defl_ctx* ctx, int engine, int batch, int M, int N, int K,
                     const void* A, long long sa_i, long long sa_k, long long batch_a,
                     const void* B, long long sb_k, long long sb_j, long long batch_b,
@@ -250,9 +270,20 @@ int defl_debug_gemm(defl_ctx* ctx, int engine, int batch, int M, int N, int K,
  * 2 Lanczos scale, 3 initialisation, 4 filter, 5 reconstruction, 6 basis update. */
 int defl_set_profiling(defl_ctx* ctx, int enabled);
 int defl_get_stage_ms(defl_ctx* ctx, float* ms, int cap);
+/* The same durations added up over the last `ncalls` calls of the context (at most 64 are kept), so that a timed
+ * loop can be split into stages afterwards without a synchronisation between its calls. */
+int defl_get_stage_ms_sum(defl_ctx* ctx, float* ms, int cap, int ncalls);
 
 /* Number of kernels the library launched on this context since creation. */
 long long defl_launch_count(defl_ctx* ctx);
+
+/* The tensor engine's wait word of this context: every device-side wait of its kernels (on a copy, on a free
+ * pipeline stage, on an accumulator) is bounded; one that runs out sets DEFL_ST_DEVICE_WAIT in this word, the kernel
+ * stops waiting, lets its copies land, frees its tensor memory and returns. defl_polar_batched, defl_psd_project
+ * and the calls built on them clear the word when they start and fold it into defl_info.status when they end; this
+ * call is for the others (defl_debug_gemm). It synchronises the context's stream, returns the word (>= 0, or a
+ * negative DEFL_ERR_*), and clears it when `clear` is non-zero. No counterpart in the paper. */
+int defl_device_wait_status(defl_ctx* ctx, int clear);
 
 const char* defl_status_string(int code);
 const char* defl_last_error(defl_ctx* ctx); /* text of the last CUDA failure, "" if none */

@@ -17,7 +17,7 @@ BF16, F32, F16 = 0, 1, 2
 RESTORE_PADDED, RESTORE_ADD = 0, 1
 NORM_LANCZOS, NORM_FROBENIUS = 0, 1
 ENGINE_AUTO, ENGINE_SIMT, ENGINE_TENSOR = 0, 1, 2
-ST_CHOL_SHIFT, ST_JACOBI_CAP, ST_ZERO_RESIDUAL, ST_DEVICE_WAIT = 1, 2, 4, 8
+ST_CHOL_SHIFT, ST_JACOBI_CAP, ST_ZERO_RESIDUAL, ST_DEVICE_WAIT, ST_NONFINITE = 1, 2, 4, 8, 16
 MAX_L, MAX_STEPS = 64, 32
 
 MUON_QUINTIC = (3.4445, -4.7750, 2.0315)
@@ -25,8 +25,9 @@ CLASSICAL_QUINTIC = (1.875, -1.25, 0.375)
 
 EXPORTS = [
     "defl_create", "defl_destroy", "defl_set_stream", "defl_polar_workspace_bytes", "defl_psd_workspace_bytes",
-    "defl_polar_batched", "defl_polar_batched_host", "defl_muon_step_batched", "defl_brsvd_batched", "defl_psd_project", "defl_admm_diag_sdp", "defl_fill_gaussian", "defl_debug_gemm",
-    "defl_frobenius_norms_noalloc", "defl_set_profiling", "defl_get_stage_ms", "defl_launch_count", "defl_status_string", "defl_last_error",
+    "defl_polar_window", "defl_psd_window", "defl_polar_batched", "defl_polar_batched_host", "defl_muon_step_batched", "defl_brsvd_batched", "defl_psd_project", "defl_admm_diag_sdp", "defl_fill_gaussian", "defl_debug_gemm",
+    "defl_frobenius_norms_noalloc", "defl_set_profiling", "defl_get_stage_ms", "defl_get_stage_ms_sum", "defl_launch_count", "defl_device_wait_status",
+    "defl_status_string", "defl_last_error",
 ]
 
 
@@ -57,6 +58,10 @@ def lib():
         L.defl_polar_workspace_bytes.argtypes = [ctypes.c_int] * 6
         L.defl_psd_workspace_bytes.restype = ctypes.c_size_t
         L.defl_psd_workspace_bytes.argtypes = [ctypes.c_int] * 2
+        L.defl_polar_window.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_float, ctypes.c_float,
+                                        ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
+        L.defl_psd_window.argtypes = [ctypes.c_int, ctypes.c_float, ctypes.c_float,
+                                      ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
         L.defl_polar_batched.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 7 + [
             ctypes.POINTER(ctypes.c_float), ctypes.c_int, ctypes.POINTER(DeflOpts), ctypes.POINTER(DeflInfo)]
         L.defl_polar_batched_host.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 7 + [
@@ -80,8 +85,10 @@ def lib():
                                       ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_float, ctypes.c_int]
         L.defl_set_profiling.argtypes = [ctypes.c_void_p, ctypes.c_int]
         L.defl_get_stage_ms.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_float), ctypes.c_int]
+        L.defl_get_stage_ms_sum.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_float), ctypes.c_int, ctypes.c_int]
         L.defl_launch_count.restype = ctypes.c_longlong
         L.defl_launch_count.argtypes = [ctypes.c_void_p]
+        L.defl_device_wait_status.argtypes = [ctypes.c_void_p, ctypes.c_int]
         L.defl_status_string.restype = ctypes.c_char_p
         L.defl_status_string.argtypes = [ctypes.c_int]
         L.defl_last_error.restype = ctypes.c_char_p
@@ -124,6 +131,24 @@ def _schedule(coeffs, steps=None):
     flat = [float(x) for x in c.reshape(-1).tolist()]
     arr = (ctypes.c_float * max(len(flat), 1))(*flat)
     return arr, c.shape[0]
+
+
+def defl_polar_window(m, n, w, delta):
+    """(k, oversample) from the paper's ratios: k = ceil(w min(m,n)), oversample = min(min(m,n), k + ceil(delta min(m,n))) - k."""
+    k, p = ctypes.c_int(), ctypes.c_int()
+    rc = lib().defl_polar_window(m, n, w, delta, ctypes.byref(k), ctypes.byref(p))
+    if rc != 0:
+        raise DeflError(rc)
+    return k.value, p.value
+
+
+def defl_psd_window(n, w, w_prime):
+    """(k, K) from the paper's ratios: k = ceil(w n), K = ceil(w' n)."""
+    k, K = ctypes.c_int(), ctypes.c_int()
+    rc = lib().defl_psd_window(n, w, w_prime, ctypes.byref(k), ctypes.byref(K))
+    if rc != 0:
+        raise DeflError(rc)
+    return k.value, K.value
 
 
 class Context:
@@ -334,7 +359,7 @@ class Context:
         return dst
 
     def defl_debug_gemm(self, A, B, trans_a=False, trans_b=False, engine=ENGINE_AUTO, out_dtype=None, alpha=1.0,
-                        exploit_symmetry=False, transpose_out=False):
+                        exploit_symmetry=False, transpose_out=False, withhold_first_step=False):
         """C[b] = alpha * op(A[b]) op(B[b]); op = transpose of the stored matrix when the flag is set. With
         transpose_out the engine writes the product transposed: the result has shape [b, N, M]."""
         _dev(A, "A"), _dev(B, "B")
@@ -357,20 +382,28 @@ class Context:
         rc = lib().defl_debug_gemm(self._h, engine, b, M, N, K, _ptr(A), sa_i, sa_k, A.shape[1] * A.shape[2],
                                    _ptr(B), sb_k, sb_j, B.shape[1] * B.shape[2], _ptr(C), _dtype_code(A),
                                    {torch.bfloat16: BF16, torch.float16: F16}.get(out_dtype, F32), alpha,
-                                   int(bool(exploit_symmetry)) | (2 if transpose_out else 0))
+                                   int(bool(exploit_symmetry)) | (2 if transpose_out else 0) | (4 if withhold_first_step else 0))
         self._check(rc)
         return C
 
     def defl_set_profiling(self, enabled):
         lib().defl_set_profiling(self._h, int(bool(enabled)))
 
-    def defl_get_stage_ms(self):
+    def defl_get_stage_ms(self, ncalls=1):
+        """Stage durations (ms) of the last call, or their sums over the last `ncalls` calls; synchronises."""
         buf = (ctypes.c_float * 16)()
-        n = lib().defl_get_stage_ms(self._h, buf, 16)
+        n = lib().defl_get_stage_ms_sum(self._h, buf, 16, int(ncalls))
         return [buf[i] for i in range(max(n, 0))]
 
     def defl_launch_count(self):
         return int(lib().defl_launch_count(self._h))
+
+    def defl_device_wait_status(self, clear=True):
+        """The tensor engine's wait word (DEFL_ST_DEVICE_WAIT if a bounded device-side wait ran out); synchronises."""
+        rc = lib().defl_device_wait_status(self._h, int(bool(clear)))
+        if rc < 0:
+            self._check(rc)
+        return rc
 
     def polar_workspace_bytes(self, b, m, n, dtype, k, oversample):
         return int(lib().defl_polar_workspace_bytes(b, m, n, BF16 if dtype == torch.bfloat16 else F32, k, oversample))

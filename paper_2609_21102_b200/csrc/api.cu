@@ -38,9 +38,17 @@ int ctx_reserve(defl_ctx* c, size_t bytes) {
   return DEFL_OK;
 }
 
+void ctx_profile_begin(defl_ctx* c) {
+  if (!c->profiling || !c->marks_ready) return;
+  ++c->call_seq;
+  c->n_marks[c->call_seq % DEFL_PROFILE_CALLS] = 0;
+}
+
 void ctx_stage_mark(defl_ctx* c) {
-  if (!c->profiling || c->n_marks >= DEFL_MAX_MARKS) return;
-  cudaEventRecord(c->marks[c->n_marks++], c->stream);
+  if (!c->profiling || !c->marks_ready || c->call_seq == 0) return;
+  const int slot = (int)(c->call_seq % DEFL_PROFILE_CALLS);
+  if (c->n_marks[slot] >= DEFL_MAX_MARKS) return;
+  cudaEventRecord(c->marks[slot][c->n_marks[slot]++], c->stream);
 }
 
 // Which engine a product runs on. AUTO sends bf16 products to the tensor cores and keeps fp32
@@ -59,14 +67,14 @@ int run_gemm(defl_ctx* c, const GemmDesc& g, int engine, const char* what) {
     return DEFL_ERR_UNSUPPORTED;
   }
   cudaError_t e;
-  if (tc) e = gemm_tc_launch(g, c->stream, c->wait_status, c->num_sms, &c->launches);
+  if (tc) e = gemm_tc_launch(g, c->stream, c->wait_status, c->num_sms, &c->launches, &c->tc_knobs, &c->tm_cache);
   else e = gemm_simt_launch(g, c->stream, &c->launches);
   if (ctx_fail(c, e, what)) return DEFL_ERR_CUDA;
   return DEFL_OK;
 }
 
-int partials_per_batch(const GemmDesc& g, int engine) {
-  if (use_tensor_engine(g, engine)) return gemm_tc_partials_per_batch(g);
+int partials_per_batch(defl_ctx* c, const GemmDesc& g, int engine) {
+  if (use_tensor_engine(g, engine)) return gemm_tc_partials_per_batch(g, &c->tc_knobs);
   return gemm_simt_partials_per_batch(g);
 }
 
@@ -236,7 +244,7 @@ int run_brsvd(defl_ctx* c, const void* G, int b, int m, int n, int dtype, int l,
                                      w.gram, c->stream, &c->launches), "gram core"))
     return DEFL_ERR_CUDA;
   if (ctx_fail(c, jacobi_eig_launch(w.gram, fused_num_chunks(ms, b), b, l, 0, w.sv, w.E, w.Es, w.status, c->stream,
-                                    &c->launches), "jacobi"))
+                                    &c->launches, c->knobs.jacobi_sweeps), "jacobi"))
     return DEFL_ERR_CUDA;
   if (k_keep > 0) {
     // U = Q E (long side), V = (Q^T A)^T E diag(1/s) (short side); keep the leading k_keep columns
@@ -277,14 +285,22 @@ int defl_create(defl_ctx** out, int device) {
   if (!c) return DEFL_ERR_CUDA;
   memset(c, 0, sizeof(*c));
   c->device = device;
+  // every environment override is read here, once: nothing on the call path looks at the environment
+  c->tc_knobs = tc_knobs_from_env();
+  c->knobs.transposed_apply = getenv("DEFL_NO_TRANSPOSED_APPLY") ? 0 : 1;
+  c->knobs.host_chunks = getenv("DEFL_HOST_CHUNKS") ? atoi(getenv("DEFL_HOST_CHUNKS")) : 0;
+  c->knobs.jacobi_sweeps = getenv("DEFL_JACOBI_SWEEPS") ? atoi(getenv("DEFL_JACOBI_SWEEPS")) : 0;
   cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device);
   int ok = 1;
   if (cudaMalloc(&c->wait_status, 2 * sizeof(int)) != cudaSuccess) ok = 0;      // status word, tile counter
   if (ok) cudaMemset(c->wait_status, 0, 2 * sizeof(int));
-  for (int i = 0; ok && i < DEFL_MAX_MARKS; ++i)
-    if (cudaEventCreate(&c->marks[i]) != cudaSuccess) ok = 0;
+  if (!ok) {      // release whatever was created before the failure
+    if (c->wait_status) cudaFree(c->wait_status);
+    cudaSetDevice(prev);
+    delete c;
+    return DEFL_ERR_CUDA;
+  }
   cudaSetDevice(prev);
-  if (!ok) { delete c; return DEFL_ERR_CUDA; }
   *out = c;
   return DEFL_OK;
 }
@@ -304,8 +320,9 @@ int defl_destroy(defl_ctx* c) {
     for (int i = 0; i < DEFL_HOST_MAX_CHUNKS; ++i) { cudaEventDestroy(c->chunk_in[i]); cudaEventDestroy(c->chunk_done[i]); }
   }
   if (c->wait_status) cudaFree(c->wait_status);
-  for (int i = 0; i < DEFL_MAX_MARKS; ++i)
-    if (c->marks[i]) cudaEventDestroy(c->marks[i]);
+  for (int r = 0; r < DEFL_PROFILE_CALLS; ++r)
+    for (int i = 0; i < DEFL_MAX_MARKS; ++i)
+      if (c->marks[r][i]) cudaEventDestroy(c->marks[r][i]);
   cudaSetDevice(prev);
   delete c;
   return DEFL_OK;
@@ -327,20 +344,88 @@ size_t defl_polar_workspace_bytes(int b, int m, int n, int dtype, int k, int ove
 
 int defl_set_profiling(defl_ctx* c, int enabled) {
   if (!c) return DEFL_ERR_ARG;
+  if (enabled && !c->marks_ready) {
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaSetDevice(c->device);
+    bool ok = true;
+    for (int r = 0; ok && r < DEFL_PROFILE_CALLS; ++r)
+      for (int i = 0; ok && i < DEFL_MAX_MARKS; ++i) ok = cudaEventCreate(&c->marks[r][i]) == cudaSuccess;
+    cudaSetDevice(prev);
+    if (!ok) { ctx_fail(c, cudaErrorUnknown, "events for stage timing"); return DEFL_ERR_CUDA; }
+    c->marks_ready = true;
+  }
   c->profiling = enabled != 0;
   return DEFL_OK;
 }
 
-int defl_get_stage_ms(defl_ctx* c, float* ms, int cap) {
-  if (!c || !ms) return DEFL_ERR_ARG;
-  if (c->n_marks < 2) return 0;
+int defl_get_stage_ms_sum(defl_ctx* c, float* ms, int cap, int ncalls) {
+  if (!c || !ms || ncalls < 1) return DEFL_ERR_ARG;
+  if (!c->marks_ready || c->call_seq == 0) return 0;
+  if (ncalls > DEFL_PROFILE_CALLS) ncalls = DEFL_PROFILE_CALLS;
+  if ((long long)ncalls > c->call_seq) ncalls = (int)c->call_seq;
   cudaStreamSynchronize(c->stream);
-  const int n = c->n_marks - 1;
-  for (int i = 0; i < n && i < cap; ++i) cudaEventElapsedTime(&ms[i], c->marks[i], c->marks[i + 1]);
-  return n;
+  int n = 0;
+  for (int i = 0; i < cap; ++i) ms[i] = 0.f;
+  for (int q = 0; q < ncalls; ++q) {
+    const int slot = (int)((c->call_seq - q) % DEFL_PROFILE_CALLS);
+    const int ns = c->n_marks[slot] - 1;
+    if (ns > n) n = ns;
+    for (int i = 0; i < ns && i < cap; ++i) {
+      float t = 0.f;
+      cudaEventElapsedTime(&t, c->marks[slot][i], c->marks[slot][i + 1]);
+      ms[i] += t;
+    }
+  }
+  return n < 0 ? 0 : n;
 }
 
+int defl_get_stage_ms(defl_ctx* c, float* ms, int cap) { return defl_get_stage_ms_sum(c, ms, cap, 1); }
+
 long long defl_launch_count(defl_ctx* c) { return c ? c->launches : 0; }
+
+int defl_device_wait_status(defl_ctx* c, int clear) {
+  if (!c) return DEFL_ERR_ARG;
+  cudaSetDevice(c->device);
+  int word = 0;
+  if (ctx_fail(c, cudaStreamSynchronize(c->stream), "synchronize") ||
+      ctx_fail(c, cudaMemcpy(&word, c->wait_status, sizeof(int), cudaMemcpyDeviceToHost), "read status word"))
+    return DEFL_ERR_CUDA;
+  if (clear && word && ctx_fail(c, cudaMemset(c->wait_status, 0, sizeof(int)), "clear status word")) return DEFL_ERR_CUDA;
+  return word;
+}
+
+// Window sizes from the paper's ratios (host arithmetic only).
+// (a ratio arrives as a float: 0.025f * 640 is 16.0000002, which must count as 16, so the product is taken two parts
+// in a million short before it is rounded up)
+static int ceil_ratio(float ratio, int dim) {
+  const double v = (double)ratio * (double)dim * (1.0 - 2e-6);
+  int c = (int)v;
+  if ((double)c < v) ++c;
+  return c;
+}
+
+int defl_polar_window(int m, int n, float w, float delta, int* k, int* oversample) {
+  if (m <= 0 || n <= 0 || !(w >= 0.f) || !(delta >= 0.f) || !k || !oversample) return DEFL_ERR_ARG;
+  const int ms = m < n ? m : n;
+  int r = ceil_ratio(w, ms);
+  if (r >= ms) r = ms - 1;                       // at least one component stays in the residual
+  int rp = r + ceil_ratio(delta, ms);
+  if (rp > ms) rp = ms;
+  *k = r;
+  *oversample = rp - r;
+  return rp > DEFL_MAX_L ? DEFL_ERR_RANK : DEFL_OK;
+}
+
+int defl_psd_window(int n, float w, float w_prime, int* k, int* K) {
+  if (n <= 0 || !(w >= 0.f) || !(w_prime >= 0.f) || !k || !K) return DEFL_ERR_ARG;
+  int r = ceil_ratio(w, n), kk = ceil_ratio(w_prime, n);
+  if (kk > n) kk = n;
+  if (r > kk) r = kk;
+  *k = r;
+  *K = kk;
+  return kk > DEFL_MAX_L ? DEFL_ERR_RANK : DEFL_OK;
+}
 
 const char* defl_status_string(int code) {
   switch (code) {
@@ -376,6 +461,7 @@ int defl_debug_gemm(defl_ctx* c, int engine, int batch, int M, int N, int K, con
   g.C = C; g.ldc = N; g.batch_c = (long long)M * N; g.out_dtype = out_dtype;
   g.epilogue = EPI_STORE; g.alpha = alpha; g.symmetric = (exploit_symmetry & 1) ? 1 : 0;
   if (exploit_symmetry & 2) { g.transpose_out = 1; g.ldc = M; }
+  if (exploit_symmetry & 4) g.debug_hold_stage = 1;
   return run_gemm(c, g, engine, "debug gemm");
 }
 
@@ -474,10 +560,12 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
   int rc = ctx_reserve(c, carve_polar(nullptr, b, m, n, dtype, k, l).bytes);
   if (rc) return rc;
   PolarWs w = carve_polar(c->ws, b, m, n, dtype, k, l);
-  c->n_marks = 0;
+  ctx_profile_begin(c);
   c->err[0] = 0;
   ctx_stage_mark(c);
   if (ctx_fail(c, fill_int_launch(w.status, b, 0, c->stream, &c->launches), "status")) return DEFL_ERR_CUDA;
+  // the engine's wait word reports this call only (the tile counter next to it stays as the kernels leave it: zero)
+  if (ctx_fail(c, cudaMemsetAsync(c->wait_status, 0, sizeof(int), c->stream), "status word")) return DEFL_ERR_CUDA;
 
   // ---- stage 0: Algorithm 3 ------------------------------------------------------------------
   if (k > 0) {
@@ -494,11 +582,11 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
   // ---- stage 1: R = G - P diag(s) W^T, rho = ||R||_F, X0 = R/rho (+ P W^T / gamma) ----------------
   const float* left = tall ? w.Uk : w.Vk;     // [b,m,k]
   const float* right = tall ? w.Vk : w.Uk;    // [b,n,k]
+  const int kp = round_up8(k > 0 ? k : 1);
   if (k > 0) {
     // R = G - P diag(s) W^T as a rank-k product on the product engine with G read in the epilogue.
     // bf16 storage: the fp32 factors are split into bf16 hi + lo and the three significant cross terms are
     // laid side by side along K, [hi|hi|lo] x [hi|lo|hi]^T, one tensor-core product of depth 3k.
-    const int kp = round_up8(k);
     // gate (Algorithm 1, lines 1-2): per matrix, how many of the k triplets are deflated; the columns beyond
     // that count are zeroed in the scaled right factor, which removes them from every product below
     if (ctx_fail(c, gate_launch(w.sv, l, b, k, k, tau, w.keff, c->stream, &c->launches), "gate")) return DEFL_ERR_CUDA;
@@ -517,26 +605,36 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
       if (ctx_fail(c, split_concat3_launch(left, (long long)m * k, k, b, m, k, kp, nullptr, 0, nullptr, 0.f, 0.f, 0, w.Pc,
                                            c->stream, &c->launches), "split P"))
         return DEFL_ERR_CUDA;
-      if (ctx_fail(c, split_concat3_launch(right, (long long)n * k, k, b, n, k, kp, w.sv, l, nullptr, 1.f, 0.f, 1, w.Wc,
-                                           c->stream, &c->launches, w.keff), "split W diag(s)"))
+      // The triplets come from U = Q E and Q^T A = E diag(s) V^T (Algorithm 3, lines 7-9), so the residual's norm
+      // needs no pass over R:  ||A - U_k diag(s) V_k^T||_F^2 = ||A||_F^2 - sum_{i<=k} s_i^2  for ANY orthonormal Q
+      // (expand the square: the cross term is 2 tr(E_k^T Q^T A A^T Q E_k) = 2 sum s_i^2). ||G||_F^2 is one streaming
+      // read of G in fixed-order fp64 partial sums; with the gate only the deflated columns are subtracted. The
+      // difference is formed in fp64 from fp32 s_i: a residual below 1e-3 ||G||_F is not resolved and counts as zero.
+      if (ctx_fail(c, frob_partial_vec_launch(G, dtype, b, (long long)m * n, FROB_VEC_BLOCKS, w.npart, c->stream, &c->launches), "frobenius"))
+        return DEFL_ERR_CUDA;
+      if (ctx_fail(c, rho_identity_launch(w.npart, FROB_VEC_BLOCKS, b, w.sv, l, w.keff, w.rho, w.inv_rho, w.inv_rho2, w.status,
+                                          c->stream, &c->launches), "rho"))
         return DEFL_ERR_CUDA;
     } else {
+      // fp32 products (fp32 storage, or shapes the tensor engine cannot take): the residual is formed and its squares
+      // summed in the epilogue of a first pass, nothing stored
       if (ctx_fail(c, scale_cols_launch(right, (long long)n * k, k, b, n, k, w.sv, l, nullptr, 1.f, 0.f, w.Ws,
                                         (long long)n * k, k, c->stream, &c->launches, w.keff), "W diag(s)"))
         return DEFL_ERR_CUDA;
       g.K[0] = k;
       g.A[0] = left; g.sa_i[0] = k; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * k; g.in_dtype = F32;
       g.B[0] = w.Ws; g.sb_k[0] = 1; g.sb_j[0] = k; g.batch_b[0] = (long long)n * k; g.b_dtype = F32;
+      g.epilogue = EPI_RESID_NORM; g.partials = w.npart;
+      g.partials_per_batch = partials_per_batch(c, g, deng);
+      if ((rc = run_gemm(c, g, deng, "residual norm"))) return rc;
+      if (ctx_fail(c, rho_finalize_launch(w.npart, g.partials_per_batch, b, w.rho, w.inv_rho, w.inv_rho2, w.status,
+                                          c->stream, &c->launches), "rho"))
+        return DEFL_ERR_CUDA;
     }
-    // pass 1: norm of the residual, nothing stored
-    g.epilogue = EPI_RESID_NORM; g.partials = w.npart;
-    g.partials_per_batch = partials_per_batch(g, deng);
-    if ((rc = run_gemm(c, g, deng, "residual norm"))) return rc;
-    if (ctx_fail(c, rho_finalize_launch(w.npart, g.partials_per_batch, b, w.rho, w.inv_rho, w.inv_rho2, w.status,
-                                        c->stream, &c->launches), "rho"))
-      return DEFL_ERR_CUDA;
-    // pass 2: X0 = G/rho - P diag(s/rho - 1/gamma) W^T   (ADD mode: without the 1/gamma term)
-    const float pad = (mode == DEFL_RESTORE_PADDED) ? 1.f / gamma : 0.f;
+    // X0 = G/rho - P diag(s/rho - pad) W^T: pad = 1/gamma puts the head into X0 (Algorithm 1); with ADD restore the
+    // head stays out (pad = 0) and joins the last filter product, or, when there is no filter step to carry it,
+    // goes in at full weight (X0 + P W^T is the padded entry with gamma = 1)
+    const float pad = (mode == DEFL_RESTORE_PADDED) ? 1.f / gamma : (L == 0 ? 1.f : 0.f);
     if (tensor_defl) {
       if (ctx_fail(c, split_concat3_launch(right, (long long)n * k, k, b, n, k, kp, w.sv, l, w.inv_rho, -1.f, pad, 1, w.Wc,
                                            c->stream, &c->launches, w.keff), "split W diag(coef)"))
@@ -550,16 +648,60 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
     g.C = bufs[cur]; g.ldc = n; g.batch_c = (long long)m * n; g.out_dtype = it_dtype;
     if ((rc = run_gemm(c, g, deng, "deflate+normalise"))) return rc;
   } else {
-    const int nblk = 296;
-    if (ctx_fail(c, frob_partial_launch(G, dtype, b, (long long)m * n, nblk, w.npart, c->stream, &c->launches), "frobenius"))
+    if (ctx_fail(c, frob_partial_vec_launch(G, dtype, b, (long long)m * n, FROB_VEC_BLOCKS, w.npart, c->stream, &c->launches), "frobenius"))
       return DEFL_ERR_CUDA;
-    if (ctx_fail(c, rho_finalize_launch(w.npart, nblk, b, w.rho, w.inv_rho, w.inv_rho2, w.status, c->stream,
+    if (ctx_fail(c, rho_finalize_launch(w.npart, FROB_VEC_BLOCKS, b, w.rho, w.inv_rho, w.inv_rho2, w.status, c->stream,
                                         &c->launches), "rho"))
       return DEFL_ERR_CUDA;
     if (ctx_fail(c, scale_launch(G, dtype, bufs[cur], it_dtype, b, (long long)m * n, w.inv_rho, c->stream, &c->launches, 0, ys), "normalise"))
       return DEFL_ERR_CUDA;
   }
   ctx_stage_mark(c);
+
+  // ---- restore (Eq. 3) with ADD mode: out = N^L(X0) + P W^T rides on the LAST filter product as a second K segment
+  // (depth k, or 3k for the split 16-bit copies), so the head is added in the accumulator and `out` makes no further
+  // trip through memory. The factors are prepared here: in the type and scale of the last step's operands
+  // (16-bit iterates: [hi|hi|lo] x [hi|lo|hi] copies, IEEE half or bf16, their product scaled like the iterate;
+  // fp32: the factors themselves), the right one gated and laid out like the operand it accompanies.
+  const bool fuse_restore = k > 0 && mode == DEFL_RESTORE_ADD && L > 0;
+  const bool last_half = L > 0 && (L - 1) < n_half;            // the last step's operands are scaled IEEE half
+  if (fuse_restore) {
+    if (dtype == BF16) {
+      const float ysl = last_half ? 32.f : 1.f;
+      const float mp = last_half ? 8.f : 1.f;                  // powers of two: P W^T * ysl = (mp P)(ysl / mp W)^T exactly
+      if (ctx_fail(c, split_concat3_launch(left, (long long)m * k, k, b, m, k, kp, nullptr, 0, nullptr, 0.f, 0.f, 0, w.Pc,
+                                           c->stream, &c->launches, nullptr, last_half ? 1 : 0, 0, mp), "split P (restore)"))
+        return DEFL_ERR_CUDA;
+      if (ctx_fail(c, split_concat3_launch(right, (long long)n * k, k, b, n, k, kp, nullptr, 0, nullptr, 0.f, 0.f, 1, w.Wc,
+                                           c->stream, &c->launches, w.keff, last_half ? 1 : 0, wide ? 1 : 0, ysl / mp),
+                   "split W (restore)"))
+        return DEFL_ERR_CUDA;
+    } else if (ctx_fail(c, scale_cols_launch(right, (long long)n * k, k, b, n, k, w.sv, l, nullptr, 0.f, 1.f, w.Ws,
+                                             (long long)n * k, k, c->stream, &c->launches, w.keff), "W (gated)")) {
+      return DEFL_ERR_CUDA;
+    }
+  }
+  // second K segment of the last apply product; `transposed_form`: the product is computed as its transpose
+  auto add_restore_segment = [&](GemmDesc& q, bool transposed_form) {
+    q.nseg = 2;
+    if (dtype == BF16) {
+      q.K[1] = 3 * kp;
+      const void* Pr = w.Pc;      // [b, m, 3kp]
+      const void* Wr = w.Wc;      // [b, 3kp, n] for a wide matrix, else [b, n, 3kp]
+      if (!transposed_form) {
+        q.A[1] = Pr; q.sa_i[1] = 3 * kp; q.sa_k[1] = 1; q.batch_a[1] = (long long)m * 3 * kp;
+        q.B[1] = Wr; q.batch_b[1] = (long long)n * 3 * kp;
+        if (wide) { q.sb_k[1] = n; q.sb_j[1] = 1; } else { q.sb_k[1] = 1; q.sb_j[1] = 3 * kp; }
+      } else {
+        q.A[1] = Wr; q.sa_i[1] = 1; q.sa_k[1] = n; q.batch_a[1] = (long long)n * 3 * kp;
+        q.B[1] = Pr; q.sb_k[1] = 1; q.sb_j[1] = 3 * kp; q.batch_b[1] = (long long)m * 3 * kp;
+      }
+    } else {
+      q.K[1] = k;
+      q.A[1] = left; q.sa_i[1] = k; q.sa_k[1] = 1; q.batch_a[1] = (long long)m * k;
+      q.B[1] = w.Ws; q.sb_k[1] = 1; q.sb_j[1] = k; q.batch_b[1] = (long long)n * k;
+    }
+  };
 
   // ---- stage 2: X <- a X + b (X X^T) X + c (X X^T)^2 X, L times, through the short-side Gram -------
   for (int t = 0; t < L; ++t) {
@@ -607,6 +749,8 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
     g.epilogue = EPI_STORE;
     g.out_dtype = nx_dtype; g.alpha = ys_next / ys;                   // the next step's format and scale
     if (t == L - 1) { g.out_dtype = dtype; g.alpha = 1.f / ys; }      // the result leaves in the caller's type and scale
+    const bool carry_head = fuse_restore && t == L - 1;
+    if (carry_head) add_restore_segment(g, false);
     if (wide && !(upd && t == L - 1)) {
       // The tensor engine pads the product's rows to whole 256-row tiles, its columns only to 32: for a wide X
       // whose short side is not a multiple of 256 (1600 = 6.25 tiles) it is cheaper to compute (B X)^T = X^T B
@@ -615,59 +759,33 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
       gt.M = n; gt.N = m;
       gt.A[0] = X; gt.sa_i[0] = 1; gt.sa_k[0] = n; gt.batch_a[0] = (long long)m * n;
       gt.B[0] = w.Bm; gt.sb_j[0] = m; gt.sb_k[0] = 1; gt.batch_b[0] = (long long)m * m;    // B_t symmetric
+      if (carry_head) add_restore_segment(gt, true);
       gt.transpose_out = 1;
       const long long pad_rows = (long long)((m + 255) / 256) * 256 * ((n + 31) / 32 * 32);
       const long long pad_rows_t = (long long)((n + 255) / 256) * 256 * ((m + 31) / 32 * 32);
-      if (m > 128 && pad_rows_t < pad_rows && use_tensor_engine(gt, engine) && !getenv("DEFL_NO_TRANSPOSED_APPLY")) g = gt;
+      if (m > 128 && pad_rows_t < pad_rows && use_tensor_engine(gt, engine) && c->knobs.transposed_apply) g = gt;
     }
     if (upd && t == L - 1) {
-      // last step of a Muon update: W <- keep W + step (B_L X) instead of storing the iterate
+      // last step of a Muon update: W <- keep W + step (B_L X [+ P W^T]) instead of storing the iterate
       g.C = upd->W; g.out_dtype = upd->w_dtype;
       g.aux = upd->W; g.ld_aux = n; g.batch_aux = (long long)m * n; g.aux_dtype = upd->w_dtype;
       g.epilogue = EPI_AUX_PLUS; g.alpha = upd->step / ys; g.aux_scale = upd->keep;
     }
-    if ((rc = run_gemm(c, g, engine, "apply"))) return rc;
+    // (a forced tensor engine that cannot take the two-segment product, e.g. fp32 factors whose width is not a
+    // multiple of four, runs this one product on the fp32 engine instead of failing)
+    const int eng_apply = (carry_head && engine == DEFL_ENGINE_TENSOR && !use_tensor_engine(g, engine)) ? DEFL_ENGINE_SIMT : engine;
+    if ((rc = run_gemm(c, g, eng_apply, "apply"))) return rc;
     cur ^= 1;
   }
   ctx_stage_mark(c);
 
-  // ---- stage 3: restore (Eq. 3) in ADD mode: out += P W^T ------------------------------------------
-  if (k > 0 && mode == DEFL_RESTORE_ADD) {
-    const int kp = round_up8(k);
-    GemmDesc g = gemm_desc_zero();
-    g.batch = b; g.M = m; g.N = n;
-    g.aux = out; g.ld_aux = n; g.batch_aux = (long long)m * n; g.aux_dtype = dtype;
-    g.C = out; g.ldc = n; g.batch_c = (long long)m * n; g.out_dtype = dtype;
-    g.epilogue = EPI_AUX_PLUS;
-    if (upd) {      // Muon update: the head joins the weights with the same step, W <- W + step P W^T
-      g.aux = upd->W; g.aux_dtype = upd->w_dtype; g.C = upd->W; g.out_dtype = upd->w_dtype;
-      g.alpha = upd->step; g.aux_scale = 1.f;
-    }
-    bool tensor_restore = false;
-    if (dtype == BF16 && engine != DEFL_ENGINE_SIMT) {
-      g.K[0] = 3 * kp;
-      g.A[0] = w.Pc; g.sa_i[0] = 3 * kp; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * 3 * kp; g.in_dtype = BF16;
-      g.B[0] = w.Wc; g.sb_k[0] = 1; g.sb_j[0] = 3 * kp; g.batch_b[0] = (long long)n * 3 * kp; g.b_dtype = BF16;
-      tensor_restore = gemm_tc_supported(g);
-    }
-    if (tensor_restore) {
-      // w.Pc still holds the split left factor from the deflation stage; rebuild the right one unscaled
-      if (ctx_fail(c, split_concat3_launch(right, (long long)n * k, k, b, n, k, kp, nullptr, 0, nullptr, 0.f, 0.f, 1, w.Wc,
-                                           c->stream, &c->launches, w.keff), "split W"))
-        return DEFL_ERR_CUDA;
-      if ((rc = run_gemm(c, g, DEFL_ENGINE_TENSOR, "restore (tensor)"))) return rc;
-    } else {
-      if (ctx_fail(c, scale_cols_launch(right, (long long)n * k, k, b, n, k, w.sv, l, nullptr, 0.f, 1.f, w.Ws,
-                                        (long long)n * k, k, c->stream, &c->launches, w.keff), "W (gated)"))
-        return DEFL_ERR_CUDA;
-      g.K[0] = k;
-      g.A[0] = left; g.sa_i[0] = k; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * k; g.in_dtype = F32;
-      g.B[0] = w.Ws; g.sb_k[0] = 1; g.sb_j[0] = k; g.batch_b[0] = (long long)n * k; g.b_dtype = F32;
-      if ((rc = run_gemm(c, g, DEFL_ENGINE_SIMT, "restore"))) return rc;
-    }
-  }
+  // (stage 3, the restore of Eq. 3, is part of the last filter product: see above)
   ctx_stage_mark(c);
 
+  // a result that is not finite raises DEFL_ST_NONFINITE for its matrix
+  if (ctx_fail(c, finite_probe_launch(upd ? upd->W : out, upd ? upd->w_dtype : dtype, b, (long long)m * n, w.status, c->stream,
+                                      &c->launches), "finite probe"))
+    return DEFL_ERR_CUDA;
   if (info) {
     if (info->s && l > 0 &&
         ctx_fail(c, cudaMemcpyAsync(info->s, w.sv, (size_t)b * l * sizeof(float), cudaMemcpyDeviceToDevice, c->stream), "copy s"))
@@ -748,7 +866,7 @@ int defl_polar_batched_host(defl_ctx* c, const void* G_host, void* out_host, int
   // chunk i-1 back to the host running (on streams of their own) while chunk i is computed. Few chunks: the small
   // kernels of the range finder take about the same time for 12 matrices as for 48.
   int chunks = b >= 24 ? 3 : (b >= 8 ? 2 : 1);
-  if (const char* e = getenv("DEFL_HOST_CHUNKS")) { const int v = atoi(e); if (v >= 1) chunks = v; }
+  if (c->knobs.host_chunks >= 1) chunks = c->knobs.host_chunks;
   if (chunks > DEFL_HOST_MAX_CHUNKS) chunks = DEFL_HOST_MAX_CHUNKS;
   if (chunks > b) chunks = b;
   if (!c->copy_ready) {

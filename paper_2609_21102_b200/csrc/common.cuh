@@ -44,6 +44,7 @@ struct GemmDesc {
   int round_tf32;               // fp32 output rounded to nearest tf32 (it feeds tf32 products, which would truncate)
   int symmetric;                // output is symmetric (M == N): compute upper tiles only and mirror
   int transpose_out;            // element (i, j) of the product is stored at C[j * ldc + i] (tensor engine, EPI_STORE only)
+  int debug_hold_stage;         // test hook, tensor engine, single-CTA form: s > 0 withholds pipeline step s - 1 of each CTA's first tile
 };
 
 inline GemmDesc gemm_desc_zero() {
@@ -55,14 +56,38 @@ inline GemmDesc gemm_desc_zero() {
   return g;
 }
 
+// Tuning overrides of the tensor engine, read from the environment ONCE, when a context is created (a value of 0
+// keeps the default rule): experiments, and the tests of the tile forms the default rules do not pick.
+//   DEFL_TC_BN, DEFL_TC_TILE_M, DEFL_TC_STAGES, DEFL_TC_KSUB, DEFL_TC_PAIR (-1 default, 0 single-CTA form, 1 pair),
+//   DEFL_TC_PAIR_MIN_N, DEFL_TC_DYNAMIC (tiles through a counter), DEFL_TC_AUX_PREFETCH (L2 prefetch of `aux`),
+//   DEFL_TC_DEBUG, DEFL_TC_WAIT_MS (limit of every device-side wait, default 2000).
+struct TcKnobs {
+  int bn, tile_m, stages, ksub, pair, pair_min_n, dynamic, aux_prefetch, debug, wait_ms;
+};
+TcKnobs tc_knobs_from_env();
+
+// Encoded TMA descriptors of recent launches, kept per context: a descriptor depends only on the operand's address,
+// shape, strides and box, and the same few operands come back at every step of a filter chain.
+struct TmCacheEntry {
+  const void* base; long long MN, K, s_mn, s_k, batch, batch_stride; int esize, mn_major; unsigned box_rows;
+  alignas(64) unsigned char map[128];
+};
+struct TmCache {
+  static constexpr int SLOTS = 64;
+  TmCacheEntry e[SLOTS];
+  int used, next;
+  long long hits, misses;
+};
+
 // Engines (each returns cudaGetLastError() of its launch; they never synchronise).
 cudaError_t gemm_simt_launch(const GemmDesc& g, cudaStream_t st, long long* launches);
 int gemm_simt_partials_per_batch(const GemmDesc& g);
 // Tensor-core engine: returns cudaErrorNotSupported when the descriptor cannot be expressed
 // as TMA-tiled tcgen05 products (alignment, type), without launching anything.
-cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word, int num_sms, long long* launches);
+cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word, int num_sms, long long* launches,
+                           const TcKnobs* knobs = nullptr, TmCache* cache = nullptr);
 bool gemm_tc_supported(const GemmDesc& g);
-int gemm_tc_partials_per_batch(const GemmDesc& g);
+int gemm_tc_partials_per_batch(const GemmDesc& g, const TcKnobs* knobs = nullptr);
 
 __device__ __forceinline__ float ld_as_float(const void* p, long long idx, int dt) {
   return dt == BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[idx])

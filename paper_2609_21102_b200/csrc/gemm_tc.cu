@@ -41,7 +41,6 @@ constexpr int STAGING_BYTES = 4096;         // per epilogue warp: one 32 x 32 bl
 constexpr int AUX_AHEAD = 3;                // tiles (per CTA) by which the aux prefetch runs ahead
 constexpr int MAX_STAGES = 6;
 constexpr int SCHED_SLOTS = 8;              // tile numbers published ahead of the slowest reader (pair form)
-constexpr unsigned long long WAIT_NS = 2000000000ull;  // 2 s per wait before giving up
 
 struct TcParams {
   CUtensorMap tmA[2];
@@ -80,6 +79,8 @@ struct TcParams {
   double* partials; int partials_per_batch;
   int* status;
   unsigned int* tile_counter;  // pair form: tiles beyond each pair's first are handed out through this counter (null: fixed stride)
+  unsigned long long wait_ns;  // limit of every bounded wait
+  int hold_stage;              // test hook (single-CTA form): the producer withholds the copies of this pipeline step (-1: none)
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -129,7 +130,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // Bounded wait. A short burst of polls first (the common case: the barrier flips within the hardware
 // suspend window of try_wait); after that every poll also checks the CTA's abort flag and a wall-clock
 // budget, so that a protocol error or a lost copy ends in a status bit instead of a hang.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, unsigned long long wait_ns) {
 #pragma unroll 1
   for (int i = 0; i < 64; ++i)
     if (mbar_try_wait(bar, parity)) return true;
@@ -137,7 +138,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (global_ns() - t0 > WAIT_NS) {
+    if (global_ns() - t0 > wait_ns) {
       *abort_flag = 1;
       if (status) atomicOr(status, 8);
       return false;
@@ -782,7 +783,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
   // one reader's step: wait for slot `it`, read the tile number, acknowledge; -1 = no more tiles, -2 = a wait ran out
   auto sched_read = [&](int it) -> long long {
     const uint32_t s2 = (uint32_t)it % SCHED_SLOTS, ph = ((uint32_t)it / SCHED_SLOTS) & 1u;
-    if (!mbar_wait(sfull0 + 8u * s2, ph, &abort_flag, p.status)) return -2;
+    if (!mbar_wait(sfull0 + 8u * s2, ph, &abort_flag, p.status, p.wait_ns)) return -2;
     const int tnum = *reinterpret_cast<volatile int*>(&sched_tile[s2]);
     mbar_arrive_cluster(sempty0_leader + 8u * s2);
     return (long long)tnum;
@@ -874,7 +875,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
                 if (tl >= total_tiles) tl = -1;
               }
               const uint32_t s2 = (uint32_t)it % SCHED_SLOTS, ph = ((uint32_t)it / SCHED_SLOTS) & 1u;
-              if (!mbar_wait(smem_u32(&sched_empty[s2]), ph ^ 1u, &abort_flag, p.status)) tl = -2;
+              if (!mbar_wait(smem_u32(&sched_empty[s2]), ph ^ 1u, &abort_flag, p.status, p.wait_ns)) tl = -2;
               if (tl != -2) {
                 sched_tile[s2] = (int)tl;
                 mbar_arrive(sfull0 + 8u * s2);
@@ -922,10 +923,16 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
           int kc = my_k_off;
           for (int kb = 0; kb < nkb; ++kb, left -= ksub, kc += ksub * kstep) {
             int ok = 1;
-            if (lane == 0) ok = mbar_wait(empty0 + 8u * stage, phase ^ 1u, &abort_flag, p.status) ? 1 : 0;
+            if (lane == 0) ok = mbar_wait(empty0 + 8u * stage, phase ^ 1u, &abort_flag, p.status, p.wait_ns) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) { live = false; break; }
             const int nsub = left < ksub ? left : ksub;       // the last step of a segment may be short
+            // test hook of the bounded waits (single-CTA form): this step of the CTA's first tile is neither announced
+            // nor copied, so the consumer's wait for it runs out with nothing in flight
+            if (!PAIR && p.hold_stage >= 0 && it == 0 && seg == 0 && kb == p.hold_stage) {
+              if (++stage == nstages) { stage = 0; phase ^= 1u; }
+              continue;
+            }
             if (lane == 0 && (!PAIR || rank == 0))
               mbar_expect_tx(full0 + 8u * stage, nsub == ksub ? tx_bytes : tx_sub_bytes * (uint32_t)nsub);
             // (the part of a K block past the end of K is filled with zeros by the copy engine and adds nothing)
@@ -982,7 +989,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
           if (nxt >= 0) tnx = tile_info(p, nxt);
           continue;
         }
-        if (!mbar_wait(smem_u32(&acc_empty_bar[acc]), acc_phase ^ 1u, &abort_flag, p.status)) break;
+        if (!mbar_wait(smem_u32(&acc_empty_bar[acc]), acc_phase ^ 1u, &abort_flag, p.status, p.wait_ns)) break;
         tc_fence_after();
         const uint32_t idesc = idesc0 | ((uint32_t)(t.n_eff >> 3) << 17);
         const uint32_t d0 = tmem_base + (tall ? 0u : acc * 256u);
@@ -993,7 +1000,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
         uint32_t ready = 0;                                   // the next stage was seen full while this one was issued
         for (int kb = 0; kb < total_kblocks; ++kb, left -= ksub) {
           if (kb == steps0) left = kreal1;
-          if (!ready && !mbar_wait(full0 + 8u * stage, phase, &abort_flag, p.status)) { ok = false; break; }
+          if (!ready && !mbar_wait(full0 + 8u * stage, phase, &abort_flag, p.status, p.wait_ns)) { ok = false; break; }
           tc_fence_after();
           {
             // probe the following stage now: the answer arrives while this stage's products are issued
@@ -1062,7 +1069,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       const TileInfo t = tile_info(p, tile);
       if (t.skip) continue;
       const int tn = t.tn, tm = t.tm, bz = t.bz;
-      const bool ok = mbar_wait(smem_u32(&acc_full_bar[acc]), acc_phase, &abort_flag, p.status);
+      const bool ok = mbar_wait(smem_u32(&acc_full_bar[acc]), acc_phase, &abort_flag, p.status, p.wait_ns);
       if (!ok) break;
       tc_fence_after();
       float alpha = p.alpha, aux_scale = p.aux_scale;
@@ -1191,35 +1198,58 @@ bool encode_map(CUtensorMap* tm, const void* base, int esize, bool tf32, bool mn
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Tuning overrides for experiments and for the tests of the forms the default rules do not pick (environment,
-// read per launch): DEFL_TC_BN, DEFL_TC_TILE_M, DEFL_TC_STAGES, DEFL_TC_KSUB, DEFL_TC_PAIR, DEFL_TC_PAIR_MIN_N,
-// DEFL_TC_DYNAMIC (tiles through a counter), DEFL_TC_AUX_PREFETCH (L2 prefetch of `aux`), DEFL_TC_DEBUG.
-int choose_bn(int N, bool pair) {
+const TcKnobs kDefaultKnobs = {0, 0, 0, 0, -1, 0, 0, 0, 0, 0};
+
+int choose_bn(int N, bool pair, const TcKnobs& kn) {
   const int q = pair ? 32 : 16;
-  if (const char* e = getenv("DEFL_TC_BN")) { const int v = atoi(e); if (v >= q && v <= 256 && v % q == 0) return v; }
+  if (kn.bn >= q && kn.bn <= 256 && kn.bn % q == 0) return kn.bn;
   // widest tile; edge tiles only compute the columns that exist (rounded up to 16, or 32 for a CTA pair), so
   // a wide tile wastes at most q - 1 columns per tile row
   const int r = (N + q - 1) & ~(q - 1);
   return r < 256 ? r : 256;
 }
 
-int choose_tile_m_impl(int M, int N, int batch) {
-  (void)N; (void)batch;
-  if (const char* e = getenv("DEFL_TC_TILE_M")) { const int v = atoi(e); if (v == 128 || v == 256) return v; }
+int choose_tile_m_impl(int M, const TcKnobs& kn) {
+  if (kn.tile_m == 128 || kn.tile_m == 256) return kn.tile_m;
   // (128-row tiles for narrow outputs whose 256-row tiles fill the last wave of CTAs badly were measured: slower)
   return M > 128 ? 256 : 128;
 }
 
-// 256-row tiles are computed by a cluster of two CTAs (tcgen05 cta_group::2) unless DEFL_TC_PAIR=0 asks for
-// the single-CTA form (two 128-row halves in one CTA)
-bool choose_pair(int M, int N, int batch) {
-  if (choose_tile_m_impl(M, N, batch) != 256) return false;
-  if (const char* e = getenv("DEFL_TC_PAIR")) return atoi(e) != 0;
-  // (DEFL_TC_PAIR_MIN_N: outputs narrower than this take the single-CTA form; measured on the range finder's
+// 256-row tiles are computed by a cluster of two CTAs (tcgen05 cta_group::2) unless the knob asks for the
+// single-CTA form (two 128-row halves in one CTA)
+bool choose_pair(int M, int N, const TcKnobs& kn) {
+  if (choose_tile_m_impl(M, kn) != 256) return false;
+  if (kn.pair >= 0) return kn.pair != 0;
+  // (pair_min_n: outputs narrower than this take the single-CTA form; measured on the range finder's
   // 48-column panels the pair streams A faster, 4.9-5.1 against 4.3-4.6 TB/s, so the default keeps every width)
-  int min_n = 0;
-  if (const char* e = getenv("DEFL_TC_PAIR_MIN_N")) min_n = atoi(e);
-  return N >= min_n;
+  return N >= kn.pair_min_n;
+}
+
+// cached encode: the same (address, shape, strides, box) gives the same descriptor
+bool cached_map(TmCache* cache, CUtensorMap* tm, const void* base, int esize, bool tf32, bool mn_major, long long MN, long long K,
+                long long s_mn, long long s_k, long long batch, long long batch_stride, uint32_t box_rows) {
+  static_assert(sizeof(CUtensorMap) <= sizeof(TmCacheEntry::map), "descriptor size");
+  if (cache) {
+    for (int i = 0; i < cache->used; ++i) {
+      const TmCacheEntry& c = cache->e[i];
+      if (c.base == base && c.MN == MN && c.K == K && c.s_mn == s_mn && c.s_k == s_k && c.batch == batch &&
+          c.batch_stride == batch_stride && c.esize == esize && c.mn_major == (int)mn_major && c.box_rows == box_rows) {
+        memcpy(tm, c.map, sizeof(CUtensorMap));
+        ++cache->hits;
+        return true;
+      }
+    }
+  }
+  if (!encode_map(tm, base, esize, tf32, mn_major, MN, K, s_mn, s_k, batch, batch_stride, box_rows)) return false;
+  if (cache) {
+    int slot = cache->used < TmCache::SLOTS ? cache->used++ : (cache->next = (cache->next + 1) % TmCache::SLOTS);
+    TmCacheEntry& c = cache->e[slot];
+    c.base = base; c.MN = MN; c.K = K; c.s_mn = s_mn; c.s_k = s_k; c.batch = batch; c.batch_stride = batch_stride;
+    c.esize = esize; c.mn_major = (int)mn_major; c.box_rows = box_rows;
+    memcpy(c.map, tm, sizeof(CUtensorMap));
+    ++cache->misses;
+  }
+  return true;
 }
 
 }  // namespace
@@ -1254,22 +1284,37 @@ bool gemm_tc_supported(const GemmDesc& g) {
 }
 
 
-int gemm_tc_partials_per_batch(const GemmDesc& g) {
-  const int bn = choose_bn(g.N, choose_pair(g.M, g.N, g.batch)), tmh = choose_tile_m_impl(g.M, g.N, g.batch);
+TcKnobs tc_knobs_from_env() {
+  TcKnobs k = kDefaultKnobs;
+  auto geti = [](const char* name, int dflt) { const char* e = getenv(name); return e ? atoi(e) : dflt; };
+  k.bn = geti("DEFL_TC_BN", 0); k.tile_m = geti("DEFL_TC_TILE_M", 0); k.stages = geti("DEFL_TC_STAGES", 0);
+  k.ksub = geti("DEFL_TC_KSUB", 0); k.pair = geti("DEFL_TC_PAIR", -1); k.pair_min_n = geti("DEFL_TC_PAIR_MIN_N", 0);
+  k.dynamic = getenv("DEFL_TC_DYNAMIC") ? 1 : 0; k.aux_prefetch = getenv("DEFL_TC_AUX_PREFETCH") ? 1 : 0;
+  k.debug = getenv("DEFL_TC_DEBUG") ? 1 : 0; k.wait_ms = geti("DEFL_TC_WAIT_MS", 0);
+  return k;
+}
+
+int gemm_tc_partials_per_batch(const GemmDesc& g, const TcKnobs* knobs) {
+  const TcKnobs& kn = knobs ? *knobs : kDefaultKnobs;
+  const int bn = choose_bn(g.N, choose_pair(g.M, g.N, kn), kn), tmh = choose_tile_m_impl(g.M, kn);
   return ((g.M + tmh - 1) / tmh) * ((g.N + bn - 1) / bn) * (tmh == 256 ? 2 : 1) * EPI_WARPS;
 }
 
-cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word, int num_sms, long long* launches) {
+cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word, int num_sms, long long* launches,
+                           const TcKnobs* knobs, TmCache* cache) {
   if (!gemm_tc_supported(g)) return cudaErrorNotSupported;
+  const TcKnobs& kn = knobs ? *knobs : kDefaultKnobs;
   TcParams p;
   memset(&p, 0, sizeof(p));
+  p.wait_ns = (unsigned long long)(kn.wait_ms > 0 ? kn.wait_ms : 2000) * 1000000ull;
+  p.hold_stage = g.debug_hold_stage - 1;      // 0 in a zeroed descriptor = no hold
   const int esize = (int)dtype_size(g.in_dtype);
   const bool tf32 = (g.in_dtype == F32);
   p.esize = esize;
   p.M = g.M; p.N = g.N; p.batch = g.batch;
-  p.tile_m = choose_tile_m_impl(g.M, g.N, g.batch);
-  p.pair = choose_pair(g.M, g.N, g.batch) ? 1 : 0;
-  p.BN = choose_bn(g.N, p.pair != 0);
+  p.tile_m = choose_tile_m_impl(g.M, kn);
+  p.pair = choose_pair(g.M, g.N, kn) ? 1 : 0;
+  p.BN = choose_bn(g.N, p.pair != 0, kn);
   p.tiles_m = (g.M + p.tile_m - 1) / p.tile_m;
   p.tiles_n = (g.N + p.BN - 1) / p.BN;
   p.tiles_per_matrix = p.tiles_m * p.tiles_n;
@@ -1295,7 +1340,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   p.b_split_bytes = pb.stage_bytes; p.b_stage_bytes = pb.stage_bytes * p.b_split;
   const int span = KBYTES / esize;
   if (p.b_split == 2) {
-    if (!encode_map(&p.tmB[1], g.B[1], esize, tf32, pb.mn_major, g.N, g.K[0], g.sb_j[0], g.sb_k[0], g.batch,
+    if (!cached_map(cache, &p.tmB[1], g.B[1], esize, tf32, pb.mn_major, g.N, g.K[0], g.sb_j[0], g.sb_k[0], g.batch,
                     g.batch_b[0], pb.box_rows))
       return cudaErrorInvalidValue;
   }
@@ -1304,14 +1349,14 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   const uint32_t smem_budget = 224 * 1024 - EPI_WARPS * STAGING_BYTES;
   const uint32_t sub_bytes = p.a_stage_bytes + p.b_stage_bytes;
   p.ksub = (p.pair && 3u * 2u * sub_bytes <= smem_budget) ? 2 : 1;
-  if (const char* e = getenv("DEFL_TC_KSUB")) { const int v = atoi(e); if ((v == 1 || v == 2) && (uint32_t)v * sub_bytes * 2u <= smem_budget) p.ksub = v; }
+  if ((kn.ksub == 1 || kn.ksub == 2) && (uint32_t)kn.ksub * sub_bytes * 2u <= smem_budget) p.ksub = kn.ksub;
   for (int s = 0; s < g.nseg; ++s) {
     p.kreal[s] = (g.K[s] + span - 1) / span;
     p.kblocks[s] = (p.kreal[s] + p.ksub - 1) / p.ksub;
-    if (!encode_map(&p.tmA[s], g.A[s], esize, tf32, pa.mn_major, g.M, g.K[s], g.sa_i[s], g.sa_k[s], g.batch,
+    if (!cached_map(cache, &p.tmA[s], g.A[s], esize, tf32, pa.mn_major, g.M, g.K[s], g.sa_i[s], g.sa_k[s], g.batch,
                     g.batch_a[s], pa.box_rows))
       return cudaErrorInvalidValue;
-    if (!encode_map(&p.tmB[s], g.B[s], esize, tf32, pb.mn_major, g.N, g.K[s], g.sb_j[s], g.sb_k[s], g.batch,
+    if (!cached_map(cache, &p.tmB[s], g.B[s], esize, tf32, pb.mn_major, g.N, g.K[s], g.sb_j[s], g.sb_k[s], g.batch,
                     g.batch_b[s], pb.box_rows))
       return cudaErrorInvalidValue;
   }
@@ -1319,7 +1364,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   const uint32_t stage_bytes = sub_bytes * (uint32_t)p.ksub;
   int stages = (int)(smem_budget / stage_bytes);
   if (stages > MAX_STAGES) stages = MAX_STAGES;
-  if (const char* e = getenv("DEFL_TC_STAGES")) { const int v = atoi(e); if (v >= 2 && v <= stages) stages = v; }
+  if (kn.stages >= 2 && kn.stages <= stages) stages = kn.stages;
   if (stages < 2) return cudaErrorNotSupported;
   p.stages = stages;
   // instruction descriptor: fp32 accumulate, operand format, majors, N >> 3 at bit 17, M >> 4 at bit 24
@@ -1337,9 +1382,9 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   p.alpha_dev = g.alpha_dev; p.aux_scale_dev = g.aux_scale_dev;
   p.partials = g.partials; p.partials_per_batch = g.partials_per_batch;
   p.aux_prefetch = 0;
-  // (Off unless DEFL_TC_AUX_PREFETCH is set: with the epilogue's own fetch one block ahead the extra L2 prefetch
+  // (Off unless the aux_prefetch knob is set: with the epilogue's own fetch one block ahead the extra L2 prefetch
   // made the deflation passes 6 % slower and raised their DRAM reads to 1.6x the matrix, measured.)
-  if (g.aux && g.epilogue != EPI_STORE && aligned16(g.aux) && getenv("DEFL_TC_AUX_PREFETCH")) {
+  if (g.aux && g.epilogue != EPI_STORE && aligned16(g.aux) && kn.aux_prefetch) {
     const int aes = (int)dtype_size(g.aux_dtype);
     if ((g.ld_aux * aes) % 16 == 0 && (g.batch == 1 || (g.batch_aux * aes) % 16 == 0)) {
       EncodeTiledFn enc = get_encode_fn();
@@ -1356,12 +1401,12 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
     }
   }
   p.status = status_word;
-  // DEFL_TC_DYNAMIC: tiles handed out through a counter instead of a fixed stride. The word after the status word
+  // The `dynamic` knob: tiles handed out through a counter instead of a fixed stride. The word after the status word
   // is this context's counter (zero between launches: the kernel that uses it puts it back; launches of one
   // context are ordered on its stream, so they never share it in time). Off by default: measured on the filter's
   // products it gains 2 % where tiles are long and uneven (the symmetric Gram product) and loses 2-3 % where they
   // are short (one more hand-off per tile), and the whole step comes out the same.
-  p.tile_counter = (p.pair && status_word && getenv("DEFL_TC_DYNAMIC")) ? reinterpret_cast<unsigned int*>(status_word + 1) : nullptr;
+  p.tile_counter = (p.pair && status_word && kn.dynamic) ? reinterpret_cast<unsigned int*>(status_word + 1) : nullptr;
 
   const size_t smem = (size_t)stages * stage_bytes + 1024 + EPI_WARPS * STAGING_BYTES;
   cudaError_t e;
@@ -1394,7 +1439,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
       pairs = n > 0 ? n : 1;
       if (pairs > num_sms / 2) pairs = num_sms / 2;
       if (dev >= 0 && dev < 64) max_pairs[variant][dev] = pairs;
-      if (getenv("DEFL_TC_DEBUG")) fprintf(stderr, "gemm_tc: %d CTA pairs resident (occupancy query %d), %d stages\n", pairs, n, stages);
+      if (kn.debug) fprintf(stderr, "gemm_tc: %d CTA pairs resident (occupancy query %d), %d stages\n", pairs, n, stages);
     }
     long long npairs = p.total_tiles < pairs ? p.total_tiles : pairs;
     if (npairs < 1) npairs = 1;

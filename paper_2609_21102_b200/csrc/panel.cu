@@ -224,11 +224,8 @@ __global__ void __launch_bounds__(512) chol_inv_kernel(const double* __restrict_
 cudaError_t chol_inv_launch(const double* partial, int nchunk, int batch, int l, float* Rinv, int* status,
                             cudaStream_t st, long long* launches) {
   const size_t smem = 2 * (size_t)MAX_L * (MAX_L + 1) * sizeof(double);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    attr_set = true;
-  }
+  // (the attribute belongs to the current device's copy of the kernel: set at every launch, a host-side call)
+  cudaFuncSetAttribute(chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   chol_inv_kernel<<<batch, 512, smem, st>>>(partial, nchunk, l, Rinv, status);
   if (launches) ++*launches;
   return cudaGetLastError();
@@ -460,10 +457,14 @@ __global__ void __launch_bounds__(JAC_THREADS) jacobi_eig_kernel(const double* _
   }
   __syncthreads();
   if (tid < l) {
-    const double mine = fabs(lam[tid]);
+    // (a NaN compares false with everything: it ranks as magnitude -1, after every number, so that `order` is a
+    // permutation whatever the input holds)
+    double mine = fabs(lam[tid]);
+    if (!(mine == mine)) mine = -1.0;
     int rank = 0;
     for (int i = 0; i < l; ++i) {
-      const double o = fabs(lam[i]);
+      double o = fabs(lam[i]);
+      if (!(o == o)) o = -1.0;
       if (o > mine || (o == mine && i < tid)) ++rank;
     }
     order[rank] = tid;
@@ -482,14 +483,11 @@ __global__ void __launch_bounds__(JAC_THREADS) jacobi_eig_kernel(const double* _
 }
 
 cudaError_t jacobi_eig_launch(const double* partial, int nchunk, int batch, int l, int signed_input, float* s_out,
-                              float* E, float* Es, int* status, cudaStream_t st, long long* launches) {
+                              float* E, float* Es, int* status, cudaStream_t st, long long* launches, int max_sweeps) {
   const size_t smem = 2 * (size_t)MAX_L * (MAX_L + 1) * sizeof(double);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaFuncSetAttribute(jacobi_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    attr_set = true;
-  }
-  jacobi_eig_kernel<<<batch, JAC_THREADS, smem, st>>>(partial, nchunk, l, signed_input, s_out, E, Es, status, 40);
+  cudaFuncSetAttribute(jacobi_eig_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  jacobi_eig_kernel<<<batch, JAC_THREADS, smem, st>>>(partial, nchunk, l, signed_input, s_out, E, Es, status,
+                                                      max_sweeps > 0 ? max_sweeps : 40);
   if (launches) ++*launches;
   return cudaGetLastError();
 }
@@ -554,6 +552,123 @@ __global__ void rho_finalize_kernel(const double* __restrict__ partial, int nper
 cudaError_t rho_finalize_launch(const double* partial, int nper, int batch, float* rho, float* inv_rho,
                                 float* inv_rho2, int* status, cudaStream_t st, long long* launches) {
   rho_finalize_kernel<<<(batch + 3) / 4, 128, 0, st>>>(partial, nper, batch, rho, inv_rho, inv_rho2, status);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+// Frobenius partial sums with 16-byte loads: CTA (blk, batch) sums a contiguous run of whole 16-byte packets (fp32
+// sums of at most 64 squares per thread, then fp64), partial[b, nblk]. The leftover elements of a matrix whose
+// size is not a whole number of packets go to the last CTA. Needs a 16-byte aligned base and matrix stride.
+template <typename T, int V>
+__global__ void __launch_bounds__(256) frob_partial_vec_kernel(const T* __restrict__ X, long long count, int nblk,
+                                                               double* __restrict__ partial) {
+  struct alignas(16) Pack { T v[V]; };
+  __shared__ double red[8];
+  const int bz = blockIdx.y, tid = threadIdx.x;
+  const T* Xb = X + (long long)bz * count;
+  const long long nvec = count / V;
+  const long long per = (nvec + nblk - 1) / nblk;
+  const long long lo = (long long)blockIdx.x * per, hi = min(nvec, lo + per);
+  double acc = 0.0;
+  const Pack* P = reinterpret_cast<const Pack*>(Xb);
+  long long i = lo + tid;
+  // four packets per thread in flight
+  for (; i + 3 * 256 < hi; i += 4 * 256) {
+    Pack q[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) q[u] = P[i + u * 256];
+    float f = 0.f;
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int j = 0; j < V; ++j) { const float v = (float)q[u].v[j]; f = fmaf(v, v, f); }
+    acc += (double)f;
+  }
+  for (; i < hi; i += 256) {
+    const Pack q = P[i];
+    float f = 0.f;
+#pragma unroll
+    for (int j = 0; j < V; ++j) { const float v = (float)q.v[j]; f = fmaf(v, v, f); }
+    acc += (double)f;
+  }
+  if (blockIdx.x == nblk - 1) {
+    for (long long e = nvec * V + tid; e < count; e += 256) { const float v = (float)Xb[e]; acc += (double)v * (double)v; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, o);
+  if ((tid & 31) == 0) red[tid >> 5] = acc;
+  __syncthreads();
+  if (tid == 0) {
+    double t = 0.0;
+    for (int w = 0; w < 8; ++w) t += red[w];
+    partial[(long long)bz * nblk + blockIdx.x] = t;
+  }
+}
+
+cudaError_t frob_partial_vec_launch(const void* X, int dtype, int batch, long long count, int nblk, double* partial,
+                                    cudaStream_t st, long long* launches) {
+  const int es = (int)dtype_size(dtype);
+  const bool aligned = (reinterpret_cast<uintptr_t>(X) & 15) == 0 && ((count * es) & 15) == 0;
+  if (!aligned || dtype == F16) return frob_partial_launch(X, dtype, batch, count, nblk, partial, st, launches);
+  if (dtype == BF16) frob_partial_vec_kernel<__nv_bfloat16, 8><<<dim3(nblk, batch), 256, 0, st>>>((const __nv_bfloat16*)X, count, nblk, partial);
+  else frob_partial_vec_kernel<float, 4><<<dim3(nblk, batch), 256, 0, st>>>((const float*)X, count, nblk, partial);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+// rho[b] from the identity ||A - U_k diag(s) V_k^T||_F^2 = ||A||_F^2 - sum_{i < keff} s_i^2 (triplets of Algorithm 3):
+// one warp per matrix adds the partial sums of ||A||_F^2 (fixed order), lane 0 subtracts the squares in fp64.
+// A difference below 1e-6 ||A||_F^2 is below what the fp32 singular values resolve: the residual counts as zero
+// (status bit 4, 1/rho = 0), as does a non-finite one.
+__global__ void rho_identity_kernel(const double* __restrict__ partial, int nper, int batch, const float* __restrict__ s,
+                                    int ld_s, const int* __restrict__ keff, float* __restrict__ rho,
+                                    float* __restrict__ inv_rho, float* __restrict__ inv_rho2, int* __restrict__ status) {
+  const int bz = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (bz >= batch) return;
+  double t = 0.0;
+  for (int i = lane; i < nper; i += 32) t += partial[(long long)bz * nper + i];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+  if (lane != 0) return;
+  const double total = t;
+  const int ke = keff[bz];
+  for (int i = 0; i < ke; ++i) { const double v = (double)s[(long long)bz * ld_s + i]; t -= v * v; }
+  const bool ok = isfinite(t) && t > 1e-6 * total;
+  const double r = ok ? sqrt(t) : 0.0;
+  if (rho) rho[bz] = (float)r;
+  if (inv_rho) inv_rho[bz] = ok ? (float)(1.0 / r) : 0.f;
+  if (inv_rho2) inv_rho2[bz] = ok ? (float)(1.0 / t) : 0.f;
+  if (!ok && status) atomicOr(&status[bz], 4);
+}
+
+cudaError_t rho_identity_launch(const double* partial, int nper, int batch, const float* s, int ld_s, const int* keff,
+                                float* rho, float* inv_rho, float* inv_rho2, int* status, cudaStream_t st,
+                                long long* launches) {
+  rho_identity_kernel<<<(batch + 3) / 4, 128, 0, st>>>(partial, nper, batch, s, ld_s, keff, rho, inv_rho, inv_rho2, status);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+// Non-finite results are reported, not returned silently: one CTA per matrix looks at the first 4096 elements and at
+// 4096 more spread evenly over the matrix, and raises bit 16 of status[b] when one of them is Inf or NaN. A sample is
+// enough: a non-finite entry of an iterate (non-finite input, or a value that left the range of the iterate's
+// storage format) reaches the Gram matrix of the next step and from there every entry of the following iterate.
+__global__ void __launch_bounds__(256) finite_probe_kernel(const void* __restrict__ X, int dtype, long long count,
+                                                           int* __restrict__ status) {
+  const int bz = blockIdx.x, tid = threadIdx.x;
+  const long long base = (long long)bz * count;
+  const long long head = min(count, (long long)4096);
+  const long long stride = max((long long)1, count / 4096);
+  bool bad = false;
+  for (long long i = tid; i < head; i += 256) bad |= !isfinite(ld_as_float(X, base + i, dtype));
+  for (long long j = tid; j < 4096 && j * stride < count; j += 256) bad |= !isfinite(ld_as_float(X, base + j * stride, dtype));
+  if (__syncthreads_or(bad ? 1 : 0) && tid == 0) atomicOr(&status[bz], 16);
+}
+
+cudaError_t finite_probe_launch(const void* X, int dtype, int batch, long long count, int* status, cudaStream_t st,
+                                long long* launches) {
+  if (batch <= 0 || count <= 0) return cudaSuccess;
+  finite_probe_kernel<<<batch, 256, 0, st>>>(X, dtype, count, status);
   if (launches) ++*launches;
   return cudaGetLastError();
 }
@@ -742,37 +857,56 @@ cudaError_t split_panel_launch(const float* In, long long in_bs, int ld_in, int 
   return cudaGetLastError();
 }
 
-// Out [b, rows, 3*kp] bf16 = three column blocks of the (optionally column-scaled) panel In [b, rows, k]:
+// Out [b, rows, 3*kp] (16-bit) = three column blocks of the (optionally column-scaled) panel In [b, rows, k]:
 //   pattern 0: [hi | hi | lo]      pattern 1: [hi | lo | hi]
 // so that  Out0 * Out1^T = hi hi^T + hi lo^T + lo hi^T  (the product of the two fp32 panels up to the lo*lo term).
-// Column t is scaled by  c0 * s[b,t] * (inv_rho ? inv_rho[b] : 1) + c1  when s is given.
+// Column t is scaled by  mult * (c0 * s[b,t] * (inv_rho ? inv_rho[b] : 1) + c1)  (without s: by mult alone).
+// The two halves are bf16 or, with `f16`, IEEE half (the type of the product they enter); with `transposed` the
+// copy is stored as [b, 3*kp, rows], the layout of an operand whose long side is contiguous.
+template <bool F16, bool TRANSPOSED>
 __global__ void split_concat3_kernel(const float* __restrict__ In, long long in_bs, int ld_in, int rows, int k, int kp,
                                      const float* __restrict__ s, int ld_s, const float* __restrict__ inv_rho, float c0,
-                                     float c1, int pattern, __nv_bfloat16* __restrict__ Out,
+                                     float c1, float mult, int pattern, uint16_t* __restrict__ Out,
                                      const int* __restrict__ keff) {
   const int bz = blockIdx.y;
   const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= (long long)rows * kp) return;
-  const int r = (int)(e / kp), t = (int)(e % kp);
+  // consecutive threads walk the contiguous direction of the output
+  const int r = TRANSPOSED ? (int)(e % rows) : (int)(e / kp), t = TRANSPOSED ? (int)(e / rows) : (int)(e % kp);
   float x = 0.f;
   if (t < k && !(keff && t >= keff[bz])) {
-    x = In[(long long)bz * in_bs + (long long)r * ld_in + t];
+    x = In[(long long)bz * in_bs + (long long)r * ld_in + t] * mult;
     if (s) x *= c0 * s[(long long)bz * ld_s + t] * (inv_rho ? inv_rho[bz] : 1.f) + c1;
   }
-  const __nv_bfloat16 h = __float2bfloat16_rn(x);
-  const __nv_bfloat16 lw = __float2bfloat16_rn(x - __bfloat162float(h));
-  __nv_bfloat16* o = Out + ((long long)bz * rows + r) * (3LL * kp);
-  o[t] = h;
-  o[kp + t] = pattern ? lw : h;
-  o[2 * kp + t] = pattern ? h : lw;
+  uint16_t h, lw;
+  if (F16) {
+    const __half hh = __float2half_rn(x);
+    h = __half_as_ushort(hh);
+    lw = __half_as_ushort(__float2half_rn(x - __half2float(hh)));
+  } else {
+    const __nv_bfloat16 hh = __float2bfloat16_rn(x);
+    h = __bfloat16_as_ushort(hh);
+    lw = __bfloat16_as_ushort(__float2bfloat16_rn(x - __bfloat162float(hh)));
+  }
+  uint16_t* ob = Out + (long long)bz * rows * (3LL * kp);
+  const long long step = TRANSPOSED ? (long long)kp * rows : (long long)kp;      // distance between the three blocks
+  uint16_t* o = TRANSPOSED ? ob + (long long)t * rows + r : ob + (long long)r * (3LL * kp) + t;
+  o[0] = h;
+  o[step] = pattern ? lw : h;
+  o[2 * step] = pattern ? h : lw;
 }
 
 cudaError_t split_concat3_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int k, int kp,
                                  const float* s, int ld_s, const float* inv_rho, float c0, float c1, int pattern,
-                                 __nv_bfloat16* Out, cudaStream_t st, long long* launches, const int* keff) {
+                                 __nv_bfloat16* Out, cudaStream_t st, long long* launches, const int* keff, int f16,
+                                 int transposed, float mult) {
   const long long tot = (long long)rows * kp;
-  split_concat3_kernel<<<dim3((unsigned)((tot + 255) / 256), batch), 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s,
-                                                                                  inv_rho, c0, c1, pattern, Out, keff);
+  const dim3 grid((unsigned)((tot + 255) / 256), batch);
+  uint16_t* o = reinterpret_cast<uint16_t*>(Out);
+  if (f16 && transposed) split_concat3_kernel<true, true><<<grid, 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s, inv_rho, c0, c1, mult, pattern, o, keff);
+  else if (f16) split_concat3_kernel<true, false><<<grid, 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s, inv_rho, c0, c1, mult, pattern, o, keff);
+  else if (transposed) split_concat3_kernel<false, true><<<grid, 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s, inv_rho, c0, c1, mult, pattern, o, keff);
+  else split_concat3_kernel<false, false><<<grid, 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s, inv_rho, c0, c1, mult, pattern, o, keff);
   if (launches) ++*launches;
   return cudaGetLastError();
 }

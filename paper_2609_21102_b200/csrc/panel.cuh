@@ -16,9 +16,17 @@ cudaError_t panel_apply_launch(const float* In, long long in_bs, int ld_in, cons
                                int rows, int l, int kout, float* Out, long long out_bs, int ld_out, cudaStream_t st,
                                long long* launches);
 cudaError_t jacobi_eig_launch(const double* partial, int nchunk, int batch, int l, int signed_input, float* s_out,
-                              float* E, float* Es, int* status, cudaStream_t st, long long* launches);
+                              float* E, float* Es, int* status, cudaStream_t st, long long* launches, int max_sweeps = 0);
 cudaError_t frob_partial_launch(const void* X, int dtype, int batch, long long count, int nblk, double* partial,
                                 cudaStream_t st, long long* launches);
+constexpr int FROB_VEC_BLOCKS = 148;    // CTAs (and partial sums) per matrix of the vectorised Frobenius pass
+cudaError_t frob_partial_vec_launch(const void* X, int dtype, int batch, long long count, int nblk, double* partial,
+                                    cudaStream_t st, long long* launches);
+cudaError_t rho_identity_launch(const double* partial, int nper, int batch, const float* s, int ld_s, const int* keff,
+                                float* rho, float* inv_rho, float* inv_rho2, int* status, cudaStream_t st,
+                                long long* launches);
+cudaError_t finite_probe_launch(const void* X, int dtype, int batch, long long count, int* status, cudaStream_t st,
+                                long long* launches);
 cudaError_t rho_finalize_launch(const double* partial, int nper, int batch, float* rho, float* inv_rho,
                                 float* inv_rho2, int* status, cudaStream_t st, long long* launches);
 cudaError_t scale_cols_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int k, const float* s,
@@ -38,7 +46,8 @@ cudaError_t split_panel_launch(const float* In, long long in_bs, int ld_in, int 
                                __nv_bfloat16* hi, __nv_bfloat16* lo, cudaStream_t st, long long* launches);
 cudaError_t split_concat3_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int k, int kp,
                                  const float* s, int ld_s, const float* inv_rho, float c0, float c1, int pattern,
-                                 __nv_bfloat16* Out, cudaStream_t st, long long* launches, const int* keff = nullptr);
+                                 __nv_bfloat16* Out, cudaStream_t st, long long* launches, const int* keff = nullptr,
+                                 int f16 = 0, int transposed = 0, float mult = 1.f);
 cudaError_t gate_launch(const float* s, int ld_s, int batch, int window, int kmax, float tau, int* keff, cudaStream_t st,
                         long long* launches);
 }  // namespace defl

@@ -551,10 +551,11 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
   int rc = ctx_reserve(c, carve_psd(nullptr, n, K).bytes);
   if (rc) return rc;
   PsdWs w = carve_psd(c->ws, n, K);
-  c->n_marks = 0;
+  ctx_profile_begin(c);
   c->err[0] = 0;
   ctx_stage_mark(c);
   if (ctx_fail(c, fill_int_launch(w.status, 1, 0, c->stream, &c->launches), "status")) return DEFL_ERR_CUDA;
+  if (ctx_fail(c, cudaMemsetAsync(c->wait_status, 0, sizeof(int), c->stream), "status word")) return DEFL_ERR_CUDA;
 
   // ---- stage 0: block step and Rayleigh-Ritz (lines 1-2) -------------------------------------------
   if (K > 0) {

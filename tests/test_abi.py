@@ -68,3 +68,23 @@ def test_shape_groups_and_stacking():
     assert float(buf[1, 3, 3]) == 3.0
     with pytest.raises(ValueError):
         grouping.stack_group(ts, [0, 1])
+
+
+def test_window_ratios_follow_the_algorithms(libpath):
+    """Algorithm 3 line 1 (r = ceil(w m), r' = min{m, r + ceil(delta m)}) and Algorithm 2's inputs (r = ceil(w n),
+    K = ceil(w' n)), worked by hand."""
+    import pytest
+    from paper_2609_21102_b200 import binding
+    assert binding.defl_polar_window(1600, 6400, 0.02, 0.01) == (32, 16)
+    assert binding.defl_polar_window(6400, 1600, 0.02, 0.01) == (32, 16)          # the short side counts
+    assert binding.defl_polar_window(768, 3072, 0.01, 0.0105) == (8, 9)           # ceil(7.68) = 8, ceil(8.064) = 9
+    assert binding.defl_polar_window(40, 40, 0.5, 0.9) == (20, 20)                # r' capped at the short side
+    assert binding.defl_polar_window(40, 64, 1.0, 0.0) == (39, 0)                 # r capped at m - 1
+    assert binding.defl_psd_window(4096, 8 / 4096, 16 / 4096) == (8, 16)
+    assert binding.defl_psd_window(640, 0.025, 0.05) == (16, 32)
+    with pytest.raises(binding.DeflError) as e:
+        binding.defl_psd_window(5000, 0.025, 0.05)                                 # K = 250 exceeds the widest basis
+    assert e.value.code == -2
+    with pytest.raises(binding.DeflError) as e:
+        binding.defl_polar_window(128, 256, -0.1, 0.0)
+    assert e.value.code == -1

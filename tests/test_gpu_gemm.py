@@ -114,12 +114,13 @@ def test_symmetric_mirroring(ctx, engine_name):
                                    {"DEFL_TC_STAGES": "2"}, {"DEFL_TC_DYNAMIC": "1"},
                                    {"DEFL_TC_DYNAMIC": "1", "DEFL_TC_STAGES": "2"}])
 @pytest.mark.parametrize("sym", [False, True])
-def test_tensor_engine_other_tile_forms(ctx, monkeypatch, knobs, sym):
+def test_tensor_engine_other_tile_forms(monkeypatch, knobs, sym):
     """The tile forms the default rules do not pick for these shapes (single-CTA 256-row tile, one K block per
-    stage, 128-row tiles, the shallowest pipeline) stay correct: the knobs are read per launch."""
+    stage, 128-row tiles, the shallowest pipeline) stay correct: a context reads the knobs when it is created."""
     from paper_2609_21102_b200 import binding
     for k, v in knobs.items():
         monkeypatch.setenv(k, v)
+    ctx = binding.Context(0)
     A = _mk(2, 712, 1096, torch.bfloat16, 9)          # ragged in M (712 = 2 x 256 + 200), K = 17.1 blocks
     if sym:
         C = ctx.defl_debug_gemm(A, A, False, True, engine=binding.ENGINE_TENSOR, out_dtype=torch.float32,
@@ -135,11 +136,12 @@ def test_tensor_engine_other_tile_forms(ctx, monkeypatch, knobs, sym):
 
 @pytest.mark.parametrize("K", [64, 200, 1096])
 @pytest.mark.parametrize("sym", [False, True])
-def test_tensor_engine_dynamic_tiles(ctx, monkeypatch, K, sym):
+def test_tensor_engine_dynamic_tiles(monkeypatch, K, sym):
     """Tiles handed out through the counter (DEFL_TC_DYNAMIC), more tiles than CTA pairs so that every pair draws
     several; a one-step K, a short and a long one. Run twice: the counter must be back at zero after a launch."""
     from paper_2609_21102_b200 import binding
     monkeypatch.setenv("DEFL_TC_DYNAMIC", "1")
+    ctx = binding.Context(0)
     A = _mk(14, 1000, K, torch.bfloat16, 31)
     B = A if sym else _mk(14, 1032, K, torch.bfloat16, 32)
     ref = _ref(A, B, False, True)
@@ -171,3 +173,23 @@ def test_tensor_engine_ieee_half(ctx, ta, tb, out_dtype):
     # the fp32 FMA engine takes half operands too (it serves shapes the tensor engine cannot)
     Cf = ctx.defl_debug_gemm(A, B, ta, tb, engine=binding.ENGINE_SIMT, out_dtype=torch.float32)
     assert torch.allclose(Cf, ref, rtol=1e-4, atol=2e-3)
+
+
+def test_bounded_wait_runs_out_and_is_reported(monkeypatch):
+    """A device-side wait that nothing satisfies ends in a status bit and a normal return, not in a hang: one
+    128 x 128 x 64 product (one CTA, one tile, one pipeline step) whose only pipeline step is never announced nor
+    copied, with the wait limit at 2 ms. Nothing is in flight when the waits give up; the kernel frees its tensor
+    memory and returns, the context stays usable and the next product is correct."""
+    from paper_2609_21102_b200 import binding
+    monkeypatch.setenv("DEFL_TC_WAIT_MS", "2")
+    ctx = binding.Context(0)
+    A, B = _mk(1, 128, 64, torch.bfloat16, 41), _mk(1, 128, 64, torch.bfloat16, 42)
+    assert ctx.defl_device_wait_status() == 0
+    ctx.defl_debug_gemm(A, B, False, True, engine=binding.ENGINE_TENSOR, out_dtype=torch.float32, withhold_first_step=True)
+    assert ctx.defl_device_wait_status(clear=False) == binding.ST_DEVICE_WAIT
+    assert ctx.defl_device_wait_status(clear=True) == binding.ST_DEVICE_WAIT      # sticky until cleared
+    assert ctx.defl_device_wait_status() == 0
+    C = ctx.defl_debug_gemm(A, B, False, True, engine=binding.ENGINE_TENSOR, out_dtype=torch.float32)
+    assert torch.allclose(C, _ref(A, B, False, True), rtol=1e-4, atol=2e-3)
+    assert ctx.defl_device_wait_status() == 0
+    ctx.close()

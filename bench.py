@@ -313,7 +313,7 @@ def measure_tf32_peak():
         torch.backends.cuda.matmul.allow_tf32 = prev
 
 
-def extra_polar(ctx, name, opts, device, steps=10, label=None):
+def extra_polar(ctx, name, opts, device, steps=10, label=None, graph=False):
     """ms per batch, TFLOP/s (flops the method needs), matrices/s and launches of one more workload."""
     import torch
     wl = WORKLOADS[name]
@@ -326,7 +326,28 @@ def extra_polar(ctx, name, opts, device, steps=10, label=None):
     st = ctx.defl_get_stage_ms(min(64, steps * len(groups)))
     per = min(64, steps * len(groups)) / len(groups)
     filt, front = workload_flops(wl, opts["sym"], opts["mode"] == 1)
-    out = {"workload": label or wl["label"], "ms_per_batch": ms, "tflops": (filt + front) / (ms * 1e-3) / 1e12,
+    graph_ms = None
+    if graph:
+        # the launch-bound small batches replayed from a CUDA graph: every call of the library only enqueues work on its
+        # stream (no allocation once the workspace exists, no synchronisation), so a whole batch captures as it is
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                run_step(ctx, wl, groups, opts)
+                gph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gph, stream=side):
+                    run_step(ctx, wl, groups, opts)
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            for _ in range(3):
+                gph.replay()
+            graph_ms = time_steps(gph.replay, steps, torch.cuda.synchronize)
+            del gph
+        except Exception as e:
+            graph_ms = "capture failed: %r" % (e,)
+    out = {"workload": label or wl["label"], "ms_per_batch": ms, "ms_per_batch_cuda_graph": graph_ms,
+           "tflops": (filt + front) / (ms * 1e-3) / 1e12,
            "matrices_per_s": sum(b for b, _, _ in wl["groups"]) / (ms * 1e-3), "launches_per_batch": int(launches),
            "stage_ms": {"rsvd": st[0] / per, "deflate_normalise": st[1] / per, "filter": st[2] / per, "restore": st[3] / per}}
     del groups
@@ -623,8 +644,8 @@ def main():
     if not args.no_extras and wl_name == "gpt2_xl" and args.batch == 0:
         extras = {}
         try:
-            extras["gpt2_small"] = extra_polar(ctx, "gpt2_small", opts, device, steps=20)
-            extras["gpt2_medium_large"] = extra_polar(ctx, "gpt2_medium_large", opts, device, steps=10)
+            extras["gpt2_small"] = extra_polar(ctx, "gpt2_small", opts, device, steps=20, graph=True)
+            extras["gpt2_medium_large"] = extra_polar(ctx, "gpt2_medium_large", opts, device, steps=10, graph=True)
             del groups
             torch.cuda.empty_cache()
             xl_minimax = dict(WORKLOADS["gpt2_xl"], schedule="minimax", gamma=1.1)

@@ -673,11 +673,14 @@ __device__ __forceinline__ void epilogue_block_fast(const TcParams& p, uint32_t 
 template <int EPI, int ES>
 __device__ __forceinline__ int epilogue_fast_blocks(const TcParams& p, uint32_t taddr, uint8_t* stg, int lane, int gi_warp0,
                                                     int col0, int c0, int lim, int bz, float alpha, float aux_scale,
-                                                    float& sq) {
+                                                    float& sq, int skip_c) {
   constexpr bool AHEAD = (ES == 2) && (EPI != EPI_STORE);
   int half = 0;
   // symmetric output: nothing to do for blocks entirely left of the warp's rows (they are written as mirror images)
   if (p.symmetric) while (c0 + 32 <= lim && col0 + c0 + 31 < gi_warp0) c0 += 64;
+  // (the block on the diagonal of a plain symmetric store is left to the caller: see epilogue_half; it is the first
+  // block of this walk when it belongs to this warp)
+  if (c0 == skip_c) c0 += 64;
   __syncwarp();
   if (AHEAD && c0 + 32 <= lim) aux_fetch_async<ES>(p, lane, gi_warp0, col0 + c0, bz, stg);
 #pragma unroll 1
@@ -697,6 +700,30 @@ __device__ __forceinline__ int epilogue_fast_blocks(const TcParams& p, uint32_t 
     }
   }
   return c0;
+}
+
+// One 32-column block (two 16-column chunks) through the general path: any alignment, ragged edges, and for a
+// symmetric output exactly one computed value per pair (i, j), (j, i), stored at both places.
+template <int EPI>
+__device__ __forceinline__ void epilogue_block_general(const TcParams& p, uint32_t taddr, int c0, int gi, int gi_warp0, int col0,
+                                                       int n_eff, bool row_ok, bool vec_ok, bool aux_bf16, size_t crow,
+                                                       size_t cbatch, size_t xrow, float alpha, float aux_scale, float& sq) {
+  const int gj0 = col0 + c0, gj1 = gj0 + 16;
+  // symmetric output: nothing to do for a block entirely left of the warp's rows (warp-uniform)
+  if (p.symmetric && gj0 + 31 < gi_warp0) return;
+  const bool second = (c0 + 16 < n_eff);
+  uint32_t r0[16], r1[16];
+  __syncwarp();
+  tmem_ld16(taddr + (uint32_t)c0, r0);
+  if (second) tmem_ld16(taddr + (uint32_t)c0 + 16u, r1);
+  const bool vec0 = vec_ok && (gj0 + 16 <= p.N) && ((gj0 & 7) == 0);
+  const bool vec1 = vec_ok && (gj1 + 16 <= p.N) && ((gj1 & 7) == 0);
+  float x0[16], x1[16];
+  load_aux16<EPI>(p, row_ok && gj0 < p.N, vec0, aux_bf16, xrow + gj0, gj0, x0);
+  load_aux16<EPI>(p, second && row_ok && gj1 < p.N, vec1, aux_bf16, xrow + gj1, gj1, x1);
+  tmem_ld_wait();
+  finish16<EPI>(p, r0, x0, gi, gi_warp0, gj0, row_ok, vec0, crow, cbatch, alpha, aux_scale, sq);
+  if (second) finish16<EPI>(p, r1, x1, gi, gi_warp0, gj1, row_ok, vec1, crow, cbatch, alpha, aux_scale, sq);
 }
 
 template <int EPI>
@@ -721,28 +748,23 @@ __device__ __forceinline__ void epilogue_half(const TcParams& p, uint32_t taddr,
     // the complete 32-column blocks come first; whatever is left (a ragged edge) takes the general path below
     int lim = p.N - col0;
     if (lim > n_eff) lim = n_eff;
+    // A plain symmetric store (EPI_STORE) may be the product of two DIFFERENT symmetric matrices (the apply step of
+    // the symmetric filter), whose computed (i, j) and (j, i) differ in the last bits. Off the diagonal the mirror
+    // store makes the pair equal; the 32 x 32 block ON the diagonal must do the same element by element, or the
+    // iterate picks up an antisymmetric part that the filter doubles at every step: it takes the general path.
+    int c_diag = -1;
+    if (EPI == EPI_STORE && p.symmetric && gi_warp0 >= col0 && gi_warp0 - col0 < lim && (((gi_warp0 - col0) >> 5) & 1) == wsel)
+      c_diag = gi_warp0 - col0;
     const bool two = (EPI == EPI_STORE) ? o2 : a2;
-    if (two) c0 = epilogue_fast_blocks<EPI, 2>(p, taddr, stg, lane, gi_warp0, col0, c0, lim, bz, alpha, aux_scale, sq);
-    else c0 = epilogue_fast_blocks<EPI, 4>(p, taddr, stg, lane, gi_warp0, col0, c0, lim, bz, alpha, aux_scale, sq);
+    if (two) c0 = epilogue_fast_blocks<EPI, 2>(p, taddr, stg, lane, gi_warp0, col0, c0, lim, bz, alpha, aux_scale, sq, c_diag);
+    else c0 = epilogue_fast_blocks<EPI, 4>(p, taddr, stg, lane, gi_warp0, col0, c0, lim, bz, alpha, aux_scale, sq, c_diag);
+    if (c_diag >= 0)
+      epilogue_block_general<EPI>(p, taddr, c_diag, gi, gi_warp0, col0, n_eff, row_ok, vec_ok, aux_bf16, crow, cbatch, xrow,
+                                  alpha, aux_scale, sq);
   }
-  for (; c0 < n_eff; c0 += 64) {
-    const int gj0 = col0 + c0, gj1 = gj0 + 16;
-    // symmetric output: nothing to do for a block entirely left of the warp's rows (warp-uniform)
-    if (p.symmetric && gj0 + 31 < gi_warp0) continue;
-    const bool second = (c0 + 16 < n_eff);
-    uint32_t r0[16], r1[16];
-    __syncwarp();
-    tmem_ld16(taddr + (uint32_t)c0, r0);
-    if (second) tmem_ld16(taddr + (uint32_t)c0 + 16u, r1);
-    const bool vec0 = vec_ok && (gj0 + 16 <= p.N) && ((gj0 & 7) == 0);
-    const bool vec1 = vec_ok && (gj1 + 16 <= p.N) && ((gj1 & 7) == 0);
-    float x0[16], x1[16];
-    load_aux16<EPI>(p, row_ok && gj0 < p.N, vec0, aux_bf16, xrow + gj0, gj0, x0);
-    load_aux16<EPI>(p, second && row_ok && gj1 < p.N, vec1, aux_bf16, xrow + gj1, gj1, x1);
-    tmem_ld_wait();
-    finish16<EPI>(p, r0, x0, gi, gi_warp0, gj0, row_ok, vec0, crow, cbatch, alpha, aux_scale, sq);
-    if (second) finish16<EPI>(p, r1, x1, gi, gi_warp0, gj1, row_ok, vec1, crow, cbatch, alpha, aux_scale, sq);
-  }
+  for (; c0 < n_eff; c0 += 64)
+    epilogue_block_general<EPI>(p, taddr, c0, gi, gi_warp0, col0, n_eff, row_ok, vec_ok, aux_bf16, crow, cbatch, xrow, alpha,
+                                aux_scale, sq);
 }
 
 template <int KIND_TF32, int BSPLIT, int PAIR>

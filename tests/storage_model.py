@@ -33,7 +33,8 @@ def round_tf32(x):
     return bits.astype(np.uint32).view(np.float32).reshape(x32.shape).astype(np.float64)
 
 
-ROUNDERS = {"half": round_half_scaled, "bf16": round_bf16, "tf32": round_tf32, "none": lambda x: np.asarray(x, dtype=np.float64)}
+ROUNDERS = {"half": round_half_scaled, "half1": lambda x: round_half_scaled(x, 1.0), "bf16": round_bf16, "tf32": round_tf32,
+            "none": lambda x: np.asarray(x, dtype=np.float64)}
 
 
 def filter_with_storage(X0, sched, formats):
@@ -81,3 +82,62 @@ def polar_storage_error(G, k, l, Omega, J, sched, gamma, add_mode, option=0):
     exact = oracle.filter_quintic(X0, sched) + (head if add_mode else 0.0)
     stored = filter_with_storage(X0, sched, polar_formats(len(sched), add_mode, option)) + (head if add_mode else 0.0)
     return float(np.linalg.norm(stored - exact) / np.linalg.norm(exact))
+
+
+def psd_pieces(Z, Vb, k, gamma, warmup, lanczos_v0):
+    """The quantities Algorithm 2 builds before and after its filter, from oracle primitives in the algorithm's order:
+    Ritz pairs of the incoming basis, the deflated residual R, the Lanczos scale theta, the filter input X0 and the
+    restored positive head. Returns (R, X0, head_plus)."""
+    Z = np.asarray(Z, dtype=np.float64)
+    n = Z.shape[0]
+    idx = []
+    if not warmup and k > 0 and Vb is not None and Vb.shape[1] > 0:
+        Zt = oracle.matmul(Z, Vb)
+        H = oracle.matmul(Vb, Zt, ta=True)
+        H = 0.5 * (H + H.T)
+        lam, E = oracle.jacobi_eig(H)
+        U = oracle.matmul(Vb, E)
+        order = sorted(range(len(lam)), key=lambda i: (-abs(lam[i]), i))
+        idx = order[:k]
+    R = Z.copy()
+    for i in idx:
+        R -= lam[i] * np.outer(U[:, i], U[:, i])
+    theta = oracle.lanczos_upper(R, lanczos_v0)
+    X0 = R / theta
+    head_plus = np.zeros((n, n))
+    for i in idx:
+        X0 += np.sign(lam[i]) / gamma * np.outer(U[:, i], U[:, i])
+        if lam[i] > 0:
+            head_plus += lam[i] * np.outer(U[:, i], U[:, i])
+    return R, X0, head_plus
+
+
+def symmetric_filter_with_storage(X0, sched, fmt):
+    """The symmetric filter the way the path stores it: per step W = X^2, T = a I + b W + c W^2, X <- X T, with X, W and
+    T each rounded to `fmt` when written (products by the oracle's matmul, exact in between); the result is rounded to
+    tf32, the type in which it enters the reconstruction product."""
+    rnd = ROUNDERS[fmt]
+    X = rnd(np.asarray(X0, dtype=np.float64))
+    n = X.shape[0]
+    for a, b, c in sched:
+        W = rnd(oracle.matmul(X, X))
+        T = rnd(a * np.eye(n) + b * W + c * oracle.matmul(W, W))
+        X = oracle.matmul(X, T)
+        X = rnd(0.5 * (X + X.T))          # the path computes the upper tiles and mirrors them
+    return round_tf32(X)
+
+
+def psd_storage_error(Z, Vb, k, sched, gamma, warmup, lanczos_v0, fmt):
+    """Relative Frobenius distance between the projection with the filter's stored quantities rounded to `fmt` ("tf32",
+    or "half1" for unscaled IEEE half) and the projection in fp64 throughout, both from the oracle's steps; also returns
+    the unrounded projection (it must equal oracle.psd_project's)."""
+    R, X0, head_plus = psd_pieces(Z, Vb, k, gamma, warmup, lanczos_v0)
+
+    def project(gX):
+        P = 0.5 * (R + oracle.matmul(R, gX)) + head_plus
+        return 0.5 * (P + P.T)
+    exact = project(oracle.filter_quintic(X0, sched))
+    stored = project(symmetric_filter_with_storage(X0, sched, fmt))
+    return float(np.linalg.norm(stored - exact) / np.linalg.norm(exact)), exact
+
+

@@ -4,17 +4,19 @@ import pytest
 import torch
 
 import oracle
+import storage_model
 from paper_2609_21102_b200 import inputs
 
 pytestmark = pytest.mark.gpu
 
 SCHED = [list(oracle.CLASSICAL_QUINTIC)] * 10
-# Per-iteration tolerance on S relative to ||S||_F. fp32 engine: rounding only. tf32 tensor engine: every product
-# rounds the iterate to 11 significant bits, a perturbation E with ||E||_F ~ 2^-11 sqrt(n) of an iterate whose
-# eigenvalues are near +-1, passed on with gain ~theta: here no large head dominates ||S||_F (theta 9-20 against
-# ||S||_F 20-60), so the relative figure is larger than on the head-dominated SDP workload of the projection tests;
-# measured 1.0e-3 to 3.8e-3 per iteration.
-TOL_ENGINE = {"fp32": 1e-4, "tf32": 6e-3, "half": 6e-3}      # "half": the filter steps in IEEE half
+# Per-iteration tolerance on S relative to ||S||_F: the library's bars (fp32 engine: rounding only; tf32 tensor engine
+# and half filter: 2e-3). On the tensor engine the error is, besides, held to what the 11-bit storage of the filter's
+# iterate, of its square and of the step's polynomial explains for that iteration's input, measured on the oracle's
+# side (storage_model.psd_storage_error), times two: a kernel that adds an error of its own (an iterate that is not
+# exactly symmetric, say, which the filter doubles at every step) fails this long before it reaches the bar.
+TOL_ENGINE = {"fp32": 1e-4, "tf32": 2e-3, "half": 2e-3}      # "half": the filter steps in IEEE half
+STORAGE = {"tf32": "tf32", "half": "half1"}
 
 
 @pytest.fixture(scope="module")
@@ -50,7 +52,7 @@ def test_every_iteration_matches_the_oracle(ctx, engine_name):
     st = {"V": V}
 
     def proj(Z, warmup):
-        states.append({"V": st["V"].copy()})
+        states.append({"V": st["V"].copy(), "Z": Z.copy(), "warm": warmup})
         P, Vn, _, _, _ = oracle.psd_project(Z, st["V"], k, SCHED, gamma=1.1, warmup=warmup, lanczos_v0=v0)
         st["V"] = Vn
         return P
@@ -66,6 +68,11 @@ def test_every_iteration_matches_the_oracle(ctx, engine_name):
                                           gamma=1.1, lanczos_start=v0d, exploit_symmetry=True, engine=engine,
                                           half_filter=(engine_name == "half"))
         tol = TOL_ENGINE[engine_name]
+        if engine_name in STORAGE:
+            model, _ = storage_model.psd_storage_error(states[-1]["Z"], states[-1]["V"], k, SCHED, 1.1, states[-1]["warm"],
+                                                       v0, STORAGE[engine_name])
+            tol = min(tol, 2.0 * model + 1e-4)
+            print("admm %s iteration %d: S error %.3e, storage model %.3e, tolerance %.3e" % (engine_name, it, _rel(Sd.cpu().double().numpy(), S1), model, tol))
         assert _rel(Sd.cpu().double().numpy(), S1) <= tol, (it, "S")
         # X_new = sigma (S - Z) is a difference of the projection and its argument: compared on the scale of S
         assert np.linalg.norm(Xd.cpu().double().numpy() - X1) <= tol * sigma * np.linalg.norm(S1), (it, "X")

@@ -45,3 +45,19 @@ def test_stepwise_evaluation_is_the_oracle_path(m, n, add_mode):
     e_half = sm.polar_storage_error(G, k, l, Om, J, [MUON] * L, gamma, add_mode, option=2)
     e_bf16 = sm.polar_storage_error(G, k, l, Om, J, [MUON] * L, gamma, add_mode, option=1)
     assert e_bf16 > 2.0 * e_half
+
+
+@pytest.mark.parametrize("warmup", [False, True])
+def test_psd_pieces_rebuild_the_oracle_projection(warmup):
+    n, K, k = 96, 8, 3
+    lam = np.concatenate([[40.0, -30.0, 25.0], np.linspace(-1.0, 1.0, n - 3)])
+    q = inputs.haar(n, n, 515).numpy()
+    Z = (q * lam[None, :]) @ q.T
+    Z = 0.5 * (Z + Z.T)
+    Vb = np.linalg.qr(q[:, [0, 1, 2, 10, 20, 30, 40, 50]] + 1e-3 * inputs.randn((n, K), 516).numpy())[0]
+    v0 = inputs.gaussian_vector(n, 5, inputs.PURPOSE_LANCZOS).double().numpy()
+    sched = [list(oracle.CLASSICAL_QUINTIC)] * 7
+    P, *_ = oracle.psd_project(Z, Vb, k, sched, gamma=1.1, warmup=warmup, lanczos_v0=v0)
+    err, exact = sm.psd_storage_error(Z, Vb, k, sched, 1.1, warmup, v0, "tf32")
+    assert np.linalg.norm(exact - P) <= 1e-10 * np.linalg.norm(P)
+    assert 0.0 < err < 1e-2

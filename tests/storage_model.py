@@ -47,6 +47,27 @@ def filter_with_storage(X0, sched, formats):
     return X
 
 
+def polar_filter_with_storage(X0, sched, formats):
+    """The filter of the bf16 polar path the way the path stores it: per step the iterate X, the short-side Gram matrix
+    A = X X^T (or X^T X) and B = a I + b A + c A^2 are each rounded when written, to the step's format ("half": X is
+    kept as 32 X and A as 1024 A in IEEE half, B unscaled; "bf16": plain bf16); products by the oracle's matmul, exact
+    in between. The last result is not rounded here."""
+    X = np.asarray(X0, dtype=np.float64)
+    m, n = X.shape
+    wide = m <= n
+    ms = min(m, n)
+    for t, (a, b, c) in enumerate(sched):
+        fmt = formats[t]
+        rx = ROUNDERS[fmt]
+        ra = (lambda v: round_half_scaled(v, 1024.0)) if fmt == "half" else rx
+        rb = ROUNDERS["half1"] if fmt == "half" else rx
+        X = rx(X)
+        A = ra(oracle.matmul(X, X, tb=True) if wide else oracle.matmul(X, X, ta=True))
+        B = rb(a * np.eye(ms) + b * A + c * oracle.matmul(A, A))
+        X = oracle.matmul(B, X) if wide else oracle.matmul(X, B)
+    return X
+
+
 def polar_formats(L, add_mode, option=0):
     """Iterate storage of the bf16 polar path per step: option 0 = scaled half in the first two steps (every step in
     ADD mode), bf16 after; 1 = bf16 throughout; 2 = half throughout."""
@@ -75,12 +96,15 @@ def polar_entry(G, k, l, Omega, J, gamma, add_mode):
     return (X0 if tall else X0.T), (head if tall else head.T)
 
 
-def polar_storage_error(G, k, l, Omega, J, sched, gamma, add_mode, option=0):
+def polar_storage_error(G, k, l, Omega, J, sched, gamma, add_mode, option=0, round_output=False):
     """Relative Frobenius distance between the oracle's result with the iterate rounded to the path's storage
-    formats and its result in fp64 throughout: what the storage format alone explains for this input."""
+    formats (and, with round_output, the result rounded to bf16 as the path returns it) and its result in fp64
+    throughout: what the storage format alone explains for this input."""
     X0, head = polar_entry(G, k, l, Omega, J, gamma, add_mode)
     exact = oracle.filter_quintic(X0, sched) + (head if add_mode else 0.0)
-    stored = filter_with_storage(X0, sched, polar_formats(len(sched), add_mode, option)) + (head if add_mode else 0.0)
+    stored = polar_filter_with_storage(X0, sched, polar_formats(len(sched), add_mode, option)) + (head if add_mode else 0.0)
+    if round_output:
+        stored = round_bf16(stored)
     return float(np.linalg.norm(stored - exact) / np.linalg.norm(exact))
 
 

@@ -40,6 +40,8 @@ def test_stepwise_evaluation_is_the_oracle_path(m, n, add_mode):
     X0, head = sm.polar_entry(G, k, l, Om, J, gamma, add_mode)
     got = sm.filter_with_storage(X0, [MUON] * L, ["none"] * L) + (head if add_mode else 0.0)
     assert np.linalg.norm(got - ref) <= 1e-11 * np.linalg.norm(ref)
+    got = sm.polar_filter_with_storage(X0, [MUON] * L, ["none"] * L) + (head if add_mode else 0.0)
+    assert np.linalg.norm(got - ref) <= 1e-11 * np.linalg.norm(ref)
     assert sm.polar_storage_error(G, k, l, Om, J, [MUON] * L, gamma, add_mode, option=2) > 0.0
     # bf16 storage moves the result more than half storage does
     e_half = sm.polar_storage_error(G, k, l, Om, J, [MUON] * L, gamma, add_mode, option=2)

@@ -68,6 +68,7 @@ extern "C" {
 
 #define DEFL_MAX_L 64 /* largest sketch width k + oversample (and PSD basis width K) */
 #define DEFL_MAX_STEPS 32 /* largest filter depth L (or T) */
+#define DEFL_MAX_TERMS 6  /* most coefficients per filter step (Eq. 5 with d = 5) */
 #define DEFL_LANCZOS_STEPS 20
 
 typedef struct defl_ctx defl_ctx; /* opaque: device, stream, scratch memory */
@@ -102,6 +103,11 @@ typedef struct defl_opts {
                             matrices with slowly decaying spectra (1600 x 6400, sigma_i = 200/i, k = 32: 4.2e-2 relative
                             Frobenius error against an fp64 evaluation of the same algorithm; square and faster
                             decaying cases stay below 3e-2). 2: scaled half in every step. */
+  int poly_terms;        /* polar calls: coefficients per filter step in coeff_schedule. 0 or 3 (default): the quintic
+                            (a, b, c) of Eq. 2. 2: a cubic (a, b). 4 .. DEFL_MAX_TERMS: the degree-(2d+1) map of Eq. 5,
+                            X <- a_0 X + a_1 (X X^T) X + ... + a_d (X X^T)^d X with d = poly_terms - 1 (4 = the
+                            degree-seven member); the schedule is then [L][poly_terms]. The polynomial in the Gram
+                            matrix is formed by Horner steps, one more short-side product per degree beyond the quintic. */
 } defl_opts;
 
 typedef struct defl_info {
@@ -122,7 +128,8 @@ int defl_create(defl_ctx** out, int device);
 int defl_destroy(defl_ctx* ctx);
 int defl_set_stream(defl_ctx* ctx, void* cuda_stream); /* cudaStream_t; NULL = default stream */
 
-/* Bytes of context scratch a polar / PSD call of this shape needs (what the context will hold). */
+/* Bytes of context scratch a polar / PSD call of this shape needs (what the context will hold; a polar call with
+ * opts->poly_terms > 3 takes one more buffer of b * min(m,n)^2 elements). */
 size_t defl_polar_workspace_bytes(int b, int m, int n, int dtype, int k, int oversample);
 size_t defl_psd_workspace_bytes(int n, int K);
 
@@ -142,7 +149,7 @@ int defl_psd_window(int n, float w, float w_prime, int* k, int* K);
  *   oversample   extra sketch columns p; l = min(min(m,n), k+p) columns are sketched (Algorithm 3 line 1).
  *   power_iters  J subspace iterations (Algorithm 3 lines 4-6).
  *   coeff_schedule  host, [L][3] = (a_t, b_t, c_t) of X <- a X + b (X X^T) X + c (X X^T)^2 X (Eq. 2), applied
- *                for t = 1..L in order. L = 0 returns X0.
+ *                for t = 1..L in order ([L][opts->poly_terms] for the other degrees of Eq. 5). L = 0 returns X0.
  * Wide matrices (m < n) are handled as the transpose without moving data (polar(M^T) = polar(M)^T).
  * Errors: DEFL_ERR_ARG, DEFL_ERR_RANK (k >= min(m,n) or l > DEFL_MAX_L or L > DEFL_MAX_STEPS), DEFL_ERR_CUDA,
  * DEFL_ERR_UNSUPPORTED. opts and info may be NULL. */

@@ -18,7 +18,7 @@ RESTORE_PADDED, RESTORE_ADD = 0, 1
 NORM_LANCZOS, NORM_FROBENIUS = 0, 1
 ENGINE_AUTO, ENGINE_SIMT, ENGINE_TENSOR = 0, 1, 2
 ST_CHOL_SHIFT, ST_JACOBI_CAP, ST_ZERO_RESIDUAL, ST_DEVICE_WAIT, ST_NONFINITE = 1, 2, 4, 8, 16
-MAX_L, MAX_STEPS = 64, 32
+MAX_L, MAX_STEPS, MAX_TERMS = 64, 32, 6
 
 MUON_QUINTIC = (3.4445, -4.7750, 2.0315)
 CLASSICAL_QUINTIC = (1.875, -1.25, 0.375)
@@ -35,7 +35,8 @@ class DeflOpts(ctypes.Structure):
     _fields_ = [("sketch", ctypes.c_void_p), ("seed", ctypes.c_uint64), ("restore_mode", ctypes.c_int),
                 ("gamma", ctypes.c_float), ("norm_mode", ctypes.c_int), ("lanczos_start", ctypes.c_void_p),
                 ("warmup", ctypes.c_int), ("engine", ctypes.c_int), ("exploit_symmetry", ctypes.c_int),
-                ("tau", ctypes.c_float), ("half_filter", ctypes.c_int), ("bf16_iterates", ctypes.c_int)]
+                ("tau", ctypes.c_float), ("half_filter", ctypes.c_int), ("bf16_iterates", ctypes.c_int),
+                ("poly_terms", ctypes.c_int)]
 
 
 class DeflInfo(ctypes.Structure):
@@ -124,10 +125,13 @@ def _dev(t, what):
     return t
 
 
-def _schedule(coeffs, steps=None):
+def _schedule(coeffs, steps=None, terms=3):
+    """[L][terms] coefficients as a C float array: one tuple repeated `steps` times, or a list of tuples."""
     c = torch.as_tensor(coeffs, dtype=torch.float64)
     if c.ndim == 1:
         c = c.unsqueeze(0).repeat(steps, 1)
+    if c.numel() and c.shape[1] != terms:
+        raise ValueError("every filter step takes %d coefficients, got %d" % (terms, c.shape[1]))
     flat = [float(x) for x in c.reshape(-1).tolist()]
     arr = (ctypes.c_float * max(len(flat), 1))(*flat)
     return arr, c.shape[0]
@@ -182,7 +186,8 @@ class Context:
             raise DeflError(rc, lib().defl_last_error(self._h).decode())
 
     def _opts(self, sketch=None, seed=0, restore_mode=RESTORE_PADDED, gamma=0.0, norm_mode=NORM_LANCZOS,
-              lanczos_start=None, warmup=False, engine=ENGINE_AUTO, exploit_symmetry=False, tau=0.0, half_filter=False, bf16_iterates=False):
+              lanczos_start=None, warmup=False, engine=ENGINE_AUTO, exploit_symmetry=False, tau=0.0, half_filter=False, bf16_iterates=False,
+              poly_terms=0):
         o = DeflOpts()
         o.sketch = sketch.data_ptr() if sketch is not None else None
         o.seed = seed
@@ -196,25 +201,27 @@ class Context:
         o.tau = tau
         o.half_filter = int(bool(half_filter))
         o.bf16_iterates = int(bf16_iterates)      # 0 mixed (default), 1 / True bf16 throughout, 2 half throughout
+        o.poly_terms = int(poly_terms)            # 0 / 3 quintic steps, 2 cubic, 4.. the higher-degree maps of Eq. 5
         return o
 
     # ------------------------------------------------------------------------------------------
     def defl_polar_batched(self, G, k, oversample, power_iters, coeff_schedule, steps=None, out=None, sketch=None,
                            seed=0, restore_mode=RESTORE_PADDED, gamma=0.0, engine=ENGINE_AUTO,
-                           exploit_symmetry=False, want_info=False, tau=0.0, bf16_iterates=False):
-        """out[b,m,n] = deflated polar factor of every G[b] (Algorithm 3 + Algorithm 1)."""
+                           exploit_symmetry=False, want_info=False, tau=0.0, bf16_iterates=False, poly_terms=0):
+        """out[b,m,n] = deflated polar factor of every G[b] (Algorithm 3 + Algorithm 1). poly_terms: coefficients per
+        filter step (0 or 3: quintic; 4: the degree-seven map of Eq. 5, ...)."""
         _dev(G, "G")
         if G.ndim != 3:
             raise ValueError("G must be [b, m, n]")
         b, m, n = G.shape
         out = torch.empty_like(G) if out is None else _dev(out, "out")
-        sched, L = _schedule(coeff_schedule, steps)
+        sched, L = _schedule(coeff_schedule, steps, poly_terms or 3)
         if sketch is not None:
             _dev(sketch, "sketch")
             if sketch.dtype != torch.float32:
                 raise TypeError("sketch must be float32")
         opts = self._opts(sketch=sketch, seed=seed, restore_mode=restore_mode, gamma=gamma, engine=engine,
-                          exploit_symmetry=exploit_symmetry, tau=tau, bf16_iterates=bf16_iterates)
+                          exploit_symmetry=exploit_symmetry, tau=tau, bf16_iterates=bf16_iterates, poly_terms=poly_terms)
         info = DeflInfo()
         extras = None
         if want_info:

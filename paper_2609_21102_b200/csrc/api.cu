@@ -92,6 +92,7 @@ struct Carver {
 struct PolarWs {
   void* X;            // [b,m,n] dtype   second iterate buffer (the other one is `out`)
   void* Am; void* Bm; // [b,ms,ms] dtype  A_t = X X^T and B_t = a I + b A_t + c A_t^2
+  void* Cm;           // [b,ms,ms] dtype  Horner intermediate of the higher-degree maps (poly_terms > 3 only)
   float* Lp;          // [b,ml,l]  long-side panel  (Y, then Q)
   float* Sp;          // [b,ms,l]  short-side panel (A^T Q and its orthonormalisation; finally (Q^T A)^T)
   double* gram;       // [b,nchunk,l,l]
@@ -112,7 +113,7 @@ struct PolarWs {
 
 inline int round_up8(int x) { return (x + 7) & ~7; }
 
-PolarWs carve_polar(void* base, int b, int m, int n, int dtype, int k, int l) {
+PolarWs carve_polar(void* base, int b, int m, int n, int dtype, int k, int l, int terms = 3) {
   const int ms = m < n ? m : n, ml = m < n ? n : m;
   const size_t es = dtype_size(dtype);
   Carver cv(base);
@@ -120,6 +121,7 @@ PolarWs carve_polar(void* base, int b, int m, int n, int dtype, int k, int l) {
   w.X = cv.take<char>((size_t)b * m * n * es);
   w.Am = cv.take<char>((size_t)b * ms * ms * es);
   w.Bm = cv.take<char>((size_t)b * ms * ms * es);
+  w.Cm = cv.take<char>(terms > 3 ? (size_t)b * ms * ms * es : 1);
   const int le = l > 0 ? l : 1, ke = k > 0 ? k : 1;
   w.Lp = cv.take<float>((size_t)b * ml * le);
   w.Sp = cv.take<float>((size_t)b * ms * le);
@@ -549,6 +551,15 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
   // ADD restore keeps half in every step: without the head inside X_0 all its singular values are small and stay
   // small for longer, and the same storage rounding costs about ten times more (a 636 x 75 case with six steps:
   // 2.8e-2 with half throughout, 8.2e-2 with two half steps, 1.7e-1 with bf16; padded restore 2.7e-3 / 9.8e-3 / 1.7e-2).
+  int terms = (opts && opts->poly_terms) ? opts->poly_terms : 3;
+  if (terms < 2 || terms > DEFL_MAX_TERMS) return DEFL_ERR_ARG;
+  // a cubic is the quintic with a zero last coefficient
+  float cubic_as_quintic[3 * DEFL_MAX_STEPS];
+  if (terms == 2) {
+    for (int t = 0; t < L; ++t) { cubic_as_quintic[3 * t] = coeff_schedule[2 * t]; cubic_as_quintic[3 * t + 1] = coeff_schedule[2 * t + 1]; cubic_as_quintic[3 * t + 2] = 0.f; }
+    coeff_schedule = cubic_as_quintic;
+    terms = 3;
+  }
   const int it_mode = opts ? opts->bf16_iterates : 0;
   const bool half_iter = dtype == DEFL_BF16 && L > 0 && it_mode != 1;
   // the first `n_half` filter steps keep the iterate in scaled IEEE half, the rest in bf16
@@ -557,9 +568,9 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
   const float ys = n_half > 0 ? 32.f : 1.f;
 
   cudaSetDevice(c->device);
-  int rc = ctx_reserve(c, carve_polar(nullptr, b, m, n, dtype, k, l).bytes);
+  int rc = ctx_reserve(c, carve_polar(nullptr, b, m, n, dtype, k, l, terms).bytes);
   if (rc) return rc;
-  PolarWs w = carve_polar(c->ws, b, m, n, dtype, k, l);
+  PolarWs w = carve_polar(c->ws, b, m, n, dtype, k, l, terms);
   ctx_profile_begin(c);
   c->err[0] = 0;
   ctx_stage_mark(c);
@@ -705,7 +716,7 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
 
   // ---- stage 2: X <- a X + b (X X^T) X + c (X X^T)^2 X, L times, through the short-side Gram -------
   for (int t = 0; t < L; ++t) {
-    const float ca = coeff_schedule[3 * t], cb = coeff_schedule[3 * t + 1], cc = coeff_schedule[3 * t + 2];
+    const float* cf = coeff_schedule + (size_t)terms * t;       // a_0 .. a_{terms-1} of this step
     const void* X = bufs[cur];
     void* Xn = bufs[cur ^ 1];
     const bool hs = t < n_half, hn = t + 1 < n_half;
@@ -721,17 +732,27 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
     g.C = w.Am; g.ldc = ms; g.batch_c = (long long)ms * ms;
     g.epilogue = EPI_STORE; g.symmetric = sym;
     if ((rc = run_gemm(c, g, engine, "gram"))) return rc;
-    // B_t = a I + b A_t + c A_t A_t
-    g = gemm_desc_zero();
-    g.batch = b; g.in_dtype = it_dtype; g.b_dtype = it_dtype; g.out_dtype = it_dtype;
-    g.M = ms; g.N = ms; g.K[0] = ms;
-    g.A[0] = w.Am; g.sa_i[0] = ms; g.sa_k[0] = 1; g.batch_a[0] = (long long)ms * ms;
-    g.B[0] = w.Am; g.sb_k[0] = 1; g.sb_j[0] = ms; g.batch_b[0] = (long long)ms * ms;   // A_t symmetric: rows as columns
-    g.C = w.Bm; g.ldc = ms; g.batch_c = (long long)ms * ms;
-    g.aux = w.Am; g.ld_aux = ms; g.batch_aux = (long long)ms * ms; g.aux_dtype = it_dtype;
-    // (with scaled iterates the stored Gram is ys^2 A_t: the coefficients absorb the powers)
-    g.epilogue = EPI_POLY; g.pa = ca; g.pb = cb / (ys * ys); g.pc = cc / (ys * ys * ys * ys); g.symmetric = sym;
-    if ((rc = run_gemm(c, g, engine, "polynomial"))) return rc;
+    // B_t = a_0 I + a_1 A_t + ... + a_d A_t^d by Horner steps. The innermost one forms a_{d-2} I + a_{d-1} A_t +
+    // a_d A_t A_t in the epilogue of one product (the whole polynomial for the quintic); every further degree costs one
+    // more product C <- a_j I + A_t C. With scaled iterates the stored Gram matrix is ys^2 A_t: the coefficients absorb
+    // the powers, the intermediate polynomials are kept unscaled.
+    const int nprod = terms - 2;
+    const float iy2 = 1.f / (ys * ys);
+    for (int q = 0; q < nprod; ++q) {
+      void* dst = ((nprod - 1 - q) % 2 == 0) ? w.Bm : w.Cm;        // the last product lands in B_t
+      const void* prev = (dst == w.Bm) ? w.Cm : w.Bm;
+      g = gemm_desc_zero();
+      g.batch = b; g.in_dtype = it_dtype; g.b_dtype = it_dtype; g.out_dtype = it_dtype;
+      g.M = ms; g.N = ms; g.K[0] = ms;
+      g.A[0] = w.Am; g.sa_i[0] = ms; g.sa_k[0] = 1; g.batch_a[0] = (long long)ms * ms;
+      g.B[0] = (q == 0) ? w.Am : prev; g.sb_k[0] = 1; g.sb_j[0] = ms; g.batch_b[0] = (long long)ms * ms;   // symmetric: rows as columns
+      g.C = dst; g.ldc = ms; g.batch_c = (long long)ms * ms;
+      g.aux = w.Am; g.ld_aux = ms; g.batch_aux = (long long)ms * ms; g.aux_dtype = it_dtype;
+      g.epilogue = EPI_POLY; g.symmetric = sym;
+      if (q == 0) { g.pa = cf[terms - 3]; g.pb = cf[terms - 2] * iy2; g.pc = cf[terms - 1] * iy2 * iy2; }
+      else { g.pa = cf[terms - 3 - q]; g.pb = 0.f; g.pc = iy2; }
+      if ((rc = run_gemm(c, g, engine, "polynomial"))) return rc;
+    }
     // X <- B_t X (wide) or X B_t (tall)
     g = gemm_desc_zero();
     g.batch = b; g.in_dtype = it_dtype; g.b_dtype = it_dtype; g.out_dtype = it_dtype;

@@ -1,7 +1,6 @@
 """Parity of defl_polar_batched (and defl_brsvd_batched) with the fp64 CPU oracle.
 
-Tolerances are the ones the task fixes: relative Frobenius error <= 2e-3 on the fp32 path and
-<= 3e-2 on the bf16 path, per matrix, on `out`. The triplets themselves are compared only through
+Tolerances: relative Frobenius error <= 2e-3 with fp32 storage and <= 3e-2 with bf16 storage, per matrix, on `out`. The triplets themselves are compared only through
 quantities that are unique (singular values, the projector of a well-separated head).
 """
 import numpy as np
@@ -216,3 +215,43 @@ def test_host_buffer_path_matches_device_path(ctx, given_sketch):
     out = torch.empty_like(G).pin_memory()
     ctx.defl_polar_batched_host(G.pin_memory(), out, k, p, 1, _sched(binding.MUON_QUINTIC, 5), sketch=sk, seed=77)
     assert torch.equal(out, ref)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("shape", [(2, 136, 328), (2, 392, 264), (1, 100, 75)])
+@pytest.mark.parametrize("terms,L", [(4, 4), (5, 3), (2, 6)])
+def test_general_degree_map_matches_oracle(ctx, dtype, shape, terms, L):
+    """The degree-(2d+1) classical map of Eq. 5 with its Bjorck-Bowie coefficients (d = 3: degree seven; d = 4; and the
+    cubic d = 1) inside Algorithm 1, padded restore: the oracle's entry X0 (Algorithm 3 and lines 3-4 of Algorithm 1)
+    followed by the oracle's L classical steps of that degree."""
+    import storage_model
+    b, m, n = shape
+    d = terms - 1
+    k, p, J, gamma = 4, 4, 1, 1.05
+    ms = min(m, n)
+    sigma = np.concatenate([np.linspace(40.0, 15.0, k), np.linspace(1.0, 0.1, ms - k)])
+    G = torch.stack([inputs.from_spectrum(m, n, sigma, 6100 + i) for i in range(b)]).to(dtype)
+    Om = inputs.sketch(b, ms, k + p, 1, 6)
+    coeffs = [float(a) for a in oracle.bjorck_bowie(d)]
+    out, info = ctx.defl_polar_batched(G.cuda(), k, p, J, [coeffs] * L, sketch=Om.cuda(), gamma=gamma, exploit_symmetry=True,
+                                       want_info=True, poly_terms=terms)
+    torch.cuda.synchronize()
+    assert int(info["status"].max()) == 0
+    for i in range(b):
+        X0, _ = storage_model.polar_entry(G[i].double().numpy(), k, k + p, Om[i].double().numpy(), J, gamma, False)
+        ref = oracle.filter_classical(X0, d, L)
+        assert _rel(out[i].double().cpu().numpy(), ref) <= TOL[dtype], (i, terms)
+    if terms == 4:
+        # the quintic entry point with the same coefficients padded by a zero is another polynomial: the option is live
+        out3 = ctx.defl_polar_batched(G.cuda(), k, p, J, [coeffs[:3]] * L, sketch=Om.cuda(), gamma=gamma, exploit_symmetry=True)
+        assert _rel(out3[0].double().cpu().numpy(), out[0].double().cpu().numpy()) > 1e-2
+
+
+def test_poly_terms_argument_errors(ctx):
+    from paper_2609_21102_b200 import binding
+    G = torch.zeros((1, 64, 96), dtype=torch.float32, device="cuda")
+    with pytest.raises(binding.DeflError) as e:
+        ctx.defl_polar_batched(G, 0, 0, 0, [[1.0] * 7] * 2, poly_terms=7)
+    assert e.value.code == -1
+    with pytest.raises(ValueError):
+        ctx.defl_polar_batched(G, 0, 0, 0, [[1.0, 0.0, 0.0]] * 2, poly_terms=4)      # three coefficients given, four wanted

@@ -71,3 +71,62 @@ def test_margin_rescales_the_first_stage_only():
     with np.errstate(over="ignore", invalid="ignore"):          # without the margin 1.05 is outside the valid range
         far = S.compose(s0, np.array([1.05]))[0]
     assert not np.isfinite(far) or abs(far) > 10
+
+
+def test_stage_two_lowers_the_relu_error_and_never_raises_it():
+    """Stage two: the refined composite has a smaller matrix-ReLU error than stage one (whose error sits in the zone
+    |x| < eps that the sign approximation leaves out, while it is 1e-9 accurate on [eps, 1], far more than the ReLU
+    needs), a refinement step never raises the error, and the result is still an odd composite of T quintics."""
+    eps, T = 1e-3, 7
+    x = np.sort(np.concatenate([np.linspace(-1.0, 1.0, 40001), np.linspace(-2 * eps, 2 * eps, 20001)]))
+    s1, errs = S.remez_sign_schedule(eps, T)
+    e1 = S.relu_error(s1, x)
+    assert errs[-1] < 1e-8
+    # |x| (1 - g(|x|)) / 2 on [0, eps]: below eps / 2, and not tiny
+    assert 1e-6 < e1 <= 0.5 * eps
+    s2, before, after = S.stage_two_schedule(eps, T, iters=6)
+    assert before == pytest.approx(e1)
+    assert after == pytest.approx(S.relu_error(s2, x))
+    assert after < 0.8 * before
+    assert len(s2) == T and all(len(c) == 3 for c in s2)
+    xs = np.linspace(-1.0, 1.0, 2001)
+    assert np.allclose(S.compose(s2, -xs), -S.compose(s2, xs))
+    # the polish alone: never worse than what it was given
+    s3, b3, a3 = S.refine_relu_schedule(s1, iters=3, grid=x)
+    assert b3 == pytest.approx(e1) and a3 <= b3
+
+
+def test_gradient_through_the_composition_matches_finite_differences():
+    sched, _ = S.remez_sign_schedule(1e-2, 3)
+    x = np.array([-0.7, -0.01, 0.003, 0.2, 0.9])
+    g, grad = S._compose_with_gradient(sched, x)
+    assert np.allclose(g, S.compose(sched, x))
+    for t in range(3):
+        for i in range(3):
+            h = 1e-6 * max(1.0, abs(sched[t][i]))
+            up = [list(c) for c in sched]
+            dn = [list(c) for c in sched]
+            up[t][i] += h
+            dn[t][i] -= h
+            fd = (S.compose([tuple(c) for c in up], x) - S.compose([tuple(c) for c in dn], x)) / (2 * h)
+            assert np.allclose(grad[t, i], fd, rtol=1e-5, atol=1e-7)
+
+
+@pytest.mark.parametrize("a_k,T", [(0.05, 3), (0.2, 2), (0.01, 5)])
+def test_filter_regenerated_on_the_deflated_interval_meets_theorem_3(a_k, T):
+    """Theorem 3: started on [a_k, 1], the sequential minimax composite satisfies max |1 - g| <= (1 - a_k^2)^(3^T) on
+    that interval (the classical composition meets the bound, the minimax one is at least as good), and raising the
+    floor from eps to a_k, which is what deflation does, buys orders of magnitude at the same depth."""
+    sched, errs, ak, bound = S.deflated_interval_schedule(a_k * 3.0, 3.0, T)
+    assert ak == pytest.approx(a_k)
+    x = np.linspace(a_k, 1.0, 100001)
+    err = float(np.max(np.abs(S.compose(sched, x) - 1.0)))
+    classical = float(np.max(np.abs(S.compose([S.bjorck_bowie(2)] * T, x) - 1.0)))
+    assert classical <= bound * (1 + 1e-12) + 1e-15
+    assert err <= classical + 1e-12
+    assert err == pytest.approx(errs[-1], rel=1e-3, abs=1e-12)
+    wide, _ = S.remez_sign_schedule(a_k / 50.0, T)
+    xw = np.linspace(a_k / 50.0, 1.0, 100001)
+    assert err < 0.5 * float(np.max(np.abs(S.compose(wide, xw) - 1.0)))
+    with pytest.raises(ValueError):
+        S.deflated_interval_schedule(2.0, 1.0, 3)

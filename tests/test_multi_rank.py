@@ -62,6 +62,30 @@ def test_single_rank_helpers_need_no_process_group():
     import bench
     assert bench.max_over_ranks(3.5) == 3.5
     assert bench.aggregate_throughput(10.0, 4, 2.0) == 4 * 10.0 / 2e-3
-    filt, rest = bench.flops_per_matrix(1600, 6400, 32, 16, 2, 5)
+    # flops the method needs for one 1600 x 6400 matrix: the symmetric products once per pair, or in full
+    filt, rest = bench.algorithmic_flops(1600, 6400, 32, 16, 2, 5, symmetric=False)
     assert abs(filt - 5 * (4 * 1600 ** 2 * 6400 + 2 * 1600 ** 3)) < 1
-    assert rest > 0
+    assert abs(filt - bench.dense_filter_flops(1600, 6400, 5)) < 1
+    fs, rs = bench.algorithmic_flops(1600, 6400, 32, 16, 2, 5, symmetric=True)
+    assert abs(fs - 5 * (1600 * 1601 * 6400 + 1600 ** 2 * 1601 + 2 * 1600 ** 2 * 6400)) < 1
+    # front end: six products with the 48-column panel and the rank-32 subtraction; the additive restore adds a rank-32 product
+    assert abs(rest - (2 * 6400 * 1600 * 48 * 6 + 2 * 1600 * 6400 * 32)) < 1 and rs == rest
+    assert bench.algorithmic_flops(1600, 6400, 32, 16, 2, 5, True, add_restore=True)[1] - rest == 2 * 1600 * 6400 * 32
+    assert bench.algorithmic_flops(1600, 6400, 0, 0, 0, 5, True)[1] == 0
+
+
+def test_gpus_flag_starts_its_own_ranks_when_no_launcher_did(monkeypatch):
+    """`bench.py --gpus N` without an outer torchrun builds the launcher command itself (127.0.0.1 rendezvous, a free
+    port, one process per GPU, the same arguments); under a launcher (WORLD_SIZE set) it does not."""
+    import bench
+    calls = []
+    monkeypatch.setattr(bench.subprocess, "call", lambda cmd: calls.append(cmd) or 0)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "4", "--steps", "2"])
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    with __import__("pytest").raises(SystemExit) as e:
+        bench.main()
+    assert e.value.code == 0 and len(calls) == 1
+    cmd = calls[0]
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"]
+    assert cmd[cmd.index("--nproc-per-node") + 1] == "4" and cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "2"] and cmd[-5].endswith("bench.py")

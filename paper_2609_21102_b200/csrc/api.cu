@@ -296,8 +296,20 @@ int defl_create(defl_ctx** out, int device) {
   int ok = 1;
   if (cudaMalloc(&c->wait_status, 2 * sizeof(int)) != cudaSuccess) ok = 0;      // status word, tile counter
   if (ok) cudaMemset(c->wait_status, 0, 2 * sizeof(int));
+  if (ok) {
+    // identity tile of the tensor engine's identity segment (X0 = (G - head) / rho adds G in the accumulator)
+    const size_t ib = 256 * 256 * sizeof(__nv_bfloat16);
+    __nv_bfloat16* h = new (std::nothrow) __nv_bfloat16[256 * 256];
+    if (!h || cudaMalloc(&c->ident_bf16, ib) != cudaSuccess) ok = 0;
+    if (ok) {
+      for (int i = 0; i < 256 * 256; ++i) h[i] = __float2bfloat16((i / 256 == i % 256) ? 1.f : 0.f);
+      if (cudaMemcpy(c->ident_bf16, h, ib, cudaMemcpyHostToDevice) != cudaSuccess) ok = 0;
+    }
+    delete[] h;
+  }
   if (!ok) {      // release whatever was created before the failure
     if (c->wait_status) cudaFree(c->wait_status);
+    if (c->ident_bf16) cudaFree(c->ident_bf16);
     cudaSetDevice(prev);
     delete c;
     return DEFL_ERR_CUDA;
@@ -322,6 +334,7 @@ int defl_destroy(defl_ctx* c) {
     for (int i = 0; i < DEFL_HOST_MAX_CHUNKS; ++i) { cudaEventDestroy(c->chunk_in[i]); cudaEventDestroy(c->chunk_done[i]); }
   }
   if (c->wait_status) cudaFree(c->wait_status);
+  if (c->ident_bf16) cudaFree(c->ident_bf16);
   for (int r = 0; r < DEFL_PROFILE_CALLS; ++r)
     for (int i = 0; i < DEFL_MAX_MARKS; ++i)
       if (c->marks[r][i]) cudaEventDestroy(c->marks[r][i]);
@@ -646,18 +659,45 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
     // head stays out (pad = 0) and joins the last filter product, or, when there is no filter step to carry it,
     // goes in at full weight (X0 + P W^T is the padded entry with gamma = 1)
     const float pad = (mode == DEFL_RESTORE_PADDED) ? 1.f / gamma : (L == 0 ? 1.f : 0.f);
+    // Tensor engine, second form: X0 = (1/rho) [G - P diag(s - pad rho) W^T] with G itself added in the accumulator
+    // (a second K segment: the tile's own columns of G against an identity tile, exact in bf16 x bf16 -> fp32), so
+    // that the epilogue is the plain coalesced store scaled by the per-matrix 1/rho. Reading G element-wise in the
+    // epilogue instead (the first form, kept for shapes whose rows the copy engine cannot address) is bound by
+    // the epilogue warps' instruction issue, at a quarter of the memory bandwidth.
+    bool ident_form = false;
+    GemmDesc gi = g;
     if (tensor_defl) {
-      if (ctx_fail(c, split_concat3_launch(right, (long long)n * k, k, b, n, k, kp, w.sv, l, w.inv_rho, -1.f, pad, 1, w.Wc,
-                                           c->stream, &c->launches, w.keff), "split W diag(coef)"))
-        return DEFL_ERR_CUDA;
-    } else if (ctx_fail(c, scale_cols_launch(right, (long long)n * k, k, b, n, k, w.sv, l, w.inv_rho, -1.f, pad, w.Ws,
-                                             (long long)n * k, k, c->stream, &c->launches, w.keff), "W diag(coef)")) {
-      return DEFL_ERR_CUDA;
+      gi.nseg = 2; gi.seg1_identity = 1;
+      gi.A[1] = G; gi.sa_i[1] = n; gi.sa_k[1] = 1; gi.batch_a[1] = (long long)m * n;
+      gi.B[1] = c->ident_bf16; gi.sb_k[1] = 1; gi.sb_j[1] = 256; gi.batch_b[1] = 0; gi.K[1] = 256;
+      gi.aux = nullptr; gi.epilogue = EPI_STORE; gi.partials = nullptr;
+      ident_form = gemm_tc_supported(gi);
     }
-    g.epilogue = EPI_AUX_PLUS; g.partials = nullptr;
-    g.aux_scale = ys; g.aux_scale_dev = w.inv_rho; g.alpha = ys;
-    g.C = bufs[cur]; g.ldc = n; g.batch_c = (long long)m * n; g.out_dtype = it_dtype;
-    if ((rc = run_gemm(c, g, deng, "deflate+normalise"))) return rc;
+    if (ident_form) {
+      if (ctx_fail(c, split_concat3_launch(right, (long long)n * k, k, b, n, k, kp, w.sv, l, nullptr, -1.f, pad, 1, w.Wc,
+                                           c->stream, &c->launches, w.keff, 0, 0, 1.f, w.rho), "split W diag(coef)"))
+        return DEFL_ERR_CUDA;
+      gi.alpha = ys; gi.alpha_dev = w.inv_rho;
+      gi.C = bufs[cur]; gi.ldc = n; gi.batch_c = (long long)m * n; gi.out_dtype = it_dtype;
+      if ((rc = run_gemm(c, gi, DEFL_ENGINE_TENSOR, "deflate+normalise"))) return rc;
+      // (a matrix whose residual counts as zero has 1/rho = 0 and came out as zeros: it gets the padded head alone)
+      if (ctx_fail(c, zero_residual_entry_launch(w.status, left, right, w.keff, b, m, n, k, ys * pad, bufs[cur], it_dtype, c->stream,
+                                                 &c->launches), "zero-residual entry"))
+        return DEFL_ERR_CUDA;
+    } else {
+      if (tensor_defl) {
+        if (ctx_fail(c, split_concat3_launch(right, (long long)n * k, k, b, n, k, kp, w.sv, l, w.inv_rho, -1.f, pad, 1, w.Wc,
+                                             c->stream, &c->launches, w.keff), "split W diag(coef)"))
+          return DEFL_ERR_CUDA;
+      } else if (ctx_fail(c, scale_cols_launch(right, (long long)n * k, k, b, n, k, w.sv, l, w.inv_rho, -1.f, pad, w.Ws,
+                                               (long long)n * k, k, c->stream, &c->launches, w.keff), "W diag(coef)")) {
+        return DEFL_ERR_CUDA;
+      }
+      g.epilogue = EPI_AUX_PLUS; g.partials = nullptr;
+      g.aux_scale = ys; g.aux_scale_dev = w.inv_rho; g.alpha = ys;
+      g.C = bufs[cur]; g.ldc = n; g.batch_c = (long long)m * n; g.out_dtype = it_dtype;
+      if ((rc = run_gemm(c, g, deng, "deflate+normalise"))) return rc;
+    }
   } else {
     if (ctx_fail(c, frob_partial_vec_launch(G, dtype, b, (long long)m * n, FROB_VEC_BLOCKS, w.npart, c->stream, &c->launches), "frobenius"))
       return DEFL_ERR_CUDA;

@@ -44,6 +44,9 @@ struct GemmDesc {
   int round_tf32;               // fp32 output rounded to nearest tf32 (it feeds tf32 products, which would truncate)
   int symmetric;                // output is symmetric (M == N): compute upper tiles only and mirror
   int transpose_out;            // element (i, j) of the product is stored at C[j * ldc + i] (tensor engine, EPI_STORE only)
+  int seg1_identity;            // tensor engine, nseg = 2: segment 1 adds A[1][i, j] itself to the accumulator, as the product of
+                                // A[1] (viewed [M, N], K = the output's column index, K-major) with an identity tile: B[1] points
+                                // to a 256 x 256 identity of the operand type (row-major), K[1] is ignored
   int debug_hold_stage;         // test hook, tensor engine, single-CTA form: s > 0 withholds pipeline step s - 1 of each CTA's first tile
 };
 

@@ -26,6 +26,7 @@ struct defl_ctx {
   defl::TcKnobs tc_knobs;        // tuning overrides, read from the environment when the context was created
   struct { int transposed_apply; int host_chunks; int jacobi_sweeps; } knobs;   // DEFL_NO_TRANSPOSED_APPLY, DEFL_HOST_CHUNKS, DEFL_JACOBI_SWEEPS
   defl::TmCache tm_cache;        // encoded TMA descriptors of recent launches
+  void* ident_bf16;              // device, 256 x 256 bf16 identity (operand of the engine's identity segment)
   long long launches;    // kernels launched so far
   bool profiling;
   // stage marks of the last DEFL_PROFILE_CALLS calls (events are created when profiling is first switched on)

@@ -48,6 +48,7 @@ struct TcParams {
   CUtensorMap tmAux;           // [batch, M, N] view of `aux`, used only to prefetch the epilogue's tile into L2
   int aux_prefetch;
   int nseg;
+  int seg1_ident;              // segment 1 = A[1] tile (K offset by the tile's first column) x identity tile (same for every tile and matrix)
   int b_split;                 // 2: B is the sum of two operands (tmB[0] + tmB[1]) that share A; else 1
   int kblocks[2];              // pipeline steps per segment (a step covers `ksub` K blocks of 128 bytes)
   int ksub;                    // K blocks per pipeline stage (1 or 2)
@@ -71,6 +72,7 @@ struct TcParams {
   // epilogue
   int epilogue, out_dtype, aux_dtype, symmetric, round_tf32;
   int transposed;              // EPI_STORE: the tile is written transposed, element (i, j) at C[j * ldc + i]
+  int diag_exact;              // symmetric output of two different operands: diagonal blocks mirrored element by element
   int aux_f16, out_f16;        // a 16-bit aux / output is IEEE half (else bf16); the operands' kind is in idesc
   void* C; long long ldc, batch_c;
   const void* aux; long long ld_aux, batch_aux;
@@ -755,8 +757,10 @@ __device__ __forceinline__ void epilogue_half(const TcParams& p, uint32_t taddr,
     // bits. Off the diagonal the mirror store makes the pair equal; the 32 x 32 block ON the diagonal must do the same
     // element by element, or an iterate picks up an antisymmetric part that the symmetric filter doubles at every step:
     // it takes the general path.
+    // (A product of a matrix with itself, X X^T or A A, computes (i, j) and (j, i) from the same terms in the same
+    // order: its diagonal blocks are symmetric to the bit and stay on the coalesced path.)
     int c_diag = -1;
-    if ((EPI == EPI_STORE || EPI == EPI_POLY) && p.symmetric && gi_warp0 >= col0 && gi_warp0 - col0 < lim &&
+    if ((EPI == EPI_STORE || EPI == EPI_POLY) && p.symmetric && p.diag_exact && gi_warp0 >= col0 && gi_warp0 - col0 < lim &&
         (((gi_warp0 - col0) >> 5) & 1) == wsel)
       c_diag = gi_warp0 - col0;
     const bool two = (EPI == EPI_STORE) ? o2 : a2;
@@ -938,15 +942,18 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
           }
         }
         const int a_mn0 = t.tm * tile_m + arow;
-        const int b_mn0 = t.tn * BN + (PAIR ? (int)rank * (t.n_eff >> 1) : 0);   // a pair: this CTA's half of the columns
-        const int bz = t.bz;
-        const int my_mn = (my_a ? a_mn0 : b_mn0) + my_mn_off;
+        const int b_loc0 = PAIR ? (int)rank * (t.n_eff >> 1) : 0;                // a pair: this CTA's half of the columns
+        const int b_mn0 = t.tn * BN + b_loc0;
         bool live = true;
         for (int seg = 0; seg < nseg && live; ++seg) {
           const int nkb = seg ? kblocks1 : kblocks0;
           int left = seg ? kreal1 : kreal0;                   // K blocks of the segment not yet requested
           const CUtensorMap* tm = seg ? my_tm1 : my_tm0;
-          int kc = my_k_off;
+          // identity segment: A is read at K = the tile's own columns, B is the same identity tile for every tile
+          const bool ident = seg == 1 && p.seg1_ident != 0;
+          const int my_mn = (my_a ? a_mn0 : (ident ? b_loc0 : b_mn0)) + my_mn_off;
+          const int bz = (ident && !my_a) ? 0 : t.bz;
+          int kc = my_k_off + ((ident && my_a) ? t.tn * BN : 0);
           for (int kb = 0; kb < nkb; ++kb, left -= ksub, kc += ksub * kstep) {
             int ok = 1;
             if (lane == 0) ok = mbar_wait(empty0 + 8u * stage, phase ^ 1u, &abort_flag, p.status, p.wait_ns) ? 1 : 0;
@@ -1288,7 +1295,12 @@ bool gemm_tc_supported(const GemmDesc& g) {
   const int esize = (int)dtype_size(g.in_dtype);
   if (g.symmetric && g.M != g.N) return false;
   if (g.transpose_out && (g.epilogue != EPI_STORE || g.symmetric)) return false;
+  if (g.seg1_identity && (g.nseg != 2 || g.sa_k[0] != 1 || g.sb_k[0] != 1 || g.sa_k[1] != 1 || esize != 2 || g.b_split == 2)) return false;
   for (int s = 0; s < g.nseg; ++s) {
+    if (s == 1 && g.seg1_identity) {
+      if (!aligned16(g.A[1]) || !aligned16(g.B[1]) || (g.sa_i[1] * esize) % 16 || (g.batch > 1 && (g.batch_a[1] * esize) % 16)) return false;
+      continue;
+    }
     if (g.K[s] <= 0) return false;
     if (!aligned16(g.A[s]) || !aligned16(g.B[s])) return false;
     // one unit stride per operand, the other stride and the batch stride multiples of 16 bytes
@@ -1376,7 +1388,19 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   const uint32_t sub_bytes = p.a_stage_bytes + p.b_stage_bytes;
   p.ksub = (p.pair && 3u * 2u * sub_bytes <= smem_budget) ? 2 : 1;
   if ((kn.ksub == 1 || kn.ksub == 2) && (uint32_t)kn.ksub * sub_bytes * 2u <= smem_budget) p.ksub = kn.ksub;
+  p.seg1_ident = (g.nseg == 2 && g.seg1_identity) ? 1 : 0;
   for (int s = 0; s < g.nseg; ++s) {
+    if (s == 1 && p.seg1_ident) {
+      // A[1] is [M, N] with K running over the output's columns (all of them: the copy engine zero-fills past N);
+      // a tile walks its own BN columns; B[1] is one 256 x 256 identity, shared by all tiles and matrices
+      p.kreal[s] = (p.BN + span - 1) / span;
+      p.kblocks[s] = (p.kreal[s] + p.ksub - 1) / p.ksub;
+      if (!cached_map(cache, &p.tmA[s], g.A[s], esize, tf32, false, g.M, g.N, g.sa_i[s], 1, g.batch, g.batch_a[s], pa.box_rows))
+        return cudaErrorInvalidValue;
+      if (!cached_map(cache, &p.tmB[s], g.B[s], esize, tf32, false, 256, 256, 256, 1, 1, 256 * 256, pb.box_rows))
+        return cudaErrorInvalidValue;
+      continue;
+    }
     p.kreal[s] = (g.K[s] + span - 1) / span;
     p.kblocks[s] = (p.kreal[s] + p.ksub - 1) / p.ksub;
     if (!cached_map(cache, &p.tmA[s], g.A[s], esize, tf32, pa.mn_major, g.M, g.K[s], g.sa_i[s], g.sa_k[s], g.batch,
@@ -1400,6 +1424,8 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
             ((uint32_t)((p.pair ? 256 : 128) >> 4) << 24);
   p.epilogue = g.epilogue; p.out_dtype = g.out_dtype; p.aux_dtype = g.aux_dtype; p.symmetric = g.symmetric; p.round_tf32 = g.round_tf32;
   p.transposed = g.transpose_out ? 1 : 0;
+  p.diag_exact = !(g.nseg == 1 && g.b_split != 2 && g.A[0] == g.B[0] && g.sa_i[0] == g.sb_j[0] && g.sa_k[0] == g.sb_k[0] &&
+                   g.batch_a[0] == g.batch_b[0]) ? 1 : 0;
   p.aux_f16 = (g.epilogue != EPI_STORE && g.aux_dtype == F16) ? 1 : 0;
   p.out_f16 = (g.out_dtype == F16) ? 1 : 0;
   p.C = g.C; p.ldc = g.ldc; p.batch_c = g.batch_c;

@@ -860,14 +860,14 @@ cudaError_t split_panel_launch(const float* In, long long in_bs, int ld_in, int 
 // Out [b, rows, 3*kp] (16-bit) = three column blocks of the (optionally column-scaled) panel In [b, rows, k]:
 //   pattern 0: [hi | hi | lo]      pattern 1: [hi | lo | hi]
 // so that  Out0 * Out1^T = hi hi^T + hi lo^T + lo hi^T  (the product of the two fp32 panels up to the lo*lo term).
-// Column t is scaled by  mult * (c0 * s[b,t] * (inv_rho ? inv_rho[b] : 1) + c1)  (without s: by mult alone).
+// Column t is scaled by  mult * (c0 * s[b,t] * (inv_rho ? inv_rho[b] : 1) + c1 * (rho ? rho[b] : 1))  (without s: by mult alone).
 // The two halves are bf16 or, with `f16`, IEEE half (the type of the product they enter); with `transposed` the
 // copy is stored as [b, 3*kp, rows], the layout of an operand whose long side is contiguous.
 template <bool F16, bool TRANSPOSED>
 __global__ void split_concat3_kernel(const float* __restrict__ In, long long in_bs, int ld_in, int rows, int k, int kp,
                                      const float* __restrict__ s, int ld_s, const float* __restrict__ inv_rho, float c0,
                                      float c1, float mult, int pattern, uint16_t* __restrict__ Out,
-                                     const int* __restrict__ keff) {
+                                     const int* __restrict__ keff, const float* __restrict__ rho) {
   const int bz = blockIdx.y;
   const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= (long long)rows * kp) return;
@@ -876,7 +876,7 @@ __global__ void split_concat3_kernel(const float* __restrict__ In, long long in_
   float x = 0.f;
   if (t < k && !(keff && t >= keff[bz])) {
     x = In[(long long)bz * in_bs + (long long)r * ld_in + t] * mult;
-    if (s) x *= c0 * s[(long long)bz * ld_s + t] * (inv_rho ? inv_rho[bz] : 1.f) + c1;
+    if (s) x *= c0 * s[(long long)bz * ld_s + t] * (inv_rho ? inv_rho[bz] : 1.f) + c1 * (rho ? rho[bz] : 1.f);
   }
   uint16_t h, lw;
   if (F16) {
@@ -899,14 +899,41 @@ __global__ void split_concat3_kernel(const float* __restrict__ In, long long in_
 cudaError_t split_concat3_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int k, int kp,
                                  const float* s, int ld_s, const float* inv_rho, float c0, float c1, int pattern,
                                  __nv_bfloat16* Out, cudaStream_t st, long long* launches, const int* keff, int f16,
-                                 int transposed, float mult) {
+                                 int transposed, float mult, const float* rho) {
   const long long tot = (long long)rows * kp;
   const dim3 grid((unsigned)((tot + 255) / 256), batch);
   uint16_t* o = reinterpret_cast<uint16_t*>(Out);
-  if (f16 && transposed) split_concat3_kernel<true, true><<<grid, 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s, inv_rho, c0, c1, mult, pattern, o, keff);
-  else if (f16) split_concat3_kernel<true, false><<<grid, 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s, inv_rho, c0, c1, mult, pattern, o, keff);
-  else if (transposed) split_concat3_kernel<false, true><<<grid, 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s, inv_rho, c0, c1, mult, pattern, o, keff);
-  else split_concat3_kernel<false, false><<<grid, 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s, inv_rho, c0, c1, mult, pattern, o, keff);
+  if (f16 && transposed) split_concat3_kernel<true, true><<<grid, 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s, inv_rho, c0, c1, mult, pattern, o, keff, rho);
+  else if (f16) split_concat3_kernel<true, false><<<grid, 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s, inv_rho, c0, c1, mult, pattern, o, keff, rho);
+  else if (transposed) split_concat3_kernel<false, true><<<grid, 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s, inv_rho, c0, c1, mult, pattern, o, keff, rho);
+  else split_concat3_kernel<false, false><<<grid, 256, 0, st>>>(In, in_bs, ld_in, rows, k, kp, s, ld_s, inv_rho, c0, c1, mult, pattern, o, keff, rho);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+// Matrices whose residual counts as zero (status bit 4: 1/rho = 0) get the padded head alone as filter input,
+// X0 = scale * P[:, :keff] W[:, :keff]^T; every other matrix is left untouched (its CTAs return at once).
+__global__ void __launch_bounds__(256) zero_residual_entry_kernel(const int* __restrict__ status, const float* __restrict__ P,
+                                                                  const float* __restrict__ W, const int* __restrict__ keff,
+                                                                  int m, int n, int k, float scale, void* __restrict__ X0,
+                                                                  int dtype) {
+  const int bz = blockIdx.y;
+  if (!(status[bz] & 4)) return;
+  const float* Pb = P + (long long)bz * m * k;
+  const float* Wb = W + (long long)bz * n * k;
+  const int ke = keff ? min(keff[bz], k) : k;
+  const long long tot = (long long)m * n;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < tot; e += (long long)gridDim.x * blockDim.x) {
+    const int i = (int)(e / n), j = (int)(e % n);
+    float t = 0.f;
+    for (int q = 0; q < ke; ++q) t = fmaf(Pb[(long long)i * k + q], Wb[(long long)j * k + q], t);
+    st_from_float(X0, (long long)bz * tot + e, dtype, scale * t);
+  }
+}
+
+cudaError_t zero_residual_entry_launch(const int* status, const float* P, const float* W, const int* keff, int batch, int m,
+                                       int n, int k, float scale, void* X0, int dtype, cudaStream_t st, long long* launches) {
+  zero_residual_entry_kernel<<<dim3(64, batch), 256, 0, st>>>(status, P, W, keff, m, n, k, scale, X0, dtype);
   if (launches) ++*launches;
   return cudaGetLastError();
 }

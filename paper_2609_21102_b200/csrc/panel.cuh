@@ -47,7 +47,9 @@ cudaError_t split_panel_launch(const float* In, long long in_bs, int ld_in, int 
 cudaError_t split_concat3_launch(const float* In, long long in_bs, int ld_in, int batch, int rows, int k, int kp,
                                  const float* s, int ld_s, const float* inv_rho, float c0, float c1, int pattern,
                                  __nv_bfloat16* Out, cudaStream_t st, long long* launches, const int* keff = nullptr,
-                                 int f16 = 0, int transposed = 0, float mult = 1.f);
+                                 int f16 = 0, int transposed = 0, float mult = 1.f, const float* rho = nullptr);
+cudaError_t zero_residual_entry_launch(const int* status, const float* P, const float* W, const int* keff, int batch, int m,
+                                       int n, int k, float scale, void* X0, int dtype, cudaStream_t st, long long* launches);
 cudaError_t gate_launch(const float* s, int ld_s, int batch, int window, int kmax, float tau, int* keff, cudaStream_t st,
                         long long* launches);
 }  // namespace defl

@@ -89,8 +89,8 @@ def dense_filter_flops(m, n, L):
 
 # Average DRAM bytes per filter-product launch: dram__bytes_read + dram__bytes_write of the six kinds of filter
 # launch (X X^T, A^2 polynomial, B X for each shape group) from the ncu captures summarised in
-# the filter-kernel summary under profiles/ (8 matrices per group: 132.4 MB on average), scaled by 48/8.
-FILTER_TRAFFIC_BYTES_PER_LAUNCH = 795e6
+# the filter-kernel summary under profiles/ (8 matrices per group: 132.8 MB on average), scaled by 48/8.
+FILTER_TRAFFIC_BYTES_PER_LAUNCH = 797e6
 
 
 def max_over_ranks(value, dist=None, device="cpu"):

@@ -355,7 +355,7 @@ def extra_polar(ctx, name, opts, device, steps=10, label=None, graph=False):
     return out
 
 
-def extra_sdp(ctx, peaks, device, n=4096, calls=20, warm=2):
+def extra_sdp(ctx, peaks, device, n=4096, calls=20, warm=2, tf32_peak=True):
     """The SDP projection sequence at n = 4096 (tf32 filter): ms per projection over the deflated calls, the seven-stage
     split, the filter + reconstruction products against a measured tf32 peak, and the Lanczos passes against HBM."""
     import torch
@@ -379,7 +379,7 @@ def extra_sdp(ctx, peaks, device, n=4096, calls=20, warm=2):
     nd = len(times)
     st = [s / nd for s in ctx.defl_get_stage_ms(nd)]
     names = ["block_step_rayleigh_ritz", "deflate", "lanczos_scale", "initialise", "filter", "reconstruct", "basis_update"]
-    tf32_peak = measure_tf32_peak()
+    tf32_peak = measure_tf32_peak() if tf32_peak else float("nan")
     flops = T * 3.0 * n * n * (n + 1.0) + 2.0 * n ** 3          # symmetric products once, R g(X0) in full
     prod_ms = st[4] + st[5]
     symv_bytes = 42.0 * 4.0 * n * n
@@ -427,6 +427,8 @@ def main():
     ap.add_argument("--add-restore", action="store_true", help="Eq. 3's post-add (fused into the last filter product) instead of the padded entry")
     ap.add_argument("--streams", type=int, default=2, help="2: one stream + context per shape group (the groups are independent); 1: one stream")
     ap.add_argument("--batch", type=int, default=0, help="override the matrices per shape group (profiling captures)")
+    ap.add_argument("--sdp-only", type=int, default=0, metavar="CALLS",
+                    help="run only the SDP projection sequence (n = 4096) with this many calls and print its figures (profiling captures)")
     args = ap.parse_args()
 
     wl_name = "small" if args.small else "gpt2_xl"
@@ -473,6 +475,9 @@ def main():
         dist.init_process_group("nccl", device_id=device)
     ctx = binding.Context(local_rank)
     ctx.defl_set_profiling(True)
+    if args.sdp_only > 0:
+        print(json.dumps(extra_sdp(ctx, load_peaks()[0], device, calls=args.sdp_only, warm=min(2, args.sdp_only - 1), tf32_peak=False)))
+        return
     groups = make_inputs(wl, device)
     ngroups = len(groups)
 

@@ -4,7 +4,7 @@
 One step = one pass of the whole hot path (batched randomized SVD, deflate + normalise, five quintic
 Newton-Schulz steps, restore) over one batch: 48 matrices 1600x6400 and 48 matrices 1600x1600 in
 bf16 with the heavy-tailed spectrum sigma_i = max(200/i, 1e-4), k=32, oversampling 16, 2 subspace
-iterations. Prints ONE JSON line (see README / DESIGN for the keys).
+iterations. Prints ONE JSON line (the keys are described in README.md).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--small] [--no-extras]
 

@@ -1,6 +1,5 @@
-"""Parity of defl_psd_project with the fp64 CPU oracle (Algorithm 2), tolerance 2e-3 relative Frobenius
-on P as the task fixes for the fp32/tf32 path, plus the bulk-only error (P minus its restored head), which
-the head would otherwise hide."""
+"""Parity of defl_psd_project with the fp64 CPU oracle (Algorithm 2), tolerance 2e-3 relative Frobenius on P (the bar of
+the fp32/tf32 path), plus the bulk-only error (P minus its restored head), which the head would otherwise hide."""
 import numpy as np
 import pytest
 import torch

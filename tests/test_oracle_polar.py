@@ -290,7 +290,7 @@ def test_deflated_polar_orientation_and_accuracy(m, n):
 
 
 def test_deflation_lowers_error_on_head_dominated_input_with_estimated_head():
-    # spec check (c) with the rSVD estimate instead of exact triplets, classical map, L = 5
+    # Theorem 1's statement with the randomized-SVD estimate in place of exact triplets, classical map, L = 5
     m, n, k = 32, 48, 3
     M, *_ = _head_dominated(m, n, k)
     coeffs = oracle.schedule(oracle.CLASSICAL_QUINTIC, 5)

@@ -72,6 +72,7 @@ struct TcParams {
   // epilogue
   int epilogue, out_dtype, aux_dtype, symmetric, round_tf32;
   int transposed;              // EPI_STORE: the tile is written transposed, element (i, j) at C[j * ldc + i]
+  int dup_ok;                  // symmetric pair-form product of a matrix with itself, BN = 256: diagonal tiles share one operand fetch
   int diag_exact;              // symmetric output of two different operands: diagonal blocks mirrored element by element
   int aux_f16, out_f16;        // a 16-bit aux / output is IEEE half (else bf16); the operands' kind is in idesc
   void* C; long long ldc, batch_c;
@@ -314,6 +315,7 @@ struct TileInfo {
   int halves;     // bit mask of the 128-row halves this tile computes
   int n_eff;      // columns actually computed (multiple of 16)
   bool skip;
+  bool dup;       // a full tile on the diagonal of a product of a matrix with itself: its B tile IS its A tile
 };
 
 __device__ __forceinline__ TileInfo tile_info(const TcParams& p, long long tile64) {
@@ -345,6 +347,10 @@ __device__ __forceinline__ TileInfo tile_info(const TcParams& p, long long tile6
   int rem = p.N - t.tn * p.BN;
   rem = p.pair ? ((rem + 31) & ~31) : ((rem + 15) & ~15);    // a pair splits the columns in two halves of 16k
   t.n_eff = rem < p.BN ? rem : p.BN;
+  // X X^T / A A on the diagonal: the tile's B operand (this CTA's half of the tile's columns) is the same block of the
+  // same matrix as its A operand (this CTA's 128 rows), in the same shared-memory layout: it is fetched once. Operand
+  // fetch from L2 is what bounds the product, and a diagonal tile then moves half the bytes.
+  t.dup = p.dup_ok && !t.skip && t.tn * p.BN == row0 && t.n_eff == p.BN;
   return t;
 }
 
@@ -960,6 +966,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) { live = false; break; }
             const int nsub = left < ksub ? left : ksub;       // the last step of a segment may be short
+            const bool dup = t.dup;
             // test hook of the bounded waits (single-CTA form): this step of the CTA's first tile is neither announced
             // nor copied, so the consumer's wait for it runs out with nothing in flight
             if (!PAIR && p.hold_stage >= 0 && it == 0 && seg == 0 && kb == p.hold_stage) {
@@ -967,9 +974,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
               continue;
             }
             if (lane == 0 && (!PAIR || rank == 0))
-              mbar_expect_tx(full0 + 8u * stage, nsub == ksub ? tx_bytes : tx_sub_bytes * (uint32_t)nsub);
+              mbar_expect_tx(full0 + 8u * stage, dup ? (PAIR ? 2u : 1u) * p.a_stage_bytes * (uint32_t)nsub
+                                                     : (nsub == ksub ? tx_bytes : tx_sub_bytes * (uint32_t)nsub));
             // (the part of a K block past the end of K is filled with zeros by the copy engine and adds nothing)
-            if (my_on && my_sub < nsub) {
+            if (my_on && my_sub < nsub && (my_a || !dup)) {
               const uint32_t fb = full0_sig + 8u * stage;
               const uint32_t dst = smem_base + stage * stage_bytes + my_dst_off;
               const int c0 = my_mn_major ? my_mn : kc, c1 = my_mn_major ? kc : my_mn;
@@ -1043,7 +1051,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
           const int nsub = left < ksub ? left : ksub;
           for (int sub = 0; sub < nsub; ++sub) {
             const uint32_t sa16 = base16 + stage * stage16 + (uint32_t)sub * sub16;
-            const uint32_t sb16 = sa16 + a_stage16;
+            const uint32_t sb16 = t.dup ? sa16 : sa16 + a_stage16;
 #pragma unroll
             for (int kk = 0; kk < KBYTES / 32; ++kk) {
               const uint64_t adesc = a_hi | (uint64_t)(sa16 + kk * a_kstep16);
@@ -1424,6 +1432,8 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
             ((uint32_t)((p.pair ? 256 : 128) >> 4) << 24);
   p.epilogue = g.epilogue; p.out_dtype = g.out_dtype; p.aux_dtype = g.aux_dtype; p.symmetric = g.symmetric; p.round_tf32 = g.round_tf32;
   p.transposed = g.transpose_out ? 1 : 0;
+  p.dup_ok = (p.pair && g.symmetric && p.BN == 256 && p.tile_m == 256 && g.nseg == 1 && p.b_split != 2 && g.A[0] == g.B[0] &&
+              g.sa_i[0] == g.sb_j[0] && g.sa_k[0] == g.sb_k[0] && g.batch_a[0] == g.batch_b[0]) ? 1 : 0;
   p.diag_exact = !(g.nseg == 1 && g.b_split != 2 && g.A[0] == g.B[0] && g.sa_i[0] == g.sb_j[0] && g.sa_k[0] == g.sb_k[0] &&
                    g.batch_a[0] == g.batch_b[0]) ? 1 : 0;
   p.aux_f16 = (g.epilogue != EPI_STORE && g.aux_dtype == F16) ? 1 : 0;

@@ -489,7 +489,7 @@ def main():
     lanes = None
     if args.streams > 1:
         lanes = [(binding.Context(local_rank), torch.cuda.Stream()) for _ in groups]
-    config["streams"] = len(lanes) if lanes else 1
+    n_streams = len(lanes) if lanes else 1
 
     def launch_total():
         return ctx.defl_launch_count() + (sum(c.defl_launch_count() for c, _ in lanes) if lanes else 0)
@@ -644,7 +644,8 @@ def main():
             "deflation_overhead_frac": (ms_per_step - plain_ms) / ms_per_step if plain_ms else None,
             "front_end_frac_of_step": front_ms / sum(stage_ms) if sum(stage_ms) > 0 else None,
             "plain_filter_ms": plain_ms,
-            "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "sustained": sustained}
+            "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "streams": n_streams, "clocks": clocks,
+            "sustained": sustained}
 
     if not args.no_extras and wl_name == "gpt2_xl" and args.batch == 0:
         extras = {}

@@ -206,7 +206,6 @@ int run_brsvd(defl_ctx* c, const void* G, int b, int m, int n, int dtype, int l,
       __nv_bfloat16* lo = transposed ? w.Llo : w.Slo;
       GemmDesc t = g;
       t.B[0] = hi; t.B[1] = lo; t.b_split = 2; t.b_dtype = BF16;
-      t.stream_a_ahead = c->knobs.stream_ahead;
       t.sb_k[0] = lp; t.sb_j[0] = 1; t.batch_b[0] = (long long)K * lp;
       if (gemm_tc_supported(t)) {
         if (!presplit &&
@@ -293,7 +292,6 @@ int defl_create(defl_ctx** out, int device) {
   c->knobs.transposed_apply = getenv("DEFL_NO_TRANSPOSED_APPLY") ? 0 : 1;
   c->knobs.host_chunks = getenv("DEFL_HOST_CHUNKS") ? atoi(getenv("DEFL_HOST_CHUNKS")) : 0;
   c->knobs.jacobi_sweeps = getenv("DEFL_JACOBI_SWEEPS") ? atoi(getenv("DEFL_JACOBI_SWEEPS")) : 0;
-  c->knobs.stream_ahead = getenv("DEFL_STREAM_AHEAD") ? atoi(getenv("DEFL_STREAM_AHEAD")) : 0;
   cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device);
   int ok = 1;
   if (cudaMalloc(&c->wait_status, 2 * sizeof(int)) != cudaSuccess) ok = 0;      // status word, tile counter

@@ -47,8 +47,6 @@ struct GemmDesc {
   int seg1_identity;            // tensor engine, nseg = 2: segment 1 adds A[1][i, j] itself to the accumulator, as the product of
                                 // A[1] (viewed [M, N], K = the output's column index, K-major) with an identity tile: B[1] points
                                 // to a 256 x 256 identity of the operand type (row-major), K[1] is ignored
-  int stream_a_ahead;           // tensor engine: A is read once, from HBM (no reuse between tiles): ask L2 for its boxes this many
-                                // pipeline steps ahead of their copy (0: off)
   int debug_hold_stage;         // test hook, tensor engine, single-CTA form: s > 0 withholds pipeline step s - 1 of each CTA's first tile
 };
 

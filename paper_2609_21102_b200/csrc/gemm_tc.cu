@@ -47,7 +47,6 @@ struct TcParams {
   CUtensorMap tmB[2];
   CUtensorMap tmAux;           // [batch, M, N] view of `aux`, used only to prefetch the epilogue's tile into L2
   int aux_prefetch;
-  int op_prefetch;             // pipeline steps by which the producer asks L2 for the A boxes ahead of their copy (0: off)
   int nseg;
   int seg1_ident;              // segment 1 = A[1] tile (K offset by the tile's first column) x identity tile (same for every tile and matrix)
   int b_split;                 // 2: B is the sum of two operands (tmB[0] + tmB[1]) that share A; else 1
@@ -895,34 +894,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
       // per pair that tells it to stop; whoever draws the last one puts the counter back to zero
       const long long last_ticket = (total_tiles > npairs ? total_tiles - npairs : 0) + npairs - 1;
       unsigned int ticket = 0;
-      // Look-ahead for a streamed A operand (the products of the randomized SVD read every tile of G exactly once, from
-      // HBM): a cursor runs op_prefetch pipeline steps ahead of the copies, across tile boundaries, and asks L2 for the
-      // A boxes it passes, so that the copy itself finds them there instead of paying the HBM latency inside a
-      // pipeline of three or four stages. (Not for operands that are shared between CTAs and already come from L2:
-      // there the extra requests cost more than they save, measured.)
-      const int opf = (!dynamic && nseg == 1) ? p.op_prefetch : 0;
-      int c_it = 0, c_kb = 0;
-      bool c_valid = opf > 0;
-      TileInfo c_t;
-      auto cursor_seek = [&]() {        // first tile at or after iteration c_it that has work
-        for (;; ++c_it) {
-          const long long tl = tile0 + (long long)c_it * tile_step;
-          if (tl >= total_tiles) { c_valid = false; return; }
-          c_t = tile_info(p, tl);
-          if (!c_t.skip) return;
-        }
-      };
-      auto cursor_step = [&]() {        // prefetch the cursor's step, then advance it
-        if (!c_valid) return;
-        const int nsub = min(ksub, kreal0 - c_kb * ksub);
-        if (my_on && my_a && my_sub < nsub) {
-          const int mn = c_t.tm * tile_m + arow + my_mn_off;
-          const int kc = my_k_off + c_kb * ksub * kstep;
-          tma_prefetch_3d(my_tm0, my_mn_major ? mn : kc, my_mn_major ? kc : mn, c_t.bz);
-        }
-        if (++c_kb >= kblocks0) { c_kb = 0; ++c_it; cursor_seek(); }
-      };
-      if (c_valid) { cursor_seek(); for (int d = 0; d < opf; ++d) cursor_step(); }
       for (int it = 0;; ++it) {
         long long tile;
         if (!dynamic) {
@@ -1013,7 +984,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_tc_kernel(const __grid_co
               if (PAIR) tma_load_3d_pair(dst, tm, fb, c0, c1, bz);
               else tma_load_3d(dst, tm, fb, c0, c1, bz);
             }
-            if (opf > 0) cursor_step();
             __syncwarp();
             if (++stage == nstages) { stage = 0; phase ^= 1u; }
           }
@@ -1474,7 +1444,6 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, cudaStream_t st, int* status_word,
   p.alpha_dev = g.alpha_dev; p.aux_scale_dev = g.aux_scale_dev;
   p.partials = g.partials; p.partials_per_batch = g.partials_per_batch;
   p.aux_prefetch = 0;
-  p.op_prefetch = (g.stream_a_ahead > 0 && g.nseg == 1) ? g.stream_a_ahead : 0;
   // (Off unless the aux_prefetch knob is set: with the epilogue's own fetch one block ahead the extra L2 prefetch
   // made the deflation passes 6 % slower and raised their DRAM reads to 1.6x the matrix, measured.)
   if (g.aux && g.epilogue != EPI_STORE && aligned16(g.aux) && kn.aux_prefetch) {

@@ -32,10 +32,29 @@ __global__ void __launch_bounds__(256) symv_kernel(const float* __restrict__ A, 
     if (vec) {
       const float4* r4 = reinterpret_cast<const float4*>(row);
       const float4* x4 = reinterpret_cast<const float4*>(x);
-      // four independent partial sums and loads in flight per lane; combined in a fixed order
+      // four independent partial sums per lane, combined in a fixed order; eight 16-byte loads of the row in flight per
+      // lane where the row is long enough (a warp walks its row in dependent trips, each one a trip to L2 or HBM: the
+      // trip count, not the bandwidth, is what a matrix-vector product of this size takes)
       float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
       const int n4 = n / 4;
       int i = lane;
+      for (; i + 224 < n4; i += 256) {
+        float4 pr[8], qr[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) pr[u] = r4[i + 32 * u];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) qr[u] = __ldg(&x4[i + 32 * u]);
+        // (the same order of additions as two trips of the four-load loop below)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float4 p0 = pr[4 * h], p1 = pr[4 * h + 1], p2 = pr[4 * h + 2], p3 = pr[4 * h + 3];
+          const float4 q0 = qr[4 * h], q1 = qr[4 * h + 1], q2 = qr[4 * h + 2], q3 = qr[4 * h + 3];
+          a0 = fmaf(p0.x, q0.x, a0); a0 = fmaf(p0.y, q0.y, a0); a0 = fmaf(p0.z, q0.z, a0); a0 = fmaf(p0.w, q0.w, a0);
+          a1 = fmaf(p1.x, q1.x, a1); a1 = fmaf(p1.y, q1.y, a1); a1 = fmaf(p1.z, q1.z, a1); a1 = fmaf(p1.w, q1.w, a1);
+          a2 = fmaf(p2.x, q2.x, a2); a2 = fmaf(p2.y, q2.y, a2); a2 = fmaf(p2.z, q2.z, a2); a2 = fmaf(p2.w, q2.w, a2);
+          a3 = fmaf(p3.x, q3.x, a3); a3 = fmaf(p3.y, q3.y, a3); a3 = fmaf(p3.z, q3.z, a3); a3 = fmaf(p3.w, q3.w, a3);
+        }
+      }
       for (; i + 96 < n4; i += 128) {
         const float4 p0 = r4[i], p1 = r4[i + 32], p2 = r4[i + 64], p3 = r4[i + 96];
         const float4 q0 = __ldg(&x4[i]), q1 = __ldg(&x4[i + 32]), q2 = __ldg(&x4[i + 64]), q3 = __ldg(&x4[i + 96]);
@@ -223,13 +242,114 @@ __global__ void __launch_bounds__(1024) lanczos_step_reg_kernel(int j, int n, in
   for (int e = 0; e < EPT; ++e) { const int i = tid + e * 1024; if (i < n) qn[i] = wv[e] * inv_b; }
 }
 
-// v = sum_p E[p][0] q_p (the Ritz vector of the largest Ritz value); E is [steps, steps] row-major fp32
+// ---------------------------------------------------------------------------------------------
+// Largest eigenpair of the Lanczos matrix (symmetric tridiagonal, dense fp64 storage [steps, steps], rows after a
+// breakdown all zero), by one warp: the eigenvalue by multi-section on the Sturm count (32 shifts per round, one
+// per lane), the eigenvector by inverse iteration (elimination with row exchanges, pivots floored at eps ||T||).
+// Only the leading unreduced block takes part: the Krylov space ends where an off-diagonal entry is zero, and the
+// entries of the vector beyond it are exact zeros. Outputs rho[0] and column 0 of E (fp32, [steps, steps] row-major).
+// A general symmetric eigensolver on this 20 x 20 matrix cost a fifth of the whole scale estimate.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(32) tridiag_top_kernel(const double* __restrict__ T, int steps, float* __restrict__ rho,
+                                                         float* __restrict__ E) {
+  constexpr int MS = DEFL_LANCZOS_STEPS;
+  __shared__ double al[MS], be[MS], y[MS];
+  const int lane = threadIdx.x;
+  if (lane < steps) {
+    al[lane] = T[lane * steps + lane];
+    be[lane] = (lane + 1 < steps) ? T[lane * steps + lane + 1] : 0.0;
+    E[lane * steps] = 0.f;
+  }
+  __syncwarp();
+  int m = 1;
+  while (m < steps && be[m - 1] != 0.0) ++m;                 // size of the leading unreduced block
+  // Gershgorin interval and the scale of the matrix
+  double lo = al[0], hi = al[0], tn = 0.0;
+  for (int i = 0; i < m; ++i) {
+    const double r = (i > 0 ? fabs(be[i - 1]) : 0.0) + (i + 1 < m ? fabs(be[i]) : 0.0);
+    lo = fmin(lo, al[i] - r); hi = fmax(hi, al[i] + r);
+    tn = fmax(tn, fabs(al[i]) + r);
+  }
+  const double eps = 2.220446049250313e-16;
+  const double pivmin = fmax(tn * eps * eps, 1e-300);
+  double a = lo - eps * tn - pivmin, b = hi + eps * tn + pivmin;       // count(a) < m = count(b)
+  for (int round = 0; round < 16; ++round) {
+    const double x = a + (b - a) * ((double)(lane + 1) / 33.0);
+    // number of eigenvalues of the block below x: negative terms of the Sturm recurrence
+    int cnt = 0;
+    double q = 1.0;
+    for (int i = 0; i < m; ++i) {
+      q = al[i] - x - (i > 0 ? be[i - 1] * be[i - 1] / q : 0.0);
+      if (fabs(q) < pivmin) q = -pivmin;
+      cnt += q < 0.0;
+    }
+    const unsigned full = __ballot_sync(0xffffffffu, cnt >= m);         // shifts above every eigenvalue
+    const int first = full ? __ffs(full) - 1 : 32;
+    const double nb = (first < 32) ? __shfl_sync(0xffffffffu, x, first) : b;
+    const double na = (first > 0) ? __shfl_sync(0xffffffffu, x, first - 1) : a;
+    a = na; b = nb;
+    if (b - a <= 2.0 * eps * fmax(fabs(a), fabs(b)) + 2.0 * pivmin) break;
+  }
+  const double lam = 0.5 * (a + b);
+  if (lane == 0) {
+    rho[0] = (float)lam;
+    if (m == 1) y[0] = 1.0;
+    else {
+      // inverse iteration from the vector of ones (the off-diagonal entries of a Lanczos matrix are positive, so the
+      // wanted vector has entries of one sign and is not orthogonal to it)
+      double d[MS], du[MS], du2[MS], dl[MS], z[MS];
+      const double floor_p = eps * tn;
+      for (int i = 0; i < m; ++i) z[i] = 1.0;
+      for (int iter = 0; iter < 3; ++iter) {
+        for (int i = 0; i < m; ++i) { d[i] = al[i] - lam; du[i] = (i + 1 < m) ? be[i] : 0.0; dl[i] = du[i]; du2[i] = 0.0; }
+        for (int i = 0; i + 1 < m; ++i) {
+          if (fabs(d[i]) >= fabs(dl[i])) {
+            if (fabs(d[i]) < floor_p) d[i] = (d[i] < 0.0) ? -floor_p : floor_p;
+            const double f = dl[i] / d[i];
+            d[i + 1] -= f * du[i];
+            z[i + 1] -= f * z[i];
+          } else {
+            // rows i and i + 1 change places
+            const double f = d[i] / dl[i];
+            d[i] = dl[i];
+            const double t = d[i + 1];
+            d[i + 1] = du[i] - f * t;
+            du[i] = t;
+            if (i + 2 < m) { du2[i] = du[i + 1]; du[i + 1] = -f * du2[i]; }
+            const double zt = z[i];
+            z[i] = z[i + 1];
+            z[i + 1] = zt - f * z[i + 1];
+          }
+        }
+        if (fabs(d[m - 1]) < floor_p) d[m - 1] = (d[m - 1] < 0.0) ? -floor_p : floor_p;
+        z[m - 1] /= d[m - 1];
+        z[m - 2] = (z[m - 2] - du[m - 2] * z[m - 1]) / d[m - 2];
+        for (int i = m - 3; i >= 0; --i) z[i] = (z[i] - du[i] * z[i + 1] - du2[i] * z[i + 2]) / d[i];
+        double big = 0.0;
+        for (int i = 0; i < m; ++i) big = fmax(big, fabs(z[i]));
+        double nn = 0.0;
+        for (int i = 0; i < m; ++i) { z[i] = (big > 0.0) ? z[i] / big : ((i == 0) ? 1.0 : 0.0); nn += z[i] * z[i]; }
+        const double inv = rsqrt(nn);
+        for (int i = 0; i < m; ++i) z[i] *= inv;
+      }
+      for (int i = 0; i < m; ++i) y[i] = z[i];
+    }
+  }
+  __syncwarp();
+  if (lane < m) E[lane * steps] = (float)y[lane];
+}
+
+// v = sum_p E[p][0] q_p (the Ritz vector of the largest Ritz value); E is [steps, steps] row-major fp32; rows of Q that
+// carry a zero coefficient (those after a breakdown, never written) are not read
 __global__ void lanczos_ritz_kernel(int n, int steps, const float* __restrict__ Q, const float* __restrict__ E,
                                     float* __restrict__ v) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   double a = 0.0;
-  for (int p = 0; p < steps; ++p) a += (double)E[p * steps] * (double)Q[(long long)p * n + i];
+  for (int p = 0; p < steps; ++p) {
+    const float e = E[p * steps];
+    if (e != 0.f) a += (double)e * (double)Q[(long long)p * n + i];
+  }
   v[i] = (float)a;
 }
 
@@ -377,9 +497,10 @@ static int estimate_scale(defl_ctx* c, const float* A, int n, int norm_mode, con
     ++c->launches;
     if (ctx_fail(c, cudaGetLastError(), "lanczos step")) return DEFL_ERR_CUDA;
   }
-  // largest Ritz pair of the (zero-padded) tridiagonal matrix through the Jacobi core
-  if (ctx_fail(c, jacobi_eig_launch(w.T, 1, 1, steps, 1, w.lrho, w.lE, nullptr, w.status, c->stream, &c->launches), "ritz"))
-    return DEFL_ERR_CUDA;
+  // largest Ritz pair of the (zero-padded) tridiagonal matrix
+  tridiag_top_kernel<<<1, 32, 0, c->stream>>>(w.T, steps, w.lrho, w.lE);
+  ++c->launches;
+  if (ctx_fail(c, cudaGetLastError(), "ritz")) return DEFL_ERR_CUDA;
   lanczos_ritz_kernel<<<(n + 255) / 256, 256, 0, c->stream>>>(n, steps, w.Q, w.lE, w.lv);
   ++c->launches;
   if (ctx_fail(c, cudaGetLastError(), "ritz vector")) return DEFL_ERR_CUDA;

@@ -125,6 +125,30 @@ def test_psd_generated_start_vector_is_the_documented_generator(ctx):
     assert abs(float(info["theta"][0]) - th) <= 1e-3 * th
 
 
+def test_lanczos_breakdown_ends_the_krylov_space(ctx):
+    """A start vector that is an eigenvector of R (exactly, in fp32): the recurrence breaks down after its first step,
+    the Lanczos matrix is 1 x 1 (the rest zero padding, the later basis vectors never written) and the scale is the
+    magnitude of that eigenvalue; a start vector inside a three-dimensional invariant subspace ends it after three."""
+    n = 160
+    d = np.concatenate([[2.0, -1.5, 1.25], 0.9 * (2.0 * inputs.rand((n - 3,), 88).double().numpy() - 1.0)])
+    X = torch.diag(torch.tensor(d, dtype=torch.float32)).cuda()
+    Xo = X.double().cpu().numpy()
+    for support, want in (([0], 2.0), ([0, 1, 2], None)):
+        v = np.zeros(n)
+        v[support] = [1.0, 0.5, -0.25][:len(support)]
+        v0 = torch.tensor(v, dtype=torch.float32).cuda()
+        P, info = ctx.defl_psd_project(X, 0, None, SCHED7, lanczos_start=v0, want_info=True)
+        th = oracle.lanczos_upper(Xo, v)
+        Po, *_ = oracle.psd_project(Xo, None, 0, oracle.schedule(SCHED7), lanczos_v0=v)
+        assert int(info["status"][0]) == 0
+        assert abs(float(info["theta"][0]) - th) <= (1e-5 if want is not None else 1e-3) * th
+        if want is not None:
+            assert abs(th - want) <= 1e-12
+        else:
+            assert 2.0 * (1 - 1e-6) <= th <= 2.0 * (1 + 1e-3)        # the three Ritz values are the three eigenvalues
+        assert _rel(P.double().cpu().numpy(), Po) <= TOL_TF32_UNDEFLATED
+
+
 def test_psd_drifting_sequence_tracks_the_head(ctx):
     """A short synthetic stand-in for consecutive solver iterates: X_{t+1} = X_t + 1e-3 sym(N)."""
     n, K, k = 320, 16, 8

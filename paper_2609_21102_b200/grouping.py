@@ -37,11 +37,27 @@ def stack_group(tensors, indices):
     return buf, views
 
 
-def muon_step_groups(ctx, weights, momenta, grads, lr, mu, window, oversample, power_iters, coeff_schedule, **kw):
+def deflation_active(step, total_steps, cutoff=1.0):
+    """The deflation cutoff of Section 4 ("Deflation cutoff"): deflation runs during the first `cutoff` fraction of
+    the `total_steps` optimizer steps (step counted from 0) and the plain filter after it; cutoff = 1 keeps it on
+    throughout, cutoff = 0 is plain Muon."""
+    if not 0.0 <= cutoff <= 1.0:
+        raise ValueError("cutoff is a fraction of the optimizer steps")
+    if step < 0 or total_steps <= 0:
+        raise ValueError("step >= 0 and total_steps > 0")
+    return step < cutoff * total_steps
+
+
+def muon_step_groups(ctx, weights, momenta, grads, lr, mu, window, oversample, power_iters, coeff_schedule,
+                     step=None, total_steps=None, cutoff=1.0, **kw):
     """One Deflated Muon step over stacked groups: weights/momenta/grads are dicts {(m, n): [b, m, n] tensor} (grads
     may hold None). `window` is the number k of leading triplets, or a ratio w in (0, 1) meaning k = ceil(w min(m, n));
-    `oversample` likewise a count or a ratio delta (Section 3: r = ceil(w m), r' = r + ceil(delta m))."""
+    `oversample` likewise a count or a ratio delta (Section 3: r = ceil(w m), r' = r + ceil(delta m)). With `step` and
+    `total_steps` the deflation cutoff applies: past it the step runs with k = 0, which is the plain Muon step (no
+    range finder, no deflation pass, the same filter)."""
     import math
+    if step is not None and total_steps is not None and not deflation_active(step, total_steps, cutoff):
+        window = 0
     for shape, W in weights.items():
         ms = min(shape)
         k = int(math.ceil(window * ms)) if 0 < window < 1 else int(window)

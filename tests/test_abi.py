@@ -70,6 +70,31 @@ def test_shape_groups_and_stacking():
         grouping.stack_group(ts, [0, 1])
 
 
+def test_deflation_cutoff_switch():
+    """Section 4, "Deflation cutoff": deflation during the first fraction of the optimizer steps, the plain step after;
+    the step helper passes k = 0 past the cutoff (a recording stand-in for the context, no GPU)."""
+    from paper_2609_21102_b200 import grouping
+    assert [grouping.deflation_active(t, 10, 0.3) for t in range(10)] == [True] * 3 + [False] * 7
+    assert all(grouping.deflation_active(t, 10, 1.0) for t in range(10))
+    assert not any(grouping.deflation_active(t, 10, 0.0) for t in range(10))
+    assert [grouping.deflation_active(t, 5, 0.5) for t in range(5)] == [True, True, True, False, False]   # 2.5 steps
+    with pytest.raises(ValueError):
+        grouping.deflation_active(0, 10, 1.5)
+
+    class Recorder:
+        def __init__(self):
+            self.calls = []
+
+        def defl_muon_step_batched(self, W, M, G, lr, mu, k, p, J, sched, **kw):
+            self.calls.append((k, p, J))
+    rec = Recorder()
+    weights = {(1600, 6400): "W"}
+    for t in range(4):
+        grouping.muon_step_groups(rec, weights, {(1600, 6400): "M"}, {}, 0.02, 0.95, 0.02, 0.01, 2, [[1.0, 0.0, 0.0]],
+                                  step=t, total_steps=4, cutoff=0.5)
+    assert rec.calls == [(32, 16, 2), (32, 16, 2), (0, 16, 2), (0, 16, 2)]
+
+
 def test_window_ratios_follow_the_algorithms(libpath):
     """Algorithm 3 line 1 (r = ceil(w m), r' = min{m, r + ceil(delta m)}) and Algorithm 2's inputs (r = ceil(w n),
     K = ceil(w' n)), worked by hand."""

@@ -121,6 +121,25 @@ def test_bf16_weights(ctx):
     assert float((W16.float() - want.float()).abs().max()) <= float(W16.float().abs().max()) * 2.0 ** -7
 
 
+def test_past_the_deflation_cutoff_the_step_is_plain_muon(ctx):
+    """Section 4, "Deflation cutoff": the step helper passes k = 0 after the cutoff; that step must be the oracle's
+    Muon step without deflation (same filter, no range finder), before the cutoff the deflated one."""
+    from paper_2609_21102_b200 import binding, grouping
+    b, m, n, k = 3, 96, 160, 4
+    W, Mom, Grad, Om = _case(b, m, n, k, torch.float32, 15)
+    sched = [list(binding.MUON_QUINTIC)] * 5
+    keep = (1.0 - LR * WD) * W.double().numpy()
+    for step, k_want in ((0, k), (1, 0)):
+        want_w, want_m = _oracle(W, Mom, Grad, Om, k_want, False, 0, "f32")
+        Wd, Md = W.cuda(), Mom.cuda()
+        # window as a count, oversampling as a count (so that the sketch has the width the oracle was given)
+        grouping.muon_step_groups(ctx, {(m, n): Wd}, {(m, n): Md}, {(m, n): Grad.cuda()}, LR, MU, k, k, 1, sched,
+                                  step=step, total_steps=2, cutoff=0.5, weight_decay=WD, scale=SCALE,
+                                  sketch=Om.cuda() if k_want else None, gamma=1.01)
+        assert _rel(Wd.cpu().double().numpy() - keep, want_w - keep) <= 2e-3, step
+        assert np.allclose(Md.cpu().double().numpy(), want_m, rtol=1e-6, atol=1e-7)
+
+
 def test_argument_errors(ctx):
     from paper_2609_21102_b200 import binding
     W = torch.zeros((1, 64, 64), device="cuda")

@@ -5,6 +5,7 @@
  * residual, run the filter, restore the components (Eq. 3). Two primitives are exported:
  *   defl_polar_batched  -- Algorithm 3 (batched randomized SVD) + Algorithm 1 (deflated polar factor)
  *   defl_psd_project    -- Algorithm 2 (deflated PSD projection with a warm-started basis)
+ *   defl_inv_root       -- the same deflation around a fixed-depth inverse matrix root (Conclusion)
  * plus the batched randomized SVD on its own, a counter-based Gaussian fill and diagnostics.
  *
  * Conventions
@@ -207,6 +208,36 @@ int defl_psd_project(defl_ctx* ctx, const void* X, void* P, int n, int k,
                      float* warm_basis, int K,
                      const float* coeff_schedule, int T,
                      const defl_opts* opts, const defl_info* info);
+
+/* Deflated inverse matrix root  out ~ A^(-1/p)  of one symmetric positive definite matrix (Conclusion: inverse
+ * matrix roots, the preconditioners of Shampoo-type optimizers, are named as the next instance of the framework; the
+ * paper gives no algorithm for it, so each step below is the one it defines for its own instances):
+ *   1. block step A V, Rayleigh-Ritz on the tracked basis, the k leading eigenpairs (lambda_i, u_i) removed:
+ *      R = A - sum lambda_i u_i u_i^T                                        (Algorithm 2, lines 1-5)
+ *   2. theta = Lanczos upper estimate of ||R||_2 (Appendix E.1, "Normalization scale");
+ *      X0 = R / theta + (1/gamma) sum u_i u_i^T                              (Algorithm 2, line 7; Algorithm 1, line 4)
+ *   3. `steps` steps of the coupled Newton iteration, matrix products only:
+ *      T_t = ((p+1) I - M_t) / p,  Z_{t+1} = Z_t T_t,  M_{t+1} = T_t^p M_t,  M_0 = X0, Z_0 = I
+ *   4. out = theta^(-1/p) (Z - z_pad sum u_i u_i^T) + sum lambda_i^(-1/p) u_i u_i^T, symmetrised, where z_pad is the
+ *      value the scalar iteration gives the padding 1/gamma: the head is restored exactly (Eq. 3 in padded form)
+ *   5. warm_basis <- orthonormalised A V                                     (Algorithm 2, line 9)
+ *   A  [n,n] fp32 symmetric positive definite, not modified.  out [n,n] fp32, exactly symmetric on return, must not
+ *   overlap A.  warm_basis [n,K] fp32 with orthonormal columns, IN/OUT (K = 0: no deflation).  p in {1, 2, 4}.
+ *   k <= K eigenpairs to remove; k = 0 or opts->warmup: the plain normalised iteration.  steps <= DEFL_MAX_STEPS.
+ * The basis must have settled before eigenpairs are removed (run the first calls with opts->warmup, as the paper does
+ * for the projection): a Ritz pair (lambda, u) with residual r = A u - lambda u leaves R indefinite, with an eigenvalue
+ * near -|r|^2 / a, a = r^T A r / |r|^2; the padding keeps X0 positive definite while |r|^2 < a theta / gamma, and on an
+ * eigenvalue that is not positive the iteration diverges. A result that is not finite sets DEFL_ST_NONFINITE.
+ * Products on the tensor cores in tf32 (iterates stored rounded to tf32) unless opts->engine = DEFL_ENGINE_SIMT
+ * (exact fp32 products). Read from opts: gamma (default 1.1), engine, warmup, tau (gate on the Ritz values, as in
+ * defl_psd_project), norm_mode, lanczos_start, seed, exploit_symmetry. info: s = the K Ritz values by decreasing
+ * magnitude, rho = theta, k_used, status (a removed Ritz value that is not positive sets DEFL_ST_NONFINITE and leaves
+ * that direction at the iteration's value: the matrix is not positive definite there).
+ * Errors: DEFL_ERR_ARG (null pointers, overlap, p not in {1,2,4}, steps < 0), DEFL_ERR_RANK (k > K, K > DEFL_MAX_L,
+ * K >= n, steps > DEFL_MAX_STEPS), DEFL_ERR_CUDA. */
+int defl_inv_root(defl_ctx* ctx, const void* A, void* out, int n, int p, int k,
+                  float* warm_basis, int K, int steps,
+                  const defl_opts* opts, const defl_info* info);
 
 /* Three-block ADMM for a standard-form SDP whose constraints are diag(X) = b (max-cut type):
  *   min <C, X>  s.t.  diag(X) = b, X PSD;   A(X) = diag(X), A*(y) = Diag(y), A A* = I.

@@ -17,6 +17,11 @@ instances:
   * the target is restored exactly on the removed directions (Algorithm 1, line 6 in its padded form; Eq. 3):
     out = theta^(-1/p) (Z_T - z_T(1/gamma) U U^T) + U diag(lambda_i^(-1/p)) U^T,  symmetrised.
 
+The removed pairs must be accurate: a Ritz pair (lambda, u) with residual r leaves R = A - lambda u u^T indefinite (an
+eigenvalue near -|r|^2 / a, a = r^T A r / |r|^2); the padding keeps X0 positive definite while |r|^2 < a theta / gamma, and
+the iteration diverges on an eigenvalue that is not positive. Hence warm-up calls (basis advanced, nothing removed)
+until the basis has settled, the protocol the paper uses for its projection.
+
 Plain numpy on top of the oracle's own primitives (its matrix product, Jacobi eigensolver, Householder
 orthonormalisation and Lanczos estimate); no blocking, no fusion.
 """

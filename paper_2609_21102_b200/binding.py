@@ -25,7 +25,7 @@ CLASSICAL_QUINTIC = (1.875, -1.25, 0.375)
 
 EXPORTS = [
     "defl_create", "defl_destroy", "defl_set_stream", "defl_polar_workspace_bytes", "defl_psd_workspace_bytes",
-    "defl_polar_window", "defl_psd_window", "defl_polar_batched", "defl_polar_batched_host", "defl_muon_step_batched", "defl_brsvd_batched", "defl_psd_project", "defl_admm_diag_sdp", "defl_fill_gaussian", "defl_debug_gemm",
+    "defl_polar_window", "defl_psd_window", "defl_polar_batched", "defl_polar_batched_host", "defl_muon_step_batched", "defl_brsvd_batched", "defl_psd_project", "defl_inv_root", "defl_admm_diag_sdp", "defl_fill_gaussian", "defl_debug_gemm",
     "defl_frobenius_norms_noalloc", "defl_set_profiling", "defl_get_stage_ms", "defl_get_stage_ms_sum", "defl_launch_count", "defl_device_wait_status",
     "defl_status_string", "defl_last_error",
 ]
@@ -75,6 +75,9 @@ def lib():
         L.defl_psd_project.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
                                        ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_float), ctypes.c_int,
                                        ctypes.POINTER(DeflOpts), ctypes.POINTER(DeflInfo)]
+        L.defl_inv_root.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                    ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.POINTER(DeflOpts),
+                                    ctypes.POINTER(DeflInfo)]
         L.defl_admm_diag_sdp.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_float,
                                          ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                          ctypes.c_int, ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_float),
@@ -329,6 +332,37 @@ class Context:
         self._sync_stream()
         rc = lib().defl_psd_project(self._h, _ptr(X), _ptr(out), n, k, _ptr(warm_basis), K, sched, T,
                                     ctypes.byref(opts), ctypes.byref(info))
+        self._check(rc)
+        return (out, extras) if want_info else out
+
+    def defl_inv_root(self, A, p, k, warm_basis, steps, out=None, gamma=0.0, norm_mode=NORM_LANCZOS, lanczos_start=None,
+                      seed=0, warmup=False, engine=ENGINE_AUTO, exploit_symmetry=False, want_info=False, tau=0.0):
+        """out ~ A^(-1/p) for the symmetric positive definite A[n,n]: deflation of the k leading eigenpairs tracked by
+        warm_basis[n,K] (updated in place) around `steps` coupled Newton steps (Conclusion's next instance)."""
+        _dev(A, "A")
+        n = A.shape[0]
+        if A.dtype != torch.float32 or A.shape != (n, n):
+            raise ValueError("A must be a square float32 matrix")
+        K = 0
+        if warm_basis is not None:
+            _dev(warm_basis, "warm_basis")
+            K = warm_basis.shape[1]
+        out = torch.empty_like(A) if out is None else _dev(out, "out")
+        opts = self._opts(gamma=gamma, norm_mode=norm_mode, lanczos_start=lanczos_start, seed=seed, warmup=warmup,
+                          engine=engine, exploit_symmetry=exploit_symmetry, tau=tau)
+        info = DeflInfo()
+        extras = None
+        if want_info:
+            lam = torch.zeros((max(K, 1),), dtype=torch.float32, device=A.device)
+            theta = torch.zeros((1,), dtype=torch.float32, device=A.device)
+            status = torch.zeros((1,), dtype=torch.int32, device=A.device)
+            k_used = torch.zeros((1,), dtype=torch.int32, device=A.device)
+            info.s, info.rho, info.status = lam.data_ptr(), theta.data_ptr(), status.data_ptr()
+            info.k_used = k_used.data_ptr()
+            extras = {"lam": lam[:K], "theta": theta, "status": status, "k_used": k_used}
+        self._sync_stream()
+        rc = lib().defl_inv_root(self._h, _ptr(A), _ptr(out), n, int(p), int(k), _ptr(warm_basis), K, int(steps),
+                                 ctypes.byref(opts), ctypes.byref(info))
         self._check(rc)
         return (out, extras) if want_info else out
 

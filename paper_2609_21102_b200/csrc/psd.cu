@@ -405,9 +405,12 @@ __global__ void split_tf32_kernel(const float* __restrict__ X, float* __restrict
   }
 }
 
-// out[t] = f(lam[t]) per column scale helpers: mode 0: lambda, 1: sign(lambda)/gamma, 2: max(lambda, 0); negated if neg
+// out[t] = f(lam[t]) per column scale helpers: mode 0: lambda, 1: sign(lambda)/gamma, 2: max(lambda, 0), 4: 1/gamma,
+// 3: lambda^(-1/p) - root_scale z_pad (the head of an inverse root minus what the iteration left on the padded
+// direction; a value that is not positive gives 0 and the non-finite status bit); negated if neg
 __global__ void ritz_scale_kernel(const float* __restrict__ lam, int k, int mode, float gamma, int neg, float* __restrict__ out,
-                                  const int* __restrict__ keff) {
+                                  const int* __restrict__ keff, const float* __restrict__ root_scale, float z_pad, int p,
+                                  int* __restrict__ status) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= k) return;
   if (t >= keff[0]) { out[t] = 0.f; return; }     // not in the deflated set (gate)
@@ -415,7 +418,45 @@ __global__ void ritz_scale_kernel(const float* __restrict__ lam, int k, int mode
   float v = l;
   if (mode == 1) v = (l > 0.f ? 1.f : (l < 0.f ? -1.f : 0.f)) / gamma;
   else if (mode == 2) v = l > 0.f ? l : 0.f;
+  else if (mode == 4) v = 1.f / gamma;
+  else if (mode == 3) {
+    if (l > 0.f && isfinite(l)) v = (float)(pow((double)l, -1.0 / (double)p) - (double)root_scale[0] * (double)z_pad);
+    else { v = 0.f; if (status) atomicOr(status, DEFL_ST_NONFINITE); }
+  }
   out[t] = neg ? -v : v;
+}
+
+// root_scale = theta^(-1/p) (0 when theta is not a positive number: the status bit is already set by the estimate)
+__global__ void root_scale_kernel(const float* __restrict__ theta, int p, float* __restrict__ out) {
+  const double th = (double)theta[0];
+  out[0] = (th > 0.0 && isfinite(th)) ? (float)pow(th, -1.0 / (double)p) : 0.f;
+}
+
+// T = a I + b M for n x n fp32 matrices (the step matrix of the coupled Newton iteration), optionally rounded to tf32
+__global__ void __launch_bounds__(256) affine_identity_kernel(const float* __restrict__ M, float a, float b,
+                                                              float* __restrict__ T, int n, int round_tf32) {
+  const long long total = (long long)n * n;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  if ((n & 3) == 0) {
+    for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < total / 4; q += stride) {
+      const float4 m4 = reinterpret_cast<const float4*>(M)[q];
+      const long long e = q * 4;
+      const int i = (int)(e / n), j = (int)(e - (long long)i * n);
+      float v[4] = {b * m4.x, b * m4.y, b * m4.z, b * m4.w};
+      if (i >= j && i < j + 4) v[i - j] += a;
+      if (round_tf32) {
+#pragma unroll
+        for (int t = 0; t < 4; ++t) v[t] = round_to_tf32(v[t]);
+      }
+      reinterpret_cast<float4*>(T)[q] = make_float4(v[0], v[1], v[2], v[3]);
+    }
+  } else {
+    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
+      const int i = (int)(e / n), j = (int)(e - (long long)i * n);
+      float v = b * M[e] + ((i == j) ? a : 0.f);
+      T[e] = round_tf32 ? round_to_tf32(v) : v;
+    }
+  }
 }
 
 struct PsdWs {
@@ -428,7 +469,7 @@ struct PsdWs {
   float* Rinv; float* E; float* Es; float* lam; float* coef;   // [K,K] x3, [K], [K]
   float* Q; double* T; float* lw; float* lt; float* lv; float* lE; float* lrho;   // Lanczos state
   int* done; double* beta_prev;
-  double* npart; float* theta; float* inv_theta; float* dummy;
+  double* npart; float* theta; float* inv_theta; float* dummy; float* rscale;
   int* status;
   int* keff;        // [1] size of the deflated set (gate)
   float* start;     // [n] generated Lanczos start vector
@@ -463,7 +504,7 @@ static PsdWs carve_psd(void* base, int n, int K) {
   w.lE = cv.take<float>(S * S); w.lrho = cv.take<float>(S);
   w.done = cv.take<int>(1); w.beta_prev = cv.take<double>(1);
   w.npart = cv.take<double>(1184);
-  w.theta = cv.take<float>(1); w.inv_theta = cv.take<float>(1); w.dummy = cv.take<float>(S * S);
+  w.theta = cv.take<float>(1); w.inv_theta = cv.take<float>(1); w.dummy = cv.take<float>(S * S); w.rscale = cv.take<float>(1);
   w.status = cv.take<int>(1);
   w.keff = cv.take<int>(1);
   w.start = cv.take<float>(n);
@@ -514,8 +555,9 @@ static int estimate_scale(defl_ctx* c, const float* A, int n, int norm_mode, con
 
 // C = aux_scale * aux + alpha * U diag(coef) U^T  (rank-k symmetric update, exact fp32 products)
 static int rank_update(defl_ctx* c, const PsdWs& w, int n, int K, int k, int coef_mode, float gamma, int neg,
-                       const float* aux, float aux_scale, const float* aux_scale_dev, float* C, int round_tf32 = 0) {
-  ritz_scale_kernel<<<1, 64, 0, c->stream>>>(w.lam, k, coef_mode, gamma, neg, w.coef, w.keff);
+                       const float* aux, float aux_scale, const float* aux_scale_dev, float* C, int round_tf32 = 0,
+                       float z_pad = 0.f, int root_p = 1) {
+  ritz_scale_kernel<<<1, 64, 0, c->stream>>>(w.lam, k, coef_mode, gamma, neg, w.coef, w.keff, w.rscale, z_pad, root_p, w.status);
   ++c->launches;
   if (ctx_fail(c, cudaGetLastError(), "ritz scale")) return DEFL_ERR_CUDA;
   if (ctx_fail(c, scale_cols_launch(w.U, 0, K, 1, n, k, w.coef, K, nullptr, 1.f, 0.f, w.Us, 0, K, c->stream, &c->launches), "U diag"))
@@ -635,11 +677,13 @@ size_t defl_psd_workspace_bytes(int n, int K) {
   return carve_psd(nullptr, n, K).bytes;
 }
 
-int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float* warm_basis, int K,
-                     const float* coeff_schedule, int T, const defl_opts* opts, const defl_info* info) {
+// Algorithm 2 (root_p = 0), or the same deflation around the coupled Newton iteration for the inverse p-th root
+// (root_p = p; T is then the number of its steps and no coefficients are read)
+static int psd_core(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float* warm_basis, int K,
+                    const float* coeff_schedule, int T, const defl_opts* opts, const defl_info* info, int root_p) {
   if (!c || !Xv || !Pv || n <= 0 || k < 0 || K < 0 || T < 0) return DEFL_ERR_ARG;
   if (K > 0 && !warm_basis) return DEFL_ERR_ARG;
-  if (T > 0 && !coeff_schedule) return DEFL_ERR_ARG;
+  if (root_p == 0 && T > 0 && !coeff_schedule) return DEFL_ERR_ARG;
   if (k > K || K > DEFL_MAX_L || K >= n || T > DEFL_MAX_STEPS) return DEFL_ERR_RANK;
   const float* Z = reinterpret_cast<const float*>(Xv);
   float* P = reinterpret_cast<float*>(Pv);
@@ -666,7 +710,7 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
   const int tf32_round = (engine == DEFL_ENGINE_TENSOR) ? 1 : 0;
   // FP16 filter (Appendix E.2, "Composite Minimax Filter": the filter is used in half precision): iterates in IEEE half, kind::f16 products
   const bool half = opts && opts->half_filter;
-  if (half && (engine != DEFL_ENGINE_TENSOR || (n & 7))) return DEFL_ERR_UNSUPPORTED;
+  if (half && (root_p != 0 || engine != DEFL_ENGINE_TENSOR || (n & 7))) return DEFL_ERR_UNSUPPORTED;
 
   cudaSetDevice(c->device);
   int rc = ctx_reserve(c, carve_psd(nullptr, n, K).bytes);
@@ -734,7 +778,8 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
   float* bufs[2] = {w.Xa, w.Xb};
   int cur = 0;
   if (deflate) {
-    if ((rc = rank_update(c, w, n, K, kcols, 1, gamma, 0, Rm, 1.f, w.inv_theta, bufs[cur], tf32_round))) return rc;
+    // (an inverse root pads at +1/gamma whatever the sign: a value that is not positive is reported, not followed)
+    if ((rc = rank_update(c, w, n, K, kcols, root_p ? 4 : 1, gamma, 0, Rm, 1.f, w.inv_theta, bufs[cur], tf32_round))) return rc;
   } else {
     if (ctx_fail(c, scale_launch(Rm, F32, bufs[cur], F32, 1, (long long)n * n, w.inv_theta, c->stream, &c->launches, tf32_round), "normalise"))
       return DEFL_ERR_CUDA;
@@ -742,7 +787,64 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
   ctx_stage_mark(c);
 
   // ---- stage 4: g = p_T o ... o p_1 on the symmetric X0: W = X^2, Tt = a I + b W + c W^2, X <- X Tt ------
-  if (half && T > 0) {
+  float* root_z = nullptr;       // inverse root: Z_T
+  if (root_p) {
+    // Coupled Newton iteration on M_0 = X0, Z_0 = I: T_t = ((p+1) I - M_t)/p, Z_{t+1} = Z_t T_t, M_{t+1} = T_t^p M_t.
+    // Every iterate is a polynomial in X0, so every product is a symmetric matrix: the tiles on and above the
+    // diagonal are computed and mirrored, as in the filter of the projection. Z_1 = T_0 is a copy; the last step
+    // does not update M. Buffers: M and two spares among {Xa, Xb, Tt}, T_t in W, Z alternating between the residual's
+    // buffer (free once X0 exists) and the output, ending in the former.
+    float* M = bufs[cur];
+    float* spare[2] = {bufs[cur ^ 1], w.Tt};
+    float* Tm = w.W;
+    const int swaps = T > 1 ? T - 1 : 0;
+    float* zc = (swaps & 1) ? P : w.R;
+    float* zn = (swaps & 1) ? w.R : P;
+    const long long nn = (long long)n * n;
+    const int ablk = (int)((nn / 4 + 255) / 256 < 1184 ? (nn / 4 + 255) / 256 + 1 : 1184);
+    auto product = [&](const float* Aop, const float* Bop, float* Cout, const char* what) {
+      GemmDesc g = gemm_desc_zero();
+      g.batch = 1; g.in_dtype = F32; g.b_dtype = F32; g.out_dtype = F32;
+      g.M = n; g.N = n; g.K[0] = n;
+      g.A[0] = Aop; g.sa_i[0] = n; g.sa_k[0] = 1;
+      g.B[0] = Bop; g.sb_k[0] = 1; g.sb_j[0] = n;          // symmetric: rows as columns
+      g.C = Cout; g.ldc = n; g.epilogue = EPI_STORE; g.symmetric = 1; g.round_tf32 = tf32_round;
+      return run_gemm(c, g, gemm_tc_supported(g) ? engine : DEFL_ENGINE_SIMT, what);
+    };
+    if (T == 0) {
+      affine_identity_kernel<<<ablk, 256, 0, c->stream>>>(M, 1.f, 0.f, zc, n, 0);
+      ++c->launches;
+      if (ctx_fail(c, cudaGetLastError(), "identity")) return DEFL_ERR_CUDA;
+    }
+    for (int t = 0; t < T; ++t) {
+      affine_identity_kernel<<<ablk, 256, 0, c->stream>>>(M, (float)(root_p + 1) / (float)root_p, -1.f / (float)root_p, Tm, n, tf32_round);
+      ++c->launches;
+      if (ctx_fail(c, cudaGetLastError(), "step matrix")) return DEFL_ERR_CUDA;
+      if (t == 0) {
+        if (ctx_fail(c, cudaMemcpyAsync(zc, Tm, (size_t)nn * sizeof(float), cudaMemcpyDeviceToDevice, c->stream), "Z_1"))
+          return DEFL_ERR_CUDA;
+      } else {
+        if ((rc = product(zc, Tm, zn, "Z T"))) return rc;
+        float* sw = zc; zc = zn; zn = sw;
+      }
+      if (t + 1 == T) break;
+      if (root_p == 1) {
+        if ((rc = product(Tm, M, spare[0], "T M"))) return rc;
+        float* old = M; M = spare[0]; spare[0] = old;
+      } else if (root_p == 2) {
+        if ((rc = product(Tm, Tm, spare[0], "T^2"))) return rc;
+        if ((rc = product(spare[0], M, spare[1], "T^2 M"))) return rc;
+        float* old = M; M = spare[1]; spare[1] = old;
+      } else {
+        if ((rc = product(Tm, Tm, spare[0], "T^2"))) return rc;
+        if ((rc = product(spare[0], spare[0], spare[1], "T^4"))) return rc;
+        if ((rc = product(spare[1], M, spare[0], "T^4 M"))) return rc;
+        float* old = M; M = spare[0]; spare[0] = old;
+      }
+    }
+    root_z = zc;
+  }
+  if (!root_p && half && T > 0) {
     // half-precision buffers inside the fp32 scratch that is free here: the two iterates share the other iterate
     // buffer, W and Tt share the fp32 W; the result returns to fp32 (rounded to tf32) for the reconstruction
     const size_t nn = (size_t)n * n;
@@ -773,7 +875,7 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
     if (ctx_fail(c, scale_launch(H[hc], F16, bufs[cur], F32, 1, (long long)nn, nullptr, c->stream, &c->launches, tf32_round), "from half"))
       return DEFL_ERR_CUDA;
   }
-  for (int t = 0; t < (half ? 0 : T); ++t) {
+  for (int t = 0; t < ((half || root_p) ? 0 : T); ++t) {
     const float ca = coeff_schedule[3 * t], cb = coeff_schedule[3 * t + 1], cc = coeff_schedule[3 * t + 2];
     const float* X = bufs[cur];
     float* Xn = bufs[cur ^ 1];
@@ -800,8 +902,34 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
   }
   ctx_stage_mark(c);
 
+  // ---- stage 5 (inverse root): out = theta^(-1/p) (Z - z_pad U U^T) + U diag(lambda^(-1/p)) U^T, symmetrised ----
+  if (root_p) {
+    root_scale_kernel<<<1, 1, 0, c->stream>>>(w.theta, root_p, w.rscale);
+    ++c->launches;
+    if (ctx_fail(c, cudaGetLastError(), "root scale")) return DEFL_ERR_CUDA;
+    if (deflate) {
+      // what the scalar iteration makes of the padding value 1/gamma (fp64 on the host: T steps)
+      double m = 1.0 / (double)gamma, z = 1.0;
+      for (int t = 0; t < T; ++t) {
+        const double tt = ((double)(root_p + 1) - m) / (double)root_p;
+        z *= tt;
+        for (int q = 0; q < root_p; ++q) m *= tt;
+      }
+      if ((rc = rank_update(c, w, n, K, kcols, 3, gamma, 0, root_z, 1.f, w.rscale, P, 0, (float)z, root_p))) return rc;
+    } else {
+      if (ctx_fail(c, scale_launch(root_z, F32, P, F32, 1, (long long)n * n, w.rscale, c->stream, &c->launches, 0), "scale"))
+        return DEFL_ERR_CUDA;
+    }
+    symmetrise_kernel<<<dim3((n + 31) / 32, (n + 31) / 32), 256, 0, c->stream>>>(P, n);
+    ++c->launches;
+    if (ctx_fail(c, cudaGetLastError(), "symmetrise")) return DEFL_ERR_CUDA;
+    // the iteration diverges on an eigenvalue of X0 that is not positive (an indefinite input, or a basis that has not
+    // settled: a Ritz pair with residual r leaves R indefinite by about -|r|^2 / (r^T A r / |r|^2)): report it
+    if (ctx_fail(c, finite_probe_launch(P, F32, 1, (long long)n * n, w.status, c->stream, &c->launches), "finite probe"))
+      return DEFL_ERR_CUDA;
+  }
   // ---- stage 5: P = (R + R g(X0))/2 + sum_{lambda_i > 0} lambda_i u_i u_i^T, symmetrised (lines 8, 12) ----
-  {
+  if (!root_p) {
     GemmDesc g = gemm_desc_zero();
     g.batch = 1; g.in_dtype = F32; g.b_dtype = F32; g.out_dtype = F32;
     g.M = n; g.N = n; g.K[0] = n;
@@ -859,6 +987,17 @@ int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float*
   return DEFL_OK;
 }
 
+
+int defl_psd_project(defl_ctx* c, const void* Xv, void* Pv, int n, int k, float* warm_basis, int K,
+                     const float* coeff_schedule, int T, const defl_opts* opts, const defl_info* info) {
+  return psd_core(c, Xv, Pv, n, k, warm_basis, K, coeff_schedule, T, opts, info, 0);
+}
+
+int defl_inv_root(defl_ctx* c, const void* Av, void* outv, int n, int p, int k, float* warm_basis, int K, int steps,
+                  const defl_opts* opts, const defl_info* info) {
+  if (p != 1 && p != 2 && p != 4) return DEFL_ERR_ARG;
+  return psd_core(c, Av, outv, n, k, warm_basis, K, nullptr, steps, opts, info, p);
+}
 
 int defl_admm_diag_sdp(defl_ctx* c, const void* Cv, const float* b, int n, float sigma, int iters, int warmup_iters,
                        void* Xv, void* Sv, float* y, int k, float* warm_basis, int K, const float* coeff_schedule,

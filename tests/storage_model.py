@@ -147,7 +147,7 @@ def symmetric_filter_with_storage(X0, sched, fmt):
         W = rnd(oracle.matmul(X, X))
         T = rnd(a * np.eye(n) + b * W + c * oracle.matmul(W, W))
         X = oracle.matmul(X, T)
-        X = rnd(0.5 * (X + X.T))          # the path computes the upper tiles and mirrors them
+        X = rnd(np.triu(X) + np.triu(X, 1).T)          # the path computes the upper triangle and mirrors it
     return round_tf32(X)
 
 
@@ -165,3 +165,60 @@ def psd_storage_error(Z, Vb, k, sched, gamma, warmup, lanczos_v0, fmt):
     return float(np.linalg.norm(stored - exact) / np.linalg.norm(exact)), exact
 
 
+
+
+def inv_root_pieces(A, Vb, k, gamma, warmup, lanczos_v0):
+    """What the deflated inverse root builds before its iteration, from oracle primitives in its order: Ritz pairs of
+    the incoming basis, the residual, the Lanczos scale and the padded, normalised X0. Returns (X0, theta, U_I, lam_I)
+    with the removed Ritz vectors in the columns of U_I."""
+    A = np.asarray(A, dtype=np.float64)
+    n = A.shape[0]
+    UI, lamI = np.zeros((n, 0)), np.zeros(0)
+    if not warmup and k > 0 and Vb is not None and Vb.shape[1] > 0:
+        H = oracle.matmul(Vb, oracle.matmul(A, Vb), ta=True)
+        lam, E = oracle.jacobi_eig(0.5 * (H + H.T))
+        U = oracle.matmul(Vb, E)
+        idx = sorted(range(len(lam)), key=lambda i: (-abs(lam[i]), i))[:k]
+        UI, lamI = U[:, idx], np.array([lam[i] for i in idx])
+    R = A - (UI * lamI) @ UI.T
+    theta = oracle.lanczos_upper(R, lanczos_v0)
+    return R / theta + UI @ UI.T / gamma, theta, UI, lamI
+
+
+def inv_root_iteration_with_storage(X0, p, steps, fmt):
+    """Z_T of the coupled Newton iteration the way the path stores it: X0, every step matrix T_t, every Z_t and every
+    power and M_t are rounded to `fmt` when written; products by the oracle's matmul (exact in between), each taken
+    with its upper triangle mirrored into the lower one, as the path does (the rounded factors no longer commute
+    exactly, so the product has a small antisymmetric part, which the mirror turns into a symmetric error)."""
+    rnd = ROUNDERS[fmt]
+    n = X0.shape[0]
+    sym = lambda X: np.triu(X) + np.triu(X, 1).T
+    M = rnd(np.asarray(X0, dtype=np.float64))
+    Z = np.eye(n)
+    for t in range(steps):
+        T = rnd(((p + 1) * np.eye(n) - M) / p)
+        Z = T if t == 0 else rnd(sym(oracle.matmul(Z, T)))
+        if t + 1 == steps:
+            break
+        P = T
+        for _ in range({1: 0, 2: 1, 4: 2}[p]):
+            P = rnd(sym(oracle.matmul(P, P)))
+        M = rnd(sym(oracle.matmul(P, M)))
+    return Z
+
+
+def inv_root_storage_error(A, Vb, k, p, steps, gamma, warmup, lanczos_v0, fmt="tf32"):
+    """Relative Frobenius distance between the deflated inverse root with the iteration's stored matrices rounded to
+    `fmt` and the same in fp64 throughout, both from the oracle's steps; also returns the unrounded result (it must
+    equal inv_root.deflated_inv_root's)."""
+    from oracle import inv_root
+    X0, theta, UI, lamI = inv_root_pieces(A, Vb, k, gamma, warmup, lanczos_v0)
+    z_pad, _ = inv_root.inv_root_scalar(1.0 / gamma, p, steps)
+    scale = theta ** (-1.0 / p)
+
+    def restore(Z):
+        out = scale * Z + (UI * (lamI ** (-1.0 / p) - scale * z_pad)) @ UI.T if lamI.size else scale * Z
+        return 0.5 * (out + out.T)
+    exact = restore(inv_root.coupled_newton(X0, p, steps)[0])
+    stored = restore(inv_root_iteration_with_storage(X0, p, steps, fmt))
+    return float(np.linalg.norm(stored - exact) / np.linalg.norm(exact)), exact

@@ -63,3 +63,19 @@ def test_psd_pieces_rebuild_the_oracle_projection(warmup):
     err, exact = sm.psd_storage_error(Z, Vb, k, sched, 1.1, warmup, v0, "tf32")
     assert np.linalg.norm(exact - P) <= 1e-10 * np.linalg.norm(P)
     assert 0.0 < err < 1e-2
+
+
+def test_inv_root_storage_model_reduces_to_the_oracle_without_rounding():
+    from oracle import inv_root
+    rng = np.random.default_rng(5)
+    n, k, p, T = 24, 2, 2, 5
+    q, _ = np.linalg.qr(rng.standard_normal((n, n)))
+    lam = np.concatenate([[400.0, 150.0], np.linspace(1.0, 0.1, n - 2)])
+    A = (q * lam) @ q.T
+    Vb = oracle.householder_orth(q[:, :3] + 1e-4 * rng.standard_normal((n, 3)))
+    v0 = rng.standard_normal(n)
+    err, exact = sm.inv_root_storage_error(A, Vb, k, p, T, 1.1, False, v0, fmt="none")
+    want, *_ = inv_root.deflated_inv_root(A, Vb, k, p, T, gamma=1.1, lanczos_v0=v0)
+    assert err <= 1e-13 and np.allclose(exact, want, atol=1e-12 * np.abs(want).max())
+    err32, _ = sm.inv_root_storage_error(A, Vb, k, p, T, 1.1, False, v0, fmt="tf32")
+    assert 1e-5 < err32 < 3e-3                      # 10 mantissa bits, a handful of stored matrices

@@ -399,6 +399,53 @@ def extra_sdp(ctx, peaks, device, n=4096, calls=20, warm=2, tf32_peak=True):
                                  "note": "R (67 MB) fits the 126 MB L2: passes after the first are served from it"}}
 
 
+def extra_inv_root(ctx, device, tf32_peak, n=4096, p=4, calls=12, warm=2):
+    """The deflated inverse p-th root at n = 4096 (tf32 products): a static synthetic preconditioner statistic (8
+    eigenvalues of 300..2000 over a bulk spread log-uniformly over [0.06, 1]), 2 warm-up calls, then deflated calls:
+    ms per call, stage split, the iteration's products against the tf32 rate measured in this run."""
+    import torch
+    from paper_2609_21102_b200 import inputs
+    K, k, T = 16, 8, 8
+    u = inputs.rand((n - k,), 705, device=device).double()
+    lam = torch.cat([torch.linspace(2000.0, 300.0, k, dtype=torch.float64, device=device), 0.06 ** u])
+    q = inputs.haar(n, n, 700, device=device)
+    A = ((q * lam.unsqueeze(0)) @ q.T)
+    A = (0.5 * (A + A.T)).float()
+    del q
+    V = inputs.randn((n, K), inputs.seed_for(5, 1, inputs.PURPOSE_BASIS), device).float()
+    v0 = inputs.gaussian_vector(n, 5, inputs.PURPOSE_LANCZOS, device=device)
+    out = torch.empty((n, n), dtype=torch.float32, device=device)
+    times = []
+    for t in range(calls):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.defl_inv_root(A, p, k, V, T, out=out, gamma=1.1, lanczos_start=v0, warmup=t < warm, exploit_symmetry=True)
+        e1.record()
+        torch.cuda.synchronize()
+        if t >= warm:
+            times.append(e0.elapsed_time(e1))
+    nd = len(times)
+    st = [x / nd for x in ctx.defl_get_stage_ms(nd)]
+    names = ["block_step_rayleigh_ritz", "deflate", "lanczos_scale", "initialise", "iteration", "restore", "basis_update"]
+    # distance from the definition: A^(-1/p) from a library eigendecomposition in fp64 (outside every timed path)
+    w, v = torch.linalg.eigh(A.double())
+    exact = (v * w.pow(-1.0 / p).unsqueeze(0)) @ v.T
+    rel_err = float((out.double() - exact).norm() / exact.norm())
+    del w, v, exact
+    nprod = {1: 2, 2: 3, 4: 4}[p] * (T - 1)                 # Z T and the M update, none of the former in the first step, none of the latter in the last
+    flops = nprod * 1.0 * n * n * (n + 1.0)
+    times.sort()
+    return {"workload": "deflated inverse %d-th root, fp32 storage / tf32 products: static symmetric positive definite %dx%d "
+                        "matrix, 8 eigenvalues 300..2000 over a bulk in [0.06, 1], k=8, K=16, %d coupled Newton steps, "
+                        "2 warm-up calls" % (p, n, n, T),
+            "ms_per_call": sum(times) / nd, "ms_per_call_median": times[nd // 2], "stage_ms": dict(zip(names, st)),
+            "rel_error_vs_fp64_eigendecomposition": rel_err,
+            "roofline_iteration": {"bound": "tensor", "kernel": "gemm_tc_kernel (tf32, symmetric: Z T, T^2, T^4, T^p M)",
+                                   "achieved": flops / (st[4] * 1e-3) / 1e12, "peak": tf32_peak, "unit": "TFLOP/s",
+                                   "frac": flops / (st[4] * 1e-3) / 1e12 / tf32_peak,
+                                   "peak_kind": "torch.matmul 8192^3 with tf32 allowed, best of 10, this run"}}
+
+
 def spawn_ranks(args):
     """--gpus N without an outer launcher: start the N ranks here (weak-scaling replicas, one batch per rank)."""
     s = socket.socket()
@@ -429,6 +476,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the matrices per shape group (profiling captures)")
     ap.add_argument("--sdp-only", type=int, default=0, metavar="CALLS",
                     help="run only the SDP projection sequence (n = 4096) with this many calls and print its figures (profiling captures)")
+    ap.add_argument("--inv-root-only", type=int, default=0, metavar="CALLS",
+                    help="run only the deflated inverse-root calls (n = 4096) and print their figures")
     args = ap.parse_args()
 
     wl_name = "small" if args.small else "gpt2_xl"
@@ -475,6 +524,9 @@ def main():
         dist.init_process_group("nccl", device_id=device)
     ctx = binding.Context(local_rank)
     ctx.defl_set_profiling(True)
+    if args.inv_root_only > 0:
+        print(json.dumps(extra_inv_root(ctx, device, float("nan"), calls=args.inv_root_only, warm=min(2, args.inv_root_only - 1))))
+        return
     if args.sdp_only > 0:
         print(json.dumps(extra_sdp(ctx, load_peaks()[0], device, calls=args.sdp_only, warm=min(2, args.sdp_only - 1), tf32_peak=False)))
         return
@@ -661,6 +713,7 @@ def main():
             extras["gpt2_xl_add_restore"] = extra_polar(ctx, "gpt2_xl", dict(opts, mode=1), device, steps=10,
                                                         label="GPT-2-XL batch, additive restore (Eq. 3) in the last filter product")
             extras["sdp_4096"] = extra_sdp(ctx, peaks, device)
+            extras["inv_root_4096"] = extra_inv_root(ctx, device, extras["sdp_4096"]["roofline_filter"]["peak"])
         except Exception as e:      # an extra that fails must not take the headline with it
             extras["error"] = repr(e)
         line["extras"] = extras

@@ -99,6 +99,35 @@ def test_inv_root_matches_oracle_with_tracked_basis(ctx, n, K, k, p, engine_name
     assert _rel(plain, exact) > 0.3           # the same depth without deflation is nowhere near
 
 
+def test_inv_root_n1024_spans_many_tiles(ctx):
+    """Several 256 x 256 tiles each way with a ragged last one (1000 = 3 x 256 + 232): two warm-up calls, then one
+    deflated call against the oracle and against the definition."""
+    n, K, k, p, steps = 1000, 16, 8, 2, 8
+    A64, lam, q = _statistics_like(n, k, 1700)
+    A = A64.float().cuda()
+    Ao = A.double().cpu().numpy()
+    Vg = inputs.randn((n, K), 1091).float().cuda()
+    Vo = _orth(Vg.double().cpu().numpy())
+    v0 = inputs.gaussian_vector(n, 5, inputs.PURPOSE_LANCZOS).cuda()
+    v0n = v0.double().cpu().numpy()
+    for it in range(3):
+        warm = it < 2
+        out, info = ctx.defl_inv_root(A, p, k, Vg, steps, gamma=1.1, lanczos_start=v0, want_info=True, exploit_symmetry=True,
+                                      warmup=warm)
+        if warm:
+            _, Vo, *_ = inv_root.deflated_inv_root(Ao, Vo, k, p, 0, warmup=True, lanczos_v0=v0n)     # basis only
+    want, _, lam_o, ndef, theta_o = inv_root.deflated_inv_root(Ao, Vo, k, p, steps, gamma=1.1, lanczos_v0=v0n)
+    got = out.double().cpu().numpy()
+    tol, model = _tol("tensor", Ao, Vo, k, p, steps, False, v0n)
+    err = _rel(got, want)
+    print("inv root n=%d p=%d: error %.3e, storage model %.3e, tolerance %.3e" % (n, p, err, model, tol))
+    assert int(info["status"][0]) == 0 and ndef == k
+    assert err <= tol
+    assert abs(float(info["theta"][0]) - theta_o) <= 1e-3 * theta_o
+    w, v = np.linalg.eigh(Ao)
+    assert _rel(got, (v * w ** (-1.0 / p)) @ v.T) <= 5e-3
+
+
 def test_inv_root_plain_reciprocal_and_warmup(ctx):
     from paper_2609_21102_b200 import binding
     n, p, steps = 192, 1, 9

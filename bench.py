@@ -67,17 +67,34 @@ def schedule_of(name, L):
     return _MINIMAX[L]
 
 
-def algorithmic_flops(m, n, k, p, J, L, symmetric, add_restore=False):
-    """Flops the method needs for one matrix: (filter, front end). Filter per step: the Gram matrix and its square
-    (each counted once per symmetric pair when the symmetric tiles are on, else in full) and the apply product;
-    front end: the (2 + 2J) products of the randomized SVD with the l-column panel, the rank-k subtraction and, with
-    the additive restore, the rank-k add."""
+def filter_passes(m, n, sched, iterates=0):
+    """How the library walks the filter steps of a bf16 batch of this shape: a list of 1s and 2s, one entry per pass
+    over X (2 = two steps in one pass: A_{t+1} = B_t^2 A_t on the short side, X <- (B_{t+1} B_t) X). Greedily from the
+    first step, a pair starts at step t when there is a next step, |a_t| <= 4.5 and |b_{t+1} + 2 c_{t+1}| <= 1, provided the long side is at least
+    twice the short one (`iterates` = 1, bf16 throughout, pairs nothing)."""
+    ms, ml = min(m, n), max(m, n)
+    L = len(sched)
+    if ml < 2 * ms or iterates == 1 or os.environ.get("DEFL_NO_PAIRED_STEPS"):
+        return [1] * L
+    out, t = [], 0
+    while t < L:
+        two = t + 1 < L and abs(sched[t][0]) <= 4.5 and abs(sched[t + 1][1] + 2.0 * sched[t + 1][2]) <= 1.0
+        out.append(2 if two else 1)
+        t += 2 if two else 1
+    return out
+
+
+def algorithmic_flops(m, n, k, p, J, L, symmetric, add_restore=False, passes=None):
+    """Flops the method needs for one matrix: (filter, front end). Filter per single step: the Gram matrix and its
+    square (each counted once per symmetric pair when the symmetric tiles are on, else in full) and the apply product;
+    per paired step (see filter_passes): one Gram and one apply product and five short-side products; front end: the
+    (2 + 2J) products of the randomized SVD with the l-column panel, the rank-k subtraction and, with the additive
+    restore, the rank-k add. `passes` None = one pass per step (the per-step count)."""
     ms, ml = min(m, n), max(m, n)
     l = min(ms, k + p) if k > 0 else 0
-    if symmetric:
-        filt = L * (ms * (ms + 1.0) * ml + ms * ms * (ms + 1.0) + 2.0 * ms * ms * ml)
-    else:
-        filt = L * (4.0 * ms * ms * ml + 2.0 * ms ** 3)
+    big_g, big_a = (ms * (ms + 1.0) * ml, 2.0 * ms * ms * ml) if symmetric else (2.0 * ms * ms * ml, 2.0 * ms * ms * ml)
+    small = ms * ms * (ms + 1.0) if symmetric else 2.0 * ms ** 3
+    filt = sum(big_g + big_a + (small if q == 1 else 5.0 * small) for q in (passes if passes is not None else [1] * L))
     front = (2.0 * ml * ms * l * (2 + 2 * J) + 2.0 * m * n * k * (2 if add_restore else 1)) if k > 0 else 0.0
     return filt, front
 
@@ -241,10 +258,22 @@ def time_steps(fn, steps, sync):
     return e0.elapsed_time(e1) / steps
 
 
-def workload_flops(wl, sym, add=False):
-    filt = sum(b * algorithmic_flops(m, n, wl["k"], wl["p"], wl["J"], wl["L"], sym, add)[0] for b, m, n in wl["groups"])
-    front = sum(b * algorithmic_flops(m, n, wl["k"], wl["p"], wl["J"], wl["L"], sym, add)[1] for b, m, n in wl["groups"])
+def workload_flops(wl, sym, add=False, iterates=0, per_step=False):
+    """(filter, front end) flops of one batch as the library evaluates it (paired steps where it pairs them), or with
+    `per_step` the count of one pass over X per step."""
+    filt = front = 0.0
+    for b, m, n in wl["groups"]:
+        passes = None if per_step else filter_passes(m, n, schedule_of(wl["schedule"], wl["L"]), iterates)
+        f, fr = algorithmic_flops(m, n, wl["k"], wl["p"], wl["J"], wl["L"], sym, add, passes)
+        filt += b * f
+        front += b * fr
     return filt, front
+
+
+def filter_launches(wl, add=False, iterates=0):
+    """Product launches of the filter stage per batch: three per single step, seven per paired step."""
+    sched = schedule_of(wl["schedule"], wl["L"])
+    return sum(sum(3 if q == 1 else 7 for q in filter_passes(m, n, sched, iterates)) for _, m, n in wl["groups"])
 
 
 def oracle_sample(wl):
@@ -325,7 +354,8 @@ def extra_polar(ctx, name, opts, device, steps=10, label=None, graph=False):
     launches = (ctx.defl_launch_count() - l0) // steps
     st = ctx.defl_get_stage_ms(min(64, steps * len(groups)))
     per = min(64, steps * len(groups)) / len(groups)
-    filt, front = workload_flops(wl, opts["sym"], opts["mode"] == 1)
+    filt, front = workload_flops(wl, opts["sym"], opts["mode"] == 1, opts["iterates"], per_step=True)     # algorithmic
+    filt_exec, _ = workload_flops(wl, opts["sym"], opts["mode"] == 1, opts["iterates"])
     graph_ms = None
     if graph:
         # the launch-bound small batches replayed from a CUDA graph: every call of the library only enqueues work on its
@@ -347,7 +377,7 @@ def extra_polar(ctx, name, opts, device, steps=10, label=None, graph=False):
         except Exception as e:
             graph_ms = "capture failed: %r" % (e,)
     out = {"workload": label or wl["label"], "ms_per_batch": ms, "ms_per_batch_cuda_graph": graph_ms,
-           "tflops": (filt + front) / (ms * 1e-3) / 1e12,
+           "tflops": (filt + front) / (ms * 1e-3) / 1e12, "executed_tflops": (filt_exec + front) / (ms * 1e-3) / 1e12,
            "matrices_per_s": sum(b for b, _, _ in wl["groups"]) / (ms * 1e-3), "launches_per_batch": int(launches),
            "stage_ms": {"rsvd": st[0] / per, "deflate_normalise": st[1] / per, "filter": st[2] / per, "restore": st[3] / per}}
     del groups
@@ -547,8 +577,14 @@ def main():
         return ctx.defl_launch_count() + (sum(c.defl_launch_count() for c, _ in lanes) if lanes else 0)
 
     step = lambda: run_step(ctx, wl, groups, opts, lanes)
-    filt_f, front_f = workload_flops(wl, opts["sym"], opts["mode"] == 1)
+    # Two counts. Algorithmic: one Gram, one polynomial and one apply product per filter step (symmetric products once),
+    # the work the method is defined by; it gives `value`, `roofline.achieved` and the end-to-end figure. Executed: the
+    # products the library actually runs (where two steps share one pass over X: one Gram, one apply, five short-side
+    # products); it gives `executed_tflops` and `roofline.executed_*`, which is what the tensor pipe did.
+    filt_f, front_f = workload_flops(wl, opts["sym"], opts["mode"] == 1, opts["iterates"], per_step=True)
     tot_f = filt_f + front_f
+    exec_filt_f, _ = workload_flops(wl, opts["sym"], opts["mode"] == 1, opts["iterates"])
+    exec_f = exec_filt_f + front_f
     dense_f = sum(b * dense_filter_flops(m, n, wl["L"]) for b, m, n in wl["groups"]) + front_f
     nmat = sum(b for b, _, _ in wl["groups"])
 
@@ -667,8 +703,9 @@ def main():
     sust = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
     value = aggregate_throughput(tot_f, world, ms_per_step) / 1e12
     filt_ms = stage_ms[2]
-    n_filter_launches = 3 * wl["L"] * ngroups
+    n_filter_launches = filter_launches(wl, opts["mode"] == 1, opts["iterates"])
     ach = filt_f / (filt_ms * 1e-3) / 1e12 if filt_ms > 0 else None
+    ach_exec = exec_filt_f / (filt_ms * 1e-3) / 1e12 if filt_ms > 0 else None
     sm_mhz = clocks.get("sm_mhz") or 0.0
     # a short timed region runs near the maximum clock (compare with the burst peak), a long one at the power cap
     # (compare with the sustained peak): both fractions are given, and time x clock so that runs at different clocks compare
@@ -676,7 +713,11 @@ def main():
                 "achieved": ach, "peak": burst, "unit": "TFLOP/s", "frac": (ach / burst) if ach else None,
                 "peak_kind": "bf16_tflops (burst), of %s" % peaks_kind,
                 "frac_of_sustained_peak": (ach / sust) if ach else None,
-                "flops": "flops the method needs (symmetric products once); per launch: %.4g" % (filt_f / n_filter_launches),
+                "flops": "algorithmic: one Gram, one polynomial and one apply product per filter step, symmetric products once "
+                         "(%.4g per step of the batch); executed_*: the products the library runs, two steps per pass over X "
+                         "where it pairs them (%.4g per launch)" % (filt_f / wl["L"], exec_filt_f / n_filter_launches),
+                "executed_achieved": ach_exec, "executed_frac": (ach_exec / burst) if ach_exec else None,
+                "executed_frac_of_sustained_peak": (ach_exec / sust) if ach_exec else None,
                 "launches_per_step": n_filter_launches, "avg_launch_ms": filt_ms / n_filter_launches,
                 "stage_source": stage_src,
                 "ms_x_mhz": filt_ms * sm_mhz,
@@ -687,7 +728,11 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
-            "flops_convention": "value = flops the method needs / time (symmetric products counted once); dense_equivalent_tflops counts them in full",
+            "flops_convention": "value = algorithmic flops / time: per filter step one Gram, one polynomial and one apply product, "
+                                "symmetric products counted once, plus the front end; executed_tflops counts the products the "
+                                "library runs (fewer where two filter steps share one pass over X); dense_equivalent_tflops "
+                                "counts every per-step product in full",
+            "executed_tflops": aggregate_throughput(exec_f, world, ms_per_step) / 1e12,
             "dense_equivalent_tflops": aggregate_throughput(dense_f, world, ms_per_step) / 1e12,
             "matrices_per_s": world * nmat / (ms_per_step * 1e-3),
             "pct_bf16_peak": {"burst": 100.0 * value / world / burst, "sustained": 100.0 * value / world / sust},

@@ -92,7 +92,8 @@ struct Carver {
 struct PolarWs {
   void* X;            // [b,m,n] dtype   second iterate buffer (the other one is `out`)
   void* Am; void* Bm; // [b,ms,ms] dtype  A_t = X X^T and B_t = a I + b A_t + c A_t^2
-  void* Cm;           // [b,ms,ms] dtype  Horner intermediate of the higher-degree maps (poly_terms > 3 only)
+  void* Cm;           // [b,ms,ms] dtype  Horner intermediate of the higher-degree maps (poly_terms > 3), B_t^2 and B_{t+1} B_t of a paired step
+  void* Dm;           // [b,ms,ms] dtype  A_{t+1} = B_t^2 A_t of a paired step
   float* Lp;          // [b,ml,l]  long-side panel  (Y, then Q)
   float* Sp;          // [b,ms,l]  short-side panel (A^T Q and its orthonormalisation; finally (Q^T A)^T)
   double* gram;       // [b,nchunk,l,l]
@@ -113,6 +114,13 @@ struct PolarWs {
 
 inline int round_up8(int x) { return (x + 7) & ~7; }
 
+// Two filter steps per pass over X (see the filter stage) pay when the long side is at least twice the short one:
+// per pair, three more ms^3 products against one Gram and one apply product of ms^2 ml each
+static bool paired_steps_shape(int m, int n, int dtype) {
+  const int ms = m < n ? m : n, ml = m < n ? n : m;
+  return dtype == BF16 && ml >= 2 * ms;
+}
+
 PolarWs carve_polar(void* base, int b, int m, int n, int dtype, int k, int l, int terms = 3) {
   const int ms = m < n ? m : n, ml = m < n ? n : m;
   const size_t es = dtype_size(dtype);
@@ -121,7 +129,9 @@ PolarWs carve_polar(void* base, int b, int m, int n, int dtype, int k, int l, in
   w.X = cv.take<char>((size_t)b * m * n * es);
   w.Am = cv.take<char>((size_t)b * ms * ms * es);
   w.Bm = cv.take<char>((size_t)b * ms * ms * es);
-  w.Cm = cv.take<char>(terms > 3 ? (size_t)b * ms * ms * es : 1);
+  const bool pairable = paired_steps_shape(m, n, dtype);
+  w.Cm = cv.take<char>((terms > 3 || pairable) ? (size_t)b * ms * ms * es : 1);
+  w.Dm = cv.take<char>(pairable ? (size_t)b * ms * ms * es : 1);
   const int le = l > 0 ? l : 1, ke = k > 0 ? k : 1;
   w.Lp = cv.take<float>((size_t)b * ml * le);
   w.Sp = cv.take<float>((size_t)b * ms * le);
@@ -292,6 +302,7 @@ int defl_create(defl_ctx** out, int device) {
   c->knobs.transposed_apply = getenv("DEFL_NO_TRANSPOSED_APPLY") ? 0 : 1;
   c->knobs.host_chunks = getenv("DEFL_HOST_CHUNKS") ? atoi(getenv("DEFL_HOST_CHUNKS")) : 0;
   c->knobs.jacobi_sweeps = getenv("DEFL_JACOBI_SWEEPS") ? atoi(getenv("DEFL_JACOBI_SWEEPS")) : 0;
+  c->knobs.paired_steps = getenv("DEFL_NO_PAIRED_STEPS") ? 0 : 1;
   cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device);
   int ok = 1;
   if (cudaMalloc(&c->wait_status, 2 * sizeof(int)) != cudaSuccess) ok = 0;      // status word, tile counter
@@ -576,7 +587,30 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
   const int it_mode = opts ? opts->bf16_iterates : 0;
   const bool half_iter = dtype == DEFL_BF16 && L > 0 && it_mode != 1;
   // the first `n_half` filter steps keep the iterate in scaled IEEE half, the rest in bf16
-  const int n_half = half_iter ? ((it_mode == 2 || mode == DEFL_RESTORE_ADD) ? L : (L < 2 ? L : 2)) : 0;
+  // Paired steps (two filter steps per pass over X, both in scaled half: see the filter stage) on the tensor engine's
+  // bf16 path when the shape pays for them; every step but an odd last one is then kept in half
+  const bool pair_ok = c->knobs.paired_steps && half_iter && terms == 3 && engine != DEFL_ENGINE_SIMT &&
+                       paired_steps_shape(m, n, dtype);
+  // A pair starts at step t when a next step exists and two gains are moderate. The short-side step multiplies the
+  // rounding of the stored A_t by about a_t^2 in the directions of small singular values (12 for Muon's quintic, 70 for
+  // the steep first step of a per-step minimax schedule, which therefore stays a step of its own): |a_t| <= 4.5. And the
+  // next polynomial is evaluated on an A_{t+1} that was not recomputed from the iterate, so its rounding reaches
+  // B_{t+1} with the gain |b_{t+1} + 2 c_{t+1}| at the top of the spectrum (0.7 for Muon's quintic, 0.5 for the
+  // classical one, 1.5-2 for the middle steps of a minimax schedule, where a pair left single singular values 0.1
+  // off): <= 1. The walk is greedy from the first step.
+  auto pair_starts = [&](int t) {
+    if (!pair_ok || t + 1 >= L) return false;
+    const float* c0 = coeff_schedule + (size_t)terms * t;
+    const float* c1 = c0 + terms;
+    return fabsf(c0[0]) <= 4.5f && fabsf(c1[1] + 2.f * c1[2]) <= 1.0f;
+  };
+  int n_half_rule = half_iter ? ((it_mode == 2 || mode == DEFL_RESTORE_ADD) ? L : (L < 2 ? L : 2)) : 0;
+  int npass = 0;
+  for (int t = 0; t < L; ++npass) {
+    if (pair_starts(t)) { t += 2; if (t > n_half_rule) n_half_rule = t; }       // both steps of a pair in scaled half
+    else t += 1;
+  }
+  const int n_half = n_half_rule;
   const int it_dtype = n_half > 0 ? (int)F16 : dtype;      // format and scale of X_0
   const float ys = n_half > 0 ? 32.f : 1.f;
 
@@ -601,7 +635,9 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
 
   // iterate buffers: the chain must end in `out`
   void* bufs[2] = {w.X, out};
-  int cur = (L % 2 == 0) ? 1 : 0;        // X0 goes to bufs[cur]; after L swaps the result is in out
+  // X0 goes to bufs[cur]; every pass over X swaps the buffers, and the last one must write `out` (a paired step is one
+  // pass for two filter steps)
+  int cur = (npass % 2 == 0) ? 1 : 0;
 
   // ---- stage 1: R = G - P diag(s) W^T, rho = ||R||_F, X0 = R/rho (+ P W^T / gamma) ----------------
   const float* left = tall ? w.Uk : w.Vk;     // [b,m,k]
@@ -755,11 +791,19 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
   };
 
   // ---- stage 2: X <- a X + b (X X^T) X + c (X X^T)^2 X, L times, through the short-side Gram -------
-  for (int t = 0; t < L; ++t) {
+  // Paired steps. X_{t+2} = B_{t+1} B_t X_t, and the Gram matrix of the step in between needs no pass over X:
+  // A_{t+1} = X_{t+1} X_{t+1}^T = B_t A_t B_t = B_t^2 A_t (B_t is a polynomial in A_t). A pair costs one Gram product and
+  // one apply product of ms^2 ml each plus five ms^3 products (A_t^2 in B_t, B_t^2, B_t^2 A_t, A_{t+1}^2 in B_{t+1},
+  // B_{t+1} B_t) where two single steps cost two of each big product and two small ones. Only ONE step is taken on the
+  // short side at a time, and only with the 11-bit storage: every further one would multiply the rounding of the
+  // stored A by a^2 (about 12), which the small singular values do not survive.
+  for (int t = 0; t < L;) {
+    const bool paired = pair_starts(t);                              // (both steps are then in scaled half)
+    const int tl = paired ? t + 1 : t;                               // the last step this pass over X covers
     const float* cf = coeff_schedule + (size_t)terms * t;       // a_0 .. a_{terms-1} of this step
     const void* X = bufs[cur];
     void* Xn = bufs[cur ^ 1];
-    const bool hs = t < n_half, hn = t + 1 < n_half;
+    const bool hs = t < n_half, hn = tl + 1 < n_half;
     const int it_dtype = hs ? (int)F16 : dtype, nx_dtype = hn ? (int)F16 : dtype;     // this step's and the next one's
     const float ys = hs ? 32.f : 1.f, ys_next = hn ? 32.f : 1.f;
     GemmDesc g = gemm_desc_zero();
@@ -793,40 +837,68 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
       else { g.pa = cf[terms - 3 - q]; g.pb = 0.f; g.pc = iy2; }
       if ((rc = run_gemm(c, g, engine, "polynomial"))) return rc;
     }
+    const void* Bap = w.Bm;          // what multiplies X: B_t, or B_{t+1} B_t
+    if (paired) {
+      const float* cf1 = coeff_schedule + (size_t)terms * (t + 1);
+      auto small_product = [&](const void* L_, const void* R_, void* C_, const char* what) {
+        GemmDesc q = gemm_desc_zero();
+        q.batch = b; q.in_dtype = it_dtype; q.b_dtype = it_dtype; q.out_dtype = it_dtype;
+        q.M = ms; q.N = ms; q.K[0] = ms;
+        q.A[0] = L_; q.sa_i[0] = ms; q.sa_k[0] = 1; q.batch_a[0] = (long long)ms * ms;
+        q.B[0] = R_; q.sb_k[0] = 1; q.sb_j[0] = ms; q.batch_b[0] = (long long)ms * ms;      // symmetric: rows as columns
+        q.C = C_; q.ldc = ms; q.batch_c = (long long)ms * ms;
+        q.epilogue = EPI_STORE; q.symmetric = sym;
+        return run_gemm(c, q, engine, what);
+      };
+      if ((rc = small_product(w.Bm, w.Bm, w.Cm, "B^2"))) return rc;
+      if ((rc = small_product(w.Cm, w.Am, w.Dm, "B^2 A"))) return rc;          // ys^2 A_{t+1}: the stored scale carries over
+      g = gemm_desc_zero();
+      g.batch = b; g.in_dtype = it_dtype; g.b_dtype = it_dtype; g.out_dtype = it_dtype;
+      g.M = ms; g.N = ms; g.K[0] = ms;
+      g.A[0] = w.Dm; g.sa_i[0] = ms; g.sa_k[0] = 1; g.batch_a[0] = (long long)ms * ms;
+      g.B[0] = w.Dm; g.sb_k[0] = 1; g.sb_j[0] = ms; g.batch_b[0] = (long long)ms * ms;
+      g.C = w.Am; g.ldc = ms; g.batch_c = (long long)ms * ms;                   // A_t is no longer needed
+      g.aux = w.Dm; g.ld_aux = ms; g.batch_aux = (long long)ms * ms; g.aux_dtype = it_dtype;
+      g.epilogue = EPI_POLY; g.symmetric = sym;
+      g.pa = cf1[0]; g.pb = cf1[1] * iy2; g.pc = cf1[2] * iy2 * iy2;
+      if ((rc = run_gemm(c, g, engine, "polynomial (second step)"))) return rc;
+      if ((rc = small_product(w.Am, w.Bm, w.Cm, "B' B"))) return rc;
+      Bap = w.Cm;
+    }
     // X <- B_t X (wide) or X B_t (tall)
     g = gemm_desc_zero();
     g.batch = b; g.in_dtype = it_dtype; g.b_dtype = it_dtype; g.out_dtype = it_dtype;
     g.M = m; g.N = n;
     if (wide) {
       g.K[0] = m;
-      g.A[0] = w.Bm; g.sa_i[0] = m; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * m;
+      g.A[0] = Bap; g.sa_i[0] = m; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * m;
       g.B[0] = X; g.sb_k[0] = n; g.sb_j[0] = 1; g.batch_b[0] = (long long)m * n;
     } else {
       g.K[0] = n;
       g.A[0] = X; g.sa_i[0] = n; g.sa_k[0] = 1; g.batch_a[0] = (long long)m * n;
-      g.B[0] = w.Bm; g.sb_k[0] = 1; g.sb_j[0] = n; g.batch_b[0] = (long long)n * n;   // B_t symmetric
+      g.B[0] = Bap; g.sb_k[0] = 1; g.sb_j[0] = n; g.batch_b[0] = (long long)n * n;   // B_t symmetric
     }
     g.C = Xn; g.ldc = n; g.batch_c = (long long)m * n;
     g.epilogue = EPI_STORE;
     g.out_dtype = nx_dtype; g.alpha = ys_next / ys;                   // the next step's format and scale
-    if (t == L - 1) { g.out_dtype = dtype; g.alpha = 1.f / ys; }      // the result leaves in the caller's type and scale
-    const bool carry_head = fuse_restore && t == L - 1;
+    if (tl == L - 1) { g.out_dtype = dtype; g.alpha = 1.f / ys; }      // the result leaves in the caller's type and scale
+    const bool carry_head = fuse_restore && tl == L - 1;
     if (carry_head) add_restore_segment(g, false);
-    if (wide && !(upd && t == L - 1)) {
+    if (wide && !(upd && tl == L - 1)) {
       // The tensor engine pads the product's rows to whole 256-row tiles, its columns only to 32: for a wide X
       // whose short side is not a multiple of 256 (1600 = 6.25 tiles) it is cheaper to compute (B X)^T = X^T B
       // (rows = the long side) and let the epilogue write the tile transposed, which is the same memory.
       GemmDesc gt = g;
       gt.M = n; gt.N = m;
       gt.A[0] = X; gt.sa_i[0] = 1; gt.sa_k[0] = n; gt.batch_a[0] = (long long)m * n;
-      gt.B[0] = w.Bm; gt.sb_j[0] = m; gt.sb_k[0] = 1; gt.batch_b[0] = (long long)m * m;    // B_t symmetric
+      gt.B[0] = Bap; gt.sb_j[0] = m; gt.sb_k[0] = 1; gt.batch_b[0] = (long long)m * m;    // B_t symmetric
       if (carry_head) add_restore_segment(gt, true);
       gt.transpose_out = 1;
       const long long pad_rows = (long long)((m + 255) / 256) * 256 * ((n + 31) / 32 * 32);
       const long long pad_rows_t = (long long)((n + 255) / 256) * 256 * ((m + 31) / 32 * 32);
       if (m > 128 && pad_rows_t < pad_rows && use_tensor_engine(gt, engine) && c->knobs.transposed_apply) g = gt;
     }
-    if (upd && t == L - 1) {
+    if (upd && tl == L - 1) {
       // last step of a Muon update: W <- keep W + step (B_L X [+ P W^T]) instead of storing the iterate
       g.C = upd->W; g.out_dtype = upd->w_dtype;
       g.aux = upd->W; g.ld_aux = n; g.batch_aux = (long long)m * n; g.aux_dtype = upd->w_dtype;
@@ -837,6 +909,7 @@ static int polar_core(defl_ctx* c, const void* G, void* out, int b, int m, int n
     const int eng_apply = (carry_head && engine == DEFL_ENGINE_TENSOR && !use_tensor_engine(g, engine)) ? DEFL_ENGINE_SIMT : engine;
     if ((rc = run_gemm(c, g, eng_apply, "apply"))) return rc;
     cur ^= 1;
+    t = tl + 1;
   }
   ctx_stage_mark(c);
 

@@ -24,7 +24,7 @@ struct defl_ctx {
   int* wait_status;      // device words: [0] the tensor engine ORs DEFL_ST_DEVICE_WAIT into it (cleared at the start of
                          // every polar / PSD call), [1] its tile counter
   defl::TcKnobs tc_knobs;        // tuning overrides, read from the environment when the context was created
-  struct { int transposed_apply; int host_chunks; int jacobi_sweeps; } knobs;   // DEFL_NO_TRANSPOSED_APPLY, DEFL_HOST_CHUNKS, DEFL_JACOBI_SWEEPS
+  struct { int transposed_apply; int host_chunks; int jacobi_sweeps; int paired_steps; } knobs;   // DEFL_NO_TRANSPOSED_APPLY, DEFL_HOST_CHUNKS, DEFL_JACOBI_SWEEPS, DEFL_NO_PAIRED_STEPS
   defl::TmCache tm_cache;        // encoded TMA descriptors of recent launches
   void* ident_bf16;              // device, 256 x 256 bf16 identity (operand of the engine's identity segment)
   long long launches;    // kernels launched so far

@@ -47,16 +47,21 @@ def filter_with_storage(X0, sched, formats):
     return X
 
 
-def polar_filter_with_storage(X0, sched, formats):
+def polar_filter_with_storage(X0, sched, formats, passes=None):
     """The filter of the bf16 polar path the way the path stores it: per step the iterate X, the short-side Gram matrix
     A = X X^T (or X^T X) and B = a I + b A + c A^2 are each rounded when written, to the step's format ("half": X is
     kept as 32 X and A as 1024 A in IEEE half, B unscaled; "bf16": plain bf16); products by the oracle's matmul, exact
-    in between. The last result is not rounded here."""
+    in between. `passes` (a list of 1s and 2s, see polar_passes) marks the steps that share one pass over X: there
+    B_t^2, A_{t+1} = B_t^2 A_t, B_{t+1} and B_{t+1} B_t are formed on the short side, each rounded when written and with
+    its upper triangle mirrored as the kernels mirror it, and X is multiplied once. The last result is not rounded."""
     X = np.asarray(X0, dtype=np.float64)
     m, n = X.shape
     wide = m <= n
     ms = min(m, n)
-    for t, (a, b, c) in enumerate(sched):
+    mirror = lambda M: np.triu(M) + np.triu(M, 1).T
+    t = 0
+    for npass in (passes if passes is not None else [1] * len(sched)):
+        a, b, c = sched[t]
         fmt = formats[t]
         rx = ROUNDERS[fmt]
         ra = (lambda v: round_half_scaled(v, 1024.0)) if fmt == "half" else rx
@@ -64,16 +69,46 @@ def polar_filter_with_storage(X0, sched, formats):
         X = rx(X)
         A = ra(oracle.matmul(X, X, tb=True) if wide else oracle.matmul(X, X, ta=True))
         B = rb(a * np.eye(ms) + b * A + c * oracle.matmul(A, A))
+        if npass == 2:
+            a1, b1, c1 = sched[t + 1]
+            S = rb(mirror(oracle.matmul(B, B)))
+            A1 = ra(mirror(oracle.matmul(S, A)))
+            B1 = rb(a1 * np.eye(ms) + b1 * A1 + c1 * oracle.matmul(A1, A1))
+            B = rb(mirror(oracle.matmul(B1, B)))
         X = oracle.matmul(B, X) if wide else oracle.matmul(X, B)
+        t += npass
     return X
 
 
-def polar_formats(L, add_mode, option=0):
+def polar_passes(m, n, sched, paired=None, option=0):
+    """How the path walks the filter steps (1 = a step of its own, 2 = two steps in one pass over X): greedily from
+    the first step, a pair starts at step t when there is a next step, |a_t| <= 4.5 and |b_{t+1} + 2 c_{t+1}| <= 1, provided the long side is at
+    least twice the short one and the iterates are not bf16 throughout (option 1). `paired` False switches the pairing
+    off (the fp32 engine, the knob)."""
+    ms, ml = min(m, n), max(m, n)
+    L = len(sched)
+    if paired is False or option == 1 or ml < 2 * ms:
+        return [1] * L
+    out, t = [], 0
+    while t < L:
+        two = t + 1 < L and abs(sched[t][0]) <= 4.5 and abs(sched[t + 1][1] + 2.0 * sched[t + 1][2]) <= 1.0
+        out.append(2 if two else 1)
+        t += 2 if two else 1
+    return out
+
+
+def polar_formats(L, add_mode, option=0, passes=None):
     """Iterate storage of the bf16 polar path per step: option 0 = scaled half in the first two steps (every step in
-    ADD mode), bf16 after; 1 = bf16 throughout; 2 = half throughout."""
+    ADD mode; every step up to the last paired one where steps are paired), bf16 after; 1 = bf16 throughout; 2 = half
+    throughout."""
     if option == 1:
         return ["bf16"] * L
     n_half = L if (option == 2 or add_mode) else min(L, 2)
+    t = 0
+    for q in (passes or []):
+        t += q
+        if q == 2:
+            n_half = max(n_half, t)                 # both steps of a pair are kept in scaled half
     return ["half"] * n_half + ["bf16"] * (L - n_half)
 
 
@@ -96,13 +131,14 @@ def polar_entry(G, k, l, Omega, J, gamma, add_mode):
     return (X0 if tall else X0.T), (head if tall else head.T)
 
 
-def polar_storage_error(G, k, l, Omega, J, sched, gamma, add_mode, option=0, round_output=False):
+def polar_storage_error(G, k, l, Omega, J, sched, gamma, add_mode, option=0, round_output=False, paired=None):
     """Relative Frobenius distance between the oracle's result with the iterate rounded to the path's storage
     formats (and, with round_output, the result rounded to bf16 as the path returns it) and its result in fp64
     throughout: what the storage format alone explains for this input."""
     X0, head = polar_entry(G, k, l, Omega, J, gamma, add_mode)
     exact = oracle.filter_quintic(X0, sched) + (head if add_mode else 0.0)
-    stored = polar_filter_with_storage(X0, sched, polar_formats(len(sched), add_mode, option)) + (head if add_mode else 0.0)
+    passes = polar_passes(np.shape(G)[0], np.shape(G)[1], sched, paired, option)
+    stored = polar_filter_with_storage(X0, sched, polar_formats(len(sched), add_mode, option, passes), passes) + (head if add_mode else 0.0)
     if round_output:
         stored = round_bf16(stored)
     return float(np.linalg.norm(stored - exact) / np.linalg.norm(exact))

@@ -243,7 +243,9 @@ def test_general_degree_map_matches_oracle(ctx, dtype, shape, terms, L):
         assert _rel(out[i].double().cpu().numpy(), ref) <= TOL[dtype], (i, terms)
     if terms == 4:
         # the quintic entry point with the same coefficients padded by a zero is another polynomial: the option is live
-        out3 = ctx.defl_polar_batched(G.cuda(), k, p, J, [coeffs[:3]] * L, sketch=Om.cuda(), gamma=gamma, exploit_symmetry=True)
+        # (that truncated polynomial grows without bound from 1 on; bf16 iterates keep the comparison finite)
+        out3 = ctx.defl_polar_batched(G.cuda(), k, p, J, [coeffs[:3]] * L, sketch=Om.cuda(), gamma=gamma, exploit_symmetry=True,
+                                      bf16_iterates=1)
         assert _rel(out3[0].double().cpu().numpy(), out[0].double().cpu().numpy()) > 1e-2
 
 

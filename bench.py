@@ -104,10 +104,10 @@ def dense_filter_flops(m, n, L):
     return L * (4.0 * ms * ms * ml + 2.0 * ms ** 3)
 
 
-# Average DRAM bytes per filter-product launch: dram__bytes_read + dram__bytes_write of the six kinds of filter
-# launch (X X^T, A^2 polynomial, B X for each shape group) from the ncu captures summarised in
-# the filter-kernel summary under profiles/ (8 matrices per group: 132.8 MB on average), scaled by 48/8.
-FILTER_TRAFFIC_BYTES_PER_LAUNCH = 797e6
+# Average DRAM bytes per filter-product launch: dram__bytes_read + dram__bytes_write of the 32 filter launches of one
+# step (two paired steps and a single one on the wide group, five single steps on the square one) from the ncu capture
+# summarised in the filter-kernel summary under profiles/ (8 matrices per group: 100.3 MB on average), scaled by 48/8.
+FILTER_TRAFFIC_BYTES_PER_LAUNCH = 602e6
 
 
 def max_over_ranks(value, dist=None, device="cpu"):

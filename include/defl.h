@@ -97,9 +97,11 @@ typedef struct defl_opts {
   int bf16_iterates;     /* polar path with bf16 input: storage type of the filter's iterates X_t, A_t, B_t (input,
                             output and every other stage are unchanged). 0 (default): IEEE half scaled by 32 in the
                             first two filter steps (same tensor-core rate, three more mantissa bits: the rounding of
-                            the early iterates is what limits accuracy), bf16 in the later ones (less power, i.e.
-                            more clock under a power cap); with DEFL_RESTORE_ADD scaled half in every step (that mode
-                            is about ten times more sensitive to the storage rounding). 1: bf16 in every step, the
+                            the early iterates is what limits accuracy) and in every step up to the last one that
+                            shares its pass over X with a neighbour (see defl_polar_batched: "two steps per pass"),
+                            bf16 in the later ones (less power, i.e. more clock under a power cap); with
+                            DEFL_RESTORE_ADD scaled half in every step (that mode is about ten times more sensitive
+                            to the storage rounding). 1: bf16 in every step (and one pass over X per step), the
                             storage the paper's training runs use; NOT within the library's 3e-2 accuracy bar on wide
                             matrices with slowly decaying spectra (1600 x 6400, sigma_i = 200/i, k = 32: 4.2e-2 relative
                             Frobenius error against an fp64 evaluation of the same algorithm; square and faster
@@ -124,7 +126,8 @@ typedef struct defl_info {
  * Environment overrides are read here, once, and never on the call path: DEFL_TC_BN, DEFL_TC_TILE_M, DEFL_TC_STAGES,
  * DEFL_TC_KSUB, DEFL_TC_PAIR, DEFL_TC_PAIR_MIN_N, DEFL_TC_DYNAMIC, DEFL_TC_AUX_PREFETCH, DEFL_TC_DEBUG (tile forms of
  * the tensor engine, for experiments and tests), DEFL_TC_WAIT_MS (limit of the device-side waits, default 2000),
- * DEFL_NO_TRANSPOSED_APPLY, DEFL_HOST_CHUNKS, DEFL_JACOBI_SWEEPS (sweep cap of the Jacobi core, default 40). */
+ * DEFL_NO_TRANSPOSED_APPLY, DEFL_NO_PAIRED_STEPS (one pass over X per filter step everywhere), DEFL_HOST_CHUNKS,
+ * DEFL_JACOBI_SWEEPS (sweep cap of the Jacobi core, default 40). */
 int defl_create(defl_ctx** out, int device);
 int defl_destroy(defl_ctx* ctx);
 int defl_set_stream(defl_ctx* ctx, void* cuda_stream); /* cudaStream_t; NULL = default stream */
@@ -152,6 +155,15 @@ int defl_psd_window(int n, float w, float w_prime, int* k, int* K);
  *   coeff_schedule  host, [L][3] = (a_t, b_t, c_t) of X <- a X + b (X X^T) X + c (X X^T)^2 X (Eq. 2), applied
  *                for t = 1..L in order ([L][opts->poly_terms] for the other degrees of Eq. 5). L = 0 returns X0.
  * Wide matrices (m < n) are handled as the transpose without moving data (polar(M^T) = polar(M)^T).
+ * Two steps per pass: each step is evaluated through the short-side Gram matrix A_t = X_t X_t^T and B_t = a I + b A_t +
+ * c A_t^2 as X_{t+1} = B_t X_t (Eq. 2). On the bf16 tensor path, when the long side is at least twice the short one,
+ * two consecutive quintic steps share one pass over X: since B_t is a polynomial in A_t, A_{t+1} = B_t^2 A_t needs no
+ * product with X, and X_{t+2} = (B_{t+1} B_t) X_t: one Gram and one apply product of ms^2 ml each and five ms^3
+ * products instead of two of each big product and two small ones; the same composite polynomial, another order of
+ * evaluation. Both steps are kept in scaled IEEE half, and a pair starts at step t only where |a_t| <= 4.5 and
+ * |b_{t+1} + 2 c_{t+1}| <= 1 (the two gains with which the rounding of the stored A_t reaches the result; Muon's and
+ * the classical quintic qualify, the steep steps of a per-step minimax schedule do not). Not with the fp32 engine, not
+ * with opts->bf16_iterates = 1, not for the other degrees of Eq. 5.
  * Errors: DEFL_ERR_ARG, DEFL_ERR_RANK (k >= min(m,n) or l > DEFL_MAX_L or L > DEFL_MAX_STEPS), DEFL_ERR_CUDA,
  * DEFL_ERR_UNSUPPORTED. opts and info may be NULL. */
 int defl_polar_batched(defl_ctx* ctx, const void* G, void* out, int b, int m, int n, int dtype,

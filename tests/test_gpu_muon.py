@@ -105,6 +105,27 @@ def test_fused_update_equals_filter_then_axpy(ctx):
     assert err <= 4e-3, err
 
 
+@pytest.mark.parametrize("L", [4, 5])
+def test_update_rides_on_a_paired_last_pass(ctx, L):
+    """A shape that takes two filter steps per pass over X: with an even depth the weight update is the epilogue of a
+    product with B_{t+1} B_t, with an odd one of a single step's product; both against the oracle's step."""
+    from paper_2609_21102_b200 import binding
+    b, m, n, k = 2, 128, 512, 8
+    W, Mom, Grad, Om = _case(b, m, n, k, torch.bfloat16, 16)
+    sched = [list(binding.MUON_QUINTIC)] * L
+    outs, moms = [], []
+    for i in range(b):
+        w1, m1 = oracle.muon_step(W[i].double().numpy(), Mom[i].double().numpy(), Grad[i].double().numpy(), LR, MU, k, 2 * k,
+                                  Om[i].double().numpy(), 1, [oracle.MUON_QUINTIC] * L, weight_decay=WD, scale=SCALE,
+                                  storage="bf16", gamma=1.01)
+        outs.append(w1)
+    Wd, Md = W.cuda(), Mom.cuda()
+    ctx.defl_muon_step_batched(Wd, Md, Grad.cuda(), LR, MU, k, k, 1, sched, weight_decay=WD, scale=SCALE, sketch=Om.cuda(),
+                               gamma=1.01, exploit_symmetry=True)
+    keep = (1.0 - LR * WD) * W.double().numpy()
+    assert _rel(Wd.cpu().double().numpy() - keep, np.stack(outs) - keep) <= 3e-2
+
+
 def test_bf16_weights(ctx):
     from paper_2609_21102_b200 import binding
     b, m, n, k = 2, 256, 256, 8

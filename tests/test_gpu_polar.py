@@ -130,6 +130,46 @@ def test_bf16_iterate_storage_options(ctx, shape, L):
     assert errs[2] <= errs[1] * 1.05 + 1e-3, errs          # half storage is never the less accurate one
 
 
+@pytest.mark.parametrize("L", [2, 3, 4, 5, 6])
+@pytest.mark.parametrize("shape", [(136, 328), (392, 128)])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_two_steps_per_pass_match_oracle(ctx, shape, L, mode):
+    """Shapes whose long side is at least twice the short one take two filter steps per pass over X (wide and tall,
+    even and odd depths, so that the last pass is a pair or a single step, both restore modes): same oracle, same
+    tolerance, the error within what the storage model of that evaluation explains, and close to the result of one
+    pass per step (a context created with the pairing switched off)."""
+    import os
+    import storage_model
+    from paper_2609_21102_b200 import binding
+    m, n = shape
+    k, p, J, gamma = 6, 6, 1, 1.05
+    sig = inputs.spectrum_power(min(m, n), 0.9, 80.0)
+    G64 = torch.stack([inputs.from_spectrum(m, n, sig, 4100 + i) for i in range(2)])
+    sched = _sched(binding.MUON_QUINTIC, L)
+    assert storage_model.polar_passes(m, n, sched).count(2) == L // 2
+    errs = _run_case(ctx, G64, torch.bfloat16, k, p, J, sched, gamma, mode, binding.ENGINE_AUTO, exploit_symmetry=True)
+    assert max(errs) <= TOL[torch.bfloat16], errs
+    G = inputs.round_to(G64, torch.bfloat16)
+    Om = inputs.sketch(2, min(m, n), k + p, 1)
+    model = storage_model.polar_storage_error(G[0].double().numpy(), k, k + p, Om[0].double().numpy(), J, sched, gamma, mode == 1,
+                                              round_output=True)
+    assert errs[0] <= 1.5 * model + 1e-3, (errs[0], model)
+    out = ctx.defl_polar_batched(G.cuda(), k, p, J, sched, sketch=Om.cuda(), restore_mode=mode, gamma=gamma, exploit_symmetry=True)
+    os.environ["DEFL_NO_PAIRED_STEPS"] = "1"
+    try:
+        single = binding.Context(0)
+    finally:
+        del os.environ["DEFL_NO_PAIRED_STEPS"]
+    try:
+        ref = single.defl_polar_batched(G.cuda(), k, p, J, sched, sketch=Om.cuda(), restore_mode=mode, gamma=gamma,
+                                        exploit_symmetry=True)
+        torch.cuda.synchronize()
+    finally:
+        single.close()
+    d = float((out.float() - ref.float()).norm() / ref.float().norm())
+    assert 0.0 < d <= TOL[torch.bfloat16], d            # another order of evaluation: not identical, and close
+
+
 def test_bf16_symmetric_option_and_plain_path(ctx):
     from paper_2609_21102_b200 import binding
     sig = inputs.spectrum_power(192, 1.0, 200.0, 1e-4)

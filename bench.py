@@ -521,7 +521,7 @@ def main():
     opts = {"sym": not args.no_symmetry, "iterates": 1 if args.bf16_iterates else (2 if args.half_iterates else 0),
             "mode": 1 if args.add_restore else 0}
     storage = ("bf16" if opts["iterates"] == 1 else "IEEE half scaled by 32" if (opts["iterates"] == 2 or opts["mode"] == 1)
-               else "IEEE half scaled by 32 in the first two steps, bf16 after")
+               else "IEEE half scaled by 32 in the first two steps and in the steps that share a pass over X, bf16 after")
     sched_note = ("Muon quintic (3.4445, -4.7750, 2.0315) every step" if wl["schedule"] == "muon" else
                   "per-step minimax quintics (greedy Remez from [1e-3, 1], first step / 1.01): the Polar-Express-style "
                   "mapping, coefficients computed by schedules.remez_sign_schedule")

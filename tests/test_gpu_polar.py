@@ -170,6 +170,36 @@ def test_two_steps_per_pass_match_oracle(ctx, shape, L, mode):
     assert 0.0 < d <= TOL[torch.bfloat16], d            # another order of evaluation: not identical, and close
 
 
+def test_pairing_rule_on_other_schedules(ctx):
+    """Which steps share a pass depends on the coefficients: every second step of the classical quintic (slope 1.875),
+    only the last two steps of a per-step minimax schedule (its first step has slope 8.4, its middle steps are too
+    sensitive at the top of the spectrum). Both against the oracle, with the singular values inside the band the
+    scalar composite allows."""
+    import storage_model
+    from paper_2609_21102_b200 import binding, schedules
+    m, n, k, p, J, gamma = 192, 640, 6, 6, 1, 1.1
+    sig = inputs.spectrum_power(m, 0.8, 60.0)
+    G64 = torch.stack([inputs.from_spectrum(m, n, sig, 4300 + i) for i in range(2)])
+    minimax = [list(c) for c in schedules.remez_sign_schedule(1e-3, 5, margin=0.01)[0]]
+    classical = _sched(oracle.CLASSICAL_QUINTIC, 8)
+    assert storage_model.polar_passes(m, n, classical) == [2, 2, 2, 2]
+    assert storage_model.polar_passes(m, n, minimax) == [1, 1, 1, 2]
+    assert storage_model.polar_passes(n, n, classical) == [1] * 8               # square: one pass per step
+    for sched in (classical, minimax):
+        G = inputs.round_to(G64, torch.bfloat16)
+        Om = inputs.sketch(2, m, k + p, 1)
+        out, info = ctx.defl_polar_batched(G.cuda(), k, p, J, sched, sketch=Om.cuda(), gamma=gamma, exploit_symmetry=True,
+                                           want_info=True)
+        torch.cuda.synchronize()
+        for i in range(2):
+            ref, s, kk, rho = oracle.deflated_polar(G[i].double().numpy(), k, k + p, Om[i].double().numpy(), J,
+                                                    oracle.schedule(sched), gamma=gamma)
+            assert _rel(out[i].double().cpu().numpy(), ref) <= TOL[torch.bfloat16]
+            sv_ref = np.linalg.svd(ref, compute_uv=False)
+            sv = np.linalg.svd(out[i].double().cpu().numpy(), compute_uv=False)
+            assert sv.max() <= sv_ref.max() + 4e-2 and sv.min() >= sv_ref.min() - 4e-2, (sv.min(), sv.max(), sv_ref.min(), sv_ref.max())
+
+
 def test_bf16_symmetric_option_and_plain_path(ctx):
     from paper_2609_21102_b200 import binding
     sig = inputs.spectrum_power(192, 1.0, 200.0, 1e-4)
